@@ -1,0 +1,503 @@
+#!/usr/bin/env python
+"""Benchmark of the ring hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--no-extras]
+
+Workload (N = 1): the data-parallel gradient bucket of the second benchmark configuration:
+reduce-scatter then all-gather over R = 8 logical ranks, 25 MiB of bf16 per rank (13,107,200
+elements, normal(0, 1e-3), seed 1), fp32 accumulation, 8 ring chunks.  One step = one pass of the
+whole path over one bucket: plan lookup, fork/join ordering, 7 x 8 reduce-scatter moves, 7 batched
+SUM steps, 7 x 8 all-gather moves.  Four bucket sets (1.6 GiB) are used in rotation so that no step
+finds its inputs in the 126 MB L2.
+
+Reported value: all-reduce bus bandwidth, S * 2(R-1)/R / t_step in GB/s (nccl-tests convention), for the
+copy-route path with at most 8 CTAs for sums; with N GPUs, N independent replicas run and the value
+is the sum of their units over the slowest replica's time.  One JSON line on stdout (rank 0).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "allreduce bus GB/s vs 8 TB/s HBM roofline; SMs used; co-run GEMM TFLOP/s loss"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+FALLBACK_BF16_TFLOPS = 1590.0
+N_BUCKET_SETS = 4
+
+# DRAM bytes (read + write) per SUM launch measured with ncu (dram__bytes_read.sum + dram__bytes_write.sum) on the
+# launch shape of this workload (8 segments of 3,276,800 bytes, 8 CTAs); see profiles/.  None until captured.
+NCU_SUM_TRAFFIC_BYTES_PER_LAUNCH = None
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-extras", action="store_true", help="skip the variant table, GEMM probe and p2p lines")
+    return ap.parse_args()
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            d = json.load(f)
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d.get("bf16_tflops", FALLBACK_BF16_TFLOPS)),
+                "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", 1400.0)), "source": "measured"}
+    except Exception:
+        return {"hbm_gbs": FALLBACK_HBM_GBS, "bf16_tflops": FALLBACK_BF16_TFLOPS, "bf16_tflops_sustained": 1400.0,
+                "source": "fallback"}
+
+
+# ---------------------------------------------------------------------------------------------------
+class ClockSampler(threading.Thread):
+    """Samples SM clock and clock-event reasons through NVML (read only) while a timed region runs."""
+
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+               0x80: "hw_power_brake_slowdown", 0x2: "applications_clocks_setting", 0x10: "sync_boost"}
+
+    def __init__(self, index: int, period_s: float = 0.002):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period_s
+        self.samples, self.reasons, self.power = [], set(), []
+        self.max_mhz = None
+        self._halt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def _reasons(self):
+        nv = self.nv
+        for fn in ("nvmlDeviceGetCurrentClocksEventReasons", "nvmlDeviceGetCurrentClocksThrottleReasons"):
+            if hasattr(nv, fn):
+                try:
+                    return int(getattr(nv, fn)(self.h))
+                except Exception:
+                    continue
+        return 0
+
+    def run(self):
+        if not self.ok:
+            return
+        while not self._halt.is_set():
+            try:
+                self.samples.append(int(self.nv.nvmlDeviceGetClockInfo(self.h, self.nv.NVML_CLOCK_SM)))
+                mask = self._reasons()
+                for bit, name in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+                self.power.append(self.nv.nvmlDeviceGetPowerUsage(self.h) / 1000.0)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def stop(self):
+        self._halt.set()
+        if self.is_alive():
+            self.join(timeout=1.0)
+        s = sorted(self.samples)
+        med = s[len(s) // 2] if s else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(s),
+                "power_w_max": max(self.power) if self.power else None}
+
+
+# ---------------------------------------------------------------------------------------------------
+def bus_factor(R):
+    return 2.0 * (R - 1) / R
+
+
+def algorithmic_hbm_bytes_allreduce(S, R):
+    """Rank-local ring on one device: every wire byte is read+written by a MOVE in both phases (2+2) and read
+    twice + written once by a SUM (3): 7 * S * (R-1)."""
+    return 7.0 * S * (R - 1)
+
+
+def reference_arm(args, world):
+    """Times the CPU oracle, as it stands, on the host cores (rank 0 only)."""
+    if world.rank != 0:
+        return
+    from oracle import ring
+    from paper_2609_34334_b200 import workloads as W
+
+    c = W.C2_DP_BUCKET
+    R, dtype = c.R, c.dtype
+    threads = ring.max_threads()
+    n = c.count
+    xs = W.rank_inputs(c.dist, c.seed, R, n, dtype, c.sigma)
+    t0 = time.perf_counter()
+    ring.ring_allreduce(xs, threads=threads)
+    t_one = time.perf_counter() - t0
+    budget = 150.0
+    frac = 1.0
+    if t_one * (args.steps + args.warmup) > budget:       # bounded sample: a prefix of every rank's bucket
+        frac = budget / (t_one * (args.steps + args.warmup))
+        n = max(R * 1024, int(n * frac) // (R * 8) * (R * 8))
+        xs = [x[:n].copy() for x in xs]
+    for _ in range(args.warmup):
+        ring.ring_allreduce(xs, threads=threads)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        ring.ring_allreduce(xs, threads=threads)
+    dt = (time.perf_counter() - t0) / args.steps
+    S = n * W.elem_size(dtype)
+    val = S * bus_factor(R) / dt / 1e9
+    sample = "all %d elements per rank" % n if frac == 1.0 else "first %d of %d elements per rank (%.1f%%)" % (n, c.count, 100.0 * n / c.count)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": "GB/s", "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": c.name, "R": R, "elements_per_rank": n, "step": "ring all-reduce by the CPU oracle"},
+        "cpu_baseline": {"value": val, "unit": "GB/s", "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------------------------------------------
+def main():
+    args = parse_args()
+    from paper_2609_34334_b200 import replicas
+
+    if args.impl == "reference":
+        world = replicas.World(rank=int(os.environ.get("RANK", "0")), size=int(os.environ.get("WORLD_SIZE", "1")))
+        reference_arm(args, world)
+        return 0
+
+    import numpy as np
+    import torch
+
+    from paper_2609_34334_b200 import binding as hb
+    from paper_2609_34334_b200 import workloads as W
+
+    if not torch.cuda.is_available():
+        sys.stderr.write("bench.py: no CUDA device; the hot path has no CPU fallback\n")
+        return 2
+    world = replicas.init_from_env()
+    dev = world.local_rank if world.distributed else 0
+    torch.cuda.set_device(dev)
+    hb.lib()
+    peaks = measured_peaks()
+    steps, warmup = max(1, args.steps), max(3, args.warmup)
+
+    c = W.C2_DP_BUCKET
+    R, n, dtype, e = c.R, c.count, c.dtype, 2
+    S = n * e
+    count = n // R
+    stream = torch.cuda.Stream()
+
+    # ---- inputs: bucket set 0 is the seeded workload; sets 1.. are the same values rotated (only timing uses them)
+    xs = W.rank_inputs(c.dist, c.seed, R, n, dtype, c.sigma)
+    send_sets, recv_sets = [], []
+    for b in range(N_BUCKET_SETS):
+        if b == 0:
+            send = [torch.from_numpy(x.view(np.int16)).to("cuda", non_blocking=False) for x in xs]
+        else:
+            send = [torch.roll(t, 4099 * b) for t in send_sets[0]]
+        send_sets.append(send)
+        recv_sets.append([torch.zeros(n, dtype=torch.int16, device="cuda") for _ in range(R)])
+    scratch = torch.empty(hb.scratch_bytes(R, n, dtype) + 256, dtype=torch.uint8, device="cuda")
+    spad = (-scratch.data_ptr()) % 256
+
+    def new_comm(path=hb.PATH_CE, **params):
+        cm = hb.Comm(R, dev)
+        cm.set_scratch(scratch.data_ptr() + spad, scratch.numel() - 256)
+        cm.set_path(path)
+        for k, v in params.items():
+            cm.set_param(k, v)
+        return cm
+
+    def step(cm, b, st):
+        """reduce-scatter into chunk r of recv[r], then all-gather in place: the two calls of the workload."""
+        recv = recv_sets[b]
+        rs_out = [recv[r].data_ptr() + r * count * e for r in range(R)]
+        cm.reduce_scatter(send_sets[b], rs_out, count, dtype, st)
+        cm.allgather(rs_out, recv, count, dtype, st)
+
+    def timed(cm, k_steps, k_warm, fn=step, sampler=None):
+        for k in range(k_warm):
+            fn(cm, k % N_BUCKET_SETS, stream)
+        stream.synchronize()
+        replicas.barrier(world)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        if sampler:
+            sampler.start()
+        e0.record(stream)
+        for k in range(k_steps):
+            fn(cm, k % N_BUCKET_SETS, stream)
+        e1.record(stream)
+        stream.synchronize()
+        torch.cuda.synchronize()
+        clocks = sampler.stop() if sampler else None
+        replicas.barrier(world)
+        return e0.elapsed_time(e1) / 1e3 / k_steps, clocks
+
+    # ---- headline: copy-route path, <= 8 CTAs for sums
+    comm = new_comm(hb.PATH_CE, sum_ctas=8)
+    sampler = ClockSampler(dev)
+    t_step, clocks = timed(comm, steps, warmup, sampler=sampler)
+    st = comm.last_stats()
+    # launches of our kernels per step: the SUM launches of the reduce-scatter (the all-gather has none on this path)
+    comm.reduce_scatter(send_sets[0], [recv_sets[0][r].data_ptr() + r * count * e for r in range(R)], count, dtype, stream)
+    stream.synchronize()
+    rs_stats = comm.last_stats()
+    launches_per_step = rs_stats["n_sum_launches"] + rs_stats["n_move_launches"]
+
+    # parity of the timed configuration on bucket set 0 (sampled: rank 0 and rank 5, full vectors)
+    parity = None
+    if world.rank == 0:
+        from oracle import ring as oracle_ring
+
+        want = oracle_ring.ring_allreduce(xs, threads=oracle_ring.max_threads())
+        step(comm, 0, stream)
+        stream.synchronize()
+        parity = all(bool((recv_sets[0][r].cpu().numpy().view(np.uint16) == want[r]).all()) for r in (0, 5))
+
+    t_slowest = replicas.max_over_ranks(world, t_step)
+    units = replicas.sum_over_ranks(world, S * bus_factor(R))
+    value = units / t_slowest / 1e9
+
+    # ---- end to end: host buffers through hoccl_host_allreduce (H2D and D2H inside the timed region)
+    per = (S + 255) // 256 * 256
+    staging = torch.empty(2 * R * per + 256, dtype=torch.uint8, device="cuda")
+    gpad = (-staging.data_ptr()) % 256
+    comm.set_staging(staging.data_ptr() + gpad, 2 * R * per)
+    h_send = [torch.from_numpy(x.view(np.int16)).pin_memory() for x in xs]
+    h_recv = [torch.zeros(n, dtype=torch.int16).pin_memory() for _ in range(R)]
+
+    def e2e_step(cm, b, st):
+        cm.host_allreduce(h_send, h_recv, n, dtype, st)
+
+    k_e2e = max(3, min(steps, 20))
+    t_e2e, _ = timed(comm, k_e2e, 3, fn=e2e_step)
+    e2e_ok = None
+    if world.rank == 0:
+        e2e_ok = bool((h_recv[3].numpy().view(np.uint16) == want[3]).all())
+    t_e2e_slowest = replicas.max_over_ranks(world, t_e2e)
+    e2e_value = units / t_e2e_slowest / 1e9
+
+    line = {
+        "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world.size, "steps": steps, "warmup": warmup,
+        "ms_per_step": t_slowest * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {
+            "workload": c.name, "R": R, "elements_per_rank": n, "bytes_per_rank": S, "ring_chunks": R,
+            "step": "hoccl_reduce_scatter + hoccl_allgather on one bucket", "path": "CE (driver copy route)",
+            "sum_ctas": 8, "executor": "cuda graph replay", "pieces_per_chunk": rs_stats["n_pieces"],
+            "l2": "inputs larger than L2: %d bucket sets of %d MiB in rotation" % (N_BUCKET_SETS, 2 * R * S >> 20),
+            "parallelism": "replicas x%d (the path does not shard)" % world.size,
+        },
+        "algbw_GBps": S / t_slowest / 1e9 * world.size,
+        "hbm_roofline": {
+            "algorithmic_bytes_per_step": algorithmic_hbm_bytes_allreduce(S, R),
+            "achieved_GBps": algorithmic_hbm_bytes_allreduce(S, R) / t_step / 1e9,
+            "frac_of_8TBps": algorithmic_hbm_bytes_allreduce(S, R) / t_step / 1e9 / NOMINAL_HBM_GBS,
+            "frac_of_measured_copy": algorithmic_hbm_bytes_allreduce(S, R) / t_step / 1e9 / peaks["hbm_gbs"],
+        },
+        "sms_used": {"sum_ctas": int(rs_stats["max_sum_ctas"]), "moves": "driver copy route (see move_needs_sm)"},
+        "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": R * S, "d2h_bytes_per_step": R * S,
+                "ms_per_step": t_e2e_slowest * 1e3, "call": "hoccl_host_allreduce (pinned host buffers)", "steps": k_e2e,
+                "matches_oracle": e2e_ok},
+        "gpu_launches": int(launches_per_step * steps),
+        "clocks": clocks,
+        "host_launch_us_per_call": st["host_launch_us"],
+        "matches_oracle": parity,
+        "peaks": peaks,
+    }
+
+    if world.rank == 0 and world.size == 1:
+        # ---- roofline of the dominant kernel (the only kernel of this path): SUM, timed per launch with CUDA events
+        prof = new_comm(hb.PATH_CE, sum_ctas=8, profile=1)
+        for k in range(3):
+            step(prof, k % N_BUCKET_SETS, stream)
+        stream.synchronize()
+        prof.profile_reset()
+        for k in range(min(steps, 40)):
+            step(prof, k % N_BUCKET_SETS, stream)
+            stream.synchronize()
+            prof.last_stats()
+        ps = prof.last_stats()
+        nl = max(1, ps["sum_kernel_launches_timed"])
+        avg_ms = ps["sum_kernel_ms"] / nl
+        bytes_per_launch = ps["sum_kernel_bytes"] / nl
+        achieved = bytes_per_launch / (avg_ms * 1e-3) / 1e9 if avg_ms > 0 else 0.0
+        line["roofline"] = {
+            "kernel": "sum2_kernel<bf16>", "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+            "frac": achieved / peaks["hbm_gbs"], "peak_source": "of " + peaks["source"],
+            "traffic": NCU_SUM_TRAFFIC_BYTES_PER_LAUNCH, "algorithmic_bytes_per_launch": bytes_per_launch,
+            "avg_launch_us": avg_ms * 1e3, "launches_timed": int(nl), "ctas": 8,
+            "note": "8 CTAs by design (SM budget for sums); per-SM rate = achieved/8",
+        }
+        prof.destroy()
+        # the same kernel without the SM budget, timed alone on 256 MiB operands (kernel quality, not the path)
+        big = 128 << 20
+        a = torch.empty(big, dtype=torch.int16, device="cuda").normal_(0, 100)
+        b2 = torch.empty(big, dtype=torch.int16, device="cuda").normal_(0, 100)
+        o = torch.empty(big, dtype=torch.int16, device="cuda")
+        full = {}
+        for ctas in (8, 148, 296, 592):
+            for _ in range(3):
+                hb.sum_launch(a, b2, o, big, dtype, ctas, stream)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            reps = 3 if ctas == 8 else 10
+            for _ in range(reps):
+                hb.sum_launch(a, b2, o, big, dtype, ctas, stream)
+            e1.record(stream)
+            stream.synchronize()
+            full[str(ctas)] = 3.0 * big * 2 / (e0.elapsed_time(e1) / 1e3 / reps) / 1e9
+        line["roofline_unconstrained"] = {
+            "kernel": "sum2_kernel<bf16>", "operands": "3 x 256 MiB, timed alone", "GBps_by_ctas": full,
+            "best_frac_of_measured": max(full.values()) / peaks["hbm_gbs"]}
+        del a, b2, o
+
+        # ---- CPU baseline: the oracle on the host cores, whole bucket, a few repetitions
+        thr = oracle_ring.max_threads()
+        reps, t0 = 0, time.perf_counter()
+        while reps < 3 or (time.perf_counter() - t0 < 2.5 and reps < 50):
+            oracle_ring.ring_allreduce(xs, threads=thr)
+            reps += 1
+        t_cpu = (time.perf_counter() - t0) / reps
+        line["cpu_baseline"] = {"value": S * bus_factor(R) / t_cpu / 1e9, "unit": "GB/s", "cores": thr, "kind": "oracle",
+                                "sample": "%d repetitions of the whole bucket (all %d elements per rank)" % (reps, n),
+                                "ms_per_step": t_cpu * 1e3}
+
+        if not args.no_extras:
+            line["extras"] = extras(hb, W, torch, np, new_comm, step, timed, stream, R, S, n, dtype, peaks, send_sets, recv_sets)
+
+    comm.destroy()
+    if world.rank == 0:
+        print(json.dumps(line), flush=True)
+    replicas.shutdown(world)
+    return 0
+
+
+def extras(hb, W, torch, np, new_comm, step, timed, stream, R, S, n, dtype, peaks, send_sets, recv_sets):
+    """Context lines: path / CTA-budget variants, whether a move needs an SM, p2p, and the co-running GEMM probe."""
+    out = {}
+    k, w = 40, 5
+    variants = [("CE", hb.PATH_CE, 8, 8), ("CE", hb.PATH_CE, 32, 8), ("CE", hb.PATH_CE, 148, 8), ("SM", hb.PATH_SM, 8, 8),
+                ("SM", hb.PATH_SM, 8, 32), ("SM", hb.PATH_SM, 148, 148), ("SM", hb.PATH_SM, 296, 296)]
+    rows = []
+    hbm = 7.0 * S * (R - 1)
+    for name, path, sc, cc in variants:
+        cm = new_comm(path, sum_ctas=sc, copy_ctas=cc)
+        t, _ = timed(cm, k, w)
+        rows.append({"path": name, "sum_ctas": sc, "copy_ctas": cc if path == hb.PATH_SM else None, "ms_per_step": t * 1e3,
+                     "busbw_GBps": S * bus_factor(R) / t / 1e9, "hbm_frac_of_8TBps": hbm / t / 1e9 / NOMINAL_HBM_GBS})
+        cm.destroy()
+    out["variants"] = rows
+    # one all-reduce call instead of two calls (all-gather of early pieces overlaps the last sums)
+    cm = new_comm(hb.PATH_CE, sum_ctas=8)
+
+    def one_call(c_, b, st):
+        c_.allreduce(send_sets[b], recv_sets[b], n, dtype, st)
+
+    t, _ = timed(cm, k, w, fn=one_call)
+    out["single_call_allreduce"] = {"ms_per_step": t * 1e3, "busbw_GBps": S * bus_factor(R) / t / 1e9}
+    # stream executor (events) instead of graph replay
+    cm.set_param("use_graph", 0)
+    t, _ = timed(cm, k, w)
+    out["stream_executor"] = {"ms_per_step": t * 1e3, "busbw_GBps": S * bus_factor(R) / t / 1e9,
+                              "host_launch_us_per_call": cm.last_stats()["host_launch_us"]}
+    cm.set_param("use_graph", 1)
+
+    # does a move need an SM?  (bounded occupancy kernel + one 64 MiB move)
+    src = send_sets[0][0]
+    dst = recv_sets[0][0]
+    nb = min(64 << 20, src.numel() * 2)
+    ce_needs, ce_end = cm.probe_move_needs_sm(hb.PATH_CE, dst, src, nb, 3000)
+    sm_needs, sm_end = cm.probe_move_needs_sm(hb.PATH_SM, dst, src, nb, 3000)
+    out["move_needs_sm"] = {"CE_driver_copy": ce_needs, "CE_move_end_us": ce_end, "SM_copy_kernel": sm_needs,
+                            "SM_move_end_us": sm_end, "occupancy_kernel_us": 3000,
+                            "note": "true = the move finished only after a kernel holding every SM had ended"}
+
+    # point to point: 64 MiB bf16 activations [4, 2048, 4096]
+    act = torch.empty(4 * 2048 * 4096, dtype=torch.int16, device="cuda").normal_(0, 100)
+    slots = [torch.empty_like(act) for _ in range(4)]
+    p2p = {}
+    for name, path in (("CE", hb.PATH_CE), ("SM8", hb.PATH_SM)):
+        cm.set_path(path)
+        cm.set_param("copy_ctas", 8)
+
+        def hop(c_, b, st):
+            c_.send(act, act.numel(), "bf16", 0, 1, st)
+            c_.recv(slots[b], act.numel(), "bf16", 0, 1, st)
+
+        t, _ = timed(cm, 20, 3, fn=hop)
+        p2p[name] = {"us_per_message": t * 1e6, "algbw_GBps": act.numel() * 2 / t / 1e9,
+                     "hbm_frac_of_8TBps": 2 * act.numel() * 2 / t / 1e9 / NOMINAL_HBM_GBS}
+    out["p2p_64MiB"] = p2p
+    cm.set_path(hb.PATH_CE)
+
+    # co-running bf16 GEMM probe (4096^3) on another stream: TFLOP/s alone and beside the collective
+    gs = torch.cuda.Stream()
+    A = torch.randn(4096, 4096, dtype=torch.bfloat16, device="cuda")
+    B = torch.randn(4096, 4096, dtype=torch.bfloat16, device="cuda")
+    C = torch.empty(4096, 4096, dtype=torch.bfloat16, device="cuda")
+    flops = 2.0 * 4096 ** 3
+
+    def gemm_tflops(cm_, n_gemm=150):
+        with torch.cuda.stream(gs):
+            for _ in range(10):
+                torch.matmul(A, B, out=C)
+        torch.cuda.synchronize()
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n_comm = 0
+        if cm_ is not None:
+            t_c, _ = timed(cm_, 10, 3)
+            n_comm = int(1.5 * n_gemm * 80e-6 / t_c) + 2
+        c0.record(stream)
+        g0.record(gs)
+        done_c = 0
+        for i in range(n_gemm):
+            with torch.cuda.stream(gs):
+                torch.matmul(A, B, out=C)
+            want_c = (i + 1) * n_comm // n_gemm
+            while done_c < want_c:
+                step(cm_, done_c % N_BUCKET_SETS, stream)
+                done_c += 1
+        g1.record(gs)
+        c1.record(stream)
+        torch.cuda.synchronize()
+        tf = flops * n_gemm / (g0.elapsed_time(g1) / 1e3) / 1e12
+        bw = (S * bus_factor(R) * done_c / (c0.elapsed_time(c1) / 1e3) / 1e9) if done_c else 0.0
+        return tf, bw
+
+    probe = {}
+    alone, _ = gemm_tflops(None)
+    probe["alone_TFLOPs"] = alone
+    for name, path, sc, cc in (("CE_sum8", hb.PATH_CE, 8, 8), ("SM_copy8_sum8", hb.PATH_SM, 8, 8), ("SM_copy32_sum8", hb.PATH_SM, 8, 32),
+                               ("SM_copy148_sum148", hb.PATH_SM, 148, 148)):
+        c2 = new_comm(path, sum_ctas=sc, copy_ctas=cc)
+        tf, bw = gemm_tflops(c2)
+        probe[name] = {"gemm_TFLOPs": tf, "loss": 1.0 - tf / alone, "comm_busbw_GBps": bw}
+        c2.destroy()
+    out["gemm_probe_4096"] = probe
+    cm.destroy()
+    return out
+
+
+if __name__ == "__main__":
+    sys.exit(main())

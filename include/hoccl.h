@@ -1,0 +1,275 @@
+/*
+ * hoccl.h - C ABI of libhoccl.so: ring collectives and point-to-point transfers over R logical
+ * ranks that live as R disjoint buffers in the HBM of ONE B200.
+ *
+ * Background.  HOCCL (the paper) runs collectives as host-issued chunked transfer schedules so that
+ * data movement leaves the SMs free (Sec. 3.1 "Overview": stream manager, point-to-point executor,
+ * collective scheduler).  This library builds the data-parallel hot path of that method for one
+ * GPU: a collective is planned on the host as a DAG of chunk MOVEs and, for reductions, per-step
+ * chunk SUMs; every MOVE is a plain device-to-device copy (driver copy route, or an SM copy kernel
+ * with a CTA budget as the comparison path); the SUM is a hand-written sm_100a kernel limited to a
+ * small CTA budget.  The paper leaves reductions out of scope (Sec. 4 "Limitations"); the ring
+ * reduce-scatter here is the textbook one in a fixed order, stated next to hoccl_allreduce.
+ *
+ * Conventions that hold for every entry point unless stated otherwise
+ *  - Pointers named `send`/`recv` are HOST arrays of R DEVICE pointers: send[r] is rank r's input
+ *    buffer X_r, recv[r] its output buffer Y_r.  The arrays are read during the call and not kept.
+ *    All device buffers belong to the caller and live on the communicator's device.
+ *  - `count` is in elements of `dtype`, NCCL style (the paper's runtime extends NCCL and is measured
+ *    with nccl-tests, Sec. 5 "Testbed"): see each collective.
+ *  - Calls are asynchronous: they enqueue work and return.  The work starts after everything
+ *    enqueued earlier on `stream` and everything enqueued later on `stream` sees it complete: the
+ *    paper's operator-level temporal ordering (abstract; Sec. 3.2 "Stream Manager").  No call
+ *    synchronises the host with the device, except where a call says so.
+ *  - Errors are return codes; nothing is enqueued when a call fails with an argument error.
+ *    count == 0 is HOCCL_OK and enqueues nothing.  X_r is never written (unless it aliases Y_r).
+ *  - Buffers of different ranks must not overlap.  In place is legal: allreduce with
+ *    send[r] == recv[r]; reduce_scatter with recv[r] == send[r] + r*count; allgather with
+ *    send[r] == recv[r] + r*count (element offsets).
+ *  - One host thread per communicator.  The library never allocates device memory: scratch and
+ *    staging are caller-owned and attached with hoccl_comm_set_scratch / hoccl_comm_set_staging.
+ *  - The CUDA device must be present: every entry point that touches the device returns
+ *    HOCCL_ERR_CUDA otherwise.  There is no CPU fallback.
+ */
+#ifndef HOCCL_H_
+#define HOCCL_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct hoccl_comm* hoccl_comm_t;
+/* a CUDA stream handle (cudaStream_t / CUstream) passed as an opaque pointer; NULL is the legacy default stream */
+typedef void* hoccl_stream_t;
+
+typedef enum {
+  HOCCL_OK = 0,
+  HOCCL_ERR_INVALID_ARG = 1, /* null pointer, rank or R out of range, src == dst, overlapping rank buffers, misaligned pointer */
+  HOCCL_ERR_UNSUPPORTED = 2, /* op other than sum, unknown dtype, unknown parameter key */
+  HOCCL_ERR_CUDA = 3,        /* a CUDA call failed (no device, bad stream, ...) */
+  HOCCL_ERR_MISMATCH = 4,    /* send/recv matched with different count or dtype; the parked post is dropped */
+  HOCCL_ERR_PENDING = 5,     /* destroy with unmatched send/recv posts */
+  HOCCL_ERR_SCRATCH = 6,     /* scratch or staging memory missing or too small */
+  HOCCL_ERR_INTERNAL = 7
+} hoccl_result_t;
+
+typedef enum { HOCCL_FLOAT32 = 0, HOCCL_BFLOAT16 = 1 } hoccl_dtype_t;
+typedef enum { HOCCL_SUM = 0 } hoccl_op_t;
+
+/*
+ * How MOVEs are carried out.
+ *  HOCCL_PATH_CE : one device-to-device cudaMemcpyAsync (or memcpy graph node) per move.  This is
+ *                  the copy-engine route of the paper (Sec. 2.3 "DMA Engines", Sec. 3.3): between two
+ *                  GPUs the driver services it with a DMA engine and no SM.  Whether a copy inside ONE
+ *                  device is also SM free is up to the driver; hoccl_probe_move_needs_sm measures it.
+ *  HOCCL_PATH_SM : the comparison baseline (the paper's "NCCL with an SM budget", Sec. 5 "Baselines"):
+ *                  all moves of a step run in one launch of an SM copy kernel with `copy_ctas` CTAs.
+ */
+typedef enum { HOCCL_PATH_CE = 0, HOCCL_PATH_SM = 1 } hoccl_path_t;
+
+typedef struct {
+  double host_launch_us; /* host time spent inside the last collective / matched p2p call (paper Sec. 5 "CPU launch overhead") */
+  long n_moves;          /* MOVE operations of the last call (copies on the CE path, segments on the SM path) */
+  long n_move_launches;  /* SM copy kernel launches of the last call (0 on the CE path) */
+  long n_sum_launches;   /* SUM kernel launches of the last call */
+  long max_sum_ctas;     /* CTAs of the widest SUM launch */
+  long max_copy_ctas;    /* CTAs of the widest SM copy launch */
+  long n_pieces;         /* pipeline pieces per ring chunk */
+  long graph_hit;        /* 1 if the call replayed a cached CUDA graph, 0 if it built one or used streams */
+  double sum_kernel_ms;  /* with parameter "profile" = 1: total device time of SUM launches since hoccl_profile_reset */
+  long sum_kernel_launches_timed;
+  double sum_kernel_bytes; /* algorithmic bytes (2 reads + 1 write per element) of those launches */
+} hoccl_stats_t;
+
+/* ---------------------------------------------------------------- communicator ----------------- */
+
+/*
+ * Creates a communicator of R logical ranks (1 <= R <= 64) on CUDA device `device`: internal
+ * streams and events only, no device memory.  Errors: INVALID_ARG (comm NULL, R out of range),
+ * CUDA (no such device).
+ */
+hoccl_result_t hoccl_comm_init(hoccl_comm_t* comm, int R, int device);
+
+/* Frees host state, streams, events and cached graphs.  Synchronises the internal streams.
+ * HOCCL_ERR_PENDING (and nothing freed) if unmatched send/recv posts remain. */
+hoccl_result_t hoccl_comm_destroy(hoccl_comm_t comm);
+
+/* Upper bound of the scratch bytes any collective needs for up to `max_count` elements of `dtype`
+ * per rank buffer (allreduce convention) with R ranks: per rank one inbox and one partial slot of
+ * one ring chunk each, padded.  0 for R == 1. */
+size_t hoccl_scratch_bytes(int R, size_t max_count, hoccl_dtype_t dtype);
+
+/* Attaches caller-owned device scratch (256-byte aligned).  Reductions need it; all-gather and p2p do
+ * not.  Contents are undefined between calls.  Collectives that overlap in time on different streams
+ * must not share a communicator. */
+hoccl_result_t hoccl_comm_set_scratch(hoccl_comm_t comm, void* dev_ptr, size_t bytes);
+
+/* Attaches caller-owned device staging memory used only by the hoccl_host_* entry points. */
+hoccl_result_t hoccl_comm_set_staging(hoccl_comm_t comm, void* dev_ptr, size_t bytes);
+
+hoccl_result_t hoccl_comm_set_path(hoccl_comm_t comm, hoccl_path_t path);
+
+/*
+ * Tuning and diagnostics.  Keys:
+ *  "sum_ctas"    CTAs of a SUM launch, 1..1024 (default 8: the SM budget for sums)
+ *  "copy_ctas"   CTAs of an SM copy launch, 1..1024 (default 8)
+ *  "piece_bytes" pipeline piece size in bytes (default 4 MiB, rounded to a multiple of 1024)
+ *  "max_pieces"  cap on pieces per ring chunk (default 8)
+ *  "lanes"       internal move streams of the stream executor, 1..8 (default 4)
+ *  "use_graph"   1 = run a cached CUDA graph built from the plan (default), 0 = streams and events
+ *  "profile"     1 = time every SUM launch with CUDA events; read the totals with hoccl_last_stats after
+ *                synchronising (with graphs only the latest replay of each cached graph is readable, so
+ *                read after every step)
+ * None of them changes a single result bit.  Errors: UNSUPPORTED (unknown key), INVALID_ARG (range).
+ */
+hoccl_result_t hoccl_comm_set_param(hoccl_comm_t comm, const char* key, long value);
+hoccl_result_t hoccl_comm_get_param(hoccl_comm_t comm, const char* key, long* value);
+
+/* ---------------------------------------------------------------- collectives ------------------ */
+
+/*
+ * Ring all-reduce (sum) = ring reduce-scatter followed by ring all-gather.
+ * send[r], recv[r]: `count` elements each.  After completion every recv[r] holds the same vector.
+ *
+ * Order of the sum (fixed; results are bit-reproducible).  The buffer is cut into R ring chunks of
+ * q = ceil(count/R) elements (trailing chunks may be short or empty).  Data travels r -> (r+1) mod R.
+ * At step s = 0..R-2 rank r sends chunk (r-1-s) mod R (its own data at s = 0, else the partial it just
+ * produced) and then adds what it received to its own chunk (r-2-s) mod R:
+ *     out[i] = round_to_dtype( float(received[i]) + float(own[i]) )     one binary32 add, RNE
+ * so element i of chunk c ends as ((x_{c+1} + x_{c+2}) + ... + x_{c+R-1}) + x_c (rank indices mod R),
+ * and the partial is stored in `dtype` at every hop (bf16 is re-rounded R-1 times).
+ * The paper has no reduction (Sec. 4 "Limitations"); moves follow its chunked, pipelined transfer
+ * schedule (Sec. 3.3 "chunk pipelining", Sec. 3.4 "Flow-size-aware chunk scheduling").
+ * Needs scratch (hoccl_scratch_bytes).  Errors: INVALID_ARG, UNSUPPORTED, SCRATCH, CUDA.
+ */
+hoccl_result_t hoccl_allreduce(const void* const* send, void* const* recv, size_t count, hoccl_dtype_t dtype,
+                               hoccl_op_t op, hoccl_comm_t comm, hoccl_stream_t stream);
+
+/*
+ * Ring reduce-scatter (sum).  send[r]: R*count elements; recv[r]: count elements = chunk r of the
+ * sum, reduced in the order given above with chunk c = elements [c*count, (c+1)*count).
+ * Needs scratch.
+ */
+hoccl_result_t hoccl_reduce_scatter(const void* const* send, void* const* recv, size_t count, hoccl_dtype_t dtype,
+                                    hoccl_op_t op, hoccl_comm_t comm, hoccl_stream_t stream);
+
+/*
+ * Ring all-gather (paper Sec. 5 "AllGather": the data-parallel pattern HOCCL targets).
+ * send[r]: count elements; recv[r]: R*count elements = send[0] | send[1] | ... | send[R-1].
+ * Pure moves: R-1 ring steps, plus the copy of the own chunk when not in place.  No scratch.
+ */
+hoccl_result_t hoccl_allgather(const void* const* send, void* const* recv, size_t count, hoccl_dtype_t dtype,
+                               hoccl_comm_t comm, hoccl_stream_t stream);
+
+/* ---------------------------------------------------------------- point to point --------------- */
+
+/*
+ * Non-blocking matched send/recv between logical ranks (paper Sec. 3.3.2 "Intra-node
+ * Communication": a post does not block the caller while the peer has not posted; the transfer
+ * happens once both sides are known).  Posts are matched per (src, dst) pair in FIFO order; either
+ * side may come first.  The first post parks {buffer, count, dtype, stream} and enqueues nothing.
+ * The second post enqueues ONE device-to-device move of count elements that runs after both
+ * posting streams have reached their post (for the first poster: its stream position at the time of
+ * the match) and that both streams then wait for.
+ * Mismatch of count or dtype at match time: HOCCL_ERR_MISMATCH from the second call, nothing is
+ * enqueued and the parked post is dropped.  Unmatched posts can never hang a stream; their number is
+ * hoccl_comm_pending().  Errors: INVALID_ARG (NULL buf, rank out of range, src == dst), CUDA.
+ */
+hoccl_result_t hoccl_send(const void* buf, size_t count, hoccl_dtype_t dtype, int src, int dst, hoccl_comm_t comm,
+                          hoccl_stream_t stream);
+hoccl_result_t hoccl_recv(void* buf, size_t count, hoccl_dtype_t dtype, int src, int dst, hoccl_comm_t comm,
+                          hoccl_stream_t stream);
+int hoccl_comm_pending(hoccl_comm_t comm);
+
+/* ---------------------------------------------------------------- host-buffer entry points ----- */
+
+/*
+ * All-reduce whose buffers are HOST memory (pinned for real asynchrony): h_send[r] / h_recv[r] are
+ * host pointers to `count` elements each.  The call copies every h_send[r] into the attached staging
+ * memory (needs 2*R*count*sizeof(dtype) bytes), runs hoccl_allreduce there and copies every rank's
+ * result back, all enqueued on `stream`.  Host-to-device traffic is driven by the copy engines
+ * (Sec. 2.3).  Errors: as hoccl_allreduce, SCRATCH if staging is missing or too small.
+ */
+hoccl_result_t hoccl_host_allreduce(const void* const* h_send, void* const* h_recv, size_t count, hoccl_dtype_t dtype,
+                                    hoccl_op_t op, hoccl_comm_t comm, hoccl_stream_t stream);
+
+/* ---------------------------------------------------------------- diagnostics ------------------ */
+
+const char* hoccl_error_string(hoccl_result_t code);
+/* Text of the last CUDA error seen by this communicator ("" if none); valid until the next call. */
+const char* hoccl_last_cuda_error(hoccl_comm_t comm);
+hoccl_result_t hoccl_last_stats(hoccl_comm_t comm, hoccl_stats_t* out);
+hoccl_result_t hoccl_profile_reset(hoccl_comm_t comm);
+
+/*
+ * Measures whether a MOVE of `bytes` bytes on the given path needs an SM.  A kernel that fills every
+ * thread slot of every SM sleeps for a fixed `spin_us` microseconds (bounded; it never waits on
+ * anything) while the move is enqueued on another stream; *needs_sm is 1 if the move finished only
+ * after that kernel ended, 0 if it finished while all SMs were taken.  *move_end_us is the move's
+ * completion time measured from the kernel's start.  Synchronises the device.  This is the
+ * single-GPU form of the paper's claim that copy-engine transfers occupy no SM (Sec. 2.3).
+ * src and dst are device buffers of at least `bytes` bytes.
+ */
+hoccl_result_t hoccl_probe_move_needs_sm(hoccl_comm_t comm, hoccl_path_t path, void* dst, const void* src, size_t bytes,
+                                         int spin_us, int* needs_sm, double* move_end_us);
+
+/*
+ * Direct launches of the two kernels (used by kernel-level tests and roofline measurements).
+ *  hoccl_sum_launch : out[i] = round_to_dtype(float(inbox[i]) + float(local[i])), i < count, with `ctas` CTAs.
+ *  hoccl_copy_launch: dst bytes <- src bytes with `ctas` CTAs.
+ * All pointers are device pointers aligned to the element size (any byte alignment for the copy).
+ */
+hoccl_result_t hoccl_sum_launch(const void* inbox, const void* local, void* out, size_t count, hoccl_dtype_t dtype,
+                                int ctas, hoccl_stream_t stream);
+hoccl_result_t hoccl_copy_launch(const void* src, void* dst, size_t bytes, int ctas, hoccl_stream_t stream);
+
+/* ---------------------------------------------------------------- plan inspection (host only) --- */
+
+/*
+ * The planner (paper Sec. 3.4: a collective becomes stages of point-to-point flows that are cut into
+ * chunks for the copy queue) is pure host code; these calls expose its output so that it can be
+ * checked without a GPU.  Addresses in a plan are byte offsets: buffer kinds below say what they are
+ * relative to.
+ */
+typedef enum { HOCCL_PLAN_ALLREDUCE = 0, HOCCL_PLAN_REDUCE_SCATTER = 1, HOCCL_PLAN_ALLGATHER = 2 } hoccl_plan_kind_t;
+typedef enum { HOCCL_OP_MOVE = 0, HOCCL_OP_SUM = 1 } hoccl_plan_op_kind_t;
+typedef enum { HOCCL_BUF_SEND = 0, HOCCL_BUF_RECV = 1, HOCCL_BUF_INBOX = 2, HOCCL_BUF_PARTIAL = 3 } hoccl_buf_kind_t;
+
+typedef struct {
+  int kind;      /* hoccl_plan_op_kind_t */
+  int phase;     /* 0 reduce-scatter, 1 all-gather, 2 own-chunk copy of an out-of-place all-gather */
+  int step;      /* ring step s */
+  int piece;     /* pipeline piece index */
+  int rank;      /* MOVE: source rank; SUM: the rank that sums */
+  int dst_rank;  /* MOVE: destination rank; SUM: same as rank */
+  int chunk;     /* ring chunk index */
+  int src_buf, dst_buf, local_buf; /* hoccl_buf_kind_t; local_buf only for SUM */
+  uint64_t src_off, dst_off, local_off; /* byte offsets from the start of those buffers (scratch: from the start of the rank's slot) */
+  uint64_t bytes;
+  int group;     /* ops of one group are issued together (one batched kernel launch or R copies) */
+} hoccl_plan_op_t;
+
+typedef struct hoccl_plan* hoccl_plan_t;
+
+/* Builds the plan for `kind` over R ranks.  `count` as in the collective; in_place as defined at the top of
+ * this file; piece_bytes / max_pieces as the parameters of the same name.  send_align: HOST array of R bytes,
+ * the low 4 bits of each rank's send pointer (NULL = all 16-byte aligned); it only decides where inside its
+ * scratch region a piece is placed so that SUM operands share their 16-byte phase.  Free with hoccl_plan_destroy. */
+hoccl_result_t hoccl_plan_build(hoccl_plan_t* plan, int kind, int R, size_t count, hoccl_dtype_t dtype, int in_place,
+                                size_t piece_bytes, int max_pieces, const unsigned char* send_align);
+/* Bytes of one rank's scratch slot (inbox or partial) under this plan; slots of rank r start at r * that. */
+size_t hoccl_plan_slot_bytes(hoccl_plan_t plan);
+void hoccl_plan_destroy(hoccl_plan_t plan);
+int hoccl_plan_num_ops(hoccl_plan_t plan);
+int hoccl_plan_num_groups(hoccl_plan_t plan);
+hoccl_result_t hoccl_plan_get_op(hoccl_plan_t plan, int index, hoccl_plan_op_t* out);
+/* Dependencies are between groups: writes up to `cap` predecessor group ids of `group` into deps, returns their number. */
+int hoccl_plan_group_deps(hoccl_plan_t plan, int group, int* deps, int cap);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HOCCL_H_ */

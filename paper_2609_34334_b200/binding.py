@@ -1,0 +1,298 @@
+"""Thin ctypes binding of libhoccl.so: same names as include/hoccl.h, argument marshalling only.
+
+Buffers are given as objects with a `data_ptr()` method (torch tensors) or as integer device
+addresses; streams as `torch.cuda.Stream`, raw integer handles or None (the current torch stream).
+Nothing here computes: every step of a collective runs inside the library.  If the library cannot
+be built or loaded the import of `lib()` raises; there is no fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+from typing import Optional, Sequence
+
+from . import build as _build
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_MISMATCH, ERR_PENDING, ERR_SCRATCH, ERR_INTERNAL = range(8)
+FLOAT32, BFLOAT16 = 0, 1
+SUM = 0
+PATH_CE, PATH_SM = 0, 1
+PLAN_ALLREDUCE, PLAN_REDUCE_SCATTER, PLAN_ALLGATHER = 0, 1, 2
+OP_MOVE, OP_SUM = 0, 1
+BUF_SEND, BUF_RECV, BUF_INBOX, BUF_PARTIAL = 0, 1, 2, 3
+
+DTYPES = {"fp32": FLOAT32, "bf16": BFLOAT16}
+
+EXPORTS = [
+    "hoccl_comm_init", "hoccl_comm_destroy", "hoccl_scratch_bytes", "hoccl_comm_set_scratch", "hoccl_comm_set_staging",
+    "hoccl_comm_set_path", "hoccl_comm_set_param", "hoccl_comm_get_param", "hoccl_allreduce", "hoccl_reduce_scatter",
+    "hoccl_allgather", "hoccl_send", "hoccl_recv", "hoccl_comm_pending", "hoccl_host_allreduce", "hoccl_error_string",
+    "hoccl_last_cuda_error", "hoccl_last_stats", "hoccl_profile_reset", "hoccl_probe_move_needs_sm", "hoccl_sum_launch",
+    "hoccl_copy_launch", "hoccl_plan_build", "hoccl_plan_destroy", "hoccl_plan_num_ops", "hoccl_plan_num_groups",
+    "hoccl_plan_get_op", "hoccl_plan_group_deps", "hoccl_plan_slot_bytes",
+]
+
+
+class Stats(ctypes.Structure):
+    _fields_ = [
+        ("host_launch_us", ctypes.c_double), ("n_moves", ctypes.c_long), ("n_move_launches", ctypes.c_long),
+        ("n_sum_launches", ctypes.c_long), ("max_sum_ctas", ctypes.c_long), ("max_copy_ctas", ctypes.c_long),
+        ("n_pieces", ctypes.c_long), ("graph_hit", ctypes.c_long), ("sum_kernel_ms", ctypes.c_double),
+        ("sum_kernel_launches_timed", ctypes.c_long), ("sum_kernel_bytes", ctypes.c_double),
+    ]
+
+    def as_dict(self):
+        return {k: getattr(self, k) for k, _ in self._fields_}
+
+
+class PlanOp(ctypes.Structure):
+    _fields_ = [
+        ("kind", ctypes.c_int), ("phase", ctypes.c_int), ("step", ctypes.c_int), ("piece", ctypes.c_int),
+        ("rank", ctypes.c_int), ("dst_rank", ctypes.c_int), ("chunk", ctypes.c_int), ("src_buf", ctypes.c_int),
+        ("dst_buf", ctypes.c_int), ("local_buf", ctypes.c_int), ("src_off", ctypes.c_uint64), ("dst_off", ctypes.c_uint64),
+        ("local_off", ctypes.c_uint64), ("bytes", ctypes.c_uint64), ("group", ctypes.c_int),
+    ]
+
+
+class HocclError(RuntimeError):
+    def __init__(self, code: int, what: str, detail: str = ""):
+        self.code = code
+        super().__init__("%s failed: %s (code %d)%s" % (what, error_string(code), code, (": " + detail) if detail else ""))
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Builds (if stale) and loads libhoccl.so.  Raises if that is not possible."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = _build.build()
+    L = ctypes.CDLL(path)
+    vp, vpp, sz, i, l = ctypes.c_void_p, ctypes.POINTER(ctypes.c_void_p), ctypes.c_size_t, ctypes.c_int, ctypes.c_long
+    sigs = {
+        "hoccl_comm_init": (i, [vpp, i, i]),
+        "hoccl_comm_destroy": (i, [vp]),
+        "hoccl_scratch_bytes": (sz, [i, sz, i]),
+        "hoccl_comm_set_scratch": (i, [vp, vp, sz]),
+        "hoccl_comm_set_staging": (i, [vp, vp, sz]),
+        "hoccl_comm_set_path": (i, [vp, i]),
+        "hoccl_comm_set_param": (i, [vp, ctypes.c_char_p, l]),
+        "hoccl_comm_get_param": (i, [vp, ctypes.c_char_p, ctypes.POINTER(l)]),
+        "hoccl_allreduce": (i, [vpp, vpp, sz, i, i, vp, vp]),
+        "hoccl_reduce_scatter": (i, [vpp, vpp, sz, i, i, vp, vp]),
+        "hoccl_allgather": (i, [vpp, vpp, sz, i, vp, vp]),
+        "hoccl_send": (i, [vp, sz, i, i, i, vp, vp]),
+        "hoccl_recv": (i, [vp, sz, i, i, i, vp, vp]),
+        "hoccl_comm_pending": (i, [vp]),
+        "hoccl_host_allreduce": (i, [vpp, vpp, sz, i, i, vp, vp]),
+        "hoccl_error_string": (ctypes.c_char_p, [i]),
+        "hoccl_last_cuda_error": (ctypes.c_char_p, [vp]),
+        "hoccl_last_stats": (i, [vp, ctypes.POINTER(Stats)]),
+        "hoccl_profile_reset": (i, [vp]),
+        "hoccl_probe_move_needs_sm": (i, [vp, i, vp, vp, sz, i, ctypes.POINTER(i), ctypes.POINTER(ctypes.c_double)]),
+        "hoccl_sum_launch": (i, [vp, vp, vp, sz, i, i, vp]),
+        "hoccl_copy_launch": (i, [vp, vp, sz, i, vp]),
+        "hoccl_plan_build": (i, [vpp, i, i, sz, i, i, sz, i, ctypes.c_char_p]),
+        "hoccl_plan_slot_bytes": (sz, [vp]),
+        "hoccl_plan_destroy": (None, [vp]),
+        "hoccl_plan_num_ops": (i, [vp]),
+        "hoccl_plan_num_groups": (i, [vp]),
+        "hoccl_plan_get_op": (i, [vp, i, ctypes.POINTER(PlanOp)]),
+        "hoccl_plan_group_deps": (i, [vp, i, ctypes.POINTER(i), i]),
+    }
+    for name, (res, args) in sigs.items():
+        fn = getattr(L, name)
+        fn.restype = res
+        fn.argtypes = args
+    _lib = L
+    return L
+
+
+def error_string(code: int) -> str:
+    return lib().hoccl_error_string(code).decode()
+
+
+def _ptr(x) -> int:
+    if x is None:
+        return 0
+    if hasattr(x, "data_ptr"):
+        return int(x.data_ptr())
+    return int(x)
+
+
+def _ptr_array(xs: Sequence):
+    arr = (ctypes.c_void_p * len(xs))()
+    for k, x in enumerate(xs):
+        arr[k] = _ptr(x)
+    return arr
+
+
+def _stream(s) -> int:
+    if s is None:
+        import torch
+
+        return int(torch.cuda.current_stream().cuda_stream)
+    if hasattr(s, "cuda_stream"):
+        return int(s.cuda_stream)
+    return int(s)
+
+
+def _dtype(d) -> int:
+    if isinstance(d, str):
+        return DTYPES[d]
+    return int(d)
+
+
+class Comm:
+    """Owner of one hoccl_comm_t.  Methods carry the C names without the prefix."""
+
+    def __init__(self, R: int, device: int = 0):
+        self._h = ctypes.c_void_p()
+        self.R = R
+        rc = lib().hoccl_comm_init(ctypes.byref(self._h), R, device)
+        if rc != OK:
+            self._h = ctypes.c_void_p()
+            raise HocclError(rc, "hoccl_comm_init")
+        self._keep = []
+
+    # -- helpers
+    def _check(self, rc: int, what: str):
+        if rc != OK:
+            raise HocclError(rc, what, self.last_cuda_error() if rc == ERR_CUDA else "")
+
+    def last_cuda_error(self) -> str:
+        return lib().hoccl_last_cuda_error(self._h).decode()
+
+    def destroy(self):
+        if self._h:
+            rc = lib().hoccl_comm_destroy(self._h)
+            if rc == OK:
+                self._h = ctypes.c_void_p()
+            return rc
+        return OK
+
+    def __del__(self):
+        try:
+            if self._h:
+                lib().hoccl_comm_destroy(self._h)
+        except Exception:
+            pass
+
+    # -- configuration
+    def set_scratch(self, buf, nbytes: Optional[int] = None):
+        if nbytes is None:
+            nbytes = buf.numel() * buf.element_size() if buf is not None else 0
+        self._keep = [b for b in self._keep if b[0] != "scratch"] + [("scratch", buf)]
+        self._check(lib().hoccl_comm_set_scratch(self._h, _ptr(buf), nbytes), "hoccl_comm_set_scratch")
+
+    def set_staging(self, buf, nbytes: Optional[int] = None):
+        if nbytes is None:
+            nbytes = buf.numel() * buf.element_size() if buf is not None else 0
+        self._keep = [b for b in self._keep if b[0] != "staging"] + [("staging", buf)]
+        self._check(lib().hoccl_comm_set_staging(self._h, _ptr(buf), nbytes), "hoccl_comm_set_staging")
+
+    def set_path(self, path: int):
+        self._check(lib().hoccl_comm_set_path(self._h, path), "hoccl_comm_set_path")
+
+    def set_param(self, key: str, value: int):
+        self._check(lib().hoccl_comm_set_param(self._h, key.encode(), value), "hoccl_comm_set_param(%s)" % key)
+
+    def get_param(self, key: str) -> int:
+        v = ctypes.c_long()
+        self._check(lib().hoccl_comm_get_param(self._h, key.encode(), ctypes.byref(v)), "hoccl_comm_get_param(%s)" % key)
+        return v.value
+
+    # -- collectives (raise on error; the *_rc variants return the code)
+    def allreduce_rc(self, send, recv, count, dtype, stream=None, op=SUM) -> int:
+        return lib().hoccl_allreduce(_ptr_array(send), _ptr_array(recv), count, _dtype(dtype), op, self._h, _stream(stream))
+
+    def reduce_scatter_rc(self, send, recv, count, dtype, stream=None, op=SUM) -> int:
+        return lib().hoccl_reduce_scatter(_ptr_array(send), _ptr_array(recv), count, _dtype(dtype), op, self._h, _stream(stream))
+
+    def allgather_rc(self, send, recv, count, dtype, stream=None) -> int:
+        return lib().hoccl_allgather(_ptr_array(send), _ptr_array(recv), count, _dtype(dtype), self._h, _stream(stream))
+
+    def allreduce(self, send, recv, count, dtype, stream=None, op=SUM):
+        self._check(self.allreduce_rc(send, recv, count, dtype, stream, op), "hoccl_allreduce")
+
+    def reduce_scatter(self, send, recv, count, dtype, stream=None, op=SUM):
+        self._check(self.reduce_scatter_rc(send, recv, count, dtype, stream, op), "hoccl_reduce_scatter")
+
+    def allgather(self, send, recv, count, dtype, stream=None):
+        self._check(self.allgather_rc(send, recv, count, dtype, stream), "hoccl_allgather")
+
+    def host_allreduce(self, h_send, h_recv, count, dtype, stream=None, op=SUM):
+        self._check(lib().hoccl_host_allreduce(_ptr_array(h_send), _ptr_array(h_recv), count, _dtype(dtype), op, self._h,
+                                               _stream(stream)), "hoccl_host_allreduce")
+
+    # -- point to point
+    def send_rc(self, buf, count, dtype, src, dst, stream=None) -> int:
+        return lib().hoccl_send(_ptr(buf), count, _dtype(dtype), src, dst, self._h, _stream(stream))
+
+    def recv_rc(self, buf, count, dtype, src, dst, stream=None) -> int:
+        return lib().hoccl_recv(_ptr(buf), count, _dtype(dtype), src, dst, self._h, _stream(stream))
+
+    def send(self, buf, count, dtype, src, dst, stream=None):
+        self._check(self.send_rc(buf, count, dtype, src, dst, stream), "hoccl_send")
+
+    def recv(self, buf, count, dtype, src, dst, stream=None):
+        self._check(self.recv_rc(buf, count, dtype, src, dst, stream), "hoccl_recv")
+
+    def pending(self) -> int:
+        return lib().hoccl_comm_pending(self._h)
+
+    # -- diagnostics
+    def last_stats(self) -> dict:
+        st = Stats()
+        self._check(lib().hoccl_last_stats(self._h, ctypes.byref(st)), "hoccl_last_stats")
+        return st.as_dict()
+
+    def profile_reset(self):
+        self._check(lib().hoccl_profile_reset(self._h), "hoccl_profile_reset")
+
+    def probe_move_needs_sm(self, path, dst, src, nbytes, spin_us=3000):
+        needs = ctypes.c_int()
+        end_us = ctypes.c_double()
+        self._check(lib().hoccl_probe_move_needs_sm(self._h, path, _ptr(dst), _ptr(src), nbytes, spin_us, ctypes.byref(needs),
+                                                    ctypes.byref(end_us)), "hoccl_probe_move_needs_sm")
+        return bool(needs.value), end_us.value
+
+
+def scratch_bytes(R: int, max_count: int, dtype) -> int:
+    return int(lib().hoccl_scratch_bytes(R, max_count, _dtype(dtype)))
+
+
+def sum_launch(inbox, local, out, count, dtype, ctas, stream=None) -> int:
+    return lib().hoccl_sum_launch(_ptr(inbox), _ptr(local), _ptr(out), count, _dtype(dtype), ctas, _stream(stream))
+
+
+def copy_launch(src, dst, nbytes, ctas, stream=None) -> int:
+    return lib().hoccl_copy_launch(_ptr(src), _ptr(dst), nbytes, ctas, _stream(stream))
+
+
+class Plan:
+    """Host-only view of the planner's output."""
+
+    def __init__(self, kind, R, count, dtype, in_place=False, piece_bytes=4 << 20, max_pieces=8, send_align=None):
+        self._h = ctypes.c_void_p()
+        align = bytes(send_align) if send_align is not None else None
+        rc = lib().hoccl_plan_build(ctypes.byref(self._h), kind, R, count, _dtype(dtype), int(in_place), piece_bytes, max_pieces,
+                                    align)
+        if rc != OK:
+            raise HocclError(rc, "hoccl_plan_build")
+        L = lib()
+        self.slot_bytes = int(L.hoccl_plan_slot_bytes(self._h))
+        self.ops = []
+        for k in range(L.hoccl_plan_num_ops(self._h)):
+            op = PlanOp()
+            assert L.hoccl_plan_get_op(self._h, k, ctypes.byref(op)) == OK
+            self.ops.append({f: getattr(op, f) for f, _ in PlanOp._fields_})
+        self.num_groups = L.hoccl_plan_num_groups(self._h)
+        self.deps = []
+        for g in range(self.num_groups):
+            buf = (ctypes.c_int * 64)()
+            n = L.hoccl_plan_group_deps(self._h, g, buf, 64)
+            self.deps.append([buf[k] for k in range(n)])
+        L.hoccl_plan_destroy(self._h)
+        self._h = None

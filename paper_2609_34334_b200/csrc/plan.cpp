@@ -1,0 +1,223 @@
+// Ring planner (see plan.h).  Ring reduce-scatter followed by ring all-gather; the paper has no
+// reduction (Sec. 4 "Limitations"), so the reduce-scatter is the textbook ring with rank r ending
+// as the owner of chunk r.
+#include "plan.h"
+
+#include <algorithm>
+
+namespace hoccl {
+
+size_t dtype_size(int dtype) { return dtype == 0 ? 4 : (dtype == 1 ? 2 : 0); }
+
+static size_t round_up(size_t v, size_t m) { return (v + m - 1) / m * m; }
+
+size_t slot_bytes_for(int R, size_t count, size_t elem) {
+  if (R <= 1 || count == 0) return 0;
+  size_t q = (count + (size_t)R - 1) / (size_t)R;
+  // one chunk plus 16 bytes of alignment slack per piece; pieces are at least 1024 bytes
+  return round_up(q * elem + (q * elem / 1024 + 2) * 16, 256);
+}
+
+void Plan::chunk_range(int c, size_t* lo, size_t* hi) const {
+  if (kind == PLAN_ALLREDUCE) {
+    size_t a = (size_t)c * chunk_elems, b = ((size_t)c + 1) * chunk_elems;
+    *lo = std::min(a, count);
+    *hi = std::min(b, count);
+  } else {
+    *lo = (size_t)c * count;
+    *hi = *lo + count;
+  }
+}
+
+namespace {
+
+int mod(int a, int R) { return ((a % R) + R) % R; }
+
+struct Builder {
+  Plan* P;
+  int cur_group = -1;
+
+  int begin_group(int kind, int phase, int step, int piece) {
+    PlanGroup g;
+    g.kind = kind;
+    g.phase = phase;
+    g.step = step;
+    g.piece = piece;
+    g.first_op = (int)P->ops.size();
+    g.num_ops = 0;
+    g.chain_dep = -1;
+    P->groups.push_back(g);
+    cur_group = (int)P->groups.size() - 1;
+    return cur_group;
+  }
+  // drops the group again if nothing was added to it; returns its id or -1
+  int end_group() {
+    int g = cur_group;
+    cur_group = -1;
+    if (P->groups[g].num_ops == 0) {
+      P->groups.pop_back();
+      return -1;
+    }
+    return g;
+  }
+  void add(PlanOp op) {
+    if (op.bytes == 0) return;
+    op.group = cur_group;
+    P->ops.push_back(op);
+    P->groups[cur_group].num_ops++;
+  }
+};
+
+// piece p of a chunk of len_bytes bytes: [off, off+len)
+void piece_span(const Plan& P, size_t len_bytes, int p, size_t* off, size_t* len) {
+  size_t a = (size_t)p * P.piece_bytes;
+  size_t b = a + P.piece_bytes;
+  a = std::min(a, len_bytes);
+  b = std::min(b, len_bytes);
+  *off = a;
+  *len = b - a;
+}
+
+}  // namespace
+
+bool build_plan(Plan* plan, int kind, int R, size_t count, int dtype, bool in_place, size_t piece_bytes, int max_pieces,
+                const unsigned char* send_align) {
+  size_t e = dtype_size(dtype);
+  if (!plan || R < 1 || e == 0 || kind < PLAN_ALLREDUCE || kind > PLAN_ALLGATHER) return false;
+  if (max_pieces < 1) max_pieces = 1;
+  if (piece_bytes < 1024) piece_bytes = 1024;
+  Plan& P = *plan;
+  P = Plan();
+  P.kind = kind;
+  P.R = R;
+  P.dtype = dtype;
+  P.count = count;
+  P.in_place = in_place;
+  P.elem = e;
+  P.chunk_elems = (kind == PLAN_ALLREDUCE) ? (count + (size_t)R - 1) / (size_t)R : count;
+  size_t chunk_bytes = P.chunk_elems * e;
+  // piece geometry: at most max_pieces pieces of equal size (multiple of 1024 bytes)
+  size_t want = (chunk_bytes + piece_bytes - 1) / piece_bytes;
+  size_t np = std::max<size_t>(1, std::min<size_t>(want, (size_t)max_pieces));
+  size_t plen = round_up((chunk_bytes + np - 1) / np, 1024);
+  if (plen == 0) plen = 1024;
+  P.piece_bytes = plen;
+  P.pieces = (int)std::max<size_t>(1, (chunk_bytes + plen - 1) / plen);
+  P.slot_bytes = (kind == PLAN_ALLGATHER || R == 1) ? 0 : round_up(chunk_bytes + 16 * (size_t)P.pieces, 256);
+  if (count == 0) return true;
+  // Where piece p of chunk c sits inside a scratch slot of rank r: every piece has its own region with 16
+  // bytes of slack, and inside it the data is shifted by the 16-byte phase of the operand it is summed with
+  // (rank r's send data of chunk c), so that the three SUM operands stay congruent modulo 16.
+  auto slot_off = [&](int r, int c, int p) -> uint64_t {
+    size_t lo, hi;
+    P.chunk_range(c, &lo, &hi);
+    size_t phase = ((send_align ? (size_t)(send_align[r] & 15) : 0) + lo * e) & 15;
+    return (uint64_t)p * (P.piece_bytes + 16) + phase;
+  };
+
+  Builder B{&P};
+  const int np_i = P.pieces;
+
+  if (R == 1) {
+    if (!in_place) {
+      for (int p = 0; p < np_i; p++) {
+        size_t off, len;
+        piece_span(P, chunk_bytes, p, &off, &len);
+        B.begin_group(OP_MOVE, PHASE_OWN, 0, p);
+        B.add(PlanOp{OP_MOVE, PHASE_OWN, 0, p, 0, 0, 0, BUF_SEND, BUF_RECV, -1, off, off, 0, len, 0});
+        B.end_group();
+      }
+    }
+    return true;
+  }
+
+  std::vector<int> last_sum(np_i, -1);   // SUM group of the previous step, per piece
+  std::vector<int> final_sum(np_i, -1);  // SUM group of step R-2, per piece
+  int prev_sum_group = -1;
+
+  if (kind != PLAN_ALLGATHER) {
+    for (int s = 0; s <= R - 2; s++) {
+      for (int p = 0; p < np_i; p++) {
+        // ---- MOVE(s, r, p): chunk c = (r-1-s) mod R leaves rank r for the inbox of rank r+1
+        int gm = B.begin_group(OP_MOVE, PHASE_RS, s, p);
+        for (int r = 0; r < R; r++) {
+          int c = mod(r - 1 - s, R);
+          size_t lo, hi, off, len;
+          P.chunk_range(c, &lo, &hi);
+          piece_span(P, (hi - lo) * e, p, &off, &len);
+          PlanOp op{OP_MOVE, PHASE_RS, s, p, r, (r + 1) % R, c, s == 0 ? BUF_SEND : BUF_PARTIAL, BUF_INBOX, -1,
+                    s == 0 ? lo * e + off : slot_off(r, c, p), slot_off((r + 1) % R, c, p), 0, len, 0};
+          B.add(op);
+        }
+        gm = B.end_group();
+        if (gm >= 0 && s > 0 && last_sum[p] >= 0) P.groups[gm].deps.push_back(last_sum[p]);
+        // ---- SUM(s, r, p): chunk c = (r-2-s) mod R: inbox + own contribution
+        int gs = B.begin_group(OP_SUM, PHASE_RS, s, p);
+        for (int r = 0; r < R; r++) {
+          int c = mod(r - 2 - s, R);
+          size_t lo, hi, off, len;
+          P.chunk_range(c, &lo, &hi);
+          piece_span(P, (hi - lo) * e, p, &off, &len);
+          bool last = (s == R - 2);
+          uint64_t out_off = last ? ((kind == PLAN_ALLREDUCE ? lo * e : 0) + off) : slot_off(r, c, p);
+          PlanOp op{OP_SUM, PHASE_RS, s, p, r, r, c, BUF_INBOX, last ? BUF_RECV : BUF_PARTIAL, BUF_SEND,
+                    slot_off(r, c, p), out_off, lo * e + off, len, 0};
+          B.add(op);
+        }
+        gs = B.end_group();
+        if (gs >= 0) {
+          if (gm >= 0) P.groups[gs].deps.push_back(gm);
+          P.groups[gs].chain_dep = prev_sum_group;
+          prev_sum_group = gs;
+          last_sum[p] = gs;
+          if (s == R - 2) final_sum[p] = gs;
+        }
+      }
+    }
+  }
+
+  if (kind != PLAN_REDUCE_SCATTER) {
+    const bool standalone = (kind == PLAN_ALLGATHER);
+    if (standalone && !in_place) {
+      // own chunk: Y_r[chunk r] <- X_r (independent of the ring: step 0 reads X_r directly)
+      for (int p = 0; p < np_i; p++) {
+        B.begin_group(OP_MOVE, PHASE_OWN, 0, p);
+        for (int r = 0; r < R; r++) {
+          size_t lo, hi, off, len;
+          P.chunk_range(r, &lo, &hi);
+          piece_span(P, (hi - lo) * e, p, &off, &len);
+          B.add(PlanOp{OP_MOVE, PHASE_OWN, 0, p, r, r, r, BUF_SEND, BUF_RECV, -1, off, lo * e + off, 0, len, 0});
+        }
+        B.end_group();
+      }
+    }
+    std::vector<int> last_ag(np_i, -1);
+    for (int s = 0; s <= R - 2; s++) {
+      for (int p = 0; p < np_i; p++) {
+        // ---- AG MOVE(s, r, p): final chunk c = (r-s) mod R goes from Y_r to the same place in Y_{r+1}
+        int g = B.begin_group(OP_MOVE, PHASE_AG, s, p);
+        for (int r = 0; r < R; r++) {
+          int c = mod(r - s, R);
+          size_t lo, hi, off, len;
+          P.chunk_range(c, &lo, &hi);
+          piece_span(P, (hi - lo) * e, p, &off, &len);
+          bool from_send = standalone && !in_place && s == 0;
+          B.add(PlanOp{OP_MOVE, PHASE_AG, s, p, r, (r + 1) % R, c, from_send ? BUF_SEND : BUF_RECV, BUF_RECV, -1,
+                       from_send ? off : lo * e + off, lo * e + off, 0, len, 0});
+        }
+        g = B.end_group();
+        if (g >= 0) {
+          if (s == 0) {
+            if (!standalone && final_sum[p] >= 0) P.groups[g].deps.push_back(final_sum[p]);
+          } else if (last_ag[p] >= 0) {
+            P.groups[g].deps.push_back(last_ag[p]);
+          }
+          last_ag[p] = g;
+        }
+      }
+    }
+  }
+  return true;
+}
+
+}  // namespace hoccl

@@ -1,0 +1,69 @@
+// Host-side planner: a ring collective becomes a DAG of groups of chunk-piece operations.
+//
+// The paper's collective scheduler turns a collective into stages of point-to-point flows and cuts
+// the flows into fixed-size chunks for the copy queue (Sec. 3.4, "Topo-aware flow schedule" and
+// "Flow-size-aware chunk scheduling").  On one device every ring step is one permutation stage
+// (rank r -> rank r+1) and all flows of a stage have the same size, so the weighted interleaving
+// degenerates to round-robin over ranks.  Pieces of a chunk give the pipelining of Sec. 3.3
+// ("chunk pipelining"): the move of piece p+1 overlaps the sum of piece p.
+//
+// Pure C++: no CUDA types, testable without a GPU.
+#pragma once
+#include <cstddef>
+#include <cstdint>
+#include <vector>
+
+namespace hoccl {
+
+enum PlanKind { PLAN_ALLREDUCE = 0, PLAN_REDUCE_SCATTER = 1, PLAN_ALLGATHER = 2 };
+enum OpKind { OP_MOVE = 0, OP_SUM = 1 };
+enum BufKind { BUF_SEND = 0, BUF_RECV = 1, BUF_INBOX = 2, BUF_PARTIAL = 3 };
+enum Phase { PHASE_RS = 0, PHASE_AG = 1, PHASE_OWN = 2 };
+
+struct PlanOp {
+  int kind;
+  int phase, step, piece;
+  int rank, dst_rank, chunk;
+  int src_buf, dst_buf, local_buf;
+  uint64_t src_off, dst_off, local_off;  // bytes from the start of the buffer (scratch: from the start of the rank's slot)
+  uint64_t bytes;
+  int group;
+};
+
+struct PlanGroup {
+  int kind;  // OpKind of every op in the group
+  int phase, step, piece;
+  int first_op, num_ops;
+  std::vector<int> deps;  // data dependencies (group ids, all smaller than this group's id)
+  int chain_dep;          // previous SUM group in issue order (-1 if none): keeps SUM launches serial
+};
+
+struct Plan {
+  int kind = 0, R = 0, dtype = 0;
+  size_t count = 0;
+  bool in_place = false;
+  size_t elem = 4;
+  size_t chunk_elems = 0;   // q: elements of a full ring chunk
+  size_t piece_bytes = 0;   // bytes of a full piece (multiple of 1024 unless the chunk is one piece)
+  int pieces = 1;
+  size_t slot_bytes = 0;    // bytes of one scratch slot (inbox or partial) of one rank, padded
+  std::vector<PlanOp> ops;
+  std::vector<PlanGroup> groups;
+
+  // element range [lo, hi) of ring chunk c inside the rank buffer that holds all R chunks
+  void chunk_range(int c, size_t* lo, size_t* hi) const;
+};
+
+size_t dtype_size(int dtype);  // 0 if unknown
+
+// upper bound of the scratch slot size (bytes) for one rank and one slot kind, whatever the piece
+// settings: one ring chunk + 16 bytes of alignment slack per piece, rounded up to 256
+size_t slot_bytes_for(int R, size_t count_allreduce_convention, size_t elem);
+
+// Returns false on invalid arguments.  `count` follows the collective's convention.  send_align (R entries
+// or NULL for "all 16-byte aligned") gives the low 4 bits of each rank's send pointer; it only decides where
+// inside its scratch region a piece is placed.
+bool build_plan(Plan* plan, int kind, int R, size_t count, int dtype, bool in_place, size_t piece_bytes, int max_pieces,
+                const unsigned char* send_align);
+
+}  // namespace hoccl

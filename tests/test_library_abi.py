@@ -1,0 +1,64 @@
+"""The C-ABI library builds, loads and exports every symbol include/hoccl.h declares (no GPU needed)."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2609_34334_b200 import binding as hb
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared_functions():
+    text = open(os.path.join(ROOT, "include", "hoccl.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(hoccl_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported():
+    L = hb.lib()
+    names = _declared_functions()
+    assert len(names) >= 25
+    for n in names:
+        assert hasattr(L, n), n
+    assert sorted(hb.EXPORTS) == names, (set(names) ^ set(hb.EXPORTS))
+
+
+def test_error_strings_and_sizes():
+    assert hb.error_string(hb.OK) == "ok"
+    for code in range(1, 8):
+        assert hb.error_string(code) and hb.error_string(code) != "ok"
+    assert hb.scratch_bytes(1, 1000, "fp32") == 0
+    assert hb.scratch_bytes(8, 0, "bf16") == 0
+    # 2 slots per rank, each one ring chunk + slack, padded to 256
+    n = 13_107_200
+    b = hb.scratch_bytes(8, n, "bf16")
+    chunk = n // 8 * 2
+    assert b >= 2 * 8 * chunk and b <= 2 * 8 * (chunk + chunk // 64 + 512)
+    assert b % 256 == 0
+
+
+def test_argument_errors_need_no_device():
+    L = hb.lib()
+    h = ctypes.c_void_p()
+    assert L.hoccl_comm_init(None, 4, 0) == hb.ERR_INVALID_ARG
+    assert L.hoccl_comm_init(ctypes.byref(h), 0, 0) == hb.ERR_INVALID_ARG
+    assert L.hoccl_comm_init(ctypes.byref(h), 65, 0) == hb.ERR_INVALID_ARG
+    assert L.hoccl_comm_destroy(None) == hb.ERR_INVALID_ARG
+    assert L.hoccl_sum_launch(None, None, None, 4, 0, 8, None) == hb.ERR_INVALID_ARG
+    assert L.hoccl_sum_launch(16, 32, 48, 4, 7, 8, None) == hb.ERR_UNSUPPORTED
+    assert L.hoccl_sum_launch(18, 32, 48, 4, 0, 8, None) == hb.ERR_INVALID_ARG      # misaligned for fp32
+    p = ctypes.c_void_p()
+    assert L.hoccl_plan_build(ctypes.byref(p), 0, 0, 10, 0, 0, 4096, 8, None) == hb.ERR_INVALID_ARG
+    assert L.hoccl_plan_build(ctypes.byref(p), 0, 4, 10, 9, 0, 4096, 8, None) == hb.ERR_UNSUPPORTED
+
+
+def test_no_device_fails_loudly():
+    """Without a CUDA device the product path reports an error; it never falls back to the CPU."""
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a device is present")
+    with pytest.raises(hb.HocclError) as ei:
+        hb.Comm(4, 0)
+    assert ei.value.code == hb.ERR_CUDA

@@ -1,0 +1,211 @@
+"""Host-only checks of the ring planner through the C ABI (hoccl_plan_*).
+
+The plan is executed here by a small interpreter (numpy copies for MOVE, numpy float32 adds for SUM)
+in RANDOM topological orders of its group DAG and compared bit for bit with the CPU oracle: a missing
+dependency, a wrong offset or a wrong chunk index shows up as a wrong result.  Structural rules are
+checked as well: rank locality of every SUM, every ring MOVE crosses exactly one rank boundary, every
+byte of every chunk is covered exactly once per step, scratch slots are never exceeded.
+"""
+import random
+
+import numpy as np
+import pytest
+
+from paper_2609_34334_b200 import binding as hb
+from paper_2609_34334_b200 import workloads as W
+
+PHASE_RS, PHASE_AG, PHASE_OWN = 0, 1, 2
+
+
+def _topo_order(num_groups, deps, rng):
+    indeg = [len(d) for d in deps]
+    users = [[] for _ in range(num_groups)]
+    for g, ds in enumerate(deps):
+        for d in ds:
+            assert 0 <= d < g, "dependencies must point to earlier groups (acyclic by construction)"
+            users[d].append(g)
+    ready = [g for g in range(num_groups) if indeg[g] == 0]
+    order = []
+    while ready:
+        g = ready.pop(rng.randrange(len(ready)))
+        order.append(g)
+        for u in users[g]:
+            indeg[u] -= 1
+            if indeg[u] == 0:
+                ready.append(u)
+    assert len(order) == num_groups
+    return order
+
+
+def _run_plan(plan, kind, R, count, dtype, xs, in_place, rng):
+    e = W.elem_size(dtype)
+    npdt = np.float32 if dtype == "fp32" else np.uint16
+    if kind == hb.PLAN_ALLREDUCE:
+        send_n, recv_n = count, count
+    elif kind == hb.PLAN_REDUCE_SCATTER:
+        send_n, recv_n = R * count, count
+    else:
+        send_n, recv_n = count, R * count
+    slot = plan.slot_bytes
+    if R > 1 and count > 0 and kind != hb.PLAN_ALLGATHER:
+        assert 0 < slot <= hb.scratch_bytes(R, send_n, dtype) // (2 * R)      # the advertised bound covers any piece setting
+    send = [x.copy().view(np.uint8) for x in xs]
+    if in_place:
+        if kind == hb.PLAN_ALLREDUCE:
+            recv = send
+        elif kind == hb.PLAN_REDUCE_SCATTER:
+            recv = [send[r][r * count * e:(r + 1) * count * e] for r in range(R)]
+        else:
+            recv = [np.zeros(recv_n * e, dtype=np.uint8) for _ in range(R)]
+            for r in range(R):
+                recv[r][r * count * e:(r + 1) * count * e] = send[r]
+                send[r] = recv[r][r * count * e:(r + 1) * count * e]
+    else:
+        recv = [np.full(recv_n * e, 0xAB, dtype=np.uint8) for _ in range(R)]
+    inbox = [np.full(slot, 0xCD, dtype=np.uint8) for _ in range(R)]
+    partial = [np.full(slot, 0xEF, dtype=np.uint8) for _ in range(R)]
+    bufs = {hb.BUF_SEND: send, hb.BUF_RECV: recv, hb.BUF_INBOX: inbox, hb.BUF_PARTIAL: partial}
+    by_group = {}
+    for op in plan.ops:
+        by_group.setdefault(op["group"], []).append(op)
+    for g in _topo_order(plan.num_groups, plan.deps, rng):
+        ops = by_group[g]
+        rng.shuffle(ops)           # ops of one group are independent of each other
+        for op in ops:
+            n = op["bytes"]
+            assert n > 0 and n % e == 0
+            src = bufs[op["src_buf"]][op["rank"]][op["src_off"]:op["src_off"] + n]
+            assert src.size == n
+            if op["kind"] == hb.OP_MOVE:
+                dst = bufs[op["dst_buf"]][op["dst_rank"]]
+                assert op["dst_off"] + n <= dst.size
+                dst[op["dst_off"]:op["dst_off"] + n] = src
+            else:
+                assert dtype == "fp32"
+                loc = bufs[op["local_buf"]][op["rank"]][op["local_off"]:op["local_off"] + n]
+                out = bufs[op["dst_buf"]][op["rank"]]
+                assert op["dst_off"] + n <= out.size
+                res = (src.view(np.float32) + loc.view(np.float32)).view(np.uint8)
+                out[op["dst_off"]:op["dst_off"] + n] = res
+    return [r.view(npdt) for r in recv]
+
+
+CASES = [(R, n, pb, mp) for R in (1, 2, 3, 4, 8) for (n, pb, mp) in
+         ((0, 4096, 8), (1, 4096, 8), (5, 1024, 4), (R * 1024, 1024, 3), (R * 1024 + 3, 1024, 8), (4099, 2048, 2), (70001, 8192, 8))]
+
+
+@pytest.mark.parametrize("R,n,piece_bytes,max_pieces", CASES)
+def test_allreduce_plan_executes_to_oracle_bits(oracle, R, n, piece_bytes, max_pieces):
+    rng = random.Random(R * 1000 + n)
+    xs = W.rank_inputs("uniform", 17, R, n, "fp32")
+    want = oracle.ring_allreduce(xs)
+    for in_place in (False, True):
+        align = [(4 * rng.randrange(4)) for _ in range(R)] if in_place else None
+        plan = hb.Plan(hb.PLAN_ALLREDUCE, R, n, "fp32", in_place, piece_bytes, max_pieces, align)
+        # SUM operands share their 16-byte phase (vector path), whatever the send pointers' alignment
+        for op in plan.ops:
+            if op["kind"] == hb.OP_SUM:
+                a = align[op["rank"]] if align else 0
+                assert op["src_off"] % 16 == (a + op["local_off"]) % 16
+                if op["dst_buf"] == hb.BUF_PARTIAL:
+                    assert op["dst_off"] % 16 == op["src_off"] % 16
+        for trial in range(2):
+            got = _run_plan(plan, hb.PLAN_ALLREDUCE, R, n, "fp32", xs, in_place, rng)
+            for r in range(R):
+                assert (got[r].view(np.uint32) == want[r].view(np.uint32)).all(), (R, n, in_place, r)
+
+
+@pytest.mark.parametrize("R", [1, 2, 4, 8])
+@pytest.mark.parametrize("count", [1, 7, 1024, 3001])
+def test_reduce_scatter_and_allgather_plans(oracle, R, count):
+    rng = random.Random(R * 77 + count)
+    xs = W.rank_inputs("uniform", 23, R, R * count, "fp32")
+    want = oracle.ring_reduce_scatter(xs)
+    for in_place in (False, True):
+        plan = hb.Plan(hb.PLAN_REDUCE_SCATTER, R, count, "fp32", in_place, 2048, 4)
+        got = _run_plan(plan, hb.PLAN_REDUCE_SCATTER, R, count, "fp32", xs, in_place, rng)
+        for r in range(R):
+            assert (got[r].view(np.uint32) == want[r].view(np.uint32)).all()
+    for dtype in ("fp32", "bf16"):
+        ys = W.rank_inputs("uniform", 29, R, count, dtype)
+        cat = np.concatenate(ys)
+        for in_place in (False, True):
+            plan = hb.Plan(hb.PLAN_ALLGATHER, R, count, dtype, in_place, 1024, 8)
+            assert all(op["kind"] == hb.OP_MOVE for op in plan.ops)
+            got = _run_plan(plan, hb.PLAN_ALLGATHER, R, count, dtype, ys, in_place, rng)
+            for r in range(R):
+                assert (got[r] == cat).all()
+
+
+@pytest.mark.parametrize("R,n", [(2, 100), (4, 1 << 20), (8, 13_107_200), (8, 1001), (5, 12345)])
+def test_structure_rules(R, n):
+    e = 4
+    plan = hb.Plan(hb.PLAN_ALLREDUCE, R, n, "fp32", False, 1 << 20, 8)
+    q = -(-n // R)
+    lo = [min(c * q, n) for c in range(R)]
+    hi = [min((c + 1) * q, n) for c in range(R)]
+    sums = [op for op in plan.ops if op["kind"] == hb.OP_SUM]
+    moves = [op for op in plan.ops if op["kind"] == hb.OP_MOVE]
+    # rank locality: a SUM touches one rank only; its operands are inbox + own send data
+    for op in sums:
+        assert op["rank"] == op["dst_rank"]
+        assert op["src_buf"] == hb.BUF_INBOX and op["local_buf"] == hb.BUF_SEND
+        assert op["chunk"] == (op["rank"] - 2 - op["step"]) % R
+        assert op["dst_buf"] == (hb.BUF_RECV if op["step"] == R - 2 else hb.BUF_PARTIAL)
+        assert op["src_off"] + op["bytes"] <= plan.slot_bytes
+    # every ring MOVE crosses exactly one rank boundary, towards rank+1
+    for op in moves:
+        assert op["phase"] in (PHASE_RS, PHASE_AG)
+        assert op["dst_rank"] == (op["rank"] + 1) % R and op["dst_rank"] != op["rank"]
+        if op["phase"] == PHASE_RS:
+            assert op["chunk"] == (op["rank"] - 1 - op["step"]) % R
+            assert op["dst_buf"] == hb.BUF_INBOX
+            assert op["src_buf"] == (hb.BUF_SEND if op["step"] == 0 else hb.BUF_PARTIAL)
+        else:
+            assert op["chunk"] == (op["rank"] - op["step"]) % R
+            assert op["src_buf"] == hb.BUF_RECV and op["dst_buf"] == hb.BUF_RECV and op["src_off"] == op["dst_off"]
+    # coverage: per (phase, step, rank) the pieces tile the chunk exactly once
+    for kind_ops, phase in ((moves, PHASE_RS), (moves, PHASE_AG), (sums, PHASE_RS)):
+        seen = {}
+        for op in kind_ops:
+            if op["phase"] != phase:
+                continue
+            seen.setdefault((op["step"], op["rank"], op["chunk"]), []).append(op)
+        assert len({(s, r) for s, r, _ in seen}) == len(seen)          # one chunk per (step, rank)
+        for (s, r, c), ops in seen.items():
+            total = sum(o["bytes"] for o in ops)
+            assert total == (hi[c] - lo[c]) * e
+            if all(o["dst_buf"] == hb.BUF_RECV for o in ops):
+                spans = sorted((o["dst_off"] - lo[c] * e, o["bytes"]) for o in ops)
+                pos = 0
+                for off, b in spans:
+                    assert off == pos
+                    pos += b
+            else:       # scratch: pieces must not overlap inside the slot
+                spans = sorted((o["dst_off"], o["bytes"]) for o in ops)
+                for (o1, b1), (o2, _) in zip(spans, spans[1:]):
+                    assert o1 + b1 <= o2
+    steps = {op["step"] for op in sums}
+    assert steps == set(range(R - 1))
+    # SUM groups form one chain (the SM budget for sums is global): each has the previous SUM group among its deps
+    sum_groups = sorted({op["group"] for op in sums})
+    for a, b in zip(sum_groups, sum_groups[1:]):
+        assert a in plan.deps[b]
+    # counts: (R-1) steps x R ranks x pieces for each of RS-move, SUM, AG-move when nothing is empty
+    if n % R == 0:
+        pieces = len({op["piece"] for op in plan.ops})
+        assert len(sums) == (R - 1) * R * pieces
+        assert len(moves) == 2 * (R - 1) * R * pieces
+
+
+def test_piece_geometry():
+    # 25 MiB bf16 bucket over 8 ranks: chunk 3,276,800 B
+    plan = hb.Plan(hb.PLAN_ALLREDUCE, 8, 13_107_200, "bf16", False, 1 << 20, 8)
+    pieces = sorted({op["piece"] for op in plan.ops})
+    assert pieces == [0, 1, 2, 3]
+    sizes = {op["bytes"] for op in plan.ops}
+    assert max(sizes) % 1024 == 0 and sum(sorted({(op["piece"], op["bytes"]) for op in plan.ops if op["rank"] == 0 and op["step"] == 0 and op["kind"] == 1}, key=lambda t: t[0])[k][1] for k in range(4)) == 3_276_800
+    one = hb.Plan(hb.PLAN_ALLREDUCE, 8, 13_107_200, "bf16", False, 64 << 20, 8)
+    assert {op["piece"] for op in one.ops} == {0}
+    capped = hb.Plan(hb.PLAN_ALLREDUCE, 2, 1 << 28, "fp32", False, 1 << 20, 8)
+    assert len({op["piece"] for op in capped.ops}) == 8
