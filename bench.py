@@ -351,9 +351,9 @@ def main():
         prof.destroy()
         # the same kernel without the SM budget, timed alone on 256 MiB operands (kernel quality, not the path)
         big = 128 << 20
-        a = torch.empty(big, dtype=torch.int16, device="cuda").normal_(0, 100)
-        b2 = torch.empty(big, dtype=torch.int16, device="cuda").normal_(0, 100)
-        o = torch.empty(big, dtype=torch.int16, device="cuda")
+        a = torch.empty(big, dtype=torch.bfloat16, device="cuda").normal_(0, 1e-3)
+        b2 = torch.empty(big, dtype=torch.bfloat16, device="cuda").normal_(0, 1e-3)
+        o = torch.empty(big, dtype=torch.bfloat16, device="cuda")
         full = {}
         for ctas in (8, 148, 296, 592):
             for _ in range(3):
@@ -433,7 +433,7 @@ def extras(hb, W, torch, np, new_comm, step, timed, stream, R, S, n, dtype, peak
                             "note": "true = the move finished only after a kernel holding every SM had ended"}
 
     # point to point: 64 MiB bf16 activations [4, 2048, 4096]
-    act = torch.empty(4 * 2048 * 4096, dtype=torch.int16, device="cuda").normal_(0, 100)
+    act = torch.empty(4 * 2048 * 4096, dtype=torch.bfloat16, device="cuda").normal_(0, 1)
     slots = [torch.empty_like(act) for _ in range(4)]
     p2p = {}
     for name, path in (("CE", hb.PATH_CE), ("SM8", hb.PATH_SM)):
