@@ -196,6 +196,41 @@ int hoccl_comm_pending(hoccl_comm_t comm);
 hoccl_result_t hoccl_host_allreduce(const void* const* h_send, void* const* h_recv, size_t count, hoccl_dtype_t dtype,
                                     hoccl_op_t op, hoccl_comm_t comm, hoccl_stream_t stream);
 
+/* ---------------------------------------------------------------- no-allocation entry point ---- */
+
+/*
+ * (The paper has no counterpart: this entry point exists for this library's users only.)
+ *
+ * hoccl_allreduce_static: the same ring all-reduce as hoccl_allreduce, bit for bit, for callers that
+ * are not allowed to allocate device memory and therefore have no scratch to attach to a communicator:
+ * for instance a communication thread running beside compute that must never cause the device-wide
+ * synchronisation an allocation can imply, or a process whose device memory was handed out once by a
+ * static memory planner.  It takes no communicator.  Its ring scratch (inbox and partial slots) is a
+ * fixed array of HOCCL_STATIC_SCRATCH_BYTES inside the library image; every GPU that loads the library
+ * holds that array until the process exits.  The call itself allocates nothing: no cudaMalloc or
+ * cudaFree, no stream, event or graph creation; it only launches kernels on `stream`, in order.
+ *
+ * send[r] / recv[r]: HOST arrays of R DEVICE pointers to `count` elements each (caller-owned; same
+ * in-place and no-overlap rules as hoccl_allreduce).  R: number of logical ranks, 1..64.  `stream` must
+ * belong to the device that is current when the call is made.
+ *
+ * Limits and sharing.  The scratch need is 2 * R * roundup256(ceil(count/R) * sizeof(dtype) + 16) bytes;
+ * a call that would need more than HOCCL_STATIC_SCRATCH_BYTES is rejected with HOCCL_ERR_SCRATCH and
+ * enqueues nothing (with R = 8 this allows a little under 16 MiB per rank buffer).  All calls on a device
+ * share the one array, which keeps whatever the last call left in it; nothing in it has to start at
+ * zero, because every byte a sum reads was written by a move of the same call first.  Two calls that
+ * overlap in time on the GPU (different streams, no ordering between them) race on the array: order them.
+ *
+ * First call.  The first call on each device looks up the array's device address (once per device, with
+ * that device current) before it launches anything; make that first call before any stream capture.
+ *
+ * Errors: INVALID_ARG (NULL or misaligned pointer, overlapping buffers, R out of range), UNSUPPORTED
+ * (dtype, op), SCRATCH (beyond the maximum), CUDA (no device, address lookup or launch failed).
+ */
+#define HOCCL_STATIC_SCRATCH_BYTES (32u << 20)
+hoccl_result_t hoccl_allreduce_static(const void* const* send, void* const* recv, size_t count, hoccl_dtype_t dtype,
+                                      hoccl_op_t op, int R, hoccl_stream_t stream);
+
 /* ---------------------------------------------------------------- diagnostics ------------------ */
 
 const char* hoccl_error_string(hoccl_result_t code);

@@ -28,7 +28,7 @@ EXPORTS = [
     "hoccl_allgather", "hoccl_send", "hoccl_recv", "hoccl_comm_pending", "hoccl_host_allreduce", "hoccl_error_string",
     "hoccl_last_cuda_error", "hoccl_last_stats", "hoccl_profile_reset", "hoccl_probe_move_needs_sm", "hoccl_sum_launch",
     "hoccl_copy_launch", "hoccl_plan_build", "hoccl_plan_destroy", "hoccl_plan_num_ops", "hoccl_plan_num_groups",
-    "hoccl_plan_get_op", "hoccl_plan_group_deps", "hoccl_plan_slot_bytes",
+    "hoccl_plan_get_op", "hoccl_plan_group_deps", "hoccl_plan_slot_bytes", "hoccl_allreduce_static",
 ]
 
 
@@ -86,6 +86,7 @@ def lib() -> ctypes.CDLL:
         "hoccl_recv": (i, [vp, sz, i, i, i, vp, vp]),
         "hoccl_comm_pending": (i, [vp]),
         "hoccl_host_allreduce": (i, [vpp, vpp, sz, i, i, vp, vp]),
+        "hoccl_allreduce_static": (i, [vpp, vpp, sz, i, i, i, vp]),
         "hoccl_error_string": (ctypes.c_char_p, [i]),
         "hoccl_last_cuda_error": (ctypes.c_char_p, [vp]),
         "hoccl_last_stats": (i, [vp, ctypes.POINTER(Stats)]),
@@ -257,6 +258,15 @@ class Comm:
         self._check(lib().hoccl_probe_move_needs_sm(self._h, path, _ptr(dst), _ptr(src), nbytes, spin_us, ctypes.byref(needs),
                                                     ctypes.byref(end_us)), "hoccl_probe_move_needs_sm")
         return bool(needs.value), end_us.value
+
+
+STATIC_SCRATCH_BYTES = 32 << 20
+
+
+def allreduce_static(send, recv, count, dtype, R, stream=None, op=SUM) -> int:
+    """hoccl_allreduce_static: all-reduce that allocates nothing and uses the library's fixed scratch array.
+    Returns the result code (OK, or ERR_SCRATCH when the buffers are too large for the fixed array)."""
+    return lib().hoccl_allreduce_static(_ptr_array(send), _ptr_array(recv), count, _dtype(dtype), op, R, _stream(stream))
 
 
 def scratch_bytes(R: int, max_count: int, dtype) -> int:
