@@ -33,9 +33,12 @@ FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0
 N_BUCKET_SETS = 4
 
-# DRAM bytes (read + write) per SUM launch measured with ncu (dram__bytes_read.sum + dram__bytes_write.sum) on the
-# launch shape of this workload (8 segments of 3,276,800 bytes, 8 CTAs); see profiles/.  None until captured.
-NCU_SUM_TRAFFIC_BYTES_PER_LAUNCH = None
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one SUM launch, from the ncu capture summarised in
+# profiles/sum2_kernel_bf16_8cta_200MiB.md: 573.44 MB of traffic for 629.15 MB of algorithmic bytes (operands of
+# 200 MiB, larger than L2; part of the output is still in L2 when the kernel ends).  Traffic grows in proportion to
+# the bytes a launch processes, so it is scaled to this workload's launch (8 segments x 3,276,800 B x 3).
+NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = 573.44 / 629.15
+SM_PORT_GBPS = 123.0   # measured mixed 2:1 read/write ceiling of one SM's memory port (bulk loads + bulk stores)
 
 
 def parse_args():
@@ -234,7 +237,8 @@ def main():
         cm.allgather(rs_out, recv, count, dtype, st)
 
     def timed(cm, k_steps, k_warm, fn=step, sampler=None):
-        for k in range(k_warm):
+        # warm-up touches every bucket set at least once, so every cached graph exists before the timed region
+        for k in range(max(k_warm, N_BUCKET_SETS)):
             fn(cm, k % N_BUCKET_SETS, stream)
         stream.synchronize()
         replicas.barrier(world)
@@ -344,9 +348,11 @@ def main():
         line["roofline"] = {
             "kernel": "sum2_kernel<bf16>", "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
             "frac": achieved / peaks["hbm_gbs"], "peak_source": "of " + peaks["source"],
-            "traffic": NCU_SUM_TRAFFIC_BYTES_PER_LAUNCH, "algorithmic_bytes_per_launch": bytes_per_launch,
+            "traffic": bytes_per_launch * NCU_TRAFFIC_PER_ALGORITHMIC_BYTE, "algorithmic_bytes_per_launch": bytes_per_launch,
             "avg_launch_us": avg_ms * 1e3, "launches_timed": int(nl), "ctas": 8,
-            "note": "8 CTAs by design (SM budget for sums); per-SM rate = achieved/8",
+            "sm_budget_ceiling_GBps": 8 * SM_PORT_GBPS, "frac_of_sm_budget_ceiling": achieved / (8 * SM_PORT_GBPS),
+            "note": "8 CTAs by design (SM budget for sums): the bound is 8 SM memory ports (~123 GB/s each for 2 reads + 1 write), "
+                    "not HBM; roofline_unconstrained is the same kernel on the whole GPU",
         }
         prof.destroy()
         # the same kernel without the SM budget, timed alone on 256 MiB operands (kernel quality, not the path)
@@ -428,9 +434,27 @@ def extras(hb, W, torch, np, new_comm, step, timed, stream, R, S, n, dtype, peak
     nb = min(64 << 20, src.numel() * 2)
     ce_needs, ce_end = cm.probe_move_needs_sm(hb.PATH_CE, dst, src, nb, 3000)
     sm_needs, sm_end = cm.probe_move_needs_sm(hb.PATH_SM, dst, src, nb, 3000)
-    out["move_needs_sm"] = {"CE_driver_copy": ce_needs, "CE_move_end_us": ce_end, "SM_copy_kernel": sm_needs,
-                            "SM_move_end_us": sm_end, "occupancy_kernel_us": 3000,
+    pinned = torch.empty(8 << 20, dtype=torch.uint8).pin_memory()
+    h2d_needs, h2d_end = cm.probe_move_needs_sm(hb.PATH_CE, dst, pinned, pinned.numel(), 3000)
+    out["move_needs_sm"] = {"CE_driver_copy_same_device_64MiB": ce_needs, "CE_move_end_us": ce_end, "SM_copy_kernel": sm_needs,
+                            "SM_move_end_us": sm_end, "control_pinned_host_to_device_8MiB": h2d_needs,
+                            "control_move_end_us": h2d_end, "occupancy_kernel_us": 3000,
                             "note": "true = the move finished only after a kernel holding every SM had ended"}
+    # host cost of one call with an idle queue (the paper's CPU launch overhead axis)
+    host_us = {}
+    for label, use_graph in (("graph_replay", 1), ("stream_executor", 0)):
+        cm.set_param("use_graph", use_graph)
+        step(cm, 0, stream)
+        stream.synchronize()
+        vals = []
+        for _ in range(15):
+            cm.allreduce(send_sets[0], recv_sets[0], n, dtype, stream)
+            vals.append(cm.last_stats()["host_launch_us"])
+            stream.synchronize()
+        vals.sort()
+        host_us[label] = vals[len(vals) // 2]
+    cm.set_param("use_graph", 1)
+    out["host_launch_us_per_allreduce_call_idle_queue"] = host_us
 
     # point to point: 64 MiB bf16 activations [4, 2048, 4096]
     act = torch.empty(4 * 2048 * 4096, dtype=torch.bfloat16, device="cuda").normal_(0, 1)

@@ -246,7 +246,9 @@ hoccl_result_t hoccl_profile_reset(hoccl_comm_t comm);
  * after that kernel ended, 0 if it finished while all SMs were taken.  *move_end_us is the move's
  * completion time measured from the kernel's start.  Synchronises the device.  This is the
  * single-GPU form of the paper's claim that copy-engine transfers occupy no SM (Sec. 2.3).
- * src and dst are device buffers of at least `bytes` bytes.
+ * src and dst are device buffers of at least `bytes` bytes.  On the CE path src may also be PINNED HOST
+ * memory: a host-to-device copy is driven by a copy engine, which makes it the control of the measurement
+ * (it must report needs_sm = 0).
  */
 hoccl_result_t hoccl_probe_move_needs_sm(hoccl_comm_t comm, hoccl_path_t path, void* dst, const void* src, size_t bytes,
                                          int spin_us, int* needs_sm, double* move_end_us);

@@ -79,6 +79,7 @@ struct hoccl_comm {
   long sum_ctas = 8, copy_ctas = 8, piece_bytes = 4 << 20, max_pieces = 8, lanes = 4, use_graph = 1, profile = 0;
   cudaStream_t lane[kMaxLanes] = {};
   cudaStream_t sum_stream = nullptr;
+  int sum_priority = 0;
   std::vector<cudaEvent_t> ev_pool;
   size_t ev_next = 0;
   void* scratch = nullptr;
@@ -366,9 +367,10 @@ hoccl_result_t build_graph(hoccl_comm* c, const Plan& P, const std::vector<RGrou
         fill_sum_batch(rg, first, n, P.dtype, P.elem, &b);
         void* args[] = {&b};
         cudaKernelNodeParams kp = {};
-        kp.func = const_cast<void*>(sum_kernel_entry(P.dtype));
+        int sum_threads = 0;
+        kp.func = const_cast<void*>(sum_kernel_entry(P.dtype, (int)c->sum_ctas, &sum_threads));
         kp.gridDim = dim3((unsigned)c->sum_ctas);
-        kp.blockDim = dim3(kThreads);
+        kp.blockDim = dim3((unsigned)sum_threads);
         kp.kernelParams = args;
         // launches of one group are chained too (they share the SM budget)
         std::vector<cudaGraphNode_t> d2 = nodes.empty() ? deps : std::vector<cudaGraphNode_t>{nodes.back()};
@@ -386,6 +388,10 @@ hoccl_result_t build_graph(hoccl_comm* c, const Plan& P, const std::vector<RGrou
         }
         cudaGraphNode_t kn;
         e = cudaGraphAddKernelNode(&kn, g, d2.data(), d2.size(), &kp);
+        if (e != cudaSuccess) break;
+        cudaLaunchAttributeValue prio = {};
+        prio.priority = c->sum_priority;
+        e = cudaGraphKernelNodeSetAttribute(kn, cudaLaunchAttributePriority, &prio);
         if (e != cudaSuccess) break;
         if (c->profile) {
           cudaGraphNode_t end_rec;
@@ -410,9 +416,10 @@ hoccl_result_t build_graph(hoccl_comm* c, const Plan& P, const std::vector<RGrou
         fill_copy_batch(rg, first, n, &b);
         void* args[] = {&b};
         cudaKernelNodeParams kp = {};
-        kp.func = const_cast<void*>(copy_kernel_entry());
+        int copy_threads = 0;
+        kp.func = const_cast<void*>(copy_kernel_entry((int)c->copy_ctas, &copy_threads));
         kp.gridDim = dim3((unsigned)c->copy_ctas);
-        kp.blockDim = dim3(kThreads);
+        kp.blockDim = dim3((unsigned)copy_threads);
         kp.kernelParams = args;
         cudaGraphNode_t kn;
         e = cudaGraphAddKernelNode(&kn, g, deps.data(), deps.size(), &kp);
@@ -649,7 +656,13 @@ hoccl_result_t hoccl_comm_init(hoccl_comm_t* comm, int R, int device) {
   cudaError_t e = cudaSetDevice(device);
   if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->num_sms, cudaDevAttrMultiProcessorCount, device);
   for (int i = 0; i < kMaxLanes && e == cudaSuccess; i++) e = cudaStreamCreateWithFlags(&c->lane[i], cudaStreamNonBlocking);
-  if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->sum_stream, cudaStreamNonBlocking);
+  // SUM launches get the highest priority: a SUM CTA needs a whole SM (1024 threads x 64 registers), and when a
+  // SUM and the next piece's copies become ready at the same moment the copies' small CTAs would otherwise take
+  // every SM first and the SUM would start only after them, which serialises the pipeline.
+  int prio_least = 0, prio_greatest = 0;
+  if (e == cudaSuccess) e = cudaDeviceGetStreamPriorityRange(&prio_least, &prio_greatest);
+  c->sum_priority = prio_greatest;
+  if (e == cudaSuccess) e = cudaStreamCreateWithPriority(&c->sum_stream, cudaStreamNonBlocking, prio_greatest);
   if (e != cudaSuccess) {
     for (int i = 0; i < kMaxLanes; i++)
       if (c->lane[i]) cudaStreamDestroy(c->lane[i]);
@@ -871,7 +884,7 @@ hoccl_result_t hoccl_probe_move_needs_sm(hoccl_comm_t c, hoccl_path_t path, void
   }
   if (e == cudaSuccess) {
     if (path == HOCCL_PATH_CE) {
-      e = cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToDevice, c->lane[1]);
+      e = cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDefault, c->lane[1]);  // src may be pinned host memory (control)
     } else {
       CopyBatch b;
       b.nseg = 1;

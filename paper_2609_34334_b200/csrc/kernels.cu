@@ -10,8 +10,10 @@
 // segments are flattened into one index space so that a small CTA budget stays balanced.  Loads and
 // stores are 16-byte vectors, fully coalesced (consecutive threads touch consecutive vectors);
 // segments whose three addresses are not congruent modulo 16 fall back to element-wise accesses.
-// No shared-memory or bulk-copy staging: with <= 8 CTAs the per-SM load/store path, not latency, is
-// the limit (measured: a bulk-copy ring of 96-192 KB per SM was slower than plain vector loads).
+// The sum streams CTA-contiguous tiles (blockDim x 4 vectors per operand) with all of a tile's loads in
+// flight before the first add.  No shared-memory or bulk-copy staging: one SM's memory port carries about
+// 123 GB/s of mixed 2:1 read/write traffic whatever issues it (bulk loads + bulk stores measured the same),
+// stores are capped at 32 B/clk per SM, and the register version already reaches 116 GB/s per SM.
 #include "kernels.cuh"
 
 #include <cuda_bf16.h>
@@ -70,6 +72,7 @@ struct Traits<1> {  // bf16
 
 // Flattened view of the batch, built once per CTA in shared memory.
 struct Flat {
+  unsigned long long tpre[kMaxSegs + 1];  // prefix sums of vector tiles (sum kernel)
   unsigned long long vpre[kMaxSegs + 1];  // prefix sums of 16-byte vectors
   unsigned long long spre[kMaxSegs + 1];  // prefix sums of element-wise items
   unsigned long long nvec[kMaxSegs];
@@ -91,8 +94,8 @@ __device__ __forceinline__ void split_segment(unsigned long long n, unsigned mis
   }
 }
 
-template <int DT>
-__global__ void __launch_bounds__(kThreads, 1) sum2_kernel(const __grid_constant__ SumBatch batch) {
+template <int DT, int U, int THREADS>
+__global__ void __launch_bounds__(THREADS, 1) sum2_kernel(const __grid_constant__ SumBatch batch) {
   using T = Traits<DT>;
   __shared__ Flat f;
   const int nseg = batch.nseg;
@@ -109,12 +112,13 @@ __global__ void __launch_bounds__(kThreads, 1) sum2_kernel(const __grid_constant
   }
   __syncthreads();
   if (threadIdx.x == 0) {
-    unsigned long long v = 0, s = 0;
-    f.vpre[0] = 0;
+    unsigned long long t = 0, s = 0;
+    const unsigned long long tile_v = (unsigned long long)U * blockDim.x;
+    f.tpre[0] = 0;
     f.spre[0] = 0;
     for (int k = 0; k < nseg; k++) {
-      v += f.nvec[k];
-      f.vpre[k + 1] = v;
+      t += (f.nvec[k] + tile_v - 1) / tile_v;
+      f.tpre[k + 1] = t;
       s += f.spre[k + 1];
       f.spre[k + 1] = s;
     }
@@ -123,33 +127,44 @@ __global__ void __launch_bounds__(kThreads, 1) sum2_kernel(const __grid_constant
   const unsigned long long total = (unsigned long long)gridDim.x * blockDim.x;
   const unsigned long long gt = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
 
-  // ---- vector body: two independent vectors per thread and iteration
+  // ---- vector body, tile by tile: a tile is a contiguous run of U * blockDim vectors of one segment; the
+  // CTA streams it with U loads per operand in flight per thread (thread t takes vectors t, t+B, t+2B, ...).
   {
-    const unsigned long long V = f.vpre[nseg];
-    int k0 = 0, k1 = 0;
-    for (unsigned long long v0 = gt; v0 < V; v0 += 2 * total) {
-      const unsigned long long v1 = v0 + total;
-      const bool two = v1 < V;
-      while (v0 >= f.vpre[k0 + 1]) k0++;
-      const unsigned long long i0 = v0 - f.vpre[k0];
-      const size_t h0 = (size_t)f.head[k0] * T::E;
-      const uint4* a0 = reinterpret_cast<const uint4*>(static_cast<const char*>(batch.seg[k0].inbox) + h0) + i0;
-      const uint4* b0 = reinterpret_cast<const uint4*>(static_cast<const char*>(batch.seg[k0].local) + h0) + i0;
-      uint4* o0 = reinterpret_cast<uint4*>(static_cast<char*>(batch.seg[k0].out) + h0) + i0;
-      uint4 va0 = __ldcs(a0), vb0 = __ldcs(b0);
-      if (two) {
-        if (k1 < k0) k1 = k0;
-        while (v1 >= f.vpre[k1 + 1]) k1++;
-        const unsigned long long i1 = v1 - f.vpre[k1];
-        const size_t h1 = (size_t)f.head[k1] * T::E;
-        const uint4* a1 = reinterpret_cast<const uint4*>(static_cast<const char*>(batch.seg[k1].inbox) + h1) + i1;
-        const uint4* b1 = reinterpret_cast<const uint4*>(static_cast<const char*>(batch.seg[k1].local) + h1) + i1;
-        uint4* o1 = reinterpret_cast<uint4*>(static_cast<char*>(batch.seg[k1].out) + h1) + i1;
-        uint4 va1 = __ldcs(a1), vb1 = __ldcs(b1);
-        *o0 = T::add_vec(va0, vb0);
-        *o1 = T::add_vec(va1, vb1);
+    const unsigned long long T_all = f.tpre[nseg];
+    const unsigned tile_v = U * blockDim.x;
+    int k = 0;
+    for (unsigned long long t = blockIdx.x; t < T_all; t += gridDim.x) {
+      while (t >= f.tpre[k + 1]) k++;
+      const unsigned long long first = (t - f.tpre[k]) * tile_v;          // first vector of the tile in segment k
+      const unsigned long long left = f.nvec[k] - first;
+      const unsigned n_here = left < tile_v ? (unsigned)left : tile_v;
+      const size_t h = (size_t)f.head[k] * T::E;
+      const uint4* a = reinterpret_cast<const uint4*>(static_cast<const char*>(batch.seg[k].inbox) + h) + first;
+      const uint4* b = reinterpret_cast<const uint4*>(static_cast<const char*>(batch.seg[k].local) + h) + first;
+      uint4* o = reinterpret_cast<uint4*>(static_cast<char*>(batch.seg[k].out) + h) + first;
+      uint4 va[U], vb[U];
+      if (n_here == tile_v) {
+#pragma unroll
+        for (int u = 0; u < U; u++) {
+          va[u] = __ldcs(a + threadIdx.x + u * blockDim.x);
+          vb[u] = __ldcs(b + threadIdx.x + u * blockDim.x);
+        }
+#pragma unroll
+        for (int u = 0; u < U; u++) o[threadIdx.x + u * blockDim.x] = T::add_vec(va[u], vb[u]);
       } else {
-        *o0 = T::add_vec(va0, vb0);
+#pragma unroll
+        for (int u = 0; u < U; u++) {
+          const unsigned i = threadIdx.x + u * blockDim.x;
+          if (i < n_here) {
+            va[u] = __ldcs(a + i);
+            vb[u] = __ldcs(b + i);
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < U; u++) {
+          const unsigned i = threadIdx.x + u * blockDim.x;
+          if (i < n_here) o[i] = T::add_vec(va[u], vb[u]);
+        }
       }
     }
   }
@@ -166,7 +181,8 @@ __global__ void __launch_bounds__(kThreads, 1) sum2_kernel(const __grid_constant
   }
 }
 
-__global__ void __launch_bounds__(kThreads, 1) copy_kernel(const __grid_constant__ CopyBatch batch) {
+template <int U, int THREADS>
+__global__ void __launch_bounds__(THREADS, 1) copy_kernel(const __grid_constant__ CopyBatch batch) {
   __shared__ Flat f;
   const int nseg = batch.nseg;
   if ((int)threadIdx.x < nseg) {
@@ -181,12 +197,13 @@ __global__ void __launch_bounds__(kThreads, 1) copy_kernel(const __grid_constant
   }
   __syncthreads();
   if (threadIdx.x == 0) {
-    unsigned long long v = 0, s = 0;
-    f.vpre[0] = 0;
+    unsigned long long t = 0, s = 0;
+    const unsigned long long tile_v = (unsigned long long)U * blockDim.x;
+    f.tpre[0] = 0;
     f.spre[0] = 0;
     for (int k = 0; k < nseg; k++) {
-      v += f.nvec[k];
-      f.vpre[k + 1] = v;
+      t += (f.nvec[k] + tile_v - 1) / tile_v;
+      f.tpre[k + 1] = t;
       s += f.spre[k + 1];
       f.spre[k + 1] = s;
     }
@@ -195,27 +212,33 @@ __global__ void __launch_bounds__(kThreads, 1) copy_kernel(const __grid_constant
   const unsigned long long total = (unsigned long long)gridDim.x * blockDim.x;
   const unsigned long long gt = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
   {
-    const unsigned long long V = f.vpre[nseg];
-    int k0 = 0, k1 = 0;
-    for (unsigned long long v0 = gt; v0 < V; v0 += 2 * total) {
-      const unsigned long long v1 = v0 + total;
-      const bool two = v1 < V;
-      while (v0 >= f.vpre[k0 + 1]) k0++;
-      const unsigned long long i0 = v0 - f.vpre[k0];
-      const uint4* a0 = reinterpret_cast<const uint4*>(static_cast<const char*>(batch.seg[k0].src) + f.head[k0]) + i0;
-      uint4* o0 = reinterpret_cast<uint4*>(static_cast<char*>(batch.seg[k0].dst) + f.head[k0]) + i0;
-      uint4 va0 = __ldcs(a0);
-      if (two) {
-        if (k1 < k0) k1 = k0;
-        while (v1 >= f.vpre[k1 + 1]) k1++;
-        const unsigned long long i1 = v1 - f.vpre[k1];
-        const uint4* a1 = reinterpret_cast<const uint4*>(static_cast<const char*>(batch.seg[k1].src) + f.head[k1]) + i1;
-        uint4* o1 = reinterpret_cast<uint4*>(static_cast<char*>(batch.seg[k1].dst) + f.head[k1]) + i1;
-        uint4 va1 = __ldcs(a1);
-        *o0 = va0;
-        *o1 = va1;
+    const unsigned long long T_all = f.tpre[nseg];
+    const unsigned tile_v = U * blockDim.x;
+    int k = 0;
+    for (unsigned long long t = blockIdx.x; t < T_all; t += gridDim.x) {
+      while (t >= f.tpre[k + 1]) k++;
+      const unsigned long long first = (t - f.tpre[k]) * tile_v;
+      const unsigned long long left = f.nvec[k] - first;
+      const unsigned n_here = left < tile_v ? (unsigned)left : tile_v;
+      const uint4* a = reinterpret_cast<const uint4*>(static_cast<const char*>(batch.seg[k].src) + f.head[k]) + first;
+      uint4* o = reinterpret_cast<uint4*>(static_cast<char*>(batch.seg[k].dst) + f.head[k]) + first;
+      uint4 va[U];
+      if (n_here == tile_v) {
+#pragma unroll
+        for (int u = 0; u < U; u++) va[u] = __ldcs(a + threadIdx.x + u * blockDim.x);
+#pragma unroll
+        for (int u = 0; u < U; u++) o[threadIdx.x + u * blockDim.x] = va[u];
       } else {
-        *o0 = va0;
+#pragma unroll
+        for (int u = 0; u < U; u++) {
+          const unsigned i = threadIdx.x + u * blockDim.x;
+          if (i < n_here) va[u] = __ldcs(a + i);
+        }
+#pragma unroll
+        for (int u = 0; u < U; u++) {
+          const unsigned i = threadIdx.x + u * blockDim.x;
+          if (i < n_here) o[i] = va[u];
+        }
       }
     }
   }
@@ -249,25 +272,40 @@ __global__ void __launch_bounds__(kThreads, 2) occupy_kernel(unsigned long long 
 
 }  // namespace
 
+// Launch shapes (measured on B200, 200 MiB operands): under a small CTA budget 1024 threads x 4 vectors per
+// operand in flight give 116 GB/s per SM (the mixed read/write ceiling of one SM's memory port is ~123 GB/s);
+// with the whole GPU 512 threads x 4 are a little faster (6.2 TB/s).
+static bool wide_grid(int ctas) { return ctas >= 64; }
+
 cudaError_t launch_sum(const SumBatch& batch, int ctas, cudaStream_t stream) {
   if (batch.nseg <= 0) return cudaSuccess;
-  if (batch.dtype == 0)
-    sum2_kernel<0><<<ctas, kThreads, 0, stream>>>(batch);
-  else
-    sum2_kernel<1><<<ctas, kThreads, 0, stream>>>(batch);
+  if (batch.dtype == 0) {
+    if (wide_grid(ctas)) sum2_kernel<0, 4, 512><<<ctas, 512, 0, stream>>>(batch);
+    else sum2_kernel<0, 4, 1024><<<ctas, 1024, 0, stream>>>(batch);
+  } else {
+    if (wide_grid(ctas)) sum2_kernel<1, 4, 512><<<ctas, 512, 0, stream>>>(batch);
+    else sum2_kernel<1, 4, 1024><<<ctas, 1024, 0, stream>>>(batch);
+  }
   return cudaGetLastError();
 }
 
 cudaError_t launch_copy(const CopyBatch& batch, int ctas, cudaStream_t stream) {
   if (batch.nseg <= 0) return cudaSuccess;
-  copy_kernel<<<ctas, kThreads, 0, stream>>>(batch);
+  if (wide_grid(ctas)) copy_kernel<4, 512><<<ctas, 512, 0, stream>>>(batch);
+  else copy_kernel<8, 1024><<<ctas, 1024, 0, stream>>>(batch);
   return cudaGetLastError();
 }
 
-const void* sum_kernel_entry(int dtype) {
-  return dtype == 0 ? reinterpret_cast<const void*>(&sum2_kernel<0>) : reinterpret_cast<const void*>(&sum2_kernel<1>);
+const void* sum_kernel_entry(int dtype, int ctas, int* threads) {
+  *threads = wide_grid(ctas) ? 512 : 1024;
+  if (dtype == 0)
+    return wide_grid(ctas) ? reinterpret_cast<const void*>(&sum2_kernel<0, 4, 512>) : reinterpret_cast<const void*>(&sum2_kernel<0, 4, 1024>);
+  return wide_grid(ctas) ? reinterpret_cast<const void*>(&sum2_kernel<1, 4, 512>) : reinterpret_cast<const void*>(&sum2_kernel<1, 4, 1024>);
 }
-const void* copy_kernel_entry() { return reinterpret_cast<const void*>(&copy_kernel); }
+const void* copy_kernel_entry(int ctas, int* threads) {
+  *threads = wide_grid(ctas) ? 512 : 1024;
+  return wide_grid(ctas) ? reinterpret_cast<const void*>(&copy_kernel<4, 512>) : reinterpret_cast<const void*>(&copy_kernel<8, 1024>);
+}
 
 cudaError_t launch_occupy_all_sms(unsigned long long ns, int num_sms, cudaStream_t stream, int* ctas_out) {
   int per_sm = 0;

@@ -7,7 +7,7 @@
 namespace hoccl {
 
 constexpr int kMaxSegs = 32;       // segments (one per rank) a single batched launch can carry
-constexpr int kThreads = 1024;     // threads per CTA of both streaming kernels
+constexpr int kThreads = 1024;     // threads per CTA of the copy and occupancy kernels (the sum picks 512 or 1024)
 
 // One SUM segment: out[i] = rn_T(f32(inbox[i]) + f32(local[i])), i < n (elements).
 struct SumSeg {
@@ -38,8 +38,8 @@ struct CopyBatch {
 cudaError_t launch_sum(const SumBatch& batch, int ctas, cudaStream_t stream);
 cudaError_t launch_copy(const CopyBatch& batch, int ctas, cudaStream_t stream);
 // Kernel entry addresses and parameter blocks for CUDA graph kernel nodes.
-const void* sum_kernel_entry(int dtype);
-const void* copy_kernel_entry();
+const void* sum_kernel_entry(int dtype, int ctas, int* threads);
+const void* copy_kernel_entry(int ctas, int* threads);
 
 // Fills every thread slot of every SM for `ns` nanoseconds (measured with %globaltimer per CTA).
 // It never waits on memory or on another agent, so it always ends by itself.

@@ -1,0 +1,65 @@
+"""Kernel microbenchmarks through the C ABI (hoccl_sum_launch / hoccl_copy_launch), one kernel at a time.
+
+    python -m paper_2609_34334_b200.microbench --kernel sum --dtype bf16 --mib 200 --ctas 8 --reps 5
+
+Operands are larger than L2 by default; timing uses CUDA events on the launching stream after warm-up.
+Prints one JSON line.  This is the small case used for ncu captures of a single kernel.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+
+import torch
+
+from . import binding as hb
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--kernel", default="sum", choices=["sum", "copy"])
+    ap.add_argument("--dtype", default="bf16", choices=["bf16", "fp32"])
+    ap.add_argument("--mib", type=int, default=200, help="MiB per operand")
+    ap.add_argument("--ctas", type=int, default=8)
+    ap.add_argument("--reps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    args = ap.parse_args()
+    torch.cuda.set_device(0)
+    nbytes = args.mib << 20
+    e = 2 if args.dtype == "bf16" else 4
+    n = nbytes // e
+    tdt = torch.bfloat16 if args.dtype == "bf16" else torch.float32
+    a = torch.empty(n, dtype=tdt, device="cuda").normal_(0, 1e-3)
+    b = torch.empty(n, dtype=tdt, device="cuda").normal_(0, 1e-3)
+    o = torch.empty(n, dtype=tdt, device="cuda")
+    st = torch.cuda.Stream()
+
+    def launch():
+        if args.kernel == "sum":
+            rc = hb.sum_launch(a, b, o, n, args.dtype, args.ctas, st)
+        else:
+            rc = hb.copy_launch(a, o, nbytes, args.ctas, st)
+        assert rc == hb.OK, rc
+
+    for _ in range(args.warmup):
+        launch()
+    st.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(st)
+    for _ in range(args.reps):
+        launch()
+    e1.record(st)
+    st.synchronize()
+    sec = e0.elapsed_time(e1) / 1e3 / args.reps
+    moved = (3 if args.kernel == "sum" else 2) * nbytes
+    if args.kernel == "sum":
+        assert torch.equal(o, (a.float() + b.float()).to(tdt)), "kernel result differs from torch's fp32 add + RNE"
+    else:
+        assert torch.equal(o, a)
+    print(json.dumps({"kernel": args.kernel, "dtype": args.dtype, "mib_per_operand": args.mib, "ctas": args.ctas,
+                      "us_per_launch": sec * 1e6, "algorithmic_bytes_per_launch": moved, "GBps": moved / sec / 1e9,
+                      "GBps_per_cta": moved / sec / 1e9 / args.ctas}))
+
+
+if __name__ == "__main__":
+    main()
