@@ -119,6 +119,9 @@ hoccl_result_t hoccl_comm_set_path(hoccl_comm_t comm, hoccl_path_t path);
  *  "piece_bytes" pipeline piece size in bytes (default 4 MiB, rounded to a multiple of 1024)
  *  "max_pieces"  cap on pieces per ring chunk (default 8)
  *  "lanes"       internal move streams of the stream executor, 1..8 (default 4)
+ *  "p2p_split"   a send/recv message of 32 MiB or more on the CE path is cut into up to this many slices that
+ *                run on different lanes, 1..8 (default 1 = one copy per message; measured: slices do not help
+ *                on one device because every driver copy already spreads over the whole GPU)
  *  "use_graph"   1 = run a cached CUDA graph built from the plan (default), 0 = streams and events
  *  "profile"     1 = time every SUM launch with CUDA events; read the totals with hoccl_last_stats after
  *                synchronising (with graphs only the latest replay of each cached graph is readable, so

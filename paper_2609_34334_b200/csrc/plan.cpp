@@ -96,7 +96,10 @@ bool build_plan(Plan* plan, int kind, int R, size_t count, int dtype, bool in_pl
   P.elem = e;
   P.chunk_elems = (kind == PLAN_ALLREDUCE) ? (count + (size_t)R - 1) / (size_t)R : count;
   size_t chunk_bytes = P.chunk_elems * e;
-  // piece geometry: at most max_pieces pieces of equal size (multiple of 1024 bytes)
+  // piece geometry: at most max_pieces pieces of equal size (multiple of 1024 bytes).  Pieces exist to overlap a
+  // piece's move with another piece's sum; a pure all-gather has no sums, and on one device many small copies only
+  // add per-copy cost, so it is cut no finer than 64 MiB.
+  if (kind == PLAN_ALLGATHER) piece_bytes = std::max<size_t>(piece_bytes, (size_t)64 << 20);
   size_t want = (chunk_bytes + piece_bytes - 1) / piece_bytes;
   size_t np = std::max<size_t>(1, std::min<size_t>(want, (size_t)max_pieces));
   size_t plen = round_up((chunk_bytes + np - 1) / np, 1024);

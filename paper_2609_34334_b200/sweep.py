@@ -1,0 +1,343 @@
+"""Message-size sweep of every operation on both paths (the fifth benchmark configuration) and the
+pipeline / gradient-stream workloads (third and fourth), through the C ABI.
+
+    python -m paper_2609_34334_b200.sweep sizes   [--min-log2 12 --max-log2 30 --ranks 2,4,8 --dtypes bf16 --ops all --out FILE]
+    python -m paper_2609_34334_b200.sweep pipeline [--microbatches 16]
+    python -m paper_2609_34334_b200.sweep gradients [--buckets 32]
+
+Sizes are per-rank buffer bytes S in the nccl-tests convention (all-reduce: send = recv = S; reduce-scatter:
+send = S; all-gather: recv = S; send/recv: S), like the sweeps the paper reports (Sec. 5 "Communication
+benchmarks").  Timing: CUDA events around back-to-back calls on one stream after warm-up, buffers rotated
+when the working set is smaller than L2.  Prints one JSON object per line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import sys
+
+import torch
+
+from . import binding as hb
+from . import workloads as W
+
+NOMINAL_HBM = 8.0e12
+L2_BYTES = 126 << 20
+
+
+def _hbm_bytes(op, S, R):
+    """Algorithmic HBM bytes of the rank-local ring on one device: S(R-1) wire bytes in total over all ranks per
+    phase; a MOVE reads and writes each (2 B), a SUM reads two and writes one (3 B)."""
+    return {"allreduce": 7.0 * S * (R - 1), "reduce_scatter": 5.0 * S * (R - 1), "allgather": 2.0 * S * (R - 1) + 2.0 * S,
+            "sendrecv": 2.0 * S}[op]
+
+
+def _bus_factor(op, R):
+    return {"allreduce": 2.0 * (R - 1) / R, "reduce_scatter": (R - 1) / R, "allgather": (R - 1) / R, "sendrecv": 1.0}[op]
+
+
+class Arena:
+    """Per-rank device buffers for one operation, several rotating sets when small."""
+
+    def __init__(self, op, R, S, dtype, nsets):
+        e = W.elem_size(dtype)
+        tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+        self.op, self.R, self.S, self.dtype, self.e = op, R, S, dtype, e
+        n = S // e
+        if op == "allreduce":
+            self.count, send_n, recv_n = n, n, n
+        elif op == "reduce_scatter":
+            self.count, send_n, recv_n = n // R, n, n // R
+        elif op == "allgather":
+            self.count, send_n, recv_n = n // R, n // R, n
+        else:
+            self.count, send_n, recv_n = n, n, n
+        ranks = R if op != "sendrecv" else 1
+        self.sets = []
+        for _ in range(nsets):
+            send = [torch.empty(max(send_n, 1), dtype=tdt, device="cuda").normal_(0, 1e-3) for _ in range(ranks)]
+            recv = [torch.zeros(max(recv_n, 1), dtype=tdt, device="cuda") for _ in range(ranks)]
+            self.sets.append((send, recv))
+
+    def call(self, comm, k, stream):
+        send, recv = self.sets[k % len(self.sets)]
+        if self.op == "allreduce":
+            comm.allreduce(send, recv, self.count, self.dtype, stream)
+        elif self.op == "reduce_scatter":
+            comm.reduce_scatter(send, recv, self.count, self.dtype, stream)
+        elif self.op == "allgather":
+            comm.allgather(send, recv, self.count, self.dtype, stream)
+        else:
+            comm.send(send[0], self.count, self.dtype, 0, 1, stream)
+            comm.recv(recv[0], self.count, self.dtype, 0, 1, stream)
+
+
+def time_op(comm, arena, stream, min_window_s=0.01, max_iters=200):
+    nsets = len(arena.sets)
+    for k in range(max(3, nsets)):
+        arena.call(comm, k, stream)
+    stream.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    arena.call(comm, 0, stream)
+    e1.record(stream)
+    stream.synchronize()
+    one = max(e0.elapsed_time(e1) / 1e3, 1e-6)
+    iters = int(min(max_iters, max(3, min_window_s / one)))
+    e0.record(stream)
+    for k in range(iters):
+        arena.call(comm, k, stream)
+    e1.record(stream)
+    stream.synchronize()
+    return e0.elapsed_time(e1) / 1e3 / iters
+
+
+def sweep_sizes(args):
+    torch.cuda.set_device(0)
+    stream = torch.cuda.Stream()
+    ops = ["allreduce", "reduce_scatter", "allgather", "sendrecv"] if args.ops == "all" else args.ops.split(",")
+    configs = [("CE", hb.PATH_CE, 8, 8), ("SM8", hb.PATH_SM, 8, 8), ("SMall", hb.PATH_SM, 148, 148)]
+    if args.configs != "all":
+        configs = [c for c in configs if c[0] in args.configs.split(",")]
+    out = open(args.out, "w") if args.out else None
+    for dtype in args.dtypes.split(","):
+        for R in [int(r) for r in args.ranks.split(",")]:
+            for lg in range(args.min_log2, args.max_log2 + 1):
+                S = 1 << lg
+                e = W.elem_size(dtype)
+                if S // e < R:
+                    continue
+                for op in ops:
+                    if op == "sendrecv" and R != 2:
+                        continue            # point to point does not depend on R
+                    ranks = R if op != "sendrecv" else 1
+                    footprint = 2 * ranks * S
+                    nsets = 1 if footprint > 2 * L2_BYTES else int(min(8, max(2, (3 * L2_BYTES) // max(footprint, 1))))
+                    if footprint * nsets > (48 << 30):
+                        nsets = 1
+                    arena = Arena(op, R, S, dtype, nsets)
+                    scratch = torch.empty(hb.scratch_bytes(R, S // e, dtype) + 256, dtype=torch.uint8, device="cuda")
+                    pad = (-scratch.data_ptr()) % 256
+                    for name, path, sc, cc in configs:
+                        comm = hb.Comm(R, 0)
+                        if scratch.numel() > 256:
+                            comm.set_scratch(scratch.data_ptr() + pad, scratch.numel() - 256)
+                        comm.set_path(path)
+                        comm.set_param("sum_ctas", sc)
+                        comm.set_param("copy_ctas", cc)
+                        t = time_op(comm, arena, stream)
+                        row = {"op": op, "R": R, "dtype": dtype, "S": S, "config": name, "sum_ctas": sc,
+                               "copy_ctas": cc if path == hb.PATH_SM else None, "us": t * 1e6, "algbw_GBps": S / t / 1e9,
+                               "busbw_GBps": S * _bus_factor(op, R) / t / 1e9,
+                               "hbm_frac_of_8TBps": _hbm_bytes(op, S, R) / t / NOMINAL_HBM, "buffer_sets": nsets}
+                        line = json.dumps(row)
+                        print(line, flush=True)
+                        if out:
+                            out.write(line + "\n")
+                        comm.destroy()
+                    del arena, scratch
+                    torch.cuda.empty_cache()
+    if out:
+        out.close()
+
+
+def pipeline(args):
+    """Stage-to-stage forwarding of bf16 activations [4, 2048, 4096] over 8 logical stages while a 4096^3 bf16
+    GEMM probe loops on another stream (the third benchmark configuration; forward wave only)."""
+    torch.cuda.set_device(0)
+    c = W.C3_PIPELINE
+    n, S = c.count, c.count * 2
+    M = args.microbatches
+    stream, gs = torch.cuda.Stream(), torch.cuda.Stream()
+    slots = [[torch.empty(n, dtype=torch.bfloat16, device="cuda") for _ in range(M)] for _ in range(c.stages)]
+    for m in range(M):
+        slots[0][m].normal_(0, 1)
+    A = torch.randn(4096, 4096, dtype=torch.bfloat16, device="cuda")
+    B = torch.randn(4096, 4096, dtype=torch.bfloat16, device="cuda")
+    C = torch.empty(4096, 4096, dtype=torch.bfloat16, device="cuda")
+    flops = 2.0 * 4096 ** 3
+
+    stage_streams = [torch.cuda.Stream() for _ in range(c.stages)]
+
+    def wave(comm):
+        # every stage posts on its own stream: the send of hop s -> s+1 on stage s's stream, the matching recv on
+        # stage s+1's stream; hop (m, s) follows hop (m, s-1) through the order of stage s's stream
+        for m in range(M):
+            for s in range(c.stages - 1):
+                comm.send(slots[s][m], n, "bf16", s, s + 1, stage_streams[s])
+                comm.recv(slots[s + 1][m], n, "bf16", s, s + 1, stage_streams[s + 1])
+
+    def fork():
+        ev = torch.cuda.Event()
+        ev.record(stream)
+        for st in stage_streams:
+            st.wait_event(ev)
+
+    def join():
+        for st in stage_streams:
+            ev = torch.cuda.Event()
+            ev.record(st)
+            stream.wait_event(ev)
+
+    def gemm_alone(n_gemm=200):
+        with torch.cuda.stream(gs):
+            for _ in range(10):
+                torch.matmul(A, B, out=C)
+            g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            g0.record(gs)
+            for _ in range(n_gemm):
+                torch.matmul(A, B, out=C)
+            g1.record(gs)
+        torch.cuda.synchronize()
+        return flops * n_gemm / (g0.elapsed_time(g1) / 1e3) / 1e12
+
+    alone = gemm_alone()
+    print(json.dumps({"workload": c.name, "gemm_alone_TFLOPs": alone}), flush=True)
+    for name, path, cc, split in (("CE", hb.PATH_CE, 8, 1), ("SM8", hb.PATH_SM, 8, 1),
+                                  ("SM32", hb.PATH_SM, 32, 1), ("SMall", hb.PATH_SM, 148, 1)):
+        comm = hb.Comm(c.stages, 0)
+        comm.set_path(path)
+        comm.set_param("copy_ctas", cc)
+        comm.set_param("p2p_split", split)
+        wave(comm)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        fork()
+        wave(comm)
+        join()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        t = e0.elapsed_time(e1) / 1e3
+        hops = (c.stages - 1) * M
+        # beside the GEMM probe: keep waves going while 200 GEMMs run
+        n_gemm = 200
+        waves = max(1, int(1.3 * n_gemm * flops / (alone * 1e12) / t) + 1)
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        c0.record(stream)
+        fork()
+        g0.record(gs)
+        done = 0
+        for i in range(n_gemm):
+            with torch.cuda.stream(gs):
+                torch.matmul(A, B, out=C)
+            while done < (i + 1) * waves // n_gemm:
+                wave(comm)
+                done += 1
+        g1.record(gs)
+        join()
+        c1.record(stream)
+        torch.cuda.synchronize()
+        tf = flops * n_gemm / (g0.elapsed_time(g1) / 1e3) / 1e12
+        tc = c0.elapsed_time(c1) / 1e3
+        ok = all(torch.equal(slots[c.stages - 1][m], slots[0][m]) for m in range(M))
+        print(json.dumps({"workload": c.name, "config": name, "copy_ctas": cc if path == hb.PATH_SM else None, "hops": hops,
+                          "message_MiB": S >> 20, "wave_ms": t * 1e3, "algbw_GBps": hops * S / t / 1e9,
+                          "hbm_frac_of_8TBps": 2.0 * hops * S / t / NOMINAL_HBM, "gemm_TFLOPs_beside": tf,
+                          "gemm_loss": 1 - tf / alone, "algbw_beside_GBps": done * hops * S / tc / 1e9 if done else 0.0,
+                          "delivered_bit_exact": ok}), flush=True)
+        comm.destroy()
+
+
+def gradients(args):
+    """GPT-6.7B shaped data-parallel all-reduce: 40 MiB bf16 buckets over R = 8 back to back, beside an
+    8192 x 4096 x 16384 bf16 GEMM probe (the fourth benchmark configuration).  A window of `--buckets` buckets is
+    timed (the full stream is 307 buckets + one of 8 MiB; every bucket is the same work)."""
+    torch.cuda.set_device(0)
+    g = W.C4_GRADIENTS
+    R, dtype = g.R, g.dtype
+    sizes = g.buckets()
+    per = sizes[0]
+    S = per * 2
+    nb = min(args.buckets, len(sizes))
+    stream, gs = torch.cuda.Stream(), torch.cuda.Stream()
+    pool = 3     # reusable per-rank bucket buffers
+    send = [[torch.empty(per, dtype=torch.bfloat16, device="cuda").normal_(0, 1e-3) for _ in range(R)] for _ in range(pool)]
+    recv = [[torch.empty(per, dtype=torch.bfloat16, device="cuda") for _ in range(R)] for _ in range(pool)]
+    scratch = torch.empty(hb.scratch_bytes(R, per, dtype) + 256, dtype=torch.uint8, device="cuda")
+    pad = (-scratch.data_ptr()) % 256
+    M, K, N = g.gemm_probe
+    A = torch.randn(M, K, dtype=torch.bfloat16, device="cuda")
+    B = torch.randn(K, N, dtype=torch.bfloat16, device="cuda")
+    C = torch.empty(M, N, dtype=torch.bfloat16, device="cuda")
+    flops = 2.0 * M * N * K
+
+    def gemm_tflops(n_gemm, comm=None, n_bucket=0):
+        with torch.cuda.stream(gs):
+            for _ in range(3):
+                torch.matmul(A, B, out=C)
+        torch.cuda.synchronize()
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        c0.record(stream)
+        g0.record(gs)
+        done = 0
+        for i in range(n_gemm):
+            with torch.cuda.stream(gs):
+                torch.matmul(A, B, out=C)
+            while comm is not None and done < (i + 1) * n_bucket // n_gemm:
+                comm.allreduce(send[done % pool], recv[done % pool], per, dtype, stream)
+                done += 1
+        g1.record(gs)
+        c1.record(stream)
+        torch.cuda.synchronize()
+        return flops * n_gemm / (g0.elapsed_time(g1) / 1e3) / 1e12, c0.elapsed_time(c1) / 1e3, done
+
+    alone, _, _ = gemm_tflops(40)
+    print(json.dumps({"workload": g.name, "buckets_total": len(sizes), "bucket_MiB": S >> 20, "last_bucket_MiB": sizes[-1] * 2 >> 20,
+                      "gemm_probe": [M, K, N], "gemm_alone_TFLOPs": alone}), flush=True)
+    for name, path, sc, cc in (("CE_sum8", hb.PATH_CE, 8, 8), ("SM_copy8_sum8", hb.PATH_SM, 8, 8), ("SM_copy32_sum8", hb.PATH_SM, 8, 32),
+                               ("SM_copy148_sum148", hb.PATH_SM, 148, 148)):
+        comm = hb.Comm(R, 0)
+        comm.set_scratch(scratch.data_ptr() + pad, scratch.numel() - 256)
+        comm.set_path(path)
+        comm.set_param("sum_ctas", sc)
+        comm.set_param("copy_ctas", cc)
+        for k in range(pool):
+            comm.allreduce(send[k], recv[k], per, dtype, stream)
+        stream.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for k in range(nb):
+            comm.allreduce(send[k % pool], recv[k % pool], per, dtype, stream)
+        e1.record(stream)
+        stream.synchronize()
+        t = e0.elapsed_time(e1) / 1e3 / nb
+        n_gemm = 40
+        t_g = n_gemm * flops / (alone * 1e12)
+        n_bucket = max(1, int(1.3 * t_g / t) + 1)
+        tf, tc, done = gemm_tflops(n_gemm, comm, n_bucket)
+        print(json.dumps({"workload": g.name, "config": name, "ms_per_bucket": t * 1e3, "busbw_GBps": S * 2 * (R - 1) / R / t / 1e9,
+                          "hbm_frac_of_8TBps": 7.0 * S * (R - 1) / t / NOMINAL_HBM,
+                          "full_stream_ms_estimate": t * 1e3 * (len(sizes) - 1 + sizes[-1] / per),
+                          "gemm_TFLOPs_beside": tf, "gemm_loss": 1 - tf / alone,
+                          "busbw_beside_GBps": done * S * 2 * (R - 1) / R / tc / 1e9}), flush=True)
+        comm.destroy()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    sub = ap.add_subparsers(dest="cmd", required=True)
+    s = sub.add_parser("sizes")
+    s.add_argument("--min-log2", type=int, default=12)
+    s.add_argument("--max-log2", type=int, default=30)
+    s.add_argument("--ranks", default="2,4,8")
+    s.add_argument("--dtypes", default="bf16")
+    s.add_argument("--ops", default="all")
+    s.add_argument("--configs", default="all")
+    s.add_argument("--out", default="")
+    p = sub.add_parser("pipeline")
+    p.add_argument("--microbatches", type=int, default=16)
+    g = sub.add_parser("gradients")
+    g.add_argument("--buckets", type=int, default=32)
+    args = ap.parse_args()
+    if not torch.cuda.is_available():
+        sys.stderr.write("sweep: no CUDA device\n")
+        return 2
+    {"sizes": sweep_sizes, "pipeline": pipeline, "gradients": gradients}[args.cmd](args)
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

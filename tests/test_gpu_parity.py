@@ -372,23 +372,32 @@ def test_send_recv_matching(oracle):
     assert comm.destroy() == hb.OK
 
 
-def test_pipeline_wave_small(oracle):
-    """Stage-to-stage forwarding: microbatch m travels 0 -> 1 -> ... -> S-1; hop s+1 depends on hop s."""
-    S, M, n, dtype = 8, 4, 65_536 + 8, "bf16"
-    comm = hb.Comm(S, 0)
-    acts = [W.normal(2, m, n, dtype) for m in range(M)]
-    slots = [[DevBuf(n * 2) for _ in range(M)] for _ in range(S)]
-    for m in range(M):
-        slots[0][m].put(acts[m])
-    st = torch.cuda.Stream()
-    for m in range(M):
-        for s in range(S - 1):
-            comm.send(slots[s][m], n, dtype, s, s + 1, st)
-            comm.recv(slots[s + 1][m], n, dtype, s, s + 1, st)
-    torch.cuda.synchronize()
-    for m in range(M):
-        assert (slots[S - 1][m].get(np.uint16) == acts[m]).all()
-    assert comm.destroy() == hb.OK
+@pytest.mark.parametrize("per_stage_streams", [False, True])
+@pytest.mark.parametrize("path", [hb.PATH_CE, hb.PATH_SM])
+def test_pipeline_wave_small(oracle, per_stage_streams, path):
+    """Stage-to-stage forwarding: microbatch m travels 0 -> 1 -> ... -> S-1; hop s+1 depends on hop s.
+    With one stream per stage the dependency runs through the matched posts only (send on stage s's stream,
+    recv on stage s+1's stream); a 40 MiB message also exercises the sliced copy."""
+    S, M, dtype = 8, 4, "bf16"
+    for n, split in ((65_536 + 8, 1), (20 * 1024 * 1024 + 8, 2)):
+        comm = hb.Comm(S, 0)
+        comm.set_path(path)
+        comm.set_param("p2p_split", split)
+        acts = [W.normal(2, m, n, dtype) for m in range(M)]
+        slots = [[DevBuf(n * 2) for _ in range(M)] for _ in range(S)]
+        for m in range(M):
+            slots[0][m].put(acts[m])
+        torch.cuda.synchronize()
+        streams = [torch.cuda.Stream() for _ in range(S)] if per_stage_streams else [torch.cuda.Stream()] * S
+        for m in range(M):
+            for s in range(S - 1):
+                comm.send(slots[s][m], n, dtype, s, s + 1, streams[s])
+                comm.recv(slots[s + 1][m], n, dtype, s, s + 1, streams[s + 1])
+        torch.cuda.synchronize()
+        for m in range(M):
+            assert (slots[S - 1][m].get(np.uint16) == oracle.sendrecv(acts[m])).all()
+            assert all(slots[s][m].guards_intact() for s in range(S))
+        assert comm.destroy() == hb.OK
 
 
 # ------------------------------------------------------------------------------- errors, host path -
