@@ -122,6 +122,8 @@ hoccl_result_t hoccl_comm_set_path(hoccl_comm_t comm, hoccl_path_t path);
  *  "p2p_split"   a send/recv message of 32 MiB or more on the CE path is cut into up to this many slices that
  *                run on different lanes, 1..8 (default 1 = one copy per message; measured: slices do not help
  *                on one device because every driver copy already spreads over the whole GPU)
+ *  "ce_sub_bytes" graph executor, CE path: a move between this many bytes and 16 MiB is issued as sub-copies of
+ *                this size (0 = off, the default)
  *  "use_graph"   1 = run a cached CUDA graph built from the plan (default), 0 = streams and events
  *  "profile"     1 = time every SUM launch with CUDA events; read the totals with hoccl_last_stats after
  *                synchronising (with graphs only the latest replay of each cached graph is readable, so
@@ -166,6 +168,16 @@ hoccl_result_t hoccl_reduce_scatter(const void* const* send, void* const* recv, 
  */
 hoccl_result_t hoccl_allgather(const void* const* send, void* const* recv, size_t count, hoccl_dtype_t dtype,
                                hoccl_comm_t comm, hoccl_stream_t stream);
+
+/*
+ * All-to-all (paper Sec. 5 "All-to-All", its second benchmarked collective).  send[r] and recv[r] hold R blocks
+ * of `count` elements; block j of recv[r] becomes block r of send[j].  Pure moves: the R(R-1) remote blocks
+ * travel in R-1 permutation stages (stage k: every rank r sends to rank (r+k) mod R: a contention-free matching,
+ * the degenerate case of the paper's stage decomposition, Sec. 3.4), plus one copy of the own block.
+ * No scratch.  There is no in-place form: send[r] and recv[r] must not overlap (INVALID_ARG otherwise).
+ */
+hoccl_result_t hoccl_alltoall(const void* const* send, void* const* recv, size_t count, hoccl_dtype_t dtype,
+                              hoccl_comm_t comm, hoccl_stream_t stream);
 
 /* ---------------------------------------------------------------- point to point --------------- */
 
@@ -274,14 +286,14 @@ hoccl_result_t hoccl_copy_launch(const void* src, void* dst, size_t bytes, int c
  * checked without a GPU.  Addresses in a plan are byte offsets: buffer kinds below say what they are
  * relative to.
  */
-typedef enum { HOCCL_PLAN_ALLREDUCE = 0, HOCCL_PLAN_REDUCE_SCATTER = 1, HOCCL_PLAN_ALLGATHER = 2 } hoccl_plan_kind_t;
+typedef enum { HOCCL_PLAN_ALLREDUCE = 0, HOCCL_PLAN_REDUCE_SCATTER = 1, HOCCL_PLAN_ALLGATHER = 2, HOCCL_PLAN_ALLTOALL = 3 } hoccl_plan_kind_t;
 typedef enum { HOCCL_OP_MOVE = 0, HOCCL_OP_SUM = 1 } hoccl_plan_op_kind_t;
 typedef enum { HOCCL_BUF_SEND = 0, HOCCL_BUF_RECV = 1, HOCCL_BUF_INBOX = 2, HOCCL_BUF_PARTIAL = 3 } hoccl_buf_kind_t;
 
 typedef struct {
   int kind;      /* hoccl_plan_op_kind_t */
-  int phase;     /* 0 reduce-scatter, 1 all-gather, 2 own-chunk copy of an out-of-place all-gather */
-  int step;      /* ring step s */
+  int phase;     /* 0 reduce-scatter, 1 all-gather, 2 own-chunk / own-block copy, 3 all-to-all stage */
+  int step;      /* ring step s (all-to-all: stage k, destination = rank + k) */
   int piece;     /* pipeline piece index */
   int rank;      /* MOVE: source rank; SUM: the rank that sums */
   int dst_rank;  /* MOVE: destination rank; SUM: same as rank */

@@ -51,6 +51,7 @@ def lib() -> ctypes.CDLL:
         L.oracle_ring_allreduce.argtypes = [ctypes.c_int, ctypes.c_size_t, ctypes.c_int, vpp, vpp, ctypes.c_int]
         L.oracle_ring_reduce_scatter.argtypes = [ctypes.c_int, ctypes.c_size_t, ctypes.c_int, vpp, vpp, ctypes.c_int]
         L.oracle_allgather.argtypes = [ctypes.c_int, ctypes.c_size_t, ctypes.c_int, vpp, vpp, ctypes.c_int]
+        L.oracle_alltoall.argtypes = [ctypes.c_int, ctypes.c_size_t, ctypes.c_int, vpp, vpp]
         L.oracle_sendrecv.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int]
         L.oracle_chain_sum.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_size_t, ctypes.c_size_t, ctypes.c_int, vpp,
                                        ctypes.c_void_p]
@@ -130,6 +131,17 @@ def allgather(xs, threads: int = 1):
     R = len(xs)
     ys = [np.empty(R * count, dtype=xs[0].dtype) for _ in range(R)]
     rc = lib().oracle_allgather(R, count, dt, _ptrs(xs), _ptrs(ys), max(1, threads))
+    assert rc == 0, rc
+    return ys
+
+
+def alltoall(xs):
+    """xs: R arrays of R*count elements.  Returns R arrays: block j of result r is block r of xs[j]."""
+    dt, n = _check(xs)
+    R = len(xs)
+    assert n % R == 0
+    ys = [np.empty_like(x) for x in xs]
+    rc = lib().oracle_alltoall(R, n // R, dt, _ptrs(xs), _ptrs(ys))
     assert rc == 0, rc
     return ys
 

@@ -14,6 +14,7 @@
  *       R separate arenas (inbox I_r, partial P_r), moves are memcpy, sums are scalar loops.
  *   oracle_allgather   : the definition (concatenation), written as the ring of moves.
  *   oracle_sendrecv    : the definition (identity on bytes).
+ *   oracle_alltoall    : the definition (block transpose).
  *   oracle_chain_sum   : closed form of the ring order for one chunk,
  *                        ((x_{c+1} + x_{c+2}) + ... + x_{c+R-1}) + x_c, used to pin the step-by-step code.
  *   oracle_sum_f64     : fp64 sum and fp64 sum of magnitudes (for the error bound).
@@ -219,6 +220,16 @@ int oracle_allgather(int R, size_t count, int dtype, const void* const* X, void*
   }
   ring_ag(R, dtype, Y, lo, hi, threads);
   free(lo);
+  return 0;
+}
+
+/* all-to-all (the paper's second benchmarked collective, Sec. 5): X[r], Y[r] hold R blocks of count elements;
+ * block j of Y[r] is block r of X[j].  Written as the definition, block by block. */
+int oracle_alltoall(int R, size_t count, int dtype, const void* const* X, void* const* Y) {
+  if (R < 1 || (dtype != DT_F32 && dtype != DT_BF16)) return -2;
+  size_t b = count * esize(dtype);
+  for (int r = 0; r < R; r++)
+    for (int j = 0; j < R; j++) memcpy((char*)Y[r] + (size_t)j * b, (const char*)X[j] + (size_t)r * b, b);
   return 0;
 }
 

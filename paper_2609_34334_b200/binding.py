@@ -16,7 +16,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_MISMATCH, ERR_PENDING, ERR_S
 FLOAT32, BFLOAT16 = 0, 1
 SUM = 0
 PATH_CE, PATH_SM = 0, 1
-PLAN_ALLREDUCE, PLAN_REDUCE_SCATTER, PLAN_ALLGATHER = 0, 1, 2
+PLAN_ALLREDUCE, PLAN_REDUCE_SCATTER, PLAN_ALLGATHER, PLAN_ALLTOALL = 0, 1, 2, 3
 OP_MOVE, OP_SUM = 0, 1
 BUF_SEND, BUF_RECV, BUF_INBOX, BUF_PARTIAL = 0, 1, 2, 3
 
@@ -25,7 +25,7 @@ DTYPES = {"fp32": FLOAT32, "bf16": BFLOAT16}
 EXPORTS = [
     "hoccl_comm_init", "hoccl_comm_destroy", "hoccl_scratch_bytes", "hoccl_comm_set_scratch", "hoccl_comm_set_staging",
     "hoccl_comm_set_path", "hoccl_comm_set_param", "hoccl_comm_get_param", "hoccl_allreduce", "hoccl_reduce_scatter",
-    "hoccl_allgather", "hoccl_send", "hoccl_recv", "hoccl_comm_pending", "hoccl_host_allreduce", "hoccl_error_string",
+    "hoccl_allgather", "hoccl_alltoall", "hoccl_send", "hoccl_recv", "hoccl_comm_pending", "hoccl_host_allreduce", "hoccl_error_string",
     "hoccl_last_cuda_error", "hoccl_last_stats", "hoccl_profile_reset", "hoccl_probe_move_needs_sm", "hoccl_sum_launch",
     "hoccl_copy_launch", "hoccl_plan_build", "hoccl_plan_destroy", "hoccl_plan_num_ops", "hoccl_plan_num_groups",
     "hoccl_plan_get_op", "hoccl_plan_group_deps", "hoccl_plan_slot_bytes", "hoccl_allreduce_static",
@@ -82,6 +82,7 @@ def lib() -> ctypes.CDLL:
         "hoccl_allreduce": (i, [vpp, vpp, sz, i, i, vp, vp]),
         "hoccl_reduce_scatter": (i, [vpp, vpp, sz, i, i, vp, vp]),
         "hoccl_allgather": (i, [vpp, vpp, sz, i, vp, vp]),
+        "hoccl_alltoall": (i, [vpp, vpp, sz, i, vp, vp]),
         "hoccl_send": (i, [vp, sz, i, i, i, vp, vp]),
         "hoccl_recv": (i, [vp, sz, i, i, i, vp, vp]),
         "hoccl_comm_pending": (i, [vp]),
@@ -213,6 +214,12 @@ class Comm:
 
     def allgather_rc(self, send, recv, count, dtype, stream=None) -> int:
         return lib().hoccl_allgather(_ptr_array(send), _ptr_array(recv), count, _dtype(dtype), self._h, _stream(stream))
+
+    def alltoall_rc(self, send, recv, count, dtype, stream=None) -> int:
+        return lib().hoccl_alltoall(_ptr_array(send), _ptr_array(recv), count, _dtype(dtype), self._h, _stream(stream))
+
+    def alltoall(self, send, recv, count, dtype, stream=None):
+        self._check(self.alltoall_rc(send, recv, count, dtype, stream), "hoccl_alltoall")
 
     def allreduce(self, send, recv, count, dtype, stream=None, op=SUM):
         self._check(self.allreduce_rc(send, recv, count, dtype, stream, op), "hoccl_allreduce")

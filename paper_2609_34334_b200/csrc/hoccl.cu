@@ -76,7 +76,7 @@ struct GraphEntry {
 struct hoccl_comm {
   int R = 0, device = 0, num_sms = 0;
   hoccl_path_t path = HOCCL_PATH_CE;
-  long sum_ctas = 8, copy_ctas = 8, piece_bytes = 4 << 20, max_pieces = 8, lanes = 4, use_graph = 1, profile = 0, p2p_split = 1;
+  long sum_ctas = 8, copy_ctas = 8, piece_bytes = 4 << 20, max_pieces = 8, lanes = 4, use_graph = 1, profile = 0, p2p_split = 1, ce_sub_bytes = 0;
   cudaStream_t lane[kMaxLanes] = {};
   cudaStream_t sum_stream = nullptr;
   int sum_priority = 0;
@@ -156,6 +156,7 @@ hoccl_result_t validate(hoccl_comm* c, Call* call) {
     bool in;
     if (call->kind == PLAN_ALLREDUCE) in = (s == d);
     else if (call->kind == PLAN_REDUCE_SCATTER) in = (d == s + (size_t)r * call->count * e);
+    else if (call->kind == PLAN_ALLTOALL) in = false;   // no in-place form: any overlap of send[r] and recv[r] is an error
     else in = (s == d + (size_t)r * call->count * e);
     if (in) n_in++;
     else if (ranges_overlap(s, call->send_bytes, d, call->recv_bytes)) return HOCCL_ERR_INVALID_ARG;
@@ -261,7 +262,7 @@ hoccl_result_t run_streams(hoccl_comm* c, const Plan& P, const std::vector<RGrou
       CU_TRY(c, touch(s, &u));
       sum_used = true;
     } else {
-      int l = move_rr++ % lanes;
+      int l = c->path == HOCCL_PATH_SM ? 0 : move_rr++ % lanes;   // SM copies share one lane: global CTA budget
       s = c->lane[l];
       CU_TRY(c, touch(s, &lane_used[l]));
     }
@@ -348,6 +349,7 @@ hoccl_result_t build_graph(hoccl_comm* c, const Plan& P, const std::vector<RGrou
   cudaGraph_t g = nullptr;
   CU_TRY(c, cudaGraphCreate(&g, 0));
   std::vector<cudaGraphNode_t> tail(groups.size(), nullptr);
+  cudaGraphNode_t last_copy_node = nullptr;
   hoccl_result_t rc = HOCCL_OK;
   auto fail = [&](cudaError_t e, const char* what) {
     rc = cuda_fail(c, e, what);
@@ -404,11 +406,19 @@ hoccl_result_t build_graph(hoccl_comm* c, const Plan& P, const std::vector<RGrou
       }
     } else if (c->path == HOCCL_PATH_CE) {
       for (const Seg& sg : rg.segs) {
-        cudaGraphNode_t n;
-        e = cudaGraphAddMemcpyNode1D(&n, g, deps.data(), deps.size(), sg.dst, sg.src, sg.bytes, cudaMemcpyDeviceToDevice);
+        // optional sub-copies: driver copies of 4-8 MiB pay a ~4 us serialised start-up that smaller ones do not
+        size_t sub = sg.bytes;
+        if (c->ce_sub_bytes > 0 && sg.bytes > (size_t)c->ce_sub_bytes && sg.bytes < ((size_t)16 << 20))
+          sub = ((size_t)c->ce_sub_bytes + 255) / 256 * 256;
+        for (size_t off = 0; off < sg.bytes && e == cudaSuccess; off += sub) {
+          cudaGraphNode_t n;
+          e = cudaGraphAddMemcpyNode1D(&n, g, deps.data(), deps.size(), sg.dst + off, sg.src + off, std::min(sub, sg.bytes - off),
+                                       cudaMemcpyDeviceToDevice);
+          if (e != cudaSuccess) break;
+          nodes.push_back(n);
+          entry->n_moves++;
+        }
         if (e != cudaSuccess) break;
-        nodes.push_back(n);
-        entry->n_moves++;
       }
     } else {
       for (size_t first = 0; first < rg.segs.size() && e == cudaSuccess; first += kMaxSegs) {
@@ -422,9 +432,13 @@ hoccl_result_t build_graph(hoccl_comm* c, const Plan& P, const std::vector<RGrou
         kp.gridDim = dim3((unsigned)c->copy_ctas);
         kp.blockDim = dim3((unsigned)copy_threads);
         kp.kernelParams = args;
+        // copy launches are chained as well: the CTA budget for copies is global, two never run at the same time
+        std::vector<cudaGraphNode_t> d2 = deps;
+        if (last_copy_node && std::find(d2.begin(), d2.end(), last_copy_node) == d2.end()) d2.push_back(last_copy_node);
         cudaGraphNode_t kn;
-        e = cudaGraphAddKernelNode(&kn, g, deps.data(), deps.size(), &kp);
+        e = cudaGraphAddKernelNode(&kn, g, d2.data(), d2.size(), &kp);
         if (e != cudaSuccess) break;
+        last_copy_node = kn;
         nodes.push_back(kn);
         entry->n_moves += (long)n;
         entry->n_move_launches++;
@@ -467,6 +481,7 @@ std::vector<uint64_t> make_key(hoccl_comm* c, const Call& call) {
   k.push_back((uint64_t)c->piece_bytes);
   k.push_back((uint64_t)c->max_pieces);
   k.push_back((uint64_t)c->profile);
+  k.push_back((uint64_t)c->ce_sub_bytes);
   k.push_back((uint64_t)(uintptr_t)c->scratch);
   for (int r = 0; r < c->R; r++) {
     k.push_back((uint64_t)(uintptr_t)call.send[r]);
@@ -765,7 +780,8 @@ static long* param_slot(hoccl_comm* c, const char* key, long* lo, long* hi) {
   } rows[] = {{"sum_ctas", &c->sum_ctas, 1, 1024},      {"copy_ctas", &c->copy_ctas, 1, 1024},
               {"piece_bytes", &c->piece_bytes, 1024, 1L << 40}, {"max_pieces", &c->max_pieces, 1, 4096},
               {"lanes", &c->lanes, 1, kMaxLanes},       {"use_graph", &c->use_graph, 0, 1},
-              {"profile", &c->profile, 0, 1},           {"p2p_split", &c->p2p_split, 1, kMaxLanes}};
+              {"profile", &c->profile, 0, 1},           {"p2p_split", &c->p2p_split, 1, kMaxLanes},
+              {"ce_sub_bytes", &c->ce_sub_bytes, 0, 1L << 40}};
   for (auto& r : rows)
     if (std::strcmp(r.name, key) == 0) {
       *lo = r.lo;
@@ -818,6 +834,14 @@ hoccl_result_t hoccl_allgather(const void* const* send, void* const* recv, size_
   if (!c) return HOCCL_ERR_INVALID_ARG;
   size_t e = dtype_size((int)dtype);
   Call call{PLAN_ALLGATHER, count, (int)dtype, false, count * e, (size_t)c->R * count * e, send, recv};
+  return run_collective(c, &call, (cudaStream_t)stream);
+}
+
+hoccl_result_t hoccl_alltoall(const void* const* send, void* const* recv, size_t count, hoccl_dtype_t dtype, hoccl_comm_t c,
+                              hoccl_stream_t stream) {
+  if (!c) return HOCCL_ERR_INVALID_ARG;
+  size_t e = dtype_size((int)dtype);
+  Call call{PLAN_ALLTOALL, count, (int)dtype, false, (size_t)c->R * count * e, (size_t)c->R * count * e, send, recv};
   return run_collective(c, &call, (cudaStream_t)stream);
 }
 

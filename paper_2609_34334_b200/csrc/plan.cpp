@@ -83,7 +83,8 @@ void piece_span(const Plan& P, size_t len_bytes, int p, size_t* off, size_t* len
 bool build_plan(Plan* plan, int kind, int R, size_t count, int dtype, bool in_place, size_t piece_bytes, int max_pieces,
                 const unsigned char* send_align) {
   size_t e = dtype_size(dtype);
-  if (!plan || R < 1 || e == 0 || kind < PLAN_ALLREDUCE || kind > PLAN_ALLGATHER) return false;
+  if (!plan || R < 1 || e == 0 || kind < PLAN_ALLREDUCE || kind > PLAN_ALLTOALL) return false;
+  if (kind == PLAN_ALLTOALL && in_place) return false;  // an in-place exchange would need a staging copy of every block
   if (max_pieces < 1) max_pieces = 1;
   if (piece_bytes < 1024) piece_bytes = 1024;
   Plan& P = *plan;
@@ -99,14 +100,14 @@ bool build_plan(Plan* plan, int kind, int R, size_t count, int dtype, bool in_pl
   // piece geometry: at most max_pieces pieces of equal size (multiple of 1024 bytes).  Pieces exist to overlap a
   // piece's move with another piece's sum; a pure all-gather has no sums, and on one device many small copies only
   // add per-copy cost, so it is cut no finer than 64 MiB.
-  if (kind == PLAN_ALLGATHER) piece_bytes = std::max<size_t>(piece_bytes, (size_t)64 << 20);
+  if (kind == PLAN_ALLGATHER || kind == PLAN_ALLTOALL) piece_bytes = std::max<size_t>(piece_bytes, (size_t)64 << 20);
   size_t want = (chunk_bytes + piece_bytes - 1) / piece_bytes;
   size_t np = std::max<size_t>(1, std::min<size_t>(want, (size_t)max_pieces));
   size_t plen = round_up((chunk_bytes + np - 1) / np, 1024);
   if (plen == 0) plen = 1024;
   P.piece_bytes = plen;
   P.pieces = (int)std::max<size_t>(1, (chunk_bytes + plen - 1) / plen);
-  P.slot_bytes = (kind == PLAN_ALLGATHER || R == 1) ? 0 : round_up(chunk_bytes + 16 * (size_t)P.pieces, 256);
+  P.slot_bytes = (kind == PLAN_ALLGATHER || kind == PLAN_ALLTOALL || R == 1) ? 0 : round_up(chunk_bytes + 16 * (size_t)P.pieces, 256);
   if (count == 0) return true;
   // Where piece p of chunk c sits inside a scratch slot of rank r: every piece has its own region with 16
   // bytes of slack, and inside it the data is shifted by the 16-byte phase of the operand it is summed with
@@ -131,6 +132,35 @@ bool build_plan(Plan* plan, int kind, int R, size_t count, int dtype, bool in_pl
         B.end_group();
       }
     }
+    return true;
+  }
+
+  if (kind == PLAN_ALLTOALL) {
+    // All-to-all as R-1 permutation stages (the matching-peeling view of the paper's stage decomposition, Sec. 3.4:
+    // stage k is the contention-free matching r -> r+k of the uniform traffic matrix) plus the own block.  All flows
+    // have the same size, so chunk service is plain round-robin over ranks.  No dependencies: blocks are disjoint.
+    for (int p = 0; p < np_i; p++) {
+      B.begin_group(OP_MOVE, PHASE_OWN, 0, p);
+      for (int r = 0; r < R; r++) {
+        size_t off, len;
+        piece_span(P, chunk_bytes, p, &off, &len);
+        uint64_t blk = (uint64_t)r * count * e + off;
+        B.add(PlanOp{OP_MOVE, PHASE_OWN, 0, p, r, r, r, BUF_SEND, BUF_RECV, -1, blk, blk, 0, len, 0});
+      }
+      B.end_group();
+    }
+    for (int k = 1; k < R; k++)
+      for (int p = 0; p < np_i; p++) {
+        B.begin_group(OP_MOVE, PHASE_A2A, k, p);
+        for (int r = 0; r < R; r++) {
+          int d = (r + k) % R;
+          size_t off, len;
+          piece_span(P, chunk_bytes, p, &off, &len);
+          B.add(PlanOp{OP_MOVE, PHASE_A2A, k, p, r, d, d, BUF_SEND, BUF_RECV, -1, (uint64_t)d * count * e + off,
+                       (uint64_t)r * count * e + off, 0, len, 0});
+        }
+        B.end_group();
+      }
     return true;
   }
 

@@ -15,10 +15,10 @@
 
 namespace hoccl {
 
-enum PlanKind { PLAN_ALLREDUCE = 0, PLAN_REDUCE_SCATTER = 1, PLAN_ALLGATHER = 2 };
+enum PlanKind { PLAN_ALLREDUCE = 0, PLAN_REDUCE_SCATTER = 1, PLAN_ALLGATHER = 2, PLAN_ALLTOALL = 3 };
 enum OpKind { OP_MOVE = 0, OP_SUM = 1 };
 enum BufKind { BUF_SEND = 0, BUF_RECV = 1, BUF_INBOX = 2, BUF_PARTIAL = 3 };
-enum Phase { PHASE_RS = 0, PHASE_AG = 1, PHASE_OWN = 2 };
+enum Phase { PHASE_RS = 0, PHASE_AG = 1, PHASE_OWN = 2, PHASE_A2A = 3 };
 
 struct PlanOp {
   int kind;

@@ -6,7 +6,7 @@ pipeline / gradient-stream workloads (third and fourth), through the C ABI.
     python -m paper_2609_34334_b200.sweep gradients [--buckets 32]
 
 Sizes are per-rank buffer bytes S in the nccl-tests convention (all-reduce: send = recv = S; reduce-scatter:
-send = S; all-gather: recv = S; send/recv: S), like the sweeps the paper reports (Sec. 5 "Communication
+send = S; all-gather: recv = S; all-to-all: send = recv = S; send/recv: S), like the sweeps the paper reports (Sec. 5 "Communication
 benchmarks").  Timing: CUDA events around back-to-back calls on one stream after warm-up, buffers rotated
 when the working set is smaller than L2.  Prints one JSON object per line.
 """
@@ -29,11 +29,12 @@ def _hbm_bytes(op, S, R):
     """Algorithmic HBM bytes of the rank-local ring on one device: S(R-1) wire bytes in total over all ranks per
     phase; a MOVE reads and writes each (2 B), a SUM reads two and writes one (3 B)."""
     return {"allreduce": 7.0 * S * (R - 1), "reduce_scatter": 5.0 * S * (R - 1), "allgather": 2.0 * S * (R - 1) + 2.0 * S,
-            "sendrecv": 2.0 * S}[op]
+            "alltoall": 2.0 * S * R, "sendrecv": 2.0 * S}[op]
 
 
 def _bus_factor(op, R):
-    return {"allreduce": 2.0 * (R - 1) / R, "reduce_scatter": (R - 1) / R, "allgather": (R - 1) / R, "sendrecv": 1.0}[op]
+    return {"allreduce": 2.0 * (R - 1) / R, "reduce_scatter": (R - 1) / R, "allgather": (R - 1) / R, "alltoall": (R - 1) / R,
+            "sendrecv": 1.0}[op]
 
 
 class Arena:
@@ -50,6 +51,8 @@ class Arena:
             self.count, send_n, recv_n = n // R, n, n // R
         elif op == "allgather":
             self.count, send_n, recv_n = n // R, n // R, n
+        elif op == "alltoall":
+            self.count, send_n, recv_n = n // R, n, n
         else:
             self.count, send_n, recv_n = n, n, n
         ranks = R if op != "sendrecv" else 1
@@ -67,6 +70,8 @@ class Arena:
             comm.reduce_scatter(send, recv, self.count, self.dtype, stream)
         elif self.op == "allgather":
             comm.allgather(send, recv, self.count, self.dtype, stream)
+        elif self.op == "alltoall":
+            comm.alltoall(send, recv, self.count, self.dtype, stream)
         else:
             comm.send(send[0], self.count, self.dtype, 0, 1, stream)
             comm.recv(recv[0], self.count, self.dtype, 0, 1, stream)
@@ -95,7 +100,7 @@ def time_op(comm, arena, stream, min_window_s=0.01, max_iters=200):
 def sweep_sizes(args):
     torch.cuda.set_device(0)
     stream = torch.cuda.Stream()
-    ops = ["allreduce", "reduce_scatter", "allgather", "sendrecv"] if args.ops == "all" else args.ops.split(",")
+    ops = ["allreduce", "reduce_scatter", "allgather", "alltoall", "sendrecv"] if args.ops == "all" else args.ops.split(",")
     configs = [("CE", hb.PATH_CE, 8, 8), ("SM8", hb.PATH_SM, 8, 8), ("SMall", hb.PATH_SM, 148, 148)]
     if args.configs != "all":
         configs = [c for c in configs if c[0] in args.configs.split(",")]

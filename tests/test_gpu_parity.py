@@ -237,6 +237,29 @@ def test_reduce_scatter_and_allgather(oracle, dtype, path):
         comm.destroy()
 
 
+@pytest.mark.parametrize("path", [hb.PATH_CE, hb.PATH_SM])
+@pytest.mark.parametrize("use_graph", [0, 1])
+def test_alltoall(oracle, path, use_graph):
+    for dtype in ("fp32", "bf16"):
+        e = W.elem_size(dtype)
+        for R, count in [(1, 7), (2, 1), (4, 4099), (8, 100_003), (5, 33)]:
+            xs = W.rank_inputs("uniform", 83, R, R * count, dtype)
+            want = oracle.alltoall(xs)
+            comm = hb.Comm(R, 0)
+            comm.set_path(path)
+            comm.set_param("use_graph", use_graph)
+            send = [DevBuf(R * count * e, (r % 3) * e).put(xs[r]) for r in range(R)]
+            recv = [DevBuf(R * count * e) for _ in range(R)]
+            comm.alltoall(send, recv, count, dtype)
+            torch.cuda.synchronize()
+            for r in range(R):
+                assert (recv[r].get(np_dtype(dtype)).view(np.uint8) == want[r].view(np.uint8)).all(), (R, count, r)
+                assert recv[r].guards_intact() and send[r].guards_intact()
+                assert (send[r].get(np_dtype(dtype)).view(np.uint8) == xs[r].view(np.uint8)).all()
+            assert comm.alltoall_rc(send, send, count, dtype) == hb.ERR_INVALID_ARG       # no in-place form
+            assert comm.destroy() == hb.OK
+
+
 def test_settings_never_change_a_bit(oracle):
     """Piece size, lane count, CTA budgets, path and executor are pure scheduling choices."""
     R, n, dtype = 8, 8 * 40000 + 8, "bf16"

@@ -294,3 +294,18 @@ def test_stored_oracle_results_unchanged(oracle):
     rs = oracle.ring_reduce_scatter(xs, threads=oracle.max_threads())
     ag = oracle.allgather(rs)
     assert (ag[3] == ys[3]).all()
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("R", [1, 2, 3, 8])
+def test_alltoall_is_block_transpose(oracle, dtype, R):
+    for count in [1, 5, 1000]:
+        xs = W.rank_inputs("uniform", 71, R, R * count, dtype)
+        ys = oracle.alltoall(xs)
+        cube = np.stack(xs).reshape(R, R, count)              # [source rank, block, element]
+        want = cube.transpose(1, 0, 2)                         # [destination rank, source rank, element]
+        for r in range(R):
+            assert (ys[r].reshape(R, count) == want[r]).all()
+        back = oracle.alltoall(ys)                             # an all-to-all is its own inverse
+        for r in range(R):
+            assert (back[r] == xs[r]).all()

@@ -42,12 +42,14 @@ def _run_plan(plan, kind, R, count, dtype, xs, in_place, rng):
     npdt = np.float32 if dtype == "fp32" else np.uint16
     if kind == hb.PLAN_ALLREDUCE:
         send_n, recv_n = count, count
+    elif kind == hb.PLAN_ALLTOALL:
+        send_n, recv_n = R * count, R * count
     elif kind == hb.PLAN_REDUCE_SCATTER:
         send_n, recv_n = R * count, count
     else:
         send_n, recv_n = count, R * count
     slot = plan.slot_bytes
-    if R > 1 and count > 0 and kind != hb.PLAN_ALLGATHER:
+    if R > 1 and count > 0 and kind in (hb.PLAN_ALLREDUCE, hb.PLAN_REDUCE_SCATTER):
         assert 0 < slot <= hb.scratch_bytes(R, send_n, dtype) // (2 * R)      # the advertised bound covers any piece setting
     send = [x.copy().view(np.uint8) for x in xs]
     if in_place:
@@ -209,3 +211,27 @@ def test_piece_geometry():
     assert {op["piece"] for op in one.ops} == {0}
     capped = hb.Plan(hb.PLAN_ALLREDUCE, 2, 1 << 28, "fp32", False, 1 << 20, 8)
     assert len({op["piece"] for op in capped.ops}) == 8
+
+
+@pytest.mark.parametrize("R", [1, 2, 5, 8])
+@pytest.mark.parametrize("count", [1, 33, 4099])
+def test_alltoall_plan(oracle, R, count):
+    rng = random.Random(R * 31 + count)
+    for dtype in ("fp32", "bf16"):
+        xs = W.rank_inputs("uniform", 37, R, R * count, dtype)
+        want = oracle.alltoall(xs)
+        plan = hb.Plan(hb.PLAN_ALLTOALL, R, count, dtype, False, 1024, 8)
+        assert all(op["kind"] == hb.OP_MOVE for op in plan.ops) and all(len(d) == 0 for d in plan.deps)
+        # every stage is a permutation: each rank sends one block and receives one block
+        stages = {}
+        for op in plan.ops:
+            stages.setdefault((op["phase"], op["step"], op["piece"]), []).append(op)
+        for (phase, k, _), ops in stages.items():
+            assert sorted(o["rank"] for o in ops) == list(range(R)) and sorted(o["dst_rank"] for o in ops) == list(range(R))
+            for o in ops:
+                assert o["dst_rank"] == (o["rank"] + (k if phase == 3 else 0)) % R
+        got = _run_plan(plan, hb.PLAN_ALLTOALL, R, count, dtype, xs, False, rng)
+        for r in range(R):
+            assert (got[r] == want[r]).all()
+    with pytest.raises(hb.HocclError):
+        hb.Plan(hb.PLAN_ALLTOALL, R, count, "fp32", True, 1024, 8)      # no in-place form
