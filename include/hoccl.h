@@ -53,7 +53,8 @@ typedef enum {
   HOCCL_ERR_MISMATCH = 4,    /* send/recv matched with different count or dtype; the parked post is dropped */
   HOCCL_ERR_PENDING = 5,     /* destroy with unmatched send/recv posts */
   HOCCL_ERR_SCRATCH = 6,     /* scratch or staging memory missing or too small */
-  HOCCL_ERR_INTERNAL = 7
+  HOCCL_ERR_INTERNAL = 7,
+  HOCCL_ERR_TIMEOUT = 8      /* handshake mode: the watchdog released a stream (asynchronous, see hoccl_comm_async_error) */
 } hoccl_result_t;
 
 typedef enum { HOCCL_FLOAT32 = 0, HOCCL_BFLOAT16 = 1 } hoccl_dtype_t;
@@ -125,6 +126,23 @@ hoccl_result_t hoccl_comm_set_path(hoccl_comm_t comm, hoccl_path_t path);
  *  "ce_sub_bytes" graph executor, CE path: a move between this many bytes and 16 MiB is issued as sub-copies of
  *                this size (0 = off, the default)
  *  "use_graph"   1 = run a cached CUDA graph built from the plan (default), 0 = streams and events
+ *  "handshake"   1 = the paper's stream manager (Sec. 3.2, Listing 1): instead of launching into the caller's
+ *                stream, the call enqueues four stream memory operations (write start flag, wait for the CPU's
+ *                acknowledgement, wait for the finish flag, reset it) and hands the schedule to a CPU proxy thread
+ *                that polls the flags in pinned host memory, runs the schedule on an internal stream and hands the
+ *                stream back.  send/recv posts are matched by the proxy AFTER each stream has reached its post, so a
+ *                post may wait for a partner that is posted later (the paper's semantics, Sec. 3.3.2); count/dtype
+ *                mismatches and unmatched posts are then reported asynchronously (hoccl_comm_async_error).
+ *                0 = off (default).  Results are identical bit for bit.  Handshake mode needs HOCCL_PATH_SM: calls on
+ *                the CE path return HOCCL_ERR_UNSUPPORTED, because on one device a driver copy issued by the proxy
+ *                can queue up behind copies that the parked stream itself has waiting and then never start.
+ *                The two sides of a send/recv must be
+ *                posted on different streams (a stream parked in its own post cannot reach the partner's).  The
+ *                first use creates the proxy: a thread, pinned host memory for 64 flag pairs and 512 bytes of
+ *                device memory (the only device allocation of the library), and loads every kernel, because
+ *                first-use work in the driver must not happen while a stream is parked.
+ *  "watchdog_ms" handshake mode: after this long (default 10000) an unmatched post is released with an abort
+ *                value and HOCCL_ERR_TIMEOUT is recorded, so no stream can wait on this library forever
  *  "profile"     1 = time every SUM launch with CUDA events; read the totals with hoccl_last_stats after
  *                synchronising (with graphs only the latest replay of each cached graph is readable, so
  *                read after every step)
@@ -198,6 +216,10 @@ hoccl_result_t hoccl_send(const void* buf, size_t count, hoccl_dtype_t dtype, in
 hoccl_result_t hoccl_recv(void* buf, size_t count, hoccl_dtype_t dtype, int src, int dst, hoccl_comm_t comm,
                           hoccl_stream_t stream);
 int hoccl_comm_pending(hoccl_comm_t comm);
+/* Handshake mode: first asynchronous failure seen by the proxy (OK, TIMEOUT, MISMATCH or CUDA); clear != 0 resets it. */
+hoccl_result_t hoccl_comm_async_error(hoccl_comm_t comm, int clear);
+/* Handshake mode: number of stream hand-overs the proxy has served so far. */
+long hoccl_comm_handshakes(hoccl_comm_t comm);
 
 /* ---------------------------------------------------------------- host-buffer entry points ----- */
 

@@ -12,7 +12,7 @@ from typing import Optional, Sequence
 
 from . import build as _build
 
-OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_MISMATCH, ERR_PENDING, ERR_SCRATCH, ERR_INTERNAL = range(8)
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_MISMATCH, ERR_PENDING, ERR_SCRATCH, ERR_INTERNAL, ERR_TIMEOUT = range(9)
 FLOAT32, BFLOAT16 = 0, 1
 SUM = 0
 PATH_CE, PATH_SM = 0, 1
@@ -25,7 +25,7 @@ DTYPES = {"fp32": FLOAT32, "bf16": BFLOAT16}
 EXPORTS = [
     "hoccl_comm_init", "hoccl_comm_destroy", "hoccl_scratch_bytes", "hoccl_comm_set_scratch", "hoccl_comm_set_staging",
     "hoccl_comm_set_path", "hoccl_comm_set_param", "hoccl_comm_get_param", "hoccl_allreduce", "hoccl_reduce_scatter",
-    "hoccl_allgather", "hoccl_alltoall", "hoccl_send", "hoccl_recv", "hoccl_comm_pending", "hoccl_host_allreduce", "hoccl_error_string",
+    "hoccl_allgather", "hoccl_alltoall", "hoccl_send", "hoccl_recv", "hoccl_comm_pending", "hoccl_comm_async_error", "hoccl_comm_handshakes", "hoccl_host_allreduce", "hoccl_error_string",
     "hoccl_last_cuda_error", "hoccl_last_stats", "hoccl_profile_reset", "hoccl_probe_move_needs_sm", "hoccl_sum_launch",
     "hoccl_copy_launch", "hoccl_plan_build", "hoccl_plan_destroy", "hoccl_plan_num_ops", "hoccl_plan_num_groups",
     "hoccl_plan_get_op", "hoccl_plan_group_deps", "hoccl_plan_slot_bytes", "hoccl_allreduce_static",
@@ -86,6 +86,8 @@ def lib() -> ctypes.CDLL:
         "hoccl_send": (i, [vp, sz, i, i, i, vp, vp]),
         "hoccl_recv": (i, [vp, sz, i, i, i, vp, vp]),
         "hoccl_comm_pending": (i, [vp]),
+        "hoccl_comm_async_error": (i, [vp, i]),
+        "hoccl_comm_handshakes": (l, [vp]),
         "hoccl_host_allreduce": (i, [vpp, vpp, sz, i, i, vp, vp]),
         "hoccl_allreduce_static": (i, [vpp, vpp, sz, i, i, i, vp]),
         "hoccl_error_string": (ctypes.c_char_p, [i]),
@@ -249,6 +251,12 @@ class Comm:
 
     def pending(self) -> int:
         return lib().hoccl_comm_pending(self._h)
+
+    def async_error(self, clear: bool = False) -> int:
+        return lib().hoccl_comm_async_error(self._h, int(clear))
+
+    def handshakes(self) -> int:
+        return int(lib().hoccl_comm_handshakes(self._h))
 
     # -- diagnostics
     def last_stats(self) -> dict:

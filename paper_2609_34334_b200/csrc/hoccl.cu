@@ -26,6 +26,7 @@
 #include "../../include/hoccl.h"
 #include "kernels.cuh"
 #include "plan.h"
+#include "proxy.h"
 
 using namespace hoccl;
 
@@ -76,7 +77,9 @@ struct GraphEntry {
 struct hoccl_comm {
   int R = 0, device = 0, num_sms = 0;
   hoccl_path_t path = HOCCL_PATH_CE;
-  long sum_ctas = 8, copy_ctas = 8, piece_bytes = 4 << 20, max_pieces = 8, lanes = 4, use_graph = 1, profile = 0, p2p_split = 1, ce_sub_bytes = 0;
+  long sum_ctas = 8, copy_ctas = 8, piece_bytes = 4 << 20, max_pieces = 8, lanes = 4, use_graph = 1, profile = 0, p2p_split = 1, ce_sub_bytes = 0,
+       handshake = 0, watchdog_ms = 10000;
+  Proxy* proxy = nullptr;
   cudaStream_t lane[kMaxLanes] = {};
   cudaStream_t sum_stream = nullptr;
   int sum_priority = 0;
@@ -517,6 +520,22 @@ void harvest_profile(hoccl_comm* c) {
   }
 }
 
+// The CPU proxy of the handshake mode is created on first use.
+hoccl_result_t ensure_proxy(hoccl_comm* c) {
+  if (c->proxy) {
+    c->proxy->set_watchdog_ms(c->watchdog_ms);
+    return HOCCL_OK;
+  }
+  Proxy* p = new Proxy(c->device, c->watchdog_ms);
+  cudaError_t e = p->init();
+  if (e != cudaSuccess) {
+    delete p;
+    return cuda_fail(c, e, "proxy init (stream memory operations)");
+  }
+  c->proxy = p;
+  return HOCCL_OK;
+}
+
 hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
   const double t0 = now_us();
   if (!c) return HOCCL_ERR_INVALID_ARG;
@@ -544,7 +563,14 @@ hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
   c->stats.n_pieces = P.pieces;
   c->stats.max_sum_ctas = 0;
   Tally tally;
-  if (c->use_graph) {
+  if (c->handshake) {
+    // Driver copies share a hardware queue with the copies the parked stream has queued behind its hand-over; a copy
+    // issued by the proxy can end up behind them and never start (observed).  Kernels do not have that problem.
+    if (c->path == HOCCL_PATH_CE) return HOCCL_ERR_UNSUPPORTED;
+    rc = ensure_proxy(c);
+    if (rc != HOCCL_OK) return rc;
+  }
+  if (c->use_graph || c->handshake) {
     std::vector<uint64_t> key = make_key(c, *call);
     GraphEntry* hit = nullptr;
     for (auto& e : c->cache)
@@ -561,7 +587,10 @@ hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
       entry.n_pieces = P.pieces;
       rc = build_graph(c, P, groups, &entry);
       if (rc != HOCCL_OK) return rc;
+      // handshake mode: place the graph on the device now; the proxy must not meet first-launch work later
+      if (c->handshake) CU_TRY(c, cudaGraphUpload(entry.exec, c->proxy->work_stream()));
       if (c->cache.size() >= kGraphCacheCap) {
+        if (c->proxy) c->proxy->drain(c->watchdog_ms);  // a queued hand-over may still refer to the victim
         size_t victim = 0;
         for (size_t i = 1; i < c->cache.size(); i++)
           if (c->cache[i].last_use < c->cache[victim].last_use) victim = i;
@@ -572,7 +601,15 @@ hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
       hit = &c->cache.back();
     }
     hit->last_use = ++c->use_counter;
-    CU_TRY(c, cudaGraphLaunch(hit->exec, user));
+    if (c->handshake) {
+      // paper Sec. 3.2: the stream hands itself to the CPU proxy, which runs the schedule and hands it back
+      ProxyTask t;
+      t.kind = ProxyTask::GRAPH;
+      t.exec = hit->exec;
+      CU_TRY(c, c->proxy->submit(user, t));
+    } else {
+      CU_TRY(c, cudaGraphLaunch(hit->exec, user));
+    }
     hit->prof_pending = !hit->prof_events.empty();
     tally.moves = hit->n_moves;
     tally.move_launches = hit->n_move_launches;
@@ -599,6 +636,29 @@ hoccl_result_t p2p_post(hoccl_comm* c, bool is_send, void* buf, size_t count, in
   if (e == 0) return HOCCL_ERR_UNSUPPORTED;
   if (src < 0 || src >= c->R || dst < 0 || dst >= c->R || src == dst) return HOCCL_ERR_INVALID_ARG;
   if ((uintptr_t)buf % e) return HOCCL_ERR_INVALID_ARG;
+  if (c->handshake) {
+    // the post is handed to the proxy at once; matching happens there, after the stream has reached the post
+    if (c->path == HOCCL_PATH_CE) return HOCCL_ERR_UNSUPPORTED;   // see run_collective
+    hoccl_result_t rc = ensure_proxy(c);
+    if (rc != HOCCL_OK) return rc;
+    ProxyTask t;
+    t.kind = ProxyTask::P2P;
+    t.is_send = is_send;
+    t.src = src;
+    t.dst = dst;
+    t.buf = buf;
+    t.count = count;
+    t.elem = e;
+    t.dtype = dtype;
+    t.path = (int)c->path;
+    t.copy_ctas = (int)c->copy_ctas;
+    CU_TRY(c, cudaSetDevice(c->device));
+    CU_TRY(c, c->proxy->submit(stream, t));
+    c->stats = hoccl_stats_t{};
+    c->stats.n_moves = 1;
+    c->stats.host_launch_us = now_us() - t0;
+    return HOCCL_OK;
+  }
   auto key = std::make_pair(src, dst);
   std::deque<Post>& q = c->pending[key];
   if (q.empty() || q.front().is_send == is_send) {
@@ -722,6 +782,12 @@ hoccl_result_t hoccl_comm_init(hoccl_comm_t* comm, int R, int device) {
 hoccl_result_t hoccl_comm_destroy(hoccl_comm_t c) {
   if (!c) return HOCCL_ERR_INVALID_ARG;
   if (c->n_pending > 0) return HOCCL_ERR_PENDING;
+  if (c->proxy) {
+    c->proxy->drain(c->watchdog_ms);
+    if (c->proxy->pending_p2p() > 0) return HOCCL_ERR_PENDING;
+    delete c->proxy;
+    c->proxy = nullptr;
+  }
   cudaSetDevice(c->device);
   for (int i = 0; i < kMaxLanes; i++)
     if (c->lane[i]) {
@@ -781,7 +847,8 @@ static long* param_slot(hoccl_comm* c, const char* key, long* lo, long* hi) {
               {"piece_bytes", &c->piece_bytes, 1024, 1L << 40}, {"max_pieces", &c->max_pieces, 1, 4096},
               {"lanes", &c->lanes, 1, kMaxLanes},       {"use_graph", &c->use_graph, 0, 1},
               {"profile", &c->profile, 0, 1},           {"p2p_split", &c->p2p_split, 1, kMaxLanes},
-              {"ce_sub_bytes", &c->ce_sub_bytes, 0, 1L << 40}};
+              {"ce_sub_bytes", &c->ce_sub_bytes, 0, 1L << 40}, {"handshake", &c->handshake, 0, 1},
+              {"watchdog_ms", &c->watchdog_ms, 10, 600000}};
   for (auto& r : rows)
     if (std::strcmp(r.name, key) == 0) {
       *lo = r.lo;
@@ -853,7 +920,25 @@ hoccl_result_t hoccl_recv(void* buf, size_t count, hoccl_dtype_t dtype, int src,
   return p2p_post(c, false, buf, count, (int)dtype, src, dst, (cudaStream_t)stream);
 }
 
-int hoccl_comm_pending(hoccl_comm_t c) { return c ? c->n_pending : 0; }
+int hoccl_comm_pending(hoccl_comm_t c) {
+  if (!c) return 0;
+  return c->n_pending + (c->proxy ? c->proxy->pending_p2p() : 0);
+}
+
+hoccl_result_t hoccl_comm_async_error(hoccl_comm_t c, int clear) {
+  if (!c) return HOCCL_ERR_INVALID_ARG;
+  if (!c->proxy) return HOCCL_OK;
+  int e = c->proxy->async_error();
+  if (clear) c->proxy->clear_error();
+  switch (e) {
+    case PROXY_OK: return HOCCL_OK;
+    case PROXY_TIMEOUT: return HOCCL_ERR_TIMEOUT;
+    case PROXY_MISMATCH: return HOCCL_ERR_MISMATCH;
+    default: return HOCCL_ERR_CUDA;
+  }
+}
+
+long hoccl_comm_handshakes(hoccl_comm_t c) { return (c && c->proxy) ? c->proxy->handshakes() : 0; }
 
 hoccl_result_t hoccl_host_allreduce(const void* const* h_send, void* const* h_recv, size_t count, hoccl_dtype_t dtype, hoccl_op_t op,
                                     hoccl_comm_t c, hoccl_stream_t stream) {
@@ -892,6 +977,7 @@ const char* hoccl_error_string(hoccl_result_t code) {
     case HOCCL_ERR_PENDING: return "unmatched send/recv posts pending";
     case HOCCL_ERR_SCRATCH: return "scratch or staging memory missing or too small";
     case HOCCL_ERR_INTERNAL: return "internal error";
+    case HOCCL_ERR_TIMEOUT: return "watchdog timeout in the stream hand-over (the stream was released)";
   }
   return "unknown error code";
 }

@@ -307,6 +307,21 @@ const void* copy_kernel_entry(int ctas, int* threads) {
   return wide_grid(ctas) ? reinterpret_cast<const void*>(&copy_kernel<4, 512>) : reinterpret_cast<const void*>(&copy_kernel<8, 1024>);
 }
 
+// Forces the module that holds these kernels to be loaded now.  Loading a kernel on first launch can synchronise the
+// device; that must never happen while a stream is parked in a hand-over that only the launching thread can finish.
+cudaError_t preload_kernels() {
+  const void* fns[] = {reinterpret_cast<const void*>(&sum2_kernel<0, 4, 512>),  reinterpret_cast<const void*>(&sum2_kernel<0, 4, 1024>),
+                       reinterpret_cast<const void*>(&sum2_kernel<1, 4, 512>),  reinterpret_cast<const void*>(&sum2_kernel<1, 4, 1024>),
+                       reinterpret_cast<const void*>(&copy_kernel<4, 512>),     reinterpret_cast<const void*>(&copy_kernel<8, 1024>),
+                       reinterpret_cast<const void*>(&occupy_kernel)};
+  for (const void* f : fns) {
+    cudaFuncAttributes a;
+    cudaError_t e = cudaFuncGetAttributes(&a, f);
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
+}
+
 cudaError_t launch_occupy_all_sms(unsigned long long ns, int num_sms, cudaStream_t stream, int* ctas_out) {
   int per_sm = 0;
   cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, occupy_kernel, kThreads, 0);

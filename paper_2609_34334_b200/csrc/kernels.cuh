@@ -41,6 +41,9 @@ cudaError_t launch_copy(const CopyBatch& batch, int ctas, cudaStream_t stream);
 const void* sum_kernel_entry(int dtype, int ctas, int* threads);
 const void* copy_kernel_entry(int ctas, int* threads);
 
+// Loads every kernel of the library on the current device (no launch).
+cudaError_t preload_kernels();
+
 // Fills every thread slot of every SM for `ns` nanoseconds (measured with %globaltimer per CTA).
 // It never waits on memory or on another agent, so it always ends by itself.
 cudaError_t launch_occupy_all_sms(unsigned long long ns, int num_sms, cudaStream_t stream, int* ctas_out);

@@ -27,7 +27,7 @@ def test_every_declared_symbol_is_exported():
 
 def test_error_strings_and_sizes():
     assert hb.error_string(hb.OK) == "ok"
-    for code in range(1, 8):
+    for code in range(1, 9):
         assert hb.error_string(code) and hb.error_string(code) != "ok"
     assert hb.scratch_bytes(1, 1000, "fp32") == 0
     assert hb.scratch_bytes(8, 0, "bf16") == 0
