@@ -197,6 +197,21 @@ hoccl_result_t hoccl_allgather(const void* const* send, void* const* recv, size_
 hoccl_result_t hoccl_alltoall(const void* const* send, void* const* recv, size_t count, hoccl_dtype_t dtype,
                               hoccl_comm_t comm, hoccl_stream_t stream);
 
+/*
+ * User-defined pattern (paper Sec. 3.4: "arbitrary user-defined collective communication patterns" go through the
+ * traffic matrix).  MPI-style all-to-allv over the R logical ranks: rank u sends sendcounts[u*R+v] elements, taken
+ * from send[u] + sdispls[u*R+v], to rank v, which stores them at recv[v] + rdispls[v*R+u] (counts and
+ * displacements are HOST arrays of R*R entries, in elements).  u == v is a local copy.
+ * The flows form the origin traffic matrix C; the collective scheduler (hoccl_sched_*) cuts it into stages by
+ * peeling matchings (Algorithm 1 with an empty RDMA domain: T = C) and, inside a stage, serves every source rank's
+ * flows from one serial queue in a size-weighted chunk interleaving (chunk = the "piece_bytes" parameter, at least
+ * 64 KiB).  Stages run one after the other.  Issued with streams and events (not cached).  No scratch.
+ * Errors: INVALID_ARG (NULL, misaligned, overlapping receive regions, a send region overlapping a receive region),
+ * UNSUPPORTED (dtype; handshake mode).
+ */
+hoccl_result_t hoccl_alltoallv(const void* const* send, const size_t* sendcounts, const size_t* sdispls, void* const* recv,
+                               const size_t* rdispls, hoccl_dtype_t dtype, hoccl_comm_t comm, hoccl_stream_t stream);
+
 /* ---------------------------------------------------------------- point to point --------------- */
 
 /*
@@ -342,6 +357,45 @@ int hoccl_plan_num_groups(hoccl_plan_t plan);
 hoccl_result_t hoccl_plan_get_op(hoccl_plan_t plan, int index, hoccl_plan_op_t* out);
 /* Dependencies are between groups: writes up to `cap` predecessor group ids of `group` into deps, returns their number. */
 int hoccl_plan_group_deps(hoccl_plan_t plan, int group, int* deps, int cap);
+
+/* ---------------------------------------------------------------- collective scheduler (host only) --- */
+
+/*
+ * The paper's collective scheduler (Sec. 3.4) for a modelled topology: G GPUs in nodes of gpus_per_node (one NVLink
+ * domain per node, the RDMA domain between nodes, symmetric peer of GPU u = u ^ 1 inside its node).
+ *   C (G x G bytes, row = source)  ->  T = C plus forwarding copies on the (u, u-bar) edges (Eq. 2-4)
+ *   ->  stages T^1..T^n by the Birkhoff-like decomposition (Algorithm 1): sum of stages = T (Eq. 5-6), at most one
+ *       RDMA flow out of and into every GPU per stage (Eq. 7), stage time tau = max over domains of largest entry /
+ *       bandwidth (Eq. 8-9), total = sum of tau (Eq. 10)
+ *   ->  per stage and per DMA engine (the source GPU of a copy) a size-weighted interleaving of fixed-size chunks.
+ * Pure host code: nothing here touches a device.  bw_* in bytes per second (<= 0 selects 400e9 / 50e9).
+ */
+typedef struct hoccl_sched* hoccl_sched_t;
+typedef enum { HOCCL_FLOW_NATIVE = 0, HOCCL_FLOW_RDMA = 1, HOCCL_FLOW_FWD_SEND = 2, HOCCL_FLOW_FWD_RECV = 3 } hoccl_flow_class_t;
+typedef struct {
+  int src, dst;                /* the edge this entry uses */
+  int cls;                     /* hoccl_flow_class_t */
+  int origin_src, origin_dst;  /* the logical flow of C it belongs to */
+  uint64_t bytes;
+  uint64_t origin_offset;      /* where these bytes start inside the logical flow */
+} hoccl_sched_flow_t;
+
+hoccl_result_t hoccl_sched_build(hoccl_sched_t* sched, int G, int gpus_per_node, double bw_nvlink, double bw_rdma,
+                                 const uint64_t* C, uint64_t chunk_bytes);
+void hoccl_sched_destroy(hoccl_sched_t sched);
+int hoccl_sched_num_stages(hoccl_sched_t sched);
+double hoccl_sched_stage_tau(hoccl_sched_t sched, int stage);
+double hoccl_sched_total_tau(hoccl_sched_t sched);
+/* max over RDMA endpoints of their traffic / bw_rdma and over NVLink edges of T / bw_nvlink: no staging can be faster */
+double hoccl_sched_lower_bound(hoccl_sched_t sched);
+/* which = -2: C, -1: T, s >= 0: the matrix of stage s.  out: G*G entries. */
+hoccl_result_t hoccl_sched_matrix(hoccl_sched_t sched, int which, uint64_t* out);
+int hoccl_sched_num_flows(hoccl_sched_t sched, int stage);
+hoccl_result_t hoccl_sched_get_flow(hoccl_sched_t sched, int stage, int index, hoccl_sched_flow_t* out);
+/* the serial chunk queue of one DMA engine in one stage: entry = (flow index in that stage, offset, bytes) */
+int hoccl_sched_queue_len(hoccl_sched_t sched, int stage, int gpu);
+hoccl_result_t hoccl_sched_queue_get(hoccl_sched_t sched, int stage, int gpu, int index, int* flow, uint64_t* offset,
+                                     uint64_t* bytes);
 
 #ifdef __cplusplus
 }

@@ -52,6 +52,8 @@ def lib() -> ctypes.CDLL:
         L.oracle_ring_reduce_scatter.argtypes = [ctypes.c_int, ctypes.c_size_t, ctypes.c_int, vpp, vpp, ctypes.c_int]
         L.oracle_allgather.argtypes = [ctypes.c_int, ctypes.c_size_t, ctypes.c_int, vpp, vpp, ctypes.c_int]
         L.oracle_alltoall.argtypes = [ctypes.c_int, ctypes.c_size_t, ctypes.c_int, vpp, vpp]
+        szp = ctypes.POINTER(ctypes.c_size_t)
+        L.oracle_alltoallv.argtypes = [ctypes.c_int, ctypes.c_int, vpp, szp, szp, vpp, szp]
         L.oracle_sendrecv.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int]
         L.oracle_chain_sum.argtypes = [ctypes.c_int, ctypes.c_int, ctypes.c_size_t, ctypes.c_size_t, ctypes.c_int, vpp,
                                        ctypes.c_void_p]
@@ -142,6 +144,18 @@ def alltoall(xs):
     assert n % R == 0
     ys = [np.empty_like(x) for x in xs]
     rc = lib().oracle_alltoall(R, n // R, dt, _ptrs(xs), _ptrs(ys))
+    assert rc == 0, rc
+    return ys
+
+
+def alltoallv(xs, sendcounts, sdispls, rdispls, recv_sizes, fill=0):
+    """xs: R send arrays; counts/displacements: R*R sequences in elements.  Returns R receive arrays of recv_sizes[v]
+    elements, pre-filled with `fill` where nothing is received."""
+    R = len(xs)
+    dt = dtype_code(xs[0])
+    ys = [np.full(int(recv_sizes[v]), fill, dtype=xs[0].dtype) for v in range(R)]
+    arr = lambda v: (ctypes.c_size_t * (R * R))(*[int(t) for t in v])
+    rc = lib().oracle_alltoallv(R, dt, _ptrs(xs), arr(sendcounts), arr(sdispls), _ptrs(ys), arr(rdispls))
     assert rc == 0, rc
     return ys
 

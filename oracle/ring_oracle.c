@@ -233,6 +233,19 @@ int oracle_alltoall(int R, size_t count, int dtype, const void* const* X, void* 
   return 0;
 }
 
+/* user-defined pattern (all-to-allv; the paper routes arbitrary patterns through its traffic matrix, Sec. 3.4):
+ * rank u sends sendcounts[u*R+v] elements from X[u] + sdispls[u*R+v] to rank v at Y[v] + rdispls[v*R+u].  The definition. */
+int oracle_alltoallv(int R, int dtype, const void* const* X, const size_t* sendcounts, const size_t* sdispls, void* const* Y,
+                     const size_t* rdispls) {
+  if (R < 1 || (dtype != DT_F32 && dtype != DT_BF16)) return -2;
+  size_t e = esize(dtype);
+  for (int u = 0; u < R; u++)
+    for (int v = 0; v < R; v++)
+      memcpy((char*)Y[v] + rdispls[(size_t)v * R + u] * e, (const char*)X[u] + sdispls[(size_t)u * R + v] * e,
+             sendcounts[(size_t)u * R + v] * e);
+  return 0;
+}
+
 /* point-to-point: the receiver's buffer becomes a byte copy of the sender's. */
 int oracle_sendrecv(const void* src, void* dst, size_t count, int dtype) {
   memmove(dst, src, count * esize(dtype));

@@ -25,10 +25,13 @@ DTYPES = {"fp32": FLOAT32, "bf16": BFLOAT16}
 EXPORTS = [
     "hoccl_comm_init", "hoccl_comm_destroy", "hoccl_scratch_bytes", "hoccl_comm_set_scratch", "hoccl_comm_set_staging",
     "hoccl_comm_set_path", "hoccl_comm_set_param", "hoccl_comm_get_param", "hoccl_allreduce", "hoccl_reduce_scatter",
-    "hoccl_allgather", "hoccl_alltoall", "hoccl_send", "hoccl_recv", "hoccl_comm_pending", "hoccl_comm_async_error", "hoccl_comm_handshakes", "hoccl_host_allreduce", "hoccl_error_string",
+    "hoccl_allgather", "hoccl_alltoall", "hoccl_alltoallv", "hoccl_send", "hoccl_recv", "hoccl_comm_pending", "hoccl_comm_async_error", "hoccl_comm_handshakes", "hoccl_host_allreduce", "hoccl_error_string",
     "hoccl_last_cuda_error", "hoccl_last_stats", "hoccl_profile_reset", "hoccl_probe_move_needs_sm", "hoccl_sum_launch",
     "hoccl_copy_launch", "hoccl_plan_build", "hoccl_plan_destroy", "hoccl_plan_num_ops", "hoccl_plan_num_groups",
     "hoccl_plan_get_op", "hoccl_plan_group_deps", "hoccl_plan_slot_bytes", "hoccl_allreduce_static",
+    "hoccl_sched_build", "hoccl_sched_destroy", "hoccl_sched_num_stages", "hoccl_sched_stage_tau", "hoccl_sched_total_tau",
+    "hoccl_sched_lower_bound", "hoccl_sched_matrix", "hoccl_sched_num_flows", "hoccl_sched_get_flow", "hoccl_sched_queue_len",
+    "hoccl_sched_queue_get",
 ]
 
 
@@ -51,6 +54,14 @@ class PlanOp(ctypes.Structure):
         ("dst_buf", ctypes.c_int), ("local_buf", ctypes.c_int), ("src_off", ctypes.c_uint64), ("dst_off", ctypes.c_uint64),
         ("local_off", ctypes.c_uint64), ("bytes", ctypes.c_uint64), ("group", ctypes.c_int),
     ]
+
+
+class SchedFlow(ctypes.Structure):
+    _fields_ = [("src", ctypes.c_int), ("dst", ctypes.c_int), ("cls", ctypes.c_int), ("origin_src", ctypes.c_int),
+                ("origin_dst", ctypes.c_int), ("bytes", ctypes.c_uint64), ("origin_offset", ctypes.c_uint64)]
+
+
+FLOW_NATIVE, FLOW_RDMA, FLOW_FWD_SEND, FLOW_FWD_RECV = 0, 1, 2, 3
 
 
 class HocclError(RuntimeError):
@@ -83,6 +94,18 @@ def lib() -> ctypes.CDLL:
         "hoccl_reduce_scatter": (i, [vpp, vpp, sz, i, i, vp, vp]),
         "hoccl_allgather": (i, [vpp, vpp, sz, i, vp, vp]),
         "hoccl_alltoall": (i, [vpp, vpp, sz, i, vp, vp]),
+        "hoccl_alltoallv": (i, [vpp, ctypes.POINTER(sz), ctypes.POINTER(sz), vpp, ctypes.POINTER(sz), i, vp, vp]),
+        "hoccl_sched_build": (i, [vpp, i, i, ctypes.c_double, ctypes.c_double, ctypes.POINTER(ctypes.c_uint64), ctypes.c_uint64]),
+        "hoccl_sched_destroy": (None, [vp]),
+        "hoccl_sched_num_stages": (i, [vp]),
+        "hoccl_sched_stage_tau": (ctypes.c_double, [vp, i]),
+        "hoccl_sched_total_tau": (ctypes.c_double, [vp]),
+        "hoccl_sched_lower_bound": (ctypes.c_double, [vp]),
+        "hoccl_sched_matrix": (i, [vp, i, ctypes.POINTER(ctypes.c_uint64)]),
+        "hoccl_sched_num_flows": (i, [vp, i]),
+        "hoccl_sched_get_flow": (i, [vp, i, i, ctypes.POINTER(SchedFlow)]),
+        "hoccl_sched_queue_len": (i, [vp, i, i]),
+        "hoccl_sched_queue_get": (i, [vp, i, i, i, ctypes.POINTER(i), ctypes.POINTER(ctypes.c_uint64), ctypes.POINTER(ctypes.c_uint64)]),
         "hoccl_send": (i, [vp, sz, i, i, i, vp, vp]),
         "hoccl_recv": (i, [vp, sz, i, i, i, vp, vp]),
         "hoccl_comm_pending": (i, [vp]),
@@ -223,6 +246,15 @@ class Comm:
     def alltoall(self, send, recv, count, dtype, stream=None):
         self._check(self.alltoall_rc(send, recv, count, dtype, stream), "hoccl_alltoall")
 
+    def alltoallv_rc(self, send, sendcounts, sdispls, recv, rdispls, dtype, stream=None) -> int:
+        R = self.R
+        arr = lambda xs: (ctypes.c_size_t * (R * R))(*[int(x) for x in xs])
+        return lib().hoccl_alltoallv(_ptr_array(send), arr(sendcounts), arr(sdispls), _ptr_array(recv), arr(rdispls), _dtype(dtype),
+                                     self._h, _stream(stream))
+
+    def alltoallv(self, send, sendcounts, sdispls, recv, rdispls, dtype, stream=None):
+        self._check(self.alltoallv_rc(send, sendcounts, sdispls, recv, rdispls, dtype, stream), "hoccl_alltoallv")
+
     def allreduce(self, send, recv, count, dtype, stream=None, op=SUM):
         self._check(self.allreduce_rc(send, recv, count, dtype, stream, op), "hoccl_allreduce")
 
@@ -321,3 +353,47 @@ class Plan:
             self.deps.append([buf[k] for k in range(n)])
         L.hoccl_plan_destroy(self._h)
         self._h = None
+
+
+class Schedule:
+    """Host-only view of the collective scheduler's output for a traffic matrix C (G x G bytes, row = source)."""
+
+    def __init__(self, C, gpus_per_node, bw_nvlink=400e9, bw_rdma=50e9, chunk_bytes=1 << 20):
+        import numpy as np
+
+        C = np.ascontiguousarray(C, dtype=np.uint64)
+        G = C.shape[0]
+        assert C.shape == (G, G)
+        L = lib()
+        h = ctypes.c_void_p()
+        rc = L.hoccl_sched_build(ctypes.byref(h), G, gpus_per_node, bw_nvlink, bw_rdma, C.ctypes.data_as(ctypes.POINTER(ctypes.c_uint64)),
+                                 chunk_bytes)
+        if rc != OK:
+            raise HocclError(rc, "hoccl_sched_build")
+        self.G = G
+
+        def mat(which):
+            out = np.zeros((G, G), dtype=np.uint64)
+            assert L.hoccl_sched_matrix(h, which, out.ctypes.data_as(ctypes.POINTER(ctypes.c_uint64))) == OK
+            return out
+
+        self.C, self.T = mat(-2), mat(-1)
+        self.total_tau = L.hoccl_sched_total_tau(h)
+        self.lower_bound = L.hoccl_sched_lower_bound(h)
+        self.stages = []
+        for s in range(L.hoccl_sched_num_stages(h)):
+            flows = []
+            for k in range(L.hoccl_sched_num_flows(h, s)):
+                f = SchedFlow()
+                assert L.hoccl_sched_get_flow(h, s, k, ctypes.byref(f)) == OK
+                flows.append({name: getattr(f, name) for name, _ in SchedFlow._fields_})
+            queues = []
+            for g in range(G):
+                q = []
+                for k in range(L.hoccl_sched_queue_len(h, s, g)):
+                    fl, off, nb = ctypes.c_int(), ctypes.c_uint64(), ctypes.c_uint64()
+                    assert L.hoccl_sched_queue_get(h, s, g, k, ctypes.byref(fl), ctypes.byref(off), ctypes.byref(nb)) == OK
+                    q.append((fl.value, off.value, nb.value))
+                queues.append(q)
+            self.stages.append({"matrix": mat(s), "tau": L.hoccl_sched_stage_tau(h, s), "flows": flows, "queues": queues})
+        L.hoccl_sched_destroy(h)

@@ -27,6 +27,7 @@
 #include "kernels.cuh"
 #include "plan.h"
 #include "proxy.h"
+#include "sched.h"
 
 using namespace hoccl;
 
@@ -964,6 +965,189 @@ hoccl_result_t hoccl_host_allreduce(const void* const* h_send, void* const* h_re
   hoccl_result_t rc = hoccl_allreduce(dsend, drecv, count, dtype, op, c, stream);
   if (rc != HOCCL_OK) return rc;
   for (int r = 0; r < R; r++) CU_TRY(c, cudaMemcpyAsync(h_recv[r], drecv[r], count * e, cudaMemcpyDeviceToHost, st));
+  return HOCCL_OK;
+}
+
+hoccl_result_t hoccl_alltoallv(const void* const* send, const size_t* sendcounts, const size_t* sdispls, void* const* recv,
+                               const size_t* rdispls, hoccl_dtype_t dtype, hoccl_comm_t c, hoccl_stream_t stream) {
+  const double t0 = now_us();
+  if (!c || !send || !recv || !sendcounts || !sdispls || !rdispls) return HOCCL_ERR_INVALID_ARG;
+  const size_t e = dtype_size((int)dtype);
+  if (e == 0) return HOCCL_ERR_UNSUPPORTED;
+  if (c->handshake) return HOCCL_ERR_UNSUPPORTED;
+  const int R = c->R;
+  for (int r = 0; r < R; r++) {
+    if (!send[r] || !recv[r]) return HOCCL_ERR_INVALID_ARG;
+    if (((uintptr_t)send[r] % e) || ((uintptr_t)recv[r] % e)) return HOCCL_ERR_INVALID_ARG;
+  }
+  // the flows of the user-defined pattern as the origin traffic matrix C (bytes); one NVLink domain, no RDMA
+  Topology topo;
+  topo.G = R;
+  topo.gpus_per_node = R;
+  std::vector<uint64_t> C((size_t)R * R);
+  uint64_t total = 0;
+  for (int u = 0; u < R; u++)
+    for (int v = 0; v < R; v++) {
+      C[(size_t)u * R + v] = (uint64_t)sendcounts[(size_t)u * R + v] * e;
+      total += C[(size_t)u * R + v];
+    }
+  // receive regions of one rank must not overlap each other, and no send region may overlap a receive region
+  for (int v = 0; v < R; v++)
+    for (int a = 0; a < R; a++) {
+      const char* ra = (const char*)recv[v] + rdispls[(size_t)v * R + a] * e;
+      const size_t la = C[(size_t)a * R + v];
+      for (int b = a + 1; b < R; b++)
+        if (ranges_overlap(ra, la, (const char*)recv[v] + rdispls[(size_t)v * R + b] * e, C[(size_t)b * R + v])) return HOCCL_ERR_INVALID_ARG;
+      for (int u = 0; u < R; u++)
+        for (int w = 0; w < R; w++)
+          if (ranges_overlap(ra, la, (const char*)send[u] + sdispls[(size_t)u * R + w] * e, C[(size_t)u * R + w])) return HOCCL_ERR_INVALID_ARG;
+    }
+  c->stats = hoccl_stats_t{};
+  if (total == 0) return HOCCL_OK;
+  Schedule S;
+  if (!build_schedule(topo, C, (uint64_t)std::max<long>(c->piece_bytes, 65536), &S)) return HOCCL_ERR_INTERNAL;
+  CU_TRY(c, cudaSetDevice(c->device));
+  cudaStream_t user = (cudaStream_t)stream;
+  const int lanes = c->path == HOCCL_PATH_SM ? 1 : (int)std::max<long>(1, std::min<long>(c->lanes, kMaxLanes));
+  c->ev_next = 0;
+  cudaEvent_t fork = next_event(c);
+  if (!fork) return cuda_fail(c, cudaErrorMemoryAllocation, "event pool");
+  CU_TRY(c, cudaEventRecord(fork, user));
+  for (int l = 0; l < lanes; l++) CU_TRY(c, cudaStreamWaitEvent(c->lane[l], fork, 0));
+  long moves = 0, launches = 0;
+  for (size_t si = 0; si < S.stages.size(); si++) {
+    const Stage& st = S.stages[si];
+    // every DMA queue (one per source rank) is a serial chain on its lane, in the interleaved chunk order
+    for (int g = 0; g < R; g++) {
+      cudaStream_t lane = c->lane[g % lanes];
+      for (const ChunkItem& it : st.queues[g]) {
+        const StageFlow& f = st.flows[it.flow];
+        const size_t so = sdispls[(size_t)f.origin_src * R + f.origin_dst] * e + f.origin_offset + it.offset;
+        const size_t dofs = rdispls[(size_t)f.origin_dst * R + f.origin_src] * e + f.origin_offset + it.offset;
+        const char* src = (const char*)send[f.origin_src] + so;
+        char* dst = (char*)recv[f.origin_dst] + dofs;
+        if (c->path == HOCCL_PATH_CE) {
+          CU_TRY(c, cudaMemcpyAsync(dst, src, it.bytes, cudaMemcpyDeviceToDevice, lane));
+        } else {
+          CopyBatch b;
+          b.nseg = 1;
+          b.pad = 0;
+          b.seg[0] = CopySeg{src, dst, (unsigned long long)it.bytes};
+          CU_TRY(c, launch_copy(b, (int)c->copy_ctas, lane));
+          launches++;
+        }
+        moves++;
+      }
+    }
+    // stages run one after the other (the paper's serial stages): barrier over the lanes
+    if (si + 1 < S.stages.size() && lanes > 1) {
+      std::vector<cudaEvent_t> evs(lanes);
+      for (int l = 0; l < lanes; l++) {
+        evs[l] = next_event(c);
+        if (!evs[l]) return cuda_fail(c, cudaErrorMemoryAllocation, "event pool");
+        CU_TRY(c, cudaEventRecord(evs[l], c->lane[l]));
+      }
+      for (int l = 0; l < lanes; l++)
+        for (int m = 0; m < lanes; m++)
+          if (m != l) CU_TRY(c, cudaStreamWaitEvent(c->lane[l], evs[m], 0));
+    }
+  }
+  for (int l = 0; l < lanes; l++) {
+    cudaEvent_t ev = next_event(c);
+    if (!ev) return cuda_fail(c, cudaErrorMemoryAllocation, "event pool");
+    CU_TRY(c, cudaEventRecord(ev, c->lane[l]));
+    CU_TRY(c, cudaStreamWaitEvent(user, ev, 0));
+  }
+  c->stats.n_moves = moves;
+  c->stats.n_move_launches = launches;
+  c->stats.max_copy_ctas = launches ? c->copy_ctas : 0;
+  c->stats.n_pieces = (long)S.stages.size();
+  c->stats.host_launch_us = now_us() - t0;
+  return HOCCL_OK;
+}
+
+// ---------------------------------------------------------------- scheduler inspection (host only) ----
+struct hoccl_sched {
+  Schedule s;
+};
+
+hoccl_result_t hoccl_sched_build(hoccl_sched_t* out, int G, int gpus_per_node, double bw_nvlink, double bw_rdma, const uint64_t* C,
+                                 uint64_t chunk_bytes) {
+  if (!out) return HOCCL_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!C || G < 1 || G > 256 || gpus_per_node < 1 || chunk_bytes == 0) return HOCCL_ERR_INVALID_ARG;
+  Topology t;
+  t.G = G;
+  t.gpus_per_node = gpus_per_node;
+  if (bw_nvlink > 0) t.bw_nvlink = bw_nvlink;
+  if (bw_rdma > 0) t.bw_rdma = bw_rdma;
+  hoccl_sched* h = new hoccl_sched();
+  std::vector<uint64_t> Cv(C, C + (size_t)G * G);
+  if (!build_schedule(t, Cv, chunk_bytes, &h->s)) {
+    delete h;
+    return HOCCL_ERR_INVALID_ARG;
+  }
+  *out = h;
+  return HOCCL_OK;
+}
+
+void hoccl_sched_destroy(hoccl_sched_t s) { delete s; }
+int hoccl_sched_num_stages(hoccl_sched_t s) { return s ? (int)s->s.stages.size() : 0; }
+double hoccl_sched_stage_tau(hoccl_sched_t s, int stage) {
+  return (s && stage >= 0 && stage < (int)s->s.stages.size()) ? s->s.stages[stage].tau : -1.0;
+}
+double hoccl_sched_total_tau(hoccl_sched_t s) { return s ? s->s.total_tau : -1.0; }
+double hoccl_sched_lower_bound(hoccl_sched_t s) { return s ? s->s.lower_bound : -1.0; }
+
+hoccl_result_t hoccl_sched_matrix(hoccl_sched_t s, int which, uint64_t* out) {
+  if (!s || !out) return HOCCL_ERR_INVALID_ARG;
+  const int G = s->s.topo.G;
+  const size_t n = (size_t)G * G;
+  if (which == -1) {
+    std::copy(s->s.T.begin(), s->s.T.end(), out);
+  } else if (which == -2) {
+    std::copy(s->s.C.begin(), s->s.C.end(), out);
+  } else if (which >= 0 && which < (int)s->s.stages.size()) {
+    std::fill(out, out + n, 0);
+    for (const StageFlow& f : s->s.stages[which].flows) out[(size_t)f.u * G + f.v] += f.bytes;
+  } else {
+    return HOCCL_ERR_INVALID_ARG;
+  }
+  return HOCCL_OK;
+}
+
+int hoccl_sched_num_flows(hoccl_sched_t s, int stage) {
+  return (s && stage >= 0 && stage < (int)s->s.stages.size()) ? (int)s->s.stages[stage].flows.size() : -1;
+}
+
+hoccl_result_t hoccl_sched_get_flow(hoccl_sched_t s, int stage, int index, hoccl_sched_flow_t* out) {
+  if (!s || !out || stage < 0 || stage >= (int)s->s.stages.size()) return HOCCL_ERR_INVALID_ARG;
+  const Stage& st = s->s.stages[stage];
+  if (index < 0 || index >= (int)st.flows.size()) return HOCCL_ERR_INVALID_ARG;
+  const StageFlow& f = st.flows[index];
+  out->src = f.u;
+  out->dst = f.v;
+  out->cls = f.cls;
+  out->origin_src = f.origin_src;
+  out->origin_dst = f.origin_dst;
+  out->bytes = f.bytes;
+  out->origin_offset = f.origin_offset;
+  return HOCCL_OK;
+}
+
+int hoccl_sched_queue_len(hoccl_sched_t s, int stage, int gpu) {
+  if (!s || stage < 0 || stage >= (int)s->s.stages.size() || gpu < 0 || gpu >= s->s.topo.G) return -1;
+  return (int)s->s.stages[stage].queues[gpu].size();
+}
+
+hoccl_result_t hoccl_sched_queue_get(hoccl_sched_t s, int stage, int gpu, int index, int* flow, uint64_t* offset, uint64_t* bytes) {
+  if (!s || !flow || !offset || !bytes || stage < 0 || stage >= (int)s->s.stages.size() || gpu < 0 || gpu >= s->s.topo.G)
+    return HOCCL_ERR_INVALID_ARG;
+  const auto& q = s->s.stages[stage].queues[gpu];
+  if (index < 0 || index >= (int)q.size()) return HOCCL_ERR_INVALID_ARG;
+  *flow = q[index].flow;
+  *offset = q[index].offset;
+  *bytes = q[index].bytes;
   return HOCCL_OK;
 }
 

@@ -260,6 +260,35 @@ def test_alltoall(oracle, path, use_graph):
             assert comm.destroy() == hb.OK
 
 
+@pytest.mark.parametrize("path", [hb.PATH_CE, hb.PATH_SM])
+def test_alltoallv_user_defined_pattern(oracle, path):
+    from test_oracle_pins import _random_pattern
+    for dtype in ("fp32", "bf16"):
+        e = W.elem_size(dtype)
+        for R, max_count, piece in [(2, 100, 65536), (4, 200_000, 65536), (8, 60_000, 131072), (5, 3, 65536)]:
+            rng = np.random.default_rng(R * 7 + max_count)
+            counts, sd, rd, send_sizes, recv_sizes = _random_pattern(R, rng, max_count)
+            xs = [W.uniform(56, u, send_sizes[u], dtype) for u in range(R)]
+            fill = np.frombuffer(bytes([0xA5]) * e, dtype=np_dtype(dtype))[0]
+            want = oracle.alltoallv(xs, counts.ravel(), sd.ravel(), rd.ravel(), recv_sizes, fill=fill)
+            comm = hb.Comm(R, 0)
+            comm.set_path(path)
+            comm.set_param("piece_bytes", piece)
+            send = [DevBuf(send_sizes[u] * e).put(xs[u]) for u in range(R)]
+            recv = [DevBuf(recv_sizes[v] * e) for v in range(R)]           # DevBuf pre-fills with 0xA5 bytes
+            comm.alltoallv(send, counts.ravel(), sd.ravel(), recv, rd.ravel(), dtype)
+            torch.cuda.synchronize()
+            for v in range(R):
+                assert (recv[v].get(np_dtype(dtype)).view(np.uint8) == want[v].view(np.uint8)).all(), (R, v)
+                assert recv[v].guards_intact() and send[v].guards_intact()
+            # overlapping receive regions are refused
+            bad = rd.copy()
+            if R >= 2 and counts[0, 1] > 0 and counts[1, 1] > 0:
+                bad[1, 0] = bad[1, 1]
+                assert comm.alltoallv_rc(send, counts.ravel(), sd.ravel(), recv, bad.ravel(), dtype) == hb.ERR_INVALID_ARG
+            assert comm.destroy() == hb.OK
+
+
 def test_settings_never_change_a_bit(oracle):
     """Piece size, lane count, CTA budgets, path and executor are pure scheduling choices."""
     R, n, dtype = 8, 8 * 40000 + 8, "bf16"

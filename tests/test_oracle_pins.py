@@ -309,3 +309,39 @@ def test_alltoall_is_block_transpose(oracle, dtype, R):
         back = oracle.alltoall(ys)                             # an all-to-all is its own inverse
         for r in range(R):
             assert (back[r] == xs[r]).all()
+
+
+def _random_pattern(R, rng, max_count=500):
+    """Counts and displacements of a random user-defined pattern (elements), with gaps between regions."""
+    counts = rng.integers(0, max_count, size=(R, R))
+    counts[rng.random((R, R)) < 0.25] = 0
+    sd = np.zeros((R, R), dtype=np.int64)
+    rd = np.zeros((R, R), dtype=np.int64)
+    send_sizes, recv_sizes = [], []
+    for u in range(R):
+        pos = 3
+        for v in rng.permutation(R):
+            sd[u, v] = pos
+            pos += counts[u, v] + int(rng.integers(0, 5))
+        send_sizes.append(pos + 2)
+    for v in range(R):
+        pos = 1
+        for u in rng.permutation(R):
+            rd[v, u] = pos
+            pos += counts[u, v] + int(rng.integers(0, 5))
+        recv_sizes.append(pos + 4)
+    return counts, sd, rd, send_sizes, recv_sizes
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("R", [1, 2, 5, 8])
+def test_alltoallv_is_the_definition(oracle, dtype, R):
+    rng = np.random.default_rng(R + 100)
+    counts, sd, rd, send_sizes, recv_sizes = _random_pattern(R, rng)
+    xs = [W.uniform(55, u, send_sizes[u], dtype) for u in range(R)]
+    ys = oracle.alltoallv(xs, counts.ravel(), sd.ravel(), rd.ravel(), recv_sizes, fill=7)
+    for v in range(R):
+        want = np.full(recv_sizes[v], 7, dtype=xs[0].dtype)
+        for u in range(R):
+            want[rd[v, u]:rd[v, u] + counts[u, v]] = xs[u][sd[u, v]:sd[u, v] + counts[u, v]]
+        assert (ys[v] == want).all()
