@@ -421,6 +421,25 @@ def extras(hb, W, torch, np, new_comm, step, timed, stream, R, S, n, dtype, peak
 
     t, _ = timed(cm, k, w, fn=one_call)
     out["single_call_allreduce"] = {"ms_per_step": t * 1e3, "busbw_GBps": S * bus_factor(R) / t / 1e9}
+    # comparison point: the whole reduction in one kernel (same bits, not rank local), by CTA budget
+    op_rows = []
+    for ctas in (8, 32, 148):
+        c1 = new_comm(hb.PATH_CE, sum_ctas=ctas, onepass=1)
+        t, _ = timed(c1, k, w, fn=one_call)
+        op_rows.append({"ctas": ctas, "ms_per_step": t * 1e3, "busbw_GBps": S * bus_factor(R) / t / 1e9,
+                        "bytes_per_step": 2.0 * R * S, "GBps": 2.0 * R * S / t / 1e9})
+        c1.destroy()
+    out["onepass_allreduce"] = op_rows
+    # handshake mode (CPU proxy + stream memory operations) on the SM path, against the same path launched directly
+    hs = {}
+    for label, flag in (("direct", 0), ("handshake", 1)):
+        c1 = new_comm(hb.PATH_SM, sum_ctas=8, copy_ctas=32, handshake=flag)
+        t, _ = timed(c1, k, w)
+        hs[label] = {"ms_per_step": t * 1e3, "busbw_GBps": S * bus_factor(R) / t / 1e9}
+        if flag:
+            hs["handshakes_served"] = c1.handshakes()
+        c1.destroy()
+    out["handshake_mode_SM_copy32_sum8"] = hs
     # stream executor (events) instead of graph replay
     cm.set_param("use_graph", 0)
     t, _ = timed(cm, k, w)
@@ -512,9 +531,10 @@ def extras(hb, W, torch, np, new_comm, step, timed, stream, R, S, n, dtype, peak
     probe = {}
     alone, _ = gemm_tflops(None)
     probe["alone_TFLOPs"] = alone
-    for name, path, sc, cc in (("CE_sum8", hb.PATH_CE, 8, 8), ("SM_copy8_sum8", hb.PATH_SM, 8, 8), ("SM_copy32_sum8", hb.PATH_SM, 8, 32),
-                               ("SM_copy148_sum148", hb.PATH_SM, 148, 148)):
-        c2 = new_comm(path, sum_ctas=sc, copy_ctas=cc)
+    for name, path, sc, cc, op in (("CE_sum8", hb.PATH_CE, 8, 8, 0), ("SM_copy8_sum8", hb.PATH_SM, 8, 8, 0),
+                                   ("SM_copy32_sum8", hb.PATH_SM, 8, 32, 0), ("SM_copy148_sum148", hb.PATH_SM, 148, 148, 0),
+                                   ("onepass_8", hb.PATH_CE, 8, 8, 1)):
+        c2 = new_comm(path, sum_ctas=sc, copy_ctas=cc, onepass=op)
         tf, bw = gemm_tflops(c2)
         probe[name] = {"gemm_TFLOPs": tf, "loss": 1.0 - tf / alone, "comm_busbw_GBps": bw}
         c2.destroy()

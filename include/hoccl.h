@@ -125,6 +125,11 @@ hoccl_result_t hoccl_comm_set_path(hoccl_comm_t comm, hoccl_path_t path);
  *                on one device because every driver copy already spreads over the whole GPU)
  *  "ce_sub_bytes" graph executor, CE path: a move between this many bytes and 16 MiB is issued as sub-copies of
  *                this size (0 = off, the default)
+ *  "onepass"     1 = all-reduce and reduce-scatter run as ONE kernel ("sum_ctas" CTAs) that reduces every element in
+ *                registers in the ring's order and rounding and writes it to its destinations: the same bits, R reads
+ *                + R (or 1) writes per element instead of 7(R-1) bytes per wire byte, no moves, no scratch.  It is not
+ *                rank local (one kernel reads every rank's buffer), so it only makes sense on one device and is kept
+ *                as the comparison point that shows what the rank-local schedule costs.  0 = off (default).
  *  "use_graph"   1 = run a cached CUDA graph built from the plan (default), 0 = streams and events
  *  "handshake"   1 = the paper's stream manager (Sec. 3.2, Listing 1): instead of launching into the caller's
  *                stream, the call enqueues four stream memory operations (write start flag, wait for the CPU's

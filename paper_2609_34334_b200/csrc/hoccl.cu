@@ -79,7 +79,7 @@ struct hoccl_comm {
   int R = 0, device = 0, num_sms = 0;
   hoccl_path_t path = HOCCL_PATH_CE;
   long sum_ctas = 8, copy_ctas = 8, piece_bytes = 4 << 20, max_pieces = 8, lanes = 4, use_graph = 1, profile = 0, p2p_split = 1, ce_sub_bytes = 0,
-       handshake = 0, watchdog_ms = 10000;
+       handshake = 0, watchdog_ms = 10000, onepass = 0;
   Proxy* proxy = nullptr;
   cudaStream_t lane[kMaxLanes] = {};
   cudaStream_t sum_stream = nullptr;
@@ -547,6 +547,31 @@ hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
   if (call->count == 0) return HOCCL_OK;
   CU_TRY(c, cudaSetDevice(c->device));
 
+  if (c->onepass && !c->handshake && (call->kind == PLAN_ALLREDUCE || call->kind == PLAN_REDUCE_SCATTER)) {
+    // comparison point: the whole reduction in one kernel, same order and rounding as the ring, no moves, no scratch
+    OnePassArgs a;
+    a.R = c->R;
+    a.dtype = call->dtype;
+    a.write_all = call->kind == PLAN_ALLREDUCE ? 1 : 0;
+    a.pad = 0;
+    if (call->kind == PLAN_ALLREDUCE) {
+      a.count = call->count;
+      a.q = (call->count + (size_t)c->R - 1) / (size_t)c->R;
+    } else {
+      a.count = (unsigned long long)call->count * c->R;
+      a.q = call->count;
+    }
+    for (int r = 0; r < c->R; r++) {
+      a.x[r] = call->send[r];
+      a.y[r] = call->recv[r];
+    }
+    CU_TRY(c, launch_onepass(a, (int)c->sum_ctas, user));
+    c->stats.n_sum_launches = 1;
+    c->stats.max_sum_ctas = c->sum_ctas;
+    c->stats.n_pieces = 1;
+    c->stats.host_launch_us = now_us() - t0;
+    return HOCCL_OK;
+  }
   Plan P;
   unsigned char align[kMaxRanks];
   for (int r = 0; r < c->R; r++) align[r] = (unsigned char)((uintptr_t)call->send[r] & 15);
@@ -849,7 +874,7 @@ static long* param_slot(hoccl_comm* c, const char* key, long* lo, long* hi) {
               {"lanes", &c->lanes, 1, kMaxLanes},       {"use_graph", &c->use_graph, 0, 1},
               {"profile", &c->profile, 0, 1},           {"p2p_split", &c->p2p_split, 1, kMaxLanes},
               {"ce_sub_bytes", &c->ce_sub_bytes, 0, 1L << 40}, {"handshake", &c->handshake, 0, 1},
-              {"watchdog_ms", &c->watchdog_ms, 10, 600000}};
+              {"watchdog_ms", &c->watchdog_ms, 10, 600000},    {"onepass", &c->onepass, 0, 1}};
   for (auto& r : rows)
     if (std::strcmp(r.name, key) == 0) {
       *lo = r.lo;

@@ -254,6 +254,93 @@ __global__ void __launch_bounds__(THREADS, 1) copy_kernel(const __grid_constant_
   }
 }
 
+// ---- one-pass ring reduction (comparison point) -------------------------------------------------------------------
+template <int DT, int THREADS>
+__global__ void __launch_bounds__(THREADS, 1) onepass_kernel(const __grid_constant__ OnePassArgs a) {
+  using T = Traits<DT>;
+  __shared__ unsigned long long tpre[kMaxOnePassRanks + 1], spre[kMaxOnePassRanks + 1], lo_s[kMaxOnePassRanks], nvec_s[kMaxOnePassRanks];
+  __shared__ int vec_ok;
+  const int R = a.R;
+  if (threadIdx.x == 0) {
+    bool ok = ((a.q * T::E) % 16) == 0;
+    for (int r = 0; r < R; r++) ok = ok && (((uintptr_t)a.x[r] | (uintptr_t)a.y[r]) & 15) == 0;
+    vec_ok = ok ? 1 : 0;
+    unsigned long long t = 0, sc = 0;
+    tpre[0] = 0;
+    spre[0] = 0;
+    for (int c = 0; c < R; c++) {
+      unsigned long long lo = (unsigned long long)c * a.q, hi = lo + a.q;
+      if (lo > a.count) lo = a.count;
+      if (hi > a.count) hi = a.count;
+      const unsigned long long len = hi - lo;
+      const unsigned long long nv = ok ? len / T::VE : 0;
+      lo_s[c] = lo;
+      nvec_s[c] = nv;
+      t += (nv + blockDim.x - 1) / blockDim.x;
+      tpre[c + 1] = t;
+      sc += len - nv * T::VE;
+      spre[c + 1] = sc;
+    }
+  }
+  __syncthreads();
+  // vector part: one 16-byte vector per thread and tile, the R operands loaded in batches of 8 before they are added
+  {
+    int c = 0;
+    for (unsigned long long t = blockIdx.x; t < tpre[R]; t += gridDim.x) {
+      while (t >= tpre[c + 1]) c++;
+      const unsigned long long v = (t - tpre[c]) * blockDim.x + threadIdx.x;
+      if (v >= nvec_s[c]) continue;
+      const size_t byte_off = (size_t)(lo_s[c] + v * T::VE) * T::E;
+      uint4 acc;
+      for (int k0 = 1; k0 <= R; k0 += 8) {
+        uint4 buf[8];
+#pragma unroll
+        for (int j = 0; j < 8; j++)
+          if (k0 + j <= R) buf[j] = __ldcs(reinterpret_cast<const uint4*>(static_cast<const char*>(a.x[(c + k0 + j) % R]) + byte_off));
+#pragma unroll
+        for (int j = 0; j < 8; j++)
+          if (k0 + j <= R) acc = (k0 + j == 1) ? buf[j] : T::add_vec(acc, buf[j]);
+      }
+      if (a.write_all) {
+        for (int r = 0; r < R; r++) *reinterpret_cast<uint4*>(static_cast<char*>(a.y[r]) + byte_off) = acc;
+      } else {
+        *reinterpret_cast<uint4*>(static_cast<char*>(a.y[c]) + (size_t)v * 16) = acc;
+      }
+    }
+  }
+  // element-wise part: chunk tails, or everything when a buffer or the chunk size is not 16-byte aligned
+  {
+    const unsigned long long total = (unsigned long long)gridDim.x * blockDim.x;
+    int c = 0;
+    for (unsigned long long j = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; j < spre[R]; j += total) {
+      while (j >= spre[c + 1]) c++;
+      const unsigned long long local = nvec_s[c] * T::VE + (j - spre[c]);   // element inside chunk c
+      const unsigned long long i = lo_s[c] + local;
+      if (DT == 0) {
+        float acc = static_cast<const float*>(a.x[(c + 1) % R])[i];
+        for (int k = 2; k <= R; k++) acc = __fadd_rn(acc, static_cast<const float*>(a.x[(c + k) % R])[i]);
+        if (a.write_all) {
+          for (int r = 0; r < R; r++) static_cast<float*>(a.y[r])[i] = acc;
+        } else {
+          static_cast<float*>(a.y[c])[local] = acc;
+        }
+      } else {
+        unsigned short acc = static_cast<const unsigned short*>(a.x[(c + 1) % R])[i];
+        for (int k = 2; k <= R; k++) {
+          float s = __fadd_rn(__uint_as_float((uint32_t)acc << 16),
+                              __uint_as_float((uint32_t) static_cast<const unsigned short*>(a.x[(c + k) % R])[i] << 16));
+          acc = __bfloat16_as_ushort(__float2bfloat16_rn(s));
+        }
+        if (a.write_all) {
+          for (int r = 0; r < R; r++) static_cast<unsigned short*>(a.y[r])[i] = acc;
+        } else {
+          static_cast<unsigned short*>(a.y[c])[local] = acc;
+        }
+      }
+    }
+  }
+}
+
 __device__ __forceinline__ unsigned long long global_ns() {
   unsigned long long t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
@@ -296,6 +383,19 @@ cudaError_t launch_copy(const CopyBatch& batch, int ctas, cudaStream_t stream) {
   return cudaGetLastError();
 }
 
+cudaError_t launch_onepass(const OnePassArgs& args, int ctas, cudaStream_t stream) {
+  if (args.count == 0) return cudaSuccess;
+  // more threads under a CTA budget: the loads in flight per SM set the rate there
+  if (wide_grid(ctas)) {
+    if (args.dtype == 0) onepass_kernel<0, 512><<<ctas, 512, 0, stream>>>(args);
+    else onepass_kernel<1, 512><<<ctas, 512, 0, stream>>>(args);
+  } else {
+    if (args.dtype == 0) onepass_kernel<0, 1024><<<ctas, 1024, 0, stream>>>(args);
+    else onepass_kernel<1, 1024><<<ctas, 1024, 0, stream>>>(args);
+  }
+  return cudaGetLastError();
+}
+
 const void* sum_kernel_entry(int dtype, int ctas, int* threads) {
   *threads = wide_grid(ctas) ? 512 : 1024;
   if (dtype == 0)
@@ -313,7 +413,9 @@ cudaError_t preload_kernels() {
   const void* fns[] = {reinterpret_cast<const void*>(&sum2_kernel<0, 4, 512>),  reinterpret_cast<const void*>(&sum2_kernel<0, 4, 1024>),
                        reinterpret_cast<const void*>(&sum2_kernel<1, 4, 512>),  reinterpret_cast<const void*>(&sum2_kernel<1, 4, 1024>),
                        reinterpret_cast<const void*>(&copy_kernel<4, 512>),     reinterpret_cast<const void*>(&copy_kernel<8, 1024>),
-                       reinterpret_cast<const void*>(&occupy_kernel)};
+                       reinterpret_cast<const void*>(&occupy_kernel),           reinterpret_cast<const void*>(&onepass_kernel<0, 512>),
+                       reinterpret_cast<const void*>(&onepass_kernel<1, 512>),  reinterpret_cast<const void*>(&onepass_kernel<0, 1024>),
+                       reinterpret_cast<const void*>(&onepass_kernel<1, 1024>)};
   for (const void* f : fns) {
     cudaFuncAttributes a;
     cudaError_t e = cudaFuncGetAttributes(&a, f);

@@ -34,6 +34,22 @@ struct CopyBatch {
   CopySeg seg[kMaxSegs];
 };
 
+// One-pass variant of the ring reduction (comparison point, not rank local): every element is reduced in registers in
+// the ring's order, chunk c as ((x_{c+1} + x_{c+2}) + ... ) + x_c with a rounding to the I/O dtype after every add, and
+// written to its destinations directly.  Same bits as the ring, R reads + R (or 1) writes per element instead of 7(R-1).
+constexpr int kMaxOnePassRanks = 64;
+struct OnePassArgs {
+  int R;
+  int dtype;
+  int write_all;             // 1: all-reduce (every y[r] gets every chunk); 0: reduce-scatter (chunk c goes to y[c] at offset 0)
+  int pad;
+  unsigned long long count;  // elements of the reduced vector (all-reduce: per rank; reduce-scatter: R * per-rank count)
+  unsigned long long q;      // elements of a full ring chunk
+  const void* x[kMaxOnePassRanks];
+  void* y[kMaxOnePassRanks];
+};
+cudaError_t launch_onepass(const OnePassArgs& args, int ctas, cudaStream_t stream);
+
 // Enqueue helpers (return the CUDA error of the launch).
 cudaError_t launch_sum(const SumBatch& batch, int ctas, cudaStream_t stream);
 cudaError_t launch_copy(const CopyBatch& batch, int ctas, cudaStream_t stream);

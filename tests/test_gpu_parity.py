@@ -289,6 +289,36 @@ def test_alltoallv_user_defined_pattern(oracle, path):
             assert comm.destroy() == hb.OK
 
 
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_onepass_reduction_gives_the_ring_bits(oracle, dtype):
+    """The one-kernel comparison variant reduces in the ring's order and rounding: same bits as the oracle."""
+    e = W.elem_size(dtype)
+    for R, n in SMALL + [(8, 8 * 65_536), (4, 4 * 100_000 + 8), (7, 7 * 4096)]:
+        xs = W.rank_inputs("normal", 300 + n % 11, R, n, dtype, 1.0)
+        want = oracle.ring_allreduce(xs)
+        for ctas in (3, 148):
+            comm = make_comm(R, n, dtype, hb.PATH_CE, onepass=1, sum_ctas=ctas)
+            for in_place in (False, True):
+                got = run_allreduce(comm, xs, dtype, in_place)
+                for r in range(R):
+                    assert same_bits(got[r], want[r], dtype), (R, n, r, in_place, ctas)
+            offs = [e * (r % 3) for r in range(R)]              # unaligned buffers take the element-wise path
+            got = run_allreduce(comm, xs, dtype, False, offs)
+            for r in range(R):
+                assert same_bits(got[r], want[r], dtype)
+            assert comm.last_stats()["n_sum_launches"] == 1 and comm.last_stats()["n_moves"] == 0
+            if n % R == 0:
+                count = n // R
+                wrs = oracle.ring_reduce_scatter(xs)
+                send = [DevBuf(n * e).put(xs[r]) for r in range(R)]
+                recv = [DevBuf(count * e) for _ in range(R)]
+                comm.reduce_scatter(send, recv, count, dtype)
+                torch.cuda.synchronize()
+                for r in range(R):
+                    assert same_bits(recv[r].get(np_dtype(dtype)), wrs[r], dtype) and recv[r].guards_intact()
+            comm.destroy()
+
+
 def test_settings_never_change_a_bit(oracle):
     """Piece size, lane count, CTA budgets, path and executor are pure scheduling choices."""
     R, n, dtype = 8, 8 * 40000 + 8, "bf16"
