@@ -482,6 +482,33 @@ def test_pipeline_wave_small(oracle, per_stage_streams, path):
         assert comm.destroy() == hb.OK
 
 
+def test_config3_pipeline_full_size(oracle):
+    """bf16 activations [4, 2048, 4096] (64 MiB per message) over 8 stages and 16 microbatches, one stream per stage,
+    copy-route path: every microbatch arrives bit for bit.  Microbatch m is the seeded block rotated by m * 4099."""
+    c = W.C3_PIPELINE
+    n = c.count
+    base = W.normal(c.seed, 0, n, c.dtype, 1.0)
+    want = oracle.sendrecv(base)
+    dev = torch.from_numpy(base.view(np.int16)).cuda()
+    comm = hb.Comm(c.stages, 0)
+    slots = [[torch.zeros(n, dtype=torch.int16, device="cuda") for _ in range(c.microbatches)] for _ in range(c.stages)]
+    for m in range(c.microbatches):
+        slots[0][m].copy_(torch.roll(dev, 4099 * m))
+    torch.cuda.synchronize()
+    streams = [torch.cuda.Stream() for _ in range(c.stages)]
+    for m in range(c.microbatches):
+        for s in range(c.stages - 1):
+            comm.send(slots[s][m], n, c.dtype, s, s + 1, streams[s])
+            comm.recv(slots[s + 1][m], n, c.dtype, s, s + 1, streams[s + 1])
+    torch.cuda.synchronize()
+    assert comm.pending() == 0
+    expect = torch.from_numpy(want.view(np.int16)).cuda()
+    for m in range(c.microbatches):
+        for s in range(1, c.stages):
+            assert torch.equal(slots[s][m], torch.roll(expect, 4099 * m)), (m, s)
+    assert comm.destroy() == hb.OK
+
+
 # ------------------------------------------------------------------------------- errors, host path -
 def test_argument_errors_enqueue_nothing():
     R, n = 4, 4096
