@@ -1,0 +1,580 @@
+// The C ABI declared in include/hoccl.h: communicator life cycle, parameters, collectives, send/recv, the user-defined
+// pattern executor, diagnostics, and the host-only planner / scheduler inspection calls.
+#include "comm.h"
+
+using namespace hoccl;
+
+extern "C" {
+
+hoccl_result_t hoccl_comm_init(hoccl_comm_t* comm, int R, int device) {
+  if (!comm || R < 1 || R > kMaxRanks) return HOCCL_ERR_INVALID_ARG;
+  *comm = nullptr;
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || device < 0 || device >= ndev) {
+    cudaGetLastError();
+    return HOCCL_ERR_CUDA;
+  }
+  hoccl_comm* c = new hoccl_comm();
+  c->R = R;
+  c->device = device;
+  cudaError_t e = cudaSetDevice(device);
+  if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->num_sms, cudaDevAttrMultiProcessorCount, device);
+  for (int i = 0; i < kMaxLanes && e == cudaSuccess; i++) e = cudaStreamCreateWithFlags(&c->lane[i], cudaStreamNonBlocking);
+  // SUM launches get the highest priority: a SUM CTA needs a whole SM (1024 threads x 64 registers), and when a
+  // SUM and the next piece's copies become ready at the same moment the copies' small CTAs would otherwise take
+  // every SM first and the SUM would start only after them, which serialises the pipeline.
+  int prio_least = 0, prio_greatest = 0;
+  if (e == cudaSuccess) e = cudaDeviceGetStreamPriorityRange(&prio_least, &prio_greatest);
+  c->sum_priority = prio_greatest;
+  if (e == cudaSuccess) e = cudaStreamCreateWithPriority(&c->sum_stream, cudaStreamNonBlocking, prio_greatest);
+  if (e != cudaSuccess) {
+    for (int i = 0; i < kMaxLanes; i++)
+      if (c->lane[i]) cudaStreamDestroy(c->lane[i]);
+    if (c->sum_stream) cudaStreamDestroy(c->sum_stream);
+    delete c;
+    return HOCCL_ERR_CUDA;
+  }
+  *comm = c;
+  return HOCCL_OK;
+}
+
+hoccl_result_t hoccl_comm_destroy(hoccl_comm_t c) {
+  if (!c) return HOCCL_ERR_INVALID_ARG;
+  if (c->n_pending > 0) return HOCCL_ERR_PENDING;
+  if (c->proxy) {
+    c->proxy->drain(c->watchdog_ms);
+    if (c->proxy->pending_p2p() > 0) return HOCCL_ERR_PENDING;
+    delete c->proxy;
+    c->proxy = nullptr;
+  }
+  cudaSetDevice(c->device);
+  for (int i = 0; i < kMaxLanes; i++)
+    if (c->lane[i]) {
+      cudaStreamSynchronize(c->lane[i]);
+      cudaStreamDestroy(c->lane[i]);
+    }
+  if (c->sum_stream) {
+    cudaStreamSynchronize(c->sum_stream);
+    cudaStreamDestroy(c->sum_stream);
+  }
+  for (auto& e : c->cache) destroy_entry(&e);
+  for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
+  for (auto& p : c->prof_pool) {
+    cudaEventDestroy(p.first);
+    cudaEventDestroy(p.second);
+  }
+  for (auto& p : c->prof_open) {
+    cudaEventDestroy(p.first.first);
+    cudaEventDestroy(p.first.second);
+  }
+  delete c;
+  return HOCCL_OK;
+}
+
+size_t hoccl_scratch_bytes(int R, size_t max_count, hoccl_dtype_t dtype) {
+  size_t e = dtype_size((int)dtype);
+  if (R <= 1 || e == 0 || max_count == 0) return 0;
+  return 2 * (size_t)R * slot_bytes_for(R, max_count, e);
+}
+
+hoccl_result_t hoccl_comm_set_scratch(hoccl_comm_t c, void* dev_ptr, size_t bytes) {
+  if (!c || ((uintptr_t)dev_ptr & 255)) return HOCCL_ERR_INVALID_ARG;
+  c->scratch = dev_ptr;
+  c->scratch_bytes = dev_ptr ? bytes : 0;
+  return HOCCL_OK;
+}
+
+hoccl_result_t hoccl_comm_set_staging(hoccl_comm_t c, void* dev_ptr, size_t bytes) {
+  if (!c || ((uintptr_t)dev_ptr & 255)) return HOCCL_ERR_INVALID_ARG;
+  c->staging = dev_ptr;
+  c->staging_bytes = dev_ptr ? bytes : 0;
+  return HOCCL_OK;
+}
+
+hoccl_result_t hoccl_comm_set_path(hoccl_comm_t c, hoccl_path_t path) {
+  if (!c || (path != HOCCL_PATH_CE && path != HOCCL_PATH_SM)) return HOCCL_ERR_INVALID_ARG;
+  c->path = path;
+  return HOCCL_OK;
+}
+
+static long* param_slot(hoccl_comm* c, const char* key, long* lo, long* hi) {
+  struct Row {
+    const char* name;
+    long* p;
+    long lo, hi;
+  } rows[] = {{"sum_ctas", &c->sum_ctas, 1, 1024},      {"copy_ctas", &c->copy_ctas, 1, 1024},
+              {"piece_bytes", &c->piece_bytes, 1024, 1L << 40}, {"max_pieces", &c->max_pieces, 1, 4096},
+              {"lanes", &c->lanes, 1, kMaxLanes},       {"use_graph", &c->use_graph, 0, 1},
+              {"profile", &c->profile, 0, 1},           {"p2p_split", &c->p2p_split, 1, kMaxLanes},
+              {"ce_sub_bytes", &c->ce_sub_bytes, 0, 1L << 40}, {"handshake", &c->handshake, 0, 1},
+              {"watchdog_ms", &c->watchdog_ms, 10, 600000},    {"onepass", &c->onepass, 0, 1}};
+  for (auto& r : rows)
+    if (std::strcmp(r.name, key) == 0) {
+      *lo = r.lo;
+      *hi = r.hi;
+      return r.p;
+    }
+  return nullptr;
+}
+
+hoccl_result_t hoccl_comm_set_param(hoccl_comm_t c, const char* key, long value) {
+  if (!c || !key) return HOCCL_ERR_INVALID_ARG;
+  long lo, hi;
+  long* p = param_slot(c, key, &lo, &hi);
+  if (!p) return HOCCL_ERR_UNSUPPORTED;
+  if (value < lo || value > hi) return HOCCL_ERR_INVALID_ARG;
+  if (std::strcmp(key, "piece_bytes") == 0) value = (value + 1023) / 1024 * 1024;
+  *p = value;
+  return HOCCL_OK;
+}
+
+hoccl_result_t hoccl_comm_get_param(hoccl_comm_t c, const char* key, long* value) {
+  if (!c || !key || !value) return HOCCL_ERR_INVALID_ARG;
+  long lo, hi;
+  long* p = param_slot(c, key, &lo, &hi);
+  if (!p) return HOCCL_ERR_UNSUPPORTED;
+  *value = *p;
+  return HOCCL_OK;
+}
+
+hoccl_result_t hoccl_allreduce(const void* const* send, void* const* recv, size_t count, hoccl_dtype_t dtype, hoccl_op_t op,
+                               hoccl_comm_t c, hoccl_stream_t stream) {
+  if (!c) return HOCCL_ERR_INVALID_ARG;
+  if (op != HOCCL_SUM) return HOCCL_ERR_UNSUPPORTED;
+  size_t e = dtype_size((int)dtype);
+  Call call{PLAN_ALLREDUCE, count, (int)dtype, false, count * e, count * e, send, recv};
+  return run_collective(c, &call, (cudaStream_t)stream);
+}
+
+hoccl_result_t hoccl_reduce_scatter(const void* const* send, void* const* recv, size_t count, hoccl_dtype_t dtype, hoccl_op_t op,
+                                    hoccl_comm_t c, hoccl_stream_t stream) {
+  if (!c) return HOCCL_ERR_INVALID_ARG;
+  if (op != HOCCL_SUM) return HOCCL_ERR_UNSUPPORTED;
+  size_t e = dtype_size((int)dtype);
+  Call call{PLAN_REDUCE_SCATTER, count, (int)dtype, false, (size_t)c->R * count * e, count * e, send, recv};
+  return run_collective(c, &call, (cudaStream_t)stream);
+}
+
+hoccl_result_t hoccl_allgather(const void* const* send, void* const* recv, size_t count, hoccl_dtype_t dtype, hoccl_comm_t c,
+                               hoccl_stream_t stream) {
+  if (!c) return HOCCL_ERR_INVALID_ARG;
+  size_t e = dtype_size((int)dtype);
+  Call call{PLAN_ALLGATHER, count, (int)dtype, false, count * e, (size_t)c->R * count * e, send, recv};
+  return run_collective(c, &call, (cudaStream_t)stream);
+}
+
+hoccl_result_t hoccl_alltoall(const void* const* send, void* const* recv, size_t count, hoccl_dtype_t dtype, hoccl_comm_t c,
+                              hoccl_stream_t stream) {
+  if (!c) return HOCCL_ERR_INVALID_ARG;
+  size_t e = dtype_size((int)dtype);
+  Call call{PLAN_ALLTOALL, count, (int)dtype, false, (size_t)c->R * count * e, (size_t)c->R * count * e, send, recv};
+  return run_collective(c, &call, (cudaStream_t)stream);
+}
+
+hoccl_result_t hoccl_send(const void* buf, size_t count, hoccl_dtype_t dtype, int src, int dst, hoccl_comm_t c, hoccl_stream_t stream) {
+  return p2p_post(c, true, const_cast<void*>(buf), count, (int)dtype, src, dst, (cudaStream_t)stream);
+}
+
+hoccl_result_t hoccl_recv(void* buf, size_t count, hoccl_dtype_t dtype, int src, int dst, hoccl_comm_t c, hoccl_stream_t stream) {
+  return p2p_post(c, false, buf, count, (int)dtype, src, dst, (cudaStream_t)stream);
+}
+
+int hoccl_comm_pending(hoccl_comm_t c) {
+  if (!c) return 0;
+  return c->n_pending + (c->proxy ? c->proxy->pending_p2p() : 0);
+}
+
+hoccl_result_t hoccl_comm_async_error(hoccl_comm_t c, int clear) {
+  if (!c) return HOCCL_ERR_INVALID_ARG;
+  if (!c->proxy) return HOCCL_OK;
+  int e = c->proxy->async_error();
+  if (clear) c->proxy->clear_error();
+  switch (e) {
+    case PROXY_OK: return HOCCL_OK;
+    case PROXY_TIMEOUT: return HOCCL_ERR_TIMEOUT;
+    case PROXY_MISMATCH: return HOCCL_ERR_MISMATCH;
+    default: return HOCCL_ERR_CUDA;
+  }
+}
+
+long hoccl_comm_handshakes(hoccl_comm_t c) { return (c && c->proxy) ? c->proxy->handshakes() : 0; }
+
+hoccl_result_t hoccl_host_allreduce(const void* const* h_send, void* const* h_recv, size_t count, hoccl_dtype_t dtype, hoccl_op_t op,
+                                    hoccl_comm_t c, hoccl_stream_t stream) {
+  if (!c || !h_send || !h_recv) return HOCCL_ERR_INVALID_ARG;
+  if (op != HOCCL_SUM) return HOCCL_ERR_UNSUPPORTED;
+  size_t e = dtype_size((int)dtype);
+  if (e == 0) return HOCCL_ERR_UNSUPPORTED;
+  const int R = c->R;
+  for (int r = 0; r < R; r++)
+    if (!h_send[r] || !h_recv[r]) return HOCCL_ERR_INVALID_ARG;
+  if (count == 0) return HOCCL_OK;
+  const size_t per = (count * e + 255) / 256 * 256;
+  if (!c->staging || c->staging_bytes < 2 * (size_t)R * per) return HOCCL_ERR_SCRATCH;
+  CU_TRY(c, cudaSetDevice(c->device));
+  cudaStream_t st = (cudaStream_t)stream;
+  const void* dsend[kMaxRanks];
+  void* drecv[kMaxRanks];
+  for (int r = 0; r < R; r++) {
+    dsend[r] = (char*)c->staging + (size_t)r * per;
+    drecv[r] = (char*)c->staging + (size_t)(R + r) * per;
+    CU_TRY(c, cudaMemcpyAsync(const_cast<void*>(dsend[r]), h_send[r], count * e, cudaMemcpyHostToDevice, st));
+  }
+  hoccl_result_t rc = hoccl_allreduce(dsend, drecv, count, dtype, op, c, stream);
+  if (rc != HOCCL_OK) return rc;
+  for (int r = 0; r < R; r++) CU_TRY(c, cudaMemcpyAsync(h_recv[r], drecv[r], count * e, cudaMemcpyDeviceToHost, st));
+  return HOCCL_OK;
+}
+
+hoccl_result_t hoccl_alltoallv(const void* const* send, const size_t* sendcounts, const size_t* sdispls, void* const* recv,
+                               const size_t* rdispls, hoccl_dtype_t dtype, hoccl_comm_t c, hoccl_stream_t stream) {
+  const double t0 = now_us();
+  if (!c || !send || !recv || !sendcounts || !sdispls || !rdispls) return HOCCL_ERR_INVALID_ARG;
+  const size_t e = dtype_size((int)dtype);
+  if (e == 0) return HOCCL_ERR_UNSUPPORTED;
+  if (c->handshake) return HOCCL_ERR_UNSUPPORTED;
+  const int R = c->R;
+  for (int r = 0; r < R; r++) {
+    if (!send[r] || !recv[r]) return HOCCL_ERR_INVALID_ARG;
+    if (((uintptr_t)send[r] % e) || ((uintptr_t)recv[r] % e)) return HOCCL_ERR_INVALID_ARG;
+  }
+  // the flows of the user-defined pattern as the origin traffic matrix C (bytes); one NVLink domain, no RDMA
+  Topology topo;
+  topo.G = R;
+  topo.gpus_per_node = R;
+  std::vector<uint64_t> C((size_t)R * R);
+  uint64_t total = 0;
+  for (int u = 0; u < R; u++)
+    for (int v = 0; v < R; v++) {
+      C[(size_t)u * R + v] = (uint64_t)sendcounts[(size_t)u * R + v] * e;
+      total += C[(size_t)u * R + v];
+    }
+  // receive regions of one rank must not overlap each other, and no send region may overlap a receive region
+  for (int v = 0; v < R; v++)
+    for (int a = 0; a < R; a++) {
+      const char* ra = (const char*)recv[v] + rdispls[(size_t)v * R + a] * e;
+      const size_t la = C[(size_t)a * R + v];
+      for (int b = a + 1; b < R; b++)
+        if (ranges_overlap(ra, la, (const char*)recv[v] + rdispls[(size_t)v * R + b] * e, C[(size_t)b * R + v])) return HOCCL_ERR_INVALID_ARG;
+      for (int u = 0; u < R; u++)
+        for (int w = 0; w < R; w++)
+          if (ranges_overlap(ra, la, (const char*)send[u] + sdispls[(size_t)u * R + w] * e, C[(size_t)u * R + w])) return HOCCL_ERR_INVALID_ARG;
+    }
+  c->stats = hoccl_stats_t{};
+  if (total == 0) return HOCCL_OK;
+  Schedule S;
+  if (!build_schedule(topo, C, (uint64_t)std::max<long>(c->piece_bytes, 65536), &S)) return HOCCL_ERR_INTERNAL;
+  CU_TRY(c, cudaSetDevice(c->device));
+  cudaStream_t user = (cudaStream_t)stream;
+  const int lanes = c->path == HOCCL_PATH_SM ? 1 : (int)std::max<long>(1, std::min<long>(c->lanes, kMaxLanes));
+  c->ev_next = 0;
+  cudaEvent_t fork = next_event(c);
+  if (!fork) return cuda_fail(c, cudaErrorMemoryAllocation, "event pool");
+  CU_TRY(c, cudaEventRecord(fork, user));
+  for (int l = 0; l < lanes; l++) CU_TRY(c, cudaStreamWaitEvent(c->lane[l], fork, 0));
+  long moves = 0, launches = 0;
+  for (size_t si = 0; si < S.stages.size(); si++) {
+    const Stage& st = S.stages[si];
+    // every DMA queue (one per source rank) is a serial chain on its lane, in the interleaved chunk order
+    for (int g = 0; g < R; g++) {
+      cudaStream_t lane = c->lane[g % lanes];
+      for (const ChunkItem& it : st.queues[g]) {
+        const StageFlow& f = st.flows[it.flow];
+        const size_t so = sdispls[(size_t)f.origin_src * R + f.origin_dst] * e + f.origin_offset + it.offset;
+        const size_t dofs = rdispls[(size_t)f.origin_dst * R + f.origin_src] * e + f.origin_offset + it.offset;
+        const char* src = (const char*)send[f.origin_src] + so;
+        char* dst = (char*)recv[f.origin_dst] + dofs;
+        if (c->path == HOCCL_PATH_CE) {
+          CU_TRY(c, cudaMemcpyAsync(dst, src, it.bytes, cudaMemcpyDeviceToDevice, lane));
+        } else {
+          CopyBatch b;
+          b.nseg = 1;
+          b.pad = 0;
+          b.seg[0] = CopySeg{src, dst, (unsigned long long)it.bytes};
+          CU_TRY(c, launch_copy(b, (int)c->copy_ctas, lane));
+          launches++;
+        }
+        moves++;
+      }
+    }
+    // stages run one after the other (the paper's serial stages): barrier over the lanes
+    if (si + 1 < S.stages.size() && lanes > 1) {
+      std::vector<cudaEvent_t> evs(lanes);
+      for (int l = 0; l < lanes; l++) {
+        evs[l] = next_event(c);
+        if (!evs[l]) return cuda_fail(c, cudaErrorMemoryAllocation, "event pool");
+        CU_TRY(c, cudaEventRecord(evs[l], c->lane[l]));
+      }
+      for (int l = 0; l < lanes; l++)
+        for (int m = 0; m < lanes; m++)
+          if (m != l) CU_TRY(c, cudaStreamWaitEvent(c->lane[l], evs[m], 0));
+    }
+  }
+  for (int l = 0; l < lanes; l++) {
+    cudaEvent_t ev = next_event(c);
+    if (!ev) return cuda_fail(c, cudaErrorMemoryAllocation, "event pool");
+    CU_TRY(c, cudaEventRecord(ev, c->lane[l]));
+    CU_TRY(c, cudaStreamWaitEvent(user, ev, 0));
+  }
+  c->stats.n_moves = moves;
+  c->stats.n_move_launches = launches;
+  c->stats.max_copy_ctas = launches ? c->copy_ctas : 0;
+  c->stats.n_pieces = (long)S.stages.size();
+  c->stats.host_launch_us = now_us() - t0;
+  return HOCCL_OK;
+}
+
+// ---------------------------------------------------------------- scheduler inspection (host only) ----
+struct hoccl_sched {
+  Schedule s;
+};
+
+hoccl_result_t hoccl_sched_build(hoccl_sched_t* out, int G, int gpus_per_node, double bw_nvlink, double bw_rdma, const uint64_t* C,
+                                 uint64_t chunk_bytes) {
+  if (!out) return HOCCL_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!C || G < 1 || G > 256 || gpus_per_node < 1 || chunk_bytes == 0) return HOCCL_ERR_INVALID_ARG;
+  Topology t;
+  t.G = G;
+  t.gpus_per_node = gpus_per_node;
+  if (bw_nvlink > 0) t.bw_nvlink = bw_nvlink;
+  if (bw_rdma > 0) t.bw_rdma = bw_rdma;
+  hoccl_sched* h = new hoccl_sched();
+  std::vector<uint64_t> Cv(C, C + (size_t)G * G);
+  if (!build_schedule(t, Cv, chunk_bytes, &h->s)) {
+    delete h;
+    return HOCCL_ERR_INVALID_ARG;
+  }
+  *out = h;
+  return HOCCL_OK;
+}
+
+void hoccl_sched_destroy(hoccl_sched_t s) { delete s; }
+int hoccl_sched_num_stages(hoccl_sched_t s) { return s ? (int)s->s.stages.size() : 0; }
+double hoccl_sched_stage_tau(hoccl_sched_t s, int stage) {
+  return (s && stage >= 0 && stage < (int)s->s.stages.size()) ? s->s.stages[stage].tau : -1.0;
+}
+double hoccl_sched_total_tau(hoccl_sched_t s) { return s ? s->s.total_tau : -1.0; }
+double hoccl_sched_lower_bound(hoccl_sched_t s) { return s ? s->s.lower_bound : -1.0; }
+
+hoccl_result_t hoccl_sched_matrix(hoccl_sched_t s, int which, uint64_t* out) {
+  if (!s || !out) return HOCCL_ERR_INVALID_ARG;
+  const int G = s->s.topo.G;
+  const size_t n = (size_t)G * G;
+  if (which == -1) {
+    std::copy(s->s.T.begin(), s->s.T.end(), out);
+  } else if (which == -2) {
+    std::copy(s->s.C.begin(), s->s.C.end(), out);
+  } else if (which >= 0 && which < (int)s->s.stages.size()) {
+    std::fill(out, out + n, 0);
+    for (const StageFlow& f : s->s.stages[which].flows) out[(size_t)f.u * G + f.v] += f.bytes;
+  } else {
+    return HOCCL_ERR_INVALID_ARG;
+  }
+  return HOCCL_OK;
+}
+
+int hoccl_sched_num_flows(hoccl_sched_t s, int stage) {
+  return (s && stage >= 0 && stage < (int)s->s.stages.size()) ? (int)s->s.stages[stage].flows.size() : -1;
+}
+
+hoccl_result_t hoccl_sched_get_flow(hoccl_sched_t s, int stage, int index, hoccl_sched_flow_t* out) {
+  if (!s || !out || stage < 0 || stage >= (int)s->s.stages.size()) return HOCCL_ERR_INVALID_ARG;
+  const Stage& st = s->s.stages[stage];
+  if (index < 0 || index >= (int)st.flows.size()) return HOCCL_ERR_INVALID_ARG;
+  const StageFlow& f = st.flows[index];
+  out->src = f.u;
+  out->dst = f.v;
+  out->cls = f.cls;
+  out->origin_src = f.origin_src;
+  out->origin_dst = f.origin_dst;
+  out->bytes = f.bytes;
+  out->origin_offset = f.origin_offset;
+  return HOCCL_OK;
+}
+
+int hoccl_sched_queue_len(hoccl_sched_t s, int stage, int gpu) {
+  if (!s || stage < 0 || stage >= (int)s->s.stages.size() || gpu < 0 || gpu >= s->s.topo.G) return -1;
+  return (int)s->s.stages[stage].queues[gpu].size();
+}
+
+hoccl_result_t hoccl_sched_queue_get(hoccl_sched_t s, int stage, int gpu, int index, int* flow, uint64_t* offset, uint64_t* bytes) {
+  if (!s || !flow || !offset || !bytes || stage < 0 || stage >= (int)s->s.stages.size() || gpu < 0 || gpu >= s->s.topo.G)
+    return HOCCL_ERR_INVALID_ARG;
+  const auto& q = s->s.stages[stage].queues[gpu];
+  if (index < 0 || index >= (int)q.size()) return HOCCL_ERR_INVALID_ARG;
+  *flow = q[index].flow;
+  *offset = q[index].offset;
+  *bytes = q[index].bytes;
+  return HOCCL_OK;
+}
+
+const char* hoccl_error_string(hoccl_result_t code) {
+  switch (code) {
+    case HOCCL_OK: return "ok";
+    case HOCCL_ERR_INVALID_ARG: return "invalid argument";
+    case HOCCL_ERR_UNSUPPORTED: return "unsupported operation, dtype or parameter";
+    case HOCCL_ERR_CUDA: return "CUDA error";
+    case HOCCL_ERR_MISMATCH: return "send/recv mismatch";
+    case HOCCL_ERR_PENDING: return "unmatched send/recv posts pending";
+    case HOCCL_ERR_SCRATCH: return "scratch or staging memory missing or too small";
+    case HOCCL_ERR_INTERNAL: return "internal error";
+    case HOCCL_ERR_TIMEOUT: return "watchdog timeout in the stream hand-over (the stream was released)";
+  }
+  return "unknown error code";
+}
+
+const char* hoccl_last_cuda_error(hoccl_comm_t c) { return c ? c->cuda_err.c_str() : ""; }
+
+hoccl_result_t hoccl_last_stats(hoccl_comm_t c, hoccl_stats_t* out) {
+  if (!c || !out) return HOCCL_ERR_INVALID_ARG;
+  // profile numbers: read events of work that has completed (the caller synchronises first)
+  harvest_profile(c);
+  *out = c->stats;
+  out->sum_kernel_ms = c->prof_ms;
+  out->sum_kernel_launches_timed = c->prof_n;
+  out->sum_kernel_bytes = c->prof_bytes;
+  return HOCCL_OK;
+}
+
+hoccl_result_t hoccl_profile_reset(hoccl_comm_t c) {
+  if (!c) return HOCCL_ERR_INVALID_ARG;
+  harvest_profile(c);
+  c->prof_ms = 0;
+  c->prof_bytes = 0;
+  c->prof_n = 0;
+  return HOCCL_OK;
+}
+
+hoccl_result_t hoccl_probe_move_needs_sm(hoccl_comm_t c, hoccl_path_t path, void* dst, const void* src, size_t bytes, int spin_us,
+                                         int* needs_sm, double* move_end_us) {
+  if (!c || !dst || !src || !needs_sm || bytes == 0 || spin_us < 100 || spin_us > 20000) return HOCCL_ERR_INVALID_ARG;
+  CU_TRY(c, cudaSetDevice(c->device));
+  CU_TRY(c, cudaDeviceSynchronize());
+  cudaEvent_t a0, a1, b1;
+  CU_TRY(c, cudaEventCreate(&a0));
+  CU_TRY(c, cudaEventCreate(&a1));
+  CU_TRY(c, cudaEventCreate(&b1));
+  hoccl_result_t rc = HOCCL_OK;
+  cudaError_t e = cudaEventRecord(a0, c->lane[0]);
+  int ctas = 0;
+  if (e == cudaSuccess) e = launch_occupy_all_sms((unsigned long long)spin_us * 1000ull, c->num_sms, c->lane[0], &ctas);
+  if (e == cudaSuccess) e = cudaEventRecord(a1, c->lane[0]);
+  // let the occupying kernel become resident before the move is enqueued
+  const double t0 = now_us();
+  while (now_us() - t0 < std::min(300.0, spin_us * 0.25)) {
+  }
+  if (e == cudaSuccess) {
+    if (path == HOCCL_PATH_CE) {
+      e = cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDefault, c->lane[1]);  // src may be pinned host memory (control)
+    } else {
+      CopyBatch b;
+      b.nseg = 1;
+      b.pad = 0;
+      b.seg[0] = CopySeg{src, dst, (unsigned long long)bytes};
+      e = launch_copy(b, (int)c->copy_ctas, c->lane[1]);
+    }
+  }
+  if (e == cudaSuccess) e = cudaEventRecord(b1, c->lane[1]);
+  if (e == cudaSuccess) e = cudaDeviceSynchronize();
+  float spin_ms = 0, end_ms = 0;
+  if (e == cudaSuccess) e = cudaEventElapsedTime(&spin_ms, a0, a1);
+  if (e == cudaSuccess) e = cudaEventElapsedTime(&end_ms, a0, b1);
+  if (e != cudaSuccess) rc = cuda_fail(c, e, "probe_move_needs_sm");
+  else {
+    *needs_sm = end_ms >= 0.9f * spin_ms ? 1 : 0;
+    if (move_end_us) *move_end_us = end_ms * 1e3;
+  }
+  cudaEventDestroy(a0);
+  cudaEventDestroy(a1);
+  cudaEventDestroy(b1);
+  return rc;
+}
+
+hoccl_result_t hoccl_sum_launch(const void* inbox, const void* local, void* out, size_t count, hoccl_dtype_t dtype, int ctas,
+                                hoccl_stream_t stream) {
+  size_t e = dtype_size((int)dtype);
+  if (e == 0) return HOCCL_ERR_UNSUPPORTED;
+  if (!inbox || !local || !out || ctas < 1 || ctas > 1024) return HOCCL_ERR_INVALID_ARG;
+  if (((uintptr_t)inbox % e) || ((uintptr_t)local % e) || ((uintptr_t)out % e)) return HOCCL_ERR_INVALID_ARG;
+  if (count == 0) return HOCCL_OK;
+  SumBatch b;
+  b.nseg = 1;
+  b.dtype = (int)dtype;
+  b.seg[0] = SumSeg{inbox, local, out, (unsigned long long)count};
+  return launch_sum(b, ctas, (cudaStream_t)stream) == cudaSuccess ? HOCCL_OK : HOCCL_ERR_CUDA;
+}
+
+hoccl_result_t hoccl_copy_launch(const void* src, void* dst, size_t bytes, int ctas, hoccl_stream_t stream) {
+  if (!src || !dst || ctas < 1 || ctas > 1024) return HOCCL_ERR_INVALID_ARG;
+  if (bytes == 0) return HOCCL_OK;
+  CopyBatch b;
+  b.nseg = 1;
+  b.pad = 0;
+  b.seg[0] = CopySeg{src, dst, (unsigned long long)bytes};
+  return launch_copy(b, ctas, (cudaStream_t)stream) == cudaSuccess ? HOCCL_OK : HOCCL_ERR_CUDA;
+}
+
+// ---------------------------------------------------------------- plan inspection ----------------
+struct hoccl_plan {
+  Plan p;
+};
+
+hoccl_result_t hoccl_plan_build(hoccl_plan_t* plan, int kind, int R, size_t count, hoccl_dtype_t dtype, int in_place, size_t piece_bytes,
+                                int max_pieces, const unsigned char* send_align) {
+  if (!plan) return HOCCL_ERR_INVALID_ARG;
+  *plan = nullptr;
+  if (R < 1 || R > kMaxRanks) return HOCCL_ERR_INVALID_ARG;
+  if (dtype_size((int)dtype) == 0) return HOCCL_ERR_UNSUPPORTED;
+  hoccl_plan* h = new hoccl_plan();
+  if (!build_plan(&h->p, kind, R, count, (int)dtype, in_place != 0, piece_bytes, max_pieces, send_align)) {
+    delete h;
+    return HOCCL_ERR_INVALID_ARG;
+  }
+  *plan = h;
+  return HOCCL_OK;
+}
+
+void hoccl_plan_destroy(hoccl_plan_t plan) { delete plan; }
+size_t hoccl_plan_slot_bytes(hoccl_plan_t plan) { return plan ? plan->p.slot_bytes : 0; }
+int hoccl_plan_num_ops(hoccl_plan_t plan) { return plan ? (int)plan->p.ops.size() : 0; }
+int hoccl_plan_num_groups(hoccl_plan_t plan) { return plan ? (int)plan->p.groups.size() : 0; }
+
+hoccl_result_t hoccl_plan_get_op(hoccl_plan_t plan, int index, hoccl_plan_op_t* out) {
+  if (!plan || !out || index < 0 || index >= (int)plan->p.ops.size()) return HOCCL_ERR_INVALID_ARG;
+  const PlanOp& o = plan->p.ops[index];
+  out->kind = o.kind;
+  out->phase = o.phase;
+  out->step = o.step;
+  out->piece = o.piece;
+  out->rank = o.rank;
+  out->dst_rank = o.dst_rank;
+  out->chunk = o.chunk;
+  out->src_buf = o.src_buf;
+  out->dst_buf = o.dst_buf;
+  out->local_buf = o.local_buf;
+  out->src_off = o.src_off;
+  out->dst_off = o.dst_off;
+  out->local_off = o.local_off;
+  out->bytes = o.bytes;
+  out->group = o.group;
+  return HOCCL_OK;
+}
+
+int hoccl_plan_group_deps(hoccl_plan_t plan, int group, int* deps, int cap) {
+  if (!plan || group < 0 || group >= (int)plan->p.groups.size()) return -1;
+  const PlanGroup& g = plan->p.groups[group];
+  int n = 0;
+  for (int d : g.deps) {
+    if (deps && n < cap) deps[n] = d;
+    n++;
+  }
+  if (g.chain_dep >= 0 && std::find(g.deps.begin(), g.deps.end(), g.chain_dep) == g.deps.end()) {
+    if (deps && n < cap) deps[n] = g.chain_dep;
+    n++;
+  }
+  return n;
+}
+
+
+}  // extern "C"

@@ -1,0 +1,143 @@
+// Shared internals of libhoccl: the communicator object and small helpers used by the executors, the point-to-point
+// path, the pattern executor and the C ABI.
+#pragma once
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <chrono>
+#include <cstdio>
+#include <cstring>
+#include <deque>
+#include <map>
+#include <string>
+#include <utility>
+#include <vector>
+
+#include "../../include/hoccl.h"
+#include "kernels.cuh"
+#include "plan.h"
+#include "proxy.h"
+#include "sched.h"
+
+namespace hoccl {
+
+constexpr int kMaxRanks = 64;
+constexpr int kMaxLanes = 8;
+constexpr size_t kGraphCacheCap = 48;
+
+inline double now_us() {
+  return std::chrono::duration<double, std::micro>(std::chrono::steady_clock::now().time_since_epoch()).count();
+}
+
+struct Seg {
+  const char* src;    // MOVE: source; SUM: inbox
+  const char* local;  // SUM only
+  char* dst;
+  uint64_t bytes;
+};
+
+struct RGroup {
+  int kind;
+  std::vector<Seg> segs;
+  std::vector<int> deps;
+  int chain_dep;
+};
+
+struct Post {
+  bool is_send;
+  void* buf;
+  size_t count;
+  int dtype;
+  cudaStream_t stream;
+};
+
+struct GraphEntry {
+  std::vector<uint64_t> key;
+  cudaGraphExec_t exec = nullptr;
+  uint64_t last_use = 0;
+  long n_moves = 0, n_move_launches = 0, n_sum_launches = 0, n_pieces = 0;
+  std::vector<std::pair<cudaEvent_t, cudaEvent_t>> prof_events;  // owned; only with profile = 1
+  std::vector<double> prof_bytes;
+  bool prof_pending = false;  // replayed since the profile events were last read
+};
+
+}  // namespace hoccl
+
+struct hoccl_comm {
+  int R = 0, device = 0, num_sms = 0;
+  hoccl_path_t path = HOCCL_PATH_CE;
+  long sum_ctas = 8, copy_ctas = 8, piece_bytes = 4 << 20, max_pieces = 8, lanes = 4, use_graph = 1, profile = 0, p2p_split = 1, ce_sub_bytes = 0,
+       handshake = 0, watchdog_ms = 10000, onepass = 0;
+  hoccl::Proxy* proxy = nullptr;
+  cudaStream_t lane[hoccl::kMaxLanes] = {};
+  cudaStream_t sum_stream = nullptr;
+  int sum_priority = 0;
+  std::vector<cudaEvent_t> ev_pool;
+  size_t ev_next = 0;
+  void* scratch = nullptr;
+  size_t scratch_bytes = 0;
+  void* staging = nullptr;
+  size_t staging_bytes = 0;
+  std::map<std::pair<int, int>, std::deque<hoccl::Post>> pending;
+  int n_pending = 0;
+  unsigned p2p_rr = 0;
+  std::vector<hoccl::GraphEntry> cache;
+  uint64_t use_counter = 0;
+  hoccl_stats_t stats = {};
+  std::string cuda_err;
+  // profile accumulation
+  std::vector<std::pair<cudaEvent_t, cudaEvent_t>> prof_pool;   // timing events of the stream executor
+  std::vector<std::pair<std::pair<cudaEvent_t, cudaEvent_t>, double>> prof_open;  // recorded, not yet read
+  double prof_ms = 0, prof_bytes = 0;
+  long prof_n = 0;
+};
+
+namespace hoccl {
+
+inline hoccl_result_t cuda_fail(hoccl_comm* c, cudaError_t e, const char* what) {
+  if (c) {
+    c->cuda_err = std::string(what) + ": " + cudaGetErrorString(e);
+  }
+  return HOCCL_ERR_CUDA;
+}
+
+#define CU_TRY(c, call)                                   \
+  do {                                                    \
+    cudaError_t e__ = (call);                             \
+    if (e__ != cudaSuccess) return cuda_fail(c, e__, #call); \
+  } while (0)
+
+inline cudaEvent_t next_event(hoccl_comm* c) {
+  if (c->ev_next == c->ev_pool.size()) {
+    cudaEvent_t e = nullptr;
+    if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    c->ev_pool.push_back(e);
+  }
+  return c->ev_pool[c->ev_next++];
+}
+
+inline bool ranges_overlap(const char* a, size_t an, const char* b, size_t bn) {
+  if (an == 0 || bn == 0) return false;
+  return a < b + bn && b < a + an;
+}
+
+struct Call {
+  int kind;  // PlanKind
+  size_t count;
+  int dtype;
+  bool in_place;
+  size_t send_bytes, recv_bytes;
+  const void* const* send;
+  void* const* recv;
+};
+
+
+// exec.cu
+hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user);
+hoccl_result_t ensure_proxy(hoccl_comm* c);
+void harvest_profile(hoccl_comm* c);
+void destroy_entry(GraphEntry* e);
+// p2p.cu
+hoccl_result_t p2p_post(hoccl_comm* c, bool is_send, void* buf, size_t count, int dtype, int src, int dst, cudaStream_t stream);
+
+}  // namespace hoccl

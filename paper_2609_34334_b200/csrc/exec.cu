@@ -1,0 +1,529 @@
+// libhoccl: communicator, executors and the C ABI declared in include/hoccl.h.
+//
+// A collective call = plan (host, plan.cpp) -> resolve the plan's buffer offsets against the caller's
+// pointers -> issue.  Two issue engines consume the same plan and give the same bits:
+//   * graph executor (default): the plan's group DAG becomes an explicit CUDA graph (memcpy nodes for
+//     moves on the copy route, kernel nodes for sums and SM copies), instantiated once per distinct
+//     call signature, cached, and replayed with one cudaGraphLaunch into the caller's stream.  A graph
+//     launch is stream ordered, which is exactly the operator-level ordering the paper's stream
+//     manager provides (Sec. 3.2), and it removes the per-operation host cost that the paper reports
+//     as its launch overhead (Sec. 5 "CPU launch overhead").
+//   * stream executor: internal move lanes plus one sum stream, ordered with CUDA events
+//     (fork from the caller's stream, join back into it).
+// SUM launches are chained (one at a time) so that the SM budget for sums is global, not per piece.
+#include "comm.h"
+
+namespace hoccl {
+
+hoccl_result_t validate(hoccl_comm* c, Call* call) {
+  const int R = c->R;
+  const size_t e = dtype_size(call->dtype);
+  if (!call->send || !call->recv) return HOCCL_ERR_INVALID_ARG;
+  for (int r = 0; r < R; r++) {
+    if (!call->send[r] || !call->recv[r]) return HOCCL_ERR_INVALID_ARG;
+    if (((uintptr_t)call->send[r] % e) || ((uintptr_t)call->recv[r] % e)) return HOCCL_ERR_INVALID_ARG;
+  }
+  // in-place forms
+  int n_in = 0;
+  for (int r = 0; r < R; r++) {
+    const char* s = (const char*)call->send[r];
+    const char* d = (const char*)call->recv[r];
+    bool in;
+    if (call->kind == PLAN_ALLREDUCE) in = (s == d);
+    else if (call->kind == PLAN_REDUCE_SCATTER) in = (d == s + (size_t)r * call->count * e);
+    else if (call->kind == PLAN_ALLTOALL) in = false;   // no in-place form: any overlap of send[r] and recv[r] is an error
+    else in = (s == d + (size_t)r * call->count * e);
+    if (in) n_in++;
+    else if (ranges_overlap(s, call->send_bytes, d, call->recv_bytes)) return HOCCL_ERR_INVALID_ARG;
+  }
+  if (n_in != 0 && n_in != R) return HOCCL_ERR_INVALID_ARG;
+  call->in_place = (n_in == R);
+  // buffers of different ranks must be disjoint
+  for (int a = 0; a < R; a++)
+    for (int b = a + 1; b < R; b++) {
+      const char *sa = (const char*)call->send[a], *sb = (const char*)call->send[b];
+      const char *da = (const char*)call->recv[a], *db = (const char*)call->recv[b];
+      if (ranges_overlap(sa, call->send_bytes, sb, call->send_bytes) || ranges_overlap(da, call->recv_bytes, db, call->recv_bytes) ||
+          ranges_overlap(sa, call->send_bytes, db, call->recv_bytes) || ranges_overlap(da, call->recv_bytes, sb, call->send_bytes))
+        return HOCCL_ERR_INVALID_ARG;
+    }
+  return HOCCL_OK;
+}
+
+// Turns plan offsets into addresses (the plan already places pieces inside the scratch slots).
+void resolve(hoccl_comm* c, const Plan& P, const Call& call, std::vector<RGroup>* out) {
+  const int R = P.R;
+  char* inbox0 = (char*)c->scratch;
+  char* partial0 = inbox0 + (size_t)R * P.slot_bytes;
+  auto addr = [&](int buf, int rank, int chunk, uint64_t off) -> char* {
+    (void)chunk;
+    switch (buf) {
+      case BUF_SEND: return (char*)call.send[rank] + off;
+      case BUF_RECV: return (char*)call.recv[rank] + off;
+      case BUF_INBOX: return inbox0 + (size_t)rank * P.slot_bytes + off;
+      default: return partial0 + (size_t)rank * P.slot_bytes + off;
+    }
+  };
+  out->clear();
+  out->resize(P.groups.size());
+  for (size_t g = 0; g < P.groups.size(); g++) {
+    const PlanGroup& pg = P.groups[g];
+    RGroup& rg = (*out)[g];
+    rg.kind = pg.kind;
+    rg.deps = pg.deps;
+    rg.chain_dep = pg.chain_dep;
+    for (int i = 0; i < pg.num_ops; i++) {
+      const PlanOp& op = P.ops[pg.first_op + i];
+      Seg s;
+      s.bytes = op.bytes;
+      if (op.kind == OP_MOVE) {
+        s.src = addr(op.src_buf, op.rank, op.chunk, op.src_off);
+        s.dst = addr(op.dst_buf, op.dst_rank, op.chunk, op.dst_off);
+        s.local = nullptr;
+      } else {
+        s.src = addr(op.src_buf, op.rank, op.chunk, op.src_off);
+        s.local = addr(op.local_buf, op.rank, op.chunk, op.local_off);
+        s.dst = addr(op.dst_buf, op.rank, op.chunk, op.dst_off);
+      }
+      rg.segs.push_back(s);
+    }
+  }
+}
+
+void fill_sum_batch(const RGroup& g, size_t first, size_t n, int dtype, size_t elem, SumBatch* b) {
+  b->nseg = (int)n;
+  b->dtype = dtype;
+  for (size_t i = 0; i < n; i++) {
+    const Seg& s = g.segs[first + i];
+    b->seg[i] = SumSeg{s.src, s.local, s.dst, (unsigned long long)(s.bytes / elem)};
+  }
+}
+void fill_copy_batch(const RGroup& g, size_t first, size_t n, CopyBatch* b) {
+  b->nseg = (int)n;
+  b->pad = 0;
+  for (size_t i = 0; i < n; i++) {
+    const Seg& s = g.segs[first + i];
+    b->seg[i] = CopySeg{s.src, s.dst, (unsigned long long)s.bytes};
+  }
+}
+
+struct Tally {
+  long moves = 0, move_launches = 0, sum_launches = 0;
+};
+
+// ------------------------------------------------------------------ stream executor -------------
+hoccl_result_t run_streams(hoccl_comm* c, const Plan& P, const std::vector<RGroup>& groups, cudaStream_t user, Tally* tally) {
+  const int lanes = (int)std::max<long>(1, std::min<long>(c->lanes, kMaxLanes));
+  c->ev_next = 0;
+  std::vector<cudaStream_t> where(groups.size(), nullptr);
+  std::vector<cudaEvent_t> done(groups.size(), nullptr);
+  std::vector<char> lane_used(lanes, 0);
+  bool sum_used = false;
+  cudaEvent_t fork = next_event(c);
+  if (!fork) return cuda_fail(c, cudaErrorMemoryAllocation, "event pool");
+  CU_TRY(c, cudaEventRecord(fork, user));
+  auto touch = [&](cudaStream_t s, char* used) -> cudaError_t {
+    if (*used) return cudaSuccess;
+    *used = 1;
+    return cudaStreamWaitEvent(s, fork, 0);
+  };
+  int move_rr = 0;
+  for (size_t g = 0; g < groups.size(); g++) {
+    const RGroup& rg = groups[g];
+    cudaStream_t s;
+    if (rg.kind == OP_SUM) {
+      s = c->sum_stream;
+      char u = sum_used ? 1 : 0;
+      CU_TRY(c, touch(s, &u));
+      sum_used = true;
+    } else {
+      int l = c->path == HOCCL_PATH_SM ? 0 : move_rr++ % lanes;   // SM copies share one lane: global CTA budget
+      s = c->lane[l];
+      CU_TRY(c, touch(s, &lane_used[l]));
+    }
+    where[g] = s;
+    for (int d : rg.deps)
+      if (where[d] != s) CU_TRY(c, cudaStreamWaitEvent(s, done[d], 0));
+    // chain_dep needs no event here: every SUM is on the one sum stream
+    if (rg.kind == OP_SUM) {
+      for (size_t first = 0; first < rg.segs.size(); first += kMaxSegs) {
+        size_t n = std::min<size_t>(kMaxSegs, rg.segs.size() - first);
+        SumBatch b;
+        fill_sum_batch(rg, first, n, P.dtype, P.elem, &b);
+        std::pair<cudaEvent_t, cudaEvent_t> pe{nullptr, nullptr};
+        if (c->profile) {
+          if (c->prof_pool.empty()) {
+            cudaEvent_t a, z;
+            CU_TRY(c, cudaEventCreate(&a));
+            CU_TRY(c, cudaEventCreate(&z));
+            pe = {a, z};
+          } else {
+            pe = c->prof_pool.back();
+            c->prof_pool.pop_back();
+          }
+          CU_TRY(c, cudaEventRecord(pe.first, s));
+        }
+        CU_TRY(c, launch_sum(b, (int)c->sum_ctas, s));
+        if (c->profile) {
+          CU_TRY(c, cudaEventRecord(pe.second, s));
+          double bytes = 0;
+          for (size_t i = 0; i < n; i++) bytes += 3.0 * (double)rg.segs[first + i].bytes;
+          c->prof_open.push_back({pe, bytes});
+        }
+        tally->sum_launches++;
+      }
+    } else if (c->path == HOCCL_PATH_CE) {
+      for (const Seg& sg : rg.segs) {
+        CU_TRY(c, cudaMemcpyAsync(sg.dst, sg.src, sg.bytes, cudaMemcpyDeviceToDevice, s));
+        tally->moves++;
+      }
+    } else {
+      for (size_t first = 0; first < rg.segs.size(); first += kMaxSegs) {
+        size_t n = std::min<size_t>(kMaxSegs, rg.segs.size() - first);
+        CopyBatch b;
+        fill_copy_batch(rg, first, n, &b);
+        CU_TRY(c, launch_copy(b, (int)c->copy_ctas, s));
+        tally->moves += (long)n;
+        tally->move_launches++;
+      }
+    }
+    cudaEvent_t ev = next_event(c);
+    if (!ev) return cuda_fail(c, cudaErrorMemoryAllocation, "event pool");
+    CU_TRY(c, cudaEventRecord(ev, s));
+    done[g] = ev;
+  }
+  // join: the caller's stream waits for every internal stream that was used
+  for (int l = 0; l < lanes; l++)
+    if (lane_used[l]) {
+      cudaEvent_t ev = next_event(c);
+      if (!ev) return cuda_fail(c, cudaErrorMemoryAllocation, "event pool");
+      CU_TRY(c, cudaEventRecord(ev, c->lane[l]));
+      CU_TRY(c, cudaStreamWaitEvent(user, ev, 0));
+    }
+  if (sum_used) {
+    cudaEvent_t ev = next_event(c);
+    if (!ev) return cuda_fail(c, cudaErrorMemoryAllocation, "event pool");
+    CU_TRY(c, cudaEventRecord(ev, c->sum_stream));
+    CU_TRY(c, cudaStreamWaitEvent(user, ev, 0));
+  }
+  return HOCCL_OK;
+}
+
+// ------------------------------------------------------------------ graph executor --------------
+void destroy_entry(GraphEntry* e) {
+  if (e->exec) cudaGraphExecDestroy(e->exec);
+  for (auto& p : e->prof_events) {
+    cudaEventDestroy(p.first);
+    cudaEventDestroy(p.second);
+  }
+  e->exec = nullptr;
+  e->prof_events.clear();
+}
+
+hoccl_result_t build_graph(hoccl_comm* c, const Plan& P, const std::vector<RGroup>& groups, GraphEntry* entry) {
+  cudaGraph_t g = nullptr;
+  CU_TRY(c, cudaGraphCreate(&g, 0));
+  std::vector<cudaGraphNode_t> tail(groups.size(), nullptr);
+  cudaGraphNode_t last_copy_node = nullptr;
+  hoccl_result_t rc = HOCCL_OK;
+  auto fail = [&](cudaError_t e, const char* what) {
+    rc = cuda_fail(c, e, what);
+  };
+  for (size_t gi = 0; gi < groups.size() && rc == HOCCL_OK; gi++) {
+    const RGroup& rg = groups[gi];
+    std::vector<cudaGraphNode_t> deps;
+    for (int d : rg.deps)
+      if (tail[d]) deps.push_back(tail[d]);
+    if (rg.chain_dep >= 0 && tail[rg.chain_dep] && std::find(rg.deps.begin(), rg.deps.end(), rg.chain_dep) == rg.deps.end())
+      deps.push_back(tail[rg.chain_dep]);
+    std::vector<cudaGraphNode_t> nodes;
+    cudaError_t e = cudaSuccess;
+    if (rg.kind == OP_SUM) {
+      for (size_t first = 0; first < rg.segs.size() && e == cudaSuccess; first += kMaxSegs) {
+        size_t n = std::min<size_t>(kMaxSegs, rg.segs.size() - first);
+        SumBatch b;
+        fill_sum_batch(rg, first, n, P.dtype, P.elem, &b);
+        void* args[] = {&b};
+        cudaKernelNodeParams kp = {};
+        int sum_threads = 0;
+        kp.func = const_cast<void*>(sum_kernel_entry(P.dtype, (int)c->sum_ctas, &sum_threads));
+        kp.gridDim = dim3((unsigned)c->sum_ctas);
+        kp.blockDim = dim3((unsigned)sum_threads);
+        kp.kernelParams = args;
+        // launches of one group are chained too (they share the SM budget)
+        std::vector<cudaGraphNode_t> d2 = nodes.empty() ? deps : std::vector<cudaGraphNode_t>{nodes.back()};
+        cudaGraphNode_t start_rec = nullptr;
+        std::pair<cudaEvent_t, cudaEvent_t> pe{nullptr, nullptr};
+        if (c->profile) {
+          if ((e = cudaEventCreate(&pe.first)) != cudaSuccess) break;
+          if ((e = cudaEventCreate(&pe.second)) != cudaSuccess) break;
+          entry->prof_events.push_back(pe);
+          double bytes = 0;
+          for (size_t i = 0; i < n; i++) bytes += 3.0 * (double)rg.segs[first + i].bytes;
+          entry->prof_bytes.push_back(bytes);
+          if ((e = cudaGraphAddEventRecordNode(&start_rec, g, d2.data(), d2.size(), pe.first)) != cudaSuccess) break;
+          d2.assign(1, start_rec);
+        }
+        cudaGraphNode_t kn;
+        e = cudaGraphAddKernelNode(&kn, g, d2.data(), d2.size(), &kp);
+        if (e != cudaSuccess) break;
+        cudaLaunchAttributeValue prio = {};
+        prio.priority = c->sum_priority;
+        e = cudaGraphKernelNodeSetAttribute(kn, cudaLaunchAttributePriority, &prio);
+        if (e != cudaSuccess) break;
+        if (c->profile) {
+          cudaGraphNode_t end_rec;
+          if ((e = cudaGraphAddEventRecordNode(&end_rec, g, &kn, 1, pe.second)) != cudaSuccess) break;
+          kn = end_rec;
+        }
+        nodes.assign(1, kn);
+        entry->n_sum_launches++;
+      }
+    } else if (c->path == HOCCL_PATH_CE) {
+      for (const Seg& sg : rg.segs) {
+        // optional sub-copies: driver copies of 4-8 MiB pay a ~4 us serialised start-up that smaller ones do not
+        size_t sub = sg.bytes;
+        if (c->ce_sub_bytes > 0 && sg.bytes > (size_t)c->ce_sub_bytes && sg.bytes < ((size_t)16 << 20))
+          sub = ((size_t)c->ce_sub_bytes + 255) / 256 * 256;
+        for (size_t off = 0; off < sg.bytes && e == cudaSuccess; off += sub) {
+          cudaGraphNode_t n;
+          e = cudaGraphAddMemcpyNode1D(&n, g, deps.data(), deps.size(), sg.dst + off, sg.src + off, std::min(sub, sg.bytes - off),
+                                       cudaMemcpyDeviceToDevice);
+          if (e != cudaSuccess) break;
+          nodes.push_back(n);
+          entry->n_moves++;
+        }
+        if (e != cudaSuccess) break;
+      }
+    } else {
+      for (size_t first = 0; first < rg.segs.size() && e == cudaSuccess; first += kMaxSegs) {
+        size_t n = std::min<size_t>(kMaxSegs, rg.segs.size() - first);
+        CopyBatch b;
+        fill_copy_batch(rg, first, n, &b);
+        void* args[] = {&b};
+        cudaKernelNodeParams kp = {};
+        int copy_threads = 0;
+        kp.func = const_cast<void*>(copy_kernel_entry((int)c->copy_ctas, &copy_threads));
+        kp.gridDim = dim3((unsigned)c->copy_ctas);
+        kp.blockDim = dim3((unsigned)copy_threads);
+        kp.kernelParams = args;
+        // copy launches are chained as well: the CTA budget for copies is global, two never run at the same time
+        std::vector<cudaGraphNode_t> d2 = deps;
+        if (last_copy_node && std::find(d2.begin(), d2.end(), last_copy_node) == d2.end()) d2.push_back(last_copy_node);
+        cudaGraphNode_t kn;
+        e = cudaGraphAddKernelNode(&kn, g, d2.data(), d2.size(), &kp);
+        if (e != cudaSuccess) break;
+        last_copy_node = kn;
+        nodes.push_back(kn);
+        entry->n_moves += (long)n;
+        entry->n_move_launches++;
+      }
+    }
+    if (e != cudaSuccess) {
+      fail(e, "graph node");
+      break;
+    }
+    if (nodes.size() == 1) {
+      tail[gi] = nodes[0];
+    } else if (nodes.size() > 1) {
+      cudaGraphNode_t join;
+      e = cudaGraphAddEmptyNode(&join, g, nodes.data(), nodes.size());
+      if (e != cudaSuccess) {
+        fail(e, "graph join node");
+        break;
+      }
+      tail[gi] = join;
+    }
+  }
+  if (rc == HOCCL_OK) {
+    cudaError_t e = cudaGraphInstantiate(&entry->exec, g, 0);
+    if (e != cudaSuccess) rc = cuda_fail(c, e, "cudaGraphInstantiate");
+  }
+  cudaGraphDestroy(g);
+  if (rc != HOCCL_OK) destroy_entry(entry);
+  return rc;
+}
+
+std::vector<uint64_t> make_key(hoccl_comm* c, const Call& call) {
+  std::vector<uint64_t> k;
+  k.reserve(12 + 2 * c->R);
+  k.push_back((uint64_t)call.kind);
+  k.push_back((uint64_t)call.count);
+  k.push_back((uint64_t)call.dtype);
+  k.push_back((uint64_t)c->path);
+  k.push_back((uint64_t)c->sum_ctas);
+  k.push_back((uint64_t)c->copy_ctas);
+  k.push_back((uint64_t)c->piece_bytes);
+  k.push_back((uint64_t)c->max_pieces);
+  k.push_back((uint64_t)c->profile);
+  k.push_back((uint64_t)c->ce_sub_bytes);
+  k.push_back((uint64_t)(uintptr_t)c->scratch);
+  for (int r = 0; r < c->R; r++) {
+    k.push_back((uint64_t)(uintptr_t)call.send[r]);
+    k.push_back((uint64_t)(uintptr_t)call.recv[r]);
+  }
+  return k;
+}
+
+// reads back the profile events of finished work (the caller has synchronised)
+void harvest_profile(hoccl_comm* c) {
+  for (auto& rec : c->prof_open) {
+    float ms = 0;
+    if (cudaEventElapsedTime(&ms, rec.first.first, rec.first.second) == cudaSuccess) {
+      c->prof_ms += ms;
+      c->prof_bytes += rec.second;
+      c->prof_n++;
+    }
+    c->prof_pool.push_back(rec.first);
+  }
+  c->prof_open.clear();
+  // cached graphs keep their own events; a replay overwrites them, so only the latest replay is readable
+  for (auto& e : c->cache) {
+    if (!e.prof_pending) continue;
+    e.prof_pending = false;
+    for (size_t i = 0; i < e.prof_events.size(); i++) {
+      float ms = 0;
+      if (cudaEventElapsedTime(&ms, e.prof_events[i].first, e.prof_events[i].second) == cudaSuccess) {
+        c->prof_ms += ms;
+        c->prof_bytes += e.prof_bytes[i];
+        c->prof_n++;
+      }
+    }
+  }
+}
+
+// The CPU proxy of the handshake mode is created on first use.
+hoccl_result_t ensure_proxy(hoccl_comm* c) {
+  if (c->proxy) {
+    c->proxy->set_watchdog_ms(c->watchdog_ms);
+    return HOCCL_OK;
+  }
+  Proxy* p = new Proxy(c->device, c->watchdog_ms);
+  cudaError_t e = p->init();
+  if (e != cudaSuccess) {
+    delete p;
+    return cuda_fail(c, e, "proxy init (stream memory operations)");
+  }
+  c->proxy = p;
+  return HOCCL_OK;
+}
+
+hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
+  const double t0 = now_us();
+  if (!c) return HOCCL_ERR_INVALID_ARG;
+  if (dtype_size(call->dtype) == 0) return HOCCL_ERR_UNSUPPORTED;
+  hoccl_result_t rc = validate(c, call);
+  if (rc != HOCCL_OK) return rc;
+  c->stats = hoccl_stats_t{};
+  if (call->count == 0) return HOCCL_OK;
+  CU_TRY(c, cudaSetDevice(c->device));
+
+  if (c->onepass && !c->handshake && (call->kind == PLAN_ALLREDUCE || call->kind == PLAN_REDUCE_SCATTER)) {
+    // comparison point: the whole reduction in one kernel, same order and rounding as the ring, no moves, no scratch
+    OnePassArgs a;
+    a.R = c->R;
+    a.dtype = call->dtype;
+    a.write_all = call->kind == PLAN_ALLREDUCE ? 1 : 0;
+    a.pad = 0;
+    if (call->kind == PLAN_ALLREDUCE) {
+      a.count = call->count;
+      a.q = (call->count + (size_t)c->R - 1) / (size_t)c->R;
+    } else {
+      a.count = (unsigned long long)call->count * c->R;
+      a.q = call->count;
+    }
+    for (int r = 0; r < c->R; r++) {
+      a.x[r] = call->send[r];
+      a.y[r] = call->recv[r];
+    }
+    CU_TRY(c, launch_onepass(a, (int)c->sum_ctas, user));
+    c->stats.n_sum_launches = 1;
+    c->stats.max_sum_ctas = c->sum_ctas;
+    c->stats.n_pieces = 1;
+    c->stats.host_launch_us = now_us() - t0;
+    return HOCCL_OK;
+  }
+  Plan P;
+  unsigned char align[kMaxRanks];
+  for (int r = 0; r < c->R; r++) align[r] = (unsigned char)((uintptr_t)call->send[r] & 15);
+  if (!build_plan(&P, call->kind, c->R, call->count, call->dtype, call->in_place, (size_t)c->piece_bytes, (int)c->max_pieces, align))
+    return HOCCL_ERR_INVALID_ARG;
+  if (P.slot_bytes) {
+    size_t need = 2 * (size_t)c->R * P.slot_bytes;
+    if (!c->scratch || c->scratch_bytes < need) return HOCCL_ERR_SCRATCH;
+    // scratch must not overlap any rank buffer
+    for (int r = 0; r < c->R; r++)
+      if (ranges_overlap((const char*)c->scratch, need, (const char*)call->send[r], call->send_bytes) ||
+          ranges_overlap((const char*)c->scratch, need, (const char*)call->recv[r], call->recv_bytes))
+        return HOCCL_ERR_INVALID_ARG;
+  }
+  c->stats.n_pieces = P.pieces;
+  c->stats.max_sum_ctas = 0;
+  Tally tally;
+  if (c->handshake) {
+    // Driver copies share a hardware queue with the copies the parked stream has queued behind its hand-over; a copy
+    // issued by the proxy can end up behind them and never start (observed).  Kernels do not have that problem.
+    if (c->path == HOCCL_PATH_CE) return HOCCL_ERR_UNSUPPORTED;
+    rc = ensure_proxy(c);
+    if (rc != HOCCL_OK) return rc;
+  }
+  if (c->use_graph || c->handshake) {
+    std::vector<uint64_t> key = make_key(c, *call);
+    GraphEntry* hit = nullptr;
+    for (auto& e : c->cache)
+      if (e.key == key) {
+        hit = &e;
+        break;
+      }
+    c->stats.graph_hit = hit ? 1 : 0;
+    if (!hit) {
+      std::vector<RGroup> groups;
+      resolve(c, P, *call, &groups);
+      GraphEntry entry;
+      entry.key = key;
+      entry.n_pieces = P.pieces;
+      rc = build_graph(c, P, groups, &entry);
+      if (rc != HOCCL_OK) return rc;
+      // handshake mode: place the graph on the device now; the proxy must not meet first-launch work later
+      if (c->handshake) CU_TRY(c, cudaGraphUpload(entry.exec, c->proxy->work_stream()));
+      if (c->cache.size() >= kGraphCacheCap) {
+        if (c->proxy) c->proxy->drain(c->watchdog_ms);  // a queued hand-over may still refer to the victim
+        size_t victim = 0;
+        for (size_t i = 1; i < c->cache.size(); i++)
+          if (c->cache[i].last_use < c->cache[victim].last_use) victim = i;
+        destroy_entry(&c->cache[victim]);
+        c->cache.erase(c->cache.begin() + victim);
+      }
+      c->cache.push_back(std::move(entry));
+      hit = &c->cache.back();
+    }
+    hit->last_use = ++c->use_counter;
+    if (c->handshake) {
+      // paper Sec. 3.2: the stream hands itself to the CPU proxy, which runs the schedule and hands it back
+      ProxyTask t;
+      t.kind = ProxyTask::GRAPH;
+      t.exec = hit->exec;
+      CU_TRY(c, c->proxy->submit(user, t));
+    } else {
+      CU_TRY(c, cudaGraphLaunch(hit->exec, user));
+    }
+    hit->prof_pending = !hit->prof_events.empty();
+    tally.moves = hit->n_moves;
+    tally.move_launches = hit->n_move_launches;
+    tally.sum_launches = hit->n_sum_launches;
+  } else {
+    std::vector<RGroup> groups;
+    resolve(c, P, *call, &groups);
+    rc = run_streams(c, P, groups, user, &tally);
+    if (rc != HOCCL_OK) return rc;
+  }
+  c->stats.n_moves = tally.moves;
+  c->stats.n_move_launches = tally.move_launches;
+  c->stats.n_sum_launches = tally.sum_launches;
+  c->stats.max_sum_ctas = tally.sum_launches ? c->sum_ctas : 0;
+  c->stats.max_copy_ctas = tally.move_launches ? c->copy_ctas : 0;
+  c->stats.host_launch_us = now_us() - t0;
+  return HOCCL_OK;
+}
+
+}  // namespace hoccl
