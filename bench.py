@@ -430,6 +430,14 @@ def extras(hb, W, torch, np, new_comm, step, timed, stream, R, S, n, dtype, peak
                         "bytes_per_step": 2.0 * R * S, "GBps": 2.0 * R * S / t / 1e9})
         c1.destroy()
     out["onepass_allreduce"] = op_rows
+    # second comparison point: fused sum-and-forward (a SUM stores into the next rank's inbox; moves only at step 0)
+    fw_rows = []
+    for name, path, sc, cc in (("CE", hb.PATH_CE, 8, 8), ("SM", hb.PATH_SM, 148, 148)):
+        c1 = new_comm(path, sum_ctas=sc, copy_ctas=cc, forward=1)
+        t, _ = timed(c1, k, w)
+        fw_rows.append({"path": name, "sum_ctas": sc, "ms_per_step": t * 1e3, "busbw_GBps": S * bus_factor(R) / t / 1e9})
+        c1.destroy()
+    out["forward_variant"] = fw_rows
     # handshake mode (CPU proxy + stream memory operations) on the SM path, against the same path launched directly
     hs = {}
     for label, flag in (("direct", 0), ("handshake", 1)):

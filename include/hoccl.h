@@ -130,6 +130,10 @@ hoccl_result_t hoccl_comm_set_path(hoccl_comm_t comm, hoccl_path_t path);
  *                + R (or 1) writes per element instead of 7(R-1) bytes per wire byte, no moves, no scratch.  It is not
  *                rank local (one kernel reads every rank's buffer), so it only makes sense on one device and is kept
  *                as the comparison point that shows what the rank-local schedule costs.  0 = off (default).
+ *  "forward"     1 = fused sum-and-forward variant of the ring reduce-scatter: the SUM of step s writes its result
+ *                straight into the next rank's inbox, so only step 0 needs moves (3 instead of 5 bytes of traffic per
+ *                wire byte in that phase).  Same bits.  A SUM then stores into another rank's memory, as SM-driven
+ *                libraries do: it is the second comparison point for what rank locality costs.  0 = off (default).
  *  "use_graph"   1 = run a cached CUDA graph built from the plan (default), 0 = streams and events
  *  "handshake"   1 = the paper's stream manager (Sec. 3.2, Listing 1): instead of launching into the caller's
  *                stream, the call enqueues four stream memory operations (write start flag, wait for the CPU's
@@ -328,7 +332,8 @@ hoccl_result_t hoccl_copy_launch(const void* src, void* dst, size_t bytes, int c
  * checked without a GPU.  Addresses in a plan are byte offsets: buffer kinds below say what they are
  * relative to.
  */
-typedef enum { HOCCL_PLAN_ALLREDUCE = 0, HOCCL_PLAN_REDUCE_SCATTER = 1, HOCCL_PLAN_ALLGATHER = 2, HOCCL_PLAN_ALLTOALL = 3 } hoccl_plan_kind_t;
+typedef enum { HOCCL_PLAN_ALLREDUCE = 0, HOCCL_PLAN_REDUCE_SCATTER = 1, HOCCL_PLAN_ALLGATHER = 2, HOCCL_PLAN_ALLTOALL = 3,
+               HOCCL_PLAN_ALLREDUCE_FWD = 4, HOCCL_PLAN_REDUCE_SCATTER_FWD = 5 /* the "forward" variants */ } hoccl_plan_kind_t;
 typedef enum { HOCCL_OP_MOVE = 0, HOCCL_OP_SUM = 1 } hoccl_plan_op_kind_t;
 typedef enum { HOCCL_BUF_SEND = 0, HOCCL_BUF_RECV = 1, HOCCL_BUF_INBOX = 2, HOCCL_BUF_PARTIAL = 3 } hoccl_buf_kind_t;
 
@@ -338,7 +343,7 @@ typedef struct {
   int step;      /* ring step s (all-to-all: stage k, destination = rank + k) */
   int piece;     /* pipeline piece index */
   int rank;      /* MOVE: source rank; SUM: the rank that sums */
-  int dst_rank;  /* MOVE: destination rank; SUM: same as rank */
+  int dst_rank;  /* MOVE: destination rank; SUM: same as rank (forward variants: the rank whose slot receives the result) */
   int chunk;     /* ring chunk index */
   int src_buf, dst_buf, local_buf; /* hoccl_buf_kind_t; local_buf only for SUM */
   uint64_t src_off, dst_off, local_off; /* byte offsets from the start of those buffers (scratch: from the start of the rank's slot) */

@@ -16,7 +16,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_MISMATCH, ERR_PENDING, ERR_S
 FLOAT32, BFLOAT16 = 0, 1
 SUM = 0
 PATH_CE, PATH_SM = 0, 1
-PLAN_ALLREDUCE, PLAN_REDUCE_SCATTER, PLAN_ALLGATHER, PLAN_ALLTOALL = 0, 1, 2, 3
+PLAN_ALLREDUCE, PLAN_REDUCE_SCATTER, PLAN_ALLGATHER, PLAN_ALLTOALL, PLAN_ALLREDUCE_FWD, PLAN_REDUCE_SCATTER_FWD = range(6)
 OP_MOVE, OP_SUM = 0, 1
 BUF_SEND, BUF_RECV, BUF_INBOX, BUF_PARTIAL = 0, 1, 2, 3
 

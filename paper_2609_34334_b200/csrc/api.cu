@@ -107,7 +107,8 @@ static long* param_slot(hoccl_comm* c, const char* key, long* lo, long* hi) {
               {"lanes", &c->lanes, 1, kMaxLanes},       {"use_graph", &c->use_graph, 0, 1},
               {"profile", &c->profile, 0, 1},           {"p2p_split", &c->p2p_split, 1, kMaxLanes},
               {"ce_sub_bytes", &c->ce_sub_bytes, 0, 1L << 40}, {"handshake", &c->handshake, 0, 1},
-              {"watchdog_ms", &c->watchdog_ms, 10, 600000},    {"onepass", &c->onepass, 0, 1}};
+              {"watchdog_ms", &c->watchdog_ms, 10, 600000},    {"onepass", &c->onepass, 0, 1},
+              {"forward", &c->forward, 0, 1}};
   for (auto& r : rows)
     if (std::strcmp(r.name, key) == 0) {
       *lo = r.lo;

@@ -83,7 +83,7 @@ void resolve(hoccl_comm* c, const Plan& P, const Call& call, std::vector<RGroup>
       } else {
         s.src = addr(op.src_buf, op.rank, op.chunk, op.src_off);
         s.local = addr(op.local_buf, op.rank, op.chunk, op.local_off);
-        s.dst = addr(op.dst_buf, op.rank, op.chunk, op.dst_off);
+        s.dst = addr(op.dst_buf, op.dst_rank, op.chunk, op.dst_off);  // dst_rank == rank except in the forward variant
       }
       rg.segs.push_back(s);
     }
@@ -357,6 +357,7 @@ std::vector<uint64_t> make_key(hoccl_comm* c, const Call& call) {
   k.push_back((uint64_t)c->max_pieces);
   k.push_back((uint64_t)c->profile);
   k.push_back((uint64_t)c->ce_sub_bytes);
+  k.push_back((uint64_t)c->forward);
   k.push_back((uint64_t)(uintptr_t)c->scratch);
   for (int r = 0; r < c->R; r++) {
     k.push_back((uint64_t)(uintptr_t)call.send[r]);
@@ -446,7 +447,10 @@ hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
   Plan P;
   unsigned char align[kMaxRanks];
   for (int r = 0; r < c->R; r++) align[r] = (unsigned char)((uintptr_t)call->send[r] & 15);
-  if (!build_plan(&P, call->kind, c->R, call->count, call->dtype, call->in_place, (size_t)c->piece_bytes, (int)c->max_pieces, align))
+  int plan_kind = call->kind;
+  if (c->forward && call->kind == PLAN_ALLREDUCE) plan_kind = PLAN_ALLREDUCE_FWD;
+  if (c->forward && call->kind == PLAN_REDUCE_SCATTER) plan_kind = PLAN_REDUCE_SCATTER_FWD;
+  if (!build_plan(&P, plan_kind, c->R, call->count, call->dtype, call->in_place, (size_t)c->piece_bytes, (int)c->max_pieces, align))
     return HOCCL_ERR_INVALID_ARG;
   if (P.slot_bytes) {
     size_t need = 2 * (size_t)c->R * P.slot_bytes;

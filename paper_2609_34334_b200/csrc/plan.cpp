@@ -83,13 +83,17 @@ void piece_span(const Plan& P, size_t len_bytes, int p, size_t* off, size_t* len
 bool build_plan(Plan* plan, int kind, int R, size_t count, int dtype, bool in_place, size_t piece_bytes, int max_pieces,
                 const unsigned char* send_align) {
   size_t e = dtype_size(dtype);
-  if (!plan || R < 1 || e == 0 || kind < PLAN_ALLREDUCE || kind > PLAN_ALLTOALL) return false;
+  if (!plan || R < 1 || e == 0 || kind < PLAN_ALLREDUCE || kind > PLAN_REDUCE_SCATTER_FWD) return false;
+  const bool forward = (kind == PLAN_ALLREDUCE_FWD || kind == PLAN_REDUCE_SCATTER_FWD);
+  if (kind == PLAN_ALLREDUCE_FWD) kind = PLAN_ALLREDUCE;
+  if (kind == PLAN_REDUCE_SCATTER_FWD) kind = PLAN_REDUCE_SCATTER;
   if (kind == PLAN_ALLTOALL && in_place) return false;  // an in-place exchange would need a staging copy of every block
   if (max_pieces < 1) max_pieces = 1;
   if (piece_bytes < 1024) piece_bytes = 1024;
   Plan& P = *plan;
   P = Plan();
   P.kind = kind;
+  P.forward = forward;
   P.R = R;
   P.dtype = dtype;
   P.count = count;
@@ -171,9 +175,12 @@ bool build_plan(Plan* plan, int kind, int R, size_t count, int dtype, bool in_pl
   if (kind != PLAN_ALLGATHER) {
     for (int s = 0; s <= R - 2; s++) {
       for (int p = 0; p < np_i; p++) {
-        // ---- MOVE(s, r, p): chunk c = (r-1-s) mod R leaves rank r for the inbox of rank r+1
+        // ---- MOVE(s, r, p): chunk c = (r-1-s) mod R leaves rank r for the inbox of rank r+1.
+        // Forward variant: only step 0 moves; afterwards SUM(s-1) has already written into the next rank's slot.  The
+        // two scratch slots of a rank then alternate as inbox (even steps: INBOX, odd steps: PARTIAL), because a SUM
+        // launch reads every rank's current inbox while it writes every rank's next one.
         int gm = B.begin_group(OP_MOVE, PHASE_RS, s, p);
-        for (int r = 0; r < R; r++) {
+        for (int r = 0; r < R && !(forward && s > 0); r++) {
           int c = mod(r - 1 - s, R);
           size_t lo, hi, off, len;
           P.chunk_range(c, &lo, &hi);
@@ -195,11 +202,20 @@ bool build_plan(Plan* plan, int kind, int R, size_t count, int dtype, bool in_pl
           uint64_t out_off = last ? ((kind == PLAN_ALLREDUCE ? lo * e : 0) + off) : slot_off(r, c, p);
           PlanOp op{OP_SUM, PHASE_RS, s, p, r, r, c, BUF_INBOX, last ? BUF_RECV : BUF_PARTIAL, BUF_SEND,
                     slot_off(r, c, p), out_off, lo * e + off, len, 0};
+          if (forward) {
+            op.src_buf = (s % 2 == 0) ? BUF_INBOX : BUF_PARTIAL;
+            if (!last) {
+              op.dst_rank = (r + 1) % R;
+              op.dst_buf = ((s + 1) % 2 == 0) ? BUF_INBOX : BUF_PARTIAL;
+              op.dst_off = slot_off((r + 1) % R, c, p);
+            }
+          }
           B.add(op);
         }
         gs = B.end_group();
         if (gs >= 0) {
           if (gm >= 0) P.groups[gs].deps.push_back(gm);
+          if (forward && s > 0 && last_sum[p] >= 0) P.groups[gs].deps.push_back(last_sum[p]);
           P.groups[gs].chain_dep = prev_sum_group;
           prev_sum_group = gs;
           last_sum[p] = gs;

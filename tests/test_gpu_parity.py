@@ -319,6 +319,35 @@ def test_onepass_reduction_gives_the_ring_bits(oracle, dtype):
             comm.destroy()
 
 
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("path", [hb.PATH_CE, hb.PATH_SM])
+def test_forward_variant_gives_the_ring_bits(oracle, dtype, path):
+    """Fused sum-and-forward (a SUM stores into the next rank's inbox): same bits as the rank-local ring."""
+    e = W.elem_size(dtype)
+    for R, n in SMALL + [(8, 8 * 65_536)]:
+        xs = W.rank_inputs("normal", 400 + n % 7, R, n, dtype, 1.0)
+        want = oracle.ring_allreduce(xs)
+        for use_graph in (1, 0):
+            comm = make_comm(R, n, dtype, path, forward=1, use_graph=use_graph, piece_bytes=8192, max_pieces=3)
+            for in_place in (False, True):
+                got = run_allreduce(comm, xs, dtype, in_place)
+                for r in range(R):
+                    assert same_bits(got[r], want[r], dtype), (R, n, r, in_place, use_graph)
+            if R > 1:
+                st = comm.last_stats()
+                assert st["n_moves"] <= 2 * R * st["n_pieces"] * (R - 1)      # fewer moves than the rank-local ring
+            if n % R == 0 and R > 1:
+                count = n // R
+                wrs = oracle.ring_reduce_scatter(xs)
+                send = [DevBuf(n * e).put(xs[r]) for r in range(R)]
+                recv = [DevBuf(count * e) for _ in range(R)]
+                comm.reduce_scatter(send, recv, count, dtype)
+                torch.cuda.synchronize()
+                for r in range(R):
+                    assert same_bits(recv[r].get(np_dtype(dtype)), wrs[r], dtype) and recv[r].guards_intact()
+            comm.destroy()
+
+
 def test_settings_never_change_a_bit(oracle):
     """Piece size, lane count, CTA budgets, path and executor are pure scheduling choices."""
     R, n, dtype = 8, 8 * 40000 + 8, "bf16"
@@ -331,6 +360,9 @@ def test_settings_never_change_a_bit(oracle):
         dict(path=hb.PATH_SM, use_graph=1, piece_bytes=1 << 20, max_pieces=1, sum_ctas=148, copy_ctas=148),
         dict(path=hb.PATH_SM, use_graph=0, piece_bytes=16384, max_pieces=3, sum_ctas=3, copy_ctas=5),
         dict(path=hb.PATH_CE, use_graph=1, profile=1),
+        dict(path=hb.PATH_CE, use_graph=1, forward=1, piece_bytes=4096, max_pieces=16),
+        dict(path=hb.PATH_SM, use_graph=0, forward=1, piece_bytes=65536, max_pieces=4, lanes=2),
+        dict(path=hb.PATH_CE, onepass=1, sum_ctas=5),
     ]
     for s in settings:
         s = dict(s)

@@ -40,6 +40,8 @@ def _topo_order(num_groups, deps, rng):
 def _run_plan(plan, kind, R, count, dtype, xs, in_place, rng):
     e = W.elem_size(dtype)
     npdt = np.float32 if dtype == "fp32" else np.uint16
+    base = {hb.PLAN_ALLREDUCE_FWD: hb.PLAN_ALLREDUCE, hb.PLAN_REDUCE_SCATTER_FWD: hb.PLAN_REDUCE_SCATTER}.get(kind, kind)
+    kind = base
     if kind == hb.PLAN_ALLREDUCE:
         send_n, recv_n = count, count
     elif kind == hb.PLAN_ALLTOALL:
@@ -85,7 +87,7 @@ def _run_plan(plan, kind, R, count, dtype, xs, in_place, rng):
             else:
                 assert dtype == "fp32"
                 loc = bufs[op["local_buf"]][op["rank"]][op["local_off"]:op["local_off"] + n]
-                out = bufs[op["dst_buf"]][op["rank"]]
+                out = bufs[op["dst_buf"]][op["dst_rank"]]
                 assert op["dst_off"] + n <= out.size
                 res = (src.view(np.float32) + loc.view(np.float32)).view(np.uint8)
                 out[op["dst_off"]:op["dst_off"] + n] = res
@@ -235,3 +237,28 @@ def test_alltoall_plan(oracle, R, count):
             assert (got[r] == want[r]).all()
     with pytest.raises(hb.HocclError):
         hb.Plan(hb.PLAN_ALLTOALL, R, count, "fp32", True, 1024, 8)      # no in-place form
+
+
+@pytest.mark.parametrize("R,n,piece_bytes,max_pieces", [c for c in CASES if c[0] > 1 and c[1] > 0])
+def test_forward_variant_plans_execute_to_oracle_bits(oracle, R, n, piece_bytes, max_pieces):
+    """Fused sum-and-forward: no moves after step 0, a SUM stores into the next rank's other slot; same bits."""
+    rng = random.Random(R * 999 + n)
+    xs = W.rank_inputs("uniform", 19, R, n, "fp32")
+    want = oracle.ring_allreduce(xs)
+    for in_place in (False, True):
+        plan = hb.Plan(hb.PLAN_ALLREDUCE_FWD, R, n, "fp32", in_place, piece_bytes, max_pieces)
+        rs_moves = [op for op in plan.ops if op["kind"] == hb.OP_MOVE and op["phase"] == 0]
+        assert all(op["step"] == 0 for op in rs_moves)
+        for op in plan.ops:
+            if op["kind"] == hb.OP_SUM and op["step"] < R - 2:
+                assert op["dst_rank"] == (op["rank"] + 1) % R and op["dst_buf"] != op["src_buf"]
+        for trial in range(2):
+            got = _run_plan(plan, hb.PLAN_ALLREDUCE_FWD, R, n, "fp32", xs, in_place, rng)
+            for r in range(R):
+                assert (got[r].view(np.uint32) == want[r].view(np.uint32)).all(), (R, n, in_place, r)
+    if n % R == 0:
+        wrs = oracle.ring_reduce_scatter(xs)
+        plan = hb.Plan(hb.PLAN_REDUCE_SCATTER_FWD, R, n // R, "fp32", False, piece_bytes, max_pieces)
+        got = _run_plan(plan, hb.PLAN_REDUCE_SCATTER_FWD, R, n // R, "fp32", xs, False, rng)
+        for r in range(R):
+            assert (got[r].view(np.uint32) == wrs[r].view(np.uint32)).all()
