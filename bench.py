@@ -329,7 +329,7 @@ def main():
         "peaks": peaks,
     }
 
-    if world.rank == 0 and world.size == 1:
+    if world.rank == 0:
         # ---- roofline of the dominant kernel (the only kernel of this path): SUM, timed per launch with CUDA events
         prof = new_comm(hb.PATH_CE, sum_ctas=8, profile=1)
         for k in range(3):
@@ -377,6 +377,7 @@ def main():
             "best_frac_of_measured": max(full.values()) / peaks["hbm_gbs"]}
         del a, b2, o
 
+    if world.rank == 0 and world.size == 1:
         # ---- CPU baseline: the oracle on the host cores, whole bucket, a few repetitions
         thr = oracle_ring.max_threads()
         reps, t0 = 0, time.perf_counter()
