@@ -355,6 +355,13 @@ def main():
                     "not HBM; roofline_unconstrained is the same kernel on the whole GPU",
         }
         prof.destroy()
+        # SM footprint of this library's kernels per step (SMs x busy time) and the paper's contention rate (Eq. 1) with
+        # compute taken as active for the whole step: I = sum over kernels of CTAs x duration / (N_SM x step time)
+        n_sm = torch.cuda.get_device_properties(dev).multi_processor_count
+        sum_us_per_step = avg_ms * 1e3 * rs_stats["n_sum_launches"]
+        line["sms_used"].update({"sum_launches_per_step": int(rs_stats["n_sum_launches"]), "sum_busy_us_per_step": sum_us_per_step,
+                                 "footprint_sm_us_per_step": 8 * sum_us_per_step, "n_sm": n_sm,
+                                 "contention_rate_of_sums": 8 * sum_us_per_step / (n_sm * t_step * 1e6)})
         # the same kernel without the SM budget, timed alone on 256 MiB operands (kernel quality, not the path)
         big = 128 << 20
         a = torch.empty(big, dtype=torch.bfloat16, device="cuda").normal_(0, 1e-3)

@@ -26,8 +26,10 @@
  *  - Buffers of different ranks must not overlap.  In place is legal: allreduce with
  *    send[r] == recv[r]; reduce_scatter with recv[r] == send[r] + r*count; allgather with
  *    send[r] == recv[r] + r*count (element offsets).
- *  - One host thread per communicator.  The library never allocates device memory: scratch and
- *    staging are caller-owned and attached with hoccl_comm_set_scratch / hoccl_comm_set_staging.
+ *  - One host thread per communicator.  Device memory is the caller's: scratch and staging are
+ *    attached with hoccl_comm_set_scratch / hoccl_comm_set_staging.  The two exceptions are stated where
+ *    they apply: handshake mode allocates 512 bytes once, and hoccl_allreduce_static uses a fixed array
+ *    that is part of the library image.
  *  - The CUDA device must be present: every entry point that touches the device returns
  *    HOCCL_ERR_CUDA otherwise.  There is no CPU fallback.
  */
