@@ -392,9 +392,13 @@ def main():
             oracle_ring.ring_allreduce(xs, threads=thr)
             reps += 1
         t_cpu = (time.perf_counter() - t0) / reps
+        t1 = time.perf_counter()
+        oracle_ring.ring_allreduce(xs, threads=1)          # the canonical single-thread run (the parity reference)
+        t_single = time.perf_counter() - t1
         line["cpu_baseline"] = {"value": S * bus_factor(R) / t_cpu / 1e9, "unit": "GB/s", "cores": thr, "kind": "oracle",
                                 "sample": "%d repetitions of the whole bucket (all %d elements per rank)" % (reps, n),
-                                "ms_per_step": t_cpu * 1e3}
+                                "ms_per_step": t_cpu * 1e3, "single_thread_value": S * bus_factor(R) / t_single / 1e9,
+                                "single_thread_ms_per_step": t_single * 1e3}
 
         if not args.no_extras:
             line["extras"] = extras(hb, W, torch, np, new_comm, step, timed, stream, R, S, n, dtype, peaks, send_sets, recv_sets)
