@@ -127,6 +127,37 @@ def test_allreduce_small_and_ragged(oracle, dtype, path, use_graph):
         assert comm.destroy() == hb.OK
 
 
+@pytest.mark.parametrize("R", [16, 33, 64])
+def test_many_ranks_split_a_step_over_several_launches(oracle, R):
+    """More than 32 ranks: the segments of one ring step no longer fit one batched launch."""
+    for dtype, n in (("bf16", R * 1000 + 5), ("fp32", R * 257)):
+        xs = W.rank_inputs("uniform", 500 + R, R, n, dtype)
+        want = oracle.ring_allreduce(xs)
+        for path in (hb.PATH_CE, hb.PATH_SM):
+            for use_graph in (1, 0):
+                comm = make_comm(R, n, dtype, path, use_graph=use_graph, piece_bytes=2048, max_pieces=2)
+                got = run_allreduce(comm, xs, dtype)
+                for r in range(R):
+                    assert same_bits(got[r], want[r], dtype), (R, dtype, path, use_graph, r)
+                comm.destroy()
+        comm = make_comm(R, n, dtype, hb.PATH_CE, onepass=1)
+        got = run_allreduce(comm, xs, dtype)
+        assert all(same_bits(got[r], want[r], dtype) for r in range(R))
+        comm.destroy()
+        count = 100
+        ys = W.rank_inputs("uniform", 600 + R, R, R * count, dtype)
+        wa = oracle.alltoall(ys)
+        comm = hb.Comm(R, 0)
+        e = W.elem_size(dtype)
+        send = [DevBuf(R * count * e).put(ys[r]) for r in range(R)]
+        recv = [DevBuf(R * count * e) for _ in range(R)]
+        comm.alltoall(send, recv, count, dtype)
+        torch.cuda.synchronize()
+        for r in range(R):
+            assert (recv[r].get(np_dtype(dtype)).view(np.uint8) == wa[r].view(np.uint8)).all()
+        comm.destroy()
+
+
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
 def test_allreduce_unaligned_rank_buffers(oracle, dtype):
     e = W.elem_size(dtype)
