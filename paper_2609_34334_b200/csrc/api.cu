@@ -124,7 +124,10 @@ hoccl_result_t hoccl_comm_set_param(hoccl_comm_t c, const char* key, long value)
   long* p = param_slot(c, key, &lo, &hi);
   if (!p) return HOCCL_ERR_UNSUPPORTED;
   if (value < lo || value > hi) return HOCCL_ERR_INVALID_ARG;
-  if (std::strcmp(key, "piece_bytes") == 0) value = (value + 1023) / 1024 * 1024;
+  if (std::strcmp(key, "piece_bytes") == 0) {
+    value = (value + 1023) / 1024 * 1024;
+    c->piece_bytes_set = true;
+  }
   *p = value;
   return HOCCL_OK;
 }

@@ -354,6 +354,7 @@ std::vector<uint64_t> make_key(hoccl_comm* c, const Call& call) {
   k.push_back((uint64_t)c->sum_ctas);
   k.push_back((uint64_t)c->copy_ctas);
   k.push_back((uint64_t)c->piece_bytes);
+  k.push_back((uint64_t)c->piece_bytes_set);
   k.push_back((uint64_t)c->max_pieces);
   k.push_back((uint64_t)c->profile);
   k.push_back((uint64_t)c->ce_sub_bytes);
@@ -450,7 +451,17 @@ hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
   int plan_kind = call->kind;
   if (c->forward && call->kind == PLAN_ALLREDUCE) plan_kind = PLAN_ALLREDUCE_FWD;
   if (c->forward && call->kind == PLAN_REDUCE_SCATTER) plan_kind = PLAN_REDUCE_SCATTER_FWD;
-  if (!build_plan(&P, plan_kind, c->R, call->count, call->dtype, call->in_place, (size_t)c->piece_bytes, (int)c->max_pieces, align))
+  // Piece size: the caller's, else 4 MiB; on the SM path under CTA budgets a reduction is cut into at least two pieces
+  // (the copy kernel of one piece then overlaps the sum kernel of the other: measured 1.6x on a 3 MiB chunk with 8 + 8
+  // CTAs), which does not pay with driver copies or whole-GPU grids.
+  size_t piece_bytes = (size_t)c->piece_bytes;
+  if (!c->piece_bytes_set && c->path == HOCCL_PATH_SM && std::max(c->sum_ctas, c->copy_ctas) < 64 &&
+      (call->kind == PLAN_ALLREDUCE || call->kind == PLAN_REDUCE_SCATTER)) {
+    const size_t q = call->kind == PLAN_ALLREDUCE ? (call->count + c->R - 1) / c->R : call->count;
+    const size_t chunk = q * dtype_size(call->dtype);
+    if (chunk >= ((size_t)1 << 20)) piece_bytes = std::min(piece_bytes, (chunk / 2 + 1023) / 1024 * 1024);
+  }
+  if (!build_plan(&P, plan_kind, c->R, call->count, call->dtype, call->in_place, piece_bytes, (int)c->max_pieces, align))
     return HOCCL_ERR_INVALID_ARG;
   if (P.slot_bytes) {
     size_t need = 2 * (size_t)c->R * P.slot_bytes;
