@@ -450,6 +450,14 @@ def extras(hb, W, torch, np, new_comm, step, timed, stream, R, S, n, dtype, peak
         fw_rows.append({"path": name, "sum_ctas": sc, "ms_per_step": t * 1e3, "busbw_GBps": S * bus_factor(R) / t / 1e9})
         c1.destroy()
     out["forward_variant"] = fw_rows
+    # the one route on a single device that really uses no SM for moves: bounce through pinned host memory
+    host_stage = torch.empty(400 << 20, dtype=torch.uint8).pin_memory()
+    c1 = new_comm(hb.PATH_CE_HOST, sum_ctas=8)
+    c1.set_host_staging(host_stage)
+    t, _ = timed(c1, 6, 3)
+    out["host_bounce_path"] = {"ms_per_step": t * 1e3, "busbw_GBps": S * bus_factor(R) / t / 1e9,
+                               "pcie_bytes_per_step_each_way": 2.0 * S * (R - 1)}
+    c1.destroy()
     # handshake mode (CPU proxy + stream memory operations) on the SM path, against the same path launched directly
     hs = {}
     for label, flag in (("direct", 0), ("handshake", 1)):
@@ -475,7 +483,10 @@ def extras(hb, W, torch, np, new_comm, step, timed, stream, R, S, n, dtype, peak
     sm_needs, sm_end = cm.probe_move_needs_sm(hb.PATH_SM, dst, src, nb, 3000)
     pinned = torch.empty(8 << 20, dtype=torch.uint8).pin_memory()
     h2d_needs, h2d_end = cm.probe_move_needs_sm(hb.PATH_CE, dst, pinned, pinned.numel(), 3000)
-    out["move_needs_sm"] = {"CE_driver_copy_same_device_64MiB": ce_needs, "CE_move_end_us": ce_end, "SM_copy_kernel": sm_needs,
+    cm.set_host_staging(host_stage)
+    hb_needs, hb_end = cm.probe_move_needs_sm(hb.PATH_CE_HOST, dst, src, min(nb, 16 << 20), 3000)
+    out["move_needs_sm"] = {"CE_HOST_bounce_16MiB": hb_needs, "CE_HOST_move_end_us": hb_end,
+                            "CE_driver_copy_same_device_64MiB": ce_needs, "CE_move_end_us": ce_end, "SM_copy_kernel": sm_needs,
                             "SM_move_end_us": sm_end, "control_pinned_host_to_device_8MiB": h2d_needs,
                             "control_move_end_us": h2d_end, "occupancy_kernel_us": 3000,
                             "note": "true = the move finished only after a kernel holding every SM had ended"}
@@ -553,8 +564,10 @@ def extras(hb, W, torch, np, new_comm, step, timed, stream, R, S, n, dtype, peak
     probe["alone_TFLOPs"] = alone
     for name, path, sc, cc, op in (("CE_sum8", hb.PATH_CE, 8, 8, 0), ("SM_copy8_sum8", hb.PATH_SM, 8, 8, 0),
                                    ("SM_copy32_sum8", hb.PATH_SM, 8, 32, 0), ("SM_copy148_sum148", hb.PATH_SM, 148, 148, 0),
-                                   ("onepass_8", hb.PATH_CE, 8, 8, 1)):
+                                   ("onepass_8", hb.PATH_CE, 8, 8, 1), ("CE_HOST_sum8", hb.PATH_CE_HOST, 8, 8, 0)):
         c2 = new_comm(path, sum_ctas=sc, copy_ctas=cc, onepass=op)
+        if path == hb.PATH_CE_HOST:
+            c2.set_host_staging(host_stage)
         tf, bw = gemm_tflops(c2)
         probe[name] = {"gemm_TFLOPs": tf, "loss": 1.0 - tf / alone, "comm_busbw_GBps": bw}
         c2.destroy()

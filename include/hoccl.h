@@ -68,10 +68,16 @@ typedef enum { HOCCL_SUM = 0 } hoccl_op_t;
  *                  the copy-engine route of the paper (Sec. 2.3 "DMA Engines", Sec. 3.3): between two
  *                  GPUs the driver services it with a DMA engine and no SM.  Whether a copy inside ONE
  *                  device is also SM free is up to the driver; hoccl_probe_move_needs_sm measures it.
+ *  HOCCL_PATH_CE_HOST : every move is a device-to-host copy into PINNED host staging followed by a host-to-device
+ *                  copy out of it.  Both legs are served by the copy engines (Sec. 2.3), so this is the one route
+ *                  on a single device that really occupies no SM (hoccl_probe_move_needs_sm confirms it); the price
+ *                  is PCIe bandwidth.  Needs hoccl_comm_set_host_staging with room for every move of a call
+ *                  (all-reduce: 2 * S * (R-1) bytes plus 256 per move).  Not available for hoccl_alltoallv or
+ *                  in handshake mode.
  *  HOCCL_PATH_SM : the comparison baseline (the paper's "NCCL with an SM budget", Sec. 5 "Baselines"):
  *                  all moves of a step run in one launch of an SM copy kernel with `copy_ctas` CTAs.
  */
-typedef enum { HOCCL_PATH_CE = 0, HOCCL_PATH_SM = 1 } hoccl_path_t;
+typedef enum { HOCCL_PATH_CE = 0, HOCCL_PATH_SM = 1, HOCCL_PATH_CE_HOST = 2 } hoccl_path_t;
 
 typedef struct {
   double host_launch_us; /* host time spent inside the last collective / matched p2p call (paper Sec. 5 "CPU launch overhead") */
@@ -112,6 +118,10 @@ hoccl_result_t hoccl_comm_set_scratch(hoccl_comm_t comm, void* dev_ptr, size_t b
 
 /* Attaches caller-owned device staging memory used only by the hoccl_host_* entry points. */
 hoccl_result_t hoccl_comm_set_staging(hoccl_comm_t comm, void* dev_ptr, size_t bytes);
+
+/* Attaches caller-owned PINNED host memory (cudaHostAlloc / cudaHostRegister) used by HOCCL_PATH_CE_HOST.
+ * INVALID_ARG if the pointer is not page-locked host memory. */
+hoccl_result_t hoccl_comm_set_host_staging(hoccl_comm_t comm, void* pinned_host_ptr, size_t bytes);
 
 hoccl_result_t hoccl_comm_set_path(hoccl_comm_t comm, hoccl_path_t path);
 

@@ -15,7 +15,7 @@ from . import build as _build
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_MISMATCH, ERR_PENDING, ERR_SCRATCH, ERR_INTERNAL, ERR_TIMEOUT = range(9)
 FLOAT32, BFLOAT16 = 0, 1
 SUM = 0
-PATH_CE, PATH_SM = 0, 1
+PATH_CE, PATH_SM, PATH_CE_HOST = 0, 1, 2
 PLAN_ALLREDUCE, PLAN_REDUCE_SCATTER, PLAN_ALLGATHER, PLAN_ALLTOALL, PLAN_ALLREDUCE_FWD, PLAN_REDUCE_SCATTER_FWD = range(6)
 OP_MOVE, OP_SUM = 0, 1
 BUF_SEND, BUF_RECV, BUF_INBOX, BUF_PARTIAL = 0, 1, 2, 3
@@ -23,7 +23,7 @@ BUF_SEND, BUF_RECV, BUF_INBOX, BUF_PARTIAL = 0, 1, 2, 3
 DTYPES = {"fp32": FLOAT32, "bf16": BFLOAT16}
 
 EXPORTS = [
-    "hoccl_comm_init", "hoccl_comm_destroy", "hoccl_scratch_bytes", "hoccl_comm_set_scratch", "hoccl_comm_set_staging",
+    "hoccl_comm_init", "hoccl_comm_destroy", "hoccl_scratch_bytes", "hoccl_comm_set_scratch", "hoccl_comm_set_staging", "hoccl_comm_set_host_staging",
     "hoccl_comm_set_path", "hoccl_comm_set_param", "hoccl_comm_get_param", "hoccl_allreduce", "hoccl_reduce_scatter",
     "hoccl_allgather", "hoccl_alltoall", "hoccl_alltoallv", "hoccl_send", "hoccl_recv", "hoccl_comm_pending", "hoccl_comm_async_error", "hoccl_comm_handshakes", "hoccl_host_allreduce", "hoccl_error_string",
     "hoccl_last_cuda_error", "hoccl_last_stats", "hoccl_profile_reset", "hoccl_probe_move_needs_sm", "hoccl_sum_launch",
@@ -87,6 +87,7 @@ def lib() -> ctypes.CDLL:
         "hoccl_scratch_bytes": (sz, [i, sz, i]),
         "hoccl_comm_set_scratch": (i, [vp, vp, sz]),
         "hoccl_comm_set_staging": (i, [vp, vp, sz]),
+        "hoccl_comm_set_host_staging": (i, [vp, vp, sz]),
         "hoccl_comm_set_path": (i, [vp, i]),
         "hoccl_comm_set_param": (i, [vp, ctypes.c_char_p, l]),
         "hoccl_comm_get_param": (i, [vp, ctypes.c_char_p, ctypes.POINTER(l)]),
@@ -218,6 +219,13 @@ class Comm:
             nbytes = buf.numel() * buf.element_size() if buf is not None else 0
         self._keep = [b for b in self._keep if b[0] != "staging"] + [("staging", buf)]
         self._check(lib().hoccl_comm_set_staging(self._h, _ptr(buf), nbytes), "hoccl_comm_set_staging")
+
+    def set_host_staging(self, pinned, nbytes: Optional[int] = None):
+        """Pinned host memory (e.g. a torch tensor created with pin_memory()) for the CE_HOST path."""
+        if nbytes is None:
+            nbytes = pinned.numel() * pinned.element_size() if pinned is not None else 0
+        self._keep = [b for b in self._keep if b[0] != "host_staging"] + [("host_staging", pinned)]
+        self._check(lib().hoccl_comm_set_host_staging(self._h, _ptr(pinned), nbytes), "hoccl_comm_set_host_staging")
 
     def set_path(self, path: int):
         self._check(lib().hoccl_comm_set_path(self._h, path), "hoccl_comm_set_path")

@@ -91,8 +91,22 @@ hoccl_result_t hoccl_comm_set_staging(hoccl_comm_t c, void* dev_ptr, size_t byte
   return HOCCL_OK;
 }
 
+hoccl_result_t hoccl_comm_set_host_staging(hoccl_comm_t c, void* pinned_host_ptr, size_t bytes) {
+  if (!c) return HOCCL_ERR_INVALID_ARG;
+  if (pinned_host_ptr) {
+    cudaPointerAttributes attr;
+    if (cudaPointerGetAttributes(&attr, pinned_host_ptr) != cudaSuccess || attr.type != cudaMemoryTypeHost) {
+      cudaGetLastError();
+      return HOCCL_ERR_INVALID_ARG;   // pageable memory would turn the copies into staged, synchronous ones
+    }
+  }
+  c->host_staging = static_cast<char*>(pinned_host_ptr);
+  c->host_staging_bytes = pinned_host_ptr ? bytes : 0;
+  return HOCCL_OK;
+}
+
 hoccl_result_t hoccl_comm_set_path(hoccl_comm_t c, hoccl_path_t path) {
-  if (!c || (path != HOCCL_PATH_CE && path != HOCCL_PATH_SM)) return HOCCL_ERR_INVALID_ARG;
+  if (!c || (path != HOCCL_PATH_CE && path != HOCCL_PATH_SM && path != HOCCL_PATH_CE_HOST)) return HOCCL_ERR_INVALID_ARG;
   c->path = path;
   return HOCCL_OK;
 }
@@ -236,7 +250,7 @@ hoccl_result_t hoccl_alltoallv(const void* const* send, const size_t* sendcounts
   if (!c || !send || !recv || !sendcounts || !sdispls || !rdispls) return HOCCL_ERR_INVALID_ARG;
   const size_t e = dtype_size((int)dtype);
   if (e == 0) return HOCCL_ERR_UNSUPPORTED;
-  if (c->handshake) return HOCCL_ERR_UNSUPPORTED;
+  if (c->handshake || c->path == HOCCL_PATH_CE_HOST) return HOCCL_ERR_UNSUPPORTED;
   const int R = c->R;
   for (int r = 0; r < R; r++) {
     if (!send[r] || !recv[r]) return HOCCL_ERR_INVALID_ARG;
@@ -471,6 +485,13 @@ hoccl_result_t hoccl_probe_move_needs_sm(hoccl_comm_t c, hoccl_path_t path, void
   if (e == cudaSuccess) {
     if (path == HOCCL_PATH_CE) {
       e = cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDefault, c->lane[1]);  // src may be pinned host memory (control)
+    } else if (path == HOCCL_PATH_CE_HOST) {
+      if (!c->host_staging || bytes > c->host_staging_bytes) {
+        e = cudaErrorInvalidValue;
+      } else {
+        e = cudaMemcpyAsync(c->host_staging, src, bytes, cudaMemcpyDeviceToHost, c->lane[1]);
+        if (e == cudaSuccess) e = cudaMemcpyAsync(dst, c->host_staging, bytes, cudaMemcpyHostToDevice, c->lane[1]);
+      }
     } else {
       CopyBatch b;
       b.nseg = 1;

@@ -34,6 +34,7 @@ struct Seg {
   const char* local;  // SUM only
   char* dst;
   uint64_t bytes;
+  uint64_t host_off = 0;  // HOCCL_PATH_CE_HOST: where this move bounces in the pinned host staging
 };
 
 struct RGroup {
@@ -79,6 +80,8 @@ struct hoccl_comm {
   size_t scratch_bytes = 0;
   void* staging = nullptr;
   size_t staging_bytes = 0;
+  char* host_staging = nullptr;  // pinned host memory of the CE_HOST path
+  size_t host_staging_bytes = 0;
   std::map<std::pair<int, int>, std::deque<hoccl::Post>> pending;
   int n_pending = 0;
   unsigned p2p_rr = 0;

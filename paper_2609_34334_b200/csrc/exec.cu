@@ -51,7 +51,8 @@ hoccl_result_t validate(hoccl_comm* c, Call* call) {
 }
 
 // Turns plan offsets into addresses (the plan already places pieces inside the scratch slots).
-void resolve(hoccl_comm* c, const Plan& P, const Call& call, std::vector<RGroup>* out) {
+void resolve(hoccl_comm* c, const Plan& P, const Call& call, std::vector<RGroup>* out, size_t* host_need) {
+  *host_need = 0;
   const int R = P.R;
   char* inbox0 = (char*)c->scratch;
   char* partial0 = inbox0 + (size_t)R * P.slot_bytes;
@@ -84,6 +85,10 @@ void resolve(hoccl_comm* c, const Plan& P, const Call& call, std::vector<RGroup>
         s.src = addr(op.src_buf, op.rank, op.chunk, op.src_off);
         s.local = addr(op.local_buf, op.rank, op.chunk, op.local_off);
         s.dst = addr(op.dst_buf, op.dst_rank, op.chunk, op.dst_off);  // dst_rank == rank except in the forward variant
+      }
+      if (op.kind == OP_MOVE && c->path == HOCCL_PATH_CE_HOST) {
+        s.host_off = *host_need;
+        *host_need += (s.bytes + 255) / 256 * 256;
       }
       rg.segs.push_back(s);
     }
@@ -175,6 +180,13 @@ hoccl_result_t run_streams(hoccl_comm* c, const Plan& P, const std::vector<RGrou
     } else if (c->path == HOCCL_PATH_CE) {
       for (const Seg& sg : rg.segs) {
         CU_TRY(c, cudaMemcpyAsync(sg.dst, sg.src, sg.bytes, cudaMemcpyDeviceToDevice, s));
+        tally->moves++;
+      }
+    } else if (c->path == HOCCL_PATH_CE_HOST) {
+      // two copy-engine legs through pinned host memory: no SM takes part in the move
+      for (const Seg& sg : rg.segs) {
+        CU_TRY(c, cudaMemcpyAsync(c->host_staging + sg.host_off, sg.src, sg.bytes, cudaMemcpyDeviceToHost, s));
+        CU_TRY(c, cudaMemcpyAsync(sg.dst, c->host_staging + sg.host_off, sg.bytes, cudaMemcpyHostToDevice, s));
         tally->moves++;
       }
     } else {
@@ -295,6 +307,17 @@ hoccl_result_t build_graph(hoccl_comm* c, const Plan& P, const std::vector<RGrou
         }
         if (e != cudaSuccess) break;
       }
+    } else if (c->path == HOCCL_PATH_CE_HOST) {
+      for (const Seg& sg : rg.segs) {
+        cudaGraphNode_t d2h, h2d;
+        e = cudaGraphAddMemcpyNode1D(&d2h, g, deps.data(), deps.size(), c->host_staging + sg.host_off, sg.src, sg.bytes,
+                                     cudaMemcpyDeviceToHost);
+        if (e != cudaSuccess) break;
+        e = cudaGraphAddMemcpyNode1D(&h2d, g, &d2h, 1, sg.dst, c->host_staging + sg.host_off, sg.bytes, cudaMemcpyHostToDevice);
+        if (e != cudaSuccess) break;
+        nodes.push_back(h2d);
+        entry->n_moves++;
+      }
     } else {
       for (size_t first = 0; first < rg.segs.size() && e == cudaSuccess; first += kMaxSegs) {
         size_t n = std::min<size_t>(kMaxSegs, rg.segs.size() - first);
@@ -360,6 +383,7 @@ std::vector<uint64_t> make_key(hoccl_comm* c, const Call& call) {
   k.push_back((uint64_t)c->ce_sub_bytes);
   k.push_back((uint64_t)c->forward);
   k.push_back((uint64_t)(uintptr_t)c->scratch);
+  k.push_back((uint64_t)(uintptr_t)c->host_staging);
   for (int r = 0; r < c->R; r++) {
     k.push_back((uint64_t)(uintptr_t)call.send[r]);
     k.push_back((uint64_t)(uintptr_t)call.recv[r]);
@@ -478,7 +502,7 @@ hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
   if (c->handshake) {
     // Driver copies share a hardware queue with the copies the parked stream has queued behind its hand-over; a copy
     // issued by the proxy can end up behind them and never start (observed).  Kernels do not have that problem.
-    if (c->path == HOCCL_PATH_CE) return HOCCL_ERR_UNSUPPORTED;
+    if (c->path != HOCCL_PATH_SM) return HOCCL_ERR_UNSUPPORTED;
     rc = ensure_proxy(c);
     if (rc != HOCCL_OK) return rc;
   }
@@ -493,7 +517,9 @@ hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
     c->stats.graph_hit = hit ? 1 : 0;
     if (!hit) {
       std::vector<RGroup> groups;
-      resolve(c, P, *call, &groups);
+      size_t host_need = 0;
+      resolve(c, P, *call, &groups, &host_need);
+      if (c->path == HOCCL_PATH_CE_HOST && (!c->host_staging || host_need > c->host_staging_bytes)) return HOCCL_ERR_SCRATCH;
       GraphEntry entry;
       entry.key = key;
       entry.n_pieces = P.pieces;
@@ -528,7 +554,9 @@ hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
     tally.sum_launches = hit->n_sum_launches;
   } else {
     std::vector<RGroup> groups;
-    resolve(c, P, *call, &groups);
+    size_t host_need = 0;
+    resolve(c, P, *call, &groups, &host_need);
+    if (c->path == HOCCL_PATH_CE_HOST && (!c->host_staging || host_need > c->host_staging_bytes)) return HOCCL_ERR_SCRATCH;
     rc = run_streams(c, P, groups, user, &tally);
     if (rc != HOCCL_OK) return rc;
   }

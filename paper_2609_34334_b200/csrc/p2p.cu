@@ -13,7 +13,7 @@ hoccl_result_t p2p_post(hoccl_comm* c, bool is_send, void* buf, size_t count, in
   if ((uintptr_t)buf % e) return HOCCL_ERR_INVALID_ARG;
   if (c->handshake) {
     // the post is handed to the proxy at once; matching happens there, after the stream has reached the post
-    if (c->path == HOCCL_PATH_CE) return HOCCL_ERR_UNSUPPORTED;   // see run_collective
+    if (c->path != HOCCL_PATH_SM) return HOCCL_ERR_UNSUPPORTED;   // see run_collective
     hoccl_result_t rc = ensure_proxy(c);
     if (rc != HOCCL_OK) return rc;
     ProxyTask t;
@@ -53,6 +53,29 @@ hoccl_result_t p2p_post(hoccl_comm* c, bool is_send, void* buf, size_t count, in
   if (ranges_overlap((const char*)sbuf, bytes, (const char*)dbuf, bytes)) return HOCCL_ERR_INVALID_ARG;
   CU_TRY(c, cudaSetDevice(c->device));
   const bool two_streams = (peer.stream != stream);
+  if (c->path == HOCCL_PATH_CE_HOST) {
+    // bounce through pinned host memory: two copy-engine legs, no SM.  All such moves share lane 0 and the start of
+    // the staging area, so they run one after the other.
+    if (!c->host_staging || bytes > c->host_staging_bytes) return HOCCL_ERR_SCRATCH;
+    c->ev_next = 0;
+    cudaEvent_t ea = next_event(c), eb = two_streams ? next_event(c) : nullptr, ed = next_event(c);
+    if (!ea || (two_streams && !eb) || !ed) return cuda_fail(c, cudaErrorMemoryAllocation, "event pool");
+    cudaStream_t run = c->lane[0];
+    CU_TRY(c, cudaEventRecord(ea, peer.stream));
+    CU_TRY(c, cudaStreamWaitEvent(run, ea, 0));
+    if (two_streams) {
+      CU_TRY(c, cudaEventRecord(eb, stream));
+      CU_TRY(c, cudaStreamWaitEvent(run, eb, 0));
+    }
+    CU_TRY(c, cudaMemcpyAsync(c->host_staging, sbuf, bytes, cudaMemcpyDeviceToHost, run));
+    CU_TRY(c, cudaMemcpyAsync(dbuf, c->host_staging, bytes, cudaMemcpyHostToDevice, run));
+    CU_TRY(c, cudaEventRecord(ed, run));
+    CU_TRY(c, cudaStreamWaitEvent(peer.stream, ed, 0));
+    if (two_streams) CU_TRY(c, cudaStreamWaitEvent(stream, ed, 0));
+    c->stats.n_moves = 1;
+    c->stats.host_launch_us = now_us() - t0;
+    return HOCCL_OK;
+  }
   // Large messages on the copy route are cut into up to 4 slices that run on different lanes: one driver copy of
   // 64 MiB reaches ~5.4 TB/s of HBM traffic, two to four concurrent ones ~6.5 TB/s (the same idea as keeping several
   // chunks in flight per connection, paper Sec. 3.3.1 "Multi-QP parallelism").
