@@ -369,7 +369,7 @@ hoccl_result_t build_graph(hoccl_comm* c, const Plan& P, const std::vector<RGrou
 
 std::vector<uint64_t> make_key(hoccl_comm* c, const Call& call) {
   std::vector<uint64_t> k;
-  k.reserve(12 + 2 * c->R);
+  k.reserve(16 + 2 * c->R);
   k.push_back((uint64_t)call.kind);
   k.push_back((uint64_t)call.count);
   k.push_back((uint64_t)call.dtype);
@@ -383,7 +383,9 @@ std::vector<uint64_t> make_key(hoccl_comm* c, const Call& call) {
   k.push_back((uint64_t)c->ce_sub_bytes);
   k.push_back((uint64_t)c->forward);
   k.push_back((uint64_t)(uintptr_t)c->scratch);
+  k.push_back((uint64_t)c->scratch_bytes);
   k.push_back((uint64_t)(uintptr_t)c->host_staging);
+  k.push_back((uint64_t)c->host_staging_bytes);
   for (int r = 0; r < c->R; r++) {
     k.push_back((uint64_t)(uintptr_t)call.send[r]);
     k.push_back((uint64_t)(uintptr_t)call.recv[r]);
@@ -434,10 +436,54 @@ hoccl_result_t ensure_proxy(hoccl_comm* c) {
   return HOCCL_OK;
 }
 
+// Replays a cached graph into the caller's stream (directly, or through the CPU proxy in handshake mode).
+static hoccl_result_t launch_entry(hoccl_comm* c, GraphEntry* hit, cudaStream_t user, double t0) {
+  hit->last_use = ++c->use_counter;
+  if (c->handshake) {
+    // paper Sec. 3.2: the stream hands itself to the CPU proxy, which runs the schedule and hands it back
+    ProxyTask t;
+    t.kind = ProxyTask::GRAPH;
+    t.exec = hit->exec;
+    CU_TRY(c, c->proxy->submit(user, t));
+  } else {
+    CU_TRY(c, cudaGraphLaunch(hit->exec, user));
+  }
+  hit->prof_pending = !hit->prof_events.empty();
+  c->stats.n_pieces = hit->n_pieces;
+  c->stats.n_moves = hit->n_moves;
+  c->stats.n_move_launches = hit->n_move_launches;
+  c->stats.n_sum_launches = hit->n_sum_launches;
+  c->stats.max_sum_ctas = hit->n_sum_launches ? c->sum_ctas : 0;
+  c->stats.max_copy_ctas = hit->n_move_launches ? c->copy_ctas : 0;
+  c->stats.host_launch_us = now_us() - t0;
+  return HOCCL_OK;
+}
+
 hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
   const double t0 = now_us();
   if (!c) return HOCCL_ERR_INVALID_ARG;
   if (dtype_size(call->dtype) == 0) return HOCCL_ERR_UNSUPPORTED;
+  if (!call->send || !call->recv) return HOCCL_ERR_INVALID_ARG;
+  const bool graphs = (c->use_graph || c->handshake) &&
+                      !(c->onepass && !c->handshake && (call->kind == PLAN_ALLREDUCE || call->kind == PLAN_REDUCE_SCATTER));
+  std::vector<uint64_t> key;
+  if (graphs && call->count != 0) {
+    // Fast path: a call whose signature (operation, count, dtype, every pointer, every setting that shapes the graph)
+    // was seen before was validated and planned then; replaying its graph is all that is left to do.
+    if (c->handshake && c->path != HOCCL_PATH_SM) return HOCCL_ERR_UNSUPPORTED;
+    key = make_key(c, *call);
+    for (auto& e : c->cache)
+      if (e.key == key) {
+        c->stats = hoccl_stats_t{};
+        c->stats.graph_hit = 1;
+        CU_TRY(c, cudaSetDevice(c->device));
+        if (c->handshake) {
+          hoccl_result_t prc = ensure_proxy(c);
+          if (prc != HOCCL_OK) return prc;
+        }
+        return launch_entry(c, &e, user, t0);
+      }
+  }
   hoccl_result_t rc = validate(c, call);
   if (rc != HOCCL_OK) return rc;
   c->stats = hoccl_stats_t{};
@@ -498,68 +544,45 @@ hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
   }
   c->stats.n_pieces = P.pieces;
   c->stats.max_sum_ctas = 0;
-  Tally tally;
-  if (c->handshake) {
-    // Driver copies share a hardware queue with the copies the parked stream has queued behind its hand-over; a copy
-    // issued by the proxy can end up behind them and never start (observed).  Kernels do not have that problem.
-    if (c->path != HOCCL_PATH_SM) return HOCCL_ERR_UNSUPPORTED;
-    rc = ensure_proxy(c);
-    if (rc != HOCCL_OK) return rc;
-  }
-  if (c->use_graph || c->handshake) {
-    std::vector<uint64_t> key = make_key(c, *call);
-    GraphEntry* hit = nullptr;
-    for (auto& e : c->cache)
-      if (e.key == key) {
-        hit = &e;
-        break;
-      }
-    c->stats.graph_hit = hit ? 1 : 0;
-    if (!hit) {
-      std::vector<RGroup> groups;
-      size_t host_need = 0;
-      resolve(c, P, *call, &groups, &host_need);
-      if (c->path == HOCCL_PATH_CE_HOST && (!c->host_staging || host_need > c->host_staging_bytes)) return HOCCL_ERR_SCRATCH;
-      GraphEntry entry;
-      entry.key = key;
-      entry.n_pieces = P.pieces;
-      rc = build_graph(c, P, groups, &entry);
-      if (rc != HOCCL_OK) return rc;
-      // handshake mode: place the graph on the device now; the proxy must not meet first-launch work later
-      if (c->handshake) CU_TRY(c, cudaGraphUpload(entry.exec, c->proxy->work_stream()));
-      if (c->cache.size() >= kGraphCacheCap) {
-        if (c->proxy) c->proxy->drain(c->watchdog_ms);  // a queued hand-over may still refer to the victim
-        size_t victim = 0;
-        for (size_t i = 1; i < c->cache.size(); i++)
-          if (c->cache[i].last_use < c->cache[victim].last_use) victim = i;
-        destroy_entry(&c->cache[victim]);
-        c->cache.erase(c->cache.begin() + victim);
-      }
-      c->cache.push_back(std::move(entry));
-      hit = &c->cache.back();
-    }
-    hit->last_use = ++c->use_counter;
+  std::vector<RGroup> groups;
+  size_t host_need = 0;
+  resolve(c, P, *call, &groups, &host_need);
+  if (c->path == HOCCL_PATH_CE_HOST && (!c->host_staging || host_need > c->host_staging_bytes)) return HOCCL_ERR_SCRATCH;
+  if (graphs) {
     if (c->handshake) {
-      // paper Sec. 3.2: the stream hands itself to the CPU proxy, which runs the schedule and hands it back
-      ProxyTask t;
-      t.kind = ProxyTask::GRAPH;
-      t.exec = hit->exec;
-      CU_TRY(c, c->proxy->submit(user, t));
-    } else {
-      CU_TRY(c, cudaGraphLaunch(hit->exec, user));
+      // Driver copies share a hardware queue with the copies the parked stream has queued behind its hand-over; a copy
+      // issued by the proxy can end up behind them and never start (observed).  Kernels do not have that problem.
+      // (Checked before the cache lookup; the proxy is created on first use.)
+      rc = ensure_proxy(c);
+      if (rc != HOCCL_OK) return rc;
     }
-    hit->prof_pending = !hit->prof_events.empty();
-    tally.moves = hit->n_moves;
-    tally.move_launches = hit->n_move_launches;
-    tally.sum_launches = hit->n_sum_launches;
-  } else {
-    std::vector<RGroup> groups;
-    size_t host_need = 0;
-    resolve(c, P, *call, &groups, &host_need);
-    if (c->path == HOCCL_PATH_CE_HOST && (!c->host_staging || host_need > c->host_staging_bytes)) return HOCCL_ERR_SCRATCH;
-    rc = run_streams(c, P, groups, user, &tally);
+    GraphEntry entry;
+    entry.key = key;
+    entry.n_pieces = P.pieces;
+    rc = build_graph(c, P, groups, &entry);
     if (rc != HOCCL_OK) return rc;
+    // handshake mode: place the graph on the device now; the proxy must not meet first-launch work later
+    if (c->handshake) {
+      cudaError_t ue = cudaGraphUpload(entry.exec, c->proxy->work_stream());
+      if (ue != cudaSuccess) {
+        destroy_entry(&entry);
+        return cuda_fail(c, ue, "cudaGraphUpload");
+      }
+    }
+    if (c->cache.size() >= kGraphCacheCap) {
+      if (c->proxy) c->proxy->drain(c->watchdog_ms);  // a queued hand-over may still refer to the victim
+      size_t victim = 0;
+      for (size_t i = 1; i < c->cache.size(); i++)
+        if (c->cache[i].last_use < c->cache[victim].last_use) victim = i;
+      destroy_entry(&c->cache[victim]);
+      c->cache.erase(c->cache.begin() + victim);
+    }
+    c->cache.push_back(std::move(entry));
+    return launch_entry(c, &c->cache.back(), user, t0);
   }
+  Tally tally;
+  rc = run_streams(c, P, groups, user, &tally);
+  if (rc != HOCCL_OK) return rc;
   c->stats.n_moves = tally.moves;
   c->stats.n_move_launches = tally.move_launches;
   c->stats.n_sum_launches = tally.sum_launches;
