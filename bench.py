@@ -490,6 +490,8 @@ def extras(hb, W, torch, np, new_comm, step, timed, stream, R, S, n, dtype, peak
                             "SM_move_end_us": sm_end, "control_pinned_host_to_device_8MiB": h2d_needs,
                             "control_move_end_us": h2d_end, "occupancy_kernel_us": 3000,
                             "note": "true = the move finished only after a kernel holding every SM had ended"}
+    out["copy_routes_16MiB"] = [{"route": n_, "needs_sm": s_, "end_us": round(t_, 1)}
+                                for n_, s_, t_ in cm.probe_copy_routes(dst, src, min(nb, 16 << 20), 3000)]
     # host cost of one call with an idle queue (the paper's CPU launch overhead axis)
     host_us = {}
     for label, use_graph in (("graph_replay", 1), ("stream_executor", 0)):

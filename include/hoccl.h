@@ -329,6 +329,24 @@ hoccl_result_t hoccl_probe_move_needs_sm(hoccl_comm_t comm, hoccl_path_t path, v
                                          int spin_us, int* needs_sm, double* move_end_us);
 
 /*
+ * The same measurement for every way the CUDA API offers to move bytes inside one device, one after the other:
+ * cudaMemcpyAsync, cudaMemcpyPeerAsync with both ends on this device, cuMemcpyDtoDAsync, a memcpy node of a CUDA
+ * graph, cudaMemcpy2DAsync, cudaMemsetAsync, this library's copy_kernel, and as controls a 32-bit stream memory
+ * write (what the paper's handshake uses, Listing 1) and, when pinned host staging is attached
+ * (hoccl_comm_set_host_staging, at least `bytes` bytes), a copy in each direction between device and pinned host.
+ * Writes one record per route that could be tried (at most max_out) and their number to *n_out.
+ * dst and src are disjoint device buffers of `bytes` bytes (bytes >= 4; dst is overwritten).  Synchronises the device.
+ * Errors: INVALID_ARG (null pointer, bytes < 4, spin_us outside [100, 20000]), CUDA.
+ */
+typedef struct {
+  char name[56];   /* which route */
+  int needs_sm;    /* 1: finished only after the SM-occupying kernel ended */
+  double end_us;   /* completion time, measured from the start of that kernel */
+} hoccl_route_probe_t;
+hoccl_result_t hoccl_probe_copy_routes(hoccl_comm_t comm, void* dst, const void* src, size_t bytes, int spin_us,
+                                       hoccl_route_probe_t* out, int max_out, int* n_out);
+
+/*
  * Direct launches of the two kernels (used by kernel-level tests and roofline measurements).
  *  hoccl_sum_launch : out[i] = round_to_dtype(float(inbox[i]) + float(local[i])), i < count, with `ctas` CTAs.
  *  hoccl_copy_launch: dst bytes <- src bytes with `ctas` CTAs.

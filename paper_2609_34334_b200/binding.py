@@ -26,13 +26,17 @@ EXPORTS = [
     "hoccl_comm_init", "hoccl_comm_destroy", "hoccl_scratch_bytes", "hoccl_comm_set_scratch", "hoccl_comm_set_staging", "hoccl_comm_set_host_staging",
     "hoccl_comm_set_path", "hoccl_comm_set_param", "hoccl_comm_get_param", "hoccl_allreduce", "hoccl_reduce_scatter",
     "hoccl_allgather", "hoccl_alltoall", "hoccl_alltoallv", "hoccl_send", "hoccl_recv", "hoccl_comm_pending", "hoccl_comm_async_error", "hoccl_comm_handshakes", "hoccl_host_allreduce", "hoccl_error_string",
-    "hoccl_last_cuda_error", "hoccl_last_stats", "hoccl_profile_reset", "hoccl_probe_move_needs_sm", "hoccl_sum_launch",
+    "hoccl_last_cuda_error", "hoccl_last_stats", "hoccl_profile_reset", "hoccl_probe_move_needs_sm", "hoccl_probe_copy_routes", "hoccl_sum_launch",
     "hoccl_copy_launch", "hoccl_plan_build", "hoccl_plan_destroy", "hoccl_plan_num_ops", "hoccl_plan_num_groups",
     "hoccl_plan_get_op", "hoccl_plan_group_deps", "hoccl_plan_slot_bytes", "hoccl_allreduce_static",
     "hoccl_sched_build", "hoccl_sched_destroy", "hoccl_sched_num_stages", "hoccl_sched_stage_tau", "hoccl_sched_total_tau",
     "hoccl_sched_lower_bound", "hoccl_sched_matrix", "hoccl_sched_num_flows", "hoccl_sched_get_flow", "hoccl_sched_queue_len",
     "hoccl_sched_queue_get",
 ]
+
+
+class RouteProbe(ctypes.Structure):
+    _fields_ = [("name", ctypes.c_char * 56), ("needs_sm", ctypes.c_int), ("end_us", ctypes.c_double)]
 
 
 class Stats(ctypes.Structure):
@@ -119,6 +123,7 @@ def lib() -> ctypes.CDLL:
         "hoccl_last_stats": (i, [vp, ctypes.POINTER(Stats)]),
         "hoccl_profile_reset": (i, [vp]),
         "hoccl_probe_move_needs_sm": (i, [vp, i, vp, vp, sz, i, ctypes.POINTER(i), ctypes.POINTER(ctypes.c_double)]),
+        "hoccl_probe_copy_routes": (i, [vp, vp, vp, sz, i, ctypes.POINTER(RouteProbe), i, ctypes.POINTER(i)]),
         "hoccl_sum_launch": (i, [vp, vp, vp, sz, i, i, vp]),
         "hoccl_copy_launch": (i, [vp, vp, sz, i, vp]),
         "hoccl_plan_build": (i, [vpp, i, i, sz, i, i, sz, i, ctypes.c_char_p]),
@@ -313,6 +318,14 @@ class Comm:
         self._check(lib().hoccl_probe_move_needs_sm(self._h, path, _ptr(dst), _ptr(src), nbytes, spin_us, ctypes.byref(needs),
                                                     ctypes.byref(end_us)), "hoccl_probe_move_needs_sm")
         return bool(needs.value), end_us.value
+
+    def probe_copy_routes(self, dst, src, nbytes, spin_us=3000):
+        """[(route name, needs an SM, completion time in us)] for every same-device way of moving bytes."""
+        out = (RouteProbe * 16)()
+        n = ctypes.c_int()
+        self._check(lib().hoccl_probe_copy_routes(self._h, _ptr(dst), _ptr(src), nbytes, spin_us, out, 16, ctypes.byref(n)),
+                    "hoccl_probe_copy_routes")
+        return [(out[k].name.decode(), bool(out[k].needs_sm), out[k].end_us) for k in range(n.value)]
 
 
 STATIC_SCRATCH_BYTES = 32 << 20

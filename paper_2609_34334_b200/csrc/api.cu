@@ -464,58 +464,6 @@ hoccl_result_t hoccl_profile_reset(hoccl_comm_t c) {
   return HOCCL_OK;
 }
 
-hoccl_result_t hoccl_probe_move_needs_sm(hoccl_comm_t c, hoccl_path_t path, void* dst, const void* src, size_t bytes, int spin_us,
-                                         int* needs_sm, double* move_end_us) {
-  if (!c || !dst || !src || !needs_sm || bytes == 0 || spin_us < 100 || spin_us > 20000) return HOCCL_ERR_INVALID_ARG;
-  CU_TRY(c, cudaSetDevice(c->device));
-  CU_TRY(c, cudaDeviceSynchronize());
-  cudaEvent_t a0, a1, b1;
-  CU_TRY(c, cudaEventCreate(&a0));
-  CU_TRY(c, cudaEventCreate(&a1));
-  CU_TRY(c, cudaEventCreate(&b1));
-  hoccl_result_t rc = HOCCL_OK;
-  cudaError_t e = cudaEventRecord(a0, c->lane[0]);
-  int ctas = 0;
-  if (e == cudaSuccess) e = launch_occupy_all_sms((unsigned long long)spin_us * 1000ull, c->num_sms, c->lane[0], &ctas);
-  if (e == cudaSuccess) e = cudaEventRecord(a1, c->lane[0]);
-  // let the occupying kernel become resident before the move is enqueued
-  const double t0 = now_us();
-  while (now_us() - t0 < std::min(300.0, spin_us * 0.25)) {
-  }
-  if (e == cudaSuccess) {
-    if (path == HOCCL_PATH_CE) {
-      e = cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDefault, c->lane[1]);  // src may be pinned host memory (control)
-    } else if (path == HOCCL_PATH_CE_HOST) {
-      if (!c->host_staging || bytes > c->host_staging_bytes) {
-        e = cudaErrorInvalidValue;
-      } else {
-        e = cudaMemcpyAsync(c->host_staging, src, bytes, cudaMemcpyDeviceToHost, c->lane[1]);
-        if (e == cudaSuccess) e = cudaMemcpyAsync(dst, c->host_staging, bytes, cudaMemcpyHostToDevice, c->lane[1]);
-      }
-    } else {
-      CopyBatch b;
-      b.nseg = 1;
-      b.pad = 0;
-      b.seg[0] = CopySeg{src, dst, (unsigned long long)bytes};
-      e = launch_copy(b, (int)c->copy_ctas, c->lane[1]);
-    }
-  }
-  if (e == cudaSuccess) e = cudaEventRecord(b1, c->lane[1]);
-  if (e == cudaSuccess) e = cudaDeviceSynchronize();
-  float spin_ms = 0, end_ms = 0;
-  if (e == cudaSuccess) e = cudaEventElapsedTime(&spin_ms, a0, a1);
-  if (e == cudaSuccess) e = cudaEventElapsedTime(&end_ms, a0, b1);
-  if (e != cudaSuccess) rc = cuda_fail(c, e, "probe_move_needs_sm");
-  else {
-    *needs_sm = end_ms >= 0.9f * spin_ms ? 1 : 0;
-    if (move_end_us) *move_end_us = end_ms * 1e3;
-  }
-  cudaEventDestroy(a0);
-  cudaEventDestroy(a1);
-  cudaEventDestroy(b1);
-  return rc;
-}
-
 hoccl_result_t hoccl_sum_launch(const void* inbox, const void* local, void* out, size_t count, hoccl_dtype_t dtype, int ctas,
                                 hoccl_stream_t stream) {
   size_t e = dtype_size((int)dtype);

@@ -1,6 +1,7 @@
 """Kernel microbenchmarks through the C ABI (hoccl_sum_launch / hoccl_copy_launch), one kernel at a time.
 
     python -m paper_2609_34334_b200.microbench --kernel sum --dtype bf16 --mib 200 --ctas 8 --reps 5
+    python -m paper_2609_34334_b200.microbench --kernel routes --mib 16      # which same-device copy routes need an SM
 
 Operands are larger than L2 by default; timing uses CUDA events on the launching stream after warm-up.
 Prints one JSON line.  This is the small case used for ncu captures of a single kernel.
@@ -17,7 +18,7 @@ from . import binding as hb
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--kernel", default="sum", choices=["sum", "copy"])
+    ap.add_argument("--kernel", default="sum", choices=["sum", "copy", "routes"])
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "fp32"])
     ap.add_argument("--mib", type=int, default=200, help="MiB per operand")
     ap.add_argument("--ctas", type=int, default=8)
@@ -26,6 +27,18 @@ def main():
     args = ap.parse_args()
     torch.cuda.set_device(0)
     nbytes = args.mib << 20
+    if args.kernel == "routes":
+        src = torch.full((nbytes,), 7, dtype=torch.uint8, device="cuda")
+        dst = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")
+        host = torch.empty(nbytes, dtype=torch.uint8).pin_memory()
+        comm = hb.Comm(2, 0)
+        comm.set_param("copy_ctas", args.ctas)
+        comm.set_host_staging(host)
+        rows = comm.probe_copy_routes(dst, src, nbytes, 3000)
+        comm.destroy()
+        print(json.dumps({"probe": "copy routes under a kernel that holds every SM for 3000 us", "mib": args.mib,
+                          "routes": [{"route": n, "needs_sm": s, "end_us": round(t, 1)} for n, s, t in rows]}))
+        return
     e = 2 if args.dtype == "bf16" else 4
     n = nbytes // e
     tdt = torch.bfloat16 if args.dtype == "bf16" else torch.float32

@@ -635,3 +635,25 @@ def test_probe_move_needs_sm_terminates():
     needs_ce, end_ce = comm.probe_move_needs_sm(hb.PATH_CE, b, a, a.numel(), 1500)
     assert isinstance(needs_ce, bool) and end_ce > 0         # the answer is the driver's; it is reported, not asserted
     comm.destroy()
+
+
+def test_probe_copy_routes_controls_and_copy_kernel():
+    """Every same-device route is tried in turn; what the driver does with its own copies is reported, not asserted,
+    but the controls are fixed: a stream memory write and pinned-host copies need no SM, copy_kernel needs one."""
+    comm = hb.Comm(2, 0)
+    comm.set_param("copy_ctas", 8)
+    n = 1 << 20
+    a = torch.full((n,), 3, dtype=torch.uint8, device="cuda")
+    b = torch.zeros(n, dtype=torch.uint8, device="cuda")
+    host = torch.empty(n, dtype=torch.uint8).pin_memory()
+    comm.set_host_staging(host)
+    rows = {name: (needs, end) for name, needs, end in comm.probe_copy_routes(b, a, n, 3000)}
+    assert len(rows) >= 9
+    for name, (needs, end) in rows.items():
+        assert end > 0, name
+    assert rows["copy_kernel (this library, by construction)"][0] is True
+    assert rows["control: cuStreamWriteValue32"][0] is False
+    assert rows["control: device->pinned host"][0] is False
+    assert rows["control: pinned host->device"][0] is False
+    assert torch.equal(b, a)                                  # the last route copied host (= a) back into b
+    comm.destroy()
