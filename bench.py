@@ -450,6 +450,16 @@ def extras(hb, W, torch, np, new_comm, step, timed, stream, R, S, n, dtype, peak
         fw_rows.append({"path": name, "sum_ctas": sc, "ms_per_step": t * 1e3, "busbw_GBps": S * bus_factor(R) / t / 1e9})
         c1.destroy()
     out["forward_variant"] = fw_rows
+    # SM path with the whole collective as one cooperative kernel (grid barriers instead of kernel boundaries)
+    fu_rows = []
+    for ctas in (8, 148):
+        c1 = new_comm(hb.PATH_SM, sum_ctas=ctas, copy_ctas=ctas, fused=1)
+        t, _ = timed(c1, k, w, fn=one_call)
+        fu_rows.append({"ctas": ctas, "ms_per_step": t * 1e3, "busbw_GBps": S * bus_factor(R) / t / 1e9,
+                        "launches_per_step": int(c1.last_stats()["n_move_launches"] + c1.last_stats()["n_sum_launches"]),
+                        "async_error": int(c1.async_error())})
+        c1.destroy()
+    out["fused_ring_kernel_SM_path"] = fu_rows
     # the one route on a single device that really uses no SM for moves: bounce through pinned host memory
     host_stage = torch.empty(400 << 20, dtype=torch.uint8).pin_memory()
     c1 = new_comm(hb.PATH_CE_HOST, sum_ctas=8)

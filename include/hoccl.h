@@ -148,6 +148,17 @@ hoccl_result_t hoccl_comm_set_path(hoccl_comm_t comm, hoccl_path_t path);
  *                straight into the next rank's inbox, so only step 0 needs moves (3 instead of 5 bytes of traffic per
  *                wire byte in that phase).  Same bits.  A SUM then stores into another rank's memory, as SM-driven
  *                libraries do: it is the second comparison point for what rank locality costs.  0 = off (default).
+ *  "fused"       1 = on HOCCL_PATH_SM the whole collective runs as ONE cooperative kernel that walks the ring steps with a
+ *                grid-wide barrier between dependent steps (how an SM-driven library runs a collective: the paper's
+ *                "NCCL under an SM budget" baseline, Sec. 5).  The schedule stays rank local and the bits are the same.
+ *                Its grid is min(sum_ctas, copy_ctas) CTAs (copy_ctas for pure moves), fewer for small messages.
+ *                Measured on B200: a grid barrier costs about what a kernel boundary inside a CUDA graph costs, so small
+ *                messages gain nothing; with the whole GPU, messages of 128 MiB and more run 7-20 % faster (no ramp and
+ *                tail per step).  Every barrier wait is bounded; a wait that runs out ends the kernel and is reported by
+ *                hoccl_comm_async_error as HOCCL_ERR_TIMEOUT.  The library allocates 16 bytes of device memory and 4 bytes
+ *                of pinned host memory of its own on first use (the third exception to "device memory is the caller's").
+ *                Ignored on the other paths, in handshake mode, and for plans too large for one launch (more than 896
+ *                chunk operations, i.e. beyond roughly 16 ranks), which run as a graph.  0 = off (default).
  *  "use_graph"   1 = run a cached CUDA graph built from the plan (default), 0 = streams and events
  *  "handshake"   1 = the paper's stream manager (Sec. 3.2, Listing 1): instead of launching into the caller's
  *                stream, the call enqueues four stream memory operations (write start flag, wait for the CPU's
@@ -254,7 +265,8 @@ hoccl_result_t hoccl_send(const void* buf, size_t count, hoccl_dtype_t dtype, in
 hoccl_result_t hoccl_recv(void* buf, size_t count, hoccl_dtype_t dtype, int src, int dst, hoccl_comm_t comm,
                           hoccl_stream_t stream);
 int hoccl_comm_pending(hoccl_comm_t comm);
-/* Handshake mode: first asynchronous failure seen by the proxy (OK, TIMEOUT, MISMATCH or CUDA); clear != 0 resets it. */
+/* First asynchronous failure: handshake mode, as seen by the proxy (OK, TIMEOUT, MISMATCH or CUDA); "fused" setting,
+ * TIMEOUT if a barrier wait of the whole-collective kernel ran out.  clear != 0 resets it. */
 hoccl_result_t hoccl_comm_async_error(hoccl_comm_t comm, int clear);
 /* Handshake mode: number of stream hand-overs the proxy has served so far. */
 long hoccl_comm_handshakes(hoccl_comm_t comm);

@@ -58,6 +58,8 @@ hoccl_result_t hoccl_comm_destroy(hoccl_comm_t c) {
     cudaStreamDestroy(c->sum_stream);
   }
   for (auto& e : c->cache) destroy_entry(&e);
+  if (c->ring_bar) cudaFree(c->ring_bar);
+  if (c->ring_err) cudaFreeHost(c->ring_err);
   for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
   for (auto& p : c->prof_pool) {
     cudaEventDestroy(p.first);
@@ -122,7 +124,7 @@ static long* param_slot(hoccl_comm* c, const char* key, long* lo, long* hi) {
               {"profile", &c->profile, 0, 1},           {"p2p_split", &c->p2p_split, 1, kMaxLanes},
               {"ce_sub_bytes", &c->ce_sub_bytes, 0, 1L << 40}, {"handshake", &c->handshake, 0, 1},
               {"watchdog_ms", &c->watchdog_ms, 10, 600000},    {"onepass", &c->onepass, 0, 1},
-              {"forward", &c->forward, 0, 1}};
+              {"forward", &c->forward, 0, 1},           {"fused", &c->fused, 0, 1}};
   for (auto& r : rows)
     if (std::strcmp(r.name, key) == 0) {
       *lo = r.lo;
@@ -204,6 +206,10 @@ int hoccl_comm_pending(hoccl_comm_t c) {
 
 hoccl_result_t hoccl_comm_async_error(hoccl_comm_t c, int clear) {
   if (!c) return HOCCL_ERR_INVALID_ARG;
+  if (c->ring_err && *reinterpret_cast<volatile int*>(c->ring_err) != 0) {
+    if (clear) *reinterpret_cast<volatile int*>(c->ring_err) = 0;
+    return HOCCL_ERR_TIMEOUT;   // a barrier wait of the whole-collective kernel ran out
+  }
   if (!c->proxy) return HOCCL_OK;
   int e = c->proxy->async_error();
   if (clear) c->proxy->clear_error();

@@ -60,6 +60,11 @@ struct GraphEntry {
   std::vector<std::pair<cudaEvent_t, cudaEvent_t>> prof_events;  // owned; only with profile = 1
   std::vector<double> prof_bytes;
   bool prof_pending = false;  // replayed since the profile events were last read
+  // "fused" setting: the whole plan as one cooperative kernel instead of a graph (exec stays null)
+  std::vector<char> ring_args;  // a RingArgsSmall or RingArgsLarge, by value
+  bool ring_large = false;
+  int ring_grid = 0, ring_threads = 0;
+  bool ring_has_sum = false;
 };
 
 }  // namespace hoccl
@@ -68,7 +73,7 @@ struct hoccl_comm {
   int R = 0, device = 0, num_sms = 0;
   hoccl_path_t path = HOCCL_PATH_CE;
   long sum_ctas = 8, copy_ctas = 8, piece_bytes = 4 << 20, max_pieces = 8, lanes = 4, use_graph = 1, profile = 0, p2p_split = 1, ce_sub_bytes = 0,
-       handshake = 0, watchdog_ms = 10000, onepass = 0, forward = 0;
+       handshake = 0, watchdog_ms = 10000, onepass = 0, forward = 0, fused = 0;
   bool piece_bytes_set = false;  // the caller chose a piece size: no automatic choice
   hoccl::Proxy* proxy = nullptr;
   cudaStream_t lane[hoccl::kMaxLanes] = {};
@@ -80,6 +85,9 @@ struct hoccl_comm {
   size_t scratch_bytes = 0;
   void* staging = nullptr;
   size_t staging_bytes = 0;
+  unsigned* ring_bar = nullptr;  // "fused" setting: three device words of the grid barrier (library owned, 16 bytes)
+  int* ring_err = nullptr;       // mapped pinned host word the ring kernel sets when a barrier wait ran out
+  int* ring_err_dev = nullptr;   // the same word as the device sees it
   char* host_staging = nullptr;  // pinned host memory of the CE_HOST path
   size_t host_staging_bytes = 0;
   std::map<std::pair<int, int>, std::deque<hoccl::Post>> pending;

@@ -369,7 +369,7 @@ hoccl_result_t build_graph(hoccl_comm* c, const Plan& P, const std::vector<RGrou
 
 std::vector<uint64_t> make_key(hoccl_comm* c, const Call& call) {
   std::vector<uint64_t> k;
-  k.reserve(16 + 2 * c->R);
+  k.reserve(17 + 2 * c->R);
   k.push_back((uint64_t)call.kind);
   k.push_back((uint64_t)call.count);
   k.push_back((uint64_t)call.dtype);
@@ -382,6 +382,7 @@ std::vector<uint64_t> make_key(hoccl_comm* c, const Call& call) {
   k.push_back((uint64_t)c->profile);
   k.push_back((uint64_t)c->ce_sub_bytes);
   k.push_back((uint64_t)c->forward);
+  k.push_back((uint64_t)(c->fused && c->path == HOCCL_PATH_SM && !c->handshake));
   k.push_back((uint64_t)(uintptr_t)c->scratch);
   k.push_back((uint64_t)c->scratch_bytes);
   k.push_back((uint64_t)(uintptr_t)c->host_staging);
@@ -436,9 +437,123 @@ hoccl_result_t ensure_proxy(hoccl_comm* c) {
   return HOCCL_OK;
 }
 
+// ------------------------------------------------------------------ whole-collective kernel ------
+// The barrier words and the error word of the "fused" setting are the library's own (16 bytes of device memory and
+// 4 bytes of mapped pinned host memory), allocated on first use.
+static hoccl_result_t ensure_ring_ctrl(hoccl_comm* c) {
+  if (c->ring_bar) return HOCCL_OK;
+  unsigned* bar = nullptr;
+  int* err = nullptr;
+  int* err_dev = nullptr;
+  CU_TRY(c, cudaMalloc(&bar, 16));
+  cudaError_t e = cudaMemset(bar, 0, 16);
+  if (e == cudaSuccess) e = cudaHostAlloc(&err, sizeof(int), cudaHostAllocMapped);
+  if (e == cudaSuccess) {
+    *err = 0;
+    e = cudaHostGetDevicePointer(&err_dev, err, 0);
+  }
+  if (e == cudaSuccess) e = preload_ring_kernels();
+  if (e != cudaSuccess) {
+    cudaFree(bar);
+    if (err) cudaFreeHost(err);
+    return cuda_fail(c, e, "ring kernel control words");
+  }
+  c->ring_bar = bar;
+  c->ring_err = err;
+  c->ring_err_dev = err_dev;
+  return HOCCL_OK;
+}
+
+template <typename Args, int NPH, int NSEG>
+static bool fill_ring_args(const std::vector<RGroup>& groups, int dtype, unsigned* bar, int* err_dev, Args* a, size_t* max_phase_bytes,
+                           bool* has_sum) {
+  int nph = 0, nseg = 0;
+  *max_phase_bytes = 0;
+  *has_sum = false;
+  a->dtype = dtype;
+  a->bar = bar;
+  a->host_err = err_dev;
+  for (const RGroup& g : groups) {
+    bool first_of_group = true;
+    for (size_t first = 0; first < g.segs.size(); first += kMaxSegs) {
+      const size_t n = std::min<size_t>(kMaxSegs, g.segs.size() - first);
+      if (nph >= NPH || nseg + (int)n > NSEG) return false;
+      RingPhase& ph = a->phase[nph++];
+      ph.first_seg = nseg;
+      ph.nseg = (int)n;
+      ph.kind = g.kind == OP_SUM ? 1 : 0;
+      ph.barrier_before = (first_of_group && !g.deps.empty()) ? 1 : 0;
+      first_of_group = false;
+      size_t bytes = 0;
+      for (size_t i = 0; i < n; i++) {
+        const Seg& sg = g.segs[first + i];
+        a->seg[nseg++] = RingSeg{sg.src, g.kind == OP_SUM ? sg.local : nullptr, sg.dst, (unsigned long long)sg.bytes};
+        bytes += sg.bytes;
+      }
+      *max_phase_bytes = std::max(*max_phase_bytes, bytes);
+      if (g.kind == OP_SUM) *has_sum = true;
+    }
+  }
+  a->nphase = nph;
+  return true;
+}
+
+// Turns the resolved plan into the parameter block of one ring_kernel launch.  UNSUPPORTED if the plan does not fit
+// into the kernel's parameter space (very many ranks): the caller then falls back to the graph.
+static hoccl_result_t build_ring(hoccl_comm* c, const Plan& P, const std::vector<RGroup>& groups, GraphEntry* entry) {
+  hoccl_result_t rc = ensure_ring_ctrl(c);
+  if (rc != HOCCL_OK) return rc;
+  size_t max_phase_bytes = 0;
+  bool has_sum = false;
+  entry->ring_args.assign(sizeof(RingArgsSmall), 0);
+  entry->ring_large = false;
+  if (!fill_ring_args<RingArgsSmall, kRingSmallPhases, kRingSmallSegs>(groups, P.dtype, c->ring_bar, c->ring_err_dev,
+                                                                     reinterpret_cast<RingArgsSmall*>(entry->ring_args.data()), &max_phase_bytes, &has_sum)) {
+    entry->ring_args.assign(sizeof(RingArgsLarge), 0);
+    entry->ring_large = true;
+    if (!fill_ring_args<RingArgsLarge, kRingLargePhases, kRingLargeSegs>(groups, P.dtype, c->ring_bar, c->ring_err_dev,
+                                                                       reinterpret_cast<RingArgsLarge*>(entry->ring_args.data()), &max_phase_bytes, &has_sum)) {
+      entry->ring_args.clear();
+      return HOCCL_ERR_UNSUPPORTED;
+    }
+  }
+  // CTA budget: never more than either budget of the SM path; never more CTAs than the largest phase has tiles for
+  // (a barrier costs more the more CTAs take part); never more than can be resident together.
+  long budget = has_sum ? std::min(c->sum_ctas, c->copy_ctas) : c->copy_ctas;
+  const int threads = budget >= 64 ? 512 : 1024;
+  const size_t tile_bytes = (size_t)threads * 4 * 16;
+  const long tiles = (long)((max_phase_bytes + tile_bytes - 1) / tile_bytes);
+  int max_grid = 0;
+  CU_TRY(c, ring_max_grid(threads, P.dtype, entry->ring_large, c->num_sms, &max_grid));
+  long grid = std::max<long>(1, std::min<long>(std::min<long>(budget, tiles), max_grid));
+  entry->ring_grid = (int)grid;
+  entry->ring_threads = threads;
+  entry->ring_has_sum = has_sum;
+  entry->n_moves = 0;
+  for (const RGroup& g : groups)
+    if (g.kind != OP_SUM) entry->n_moves += (long)g.segs.size();
+  entry->n_move_launches = 1;   // the one launch of the collective
+  entry->n_sum_launches = 0;
+  return HOCCL_OK;
+}
+
 // Replays a cached graph into the caller's stream (directly, or through the CPU proxy in handshake mode).
 static hoccl_result_t launch_entry(hoccl_comm* c, GraphEntry* hit, cudaStream_t user, double t0) {
   hit->last_use = ++c->use_counter;
+  if (!hit->ring_args.empty()) {
+    if (hit->ring_large)
+      CU_TRY(c, launch_ring(*reinterpret_cast<const RingArgsLarge*>(hit->ring_args.data()), hit->ring_grid, hit->ring_threads, user));
+    else
+      CU_TRY(c, launch_ring(*reinterpret_cast<const RingArgsSmall*>(hit->ring_args.data()), hit->ring_grid, hit->ring_threads, user));
+    c->stats.n_pieces = hit->n_pieces;
+    c->stats.n_moves = hit->n_moves;
+    c->stats.n_move_launches = 1;
+    c->stats.n_sum_launches = 0;
+    c->stats.max_copy_ctas = hit->ring_grid;
+    c->stats.max_sum_ctas = hit->ring_has_sum ? hit->ring_grid : 0;
+    c->stats.host_launch_us = now_us() - t0;
+    return HOCCL_OK;
+  }
   if (c->handshake) {
     // paper Sec. 3.2: the stream hands itself to the CPU proxy, which runs the schedule and hands it back
     ProxyTask t;
@@ -464,8 +579,9 @@ hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
   if (!c) return HOCCL_ERR_INVALID_ARG;
   if (dtype_size(call->dtype) == 0) return HOCCL_ERR_UNSUPPORTED;
   if (!call->send || !call->recv) return HOCCL_ERR_INVALID_ARG;
-  const bool graphs = (c->use_graph || c->handshake) &&
-                      !(c->onepass && !c->handshake && (call->kind == PLAN_ALLREDUCE || call->kind == PLAN_REDUCE_SCATTER));
+  const bool onepass_case = c->onepass && !c->handshake && (call->kind == PLAN_ALLREDUCE || call->kind == PLAN_REDUCE_SCATTER);
+  const bool fused = c->fused && c->path == HOCCL_PATH_SM && !c->handshake && !onepass_case;
+  const bool graphs = (c->use_graph || c->handshake || fused) && !onepass_case;
   std::vector<uint64_t> key;
   if (graphs && call->count != 0) {
     // Fast path: a call whose signature (operation, count, dtype, every pointer, every setting that shapes the graph)
@@ -525,13 +641,17 @@ hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
   // (the copy kernel of one piece then overlaps the sum kernel of the other: measured 1.6x on a 3 MiB chunk with 8 + 8
   // CTAs), which does not pay with driver copies or whole-GPU grids.
   size_t piece_bytes = (size_t)c->piece_bytes;
-  if (!c->piece_bytes_set && c->path == HOCCL_PATH_SM && std::max(c->sum_ctas, c->copy_ctas) < 64 &&
+  int max_pieces = (int)c->max_pieces;
+  if (fused) {   // one kernel walks the steps in order; whole chunks measured faster than pieces (fewer barriers and tails)
+    piece_bytes = (size_t)1 << 60;
+    max_pieces = 1;
+  } else if (!c->piece_bytes_set && c->path == HOCCL_PATH_SM && std::max(c->sum_ctas, c->copy_ctas) < 64 &&
       (call->kind == PLAN_ALLREDUCE || call->kind == PLAN_REDUCE_SCATTER)) {
     const size_t q = call->kind == PLAN_ALLREDUCE ? (call->count + c->R - 1) / c->R : call->count;
     const size_t chunk = q * dtype_size(call->dtype);
     if (chunk >= ((size_t)1 << 20)) piece_bytes = std::min(piece_bytes, (chunk / 2 + 1023) / 1024 * 1024);
   }
-  if (!build_plan(&P, plan_kind, c->R, call->count, call->dtype, call->in_place, piece_bytes, (int)c->max_pieces, align))
+  if (!build_plan(&P, plan_kind, c->R, call->count, call->dtype, call->in_place, piece_bytes, max_pieces, align))
     return HOCCL_ERR_INVALID_ARG;
   if (P.slot_bytes) {
     size_t need = 2 * (size_t)c->R * P.slot_bytes;
@@ -559,7 +679,8 @@ hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
     GraphEntry entry;
     entry.key = key;
     entry.n_pieces = P.pieces;
-    rc = build_graph(c, P, groups, &entry);
+    rc = fused ? build_ring(c, P, groups, &entry) : HOCCL_ERR_UNSUPPORTED;
+    if (rc == HOCCL_ERR_UNSUPPORTED) rc = build_graph(c, P, groups, &entry);   // not asked for, or too many ranks for one launch
     if (rc != HOCCL_OK) return rc;
     // handshake mode: place the graph on the device now; the proxy must not meet first-launch work later
     if (c->handshake) {

@@ -50,6 +50,41 @@ struct OnePassArgs {
 };
 cudaError_t launch_onepass(const OnePassArgs& args, int ctas, cudaStream_t stream);
 
+// Whole-collective kernel of the SM path ("fused" setting): one cooperative launch walks the plan's groups in order,
+// a grid-wide barrier between dependent groups.  This is how an SM-driven library runs a collective (one persistent
+// kernel, the paper's "NCCL under an SM budget" baseline of Sec. 5), while the schedule stays rank local: MOVE into
+// the receiver's inbox, then SUM out of it.  It removes the per-step launch cost that dominates small messages.
+struct RingSeg {
+  const void* src;     // MOVE: source; SUM: inbox
+  const void* local;   // SUM: local contribution; MOVE: nullptr
+  void* dst;
+  unsigned long long bytes;
+};
+struct RingPhase {
+  int first_seg, nseg;
+  int kind;            // 0 MOVE, 1 SUM
+  int barrier_before;  // 1: a grid barrier separates this phase from the ones before it
+};
+constexpr int kRingSmallPhases = 32, kRingSmallSegs = 256;   // 8.7 KB of kernel parameters
+constexpr int kRingLargePhases = 224, kRingLargeSegs = 896;  // 32.3 KB (the limit is 32,764 bytes)
+constexpr unsigned kRingSpinLimit = 1u << 21;                // polls of one barrier wait before the kernel gives up (~1-2 s)
+template <int NPH, int NSEG>
+struct RingArgsT {
+  int nphase;
+  int dtype;
+  unsigned* bar;   // device words {arrivals, exits, gave-up flag}; zero between launches (the kernel resets them on exit)
+  int* host_err;   // mapped pinned host word: set to 1 if a barrier wait ran out
+  RingPhase phase[NPH];
+  RingSeg seg[NSEG];
+};
+using RingArgsSmall = RingArgsT<kRingSmallPhases, kRingSmallSegs>;
+using RingArgsLarge = RingArgsT<kRingLargePhases, kRingLargeSegs>;
+// Largest cooperative grid of the ring kernel on the current device for the given thread count (512 or 1024).
+cudaError_t ring_max_grid(int threads, int dtype, bool large, int num_sms, int* grid);
+cudaError_t launch_ring(const RingArgsSmall& a, int grid, int threads, cudaStream_t stream);
+cudaError_t launch_ring(const RingArgsLarge& a, int grid, int threads, cudaStream_t stream);
+cudaError_t preload_ring_kernels();
+
 // Enqueue helpers (return the CUDA error of the launch).
 cudaError_t launch_sum(const SumBatch& batch, int ctas, cudaStream_t stream);
 cudaError_t launch_copy(const CopyBatch& batch, int ctas, cudaStream_t stream);

@@ -101,9 +101,13 @@ def sweep_sizes(args):
     torch.cuda.set_device(0)
     stream = torch.cuda.Stream()
     ops = ["allreduce", "reduce_scatter", "allgather", "alltoall", "sendrecv"] if args.ops == "all" else args.ops.split(",")
-    configs = [("CE", hb.PATH_CE, 8, 8), ("SM8", hb.PATH_SM, 8, 8), ("SMall", hb.PATH_SM, 148, 148)]
+    # name, path, SUM CTAs, copy CTAs, whole collective as one cooperative kernel
+    configs = [("CE", hb.PATH_CE, 8, 8, 0), ("SM8", hb.PATH_SM, 8, 8, 0), ("SMall", hb.PATH_SM, 148, 148, 0),
+               ("SM8fused", hb.PATH_SM, 8, 8, 1), ("SMallfused", hb.PATH_SM, 148, 148, 1)]
     if args.configs != "all":
         configs = [c for c in configs if c[0] in args.configs.split(",")]
+    else:
+        configs = configs[:3]
     out = open(args.out, "w") if args.out else None
     for dtype in args.dtypes.split(","):
         for R in [int(r) for r in args.ranks.split(",")]:
@@ -123,13 +127,14 @@ def sweep_sizes(args):
                     arena = Arena(op, R, S, dtype, nsets)
                     scratch = torch.empty(hb.scratch_bytes(R, S // e, dtype) + 256, dtype=torch.uint8, device="cuda")
                     pad = (-scratch.data_ptr()) % 256
-                    for name, path, sc, cc in configs:
+                    for name, path, sc, cc, fused in configs:
                         comm = hb.Comm(R, 0)
                         if scratch.numel() > 256:
                             comm.set_scratch(scratch.data_ptr() + pad, scratch.numel() - 256)
                         comm.set_path(path)
                         comm.set_param("sum_ctas", sc)
                         comm.set_param("copy_ctas", cc)
+                        comm.set_param("fused", fused)
                         t = time_op(comm, arena, stream)
                         row = {"op": op, "R": R, "dtype": dtype, "S": S, "config": name, "sum_ctas": sc,
                                "copy_ctas": cc if path == hb.PATH_SM else None, "us": t * 1e6, "algbw_GBps": S / t / 1e9,
