@@ -320,7 +320,7 @@ def main():
         },
         "sms_used": {"sum_ctas": int(rs_stats["max_sum_ctas"]), "moves": "driver copy route (see move_needs_sm)"},
         "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": R * S, "d2h_bytes_per_step": R * S,
-                "ms_per_step": t_e2e_slowest * 1e3, "call": "hoccl_host_allreduce (pinned host buffers)", "steps": k_e2e,
+                "ms_per_step": t_e2e_slowest * 1e3, "call": "hoccl_host_allreduce (pinned host buffers; inbound copies, ring and outbound copies pipelined over 8 pieces per chunk)", "steps": k_e2e,
                 "matches_oracle": e2e_ok},
         "gpu_launches": int(launches_per_step * steps),
         "clocks": clocks,

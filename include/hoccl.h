@@ -159,6 +159,7 @@ hoccl_result_t hoccl_comm_set_path(hoccl_comm_t comm, hoccl_path_t path);
  *                of pinned host memory of its own on first use (the third exception to "device memory is the caller's").
  *                Ignored on the other paths, in handshake mode, and for plans too large for one launch (more than 896
  *                chunk operations, i.e. beyond roughly 16 ranks), which run as a graph.  0 = off (default).
+ *  "host_pieces" pieces per ring chunk of the pipelined hoccl_host_allreduce (1..64, default 8; 1 = not pipelined)
  *  "use_graph"   1 = run a cached CUDA graph built from the plan (default), 0 = streams and events
  *  "handshake"   1 = the paper's stream manager (Sec. 3.2, Listing 1): instead of launching into the caller's
  *                stream, the call enqueues four stream memory operations (write start flag, wait for the CPU's
@@ -276,9 +277,16 @@ long hoccl_comm_handshakes(hoccl_comm_t comm);
 /*
  * All-reduce whose buffers are HOST memory (pinned for real asynchrony): h_send[r] / h_recv[r] are
  * host pointers to `count` elements each.  The call copies every h_send[r] into the attached staging
- * memory (needs 2*R*count*sizeof(dtype) bytes), runs hoccl_allreduce there and copies every rank's
- * result back, all enqueued on `stream`.  Host-to-device traffic is driven by the copy engines
- * (Sec. 2.3).  Errors: as hoccl_allreduce, SCRATCH if staging is missing or too small.
+ * memory (needs 2*R*roundup256(count*sizeof(dtype)) bytes), runs the all-reduce there and copies every rank's
+ * result back, all ordered on `stream`.  Host-to-device traffic is driven by the copy engines (Sec. 2.3).
+ * Pipelined form (default; "host_pieces" > 1 with graphs on): every ring chunk is cut into host_pieces pieces and ONE
+ * cached graph holds, per piece, the host-to-device copies (2-D copies: a piece of every chunk), the ring on that piece
+ * and the device-to-host copies, so that the inbound copies, the ring and the outbound copies of different pieces
+ * overlap (chunk pipelining, Sec. 3.3.1, applied across the PCIe link).  Chunk boundaries, and therefore every bit of
+ * the result, are those of hoccl_allreduce on the whole buffer.  Host buffers of different ranks must not overlap
+ * partially (INVALID_ARG); h_recv[r] == h_send[r] is legal.  With host_pieces = 1, use_graph = 0, handshake, onepass,
+ * fused or HOCCL_PATH_CE_HOST the three stages run one after the other.
+ * Errors: as hoccl_allreduce, SCRATCH if staging is missing or too small.
  */
 hoccl_result_t hoccl_host_allreduce(const void* const* h_send, void* const* h_recv, size_t count, hoccl_dtype_t dtype,
                                     hoccl_op_t op, hoccl_comm_t comm, hoccl_stream_t stream);

@@ -124,7 +124,8 @@ static long* param_slot(hoccl_comm* c, const char* key, long* lo, long* hi) {
               {"profile", &c->profile, 0, 1},           {"p2p_split", &c->p2p_split, 1, kMaxLanes},
               {"ce_sub_bytes", &c->ce_sub_bytes, 0, 1L << 40}, {"handshake", &c->handshake, 0, 1},
               {"watchdog_ms", &c->watchdog_ms, 10, 600000},    {"onepass", &c->onepass, 0, 1},
-              {"forward", &c->forward, 0, 1},           {"fused", &c->fused, 0, 1}};
+              {"forward", &c->forward, 0, 1},           {"fused", &c->fused, 0, 1},
+              {"host_pieces", &c->host_pieces, 1, 64}};
   for (auto& r : rows)
     if (std::strcmp(r.name, key) == 0) {
       *lo = r.lo;
@@ -242,8 +243,24 @@ hoccl_result_t hoccl_host_allreduce(const void* const* h_send, void* const* h_re
   for (int r = 0; r < R; r++) {
     dsend[r] = (char*)c->staging + (size_t)r * per;
     drecv[r] = (char*)c->staging + (size_t)(R + r) * per;
-    CU_TRY(c, cudaMemcpyAsync(const_cast<void*>(dsend[r]), h_send[r], count * e, cudaMemcpyHostToDevice, st));
   }
+  // Pipelined form: one graph holds, per piece of every ring chunk, the host-to-device copies, the ring on that piece and
+  // the device-to-host copies, so that the three overlap across pieces (PCIe is full duplex and the ring is short).
+  const bool pipelined = c->use_graph && c->host_pieces > 1 && !c->handshake && !c->onepass && c->path != HOCCL_PATH_CE_HOST &&
+                         !(c->fused && c->path == HOCCL_PATH_SM);
+  if (pipelined) {
+    // host buffers of different ranks must not overlap each other (a receive buffer is written while others are read)
+    for (int a = 0; a < R; a++)
+      for (int b = 0; b < R; b++) {
+        if (a < b && ranges_overlap((const char*)h_recv[a], count * e, (const char*)h_recv[b], count * e)) return HOCCL_ERR_INVALID_ARG;
+        if (h_send[a] != h_recv[b] && ranges_overlap((const char*)h_send[a], count * e, (const char*)h_recv[b], count * e)) return HOCCL_ERR_INVALID_ARG;
+      }
+    Call call{PLAN_ALLREDUCE, count, (int)dtype, false, count * e, count * e, dsend, drecv};
+    call.h_send = h_send;
+    call.h_recv = h_recv;
+    return run_collective(c, &call, st);
+  }
+  for (int r = 0; r < R; r++) CU_TRY(c, cudaMemcpyAsync(const_cast<void*>(dsend[r]), h_send[r], count * e, cudaMemcpyHostToDevice, st));
   hoccl_result_t rc = hoccl_allreduce(dsend, drecv, count, dtype, op, c, stream);
   if (rc != HOCCL_OK) return rc;
   for (int r = 0; r < R; r++) CU_TRY(c, cudaMemcpyAsync(h_recv[r], drecv[r], count * e, cudaMemcpyDeviceToHost, st));

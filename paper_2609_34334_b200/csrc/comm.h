@@ -52,6 +52,13 @@ struct Post {
   cudaStream_t stream;
 };
 
+// One host <-> staging copy of the pipelined host all-reduce: `rows` rows of `width` bytes at `pitch` (rows == 1: plain).
+struct HostCopy {
+  char* dev;
+  char* host;
+  size_t pitch, width, rows;
+};
+
 struct GraphEntry {
   std::vector<uint64_t> key;
   cudaGraphExec_t exec = nullptr;
@@ -60,6 +67,9 @@ struct GraphEntry {
   std::vector<std::pair<cudaEvent_t, cudaEvent_t>> prof_events;  // owned; only with profile = 1
   std::vector<double> prof_bytes;
   bool prof_pending = false;  // replayed since the profile events were last read
+  // pipelined host all-reduce: one graph per piece, and the host copies in front of and behind each of them
+  std::vector<cudaGraphExec_t> piece_exec;
+  std::vector<std::vector<HostCopy>> h2d, d2h;   // [piece]
   // "fused" setting: the whole plan as one cooperative kernel instead of a graph (exec stays null)
   std::vector<char> ring_args;  // a RingArgsSmall or RingArgsLarge, by value
   bool ring_large = false;
@@ -73,7 +83,7 @@ struct hoccl_comm {
   int R = 0, device = 0, num_sms = 0;
   hoccl_path_t path = HOCCL_PATH_CE;
   long sum_ctas = 8, copy_ctas = 8, piece_bytes = 4 << 20, max_pieces = 8, lanes = 4, use_graph = 1, profile = 0, p2p_split = 1, ce_sub_bytes = 0,
-       handshake = 0, watchdog_ms = 10000, onepass = 0, forward = 0, fused = 0;
+       handshake = 0, watchdog_ms = 10000, onepass = 0, forward = 0, fused = 0, host_pieces = 8;
   bool piece_bytes_set = false;  // the caller chose a piece size: no automatic choice
   hoccl::Proxy* proxy = nullptr;
   cudaStream_t lane[hoccl::kMaxLanes] = {};
@@ -141,6 +151,10 @@ struct Call {
   size_t send_bytes, recv_bytes;
   const void* const* send;
   void* const* recv;
+  // hoccl_host_allreduce, pipelined form: the caller's HOST buffers; send/recv then point into the device staging and
+  // the graph carries, per piece, the host-to-device copies in front of the ring and the device-to-host copies behind it
+  const void* const* h_send = nullptr;
+  void* const* h_recv = nullptr;
 };
 
 

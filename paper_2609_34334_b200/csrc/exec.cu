@@ -224,6 +224,9 @@ hoccl_result_t run_streams(hoccl_comm* c, const Plan& P, const std::vector<RGrou
 // ------------------------------------------------------------------ graph executor --------------
 void destroy_entry(GraphEntry* e) {
   if (e->exec) cudaGraphExecDestroy(e->exec);
+  for (cudaGraphExec_t pe : e->piece_exec)
+    if (pe) cudaGraphExecDestroy(pe);
+  e->piece_exec.clear();
   for (auto& p : e->prof_events) {
     cudaEventDestroy(p.first);
     cudaEventDestroy(p.second);
@@ -232,7 +235,41 @@ void destroy_entry(GraphEntry* e) {
   e->prof_events.clear();
 }
 
-hoccl_result_t build_graph(hoccl_comm* c, const Plan& P, const std::vector<RGroup>& groups, GraphEntry* entry) {
+// Host <-> staging copies of one piece of one rank (all-reduce layout): piece p of every ring chunk, i.e. rows of
+// `piece` bytes at a pitch of one chunk.  Chunks that hold the full piece go as one 2-D copy; a shorter trailing piece
+// as a 1-D copy.
+static void add_host_copies(const Plan& P, int p, char* dev, char* host, std::vector<HostCopy>* out) {
+  const size_t e = P.elem, q_bytes = P.chunk_elems * e;
+  const size_t off = (size_t)p * P.piece_bytes;
+  size_t full_rows = 0, full_len = 0;
+  for (int cidx = 0; cidx < P.R; cidx++) {
+    size_t lo, hi;
+    P.chunk_range(cidx, &lo, &hi);
+    const size_t len_bytes = (hi - lo) * e;
+    const size_t a = std::min(off, len_bytes), b = std::min(off + P.piece_bytes, len_bytes);
+    const size_t len = b - a;
+    if (len == 0) continue;
+    if (cidx == 0) full_len = len;
+    if (len == full_len && (size_t)cidx == full_rows) {
+      full_rows++;
+      continue;
+    }
+    out->push_back(HostCopy{dev + lo * e + a, host + lo * e + a, len, len, 1});
+  }
+  if (full_rows > 0) out->push_back(HostCopy{dev + off, host + off, q_bytes, full_len, full_rows});
+}
+
+static cudaError_t enqueue_host_copy(const HostCopy& hc, bool to_device, cudaStream_t s) {
+  const cudaMemcpyKind kind = to_device ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToHost;
+  void* dst = to_device ? (void*)hc.dev : (void*)hc.host;
+  const void* src = to_device ? (const void*)hc.host : (const void*)hc.dev;
+  if (hc.rows == 1) return cudaMemcpyAsync(dst, src, hc.width, kind, s);
+  return cudaMemcpy2DAsync(dst, hc.pitch, src, hc.pitch, hc.width, hc.rows, kind, s);
+}
+
+// only_piece >= 0 builds the graph of that piece alone (dependencies never cross pieces) and stores it in *out_exec.
+hoccl_result_t build_graph(hoccl_comm* c, const Plan& P, const std::vector<RGroup>& groups, GraphEntry* entry, int only_piece,
+                           cudaGraphExec_t* out_exec) {
   cudaGraph_t g = nullptr;
   CU_TRY(c, cudaGraphCreate(&g, 0));
   std::vector<cudaGraphNode_t> tail(groups.size(), nullptr);
@@ -242,6 +279,7 @@ hoccl_result_t build_graph(hoccl_comm* c, const Plan& P, const std::vector<RGrou
     rc = cuda_fail(c, e, what);
   };
   for (size_t gi = 0; gi < groups.size() && rc == HOCCL_OK; gi++) {
+    if (only_piece >= 0 && P.groups[gi].piece != only_piece) continue;
     const RGroup& rg = groups[gi];
     std::vector<cudaGraphNode_t> deps;
     for (int d : rg.deps)
@@ -359,7 +397,7 @@ hoccl_result_t build_graph(hoccl_comm* c, const Plan& P, const std::vector<RGrou
     }
   }
   if (rc == HOCCL_OK) {
-    cudaError_t e = cudaGraphInstantiate(&entry->exec, g, 0);
+    cudaError_t e = cudaGraphInstantiate(out_exec, g, 0);
     if (e != cudaSuccess) rc = cuda_fail(c, e, "cudaGraphInstantiate");
   }
   cudaGraphDestroy(g);
@@ -391,6 +429,12 @@ std::vector<uint64_t> make_key(hoccl_comm* c, const Call& call) {
     k.push_back((uint64_t)(uintptr_t)call.send[r]);
     k.push_back((uint64_t)(uintptr_t)call.recv[r]);
   }
+  k.push_back(call.h_send ? (uint64_t)c->host_pieces : 0);
+  if (call.h_send)
+    for (int r = 0; r < c->R; r++) {
+      k.push_back((uint64_t)(uintptr_t)call.h_send[r]);
+      k.push_back((uint64_t)(uintptr_t)call.h_recv[r]);
+    }
   return k;
 }
 
@@ -554,7 +598,38 @@ static hoccl_result_t launch_entry(hoccl_comm* c, GraphEntry* hit, cudaStream_t 
     c->stats.host_launch_us = now_us() - t0;
     return HOCCL_OK;
   }
-  if (c->handshake) {
+  if (!hit->piece_exec.empty()) {
+    // Pipelined host all-reduce: the inbound copies run on one internal stream, the outbound copies on another, and the
+    // caller's stream runs the ring piece by piece as each piece arrives; PCIe carries both directions at once.
+    cudaStream_t in = c->lane[0], out = c->lane[1];
+    c->ev_next = 0;
+    cudaEvent_t fork = next_event(c);
+    if (!fork) return cuda_fail(c, cudaErrorMemoryAllocation, "event pool");
+    CU_TRY(c, cudaEventRecord(fork, user));
+    CU_TRY(c, cudaStreamWaitEvent(in, fork, 0));
+    CU_TRY(c, cudaStreamWaitEvent(out, fork, 0));
+    const size_t np = hit->piece_exec.size();
+    std::vector<cudaEvent_t> arrived(np, nullptr);
+    for (size_t p = 0; p < np; p++) {
+      for (const HostCopy& hc : hit->h2d[p]) CU_TRY(c, enqueue_host_copy(hc, true, in));
+      arrived[p] = next_event(c);
+      if (!arrived[p]) return cuda_fail(c, cudaErrorMemoryAllocation, "event pool");
+      CU_TRY(c, cudaEventRecord(arrived[p], in));
+    }
+    for (size_t p = 0; p < np; p++) {
+      CU_TRY(c, cudaStreamWaitEvent(user, arrived[p], 0));
+      if (hit->piece_exec[p]) CU_TRY(c, cudaGraphLaunch(hit->piece_exec[p], user));
+      cudaEvent_t reduced = next_event(c);
+      if (!reduced) return cuda_fail(c, cudaErrorMemoryAllocation, "event pool");
+      CU_TRY(c, cudaEventRecord(reduced, user));
+      CU_TRY(c, cudaStreamWaitEvent(out, reduced, 0));
+      for (const HostCopy& hc : hit->d2h[p]) CU_TRY(c, enqueue_host_copy(hc, false, out));
+    }
+    cudaEvent_t done = next_event(c);
+    if (!done) return cuda_fail(c, cudaErrorMemoryAllocation, "event pool");
+    CU_TRY(c, cudaEventRecord(done, out));
+    CU_TRY(c, cudaStreamWaitEvent(user, done, 0));
+  } else if (c->handshake) {
     // paper Sec. 3.2: the stream hands itself to the CPU proxy, which runs the schedule and hands it back
     ProxyTask t;
     t.kind = ProxyTask::GRAPH;
@@ -580,7 +655,7 @@ hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
   if (dtype_size(call->dtype) == 0) return HOCCL_ERR_UNSUPPORTED;
   if (!call->send || !call->recv) return HOCCL_ERR_INVALID_ARG;
   const bool onepass_case = c->onepass && !c->handshake && (call->kind == PLAN_ALLREDUCE || call->kind == PLAN_REDUCE_SCATTER);
-  const bool fused = c->fused && c->path == HOCCL_PATH_SM && !c->handshake && !onepass_case;
+  const bool fused = c->fused && c->path == HOCCL_PATH_SM && !c->handshake && !onepass_case && !call->h_send;
   const bool graphs = (c->use_graph || c->handshake || fused) && !onepass_case;
   std::vector<uint64_t> key;
   if (graphs && call->count != 0) {
@@ -642,7 +717,12 @@ hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
   // CTAs), which does not pay with driver copies or whole-GPU grids.
   size_t piece_bytes = (size_t)c->piece_bytes;
   int max_pieces = (int)c->max_pieces;
-  if (fused) {   // one kernel walks the steps in order; whole chunks measured faster than pieces (fewer barriers and tails)
+  if (call->h_send) {   // pipelined host all-reduce: host_pieces pieces per chunk, whatever the chunk size
+    const size_t q = (call->count + c->R - 1) / c->R;
+    const size_t chunk = q * dtype_size(call->dtype);
+    max_pieces = (int)c->host_pieces;
+    piece_bytes = std::max<size_t>((size_t)64 << 10, ((chunk + max_pieces - 1) / max_pieces + 1023) / 1024 * 1024);
+  } else if (fused) {   // one kernel walks the steps in order; whole chunks measured faster than pieces (fewer barriers and tails)
     piece_bytes = (size_t)1 << 60;
     max_pieces = 1;
   } else if (!c->piece_bytes_set && c->path == HOCCL_PATH_SM && std::max(c->sum_ctas, c->copy_ctas) < 64 &&
@@ -679,9 +759,26 @@ hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
     GraphEntry entry;
     entry.key = key;
     entry.n_pieces = P.pieces;
-    rc = fused ? build_ring(c, P, groups, &entry) : HOCCL_ERR_UNSUPPORTED;
-    if (rc == HOCCL_ERR_UNSUPPORTED) rc = build_graph(c, P, groups, &entry);   // not asked for, or too many ranks for one launch
-    if (rc != HOCCL_OK) return rc;
+    if (call->h_send) {
+      entry.piece_exec.assign(P.pieces, nullptr);
+      entry.h2d.resize(P.pieces);
+      entry.d2h.resize(P.pieces);
+      for (int p = 0; p < P.pieces; p++) {
+        for (int r = 0; r < c->R; r++) {
+          add_host_copies(P, p, (char*)call->send[r], (char*)call->h_send[r], &entry.h2d[p]);
+          add_host_copies(P, p, (char*)call->recv[r], (char*)call->h_recv[r], &entry.d2h[p]);
+        }
+        bool any = false;
+        for (const PlanGroup& pg : P.groups) any = any || pg.piece == p;
+        if (!any) continue;   // e.g. one rank copying in place: nothing to run between the copies
+        rc = build_graph(c, P, groups, &entry, p, &entry.piece_exec[p]);
+        if (rc != HOCCL_OK) return rc;
+      }
+    } else {
+      rc = fused ? build_ring(c, P, groups, &entry) : HOCCL_ERR_UNSUPPORTED;
+      if (rc == HOCCL_ERR_UNSUPPORTED) rc = build_graph(c, P, groups, &entry, -1, &entry.exec);   // not asked for, or too many ranks for one launch
+      if (rc != HOCCL_OK) return rc;
+    }
     // handshake mode: place the graph on the device now; the proxy must not meet first-launch work later
     if (c->handshake) {
       cudaError_t ue = cudaGraphUpload(entry.exec, c->proxy->work_stream());
