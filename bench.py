@@ -261,6 +261,14 @@ def main():
     sampler = ClockSampler(dev)
     t_step, clocks = timed(comm, steps, warmup, sampler=sampler)
     st = comm.last_stats()
+    # spread: ten more windows of steps/10 steps each (median and best), same launch configuration
+    win = []
+    for _ in range(10):
+        tw, _ = timed(comm, max(5, steps // 10), 0)
+        win.append(tw * 1e3)
+    win.sort()
+    windows = {"n": 10, "steps_each": max(5, steps // 10), "median_ms_per_step": win[len(win) // 2], "best_ms_per_step": win[0],
+               "worst_ms_per_step": win[-1]}
     # launches of our kernels per step: the SUM launches of the reduce-scatter (the all-gather has none on this path)
     comm.reduce_scatter(send_sets[0], [recv_sets[0][r].data_ptr() + r * count * e for r in range(R)], count, dtype, stream)
     stream.synchronize()
@@ -325,6 +333,7 @@ def main():
         "gpu_launches": int(launches_per_step * steps),
         "clocks": clocks,
         "host_launch_us_per_call": st["host_launch_us"],
+        "windows": windows,
         "matches_oracle": parity,
         "peaks": peaks,
     }
@@ -368,7 +377,7 @@ def main():
         b2 = torch.empty(big, dtype=torch.bfloat16, device="cuda").normal_(0, 1e-3)
         o = torch.empty(big, dtype=torch.bfloat16, device="cuda")
         full = {}
-        for ctas in (8, 148, 296, 592):
+        for ctas in (8, 16, 32, 48, 64, 96, 128, 148, 296, 592):
             for _ in range(3):
                 hb.sum_launch(a, b2, o, big, dtype, ctas, stream)
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -381,7 +390,9 @@ def main():
             full[str(ctas)] = 3.0 * big * 2 / (e0.elapsed_time(e1) / 1e3 / reps) / 1e9
         line["roofline_unconstrained"] = {
             "kernel": "sum2_kernel<bf16>", "operands": "3 x 256 MiB, timed alone", "GBps_by_ctas": full,
-            "best_frac_of_measured": max(full.values()) / peaks["hbm_gbs"]}
+            "best_frac_of_measured": max(full.values()) / peaks["hbm_gbs"],
+            # the north star's "grid sized to the fewest SMs that still saturate HBM": first CTA count within 5 % of the best
+            "fewest_ctas_within_5pct_of_best": min(int(k_) for k_, v_ in full.items() if v_ >= 0.95 * max(full.values()))}
         del a, b2, o
 
     if world.rank == 0 and world.size == 1:

@@ -564,7 +564,7 @@ static hoccl_result_t build_ring(hoccl_comm* c, const Plan& P, const std::vector
   // CTA budget: never more than either budget of the SM path; never more CTAs than the largest phase has tiles for
   // (a barrier costs more the more CTAs take part); never more than can be resident together.
   long budget = has_sum ? std::min(c->sum_ctas, c->copy_ctas) : c->copy_ctas;
-  const int threads = budget >= 64 ? 512 : 1024;
+  const int threads = budget >= 128 ? 512 : 1024;
   const size_t tile_bytes = (size_t)threads * 4 * 16;
   const long tiles = (long)((max_phase_bytes + tile_bytes - 1) / tile_bytes);
   int max_grid = 0;

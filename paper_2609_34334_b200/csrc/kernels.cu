@@ -289,10 +289,14 @@ __global__ void __launch_bounds__(kThreads, 2) occupy_kernel(unsigned long long 
 
 }  // namespace
 
-// Launch shapes (measured on B200, 200 MiB operands): under a small CTA budget 1024 threads x 4 vectors per
-// operand in flight give 116 GB/s per SM (the mixed read/write ceiling of one SM's memory port is ~123 GB/s);
-// with the whole GPU 512 threads x 4 are a little faster (6.2 TB/s).
-static bool wide_grid(int ctas) { return ctas >= 64; }
+// Launch shapes (measured on B200, 256 MiB operands).  SUM: 1024 threads x 4 vectors per operand in flight give 116 GB/s
+// per SM under a small budget (the mixed read/write ceiling of one SM's memory port is ~123 GB/s) and reach 6.1 TB/s
+// (0.93 of the measured HBM peak) from 64 CTAs on; with 128 CTAs and more, 512 threads x 4 are a little faster
+// (6.35 against 6.1-6.2 TB/s).  Copy: 1024 threads x 8 vectors below 128 CTAs (5.5 TB/s at 64 CTAs); from 128 CTAs on
+// 512 x 4: on 256 MiB operands the two are equal there, but the four times smaller tile (32 KiB) balances the few-MB
+// chunks of a ring step over the grid (gradient bucket, whole GPU: 0.201 against 0.213 ms per step).
+static bool wide_grid(int ctas) { return ctas >= 128; }
+static bool wide_copy_grid(int ctas) { return ctas >= 128; }
 
 cudaError_t launch_sum(const SumBatch& batch, int ctas, cudaStream_t stream) {
   if (batch.nseg <= 0) return cudaSuccess;
@@ -308,7 +312,7 @@ cudaError_t launch_sum(const SumBatch& batch, int ctas, cudaStream_t stream) {
 
 cudaError_t launch_copy(const CopyBatch& batch, int ctas, cudaStream_t stream) {
   if (batch.nseg <= 0) return cudaSuccess;
-  if (wide_grid(ctas)) copy_kernel<4, 512><<<ctas, 512, 0, stream>>>(batch);
+  if (wide_copy_grid(ctas)) copy_kernel<4, 512><<<ctas, 512, 0, stream>>>(batch);
   else copy_kernel<8, 1024><<<ctas, 1024, 0, stream>>>(batch);
   return cudaGetLastError();
 }
@@ -333,8 +337,8 @@ const void* sum_kernel_entry(int dtype, int ctas, int* threads) {
   return wide_grid(ctas) ? reinterpret_cast<const void*>(&sum2_kernel<1, 4, 512>) : reinterpret_cast<const void*>(&sum2_kernel<1, 4, 1024>);
 }
 const void* copy_kernel_entry(int ctas, int* threads) {
-  *threads = wide_grid(ctas) ? 512 : 1024;
-  return wide_grid(ctas) ? reinterpret_cast<const void*>(&copy_kernel<4, 512>) : reinterpret_cast<const void*>(&copy_kernel<8, 1024>);
+  *threads = wide_copy_grid(ctas) ? 512 : 1024;
+  return wide_copy_grid(ctas) ? reinterpret_cast<const void*>(&copy_kernel<4, 512>) : reinterpret_cast<const void*>(&copy_kernel<8, 1024>);
 }
 
 // Forces the module that holds these kernels to be loaded now.  Loading a kernel on first launch can synchronise the

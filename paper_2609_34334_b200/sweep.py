@@ -3,7 +3,8 @@ pipeline / gradient-stream workloads (third and fourth), through the C ABI.
 
     python -m paper_2609_34334_b200.sweep sizes   [--min-log2 12 --max-log2 30 --ranks 2,4,8 --dtypes bf16 --ops all --out FILE]
     python -m paper_2609_34334_b200.sweep pipeline [--microbatches 16]
-    python -m paper_2609_34334_b200.sweep gradients [--buckets 32]
+    python -m paper_2609_34334_b200.sweep gradients [--buckets 32] [--budgets 1,2,4,8,16,32,64]
+    python -m paper_2609_34334_b200.sweep launch-cost
 
 Sizes are per-rank buffer bytes S in the nccl-tests convention (all-reduce: send = recv = S; reduce-scatter:
 send = S; all-gather: recv = S; all-to-all: send = recv = S; send/recv: S), like the sweeps the paper reports (Sec. 5 "Communication
@@ -297,8 +298,15 @@ def gradients(args):
     alone, _, _ = gemm_tflops(40)
     print(json.dumps({"workload": g.name, "buckets_total": len(sizes), "bucket_MiB": S >> 20, "last_bucket_MiB": sizes[-1] * 2 >> 20,
                       "gemm_probe": [M, K, N], "gemm_alone_TFLOPs": alone}), flush=True)
-    for name, path, sc, cc in (("CE_sum8", hb.PATH_CE, 8, 8), ("SM_copy8_sum8", hb.PATH_SM, 8, 8), ("SM_copy32_sum8", hb.PATH_SM, 8, 32),
-                               ("SM_copy148_sum148", hb.PATH_SM, 148, 148)):
+    configs = [("CE_sum8", hb.PATH_CE, 8, 8), ("SM_copy8_sum8", hb.PATH_SM, 8, 8), ("SM_copy32_sum8", hb.PATH_SM, 8, 32),
+               ("SM_copy148_sum148", hb.PATH_SM, 148, 148)]
+    if getattr(args, "budgets", ""):
+        # the copy-route path, then the SM-copy path under every CTA budget (SUM budget: the same, at most 8), then the whole GPU
+        configs = [("CE_sum8", hb.PATH_CE, 8, 8)]
+        for b in [int(x) for x in args.budgets.split(",")]:
+            configs.append(("SM_copy%d_sum%d" % (b, min(b, 8)), hb.PATH_SM, min(b, 8), b))
+        configs.append(("SM_copy148_sum148", hb.PATH_SM, 148, 148))
+    for name, path, sc, cc in configs:
         comm = hb.Comm(R, 0)
         comm.set_scratch(scratch.data_ptr() + pad, scratch.numel() - 256)
         comm.set_path(path)
@@ -326,6 +334,48 @@ def gradients(args):
         comm.destroy()
 
 
+def launch_cost(args):
+    """Host time of one all-reduce call against the number of operations it issues (the paper's CPU launch overhead
+    axis, Sec. 5): R = 8, 64 MiB bf16 per rank, chunks cut into 1..64 pieces, stream executor against graph replay, with
+    an idle queue (the stream is synchronised after every call)."""
+    torch.cuda.set_device(0)
+    R, dtype = 8, "bf16"
+    n = (64 << 20) // 2
+    stream = torch.cuda.Stream()
+    send = [torch.empty(n, dtype=torch.bfloat16, device="cuda").normal_(0, 1e-3) for _ in range(R)]
+    recv = [torch.empty(n, dtype=torch.bfloat16, device="cuda") for _ in range(R)]
+    scratch = torch.empty(hb.scratch_bytes(R, n, dtype) + 256, dtype=torch.uint8, device="cuda")
+    pad = (-scratch.data_ptr()) % 256
+    chunk = n * 2 // R
+    for path_name, path in (("CE", hb.PATH_CE), ("SM", hb.PATH_SM)):
+        for pieces in (1, 2, 4, 8, 16, 32, 64):
+            for label, use_graph in (("stream_executor", 0), ("graph_replay", 1)):
+                comm = hb.Comm(R, 0)
+                comm.set_scratch(scratch.data_ptr() + pad, scratch.numel() - 256)
+                comm.set_path(path)
+                comm.set_param("use_graph", use_graph)
+                comm.set_param("max_pieces", pieces)
+                comm.set_param("piece_bytes", max(1024, chunk // pieces))
+                vals, dev = [], []
+                for k in range(12):
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record(stream)
+                    comm.allreduce(send, recv, n, dtype, stream)
+                    e1.record(stream)
+                    st = comm.last_stats()
+                    stream.synchronize()
+                    if k >= 2:
+                        vals.append(st["host_launch_us"])
+                        dev.append(e0.elapsed_time(e1) * 1e3)
+                vals.sort()
+                dev.sort()
+                print(json.dumps({"path": path_name, "executor": label, "pieces_per_chunk": int(st["n_pieces"]),
+                                  "operations": int(st["n_moves"] + st["n_sum_launches"]), "moves": int(st["n_moves"]),
+                                  "sum_launches": int(st["n_sum_launches"]), "host_us_per_call_median": vals[len(vals) // 2],
+                                  "device_us_per_call_median": dev[len(dev) // 2]}), flush=True)
+                comm.destroy()
+
+
 def main():
     ap = argparse.ArgumentParser()
     sub = ap.add_subparsers(dest="cmd", required=True)
@@ -341,11 +391,13 @@ def main():
     p.add_argument("--microbatches", type=int, default=16)
     g = sub.add_parser("gradients")
     g.add_argument("--buckets", type=int, default=32)
+    g.add_argument("--budgets", default="", help="comma list of copy-kernel CTA budgets, e.g. 1,2,4,8,16,32,64")
+    sub.add_parser("launch-cost")
     args = ap.parse_args()
     if not torch.cuda.is_available():
         sys.stderr.write("sweep: no CUDA device\n")
         return 2
-    {"sizes": sweep_sizes, "pipeline": pipeline, "gradients": gradients}[args.cmd](args)
+    {"sizes": sweep_sizes, "pipeline": pipeline, "gradients": gradients, "launch-cost": launch_cost}[args.cmd](args)
     return 0
 
 
