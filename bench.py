@@ -436,6 +436,30 @@ def extras(hb, W, torch, np, new_comm, step, timed, stream, R, S, n, dtype, peak
                      "busbw_GBps": S * bus_factor(R) / t / 1e9, "hbm_frac_of_8TBps": hbm / t / 1e9 / NOMINAL_HBM_GBS})
         cm.destroy()
     out["variants"] = rows
+    # SM footprint of this library's kernels on the SM path (SMs x busy time per step), per-launch CUDA events in the graph
+    fp_rows = []
+    for sc, cc in ((8, 8), (8, 32), (148, 148)):
+        cm = new_comm(hb.PATH_SM, sum_ctas=sc, copy_ctas=cc, profile=1)
+        for b in range(4):
+            step(cm, b, stream)
+        stream.synchronize()
+        cm.profile_reset()
+        nst = 10
+        for b in range(nst):
+            step(cm, b % 4, stream)
+            stream.synchronize()
+            cm.last_stats()
+        ps = cm.last_stats()
+        sum_us = ps["sum_kernel_ms"] * 1e3 / nst
+        copy_us = ps["copy_kernel_ms"] * 1e3 / nst
+        fp_rows.append({"sum_ctas": sc, "copy_ctas": cc, "sum_busy_us_per_step": sum_us, "copy_busy_us_per_step": copy_us,
+                        "sum_launches_per_step": ps["sum_kernel_launches_timed"] / nst,
+                        "copy_launches_per_step": ps["copy_kernel_launches_timed"] / nst,
+                        "footprint_sm_us_per_step": sc * sum_us + cc * copy_us,
+                        "sum_GBps": ps["sum_kernel_bytes"] / max(ps["sum_kernel_ms"], 1e-9) / 1e6,
+                        "copy_GBps": ps["copy_kernel_bytes"] / max(ps["copy_kernel_ms"], 1e-9) / 1e6})
+        cm.destroy()
+    out["sm_path_footprint"] = fp_rows
     # one all-reduce call instead of two calls (all-gather of early pieces overlaps the last sums)
     cm = new_comm(hb.PATH_CE, sum_ctas=8)
 

@@ -91,6 +91,9 @@ typedef struct {
   double sum_kernel_ms;  /* with parameter "profile" = 1: total device time of SUM launches since hoccl_profile_reset */
   long sum_kernel_launches_timed;
   double sum_kernel_bytes; /* algorithmic bytes (2 reads + 1 write per element) of those launches */
+  double copy_kernel_ms;   /* the same for copy_kernel launches (SM path, graph executor) */
+  long copy_kernel_launches_timed;
+  double copy_kernel_bytes; /* algorithmic bytes (1 read + 1 write per byte) of those launches */
 } hoccl_stats_t;
 
 /* ---------------------------------------------------------------- communicator ----------------- */

@@ -475,6 +475,9 @@ hoccl_result_t hoccl_last_stats(hoccl_comm_t c, hoccl_stats_t* out) {
   out->sum_kernel_ms = c->prof_ms;
   out->sum_kernel_launches_timed = c->prof_n;
   out->sum_kernel_bytes = c->prof_bytes;
+  out->copy_kernel_ms = c->prof_copy_ms;
+  out->copy_kernel_launches_timed = c->prof_copy_n;
+  out->copy_kernel_bytes = c->prof_copy_bytes;
   return HOCCL_OK;
 }
 
@@ -484,6 +487,9 @@ hoccl_result_t hoccl_profile_reset(hoccl_comm_t c) {
   c->prof_ms = 0;
   c->prof_bytes = 0;
   c->prof_n = 0;
+  c->prof_copy_ms = 0;
+  c->prof_copy_bytes = 0;
+  c->prof_copy_n = 0;
   return HOCCL_OK;
 }
 

@@ -112,6 +112,8 @@ struct hoccl_comm {
   std::vector<std::pair<std::pair<cudaEvent_t, cudaEvent_t>, double>> prof_open;  // recorded, not yet read
   double prof_ms = 0, prof_bytes = 0;
   long prof_n = 0;
+  double prof_copy_ms = 0, prof_copy_bytes = 0;   // copy_kernel launches (graph executor)
+  long prof_copy_n = 0;
 };
 
 namespace hoccl {

@@ -371,9 +371,26 @@ hoccl_result_t build_graph(hoccl_comm* c, const Plan& P, const std::vector<RGrou
         // copy launches are chained as well: the CTA budget for copies is global, two never run at the same time
         std::vector<cudaGraphNode_t> d2 = deps;
         if (last_copy_node && std::find(d2.begin(), d2.end(), last_copy_node) == d2.end()) d2.push_back(last_copy_node);
+        std::pair<cudaEvent_t, cudaEvent_t> pe{nullptr, nullptr};
+        if (c->profile) {
+          if ((e = cudaEventCreate(&pe.first)) != cudaSuccess) break;
+          if ((e = cudaEventCreate(&pe.second)) != cudaSuccess) break;
+          entry->prof_events.push_back(pe);
+          double bytes = 0;
+          for (size_t i = 0; i < n; i++) bytes += 2.0 * (double)rg.segs[first + i].bytes;
+          entry->prof_bytes.push_back(-bytes);   // negative: a copy launch (read + write), kept apart from the sums
+          cudaGraphNode_t start_rec;
+          if ((e = cudaGraphAddEventRecordNode(&start_rec, g, d2.data(), d2.size(), pe.first)) != cudaSuccess) break;
+          d2.assign(1, start_rec);
+        }
         cudaGraphNode_t kn;
         e = cudaGraphAddKernelNode(&kn, g, d2.data(), d2.size(), &kp);
         if (e != cudaSuccess) break;
+        if (c->profile) {
+          cudaGraphNode_t end_rec;
+          if ((e = cudaGraphAddEventRecordNode(&end_rec, g, &kn, 1, pe.second)) != cudaSuccess) break;
+          kn = end_rec;
+        }
         last_copy_node = kn;
         nodes.push_back(kn);
         entry->n_moves += (long)n;
@@ -457,9 +474,15 @@ void harvest_profile(hoccl_comm* c) {
     for (size_t i = 0; i < e.prof_events.size(); i++) {
       float ms = 0;
       if (cudaEventElapsedTime(&ms, e.prof_events[i].first, e.prof_events[i].second) == cudaSuccess) {
-        c->prof_ms += ms;
-        c->prof_bytes += e.prof_bytes[i];
-        c->prof_n++;
+        if (e.prof_bytes[i] < 0) {
+          c->prof_copy_ms += ms;
+          c->prof_copy_bytes -= e.prof_bytes[i];
+          c->prof_copy_n++;
+        } else {
+          c->prof_ms += ms;
+          c->prof_bytes += e.prof_bytes[i];
+          c->prof_n++;
+        }
       }
     }
   }
