@@ -2,6 +2,7 @@
 
     python -m paper_2609_34334_b200.microbench --kernel sum --dtype bf16 --mib 200 --ctas 8 --reps 5
     python -m paper_2609_34334_b200.microbench --kernel routes --mib 16      # which same-device copy routes need an SM
+    python -m paper_2609_34334_b200.microbench --kernel ring --mib 32 --ctas 148   # all-reduce, R = 8, as one cooperative kernel
 
 Operands are larger than L2 by default; timing uses CUDA events on the launching stream after warm-up.
 Prints one JSON line.  This is the small case used for ncu captures of a single kernel.
@@ -18,7 +19,7 @@ from . import binding as hb
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--kernel", default="sum", choices=["sum", "copy", "routes"])
+    ap.add_argument("--kernel", default="sum", choices=["sum", "copy", "routes", "ring"])
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "fp32"])
     ap.add_argument("--mib", type=int, default=200, help="MiB per operand")
     ap.add_argument("--ctas", type=int, default=8)
@@ -27,6 +28,41 @@ def main():
     args = ap.parse_args()
     torch.cuda.set_device(0)
     nbytes = args.mib << 20
+    if args.kernel == "ring":
+        R = 8
+        e = 2 if args.dtype == "bf16" else 4
+        n = nbytes // e
+        tdt = torch.bfloat16 if args.dtype == "bf16" else torch.float32
+        send = [torch.empty(n, dtype=tdt, device="cuda").normal_(0, 1e-3) for _ in range(R)]
+        recv = [torch.empty(n, dtype=tdt, device="cuda") for _ in range(R)]
+        nb = hb.scratch_bytes(R, n, args.dtype)
+        scratch = torch.empty(nb + 256, dtype=torch.uint8, device="cuda")
+        comm = hb.Comm(R, 0)
+        comm.set_path(hb.PATH_SM)
+        comm.set_scratch(scratch.data_ptr() + (-scratch.data_ptr()) % 256, nb)
+        for k, v in (("fused", 1), ("sum_ctas", args.ctas), ("copy_ctas", args.ctas)):
+            comm.set_param(k, v)
+        st = torch.cuda.Stream()
+        for _ in range(args.warmup):
+            comm.allreduce(send, recv, n, args.dtype, st)
+        st.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(st)
+        for _ in range(args.reps):
+            comm.allreduce(send, recv, n, args.dtype, st)
+        e1.record(st)
+        st.synchronize()
+        sec = e0.elapsed_time(e1) / 1e3 / args.reps
+        moved = 7.0 * nbytes * (R - 1)
+        assert all(torch.equal(recv[0], recv[r]) for r in range(1, R)), "ranks disagree"
+        assert comm.async_error() == hb.OK
+        stats = comm.last_stats()
+        print(json.dumps({"kernel": "ring_kernel (all-reduce, R = 8, one cooperative launch)", "dtype": args.dtype,
+                          "mib_per_rank": args.mib, "ctas": int(stats["max_copy_ctas"]), "us_per_launch": sec * 1e6,
+                          "algorithmic_bytes_per_launch": moved, "GBps": moved / sec / 1e9,
+                          "busbw_GBps": nbytes * 2 * (R - 1) / R / sec / 1e9}))
+        comm.destroy()
+        return
     if args.kernel == "routes":
         src = torch.full((nbytes,), 7, dtype=torch.uint8, device="cuda")
         dst = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")
