@@ -155,9 +155,11 @@ hoccl_result_t hoccl_comm_set_path(hoccl_comm_t comm, hoccl_path_t path);
  *                grid-wide barrier between dependent steps (how an SM-driven library runs a collective: the paper's
  *                "NCCL under an SM budget" baseline, Sec. 5).  The schedule stays rank local and the bits are the same.
  *                Its grid is min(sum_ctas, copy_ctas) CTAs (copy_ctas for pure moves), fewer for small messages.
- *                Measured on B200: a grid barrier costs about what a kernel boundary inside a CUDA graph costs, so small
- *                messages gain nothing; with the whole GPU, messages of 128 MiB and more run 7-20 % faster (no ramp and
- *                tail per step).  Every barrier wait is bounded; a wait that runs out ends the kernel and is reported by
+ *                Measured on B200 (R = 8, bf16, whole GPU): a step inside the kernel costs ~4.6 us against ~2.7 us for a
+ *                kernel boundary inside a CUDA graph, so messages below 256 KiB per rank are slower this way; from 256 KiB
+ *                to 16 MiB and from 128 MiB on it is 8-21 % faster (no ramp and tail per step), in between equal.  Under an
+ *                8-CTA budget the graph is faster from 8 MiB on, because it overlaps a copy kernel with a sum kernel.
+ *                Every barrier wait is bounded; a wait that runs out ends the kernel and is reported by
  *                hoccl_comm_async_error as HOCCL_ERR_TIMEOUT.  The library allocates 16 bytes of device memory and 4 bytes
  *                of pinned host memory of its own on first use (the third exception to "device memory is the caller's").
  *                Ignored on the other paths, in handshake mode, and for plans too large for one launch (more than 896

@@ -9,7 +9,7 @@
 // started.
 //
 // Data written by one CTA in a phase is read by another CTA in a later phase: stores are followed by __threadfence()
-// before the arrival, the poll is an acquire load, and operands are loaded with ld.global.cg (L2, never a stale L1 line).
+// before the arrival (a release reduction), the poll is an acquire load (measured faster than relaxed polls plus one fence), and operands are loaded with ld.global.cg (L2, never a stale L1 line).
 #include <cuda_bf16.h>
 
 #include "device_common.cuh"
@@ -28,8 +28,8 @@ __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
 __device__ __forceinline__ bool grid_barrier(unsigned* bar, unsigned target, int* host_err, int* s_bail) {
   __syncthreads();
   if (threadIdx.x == 0) {
-    __threadfence();
-    atomicAdd(&bar[0], 1u);
+    // release: everything this CTA wrote (ordered before by the bar.sync above) is visible to whoever sees the arrival
+    asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(bar) : "memory");
     bool ok = true;
     unsigned it = 0;
     while (ld_acquire_u32(&bar[0]) < target) {
@@ -44,10 +44,34 @@ __device__ __forceinline__ bool grid_barrier(unsigned* bar, unsigned target, int
       *reinterpret_cast<volatile int*>(host_err) = 1;
       *s_bail = 1;
     }
-    __threadfence();
   }
   __syncthreads();
   return *reinterpret_cast<volatile int*>(s_bail) == 0;
+}
+
+// Prefix sums over the (at most 32) segments of a phase by the first warp: tile counts and element-wise item counts.
+// Every thread of the CTA calls it; lanes >= nseg contribute zero.  Ends with the CTA barrier that publishes the view.
+__device__ __forceinline__ void flatten_prefix(Flat& f, int nseg, unsigned long long my_tiles, unsigned long long my_scalars) {
+  if (threadIdx.x < 32) {
+    unsigned long long t = my_tiles, s = my_scalars;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const unsigned long long tu = __shfl_up_sync(0xffffffffu, t, d), su = __shfl_up_sync(0xffffffffu, s, d);
+      if ((int)threadIdx.x >= d) {
+        t += tu;
+        s += su;
+      }
+    }
+    if (threadIdx.x == 0) {
+      f.tpre[0] = 0;
+      f.spre[0] = 0;
+    }
+    if ((int)threadIdx.x < nseg) {
+      f.tpre[threadIdx.x + 1] = t;
+      f.spre[threadIdx.x + 1] = s;
+    }
+  }
+  __syncthreads();
 }
 
 // element-wise add with L2 loads (heads, tails and segments without a common 16-byte phase)
@@ -65,6 +89,7 @@ __device__ __forceinline__ void add_scalar_cg(const void* a, const void* b, void
 template <int DT, int U>
 __device__ __forceinline__ void sum_phase(Flat& f, const RingSeg* seg, int nseg) {
   using T = Traits<DT>;
+  unsigned long long my_tiles = 0, my_scalars = 0;
   if ((int)threadIdx.x < nseg) {
     const RingSeg& s = seg[threadIdx.x];
     unsigned ma = (unsigned)((uintptr_t)s.src & 15), mb = (unsigned)((uintptr_t)s.local & 15), mo = (unsigned)((uintptr_t)s.dst & 15);
@@ -73,22 +98,10 @@ __device__ __forceinline__ void sum_phase(Flat& f, const RingSeg* seg, int nseg)
     split_segment(s.bytes / T::E, ma, ma == mb && mb == mo, T::E, T::VE, &h, &nv, &ns);
     f.head[threadIdx.x] = h;
     f.nvec[threadIdx.x] = nv;
-    f.spre[threadIdx.x + 1] = ns;
+    my_tiles = (nv + (unsigned long long)U * blockDim.x - 1) / ((unsigned long long)U * blockDim.x);
+    my_scalars = ns;
   }
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    unsigned long long t = 0, s = 0;
-    const unsigned long long tile_v = (unsigned long long)U * blockDim.x;
-    f.tpre[0] = 0;
-    f.spre[0] = 0;
-    for (int k = 0; k < nseg; k++) {
-      t += (f.nvec[k] + tile_v - 1) / tile_v;
-      f.tpre[k + 1] = t;
-      s += f.spre[k + 1];
-      f.spre[k + 1] = s;
-    }
-  }
-  __syncthreads();
+  flatten_prefix(f, nseg, my_tiles, my_scalars);
   {
     const unsigned long long T_all = f.tpre[nseg];
     const unsigned tile_v = U * blockDim.x;
@@ -131,6 +144,7 @@ __device__ __forceinline__ void sum_phase(Flat& f, const RingSeg* seg, int nseg)
 
 template <int U>
 __device__ __forceinline__ void copy_phase(Flat& f, const RingSeg* seg, int nseg) {
+  unsigned long long my_tiles = 0, my_scalars = 0;
   if ((int)threadIdx.x < nseg) {
     const RingSeg& s = seg[threadIdx.x];
     unsigned ms = (unsigned)((uintptr_t)s.src & 15), md = (unsigned)((uintptr_t)s.dst & 15);
@@ -139,22 +153,10 @@ __device__ __forceinline__ void copy_phase(Flat& f, const RingSeg* seg, int nseg
     split_segment(s.bytes, ms, ms == md, 1, 16, &h, &nv, &ns);
     f.head[threadIdx.x] = h;
     f.nvec[threadIdx.x] = nv;
-    f.spre[threadIdx.x + 1] = ns;
+    my_tiles = (nv + (unsigned long long)U * blockDim.x - 1) / ((unsigned long long)U * blockDim.x);
+    my_scalars = ns;
   }
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    unsigned long long t = 0, s = 0;
-    const unsigned long long tile_v = (unsigned long long)U * blockDim.x;
-    f.tpre[0] = 0;
-    f.spre[0] = 0;
-    for (int k = 0; k < nseg; k++) {
-      t += (f.nvec[k] + tile_v - 1) / tile_v;
-      f.tpre[k + 1] = t;
-      s += f.spre[k + 1];
-      f.spre[k + 1] = s;
-    }
-  }
-  __syncthreads();
+  flatten_prefix(f, nseg, my_tiles, my_scalars);
   {
     const unsigned long long T_all = f.tpre[nseg];
     const unsigned tile_v = U * blockDim.x;
