@@ -316,26 +316,52 @@ hoccl_result_t hoccl_alltoallv(const void* const* send, const size_t* sendcounts
   long moves = 0, launches = 0;
   for (size_t si = 0; si < S.stages.size(); si++) {
     const Stage& st = S.stages[si];
-    // every DMA queue (one per source rank) is a serial chain on its lane, in the interleaved chunk order
-    for (int g = 0; g < R; g++) {
-      cudaStream_t lane = c->lane[g % lanes];
-      for (const ChunkItem& it : st.queues[g]) {
-        const StageFlow& f = st.flows[it.flow];
-        const size_t so = sdispls[(size_t)f.origin_src * R + f.origin_dst] * e + f.origin_offset + it.offset;
-        const size_t dofs = rdispls[(size_t)f.origin_dst * R + f.origin_src] * e + f.origin_offset + it.offset;
-        const char* src = (const char*)send[f.origin_src] + so;
-        char* dst = (char*)recv[f.origin_dst] + dofs;
-        if (c->path == HOCCL_PATH_CE) {
+    auto endpoints = [&](const ChunkItem& it, const char** src, char** dst) {
+      const StageFlow& f = st.flows[it.flow];
+      const size_t so = sdispls[(size_t)f.origin_src * R + f.origin_dst] * e + f.origin_offset + it.offset;
+      const size_t dofs = rdispls[(size_t)f.origin_dst * R + f.origin_src] * e + f.origin_offset + it.offset;
+      *src = (const char*)send[f.origin_src] + so;
+      *dst = (char*)recv[f.origin_dst] + dofs;
+    };
+    if (c->path == HOCCL_PATH_CE) {
+      // every DMA queue (one per source rank) is a serial chain on its lane, in the interleaved chunk order
+      for (int g = 0; g < R; g++) {
+        cudaStream_t lane = c->lane[g % lanes];
+        for (const ChunkItem& it : st.queues[g]) {
+          const char* src;
+          char* dst;
+          endpoints(it, &src, &dst);
           CU_TRY(c, cudaMemcpyAsync(dst, src, it.bytes, cudaMemcpyDeviceToDevice, lane));
-        } else {
-          CopyBatch b;
-          b.nseg = 1;
-          b.pad = 0;
-          b.seg[0] = CopySeg{src, dst, (unsigned long long)it.bytes};
-          CU_TRY(c, launch_copy(b, (int)c->copy_ctas, lane));
+          moves++;
+        }
+      }
+    } else {
+      // SM path: the k-th chunk of every queue goes into one batched copy launch (the queues advance in lock step,
+      // which is what R engines of equal speed would do), so a stage costs as many launches as its longest queue
+      size_t depth = 0;
+      for (int g = 0; g < R; g++) depth = std::max(depth, st.queues[g].size());
+      for (size_t k = 0; k < depth; k++) {
+        CopyBatch b;
+        b.nseg = 0;
+        b.pad = 0;
+        for (int g = 0; g < R; g++) {
+          if (k >= st.queues[g].size()) continue;
+          const ChunkItem& it = st.queues[g][k];
+          const char* src;
+          char* dst;
+          endpoints(it, &src, &dst);
+          b.seg[b.nseg++] = CopySeg{src, dst, (unsigned long long)it.bytes};
+          moves++;
+          if (b.nseg == kMaxSegs) {
+            CU_TRY(c, launch_copy(b, (int)c->copy_ctas, c->lane[0]));
+            launches++;
+            b.nseg = 0;
+          }
+        }
+        if (b.nseg > 0) {
+          CU_TRY(c, launch_copy(b, (int)c->copy_ctas, c->lane[0]));
           launches++;
         }
-        moves++;
       }
     }
     // stages run one after the other (the paper's serial stages): barrier over the lanes
