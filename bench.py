@@ -421,6 +421,47 @@ def main():
     return 0
 
 
+def small_case(hb, W, torch, np, stream):
+    """The small configuration (all-reduce over R = 4, 1,048,576 fp32 per rank, uniform[-1,1), seed 0): latency bound
+    (its algorithmic bytes take 11 us at 8 TB/s).  Time per call on both paths; the result is checked against the oracle."""
+    from oracle import ring as oracle_ring
+    c = W.C1_SMALL_ALLREDUCE
+    R, n = c.R, c.count
+    xs = W.rank_inputs(c.dist, c.seed, R, n, c.dtype)
+    want = oracle_ring.ring_allreduce(xs, threads=oracle_ring.max_threads())
+    sets = 8      # 8 x 32 MiB of buffers in rotation: larger than L2
+    send = [[torch.from_numpy(x).cuda() for x in xs] for _ in range(sets)]
+    recv = [[torch.zeros(n, dtype=torch.float32, device="cuda") for _ in range(R)] for _ in range(sets)]
+    nb = hb.scratch_bytes(R, n, c.dtype)
+    scratch = torch.empty(nb + 256, dtype=torch.uint8, device="cuda")
+    rows = {}
+    for name, path, ctas, fused in (("CE_sum8", hb.PATH_CE, 8, 0), ("SM_8", hb.PATH_SM, 8, 0), ("SM_148", hb.PATH_SM, 148, 0),
+                                    ("SM_148_one_kernel", hb.PATH_SM, 148, 1)):
+        cm = hb.Comm(R, 0)
+        cm.set_scratch(scratch.data_ptr() + (-scratch.data_ptr()) % 256, nb)
+        cm.set_path(path)
+        for key, v in (("sum_ctas", ctas), ("copy_ctas", ctas), ("fused", fused)):
+            cm.set_param(key, v)
+        for b in range(sets):
+            cm.allreduce(send[b], recv[b], n, c.dtype, stream)
+        stream.synchronize()
+        ok = all(bool((recv[0][r].cpu().numpy().view(np.uint32) == want[r].view(np.uint32)).all()) for r in range(R))
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        reps = 200
+        e0.record(stream)
+        for i in range(reps):
+            cm.allreduce(send[i % sets], recv[i % sets], n, c.dtype, stream)
+        e1.record(stream)
+        stream.synchronize()
+        t = e0.elapsed_time(e1) / 1e3 / reps
+        S1 = n * 4
+        rows[name] = {"us_per_call": t * 1e6, "busbw_GBps": S1 * 2 * (R - 1) / R / t / 1e9,
+                      "hbm_frac_of_8TBps": 7.0 * S1 * (R - 1) / t / 1e9 / NOMINAL_HBM_GBS, "matches_oracle": ok}
+        cm.destroy()
+    rows["workload"] = c.name
+    return rows
+
+
 def extras(hb, W, torch, np, new_comm, step, timed, stream, R, S, n, dtype, peaks, send_sets, recv_sets):
     """Context lines: path / CTA-budget variants, whether a move needs an SM, p2p, and the co-running GEMM probe."""
     out = {}
@@ -619,6 +660,7 @@ def extras(hb, W, torch, np, new_comm, step, timed, stream, R, S, n, dtype, peak
         probe[name] = {"gemm_TFLOPs": tf, "loss": 1.0 - tf / alone, "comm_busbw_GBps": bw}
         c2.destroy()
     out["gemm_probe_4096"] = probe
+    out["c1_small_allreduce"] = small_case(hb, W, torch, np, stream)
     cm.destroy()
     return out
 
