@@ -43,7 +43,7 @@ __global__ void __launch_bounds__(THREADS, 1) sum2_kernel(const __grid_constant_
   __syncthreads();
   if (threadIdx.x == 0) {
     unsigned long long t = 0, s = 0;
-    const unsigned long long tile_v = (unsigned long long)U * blockDim.x;
+    constexpr unsigned long long tile_v = (unsigned long long)U * THREADS;   // the launch helpers use THREADS threads: a shift, not a division
     f.tpre[0] = 0;
     f.spre[0] = 0;
     for (int k = 0; k < nseg; k++) {
@@ -128,7 +128,7 @@ __global__ void __launch_bounds__(THREADS, 1) copy_kernel(const __grid_constant_
   __syncthreads();
   if (threadIdx.x == 0) {
     unsigned long long t = 0, s = 0;
-    const unsigned long long tile_v = (unsigned long long)U * blockDim.x;
+    constexpr unsigned long long tile_v = (unsigned long long)U * THREADS;   // the launch helpers use THREADS threads: a shift, not a division
     f.tpre[0] = 0;
     f.spre[0] = 0;
     for (int k = 0; k < nseg; k++) {

@@ -86,7 +86,7 @@ __device__ __forceinline__ void add_scalar_cg(const void* a, const void* b, void
   }
 }
 
-template <int DT, int U>
+template <int DT, int U, int THREADS>
 __device__ __forceinline__ void sum_phase(Flat& f, const RingSeg* seg, int nseg) {
   using T = Traits<DT>;
   unsigned long long my_tiles = 0, my_scalars = 0;
@@ -98,7 +98,7 @@ __device__ __forceinline__ void sum_phase(Flat& f, const RingSeg* seg, int nseg)
     split_segment(s.bytes / T::E, ma, ma == mb && mb == mo, T::E, T::VE, &h, &nv, &ns);
     f.head[threadIdx.x] = h;
     f.nvec[threadIdx.x] = nv;
-    my_tiles = (nv + (unsigned long long)U * blockDim.x - 1) / ((unsigned long long)U * blockDim.x);
+    my_tiles = (nv + (unsigned long long)U * THREADS - 1) / ((unsigned long long)U * THREADS);   // a shift
     my_scalars = ns;
   }
   flatten_prefix(f, nseg, my_tiles, my_scalars);
@@ -142,7 +142,7 @@ __device__ __forceinline__ void sum_phase(Flat& f, const RingSeg* seg, int nseg)
   }
 }
 
-template <int U>
+template <int U, int THREADS>
 __device__ __forceinline__ void copy_phase(Flat& f, const RingSeg* seg, int nseg) {
   unsigned long long my_tiles = 0, my_scalars = 0;
   if ((int)threadIdx.x < nseg) {
@@ -153,7 +153,7 @@ __device__ __forceinline__ void copy_phase(Flat& f, const RingSeg* seg, int nseg
     split_segment(s.bytes, ms, ms == md, 1, 16, &h, &nv, &ns);
     f.head[threadIdx.x] = h;
     f.nvec[threadIdx.x] = nv;
-    my_tiles = (nv + (unsigned long long)U * blockDim.x - 1) / ((unsigned long long)U * blockDim.x);
+    my_tiles = (nv + (unsigned long long)U * THREADS - 1) / ((unsigned long long)U * THREADS);   // a shift
     my_scalars = ns;
   }
   flatten_prefix(f, nseg, my_tiles, my_scalars);
@@ -208,8 +208,8 @@ __global__ void __launch_bounds__(THREADS, 1) ring_kernel(const __grid_constant_
     } else {
       __syncthreads();   // the flattened view of the previous phase is about to be overwritten
     }
-    if (P.kind == 1) sum_phase<DT, 4>(f, a.seg + P.first_seg, P.nseg);
-    else copy_phase<(THREADS == 1024 ? 8 : 4)>(f, a.seg + P.first_seg, P.nseg);
+    if (P.kind == 1) sum_phase<DT, 4, THREADS>(f, a.seg + P.first_seg, P.nseg);
+    else copy_phase<(THREADS == 1024 ? 8 : 4), THREADS>(f, a.seg + P.first_seg, P.nseg);
   }
   // leave: the last CTA out clears the barrier words, so that the next launch starts from zero even after a give-up
   __syncthreads();
