@@ -520,7 +520,7 @@ def extras(hb, W, torch, np, new_comm, step, timed, stream, R, S, n, dtype, peak
     out["onepass_allreduce"] = op_rows
     # second comparison point: fused sum-and-forward (a SUM stores into the next rank's inbox; moves only at step 0)
     fw_rows = []
-    for name, path, sc, cc in (("CE", hb.PATH_CE, 8, 8), ("SM", hb.PATH_SM, 148, 148)):
+    for name, path, sc, cc in (("CE", hb.PATH_CE, 8, 8), ("SM", hb.PATH_SM, 8, 8), ("SM", hb.PATH_SM, 148, 148)):
         c1 = new_comm(path, sum_ctas=sc, copy_ctas=cc, forward=1)
         t, _ = timed(c1, k, w)
         fw_rows.append({"path": name, "sum_ctas": sc, "ms_per_step": t * 1e3, "busbw_GBps": S * bus_factor(R) / t / 1e9})
@@ -650,10 +650,11 @@ def extras(hb, W, torch, np, new_comm, step, timed, stream, R, S, n, dtype, peak
     probe = {}
     alone, _ = gemm_tflops(None)
     probe["alone_TFLOPs"] = alone
-    for name, path, sc, cc, op in (("CE_sum8", hb.PATH_CE, 8, 8, 0), ("SM_copy8_sum8", hb.PATH_SM, 8, 8, 0),
-                                   ("SM_copy32_sum8", hb.PATH_SM, 8, 32, 0), ("SM_copy148_sum148", hb.PATH_SM, 148, 148, 0),
-                                   ("onepass_8", hb.PATH_CE, 8, 8, 1), ("CE_HOST_sum8", hb.PATH_CE_HOST, 8, 8, 0)):
-        c2 = new_comm(path, sum_ctas=sc, copy_ctas=cc, onepass=op)
+    for name, path, sc, cc, op, fw in (("CE_sum8", hb.PATH_CE, 8, 8, 0, 0), ("SM_copy8_sum8", hb.PATH_SM, 8, 8, 0, 0),
+                                       ("SM_copy32_sum8", hb.PATH_SM, 8, 32, 0, 0), ("SM_copy148_sum148", hb.PATH_SM, 148, 148, 0, 0),
+                                       ("SM_forward_copy8_sum8", hb.PATH_SM, 8, 8, 0, 1),
+                                       ("onepass_8", hb.PATH_CE, 8, 8, 1, 0), ("CE_HOST_sum8", hb.PATH_CE_HOST, 8, 8, 0, 0)):
+        c2 = new_comm(path, sum_ctas=sc, copy_ctas=cc, onepass=op, forward=fw)
         if path == hb.PATH_CE_HOST:
             c2.set_host_staging(host_stage)
         tf, bw = gemm_tflops(c2)
