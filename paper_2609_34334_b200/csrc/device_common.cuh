@@ -57,16 +57,7 @@ struct Traits<1> {  // bf16
   }
 };
 
-// Flattened view of the batch, built once per CTA in shared memory.
-struct Flat {
-  unsigned long long tpre[kMaxSegs + 1];  // prefix sums of vector tiles (sum kernel)
-  unsigned long long vpre[kMaxSegs + 1];  // prefix sums of 16-byte vectors
-  unsigned long long spre[kMaxSegs + 1];  // prefix sums of element-wise items
-  unsigned long long nvec[kMaxSegs];
-  unsigned int head[kMaxSegs];            // element-wise items before the vector body
-};
-
-__device__ __forceinline__ void split_segment(unsigned long long n, unsigned mis, bool congruent, int E, int VE,
+__host__ __device__ __forceinline__ void split_segment(unsigned long long n, unsigned mis, bool congruent, int E, int VE,
                                               unsigned* head, unsigned long long* nvec, unsigned long long* nscalar) {
   if (congruent && (mis % E) == 0) {
     unsigned long long h = ((16u - mis) & 15u) / E;

@@ -293,6 +293,7 @@ hoccl_result_t build_graph(hoccl_comm* c, const Plan& P, const std::vector<RGrou
         size_t n = std::min<size_t>(kMaxSegs, rg.segs.size() - first);
         SumBatch b;
         fill_sum_batch(rg, first, n, P.dtype, P.elem, &b);
+        prepare_sum_batch(&b, (int)c->sum_ctas);
         void* args[] = {&b};
         cudaKernelNodeParams kp = {};
         int sum_threads = 0;
@@ -361,6 +362,7 @@ hoccl_result_t build_graph(hoccl_comm* c, const Plan& P, const std::vector<RGrou
         size_t n = std::min<size_t>(kMaxSegs, rg.segs.size() - first);
         CopyBatch b;
         fill_copy_batch(rg, first, n, &b);
+        prepare_copy_batch(&b, (int)c->copy_ctas);
         void* args[] = {&b};
         cudaKernelNodeParams kp = {};
         int copy_threads = 0;

@@ -27,33 +27,8 @@ namespace {
 template <int DT, int U, int THREADS>
 __global__ void __launch_bounds__(THREADS, 1) sum2_kernel(const __grid_constant__ SumBatch batch) {
   using T = Traits<DT>;
-  __shared__ Flat f;
+  const Flat& f = batch.flat;   // filled on the host for this kernel variant: no set-up phase, no barrier
   const int nseg = batch.nseg;
-  if ((int)threadIdx.x < nseg) {
-    const SumSeg& s = batch.seg[threadIdx.x];
-    unsigned ma = (unsigned)((uintptr_t)s.inbox & 15), mb = (unsigned)((uintptr_t)s.local & 15),
-             mo = (unsigned)((uintptr_t)s.out & 15);
-    unsigned long long nv, ns;
-    unsigned h;
-    split_segment(s.n, ma, ma == mb && mb == mo, T::E, T::VE, &h, &nv, &ns);
-    f.head[threadIdx.x] = h;
-    f.nvec[threadIdx.x] = nv;
-    f.spre[threadIdx.x + 1] = ns;
-  }
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    unsigned long long t = 0, s = 0;
-    constexpr unsigned long long tile_v = (unsigned long long)U * THREADS;   // the launch helpers use THREADS threads: a shift, not a division
-    f.tpre[0] = 0;
-    f.spre[0] = 0;
-    for (int k = 0; k < nseg; k++) {
-      t += (f.nvec[k] + tile_v - 1) / tile_v;
-      f.tpre[k + 1] = t;
-      s += f.spre[k + 1];
-      f.spre[k + 1] = s;
-    }
-  }
-  __syncthreads();
   const unsigned long long total = (unsigned long long)gridDim.x * blockDim.x;
   const unsigned long long gt = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
 
@@ -113,32 +88,8 @@ __global__ void __launch_bounds__(THREADS, 1) sum2_kernel(const __grid_constant_
 
 template <int U, int THREADS>
 __global__ void __launch_bounds__(THREADS, 1) copy_kernel(const __grid_constant__ CopyBatch batch) {
-  __shared__ Flat f;
+  const Flat& f = batch.flat;
   const int nseg = batch.nseg;
-  if ((int)threadIdx.x < nseg) {
-    const CopySeg& s = batch.seg[threadIdx.x];
-    unsigned ms = (unsigned)((uintptr_t)s.src & 15), md = (unsigned)((uintptr_t)s.dst & 15);
-    unsigned long long nv, ns;
-    unsigned h;
-    split_segment(s.bytes, ms, ms == md, 1, 16, &h, &nv, &ns);
-    f.head[threadIdx.x] = h;
-    f.nvec[threadIdx.x] = nv;
-    f.spre[threadIdx.x + 1] = ns;
-  }
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    unsigned long long t = 0, s = 0;
-    constexpr unsigned long long tile_v = (unsigned long long)U * THREADS;   // the launch helpers use THREADS threads: a shift, not a division
-    f.tpre[0] = 0;
-    f.spre[0] = 0;
-    for (int k = 0; k < nseg; k++) {
-      t += (f.nvec[k] + tile_v - 1) / tile_v;
-      f.tpre[k + 1] = t;
-      s += f.spre[k + 1];
-      f.spre[k + 1] = s;
-    }
-  }
-  __syncthreads();
   const unsigned long long total = (unsigned long long)gridDim.x * blockDim.x;
   const unsigned long long gt = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
   {
@@ -298,22 +249,68 @@ __global__ void __launch_bounds__(kThreads, 2) occupy_kernel(unsigned long long 
 static bool wide_grid(int ctas) { return ctas >= 128; }
 static bool wide_copy_grid(int ctas) { return ctas >= 128; }
 
+// Host side of the flattened view (same split as the device helper; tile = 4 x threads vectors for the sum, 8 x 1024 or
+// 4 x 512 for the copy: the shapes launch_sum / launch_copy pick for `ctas`).
+static void fill_flat(Flat* f, int nseg, unsigned long long tile_v, const unsigned* head, const unsigned long long* nvec,
+                      const unsigned long long* nscalar) {
+  unsigned long long t = 0, sc = 0;
+  f->tpre[0] = 0;
+  f->spre[0] = 0;
+  for (int k = 0; k < nseg; k++) {
+    f->head[k] = head[k];
+    f->nvec[k] = nvec[k];
+    t += (nvec[k] + tile_v - 1) / tile_v;
+    sc += nscalar[k];
+    f->tpre[k + 1] = t;
+    f->spre[k + 1] = sc;
+  }
+}
+
+void prepare_sum_batch(SumBatch* b, int ctas) {
+  const int E = b->dtype == 0 ? 4 : 2, VE = 16 / E;
+  const unsigned long long tile_v = 4ull * (wide_grid(ctas) ? 512 : 1024);
+  unsigned head[kMaxSegs];
+  unsigned long long nvec[kMaxSegs], nscalar[kMaxSegs];
+  for (int k = 0; k < b->nseg; k++) {
+    const SumSeg& s = b->seg[k];
+    const unsigned ma = (unsigned)((uintptr_t)s.inbox & 15), mb = (unsigned)((uintptr_t)s.local & 15), mo = (unsigned)((uintptr_t)s.out & 15);
+    split_segment(s.n, ma, ma == mb && mb == mo, E, VE, &head[k], &nvec[k], &nscalar[k]);
+  }
+  fill_flat(&b->flat, b->nseg, tile_v, head, nvec, nscalar);
+}
+
+void prepare_copy_batch(CopyBatch* b, int ctas) {
+  const unsigned long long tile_v = wide_copy_grid(ctas) ? 4ull * 512 : 8ull * 1024;
+  unsigned head[kMaxSegs];
+  unsigned long long nvec[kMaxSegs], nscalar[kMaxSegs];
+  for (int k = 0; k < b->nseg; k++) {
+    const CopySeg& s = b->seg[k];
+    const unsigned ms = (unsigned)((uintptr_t)s.src & 15), md = (unsigned)((uintptr_t)s.dst & 15);
+    split_segment(s.bytes, ms, ms == md, 1, 16, &head[k], &nvec[k], &nscalar[k]);
+  }
+  fill_flat(&b->flat, b->nseg, tile_v, head, nvec, nscalar);
+}
+
 cudaError_t launch_sum(const SumBatch& batch, int ctas, cudaStream_t stream) {
   if (batch.nseg <= 0) return cudaSuccess;
-  if (batch.dtype == 0) {
-    if (wide_grid(ctas)) sum2_kernel<0, 4, 512><<<ctas, 512, 0, stream>>>(batch);
-    else sum2_kernel<0, 4, 1024><<<ctas, 1024, 0, stream>>>(batch);
+  SumBatch b = batch;
+  prepare_sum_batch(&b, ctas);
+  if (b.dtype == 0) {
+    if (wide_grid(ctas)) sum2_kernel<0, 4, 512><<<ctas, 512, 0, stream>>>(b);
+    else sum2_kernel<0, 4, 1024><<<ctas, 1024, 0, stream>>>(b);
   } else {
-    if (wide_grid(ctas)) sum2_kernel<1, 4, 512><<<ctas, 512, 0, stream>>>(batch);
-    else sum2_kernel<1, 4, 1024><<<ctas, 1024, 0, stream>>>(batch);
+    if (wide_grid(ctas)) sum2_kernel<1, 4, 512><<<ctas, 512, 0, stream>>>(b);
+    else sum2_kernel<1, 4, 1024><<<ctas, 1024, 0, stream>>>(b);
   }
   return cudaGetLastError();
 }
 
 cudaError_t launch_copy(const CopyBatch& batch, int ctas, cudaStream_t stream) {
   if (batch.nseg <= 0) return cudaSuccess;
-  if (wide_copy_grid(ctas)) copy_kernel<4, 512><<<ctas, 512, 0, stream>>>(batch);
-  else copy_kernel<8, 1024><<<ctas, 1024, 0, stream>>>(batch);
+  CopyBatch b = batch;
+  prepare_copy_batch(&b, ctas);
+  if (wide_copy_grid(ctas)) copy_kernel<4, 512><<<ctas, 512, 0, stream>>>(b);
+  else copy_kernel<8, 1024><<<ctas, 1024, 0, stream>>>(b);
   return cudaGetLastError();
 }
 

@@ -9,6 +9,17 @@ namespace hoccl {
 constexpr int kMaxSegs = 32;       // segments (one per rank) a single batched launch can carry
 constexpr int kThreads = 1024;     // threads per CTA of the copy and occupancy kernels (the sum picks 512 or 1024)
 
+// Flattened view of a batch of segments: every segment is an element-wise head, a body of 16-byte vectors cut into
+// CTA tiles, and an element-wise tail; prefix sums put the tiles (and the element-wise items) of all segments into one
+// index space, so that any grid stays balanced.  The host fills it when it fills a batch (it knows every pointer and
+// length), so the kernels start without a set-up phase.
+struct Flat {
+  unsigned long long tpre[kMaxSegs + 1];  // prefix sums of vector tiles
+  unsigned long long spre[kMaxSegs + 1];  // prefix sums of element-wise items
+  unsigned long long nvec[kMaxSegs];      // 16-byte vectors in the body
+  unsigned int head[kMaxSegs];            // element-wise items before the body
+};
+
 // One SUM segment: out[i] = rn_T(f32(inbox[i]) + f32(local[i])), i < n (elements).
 struct SumSeg {
   const void* inbox;
@@ -20,6 +31,7 @@ struct SumBatch {
   int nseg;
   int dtype;  // 0 fp32, 1 bf16
   SumSeg seg[kMaxSegs];
+  Flat flat;  // filled by prepare_sum_batch (the launch helpers do it themselves)
 };
 
 // One copy segment: dst[0..bytes) <- src[0..bytes).
@@ -32,6 +44,7 @@ struct CopyBatch {
   int nseg;
   int pad;
   CopySeg seg[kMaxSegs];
+  Flat flat;  // filled by prepare_copy_batch (the launch helpers do it themselves)
 };
 
 // One-pass variant of the ring reduction (comparison point, not rank local): every element is reduced in registers in
@@ -88,6 +101,9 @@ cudaError_t preload_ring_kernels();
 // Enqueue helpers (return the CUDA error of the launch).
 cudaError_t launch_sum(const SumBatch& batch, int ctas, cudaStream_t stream);
 cudaError_t launch_copy(const CopyBatch& batch, int ctas, cudaStream_t stream);
+// Fill batch->flat for the kernel variant that `ctas` CTAs select (needed before a batch is handed to a graph kernel node).
+void prepare_sum_batch(SumBatch* batch, int ctas);
+void prepare_copy_batch(CopyBatch* batch, int ctas);
 // Kernel entry addresses and parameter blocks for CUDA graph kernel nodes.
 const void* sum_kernel_entry(int dtype, int ctas, int* threads);
 const void* copy_kernel_entry(int ctas, int* threads);
