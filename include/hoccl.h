@@ -155,15 +155,16 @@ hoccl_result_t hoccl_comm_set_path(hoccl_comm_t comm, hoccl_path_t path);
  *                grid-wide barrier between dependent steps (how an SM-driven library runs a collective: the paper's
  *                "NCCL under an SM budget" baseline, Sec. 5).  The schedule stays rank local and the bits are the same.
  *                Its grid is min(sum_ctas, copy_ctas) CTAs (copy_ctas for pure moves), fewer for small messages.
- *                Measured on B200 (R = 8, bf16, whole GPU): a step inside the kernel costs ~4.6 us against ~2.7 us for a
- *                kernel boundary inside a CUDA graph, so messages below 256 KiB per rank are slower this way; from 256 KiB
- *                to 16 MiB and from 128 MiB on it is 8-21 % faster (no ramp and tail per step), in between equal.  Under an
- *                8-CTA budget the graph is faster from 8 MiB on, because it overlaps a copy kernel with a sum kernel.
+ *                Measured on B200 (R = 8, bf16, whole GPU): a grid barrier costs ~4 us against ~1.5 us for a kernel
+ *                boundary inside a CUDA graph, so below 128 MiB per rank the graph of per-step kernels is faster (4 KiB
+ *                all-reduce: 31 against 96 us); from 128 MiB on the one-kernel form is 3-10 % faster (no ramp and tail
+ *                per step: 0.78-0.80 against 0.73-0.77 of the 8 TB/s roofline).  Under an 8-CTA budget the graph is
+ *                faster at every size, because it overlaps a copy kernel with a sum kernel.
  *                Every barrier wait is bounded; a wait that runs out ends the kernel and is reported by
  *                hoccl_comm_async_error as HOCCL_ERR_TIMEOUT.  The library allocates 16 bytes of device memory and 4 bytes
  *                of pinned host memory of its own on first use (the third exception to "device memory is the caller's").
- *                Ignored on the other paths, in handshake mode, and for plans too large for one launch (more than 896
- *                chunk operations, i.e. beyond roughly 16 ranks), which run as a graph.  0 = off (default).
+ *                Ignored on the other paths, in handshake mode, and for plans too large for one launch (more than 480
+ *                chunk operations or 96 steps: an all-reduce beyond 12 ranks), which run as a graph.  0 = off (default).
  *  "host_pieces" pieces per ring chunk of the pipelined hoccl_host_allreduce (1..64, default 8; 1 = not pipelined)
  *  "use_graph"   1 = run a cached CUDA graph built from the plan (default), 0 = streams and events
  *  "handshake"   1 = the paper's stream manager (Sec. 3.2, Listing 1): instead of launching into the caller's

@@ -93,6 +93,17 @@ void resolve(hoccl_comm* c, const Plan& P, const Call& call, std::vector<RGroup>
       rg.segs.push_back(s);
     }
   }
+  // SM path: the stages of an all-to-all are independent (disjoint blocks, no dependencies), so their moves go into as few
+  // batched launches as the segment table allows instead of one launch per stage
+  if (c->path == HOCCL_PATH_SM && P.kind == PLAN_ALLTOALL && out->size() > 1) {
+    bool independent = true;
+    for (const RGroup& g : *out) independent = independent && g.deps.empty() && g.kind == OP_MOVE;
+    if (independent) {
+      RGroup all = (*out)[0];
+      for (size_t g = 1; g < out->size(); g++) all.segs.insert(all.segs.end(), (*out)[g].segs.begin(), (*out)[g].segs.end());
+      out->assign(1, all);
+    }
+  }
 }
 
 void fill_sum_batch(const RGroup& g, size_t first, size_t n, int dtype, size_t elem, SumBatch* b) {
@@ -534,11 +545,10 @@ static hoccl_result_t ensure_ring_ctrl(hoccl_comm* c) {
 }
 
 template <typename Args, int NPH, int NSEG>
-static bool fill_ring_args(const std::vector<RGroup>& groups, int dtype, unsigned* bar, int* err_dev, Args* a, size_t* max_phase_bytes,
-                           bool* has_sum) {
+static bool fill_ring_args(const std::vector<RGroup>& groups, int dtype, int threads, unsigned* bar, int* err_dev, Args* a,
+                           size_t* max_phase_bytes) {
   int nph = 0, nseg = 0;
   *max_phase_bytes = 0;
-  *has_sum = false;
   a->dtype = dtype;
   a->bar = bar;
   a->host_err = err_dev;
@@ -556,11 +566,16 @@ static bool fill_ring_args(const std::vector<RGroup>& groups, int dtype, unsigne
       size_t bytes = 0;
       for (size_t i = 0; i < n; i++) {
         const Seg& sg = g.segs[first + i];
-        a->seg[nseg++] = RingSeg{sg.src, g.kind == OP_SUM ? sg.local : nullptr, sg.dst, (unsigned long long)sg.bytes};
+        RingSeg rs = {};
+        rs.src = sg.src;
+        rs.local = g.kind == OP_SUM ? sg.local : nullptr;
+        rs.dst = sg.dst;
+        rs.bytes = (unsigned long long)sg.bytes;
+        a->seg[nseg++] = rs;
         bytes += sg.bytes;
       }
+      prepare_ring_phase(a->seg + ph.first_seg, ph.nseg, ph.kind, dtype, threads);
       *max_phase_bytes = std::max(*max_phase_bytes, bytes);
-      if (g.kind == OP_SUM) *has_sum = true;
     }
   }
   a->nphase = nph;
@@ -574,22 +589,23 @@ static hoccl_result_t build_ring(hoccl_comm* c, const Plan& P, const std::vector
   if (rc != HOCCL_OK) return rc;
   size_t max_phase_bytes = 0;
   bool has_sum = false;
-  entry->ring_args.assign(sizeof(RingArgsSmall), 0);
-  entry->ring_large = false;
-  if (!fill_ring_args<RingArgsSmall, kRingSmallPhases, kRingSmallSegs>(groups, P.dtype, c->ring_bar, c->ring_err_dev,
-                                                                     reinterpret_cast<RingArgsSmall*>(entry->ring_args.data()), &max_phase_bytes, &has_sum)) {
-    entry->ring_args.assign(sizeof(RingArgsLarge), 0);
-    entry->ring_large = true;
-    if (!fill_ring_args<RingArgsLarge, kRingLargePhases, kRingLargeSegs>(groups, P.dtype, c->ring_bar, c->ring_err_dev,
-                                                                       reinterpret_cast<RingArgsLarge*>(entry->ring_args.data()), &max_phase_bytes, &has_sum)) {
-      entry->ring_args.clear();
-      return HOCCL_ERR_UNSUPPORTED;
-    }
-  }
+  for (const RGroup& g : groups) has_sum = has_sum || g.kind == OP_SUM;
   // CTA budget: never more than either budget of the SM path; never more CTAs than the largest phase has tiles for
   // (a barrier costs more the more CTAs take part); never more than can be resident together.
   long budget = has_sum ? std::min(c->sum_ctas, c->copy_ctas) : c->copy_ctas;
   const int threads = budget >= 128 ? 512 : 1024;
+  entry->ring_args.assign(sizeof(RingArgsSmall), 0);
+  entry->ring_large = false;
+  if (!fill_ring_args<RingArgsSmall, kRingSmallPhases, kRingSmallSegs>(groups, P.dtype, threads, c->ring_bar, c->ring_err_dev,
+                                                                     reinterpret_cast<RingArgsSmall*>(entry->ring_args.data()), &max_phase_bytes)) {
+    entry->ring_args.assign(sizeof(RingArgsLarge), 0);
+    entry->ring_large = true;
+    if (!fill_ring_args<RingArgsLarge, kRingLargePhases, kRingLargeSegs>(groups, P.dtype, threads, c->ring_bar, c->ring_err_dev,
+                                                                       reinterpret_cast<RingArgsLarge*>(entry->ring_args.data()), &max_phase_bytes)) {
+      entry->ring_args.clear();
+      return HOCCL_ERR_UNSUPPORTED;
+    }
+  }
   const size_t tile_bytes = (size_t)threads * 4 * 16;
   const long tiles = (long)((max_phase_bytes + tile_bytes - 1) / tile_bytes);
   int max_grid = 0;

@@ -72,14 +72,20 @@ struct RingSeg {
   const void* local;   // SUM: local contribution; MOVE: nullptr
   void* dst;
   unsigned long long bytes;
+  // filled by the host (prepare_ring_phase): the segment's split and the running totals of its phase
+  unsigned long long nvec;         // 16-byte vectors in the body
+  unsigned long long tiles_end;    // tiles of this phase up to and including this segment
+  unsigned long long scalars_end;  // element-wise items of this phase up to and including this segment
+  unsigned int head;               // element-wise items before the body
+  unsigned int pad;
 };
 struct RingPhase {
   int first_seg, nseg;
   int kind;            // 0 MOVE, 1 SUM
   int barrier_before;  // 1: a grid barrier separates this phase from the ones before it
 };
-constexpr int kRingSmallPhases = 32, kRingSmallSegs = 256;   // 8.7 KB of kernel parameters
-constexpr int kRingLargePhases = 224, kRingLargeSegs = 896;  // 32.3 KB (the limit is 32,764 bytes)
+constexpr int kRingSmallPhases = 32, kRingSmallSegs = 256;   // 16.9 KB of kernel parameters
+constexpr int kRingLargePhases = 96, kRingLargeSegs = 480;   // 32.3 KB (the limit is 32,764 bytes)
 constexpr unsigned kRingSpinLimit = 1u << 21;                // polls of one barrier wait before the kernel gives up (~1-2 s)
 template <int NPH, int NSEG>
 struct RingArgsT {
@@ -97,6 +103,8 @@ cudaError_t ring_max_grid(int threads, int dtype, bool large, int num_sms, int* 
 cudaError_t launch_ring(const RingArgsSmall& a, int grid, int threads, cudaStream_t stream);
 cudaError_t launch_ring(const RingArgsLarge& a, int grid, int threads, cudaStream_t stream);
 cudaError_t preload_ring_kernels();
+// Fills nvec / head / tiles_end / scalars_end of the nseg segments of one phase for the kernel shape `threads` selects.
+void prepare_ring_phase(RingSeg* seg, int nseg, int kind, int dtype, int threads);
 
 // Enqueue helpers (return the CUDA error of the launch).
 cudaError_t launch_sum(const SumBatch& batch, int ctas, cudaStream_t stream);

@@ -49,31 +49,6 @@ __device__ __forceinline__ bool grid_barrier(unsigned* bar, unsigned target, int
   return *reinterpret_cast<volatile int*>(s_bail) == 0;
 }
 
-// Prefix sums over the (at most 32) segments of a phase by the first warp: tile counts and element-wise item counts.
-// Every thread of the CTA calls it; lanes >= nseg contribute zero.  Ends with the CTA barrier that publishes the view.
-__device__ __forceinline__ void flatten_prefix(Flat& f, int nseg, unsigned long long my_tiles, unsigned long long my_scalars) {
-  if (threadIdx.x < 32) {
-    unsigned long long t = my_tiles, s = my_scalars;
-#pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-      const unsigned long long tu = __shfl_up_sync(0xffffffffu, t, d), su = __shfl_up_sync(0xffffffffu, s, d);
-      if ((int)threadIdx.x >= d) {
-        t += tu;
-        s += su;
-      }
-    }
-    if (threadIdx.x == 0) {
-      f.tpre[0] = 0;
-      f.spre[0] = 0;
-    }
-    if ((int)threadIdx.x < nseg) {
-      f.tpre[threadIdx.x + 1] = t;
-      f.spre[threadIdx.x + 1] = s;
-    }
-  }
-  __syncthreads();
-}
-
 // element-wise add with L2 loads (heads, tails and segments without a common 16-byte phase)
 template <int DT>
 __device__ __forceinline__ void add_scalar_cg(const void* a, const void* b, void* o, unsigned long long i) {
@@ -86,32 +61,21 @@ __device__ __forceinline__ void add_scalar_cg(const void* a, const void* b, void
   }
 }
 
+// A phase needs no set-up: the host has split every segment into head / vector body / tail and written the running
+// totals of tiles and element-wise items of the phase next to it (RingSeg::tiles_end, ::scalars_end).
 template <int DT, int U, int THREADS>
-__device__ __forceinline__ void sum_phase(Flat& f, const RingSeg* seg, int nseg) {
+__device__ __forceinline__ void sum_phase(const RingSeg* seg, int nseg) {
   using T = Traits<DT>;
-  unsigned long long my_tiles = 0, my_scalars = 0;
-  if ((int)threadIdx.x < nseg) {
-    const RingSeg& s = seg[threadIdx.x];
-    unsigned ma = (unsigned)((uintptr_t)s.src & 15), mb = (unsigned)((uintptr_t)s.local & 15), mo = (unsigned)((uintptr_t)s.dst & 15);
-    unsigned long long nv, ns;
-    unsigned h;
-    split_segment(s.bytes / T::E, ma, ma == mb && mb == mo, T::E, T::VE, &h, &nv, &ns);
-    f.head[threadIdx.x] = h;
-    f.nvec[threadIdx.x] = nv;
-    my_tiles = (nv + (unsigned long long)U * THREADS - 1) / ((unsigned long long)U * THREADS);   // a shift
-    my_scalars = ns;
-  }
-  flatten_prefix(f, nseg, my_tiles, my_scalars);
+  constexpr unsigned tile_v = U * THREADS;
   {
-    const unsigned long long T_all = f.tpre[nseg];
-    const unsigned tile_v = U * blockDim.x;
+    const unsigned long long T_all = seg[nseg - 1].tiles_end;
     int k = 0;
     for (unsigned long long t = blockIdx.x; t < T_all; t += gridDim.x) {
-      while (t >= f.tpre[k + 1]) k++;
-      const unsigned long long first = (t - f.tpre[k]) * tile_v;
-      const unsigned long long left = f.nvec[k] - first;
+      while (t >= seg[k].tiles_end) k++;
+      const unsigned long long first = (t - (k ? seg[k - 1].tiles_end : 0ull)) * tile_v;
+      const unsigned long long left = seg[k].nvec - first;
       const unsigned n_here = left < tile_v ? (unsigned)left : tile_v;
-      const size_t h = (size_t)f.head[k] * T::E;
+      const size_t h = (size_t)seg[k].head * T::E;
       const uint4* a = reinterpret_cast<const uint4*>(static_cast<const char*>(seg[k].src) + h) + first;
       const uint4* b = reinterpret_cast<const uint4*>(static_cast<const char*>(seg[k].local) + h) + first;
       uint4* o = reinterpret_cast<uint4*>(static_cast<char*>(seg[k].dst) + h) + first;
@@ -119,74 +83,61 @@ __device__ __forceinline__ void sum_phase(Flat& f, const RingSeg* seg, int nseg)
       if (n_here == tile_v) {
 #pragma unroll
         for (int u = 0; u < U; u++) {
-          va[u] = __ldcg(a + threadIdx.x + u * blockDim.x);
-          vb[u] = __ldcg(b + threadIdx.x + u * blockDim.x);
+          va[u] = __ldcg(a + threadIdx.x + u * THREADS);
+          vb[u] = __ldcg(b + threadIdx.x + u * THREADS);
         }
 #pragma unroll
-        for (int u = 0; u < U; u++) o[threadIdx.x + u * blockDim.x] = T::add_vec(va[u], vb[u]);
+        for (int u = 0; u < U; u++) o[threadIdx.x + u * THREADS] = T::add_vec(va[u], vb[u]);
       } else {
-        for (unsigned i = threadIdx.x; i < n_here; i += blockDim.x) o[i] = T::add_vec(__ldcg(a + i), __ldcg(b + i));
+        for (unsigned i = threadIdx.x; i < n_here; i += THREADS) o[i] = T::add_vec(__ldcg(a + i), __ldcg(b + i));
       }
     }
   }
   {
-    const unsigned long long total = (unsigned long long)gridDim.x * blockDim.x;
-    const unsigned long long S = f.spre[nseg];
+    const unsigned long long total = (unsigned long long)gridDim.x * THREADS;
+    const unsigned long long S = seg[nseg - 1].scalars_end;
     int k = 0;
-    for (unsigned long long j = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; j < S; j += total) {
-      while (j >= f.spre[k + 1]) k++;
-      unsigned long long i = j - f.spre[k];
-      if (i >= f.head[k]) i += f.nvec[k] * T::VE;
+    for (unsigned long long j = (unsigned long long)blockIdx.x * THREADS + threadIdx.x; j < S; j += total) {
+      while (j >= seg[k].scalars_end) k++;
+      unsigned long long i = j - (k ? seg[k - 1].scalars_end : 0ull);
+      if (i >= seg[k].head) i += seg[k].nvec * T::VE;
       add_scalar_cg<DT>(seg[k].src, seg[k].local, seg[k].dst, i);
     }
   }
 }
 
 template <int U, int THREADS>
-__device__ __forceinline__ void copy_phase(Flat& f, const RingSeg* seg, int nseg) {
-  unsigned long long my_tiles = 0, my_scalars = 0;
-  if ((int)threadIdx.x < nseg) {
-    const RingSeg& s = seg[threadIdx.x];
-    unsigned ms = (unsigned)((uintptr_t)s.src & 15), md = (unsigned)((uintptr_t)s.dst & 15);
-    unsigned long long nv, ns;
-    unsigned h;
-    split_segment(s.bytes, ms, ms == md, 1, 16, &h, &nv, &ns);
-    f.head[threadIdx.x] = h;
-    f.nvec[threadIdx.x] = nv;
-    my_tiles = (nv + (unsigned long long)U * THREADS - 1) / ((unsigned long long)U * THREADS);   // a shift
-    my_scalars = ns;
-  }
-  flatten_prefix(f, nseg, my_tiles, my_scalars);
+__device__ __forceinline__ void copy_phase(const RingSeg* seg, int nseg) {
+  constexpr unsigned tile_v = U * THREADS;
   {
-    const unsigned long long T_all = f.tpre[nseg];
-    const unsigned tile_v = U * blockDim.x;
+    const unsigned long long T_all = seg[nseg - 1].tiles_end;
     int k = 0;
     for (unsigned long long t = blockIdx.x; t < T_all; t += gridDim.x) {
-      while (t >= f.tpre[k + 1]) k++;
-      const unsigned long long first = (t - f.tpre[k]) * tile_v;
-      const unsigned long long left = f.nvec[k] - first;
+      while (t >= seg[k].tiles_end) k++;
+      const unsigned long long first = (t - (k ? seg[k - 1].tiles_end : 0ull)) * tile_v;
+      const unsigned long long left = seg[k].nvec - first;
       const unsigned n_here = left < tile_v ? (unsigned)left : tile_v;
-      const uint4* a = reinterpret_cast<const uint4*>(static_cast<const char*>(seg[k].src) + f.head[k]) + first;
-      uint4* o = reinterpret_cast<uint4*>(static_cast<char*>(seg[k].dst) + f.head[k]) + first;
+      const uint4* a = reinterpret_cast<const uint4*>(static_cast<const char*>(seg[k].src) + seg[k].head) + first;
+      uint4* o = reinterpret_cast<uint4*>(static_cast<char*>(seg[k].dst) + seg[k].head) + first;
       uint4 va[U];
       if (n_here == tile_v) {
 #pragma unroll
-        for (int u = 0; u < U; u++) va[u] = __ldcg(a + threadIdx.x + u * blockDim.x);
+        for (int u = 0; u < U; u++) va[u] = __ldcg(a + threadIdx.x + u * THREADS);
 #pragma unroll
-        for (int u = 0; u < U; u++) o[threadIdx.x + u * blockDim.x] = va[u];
+        for (int u = 0; u < U; u++) o[threadIdx.x + u * THREADS] = va[u];
       } else {
-        for (unsigned i = threadIdx.x; i < n_here; i += blockDim.x) o[i] = __ldcg(a + i);
+        for (unsigned i = threadIdx.x; i < n_here; i += THREADS) o[i] = __ldcg(a + i);
       }
     }
   }
   {
-    const unsigned long long total = (unsigned long long)gridDim.x * blockDim.x;
-    const unsigned long long S = f.spre[nseg];
+    const unsigned long long total = (unsigned long long)gridDim.x * THREADS;
+    const unsigned long long S = seg[nseg - 1].scalars_end;
     int k = 0;
-    for (unsigned long long j = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; j < S; j += total) {
-      while (j >= f.spre[k + 1]) k++;
-      unsigned long long i = j - f.spre[k];
-      if (i >= f.head[k]) i += f.nvec[k] * 16;
+    for (unsigned long long j = (unsigned long long)blockIdx.x * THREADS + threadIdx.x; j < S; j += total) {
+      while (j >= seg[k].scalars_end) k++;
+      unsigned long long i = j - (k ? seg[k - 1].scalars_end : 0ull);
+      if (i >= seg[k].head) i += seg[k].nvec * 16;
       static_cast<unsigned char*>(seg[k].dst)[i] = __ldcg(static_cast<const unsigned char*>(seg[k].src) + i);
     }
   }
@@ -194,22 +145,17 @@ __device__ __forceinline__ void copy_phase(Flat& f, const RingSeg* seg, int nseg
 
 template <int DT, int THREADS, int NPH, int NSEG>
 __global__ void __launch_bounds__(THREADS, 1) ring_kernel(const __grid_constant__ RingArgsT<NPH, NSEG> a) {
-  __shared__ Flat f;
   __shared__ int s_bail;
   if (threadIdx.x == 0) s_bail = 0;
   unsigned nbar = 0;
-  bool ok = true;
-  for (int ph = 0; ph < a.nphase && ok; ph++) {
+  for (int ph = 0; ph < a.nphase; ph++) {
     const RingPhase P = a.phase[ph];
     if (P.barrier_before) {
       nbar++;
-      ok = grid_barrier(a.bar, nbar * gridDim.x, a.host_err, &s_bail);
-      if (!ok) break;
-    } else {
-      __syncthreads();   // the flattened view of the previous phase is about to be overwritten
+      if (!grid_barrier(a.bar, nbar * gridDim.x, a.host_err, &s_bail)) break;
     }
-    if (P.kind == 1) sum_phase<DT, 4, THREADS>(f, a.seg + P.first_seg, P.nseg);
-    else copy_phase<(THREADS == 1024 ? 8 : 4), THREADS>(f, a.seg + P.first_seg, P.nseg);
+    if (P.kind == 1) sum_phase<DT, 4, THREADS>(a.seg + P.first_seg, P.nseg);
+    else copy_phase<(THREADS == 1024 ? 8 : 4), THREADS>(a.seg + P.first_seg, P.nseg);
   }
   // leave: the last CTA out clears the barrier words, so that the next launch starts from zero even after a give-up
   __syncthreads();
@@ -253,6 +199,27 @@ cudaError_t launch_ring_t(const RingArgsT<NPH, NSEG>& a, int grid, int threads, 
 
 cudaError_t launch_ring(const RingArgsSmall& a, int grid, int threads, cudaStream_t stream) { return launch_ring_t(a, grid, threads, stream); }
 cudaError_t launch_ring(const RingArgsLarge& a, int grid, int threads, cudaStream_t stream) { return launch_ring_t(a, grid, threads, stream); }
+
+void prepare_ring_phase(RingSeg* seg, int nseg, int kind, int dtype, int threads) {
+  const int E = kind == 1 ? (dtype == 0 ? 4 : 2) : 1, VE = 16 / E;
+  const unsigned long long tile_v = (unsigned long long)threads * (kind == 1 ? 4 : (threads == 1024 ? 8 : 4));
+  unsigned long long tiles = 0, scalars = 0;
+  for (int k = 0; k < nseg; k++) {
+    RingSeg& s = seg[k];
+    const unsigned ms = (unsigned)((uintptr_t)s.src & 15), md = (unsigned)((uintptr_t)s.dst & 15);
+    const bool congruent = kind == 1 ? (ms == md && ms == (unsigned)((uintptr_t)s.local & 15)) : (ms == md);
+    unsigned long long nv, ns;
+    unsigned h;
+    split_segment(s.bytes / E, ms, congruent, E, VE, &h, &nv, &ns);
+    s.head = h;
+    s.nvec = nv;
+    s.pad = 0;
+    tiles += (nv + tile_v - 1) / tile_v;
+    scalars += ns;
+    s.tiles_end = tiles;
+    s.scalars_end = scalars;
+  }
+}
 
 cudaError_t ring_max_grid(int threads, int dtype, bool large, int num_sms, int* grid) {
   int per_sm = 0;

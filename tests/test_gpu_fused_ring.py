@@ -115,9 +115,9 @@ def test_fused_reduce_scatter_allgather_alltoall(oracle, dtype):
         comm.destroy()
 
 
-@pytest.mark.parametrize("R", [16, 33])
+@pytest.mark.parametrize("R", [10, 16])
 def test_fused_many_ranks(oracle, R):
-    """16 ranks need the large parameter block; 33 ranks do not fit one launch and fall back to the graph."""
+    """10 ranks need the large parameter block; 16 ranks do not fit one launch and fall back to the graph."""
     for dtype, n in (("bf16", R * 1000 + 5), ("fp32", R * 257)):
         xs = W.rank_inputs("uniform", 500 + R, R, n, dtype)
         want = oracle.ring_allreduce(xs)
@@ -126,7 +126,7 @@ def test_fused_many_ranks(oracle, R):
         for r in range(R):
             assert same_bits(got[r], want[r], dtype), (R, dtype, r)
         st = comm.last_stats()
-        assert (st["n_sum_launches"] == 0) == (R == 16), st
+        assert (st["n_sum_launches"] == 0) == (R == 10), st
         comm.destroy()
 
 
