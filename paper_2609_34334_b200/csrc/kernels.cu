@@ -7,7 +7,8 @@
 // copy_kernel  - SM-driven byte copy with a CTA budget: the comparison path for moves (the paper's
 //                "NCCL under an SM budget", Sec. 5 "Baselines").
 // Both are batched: one launch serves all ranks of a ring step through a segment table, and the
-// segments are flattened into one index space so that a small CTA budget stays balanced.  Loads and
+// segments are flattened into one index space (by the host, which passes the prefix sums along with the
+// table: the kernels have no set-up phase and no barrier) so that a small CTA budget stays balanced.  Loads and
 // stores are 16-byte vectors, fully coalesced (consecutive threads touch consecutive vectors);
 // segments whose three addresses are not congruent modulo 16 fall back to element-wise accesses.
 // The sum streams CTA-contiguous tiles (blockDim x 4 vectors per operand) with all of a tile's loads in
