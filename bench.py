@@ -34,10 +34,10 @@ FALLBACK_BF16_TFLOPS = 1590.0
 N_BUCKET_SETS = 4
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of one SUM launch, from the ncu capture summarised in
-# profiles/sum2_kernel_bf16_8cta_200MiB.md: 573.44 MB of traffic for 629.15 MB of algorithmic bytes (operands of
+# profiles/sum2_kernel_bf16_8cta_200MiB.md: 573.88 MB of traffic for 629.15 MB of algorithmic bytes (operands of
 # 200 MiB, larger than L2; part of the output is still in L2 when the kernel ends).  Traffic grows in proportion to
 # the bytes a launch processes, so it is scaled to this workload's launch (8 segments x 3,276,800 B x 3).
-NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = 573.44 / 629.15
+NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = 573.88 / 629.15
 SM_PORT_GBPS = 123.0   # measured mixed 2:1 read/write ceiling of one SM's memory port (bulk loads + bulk stores)
 
 
