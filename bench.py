@@ -376,6 +376,11 @@ def main():
         a = torch.empty(big, dtype=torch.bfloat16, device="cuda").normal_(0, 1e-3)
         b2 = torch.empty(big, dtype=torch.bfloat16, device="cuda").normal_(0, 1e-3)
         o = torch.empty(big, dtype=torch.bfloat16, device="cuda")
+        # SMs used, counted: every CTA of an 8-CTA SUM launch (the launch shape of the timed path) reports its SM id
+        ids = torch.full((8,), -1, dtype=torch.int32, device="cuda")
+        if hb.kernel_sms("sum", a, b2, o, 8 * 3276800, dtype, 8, ids, stream) == hb.OK:
+            stream.synchronize()
+            line["sms_used"]["distinct_sms_of_one_sum_launch"] = len(set(ids.cpu().tolist()))
         full = {}
         for ctas in (8, 16, 32, 48, 64, 96, 128, 148, 296, 592):
             for _ in range(3):

@@ -381,6 +381,15 @@ hoccl_result_t hoccl_probe_copy_routes(hoccl_comm_t comm, void* dst, const void*
 hoccl_result_t hoccl_sum_launch(const void* inbox, const void* local, void* out, size_t count, hoccl_dtype_t dtype,
                                 int ctas, hoccl_stream_t stream);
 hoccl_result_t hoccl_copy_launch(const void* src, void* dst, size_t bytes, int ctas, hoccl_stream_t stream);
+/*
+ * "SMs used", counted rather than inferred (the paper's Table 1 counts the SMs that communication kernels occupy):
+ * launches the SUM kernel (kind 0: out = a + b over bytes / sizeof(dtype) elements) or the copy kernel (kind 1:
+ * out <- a, b ignored) with `ctas` CTAs, and every CTA additionally stores the id of the SM it runs on (%smid) to
+ * smid_out[block index], a device array of `ctas` 32-bit words.  The number of distinct values is the number of SMs
+ * the launch occupied.  Same kernels and launch shapes as the collectives use.
+ */
+hoccl_result_t hoccl_kernel_sms(int kind, const void* a, const void* b, void* out, size_t bytes, hoccl_dtype_t dtype, int ctas,
+                                unsigned int* smid_out, hoccl_stream_t stream);
 
 /* ---------------------------------------------------------------- plan inspection (host only) --- */
 

@@ -533,6 +533,29 @@ hoccl_result_t hoccl_sum_launch(const void* inbox, const void* local, void* out,
   return launch_sum(b, ctas, (cudaStream_t)stream) == cudaSuccess ? HOCCL_OK : HOCCL_ERR_CUDA;
 }
 
+hoccl_result_t hoccl_kernel_sms(int kind, const void* a, const void* b, void* out, size_t bytes, hoccl_dtype_t dtype, int ctas,
+                                unsigned int* smid_out, hoccl_stream_t stream) {
+  size_t e = dtype_size((int)dtype);
+  if (e == 0) return HOCCL_ERR_UNSUPPORTED;
+  if ((kind != 0 && kind != 1) || !a || !out || (kind == 0 && !b) || !smid_out || ctas < 1 || ctas > 1024) return HOCCL_ERR_INVALID_ARG;
+  if (((uintptr_t)smid_out & 3) || (kind == 0 && (((uintptr_t)a | (uintptr_t)b | (uintptr_t)out) % e))) return HOCCL_ERR_INVALID_ARG;
+  if (bytes == 0) return HOCCL_OK;
+  if (kind == 0) {
+    SumBatch sb;
+    sb.nseg = 1;
+    sb.dtype = (int)dtype;
+    sb.seg[0] = SumSeg{a, b, out, (unsigned long long)(bytes / e)};
+    sb.smid_out = smid_out;
+    return launch_sum(sb, ctas, (cudaStream_t)stream) == cudaSuccess ? HOCCL_OK : HOCCL_ERR_CUDA;
+  }
+  CopyBatch cb;
+  cb.nseg = 1;
+  cb.pad = 0;
+  cb.seg[0] = CopySeg{a, out, (unsigned long long)bytes};
+  cb.smid_out = smid_out;
+  return launch_copy(cb, ctas, (cudaStream_t)stream) == cudaSuccess ? HOCCL_OK : HOCCL_ERR_CUDA;
+}
+
 hoccl_result_t hoccl_copy_launch(const void* src, void* dst, size_t bytes, int ctas, hoccl_stream_t stream) {
   if (!src || !dst || ctas < 1 || ctas > 1024) return HOCCL_ERR_INVALID_ARG;
   if (bytes == 0) return HOCCL_OK;

@@ -30,6 +30,11 @@ __global__ void __launch_bounds__(THREADS, 1) sum2_kernel(const __grid_constant_
   using T = Traits<DT>;
   const Flat& f = batch.flat;   // filled on the host for this kernel variant: no set-up phase, no barrier
   const int nseg = batch.nseg;
+  if (batch.smid_out != nullptr && threadIdx.x == 0) {
+    unsigned id;
+    asm volatile("mov.u32 %0, %%smid;" : "=r"(id));
+    batch.smid_out[blockIdx.x] = id;
+  }
   const unsigned long long total = (unsigned long long)gridDim.x * blockDim.x;
   const unsigned long long gt = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
 
@@ -91,6 +96,11 @@ template <int U, int THREADS>
 __global__ void __launch_bounds__(THREADS, 1) copy_kernel(const __grid_constant__ CopyBatch batch) {
   const Flat& f = batch.flat;
   const int nseg = batch.nseg;
+  if (batch.smid_out != nullptr && threadIdx.x == 0) {
+    unsigned id;
+    asm volatile("mov.u32 %0, %%smid;" : "=r"(id));
+    batch.smid_out[blockIdx.x] = id;
+  }
   const unsigned long long total = (unsigned long long)gridDim.x * blockDim.x;
   const unsigned long long gt = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
   {

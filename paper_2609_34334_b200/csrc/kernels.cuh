@@ -32,6 +32,7 @@ struct SumBatch {
   int dtype;  // 0 fp32, 1 bf16
   SumSeg seg[kMaxSegs];
   Flat flat;  // filled by prepare_sum_batch (the launch helpers do it themselves)
+  unsigned int* smid_out = nullptr;  // diagnostics: if set, CTA b stores the id of the SM it runs on to smid_out[b]
 };
 
 // One copy segment: dst[0..bytes) <- src[0..bytes).
@@ -45,6 +46,7 @@ struct CopyBatch {
   int pad;
   CopySeg seg[kMaxSegs];
   Flat flat;  // filled by prepare_copy_batch (the launch helpers do it themselves)
+  unsigned int* smid_out = nullptr;  // diagnostics, as in SumBatch
 };
 
 // One-pass variant of the ring reduction (comparison point, not rank local): every element is reduced in registers in

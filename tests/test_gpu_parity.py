@@ -657,3 +657,23 @@ def test_probe_copy_routes_controls_and_copy_kernel():
     assert rows["control: pinned host->device"][0] is False
     assert torch.equal(b, a)                                  # the last route copied host (= a) back into b
     comm.destroy()
+
+
+@pytest.mark.parametrize("kind", ["sum", "copy"])
+def test_kernels_occupy_as_many_sms_as_their_cta_budget(kind):
+    """SMs used, counted: every CTA reports the SM it ran on.  Under a budget of up to 148 CTAs (one CTA per SM by
+    registers and threads) the launch occupies exactly `ctas` distinct SMs; the result is still right."""
+    n = 8 << 20
+    a = torch.empty(n, dtype=torch.bfloat16, device="cuda").normal_(0, 1e-3)
+    b = torch.empty(n, dtype=torch.bfloat16, device="cuda").normal_(0, 1e-3)
+    out = torch.empty(n, dtype=torch.bfloat16, device="cuda")
+    n_sm = torch.cuda.get_device_properties(0).multi_processor_count
+    for ctas in (1, 8, 32, n_sm):
+        ids = torch.full((ctas,), 0xFFFF, dtype=torch.int32, device="cuda")
+        assert hb.kernel_sms(kind, a, b if kind == "sum" else None, out, n * 2, "bf16", ctas, ids) == hb.OK
+        torch.cuda.synchronize()
+        got = ids.cpu().numpy()
+        assert (got >= 0).all() and (got < n_sm).all()
+        assert len(set(got.tolist())) == ctas, (kind, ctas, sorted(got.tolist()))
+        want = (a.float() + b.float()).to(torch.bfloat16) if kind == "sum" else a
+        assert torch.equal(out, want)
