@@ -323,11 +323,21 @@ hoccl_result_t hoccl_alltoallv(const void* const* send, const size_t* sendcounts
       *src = (const char*)send[f.origin_src] + so;
       *dst = (char*)recv[f.origin_dst] + dofs;
     };
+    // Service order is the scheduler's; chunks that follow one another in a queue and continue the same flow are
+    // issued as one operation (a queue that serves a single flow, the uniform case, becomes one copy per flow).
+    std::vector<std::vector<ChunkItem>> queues(R);
+    for (int g = 0; g < R; g++)
+      for (const ChunkItem& it : st.queues[g]) {
+        if (!queues[g].empty() && queues[g].back().flow == it.flow && queues[g].back().offset + queues[g].back().bytes == it.offset)
+          queues[g].back().bytes += it.bytes;
+        else
+          queues[g].push_back(it);
+      }
     if (c->path == HOCCL_PATH_CE) {
       // every DMA queue (one per source rank) is a serial chain on its lane, in the interleaved chunk order
       for (int g = 0; g < R; g++) {
         cudaStream_t lane = c->lane[g % lanes];
-        for (const ChunkItem& it : st.queues[g]) {
+        for (const ChunkItem& it : queues[g]) {
           const char* src;
           char* dst;
           endpoints(it, &src, &dst);
@@ -339,14 +349,14 @@ hoccl_result_t hoccl_alltoallv(const void* const* send, const size_t* sendcounts
       // SM path: the k-th chunk of every queue goes into one batched copy launch (the queues advance in lock step,
       // which is what R engines of equal speed would do), so a stage costs as many launches as its longest queue
       size_t depth = 0;
-      for (int g = 0; g < R; g++) depth = std::max(depth, st.queues[g].size());
+      for (int g = 0; g < R; g++) depth = std::max(depth, queues[g].size());
       for (size_t k = 0; k < depth; k++) {
         CopyBatch b;
         b.nseg = 0;
         b.pad = 0;
         for (int g = 0; g < R; g++) {
-          if (k >= st.queues[g].size()) continue;
-          const ChunkItem& it = st.queues[g][k];
+          if (k >= queues[g].size()) continue;
+          const ChunkItem& it = queues[g][k];
           const char* src;
           char* dst;
           endpoints(it, &src, &dst);

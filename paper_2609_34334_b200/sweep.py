@@ -5,6 +5,7 @@ pipeline / gradient-stream workloads (third and fourth), through the C ABI.
     python -m paper_2609_34334_b200.sweep pipeline [--microbatches 16]
     python -m paper_2609_34334_b200.sweep gradients [--buckets 32] [--budgets 1,2,4,8,16,32,64]
     python -m paper_2609_34334_b200.sweep launch-cost
+    python -m paper_2609_34334_b200.sweep alltoallv [--mib 4,64,256]
 
 Sizes are per-rank buffer bytes S in the nccl-tests convention (all-reduce: send = recv = S; reduce-scatter:
 send = S; all-gather: recv = S; all-to-all: send = recv = S; send/recv: S), like the sweeps the paper reports (Sec. 5 "Communication
@@ -376,6 +377,78 @@ def launch_cost(args):
                 comm.destroy()
 
 
+def alltoallv(args):
+    """User-defined pattern (the paper's collective scheduler, Sec. 3.4, driving hoccl_alltoallv): an expert-parallel
+    dispatch where every rank sends S bytes in total, split over the destinations either uniformly or with a skew
+    (destination weights 1/(1+k) in a per-source random order, seeded).  Time per call on both paths, host time
+    per call, and the schedule's stage count.  The uniform case is compared with hoccl_alltoall."""
+    import numpy as np
+    torch.cuda.set_device(0)
+    R, dtype, e = 8, "bf16", 2
+    stream = torch.cuda.Stream()
+    rng = np.random.default_rng(5)
+    for S in [int(x) << 20 for x in args.mib.split(",")]:
+        n = S // e
+        send = [torch.empty(n, dtype=torch.bfloat16, device="cuda").normal_(0, 1) for _ in range(R)]
+        for pattern in ("uniform", "skewed"):
+            if pattern == "uniform":
+                counts = np.full((R, R), n // R, dtype=np.int64)
+            else:
+                counts = np.zeros((R, R), dtype=np.int64)
+                for u in range(R):
+                    w = 1.0 / (1.0 + rng.permutation(R))
+                    counts[u] = np.floor(w / w.sum() * n).astype(np.int64) // 8 * 8
+            sdispls = np.concatenate([np.zeros((R, 1), dtype=np.int64), np.cumsum(counts, axis=1)[:, :-1]], axis=1)
+            recv_counts = counts.T                         # recv_counts[v][u] = what v gets from u
+            rdispls = np.concatenate([np.zeros((R, 1), dtype=np.int64), np.cumsum(recv_counts, axis=1)[:, :-1]], axis=1)
+            recv = [torch.zeros(int(recv_counts[v].sum()) + 8, dtype=torch.bfloat16, device="cuda") for v in range(R)]
+            moved = int(counts.sum()) * e
+            configs = [("CE", hb.PATH_CE, 8), ("SM8", hb.PATH_SM, 8), ("SMall", hb.PATH_SM, 148)]
+            for name, path, ctas in configs:
+                comm = hb.Comm(R, 0)
+                comm.set_path(path)
+                comm.set_param("copy_ctas", ctas)
+
+                def call():
+                    comm.alltoallv(send, counts.reshape(-1), sdispls.reshape(-1), recv, rdispls.reshape(-1), dtype, stream)
+
+                for _ in range(3):
+                    call()
+                stream.synchronize()
+                ok = all(torch.equal(recv[v][int(rdispls[v][u]):int(rdispls[v][u] + counts[u][v])],
+                                     send[u][int(sdispls[u][v]):int(sdispls[u][v] + counts[u][v])]) for u in range(R) for v in range(R))
+                iters = 10
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                for _ in range(iters):
+                    call()
+                e1.record(stream)
+                stream.synchronize()
+                t = e0.elapsed_time(e1) / 1e3 / iters
+                st = comm.last_stats()
+                row = {"op": "alltoallv", "pattern": pattern, "S": S, "config": name, "us": t * 1e6, "GBps_moved": moved / t / 1e9,
+                       "hbm_frac_of_8TBps": 2.0 * moved / t / NOMINAL_HBM, "stages": int(st["n_pieces"]), "moves": int(st["n_moves"]),
+                       "launches": int(st["n_move_launches"]), "host_us_per_call": st["host_launch_us"], "delivered_bit_exact": ok,
+                       "largest_flow_MiB": float(counts.max() * e / 2 ** 20), "smallest_flow_MiB": float(counts.min() * e / 2 ** 20)}
+                if pattern == "uniform":
+                    r2 = [torch.zeros(n, dtype=torch.bfloat16, device="cuda") for _ in range(R)]
+                    for _ in range(3):
+                        comm.alltoall(send, r2, n // R, dtype, stream)
+                    stream.synchronize()
+                    e0.record(stream)
+                    for _ in range(iters):
+                        comm.alltoall(send, r2, n // R, dtype, stream)
+                    e1.record(stream)
+                    stream.synchronize()
+                    row["alltoall_us"] = e0.elapsed_time(e1) * 1e3 / iters
+                    del r2
+                print(json.dumps(row), flush=True)
+                comm.destroy()
+            del recv
+        del send
+        torch.cuda.empty_cache()
+
+
 def main():
     ap = argparse.ArgumentParser()
     sub = ap.add_subparsers(dest="cmd", required=True)
@@ -393,11 +466,13 @@ def main():
     g.add_argument("--buckets", type=int, default=32)
     g.add_argument("--budgets", default="", help="comma list of copy-kernel CTA budgets, e.g. 1,2,4,8,16,32,64")
     sub.add_parser("launch-cost")
+    a2 = sub.add_parser("alltoallv")
+    a2.add_argument("--mib", default="4,64,256", help="comma list of MiB sent per rank")
     args = ap.parse_args()
     if not torch.cuda.is_available():
         sys.stderr.write("sweep: no CUDA device\n")
         return 2
-    {"sizes": sweep_sizes, "pipeline": pipeline, "gradients": gradients, "launch-cost": launch_cost}[args.cmd](args)
+    {"sizes": sweep_sizes, "pipeline": pipeline, "gradients": gradients, "launch-cost": launch_cost, "alltoallv": alltoallv}[args.cmd](args)
     return 0
 
 
