@@ -463,6 +463,15 @@ def small_case(hb, W, torch, np, stream):
         rows[name] = {"us_per_call": t * 1e6, "busbw_GBps": S1 * 2 * (R - 1) / R / t / 1e9,
                       "hbm_frac_of_8TBps": 7.0 * S1 * (R - 1) / t / 1e9 / NOMINAL_HBM_GBS, "matches_oracle": ok}
         cm.destroy()
+    # the oracle on the host cores for the same configuration (a reported baseline, as for the headline workload)
+    thr = oracle_ring.max_threads()
+    t0 = time.perf_counter()
+    reps = 0
+    while reps < 5 or (time.perf_counter() - t0 < 0.5 and reps < 200):
+        oracle_ring.ring_allreduce(xs, threads=thr)
+        reps += 1
+    t_cpu = (time.perf_counter() - t0) / reps
+    rows["cpu_oracle"] = {"us_per_call": t_cpu * 1e6, "busbw_GBps": n * 4 * 2 * (R - 1) / R / t_cpu / 1e9, "cores": thr}
     rows["workload"] = c.name
     return rows
 
