@@ -677,3 +677,31 @@ def test_kernels_occupy_as_many_sms_as_their_cta_budget(kind):
         assert len(set(got.tolist())) == ctas, (kind, ctas, sorted(got.tolist()))
         want = (a.float() + b.float()).to(torch.bfloat16) if kind == "sum" else a
         assert torch.equal(out, want)
+
+
+def test_graph_cache_eviction_with_work_in_flight(oracle):
+    """More distinct call signatures than the graph cache holds (48), issued back to back without host synchronisation:
+    the least recently used graphs are evicted while earlier launches may still be running; every result stays right,
+    and a signature that was evicted is simply rebuilt."""
+    R, dtype = 4, "fp32"
+    counts = [4096 + 4 * k for k in range(70)]
+    n_max = max(counts)
+    xs = W.rank_inputs("uniform", 77, R, n_max, dtype)
+    comm = make_comm(R, n_max, dtype, hb.PATH_SM, sum_ctas=8, copy_ctas=8)
+    send = [DevBuf(n_max * 4).put(xs[r]) for r in range(R)]
+    recvs = [[DevBuf(n * 4) for _ in range(R)] for n in counts]
+    stream = torch.cuda.Stream()
+    for n, recv in zip(counts, recvs):
+        comm.allreduce(send, recv, n, dtype, stream)
+        assert comm.last_stats()["graph_hit"] == 0
+    comm.allreduce(send, recvs[-1], counts[-1], dtype, stream)
+    assert comm.last_stats()["graph_hit"] == 1              # the newest entry is still cached
+    comm.allreduce(send, recvs[0], counts[0], dtype, stream)
+    assert comm.last_stats()["graph_hit"] == 0              # the oldest was evicted and is rebuilt
+    stream.synchronize()
+    for n, recv in zip(counts, recvs):
+        want = oracle.ring_allreduce([x[:n] for x in xs])
+        for r in range(R):
+            assert same_bits(recv[r].get(np.float32), want[r], dtype), (n, r)
+            assert recv[r].guards_intact()
+    assert comm.destroy() == hb.OK
