@@ -275,6 +275,14 @@ int hoccl_comm_pending(hoccl_comm_t comm);
 /* First asynchronous failure: handshake mode, as seen by the proxy (OK, TIMEOUT, MISMATCH or CUDA); "fused" setting,
  * TIMEOUT if a barrier wait of the whole-collective kernel ran out.  clear != 0 resets it. */
 hoccl_result_t hoccl_comm_async_error(hoccl_comm_t comm, int clear);
+/*
+ * Failure-detection self-test of the "fused" kernel's bounded waits, without faulting the GPU: enqueues the
+ * whole-collective kernel with two copy phases (first and second half of `bytes`, src -> dst, device pointers, bytes a
+ * multiple of 32) separated by a grid barrier that waits for one arrival more than the grid delivers.  Every CTA polls
+ * for its bounded number of rounds (a second or two), gives up, the kernel ends by itself, the second half is NOT
+ * copied, and hoccl_comm_async_error then reports HOCCL_ERR_TIMEOUT; the barrier words are clean for the next call.
+ */
+hoccl_result_t hoccl_selftest_barrier_timeout(hoccl_comm_t comm, void* dst, const void* src, size_t bytes, hoccl_stream_t stream);
 /* Handshake mode: number of stream hand-overs the proxy has served so far. */
 long hoccl_comm_handshakes(hoccl_comm_t comm);
 

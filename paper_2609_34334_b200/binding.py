@@ -25,7 +25,7 @@ DTYPES = {"fp32": FLOAT32, "bf16": BFLOAT16}
 EXPORTS = [
     "hoccl_comm_init", "hoccl_comm_destroy", "hoccl_scratch_bytes", "hoccl_comm_set_scratch", "hoccl_comm_set_staging", "hoccl_comm_set_host_staging",
     "hoccl_comm_set_path", "hoccl_comm_set_param", "hoccl_comm_get_param", "hoccl_allreduce", "hoccl_reduce_scatter",
-    "hoccl_allgather", "hoccl_alltoall", "hoccl_alltoallv", "hoccl_send", "hoccl_recv", "hoccl_comm_pending", "hoccl_comm_async_error", "hoccl_comm_handshakes", "hoccl_host_allreduce", "hoccl_error_string",
+    "hoccl_allgather", "hoccl_alltoall", "hoccl_alltoallv", "hoccl_send", "hoccl_recv", "hoccl_comm_pending", "hoccl_comm_async_error", "hoccl_comm_handshakes", "hoccl_selftest_barrier_timeout", "hoccl_host_allreduce", "hoccl_error_string",
     "hoccl_last_cuda_error", "hoccl_last_stats", "hoccl_profile_reset", "hoccl_probe_move_needs_sm", "hoccl_probe_copy_routes", "hoccl_sum_launch", "hoccl_kernel_sms",
     "hoccl_copy_launch", "hoccl_plan_build", "hoccl_plan_destroy", "hoccl_plan_num_ops", "hoccl_plan_num_groups",
     "hoccl_plan_get_op", "hoccl_plan_group_deps", "hoccl_plan_slot_bytes", "hoccl_allreduce_static",
@@ -128,6 +128,7 @@ def lib() -> ctypes.CDLL:
         "hoccl_sum_launch": (i, [vp, vp, vp, sz, i, i, vp]),
         "hoccl_copy_launch": (i, [vp, vp, sz, i, vp]),
         "hoccl_kernel_sms": (i, [i, vp, vp, vp, sz, i, i, vp, vp]),
+        "hoccl_selftest_barrier_timeout": (i, [vp, vp, vp, sz, vp]),
         "hoccl_plan_build": (i, [vpp, i, i, sz, i, i, sz, i, ctypes.c_char_p]),
         "hoccl_plan_slot_bytes": (sz, [vp]),
         "hoccl_plan_destroy": (None, [vp]),
@@ -301,6 +302,9 @@ class Comm:
 
     def async_error(self, clear: bool = False) -> int:
         return lib().hoccl_comm_async_error(self._h, int(clear))
+
+    def selftest_barrier_timeout(self, dst, src, nbytes, stream=None) -> int:
+        return lib().hoccl_selftest_barrier_timeout(self._h, _ptr(dst), _ptr(src), nbytes, _stream(stream))
 
     def handshakes(self) -> int:
         return int(lib().hoccl_comm_handshakes(self._h))

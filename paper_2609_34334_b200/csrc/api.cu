@@ -222,6 +222,12 @@ hoccl_result_t hoccl_comm_async_error(hoccl_comm_t c, int clear) {
   }
 }
 
+hoccl_result_t hoccl_selftest_barrier_timeout(hoccl_comm_t c, void* dst, const void* src, size_t bytes, hoccl_stream_t stream) {
+  if (!c || !dst || !src || bytes < 32 || (bytes & 31)) return HOCCL_ERR_INVALID_ARG;
+  CU_TRY(c, cudaSetDevice(c->device));
+  return ring_barrier_selftest(c, dst, src, bytes, (cudaStream_t)stream);
+}
+
 long hoccl_comm_handshakes(hoccl_comm_t c) { return (c && c->proxy) ? c->proxy->handshakes() : 0; }
 
 hoccl_result_t hoccl_host_allreduce(const void* const* h_send, void* const* h_recv, size_t count, hoccl_dtype_t dtype, hoccl_op_t op,

@@ -622,6 +622,32 @@ static hoccl_result_t build_ring(hoccl_comm* c, const Plan& P, const std::vector
   return HOCCL_OK;
 }
 
+// Self-test of the bounded barrier wait: two copy phases with a barrier between them that waits for one arrival more
+// than the grid can deliver.  The kernel must give up by itself, report it, and leave the barrier words clean.
+hoccl_result_t ring_barrier_selftest(hoccl_comm* c, void* dst, const void* src, size_t bytes, cudaStream_t stream) {
+  hoccl_result_t rc = ensure_ring_ctrl(c);
+  if (rc != HOCCL_OK) return rc;
+  std::vector<char> store(sizeof(RingArgsSmall), 0);
+  RingArgsSmall* a = reinterpret_cast<RingArgsSmall*>(store.data());
+  a->nphase = 2;
+  a->dtype = 0;
+  a->missing_arrivals = 1;
+  a->bar = c->ring_bar;
+  a->host_err = c->ring_err_dev;
+  const size_t half = bytes / 2;
+  for (int ph = 0; ph < 2; ph++) {
+    a->phase[ph] = RingPhase{ph, 1, 0, ph};   // phase 1 sits behind the barrier and must never run
+    RingSeg rs = {};
+    rs.src = (const char*)src + ph * half;
+    rs.dst = (char*)dst + ph * half;
+    rs.bytes = half;
+    a->seg[ph] = rs;
+    prepare_ring_phase(a->seg + ph, 1, 0, 0, 1024);
+  }
+  CU_TRY(c, launch_ring(*a, 4, 1024, stream));
+  return HOCCL_OK;
+}
+
 // Replays a cached graph into the caller's stream (directly, or through the CPU proxy in handshake mode).
 static hoccl_result_t launch_entry(hoccl_comm* c, GraphEntry* hit, cudaStream_t user, double t0) {
   hit->last_use = ++c->use_counter;

@@ -93,6 +93,8 @@ template <int NPH, int NSEG>
 struct RingArgsT {
   int nphase;
   int dtype;
+  int missing_arrivals;  // 0 in normal use; the self-test sets 1: every barrier then waits for a CTA that does not exist
+  int pad;
   unsigned* bar;   // device words {arrivals, exits, gave-up flag}; zero between launches (the kernel resets them on exit)
   int* host_err;   // mapped pinned host word: set to 1 if a barrier wait ran out
   RingPhase phase[NPH];

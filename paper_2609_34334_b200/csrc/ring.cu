@@ -152,7 +152,7 @@ __global__ void __launch_bounds__(THREADS, 1) ring_kernel(const __grid_constant_
     const RingPhase P = a.phase[ph];
     if (P.barrier_before) {
       nbar++;
-      if (!grid_barrier(a.bar, nbar * gridDim.x, a.host_err, &s_bail)) break;
+      if (!grid_barrier(a.bar, nbar * (gridDim.x + (unsigned)a.missing_arrivals), a.host_err, &s_bail)) break;
     }
     if (P.kind == 1) sum_phase<DT, 4, THREADS>(a.seg + P.first_seg, P.nseg);
     else copy_phase<(THREADS == 1024 ? 8 : 4), THREADS>(a.seg + P.first_seg, P.nseg);

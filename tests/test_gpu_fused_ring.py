@@ -156,3 +156,32 @@ def test_fused_forward_variant_and_stream_order(oracle):
     for r in range(R):
         assert same_bits(outs[r].cpu().numpy().view(np.uint16), want[r], dtype)
     comm.destroy()
+
+
+def test_bounded_barrier_wait_runs_out_and_is_reported(oracle):
+    """Failure detection without a GPU fault: a barrier that waits for an arrival nobody makes.  Every CTA gives up
+    after its bounded number of polls, the kernel ends by itself, the phase behind the barrier does not run, the
+    status says TIMEOUT, and the communicator works normally afterwards (the barrier words were cleaned)."""
+    import time
+    R, n, dtype = 4, 4 * 5000 + 1, "fp32"
+    comm = fused_comm(R, n, dtype, 8)
+    nbytes = 1 << 20
+    src = torch.full((nbytes,), 7, dtype=torch.uint8, device="cuda")
+    dst = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")
+    assert comm.async_error() == hb.OK
+    t0 = time.time()
+    assert comm.selftest_barrier_timeout(dst, src, nbytes) == hb.OK
+    torch.cuda.synchronize()
+    waited = time.time() - t0
+    assert 0.05 < waited < 30.0, waited                       # it really waited, and it really stopped by itself
+    assert comm.async_error() == hb.ERR_TIMEOUT
+    assert bool((dst[:nbytes // 2] == 7).all()) and bool((dst[nbytes // 2:] == 0).all())
+    assert comm.async_error(clear=True) == hb.ERR_TIMEOUT
+    assert comm.async_error() == hb.OK
+    xs = W.rank_inputs("uniform", 31, R, n, dtype)
+    want = oracle.ring_allreduce(xs)
+    got = run_allreduce(comm, xs, dtype)
+    for r in range(R):
+        assert same_bits(got[r], want[r], dtype)
+    assert comm.async_error() == hb.OK
+    assert comm.destroy() == hb.OK
