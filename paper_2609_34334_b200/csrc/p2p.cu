@@ -67,8 +67,33 @@ hoccl_result_t p2p_post(hoccl_comm* c, bool is_send, void* buf, size_t count, in
       CU_TRY(c, cudaEventRecord(eb, stream));
       CU_TRY(c, cudaStreamWaitEvent(run, eb, 0));
     }
-    CU_TRY(c, cudaMemcpyAsync(c->host_staging, sbuf, bytes, cudaMemcpyDeviceToHost, run));
-    CU_TRY(c, cudaMemcpyAsync(dbuf, c->host_staging, bytes, cudaMemcpyHostToDevice, run));
+    // Chunk pipelining through the staging area (paper Sec. 3.3.1: one engine fills a staging chunk while the other
+    // drains the previous one): the outbound leg of chunk k+1 runs on lane 0 while the inbound leg of chunk k runs on
+    // lane 1; PCIe carries both directions at once.
+    const size_t chunk = std::max<size_t>((size_t)c->piece_bytes, (size_t)1 << 20);
+    if (bytes <= chunk) {
+      CU_TRY(c, cudaMemcpyAsync(c->host_staging, sbuf, bytes, cudaMemcpyDeviceToHost, run));
+      CU_TRY(c, cudaMemcpyAsync(dbuf, c->host_staging, bytes, cudaMemcpyHostToDevice, run));
+    } else {
+      cudaStream_t back = c->lane[1];
+      cudaEvent_t start = next_event(c);
+      if (!start) return cuda_fail(c, cudaErrorMemoryAllocation, "event pool");
+      CU_TRY(c, cudaEventRecord(start, run));
+      CU_TRY(c, cudaStreamWaitEvent(back, start, 0));   // lane 1 joins after both posting streams, like lane 0
+      for (size_t off = 0; off < bytes; off += chunk) {
+        const size_t len = std::min(chunk, bytes - off);
+        CU_TRY(c, cudaMemcpyAsync(c->host_staging + off, (const char*)sbuf + off, len, cudaMemcpyDeviceToHost, run));
+        cudaEvent_t out = next_event(c);
+        if (!out) return cuda_fail(c, cudaErrorMemoryAllocation, "event pool");
+        CU_TRY(c, cudaEventRecord(out, run));
+        CU_TRY(c, cudaStreamWaitEvent(back, out, 0));
+        CU_TRY(c, cudaMemcpyAsync((char*)dbuf + off, c->host_staging + off, len, cudaMemcpyHostToDevice, back));
+      }
+      cudaEvent_t in_done = next_event(c);
+      if (!in_done) return cuda_fail(c, cudaErrorMemoryAllocation, "event pool");
+      CU_TRY(c, cudaEventRecord(in_done, back));
+      CU_TRY(c, cudaStreamWaitEvent(run, in_done, 0));   // lane 0 stays the serial order of all such moves
+    }
     CU_TRY(c, cudaEventRecord(ed, run));
     CU_TRY(c, cudaStreamWaitEvent(peer.stream, ed, 0));
     if (two_streams) CU_TRY(c, cudaStreamWaitEvent(stream, ed, 0));

@@ -90,3 +90,44 @@ def test_host_bounce_moves_need_no_sm_and_staging_is_checked():
     torch.cuda.synchronize()
     assert float(b[2][77]) == 4.0
     assert comm.destroy() == hb.OK
+
+
+def test_large_messages_are_pipelined_through_the_staging_area():
+    """send/recv of messages larger than one staging chunk: the two legs run chunk by chunk on two lanes.  Messages that
+    follow one another reuse the staging area in order; every message arrives bit for bit."""
+    import time
+    torch.cuda.set_device(0)
+    n = (48 << 20) + 12345 * 2                                   # bf16 elements x 2 B: 48 MiB and a ragged tail
+    comm = hb.Comm(4, 0)
+    comm.set_path(hb.PATH_CE_HOST)
+    comm.set_host_staging(torch.empty(2 * n + 4096, dtype=torch.uint8).pin_memory())
+    msgs = [torch.randint(-30000, 30000, (n,), dtype=torch.int16, device="cuda") for _ in range(3)]
+    dsts = [torch.zeros(n, dtype=torch.int16, device="cuda") for _ in range(3)]
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    for k in range(3):                                            # back to back, no host synchronisation
+        comm.send(msgs[k], n, "bf16", k, k + 1, s1)
+        comm.recv(dsts[k], n, "bf16", k, k + 1, s2)
+    torch.cuda.synchronize()
+    for k in range(3):
+        assert torch.equal(msgs[k], dsts[k]), k
+    # timing: the pipelined legs beat the same two copies issued one after the other, measured side by side
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(s1)
+    comm.send(msgs[0], n, "bf16", 0, 1, s1)
+    comm.recv(dsts[1], n, "bf16", 0, 1, s1)
+    e1.record(s1)
+    torch.cuda.synchronize()
+    assert torch.equal(msgs[0], dsts[1])
+    t_pipe = e0.elapsed_time(e1)
+    host = torch.empty(n, dtype=torch.int16).pin_memory()
+    with torch.cuda.stream(s1):
+        host.copy_(msgs[0], non_blocking=True)                    # touch the pages once
+        torch.cuda.current_stream().synchronize()
+        e0.record(s1)
+        host.copy_(msgs[0], non_blocking=True)
+        dsts[2].copy_(host, non_blocking=True)
+        e1.record(s1)
+    torch.cuda.synchronize()
+    t_seq = e0.elapsed_time(e1)
+    assert t_pipe < 0.8 * t_seq, (t_pipe, t_seq)
+    assert comm.destroy() == hb.OK
