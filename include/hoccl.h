@@ -72,8 +72,10 @@ typedef enum { HOCCL_SUM = 0 } hoccl_op_t;
  *                  copy out of it.  Both legs are served by the copy engines (Sec. 2.3), so this is the one route
  *                  on a single device that really occupies no SM (hoccl_probe_move_needs_sm confirms it); the price
  *                  is PCIe bandwidth.  Needs hoccl_comm_set_host_staging with room for every move of a call
- *                  (all-reduce: 2 * S * (R-1) bytes plus 256 per move).  Not available for hoccl_alltoallv or
- *                  in handshake mode.
+ *                  (all-reduce: 2 * S * (R-1) bytes plus 256 per move; send/recv: the message).  A send/recv message
+ *                  larger than one chunk ("piece_bytes", at least 1 MiB) is pipelined through the staging area chunk by
+ *                  chunk, the outbound leg of chunk k+1 beside the inbound leg of chunk k (Sec. 3.3.1).  Not available
+ *                  for hoccl_alltoallv or in handshake mode.
  *  HOCCL_PATH_SM : the comparison baseline (the paper's "NCCL with an SM budget", Sec. 5 "Baselines"):
  *                  all moves of a step run in one launch of an SM copy kernel with `copy_ctas` CTAs.
  */
