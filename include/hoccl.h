@@ -248,7 +248,10 @@ hoccl_result_t hoccl_alltoall(const void* const* send, void* const* recv, size_t
  * The flows form the origin traffic matrix C; the collective scheduler (hoccl_sched_*) cuts it into stages by
  * peeling matchings (Algorithm 1 with an empty RDMA domain: T = C) and, inside a stage, serves every source rank's
  * flows from one serial queue in a size-weighted chunk interleaving (chunk = the "piece_bytes" parameter, at least
- * 64 KiB).  Stages run one after the other.  Issued with streams and events (not cached).  No scratch.
+ * 64 KiB; chunks that follow one another in a queue and continue the same flow are issued as one operation).  Stages
+ * run one after the other.  With "use_graph" = 1 (default) the schedule becomes a CUDA graph that is cached under the
+ * call's full signature (every pointer, count and displacement), so a pattern that repeats on the same buffers replays
+ * it; otherwise, and with "use_graph" = 0, it is issued with streams and events.  No scratch.
  * Errors: INVALID_ARG (NULL, misaligned, overlapping receive regions, a send region overlapping a receive region),
  * UNSUPPORTED (dtype; handshake mode).
  */

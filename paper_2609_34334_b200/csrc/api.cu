@@ -296,6 +296,40 @@ hoccl_result_t hoccl_alltoallv(const void* const* send, const size_t* sendcounts
       C[(size_t)u * R + v] = (uint64_t)sendcounts[(size_t)u * R + v] * e;
       total += C[(size_t)u * R + v];
     }
+  // A pattern that was issued before with the same buffers (same counts, displacements, pointers and settings) replays
+  // its cached graph: validation, Algorithm 1 and the per-operation host cost were paid when it was built.
+  std::vector<uint64_t> key;
+  if (c->use_graph && total != 0) {
+    key.reserve(8 + 2 * (size_t)R + 3 * (size_t)R * R);
+    key.push_back(0xA11704117ull);   // tag: not a ring collective
+    key.push_back((uint64_t)dtype);
+    key.push_back((uint64_t)c->path);
+    key.push_back((uint64_t)c->copy_ctas);
+    key.push_back((uint64_t)c->piece_bytes);
+    for (int r = 0; r < R; r++) {
+      key.push_back((uint64_t)(uintptr_t)send[r]);
+      key.push_back((uint64_t)(uintptr_t)recv[r]);
+    }
+    for (size_t i = 0; i < (size_t)R * R; i++) {
+      key.push_back((uint64_t)sendcounts[i]);
+      key.push_back((uint64_t)sdispls[i]);
+      key.push_back((uint64_t)rdispls[i]);
+    }
+    for (auto& en : c->cache)
+      if (en.key == key) {
+        c->stats = hoccl_stats_t{};
+        c->stats.graph_hit = 1;
+        CU_TRY(c, cudaSetDevice(c->device));
+        en.last_use = ++c->use_counter;
+        CU_TRY(c, cudaGraphLaunch(en.exec, (cudaStream_t)stream));
+        c->stats.n_moves = en.n_moves;
+        c->stats.n_move_launches = en.n_move_launches;
+        c->stats.max_copy_ctas = en.n_move_launches ? c->copy_ctas : 0;
+        c->stats.n_pieces = en.n_pieces;
+        c->stats.host_launch_us = now_us() - t0;
+        return HOCCL_OK;
+      }
+  }
   // receive regions of one rank must not overlap each other, and no send region may overlap a receive region
   for (int v = 0; v < R; v++)
     for (int a = 0; a < R; a++) {
@@ -313,6 +347,21 @@ hoccl_result_t hoccl_alltoallv(const void* const* send, const size_t* sendcounts
   if (!build_schedule(topo, C, (uint64_t)std::max<long>(c->piece_bytes, 65536), &S)) return HOCCL_ERR_INTERNAL;
   CU_TRY(c, cudaSetDevice(c->device));
   cudaStream_t user = (cudaStream_t)stream;
+  if (c->use_graph) {
+    GraphEntry entry;
+    entry.key = key;
+    hoccl_result_t grc = build_pattern_graph(c, S, send, sdispls, recv, rdispls, e, &entry);
+    if (grc != HOCCL_OK) return grc;
+    GraphEntry* en = cache_put(c, std::move(entry));
+    en->last_use = ++c->use_counter;
+    CU_TRY(c, cudaGraphLaunch(en->exec, user));
+    c->stats.n_moves = en->n_moves;
+    c->stats.n_move_launches = en->n_move_launches;
+    c->stats.max_copy_ctas = en->n_move_launches ? c->copy_ctas : 0;
+    c->stats.n_pieces = en->n_pieces;
+    c->stats.host_launch_us = now_us() - t0;
+    return HOCCL_OK;
+  }
   const int lanes = c->path == HOCCL_PATH_SM ? 1 : (int)std::max<long>(1, std::min<long>(c->lanes, kMaxLanes));
   c->ev_next = 0;
   cudaEvent_t fork = next_event(c);

@@ -165,6 +165,9 @@ hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user);
 hoccl_result_t ensure_proxy(hoccl_comm* c);
 void harvest_profile(hoccl_comm* c);
 void destroy_entry(GraphEntry* e);
+GraphEntry* cache_put(hoccl_comm* c, GraphEntry&& entry);
+hoccl_result_t build_pattern_graph(hoccl_comm* c, const Schedule& S, const void* const* send, const size_t* sdispls, void* const* recv,
+                                   const size_t* rdispls, size_t e, GraphEntry* entry);
 hoccl_result_t ring_barrier_selftest(hoccl_comm* c, void* dst, const void* src, size_t bytes, cudaStream_t stream);
 // p2p.cu
 hoccl_result_t p2p_post(hoccl_comm* c, bool is_send, void* buf, size_t count, int dtype, int src, int dst, cudaStream_t stream);

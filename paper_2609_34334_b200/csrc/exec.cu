@@ -435,6 +435,118 @@ hoccl_result_t build_graph(hoccl_comm* c, const Plan& P, const std::vector<RGrou
   return rc;
 }
 
+// Inserts an entry into the graph cache (evicting the least recently used one when it is full) and returns it.
+GraphEntry* cache_put(hoccl_comm* c, GraphEntry&& entry) {
+  if (c->cache.size() >= kGraphCacheCap) {
+    if (c->proxy) c->proxy->drain(c->watchdog_ms);  // a queued hand-over may still refer to the victim
+    size_t victim = 0;
+    for (size_t i = 1; i < c->cache.size(); i++)
+      if (c->cache[i].last_use < c->cache[victim].last_use) victim = i;
+    destroy_entry(&c->cache[victim]);
+    c->cache.erase(c->cache.begin() + victim);
+  }
+  c->cache.push_back(std::move(entry));
+  return &c->cache.back();
+}
+
+// The schedule of a user-defined pattern (paper Sec. 3.4) as a CUDA graph: stages one after the other (a join node between
+// them), inside a stage every source rank's queue is a serial chain in the scheduler's service order (copy route), or the
+// k-th operations of all queues share one batched copy launch and the launches form one chain (SM path).
+hoccl_result_t build_pattern_graph(hoccl_comm* c, const Schedule& S, const void* const* send, const size_t* sdispls, void* const* recv,
+                                   const size_t* rdispls, size_t e, GraphEntry* entry) {
+  const int R = c->R;
+  cudaGraph_t g = nullptr;
+  CU_TRY(c, cudaGraphCreate(&g, 0));
+  cudaError_t err = cudaSuccess;
+  cudaGraphNode_t stage_dep = nullptr;
+  for (size_t si = 0; si < S.stages.size() && err == cudaSuccess; si++) {
+    const Stage& st = S.stages[si];
+    auto endpoints = [&](const ChunkItem& it, const char** src, char** dst) {
+      const StageFlow& f = st.flows[it.flow];
+      *src = (const char*)send[f.origin_src] + sdispls[(size_t)f.origin_src * R + f.origin_dst] * e + f.origin_offset + it.offset;
+      *dst = (char*)recv[f.origin_dst] + rdispls[(size_t)f.origin_dst * R + f.origin_src] * e + f.origin_offset + it.offset;
+    };
+    // chunks that follow one another in a queue and continue the same flow are one operation
+    std::vector<std::vector<ChunkItem>> queues(R);
+    for (int q = 0; q < R; q++)
+      for (const ChunkItem& it : st.queues[q]) {
+        if (!queues[q].empty() && queues[q].back().flow == it.flow && queues[q].back().offset + queues[q].back().bytes == it.offset)
+          queues[q].back().bytes += it.bytes;
+        else
+          queues[q].push_back(it);
+      }
+    std::vector<cudaGraphNode_t> tails;
+    if (c->path == HOCCL_PATH_CE) {
+      for (int q = 0; q < R && err == cudaSuccess; q++) {
+        cudaGraphNode_t prev = stage_dep;
+        for (const ChunkItem& it : queues[q]) {
+          const char* src;
+          char* dst;
+          endpoints(it, &src, &dst);
+          cudaGraphNode_t n;
+          err = cudaGraphAddMemcpyNode1D(&n, g, prev ? &prev : nullptr, prev ? 1 : 0, dst, src, it.bytes, cudaMemcpyDeviceToDevice);
+          if (err != cudaSuccess) break;
+          prev = n;
+          entry->n_moves++;
+        }
+        if (prev && prev != stage_dep) tails.push_back(prev);
+      }
+    } else {
+      size_t depth = 0;
+      for (int q = 0; q < R; q++) depth = std::max(depth, queues[q].size());
+      cudaGraphNode_t prev = stage_dep;
+      auto add_launch = [&](CopyBatch& b) {
+        prepare_copy_batch(&b, (int)c->copy_ctas);
+        void* args[] = {&b};
+        cudaKernelNodeParams kp = {};
+        int threads = 0;
+        kp.func = const_cast<void*>(copy_kernel_entry((int)c->copy_ctas, &threads));
+        kp.gridDim = dim3((unsigned)c->copy_ctas);
+        kp.blockDim = dim3((unsigned)threads);
+        kp.kernelParams = args;
+        cudaGraphNode_t n;
+        err = cudaGraphAddKernelNode(&n, g, prev ? &prev : nullptr, prev ? 1 : 0, &kp);
+        if (err == cudaSuccess) {
+          prev = n;
+          entry->n_move_launches++;
+        }
+        b.nseg = 0;
+      };
+      for (size_t k = 0; k < depth && err == cudaSuccess; k++) {
+        CopyBatch b;
+        b.nseg = 0;
+        b.pad = 0;
+        for (int q = 0; q < R && err == cudaSuccess; q++) {
+          if (k >= queues[q].size()) continue;
+          const char* src;
+          char* dst;
+          endpoints(queues[q][k], &src, &dst);
+          b.seg[b.nseg++] = CopySeg{src, dst, (unsigned long long)queues[q][k].bytes};
+          entry->n_moves++;
+          if (b.nseg == kMaxSegs) add_launch(b);
+        }
+        if (b.nseg > 0 && err == cudaSuccess) add_launch(b);
+      }
+      if (prev && prev != stage_dep) tails.push_back(prev);
+    }
+    if (err != cudaSuccess) break;
+    if (tails.size() == 1) {
+      stage_dep = tails[0];
+    } else if (tails.size() > 1) {
+      cudaGraphNode_t join;
+      err = cudaGraphAddEmptyNode(&join, g, tails.data(), tails.size());
+      if (err == cudaSuccess) stage_dep = join;
+    }
+  }
+  hoccl_result_t rc = HOCCL_OK;
+  if (err == cudaSuccess) err = cudaGraphInstantiate(&entry->exec, g, 0);
+  if (err != cudaSuccess) rc = cuda_fail(c, err, "pattern graph");
+  cudaGraphDestroy(g);
+  entry->n_pieces = (long)S.stages.size();
+  if (rc != HOCCL_OK) destroy_entry(entry);
+  return rc;
+}
+
 std::vector<uint64_t> make_key(hoccl_comm* c, const Call& call) {
   std::vector<uint64_t> k;
   k.reserve(17 + 2 * c->R);
@@ -854,16 +966,7 @@ hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
         return cuda_fail(c, ue, "cudaGraphUpload");
       }
     }
-    if (c->cache.size() >= kGraphCacheCap) {
-      if (c->proxy) c->proxy->drain(c->watchdog_ms);  // a queued hand-over may still refer to the victim
-      size_t victim = 0;
-      for (size_t i = 1; i < c->cache.size(); i++)
-        if (c->cache[i].last_use < c->cache[victim].last_use) victim = i;
-      destroy_entry(&c->cache[victim]);
-      c->cache.erase(c->cache.begin() + victim);
-    }
-    c->cache.push_back(std::move(entry));
-    return launch_entry(c, &c->cache.back(), user, t0);
+    return launch_entry(c, cache_put(c, std::move(entry)), user, t0);
   }
   Tally tally;
   rc = run_streams(c, P, groups, user, &tally);

@@ -291,8 +291,9 @@ def test_alltoall(oracle, path, use_graph):
             assert comm.destroy() == hb.OK
 
 
+@pytest.mark.parametrize("use_graph", [0, 1])
 @pytest.mark.parametrize("path", [hb.PATH_CE, hb.PATH_SM])
-def test_alltoallv_user_defined_pattern(oracle, path):
+def test_alltoallv_user_defined_pattern(oracle, path, use_graph):
     from test_oracle_pins import _random_pattern
     for dtype in ("fp32", "bf16"):
         e = W.elem_size(dtype)
@@ -305,13 +306,20 @@ def test_alltoallv_user_defined_pattern(oracle, path):
             comm = hb.Comm(R, 0)
             comm.set_path(path)
             comm.set_param("piece_bytes", piece)
+            comm.set_param("use_graph", use_graph)
             send = [DevBuf(send_sizes[u] * e).put(xs[u]) for u in range(R)]
             recv = [DevBuf(recv_sizes[v] * e) for v in range(R)]           # DevBuf pre-fills with 0xA5 bytes
-            comm.alltoallv(send, counts.ravel(), sd.ravel(), recv, rd.ravel(), dtype)
-            torch.cuda.synchronize()
-            for v in range(R):
-                assert (recv[v].get(np_dtype(dtype)).view(np.uint8) == want[v].view(np.uint8)).all(), (R, v)
-                assert recv[v].guards_intact() and send[v].guards_intact()
+            for rep in range(2):                                           # the second call replays the cached graph
+                if rep:
+                    for v in range(R):
+                        recv[v].view.fill_(0xA5)
+                comm.alltoallv(send, counts.ravel(), sd.ravel(), recv, rd.ravel(), dtype)
+                torch.cuda.synchronize()
+                if counts.sum() > 0:
+                    assert comm.last_stats()["graph_hit"] == (1 if (rep and use_graph) else 0)
+                for v in range(R):
+                    assert (recv[v].get(np_dtype(dtype)).view(np.uint8) == want[v].view(np.uint8)).all(), (R, v, rep)
+                    assert recv[v].guards_intact() and send[v].guards_intact()
             # overlapping receive regions are refused
             bad = rd.copy()
             if R >= 2 and counts[0, 1] > 0 and counts[1, 1] > 0:
