@@ -66,7 +66,8 @@ def test_host_allreduce_pipelined_and_sequential(oracle, dtype, host_pieces):
 
 @pytest.mark.parametrize("path,params", [(hb.PATH_SM, dict(sum_ctas=8, copy_ctas=8)), (hb.PATH_SM, dict(sum_ctas=148, copy_ctas=148)),
                                          (hb.PATH_CE, dict(use_graph=0)), (hb.PATH_CE, dict(forward=1)),
-                                         (hb.PATH_SM, dict(fused=1)), (hb.PATH_CE, dict(onepass=1))])
+                                         (hb.PATH_SM, dict(fused=1)), (hb.PATH_CE, dict(onepass=1)),
+                                         (hb.PATH_SM, dict(handshake=1, watchdog_ms=5000))])
 def test_host_allreduce_every_path(oracle, path, params):
     R, n, dtype = 8, 8 * 200_000 + 5, "bf16"
     xs = W.rank_inputs("normal", 71, R, n, dtype, 1e-3)
