@@ -1,8 +1,8 @@
 """GPU parity for hoccl_host_allreduce: host buffers in, host buffers out, bits equal to the oracle.
 
-The pipelined form puts, per piece of every ring chunk, the host-to-device copies, the ring and the device-to-host
-copies into one graph; the sequential form (host_pieces = 1 or use_graph = 0) copies everything in, runs the
-all-reduce and copies everything out.  Both must give the oracle's bits for every size class: ragged sizes where
+The pipelined form runs, per piece of every ring chunk, the host-to-device copies on one internal stream, the ring on
+that piece (its own cached graph) on the caller's stream and the device-to-host copies on a second internal stream; the
+sequential form (host_pieces = 1 or use_graph = 0) copies everything in, runs the all-reduce and copies everything out.  Both must give the oracle's bits for every size class: ragged sizes where
 trailing chunks are short or empty, sizes below one piece, in place on the host, and every path."""
 import numpy as np
 import pytest
