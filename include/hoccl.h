@@ -298,10 +298,11 @@ long hoccl_comm_handshakes(hoccl_comm_t comm);
  * host pointers to `count` elements each.  The call copies every h_send[r] into the attached staging
  * memory (needs 2*R*roundup256(count*sizeof(dtype)) bytes), runs the all-reduce there and copies every rank's
  * result back, all ordered on `stream`.  Host-to-device traffic is driven by the copy engines (Sec. 2.3).
- * Pipelined form (default; "host_pieces" > 1 with graphs on): every ring chunk is cut into host_pieces pieces and ONE
- * cached graph holds, per piece, the host-to-device copies (2-D copies: a piece of every chunk), the ring on that piece
- * and the device-to-host copies, so that the inbound copies, the ring and the outbound copies of different pieces
- * overlap (chunk pipelining, Sec. 3.3.1, applied across the PCIe link).  Chunk boundaries, and therefore every bit of
+ * Pipelined form (default; "host_pieces" > 1 with graphs on): every ring chunk is cut into host_pieces pieces; per
+ * piece, the host-to-device copies (2-D copies: that piece of every chunk) run on one internal stream, the ring on that
+ * piece (its own cached graph) runs on `stream` as soon as the piece has arrived, and the device-to-host copies follow on
+ * a second internal stream, so that the inbound copies, the ring and the outbound copies of different pieces overlap
+ * (chunk pipelining, Sec. 3.3.1, applied across the PCIe link); `stream` waits for the last outbound copy.  Chunk boundaries, and therefore every bit of
  * the result, are those of hoccl_allreduce on the whole buffer.  Host buffers of different ranks must not overlap
  * partially (INVALID_ARG); h_recv[r] == h_send[r] is legal.  With host_pieces = 1, use_graph = 0, handshake, onepass,
  * fused or HOCCL_PATH_CE_HOST the three stages run one after the other.
