@@ -182,7 +182,7 @@ hoccl_result_t hoccl_comm_set_path(hoccl_comm_t comm, hoccl_path_t path);
  *                The two sides of a send/recv must be
  *                posted on different streams (a stream parked in its own post cannot reach the partner's).  The
  *                first use creates the proxy: a thread, pinned host memory for 64 flag pairs and 512 bytes of
- *                device memory (the only device allocation of the library), and loads every kernel, because
+ *                device memory (one of the library's own device allocations stated in this header), and loads every kernel, because
  *                first-use work in the driver must not happen while a stream is parked.
  *  "watchdog_ms" handshake mode: after this long (default 10000) an unmatched post is released with an abort
  *                value and HOCCL_ERR_TIMEOUT is recorded, so no stream can wait on this library forever
