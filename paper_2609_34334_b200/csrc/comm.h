@@ -160,6 +160,20 @@ struct Call {
 };
 
 
+struct Tally {
+  long moves = 0, move_launches = 0, sum_launches = 0;
+};
+
+// exec.cu
+void fill_sum_batch(const RGroup& g, size_t first, size_t n, int dtype, size_t elem, SumBatch* b);
+void fill_copy_batch(const RGroup& g, size_t first, size_t n, CopyBatch* b);
+// graph.cu
+hoccl_result_t build_graph(hoccl_comm* c, const Plan& P, const std::vector<RGroup>& groups, GraphEntry* entry, int only_piece,
+                           cudaGraphExec_t* out_exec);
+void add_host_copies(const Plan& P, int p, char* dev, char* host, std::vector<HostCopy>* out);
+cudaError_t enqueue_host_copy(const HostCopy& hc, bool to_device, cudaStream_t s);
+// ring_host.cu
+hoccl_result_t build_ring(hoccl_comm* c, const Plan& P, const std::vector<RGroup>& groups, GraphEntry* entry);
 // exec.cu
 hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user);
 hoccl_result_t ensure_proxy(hoccl_comm* c);

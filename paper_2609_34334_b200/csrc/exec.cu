@@ -1,4 +1,4 @@
-// libhoccl: communicator, executors and the C ABI declared in include/hoccl.h.
+// libhoccl: how a collective call is executed (the graphs themselves are built in graph.cu, the one-kernel form in ring_host.cu).
 //
 // A collective call = plan (host, plan.cpp) -> resolve the plan's buffer offsets against the caller's
 // pointers -> issue.  Two issue engines consume the same plan and give the same bits:
@@ -123,9 +123,6 @@ void fill_copy_batch(const RGroup& g, size_t first, size_t n, CopyBatch* b) {
   }
 }
 
-struct Tally {
-  long moves = 0, move_launches = 0, sum_launches = 0;
-};
 
 // ------------------------------------------------------------------ stream executor -------------
 hoccl_result_t run_streams(hoccl_comm* c, const Plan& P, const std::vector<RGroup>& groups, cudaStream_t user, Tally* tally) {
@@ -232,321 +229,6 @@ hoccl_result_t run_streams(hoccl_comm* c, const Plan& P, const std::vector<RGrou
   return HOCCL_OK;
 }
 
-// ------------------------------------------------------------------ graph executor --------------
-void destroy_entry(GraphEntry* e) {
-  if (e->exec) cudaGraphExecDestroy(e->exec);
-  for (cudaGraphExec_t pe : e->piece_exec)
-    if (pe) cudaGraphExecDestroy(pe);
-  e->piece_exec.clear();
-  for (auto& p : e->prof_events) {
-    cudaEventDestroy(p.first);
-    cudaEventDestroy(p.second);
-  }
-  e->exec = nullptr;
-  e->prof_events.clear();
-}
-
-// Host <-> staging copies of one piece of one rank (all-reduce layout): piece p of every ring chunk, i.e. rows of
-// `piece` bytes at a pitch of one chunk.  Chunks that hold the full piece go as one 2-D copy; a shorter trailing piece
-// as a 1-D copy.
-static void add_host_copies(const Plan& P, int p, char* dev, char* host, std::vector<HostCopy>* out) {
-  const size_t e = P.elem, q_bytes = P.chunk_elems * e;
-  const size_t off = (size_t)p * P.piece_bytes;
-  size_t full_rows = 0, full_len = 0;
-  for (int cidx = 0; cidx < P.R; cidx++) {
-    size_t lo, hi;
-    P.chunk_range(cidx, &lo, &hi);
-    const size_t len_bytes = (hi - lo) * e;
-    const size_t a = std::min(off, len_bytes), b = std::min(off + P.piece_bytes, len_bytes);
-    const size_t len = b - a;
-    if (len == 0) continue;
-    if (cidx == 0) full_len = len;
-    if (len == full_len && (size_t)cidx == full_rows) {
-      full_rows++;
-      continue;
-    }
-    out->push_back(HostCopy{dev + lo * e + a, host + lo * e + a, len, len, 1});
-  }
-  if (full_rows > 0) out->push_back(HostCopy{dev + off, host + off, q_bytes, full_len, full_rows});
-}
-
-static cudaError_t enqueue_host_copy(const HostCopy& hc, bool to_device, cudaStream_t s) {
-  const cudaMemcpyKind kind = to_device ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToHost;
-  void* dst = to_device ? (void*)hc.dev : (void*)hc.host;
-  const void* src = to_device ? (const void*)hc.host : (const void*)hc.dev;
-  if (hc.rows == 1) return cudaMemcpyAsync(dst, src, hc.width, kind, s);
-  return cudaMemcpy2DAsync(dst, hc.pitch, src, hc.pitch, hc.width, hc.rows, kind, s);
-}
-
-// only_piece >= 0 builds the graph of that piece alone (dependencies never cross pieces) and stores it in *out_exec.
-hoccl_result_t build_graph(hoccl_comm* c, const Plan& P, const std::vector<RGroup>& groups, GraphEntry* entry, int only_piece,
-                           cudaGraphExec_t* out_exec) {
-  cudaGraph_t g = nullptr;
-  CU_TRY(c, cudaGraphCreate(&g, 0));
-  std::vector<cudaGraphNode_t> tail(groups.size(), nullptr);
-  cudaGraphNode_t last_copy_node = nullptr;
-  hoccl_result_t rc = HOCCL_OK;
-  auto fail = [&](cudaError_t e, const char* what) {
-    rc = cuda_fail(c, e, what);
-  };
-  for (size_t gi = 0; gi < groups.size() && rc == HOCCL_OK; gi++) {
-    if (only_piece >= 0 && P.groups[gi].piece != only_piece) continue;
-    const RGroup& rg = groups[gi];
-    std::vector<cudaGraphNode_t> deps;
-    for (int d : rg.deps)
-      if (tail[d]) deps.push_back(tail[d]);
-    if (rg.chain_dep >= 0 && tail[rg.chain_dep] && std::find(rg.deps.begin(), rg.deps.end(), rg.chain_dep) == rg.deps.end())
-      deps.push_back(tail[rg.chain_dep]);
-    std::vector<cudaGraphNode_t> nodes;
-    cudaError_t e = cudaSuccess;
-    if (rg.kind == OP_SUM) {
-      for (size_t first = 0; first < rg.segs.size() && e == cudaSuccess; first += kMaxSegs) {
-        size_t n = std::min<size_t>(kMaxSegs, rg.segs.size() - first);
-        SumBatch b;
-        fill_sum_batch(rg, first, n, P.dtype, P.elem, &b);
-        prepare_sum_batch(&b, (int)c->sum_ctas);
-        void* args[] = {&b};
-        cudaKernelNodeParams kp = {};
-        int sum_threads = 0;
-        kp.func = const_cast<void*>(sum_kernel_entry(P.dtype, (int)c->sum_ctas, &sum_threads));
-        kp.gridDim = dim3((unsigned)c->sum_ctas);
-        kp.blockDim = dim3((unsigned)sum_threads);
-        kp.kernelParams = args;
-        // launches of one group are chained too (they share the SM budget)
-        std::vector<cudaGraphNode_t> d2 = nodes.empty() ? deps : std::vector<cudaGraphNode_t>{nodes.back()};
-        cudaGraphNode_t start_rec = nullptr;
-        std::pair<cudaEvent_t, cudaEvent_t> pe{nullptr, nullptr};
-        if (c->profile) {
-          if ((e = cudaEventCreate(&pe.first)) != cudaSuccess) break;
-          if ((e = cudaEventCreate(&pe.second)) != cudaSuccess) break;
-          entry->prof_events.push_back(pe);
-          double bytes = 0;
-          for (size_t i = 0; i < n; i++) bytes += 3.0 * (double)rg.segs[first + i].bytes;
-          entry->prof_bytes.push_back(bytes);
-          if ((e = cudaGraphAddEventRecordNode(&start_rec, g, d2.data(), d2.size(), pe.first)) != cudaSuccess) break;
-          d2.assign(1, start_rec);
-        }
-        cudaGraphNode_t kn;
-        e = cudaGraphAddKernelNode(&kn, g, d2.data(), d2.size(), &kp);
-        if (e != cudaSuccess) break;
-        cudaLaunchAttributeValue prio = {};
-        prio.priority = c->sum_priority;
-        e = cudaGraphKernelNodeSetAttribute(kn, cudaLaunchAttributePriority, &prio);
-        if (e != cudaSuccess) break;
-        if (c->profile) {
-          cudaGraphNode_t end_rec;
-          if ((e = cudaGraphAddEventRecordNode(&end_rec, g, &kn, 1, pe.second)) != cudaSuccess) break;
-          kn = end_rec;
-        }
-        nodes.assign(1, kn);
-        entry->n_sum_launches++;
-      }
-    } else if (c->path == HOCCL_PATH_CE) {
-      for (const Seg& sg : rg.segs) {
-        // optional sub-copies: driver copies of 4-8 MiB pay a ~4 us serialised start-up that smaller ones do not
-        size_t sub = sg.bytes;
-        if (c->ce_sub_bytes > 0 && sg.bytes > (size_t)c->ce_sub_bytes && sg.bytes < ((size_t)16 << 20))
-          sub = ((size_t)c->ce_sub_bytes + 255) / 256 * 256;
-        for (size_t off = 0; off < sg.bytes && e == cudaSuccess; off += sub) {
-          cudaGraphNode_t n;
-          e = cudaGraphAddMemcpyNode1D(&n, g, deps.data(), deps.size(), sg.dst + off, sg.src + off, std::min(sub, sg.bytes - off),
-                                       cudaMemcpyDeviceToDevice);
-          if (e != cudaSuccess) break;
-          nodes.push_back(n);
-          entry->n_moves++;
-        }
-        if (e != cudaSuccess) break;
-      }
-    } else if (c->path == HOCCL_PATH_CE_HOST) {
-      for (const Seg& sg : rg.segs) {
-        cudaGraphNode_t d2h, h2d;
-        e = cudaGraphAddMemcpyNode1D(&d2h, g, deps.data(), deps.size(), c->host_staging + sg.host_off, sg.src, sg.bytes,
-                                     cudaMemcpyDeviceToHost);
-        if (e != cudaSuccess) break;
-        e = cudaGraphAddMemcpyNode1D(&h2d, g, &d2h, 1, sg.dst, c->host_staging + sg.host_off, sg.bytes, cudaMemcpyHostToDevice);
-        if (e != cudaSuccess) break;
-        nodes.push_back(h2d);
-        entry->n_moves++;
-      }
-    } else {
-      for (size_t first = 0; first < rg.segs.size() && e == cudaSuccess; first += kMaxSegs) {
-        size_t n = std::min<size_t>(kMaxSegs, rg.segs.size() - first);
-        CopyBatch b;
-        fill_copy_batch(rg, first, n, &b);
-        prepare_copy_batch(&b, (int)c->copy_ctas);
-        void* args[] = {&b};
-        cudaKernelNodeParams kp = {};
-        int copy_threads = 0;
-        kp.func = const_cast<void*>(copy_kernel_entry((int)c->copy_ctas, &copy_threads));
-        kp.gridDim = dim3((unsigned)c->copy_ctas);
-        kp.blockDim = dim3((unsigned)copy_threads);
-        kp.kernelParams = args;
-        // copy launches are chained as well: the CTA budget for copies is global, two never run at the same time
-        std::vector<cudaGraphNode_t> d2 = deps;
-        if (last_copy_node && std::find(d2.begin(), d2.end(), last_copy_node) == d2.end()) d2.push_back(last_copy_node);
-        std::pair<cudaEvent_t, cudaEvent_t> pe{nullptr, nullptr};
-        if (c->profile) {
-          if ((e = cudaEventCreate(&pe.first)) != cudaSuccess) break;
-          if ((e = cudaEventCreate(&pe.second)) != cudaSuccess) break;
-          entry->prof_events.push_back(pe);
-          double bytes = 0;
-          for (size_t i = 0; i < n; i++) bytes += 2.0 * (double)rg.segs[first + i].bytes;
-          entry->prof_bytes.push_back(-bytes);   // negative: a copy launch (read + write), kept apart from the sums
-          cudaGraphNode_t start_rec;
-          if ((e = cudaGraphAddEventRecordNode(&start_rec, g, d2.data(), d2.size(), pe.first)) != cudaSuccess) break;
-          d2.assign(1, start_rec);
-        }
-        cudaGraphNode_t kn;
-        e = cudaGraphAddKernelNode(&kn, g, d2.data(), d2.size(), &kp);
-        if (e != cudaSuccess) break;
-        if (c->profile) {
-          cudaGraphNode_t end_rec;
-          if ((e = cudaGraphAddEventRecordNode(&end_rec, g, &kn, 1, pe.second)) != cudaSuccess) break;
-          kn = end_rec;
-        }
-        last_copy_node = kn;
-        nodes.push_back(kn);
-        entry->n_moves += (long)n;
-        entry->n_move_launches++;
-      }
-    }
-    if (e != cudaSuccess) {
-      fail(e, "graph node");
-      break;
-    }
-    if (nodes.size() == 1) {
-      tail[gi] = nodes[0];
-    } else if (nodes.size() > 1) {
-      cudaGraphNode_t join;
-      e = cudaGraphAddEmptyNode(&join, g, nodes.data(), nodes.size());
-      if (e != cudaSuccess) {
-        fail(e, "graph join node");
-        break;
-      }
-      tail[gi] = join;
-    }
-  }
-  if (rc == HOCCL_OK) {
-    cudaError_t e = cudaGraphInstantiate(out_exec, g, 0);
-    if (e != cudaSuccess) rc = cuda_fail(c, e, "cudaGraphInstantiate");
-  }
-  cudaGraphDestroy(g);
-  if (rc != HOCCL_OK) destroy_entry(entry);
-  return rc;
-}
-
-// Inserts an entry into the graph cache (evicting the least recently used one when it is full) and returns it.
-GraphEntry* cache_put(hoccl_comm* c, GraphEntry&& entry) {
-  if (c->cache.size() >= kGraphCacheCap) {
-    if (c->proxy) c->proxy->drain(c->watchdog_ms);  // a queued hand-over may still refer to the victim
-    size_t victim = 0;
-    for (size_t i = 1; i < c->cache.size(); i++)
-      if (c->cache[i].last_use < c->cache[victim].last_use) victim = i;
-    destroy_entry(&c->cache[victim]);
-    c->cache.erase(c->cache.begin() + victim);
-  }
-  c->cache.push_back(std::move(entry));
-  return &c->cache.back();
-}
-
-// The schedule of a user-defined pattern (paper Sec. 3.4) as a CUDA graph: stages one after the other (a join node between
-// them), inside a stage every source rank's queue is a serial chain in the scheduler's service order (copy route), or the
-// k-th operations of all queues share one batched copy launch and the launches form one chain (SM path).
-hoccl_result_t build_pattern_graph(hoccl_comm* c, const Schedule& S, const void* const* send, const size_t* sdispls, void* const* recv,
-                                   const size_t* rdispls, size_t e, GraphEntry* entry) {
-  const int R = c->R;
-  cudaGraph_t g = nullptr;
-  CU_TRY(c, cudaGraphCreate(&g, 0));
-  cudaError_t err = cudaSuccess;
-  cudaGraphNode_t stage_dep = nullptr;
-  for (size_t si = 0; si < S.stages.size() && err == cudaSuccess; si++) {
-    const Stage& st = S.stages[si];
-    auto endpoints = [&](const ChunkItem& it, const char** src, char** dst) {
-      const StageFlow& f = st.flows[it.flow];
-      *src = (const char*)send[f.origin_src] + sdispls[(size_t)f.origin_src * R + f.origin_dst] * e + f.origin_offset + it.offset;
-      *dst = (char*)recv[f.origin_dst] + rdispls[(size_t)f.origin_dst * R + f.origin_src] * e + f.origin_offset + it.offset;
-    };
-    // chunks that follow one another in a queue and continue the same flow are one operation
-    std::vector<std::vector<ChunkItem>> queues(R);
-    for (int q = 0; q < R; q++)
-      for (const ChunkItem& it : st.queues[q]) {
-        if (!queues[q].empty() && queues[q].back().flow == it.flow && queues[q].back().offset + queues[q].back().bytes == it.offset)
-          queues[q].back().bytes += it.bytes;
-        else
-          queues[q].push_back(it);
-      }
-    std::vector<cudaGraphNode_t> tails;
-    if (c->path == HOCCL_PATH_CE) {
-      for (int q = 0; q < R && err == cudaSuccess; q++) {
-        cudaGraphNode_t prev = stage_dep;
-        for (const ChunkItem& it : queues[q]) {
-          const char* src;
-          char* dst;
-          endpoints(it, &src, &dst);
-          cudaGraphNode_t n;
-          err = cudaGraphAddMemcpyNode1D(&n, g, prev ? &prev : nullptr, prev ? 1 : 0, dst, src, it.bytes, cudaMemcpyDeviceToDevice);
-          if (err != cudaSuccess) break;
-          prev = n;
-          entry->n_moves++;
-        }
-        if (prev && prev != stage_dep) tails.push_back(prev);
-      }
-    } else {
-      size_t depth = 0;
-      for (int q = 0; q < R; q++) depth = std::max(depth, queues[q].size());
-      cudaGraphNode_t prev = stage_dep;
-      auto add_launch = [&](CopyBatch& b) {
-        prepare_copy_batch(&b, (int)c->copy_ctas);
-        void* args[] = {&b};
-        cudaKernelNodeParams kp = {};
-        int threads = 0;
-        kp.func = const_cast<void*>(copy_kernel_entry((int)c->copy_ctas, &threads));
-        kp.gridDim = dim3((unsigned)c->copy_ctas);
-        kp.blockDim = dim3((unsigned)threads);
-        kp.kernelParams = args;
-        cudaGraphNode_t n;
-        err = cudaGraphAddKernelNode(&n, g, prev ? &prev : nullptr, prev ? 1 : 0, &kp);
-        if (err == cudaSuccess) {
-          prev = n;
-          entry->n_move_launches++;
-        }
-        b.nseg = 0;
-      };
-      for (size_t k = 0; k < depth && err == cudaSuccess; k++) {
-        CopyBatch b;
-        b.nseg = 0;
-        b.pad = 0;
-        for (int q = 0; q < R && err == cudaSuccess; q++) {
-          if (k >= queues[q].size()) continue;
-          const char* src;
-          char* dst;
-          endpoints(queues[q][k], &src, &dst);
-          b.seg[b.nseg++] = CopySeg{src, dst, (unsigned long long)queues[q][k].bytes};
-          entry->n_moves++;
-          if (b.nseg == kMaxSegs) add_launch(b);
-        }
-        if (b.nseg > 0 && err == cudaSuccess) add_launch(b);
-      }
-      if (prev && prev != stage_dep) tails.push_back(prev);
-    }
-    if (err != cudaSuccess) break;
-    if (tails.size() == 1) {
-      stage_dep = tails[0];
-    } else if (tails.size() > 1) {
-      cudaGraphNode_t join;
-      err = cudaGraphAddEmptyNode(&join, g, tails.data(), tails.size());
-      if (err == cudaSuccess) stage_dep = join;
-    }
-  }
-  hoccl_result_t rc = HOCCL_OK;
-  if (err == cudaSuccess) err = cudaGraphInstantiate(&entry->exec, g, 0);
-  if (err != cudaSuccess) rc = cuda_fail(c, err, "pattern graph");
-  cudaGraphDestroy(g);
-  entry->n_pieces = (long)S.stages.size();
-  if (rc != HOCCL_OK) destroy_entry(entry);
-  return rc;
-}
-
 std::vector<uint64_t> make_key(hoccl_comm* c, const Call& call) {
   std::vector<uint64_t> k;
   k.reserve(17 + 2 * c->R);
@@ -626,137 +308,6 @@ hoccl_result_t ensure_proxy(hoccl_comm* c) {
     return cuda_fail(c, e, "proxy init (stream memory operations)");
   }
   c->proxy = p;
-  return HOCCL_OK;
-}
-
-// ------------------------------------------------------------------ whole-collective kernel ------
-// The barrier words and the error word of the "fused" setting are the library's own (16 bytes of device memory and
-// 4 bytes of mapped pinned host memory), allocated on first use.
-static hoccl_result_t ensure_ring_ctrl(hoccl_comm* c) {
-  if (c->ring_bar) return HOCCL_OK;
-  unsigned* bar = nullptr;
-  int* err = nullptr;
-  int* err_dev = nullptr;
-  CU_TRY(c, cudaMalloc(&bar, 16));
-  cudaError_t e = cudaMemset(bar, 0, 16);
-  if (e == cudaSuccess) e = cudaHostAlloc(&err, sizeof(int), cudaHostAllocMapped);
-  if (e == cudaSuccess) {
-    *err = 0;
-    e = cudaHostGetDevicePointer(&err_dev, err, 0);
-  }
-  if (e == cudaSuccess) e = preload_ring_kernels();
-  if (e != cudaSuccess) {
-    cudaFree(bar);
-    if (err) cudaFreeHost(err);
-    return cuda_fail(c, e, "ring kernel control words");
-  }
-  c->ring_bar = bar;
-  c->ring_err = err;
-  c->ring_err_dev = err_dev;
-  return HOCCL_OK;
-}
-
-template <typename Args, int NPH, int NSEG>
-static bool fill_ring_args(const std::vector<RGroup>& groups, int dtype, int threads, unsigned* bar, int* err_dev, Args* a,
-                           size_t* max_phase_bytes) {
-  int nph = 0, nseg = 0;
-  *max_phase_bytes = 0;
-  a->dtype = dtype;
-  a->bar = bar;
-  a->host_err = err_dev;
-  for (const RGroup& g : groups) {
-    bool first_of_group = true;
-    for (size_t first = 0; first < g.segs.size(); first += kMaxSegs) {
-      const size_t n = std::min<size_t>(kMaxSegs, g.segs.size() - first);
-      if (nph >= NPH || nseg + (int)n > NSEG) return false;
-      RingPhase& ph = a->phase[nph++];
-      ph.first_seg = nseg;
-      ph.nseg = (int)n;
-      ph.kind = g.kind == OP_SUM ? 1 : 0;
-      ph.barrier_before = (first_of_group && !g.deps.empty()) ? 1 : 0;
-      first_of_group = false;
-      size_t bytes = 0;
-      for (size_t i = 0; i < n; i++) {
-        const Seg& sg = g.segs[first + i];
-        RingSeg rs = {};
-        rs.src = sg.src;
-        rs.local = g.kind == OP_SUM ? sg.local : nullptr;
-        rs.dst = sg.dst;
-        rs.bytes = (unsigned long long)sg.bytes;
-        a->seg[nseg++] = rs;
-        bytes += sg.bytes;
-      }
-      prepare_ring_phase(a->seg + ph.first_seg, ph.nseg, ph.kind, dtype, threads);
-      *max_phase_bytes = std::max(*max_phase_bytes, bytes);
-    }
-  }
-  a->nphase = nph;
-  return true;
-}
-
-// Turns the resolved plan into the parameter block of one ring_kernel launch.  UNSUPPORTED if the plan does not fit
-// into the kernel's parameter space (very many ranks): the caller then falls back to the graph.
-static hoccl_result_t build_ring(hoccl_comm* c, const Plan& P, const std::vector<RGroup>& groups, GraphEntry* entry) {
-  hoccl_result_t rc = ensure_ring_ctrl(c);
-  if (rc != HOCCL_OK) return rc;
-  size_t max_phase_bytes = 0;
-  bool has_sum = false;
-  for (const RGroup& g : groups) has_sum = has_sum || g.kind == OP_SUM;
-  // CTA budget: never more than either budget of the SM path; never more CTAs than the largest phase has tiles for
-  // (a barrier costs more the more CTAs take part); never more than can be resident together.
-  long budget = has_sum ? std::min(c->sum_ctas, c->copy_ctas) : c->copy_ctas;
-  const int threads = budget >= 128 ? 512 : 1024;
-  entry->ring_args.assign(sizeof(RingArgsSmall), 0);
-  entry->ring_large = false;
-  if (!fill_ring_args<RingArgsSmall, kRingSmallPhases, kRingSmallSegs>(groups, P.dtype, threads, c->ring_bar, c->ring_err_dev,
-                                                                     reinterpret_cast<RingArgsSmall*>(entry->ring_args.data()), &max_phase_bytes)) {
-    entry->ring_args.assign(sizeof(RingArgsLarge), 0);
-    entry->ring_large = true;
-    if (!fill_ring_args<RingArgsLarge, kRingLargePhases, kRingLargeSegs>(groups, P.dtype, threads, c->ring_bar, c->ring_err_dev,
-                                                                       reinterpret_cast<RingArgsLarge*>(entry->ring_args.data()), &max_phase_bytes)) {
-      entry->ring_args.clear();
-      return HOCCL_ERR_UNSUPPORTED;
-    }
-  }
-  const size_t tile_bytes = (size_t)threads * 4 * 16;
-  const long tiles = (long)((max_phase_bytes + tile_bytes - 1) / tile_bytes);
-  int max_grid = 0;
-  CU_TRY(c, ring_max_grid(threads, P.dtype, entry->ring_large, c->num_sms, &max_grid));
-  long grid = std::max<long>(1, std::min<long>(std::min<long>(budget, tiles), max_grid));
-  entry->ring_grid = (int)grid;
-  entry->ring_threads = threads;
-  entry->ring_has_sum = has_sum;
-  entry->n_moves = 0;
-  for (const RGroup& g : groups)
-    if (g.kind != OP_SUM) entry->n_moves += (long)g.segs.size();
-  entry->n_move_launches = 1;   // the one launch of the collective
-  entry->n_sum_launches = 0;
-  return HOCCL_OK;
-}
-
-// Self-test of the bounded barrier wait: two copy phases with a barrier between them that waits for one arrival more
-// than the grid can deliver.  The kernel must give up by itself, report it, and leave the barrier words clean.
-hoccl_result_t ring_barrier_selftest(hoccl_comm* c, void* dst, const void* src, size_t bytes, cudaStream_t stream) {
-  hoccl_result_t rc = ensure_ring_ctrl(c);
-  if (rc != HOCCL_OK) return rc;
-  std::vector<char> store(sizeof(RingArgsSmall), 0);
-  RingArgsSmall* a = reinterpret_cast<RingArgsSmall*>(store.data());
-  a->nphase = 2;
-  a->dtype = 0;
-  a->missing_arrivals = 1;
-  a->bar = c->ring_bar;
-  a->host_err = c->ring_err_dev;
-  const size_t half = bytes / 2;
-  for (int ph = 0; ph < 2; ph++) {
-    a->phase[ph] = RingPhase{ph, 1, 0, ph};   // phase 1 sits behind the barrier and must never run
-    RingSeg rs = {};
-    rs.src = (const char*)src + ph * half;
-    rs.dst = (char*)dst + ph * half;
-    rs.bytes = half;
-    a->seg[ph] = rs;
-    prepare_ring_phase(a->seg + ph, 1, 0, 0, 1024);
-  }
-  CU_TRY(c, launch_ring(*a, 4, 1024, stream));
   return HOCCL_OK;
 }
 

@@ -1,0 +1,322 @@
+// Graph side of libhoccl: a resolved plan (or the schedule of a user-defined pattern) becomes an explicit CUDA graph:
+// memcpy nodes for moves on the copy route, kernel nodes for sums and SM copies, empty nodes as joins.  Also the graph
+// cache and the host copies of the pipelined host all-reduce.
+#include "comm.h"
+
+namespace hoccl {
+
+void destroy_entry(GraphEntry* e) {
+  if (e->exec) cudaGraphExecDestroy(e->exec);
+  for (cudaGraphExec_t pe : e->piece_exec)
+    if (pe) cudaGraphExecDestroy(pe);
+  e->piece_exec.clear();
+  for (auto& p : e->prof_events) {
+    cudaEventDestroy(p.first);
+    cudaEventDestroy(p.second);
+  }
+  e->exec = nullptr;
+  e->prof_events.clear();
+}
+
+// Host <-> staging copies of one piece of one rank (all-reduce layout): piece p of every ring chunk, i.e. rows of
+// `piece` bytes at a pitch of one chunk.  Chunks that hold the full piece go as one 2-D copy; a shorter trailing piece
+// as a 1-D copy.
+void add_host_copies(const Plan& P, int p, char* dev, char* host, std::vector<HostCopy>* out) {
+  const size_t e = P.elem, q_bytes = P.chunk_elems * e;
+  const size_t off = (size_t)p * P.piece_bytes;
+  size_t full_rows = 0, full_len = 0;
+  for (int cidx = 0; cidx < P.R; cidx++) {
+    size_t lo, hi;
+    P.chunk_range(cidx, &lo, &hi);
+    const size_t len_bytes = (hi - lo) * e;
+    const size_t a = std::min(off, len_bytes), b = std::min(off + P.piece_bytes, len_bytes);
+    const size_t len = b - a;
+    if (len == 0) continue;
+    if (cidx == 0) full_len = len;
+    if (len == full_len && (size_t)cidx == full_rows) {
+      full_rows++;
+      continue;
+    }
+    out->push_back(HostCopy{dev + lo * e + a, host + lo * e + a, len, len, 1});
+  }
+  if (full_rows > 0) out->push_back(HostCopy{dev + off, host + off, q_bytes, full_len, full_rows});
+}
+
+cudaError_t enqueue_host_copy(const HostCopy& hc, bool to_device, cudaStream_t s) {
+  const cudaMemcpyKind kind = to_device ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToHost;
+  void* dst = to_device ? (void*)hc.dev : (void*)hc.host;
+  const void* src = to_device ? (const void*)hc.host : (const void*)hc.dev;
+  if (hc.rows == 1) return cudaMemcpyAsync(dst, src, hc.width, kind, s);
+  return cudaMemcpy2DAsync(dst, hc.pitch, src, hc.pitch, hc.width, hc.rows, kind, s);
+}
+
+// only_piece >= 0 builds the graph of that piece alone (dependencies never cross pieces) and stores it in *out_exec.
+hoccl_result_t build_graph(hoccl_comm* c, const Plan& P, const std::vector<RGroup>& groups, GraphEntry* entry, int only_piece,
+                           cudaGraphExec_t* out_exec) {
+  cudaGraph_t g = nullptr;
+  CU_TRY(c, cudaGraphCreate(&g, 0));
+  std::vector<cudaGraphNode_t> tail(groups.size(), nullptr);
+  cudaGraphNode_t last_copy_node = nullptr;
+  hoccl_result_t rc = HOCCL_OK;
+  auto fail = [&](cudaError_t e, const char* what) {
+    rc = cuda_fail(c, e, what);
+  };
+  for (size_t gi = 0; gi < groups.size() && rc == HOCCL_OK; gi++) {
+    if (only_piece >= 0 && P.groups[gi].piece != only_piece) continue;
+    const RGroup& rg = groups[gi];
+    std::vector<cudaGraphNode_t> deps;
+    for (int d : rg.deps)
+      if (tail[d]) deps.push_back(tail[d]);
+    if (rg.chain_dep >= 0 && tail[rg.chain_dep] && std::find(rg.deps.begin(), rg.deps.end(), rg.chain_dep) == rg.deps.end())
+      deps.push_back(tail[rg.chain_dep]);
+    std::vector<cudaGraphNode_t> nodes;
+    cudaError_t e = cudaSuccess;
+    if (rg.kind == OP_SUM) {
+      for (size_t first = 0; first < rg.segs.size() && e == cudaSuccess; first += kMaxSegs) {
+        size_t n = std::min<size_t>(kMaxSegs, rg.segs.size() - first);
+        SumBatch b;
+        fill_sum_batch(rg, first, n, P.dtype, P.elem, &b);
+        prepare_sum_batch(&b, (int)c->sum_ctas);
+        void* args[] = {&b};
+        cudaKernelNodeParams kp = {};
+        int sum_threads = 0;
+        kp.func = const_cast<void*>(sum_kernel_entry(P.dtype, (int)c->sum_ctas, &sum_threads));
+        kp.gridDim = dim3((unsigned)c->sum_ctas);
+        kp.blockDim = dim3((unsigned)sum_threads);
+        kp.kernelParams = args;
+        // launches of one group are chained too (they share the SM budget)
+        std::vector<cudaGraphNode_t> d2 = nodes.empty() ? deps : std::vector<cudaGraphNode_t>{nodes.back()};
+        cudaGraphNode_t start_rec = nullptr;
+        std::pair<cudaEvent_t, cudaEvent_t> pe{nullptr, nullptr};
+        if (c->profile) {
+          if ((e = cudaEventCreate(&pe.first)) != cudaSuccess) break;
+          if ((e = cudaEventCreate(&pe.second)) != cudaSuccess) break;
+          entry->prof_events.push_back(pe);
+          double bytes = 0;
+          for (size_t i = 0; i < n; i++) bytes += 3.0 * (double)rg.segs[first + i].bytes;
+          entry->prof_bytes.push_back(bytes);
+          if ((e = cudaGraphAddEventRecordNode(&start_rec, g, d2.data(), d2.size(), pe.first)) != cudaSuccess) break;
+          d2.assign(1, start_rec);
+        }
+        cudaGraphNode_t kn;
+        e = cudaGraphAddKernelNode(&kn, g, d2.data(), d2.size(), &kp);
+        if (e != cudaSuccess) break;
+        cudaLaunchAttributeValue prio = {};
+        prio.priority = c->sum_priority;
+        e = cudaGraphKernelNodeSetAttribute(kn, cudaLaunchAttributePriority, &prio);
+        if (e != cudaSuccess) break;
+        if (c->profile) {
+          cudaGraphNode_t end_rec;
+          if ((e = cudaGraphAddEventRecordNode(&end_rec, g, &kn, 1, pe.second)) != cudaSuccess) break;
+          kn = end_rec;
+        }
+        nodes.assign(1, kn);
+        entry->n_sum_launches++;
+      }
+    } else if (c->path == HOCCL_PATH_CE) {
+      for (const Seg& sg : rg.segs) {
+        // optional sub-copies: driver copies of 4-8 MiB pay a ~4 us serialised start-up that smaller ones do not
+        size_t sub = sg.bytes;
+        if (c->ce_sub_bytes > 0 && sg.bytes > (size_t)c->ce_sub_bytes && sg.bytes < ((size_t)16 << 20))
+          sub = ((size_t)c->ce_sub_bytes + 255) / 256 * 256;
+        for (size_t off = 0; off < sg.bytes && e == cudaSuccess; off += sub) {
+          cudaGraphNode_t n;
+          e = cudaGraphAddMemcpyNode1D(&n, g, deps.data(), deps.size(), sg.dst + off, sg.src + off, std::min(sub, sg.bytes - off),
+                                       cudaMemcpyDeviceToDevice);
+          if (e != cudaSuccess) break;
+          nodes.push_back(n);
+          entry->n_moves++;
+        }
+        if (e != cudaSuccess) break;
+      }
+    } else if (c->path == HOCCL_PATH_CE_HOST) {
+      for (const Seg& sg : rg.segs) {
+        cudaGraphNode_t d2h, h2d;
+        e = cudaGraphAddMemcpyNode1D(&d2h, g, deps.data(), deps.size(), c->host_staging + sg.host_off, sg.src, sg.bytes,
+                                     cudaMemcpyDeviceToHost);
+        if (e != cudaSuccess) break;
+        e = cudaGraphAddMemcpyNode1D(&h2d, g, &d2h, 1, sg.dst, c->host_staging + sg.host_off, sg.bytes, cudaMemcpyHostToDevice);
+        if (e != cudaSuccess) break;
+        nodes.push_back(h2d);
+        entry->n_moves++;
+      }
+    } else {
+      for (size_t first = 0; first < rg.segs.size() && e == cudaSuccess; first += kMaxSegs) {
+        size_t n = std::min<size_t>(kMaxSegs, rg.segs.size() - first);
+        CopyBatch b;
+        fill_copy_batch(rg, first, n, &b);
+        prepare_copy_batch(&b, (int)c->copy_ctas);
+        void* args[] = {&b};
+        cudaKernelNodeParams kp = {};
+        int copy_threads = 0;
+        kp.func = const_cast<void*>(copy_kernel_entry((int)c->copy_ctas, &copy_threads));
+        kp.gridDim = dim3((unsigned)c->copy_ctas);
+        kp.blockDim = dim3((unsigned)copy_threads);
+        kp.kernelParams = args;
+        // copy launches are chained as well: the CTA budget for copies is global, two never run at the same time
+        std::vector<cudaGraphNode_t> d2 = deps;
+        if (last_copy_node && std::find(d2.begin(), d2.end(), last_copy_node) == d2.end()) d2.push_back(last_copy_node);
+        std::pair<cudaEvent_t, cudaEvent_t> pe{nullptr, nullptr};
+        if (c->profile) {
+          if ((e = cudaEventCreate(&pe.first)) != cudaSuccess) break;
+          if ((e = cudaEventCreate(&pe.second)) != cudaSuccess) break;
+          entry->prof_events.push_back(pe);
+          double bytes = 0;
+          for (size_t i = 0; i < n; i++) bytes += 2.0 * (double)rg.segs[first + i].bytes;
+          entry->prof_bytes.push_back(-bytes);   // negative: a copy launch (read + write), kept apart from the sums
+          cudaGraphNode_t start_rec;
+          if ((e = cudaGraphAddEventRecordNode(&start_rec, g, d2.data(), d2.size(), pe.first)) != cudaSuccess) break;
+          d2.assign(1, start_rec);
+        }
+        cudaGraphNode_t kn;
+        e = cudaGraphAddKernelNode(&kn, g, d2.data(), d2.size(), &kp);
+        if (e != cudaSuccess) break;
+        if (c->profile) {
+          cudaGraphNode_t end_rec;
+          if ((e = cudaGraphAddEventRecordNode(&end_rec, g, &kn, 1, pe.second)) != cudaSuccess) break;
+          kn = end_rec;
+        }
+        last_copy_node = kn;
+        nodes.push_back(kn);
+        entry->n_moves += (long)n;
+        entry->n_move_launches++;
+      }
+    }
+    if (e != cudaSuccess) {
+      fail(e, "graph node");
+      break;
+    }
+    if (nodes.size() == 1) {
+      tail[gi] = nodes[0];
+    } else if (nodes.size() > 1) {
+      cudaGraphNode_t join;
+      e = cudaGraphAddEmptyNode(&join, g, nodes.data(), nodes.size());
+      if (e != cudaSuccess) {
+        fail(e, "graph join node");
+        break;
+      }
+      tail[gi] = join;
+    }
+  }
+  if (rc == HOCCL_OK) {
+    cudaError_t e = cudaGraphInstantiate(out_exec, g, 0);
+    if (e != cudaSuccess) rc = cuda_fail(c, e, "cudaGraphInstantiate");
+  }
+  cudaGraphDestroy(g);
+  if (rc != HOCCL_OK) destroy_entry(entry);
+  return rc;
+}
+
+// Inserts an entry into the graph cache (evicting the least recently used one when it is full) and returns it.
+GraphEntry* cache_put(hoccl_comm* c, GraphEntry&& entry) {
+  if (c->cache.size() >= kGraphCacheCap) {
+    if (c->proxy) c->proxy->drain(c->watchdog_ms);  // a queued hand-over may still refer to the victim
+    size_t victim = 0;
+    for (size_t i = 1; i < c->cache.size(); i++)
+      if (c->cache[i].last_use < c->cache[victim].last_use) victim = i;
+    destroy_entry(&c->cache[victim]);
+    c->cache.erase(c->cache.begin() + victim);
+  }
+  c->cache.push_back(std::move(entry));
+  return &c->cache.back();
+}
+
+// The schedule of a user-defined pattern (paper Sec. 3.4) as a CUDA graph: stages one after the other (a join node between
+// them), inside a stage every source rank's queue is a serial chain in the scheduler's service order (copy route), or the
+// k-th operations of all queues share one batched copy launch and the launches form one chain (SM path).
+hoccl_result_t build_pattern_graph(hoccl_comm* c, const Schedule& S, const void* const* send, const size_t* sdispls, void* const* recv,
+                                   const size_t* rdispls, size_t e, GraphEntry* entry) {
+  const int R = c->R;
+  cudaGraph_t g = nullptr;
+  CU_TRY(c, cudaGraphCreate(&g, 0));
+  cudaError_t err = cudaSuccess;
+  cudaGraphNode_t stage_dep = nullptr;
+  for (size_t si = 0; si < S.stages.size() && err == cudaSuccess; si++) {
+    const Stage& st = S.stages[si];
+    auto endpoints = [&](const ChunkItem& it, const char** src, char** dst) {
+      const StageFlow& f = st.flows[it.flow];
+      *src = (const char*)send[f.origin_src] + sdispls[(size_t)f.origin_src * R + f.origin_dst] * e + f.origin_offset + it.offset;
+      *dst = (char*)recv[f.origin_dst] + rdispls[(size_t)f.origin_dst * R + f.origin_src] * e + f.origin_offset + it.offset;
+    };
+    // chunks that follow one another in a queue and continue the same flow are one operation
+    std::vector<std::vector<ChunkItem>> queues(R);
+    for (int q = 0; q < R; q++)
+      for (const ChunkItem& it : st.queues[q]) {
+        if (!queues[q].empty() && queues[q].back().flow == it.flow && queues[q].back().offset + queues[q].back().bytes == it.offset)
+          queues[q].back().bytes += it.bytes;
+        else
+          queues[q].push_back(it);
+      }
+    std::vector<cudaGraphNode_t> tails;
+    if (c->path == HOCCL_PATH_CE) {
+      for (int q = 0; q < R && err == cudaSuccess; q++) {
+        cudaGraphNode_t prev = stage_dep;
+        for (const ChunkItem& it : queues[q]) {
+          const char* src;
+          char* dst;
+          endpoints(it, &src, &dst);
+          cudaGraphNode_t n;
+          err = cudaGraphAddMemcpyNode1D(&n, g, prev ? &prev : nullptr, prev ? 1 : 0, dst, src, it.bytes, cudaMemcpyDeviceToDevice);
+          if (err != cudaSuccess) break;
+          prev = n;
+          entry->n_moves++;
+        }
+        if (prev && prev != stage_dep) tails.push_back(prev);
+      }
+    } else {
+      size_t depth = 0;
+      for (int q = 0; q < R; q++) depth = std::max(depth, queues[q].size());
+      cudaGraphNode_t prev = stage_dep;
+      auto add_launch = [&](CopyBatch& b) {
+        prepare_copy_batch(&b, (int)c->copy_ctas);
+        void* args[] = {&b};
+        cudaKernelNodeParams kp = {};
+        int threads = 0;
+        kp.func = const_cast<void*>(copy_kernel_entry((int)c->copy_ctas, &threads));
+        kp.gridDim = dim3((unsigned)c->copy_ctas);
+        kp.blockDim = dim3((unsigned)threads);
+        kp.kernelParams = args;
+        cudaGraphNode_t n;
+        err = cudaGraphAddKernelNode(&n, g, prev ? &prev : nullptr, prev ? 1 : 0, &kp);
+        if (err == cudaSuccess) {
+          prev = n;
+          entry->n_move_launches++;
+        }
+        b.nseg = 0;
+      };
+      for (size_t k = 0; k < depth && err == cudaSuccess; k++) {
+        CopyBatch b;
+        b.nseg = 0;
+        b.pad = 0;
+        for (int q = 0; q < R && err == cudaSuccess; q++) {
+          if (k >= queues[q].size()) continue;
+          const char* src;
+          char* dst;
+          endpoints(queues[q][k], &src, &dst);
+          b.seg[b.nseg++] = CopySeg{src, dst, (unsigned long long)queues[q][k].bytes};
+          entry->n_moves++;
+          if (b.nseg == kMaxSegs) add_launch(b);
+        }
+        if (b.nseg > 0 && err == cudaSuccess) add_launch(b);
+      }
+      if (prev && prev != stage_dep) tails.push_back(prev);
+    }
+    if (err != cudaSuccess) break;
+    if (tails.size() == 1) {
+      stage_dep = tails[0];
+    } else if (tails.size() > 1) {
+      cudaGraphNode_t join;
+      err = cudaGraphAddEmptyNode(&join, g, tails.data(), tails.size());
+      if (err == cudaSuccess) stage_dep = join;
+    }
+  }
+  hoccl_result_t rc = HOCCL_OK;
+  if (err == cudaSuccess) err = cudaGraphInstantiate(&entry->exec, g, 0);
+  if (err != cudaSuccess) rc = cuda_fail(c, err, "pattern graph");
+  cudaGraphDestroy(g);
+  entry->n_pieces = (long)S.stages.size();
+  if (rc != HOCCL_OK) destroy_entry(entry);
+  return rc;
+}
+
+}  // namespace hoccl
