@@ -402,6 +402,17 @@ hoccl_result_t hoccl_copy_launch(const void* src, void* dst, size_t bytes, int c
  * smid_out[block index], a device array of `ctas` 32-bit words.  The number of distinct values is the number of SMs
  * the launch occupied.  Same kernels and launch shapes as the collectives use.
  */
+/*
+ * Host only (no device needed): the flattened view the host passes to a batched SUM (kind 0) or copy (kind 1) launch for
+ * `nseg` segments given by their ADDRESSES as integers (a, b, out; b unused for the copy) and lengths (elements for the
+ * SUM, bytes for the copy) under the kernel shape that `ctas` selects.  Per segment: head (element-wise items before the
+ * 16-byte vector body), nvec (vectors in the body), and the running totals of tiles and of element-wise items;
+ * *tile_vectors is the tile size in vectors.  The kernels trust this view for every address they form, so tests check its
+ * invariants on the CPU: nothing is read or written.
+ */
+hoccl_result_t hoccl_flatten_inspect(int kind, hoccl_dtype_t dtype, int ctas, int nseg, const uint64_t* a_addr, const uint64_t* b_addr,
+                                     const uint64_t* out_addr, const uint64_t* len, uint64_t* tiles_end, uint64_t* scalars_end,
+                                     uint64_t* nvec, uint32_t* head, uint64_t* tile_vectors);
 hoccl_result_t hoccl_kernel_sms(int kind, const void* a, const void* b, void* out, size_t bytes, hoccl_dtype_t dtype, int ctas,
                                 unsigned int* smid_out, hoccl_stream_t stream);
 

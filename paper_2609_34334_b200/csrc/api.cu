@@ -598,6 +598,45 @@ hoccl_result_t hoccl_sum_launch(const void* inbox, const void* local, void* out,
   return launch_sum(b, ctas, (cudaStream_t)stream) == cudaSuccess ? HOCCL_OK : HOCCL_ERR_CUDA;
 }
 
+hoccl_result_t hoccl_flatten_inspect(int kind, hoccl_dtype_t dtype, int ctas, int nseg, const uint64_t* a_addr, const uint64_t* b_addr,
+                                     const uint64_t* out_addr, const uint64_t* len, uint64_t* tiles_end, uint64_t* scalars_end, uint64_t* nvec,
+                                     uint32_t* head, uint64_t* tile_vectors) {
+  if ((kind != 0 && kind != 1) || nseg < 1 || nseg > kMaxSegs || !a_addr || !out_addr || (kind == 0 && !b_addr) || !len || !tiles_end ||
+      !scalars_end || !nvec || !head || !tile_vectors || ctas < 1)
+    return HOCCL_ERR_INVALID_ARG;
+  if (kind == 0 && dtype_size((int)dtype) == 0) return HOCCL_ERR_UNSUPPORTED;
+  const Flat* f = nullptr;
+  SumBatch sb;
+  CopyBatch cb;
+  if (kind == 0) {
+    sb.nseg = nseg;
+    sb.dtype = (int)dtype;
+    for (int k = 0; k < nseg; k++)
+      sb.seg[k] = SumSeg{(const void*)(uintptr_t)a_addr[k], (const void*)(uintptr_t)b_addr[k], (void*)(uintptr_t)out_addr[k], len[k]};
+    prepare_sum_batch(&sb, ctas);
+    f = &sb.flat;
+    int threads = 0;
+    (void)sum_kernel_entry((int)dtype, ctas, &threads);
+    *tile_vectors = 4ull * (uint64_t)threads;
+  } else {
+    cb.nseg = nseg;
+    cb.pad = 0;
+    for (int k = 0; k < nseg; k++) cb.seg[k] = CopySeg{(const void*)(uintptr_t)a_addr[k], (void*)(uintptr_t)out_addr[k], len[k]};
+    prepare_copy_batch(&cb, ctas);
+    f = &cb.flat;
+    int threads = 0;
+    (void)copy_kernel_entry(ctas, &threads);
+    *tile_vectors = (threads == 1024 ? 8ull : 4ull) * (uint64_t)threads;
+  }
+  for (int k = 0; k < nseg; k++) {
+    tiles_end[k] = f->tpre[k + 1];
+    scalars_end[k] = f->spre[k + 1];
+    nvec[k] = f->nvec[k];
+    head[k] = f->head[k];
+  }
+  return HOCCL_OK;
+}
+
 hoccl_result_t hoccl_kernel_sms(int kind, const void* a, const void* b, void* out, size_t bytes, hoccl_dtype_t dtype, int ctas,
                                 unsigned int* smid_out, hoccl_stream_t stream) {
   size_t e = dtype_size((int)dtype);
