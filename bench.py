@@ -275,15 +275,12 @@ def main():
     rs_stats = comm.last_stats()
     launches_per_step = rs_stats["n_sum_launches"] + rs_stats["n_move_launches"]
 
-    # parity of the timed configuration on bucket set 0 (sampled: rank 0 and rank 5, full vectors)
+    # results of the timed configuration on bucket set 0 (ranks 0 and 5, full vectors), kept for the comparison with the
+    # oracle, which happens where the oracle runs: in the CPU-baseline leg below
     parity = None
-    if world.rank == 0:
-        from oracle import ring as oracle_ring
-
-        want = oracle_ring.ring_allreduce(xs, threads=oracle_ring.max_threads())
-        step(comm, 0, stream)
-        stream.synchronize()
-        parity = all(bool((recv_sets[0][r].cpu().numpy().view(np.uint16) == want[r]).all()) for r in (0, 5))
+    step(comm, 0, stream)
+    stream.synchronize()
+    got_parity = {r: recv_sets[0][r].cpu().numpy().view(np.uint16).copy() for r in (0, 5)}
 
     t_slowest = replicas.max_over_ranks(world, t_step)
     units = replicas.sum_over_ranks(world, S * bus_factor(R))
@@ -303,8 +300,7 @@ def main():
     k_e2e = max(3, min(steps, 20))
     t_e2e, _ = timed(comm, k_e2e, 3, fn=e2e_step)
     e2e_ok = None
-    if world.rank == 0:
-        e2e_ok = bool((h_recv[3].numpy().view(np.uint16) == want[3]).all())
+    got_e2e = h_recv[3].numpy().view(np.uint16).copy()
     t_e2e_slowest = replicas.max_over_ranks(world, t_e2e)
     e2e_value = units / t_e2e_slowest / 1e9
 
@@ -402,12 +398,17 @@ def main():
 
     if world.rank == 0 and world.size == 1:
         # ---- CPU baseline: the oracle on the host cores, whole bucket, a few repetitions
+        from oracle import ring as oracle_ring
+
         thr = oracle_ring.max_threads()
         reps, t0 = 0, time.perf_counter()
         while reps < 3 or (time.perf_counter() - t0 < 2.5 and reps < 50):
-            oracle_ring.ring_allreduce(xs, threads=thr)
+            want = oracle_ring.ring_allreduce(xs, threads=thr)
             reps += 1
         t_cpu = (time.perf_counter() - t0) / reps
+        # the oracle's result against what the device produced in the timed configuration and end to end
+        line["matches_oracle"] = all(bool((got_parity[r] == want[r]).all()) for r in got_parity)
+        line["e2e"]["matches_oracle"] = bool((got_e2e == want[3]).all())
         t1 = time.perf_counter()
         oracle_ring.ring_allreduce(xs, threads=1)          # the canonical single-thread run (the parity reference)
         t_single = time.perf_counter() - t1
