@@ -713,3 +713,31 @@ def test_graph_cache_eviction_with_work_in_flight(oracle):
             assert same_bits(recv[r].get(np.float32), want[r], dtype), (n, r)
             assert recv[r].guards_intact()
     assert comm.destroy() == hb.OK
+
+
+@pytest.mark.parametrize("params", [dict(), dict(path=hb.PATH_SM, sum_ctas=8, copy_ctas=8), dict(path=hb.PATH_SM, fused=1, sum_ctas=148, copy_ctas=148)])
+def test_two_communicators_on_two_streams_at_once(oracle, params):
+    """Collectives that overlap in time must not share a communicator; two communicators on two streams may run at the same
+    time and must not disturb each other (no state is shared between communicators)."""
+    R, dtype = 4, "bf16"
+    ns = (4 * 70_000 + 3, 4 * 90_000 + 1)
+    p = dict(params)
+    path = p.pop("path", hb.PATH_CE)
+    comms, sends, recvs, wants, streams = [], [], [], [], []
+    for k, n in enumerate(ns):
+        xs = W.rank_inputs("normal", 300 + k, R, n, dtype, 1e-3)
+        wants.append(oracle.ring_allreduce(xs))
+        comms.append(make_comm(R, n, dtype, path, **p))
+        sends.append([DevBuf(n * 2).put(x) for x in xs])
+        recvs.append([DevBuf(n * 2) for _ in range(R)])
+        streams.append(torch.cuda.Stream())
+    for rep in range(6):                                   # interleaved issue, no host synchronisation in between
+        for k in range(2):
+            comms[k].allreduce(sends[k], recvs[k], ns[k], dtype, streams[k])
+    torch.cuda.synchronize()
+    for k in range(2):
+        for r in range(R):
+            assert same_bits(recvs[k][r].get(np.uint16), wants[k][r], dtype), (k, r)
+            assert recvs[k][r].guards_intact() and sends[k][r].guards_intact()
+        assert comms[k].async_error() == hb.OK
+        assert comms[k].destroy() == hb.OK
