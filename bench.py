@@ -668,8 +668,9 @@ def extras(hb, W, torch, np, new_comm, step, timed, stream, R, S, n, dtype, peak
     for name, path, sc, cc, op, fw in (("CE_sum8", hb.PATH_CE, 8, 8, 0, 0), ("SM_copy8_sum8", hb.PATH_SM, 8, 8, 0, 0),
                                        ("SM_copy32_sum8", hb.PATH_SM, 8, 32, 0, 0), ("SM_copy148_sum148", hb.PATH_SM, 148, 148, 0, 0),
                                        ("SM_forward_copy8_sum8", hb.PATH_SM, 8, 8, 0, 1),
+                                       ("SM_one_kernel_8", hb.PATH_SM, 8, 8, 0, 2),
                                        ("onepass_8", hb.PATH_CE, 8, 8, 1, 0), ("CE_HOST_sum8", hb.PATH_CE_HOST, 8, 8, 0, 0)):
-        c2 = new_comm(path, sum_ctas=sc, copy_ctas=cc, onepass=op, forward=fw)
+        c2 = new_comm(path, sum_ctas=sc, copy_ctas=cc, onepass=op, forward=1 if fw == 1 else 0, fused=1 if fw == 2 else 0)
         if path == hb.PATH_CE_HOST:
             c2.set_host_staging(host_stage)
         tf, bw = gemm_tflops(c2)
