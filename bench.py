@@ -634,7 +634,7 @@ def extras(hb, W, torch, np, new_comm, step, timed, stream, R, S, n, dtype, peak
     C = torch.empty(4096, 4096, dtype=torch.bfloat16, device="cuda")
     flops = 2.0 * 4096 ** 3
 
-    def gemm_tflops(cm_, n_gemm=150):
+    def gemm_tflops(cm_, n_gemm=150, fn=step):
         with torch.cuda.stream(gs):
             for _ in range(10):
                 torch.matmul(A, B, out=C)
@@ -643,7 +643,7 @@ def extras(hb, W, torch, np, new_comm, step, timed, stream, R, S, n, dtype, peak
         c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         n_comm = 0
         if cm_ is not None:
-            t_c, _ = timed(cm_, 10, 3)
+            t_c, _ = timed(cm_, 10, 3, fn=fn)
             n_comm = int(1.5 * n_gemm * 80e-6 / t_c) + 2
         c0.record(stream)
         g0.record(gs)
@@ -653,7 +653,7 @@ def extras(hb, W, torch, np, new_comm, step, timed, stream, R, S, n, dtype, peak
                 torch.matmul(A, B, out=C)
             want_c = (i + 1) * n_comm // n_gemm
             while done_c < want_c:
-                step(cm_, done_c % N_BUCKET_SETS, stream)
+                fn(cm_, done_c % N_BUCKET_SETS, stream)
                 done_c += 1
         g1.record(gs)
         c1.record(stream)
@@ -673,7 +673,8 @@ def extras(hb, W, torch, np, new_comm, step, timed, stream, R, S, n, dtype, peak
         c2 = new_comm(path, sum_ctas=sc, copy_ctas=cc, onepass=op, forward=1 if fw == 1 else 0, fused=1 if fw == 2 else 0)
         if path == hb.PATH_CE_HOST:
             c2.set_host_staging(host_stage)
-        tf, bw = gemm_tflops(c2)
+        # the one-pass comparison kernel is one all-reduce call (reduce-scatter + all-gather would add the path's moves)
+        tf, bw = gemm_tflops(c2, fn=one_call if op else step)
         probe[name] = {"gemm_TFLOPs": tf, "loss": 1.0 - tf / alone, "comm_busbw_GBps": bw}
         c2.destroy()
     out["gemm_probe_4096"] = probe
