@@ -482,7 +482,7 @@ def extras(hb, W, torch, np, new_comm, step, timed, stream, R, S, n, dtype, peak
     out = {}
     k, w = 40, 5
     variants = [("CE", hb.PATH_CE, 8, 8), ("CE", hb.PATH_CE, 32, 8), ("CE", hb.PATH_CE, 148, 8), ("SM", hb.PATH_SM, 8, 8),
-                ("SM", hb.PATH_SM, 8, 32), ("SM", hb.PATH_SM, 148, 148), ("SM", hb.PATH_SM, 296, 296)]
+                ("SM", hb.PATH_SM, 8, 32), ("SM", hb.PATH_SM, 8, 48), ("SM", hb.PATH_SM, 148, 148), ("SM", hb.PATH_SM, 296, 296)]
     rows = []
     hbm = 7.0 * S * (R - 1)
     for name, path, sc, cc in variants:
@@ -494,7 +494,7 @@ def extras(hb, W, torch, np, new_comm, step, timed, stream, R, S, n, dtype, peak
     out["variants"] = rows
     # SM footprint of this library's kernels on the SM path (SMs x busy time per step), per-launch CUDA events in the graph
     fp_rows = []
-    for sc, cc in ((8, 8), (8, 32), (148, 148)):
+    for sc, cc in ((8, 8), (8, 32), (8, 48), (148, 148)):
         cm = new_comm(hb.PATH_SM, sum_ctas=sc, copy_ctas=cc, profile=1)
         for b in range(4):
             step(cm, b, stream)
@@ -666,7 +666,8 @@ def extras(hb, W, torch, np, new_comm, step, timed, stream, R, S, n, dtype, peak
     alone, _ = gemm_tflops(None)
     probe["alone_TFLOPs"] = alone
     for name, path, sc, cc, op, fw in (("CE_sum8", hb.PATH_CE, 8, 8, 0, 0), ("SM_copy8_sum8", hb.PATH_SM, 8, 8, 0, 0),
-                                       ("SM_copy32_sum8", hb.PATH_SM, 8, 32, 0, 0), ("SM_copy148_sum148", hb.PATH_SM, 148, 148, 0, 0),
+                                       ("SM_copy32_sum8", hb.PATH_SM, 8, 32, 0, 0), ("SM_copy48_sum8", hb.PATH_SM, 8, 48, 0, 0),
+                                       ("SM_copy148_sum148", hb.PATH_SM, 148, 148, 0, 0),
                                        ("SM_forward_copy8_sum8", hb.PATH_SM, 8, 8, 0, 1),
                                        ("SM_one_kernel_8", hb.PATH_SM, 8, 8, 0, 2),
                                        ("onepass_8", hb.PATH_CE, 8, 8, 1, 0), ("CE_HOST_sum8", hb.PATH_CE_HOST, 8, 8, 0, 0)):
