@@ -78,6 +78,11 @@ class HocclError(RuntimeError):
 _lib = None
 
 
+def library_path() -> str:
+    """Path of libhoccl.so (built first if it is missing or stale)."""
+    return _build.build()
+
+
 def lib() -> ctypes.CDLL:
     """Builds (if stale) and loads libhoccl.so.  Raises if that is not possible."""
     global _lib

@@ -62,3 +62,29 @@ def test_no_device_fails_loudly():
     with pytest.raises(hb.HocclError) as ei:
         hb.Comm(4, 0)
     assert ei.value.code == hb.ERR_CUDA
+
+
+def test_header_is_plain_c_and_a_c_program_links_against_the_library(tmp_path):
+    """The boundary is a C ABI: the header compiles as strict C99 (and as C++), and a C program that names every entry
+    point links against libhoccl.so and runs its host-only calls (no device needed)."""
+    import shutil
+    import subprocess
+    if not shutil.which("gcc"):
+        pytest.skip("no C compiler")
+    inc = os.path.join(ROOT, "include")
+    libdir = os.path.dirname(hb.library_path())
+    names = _declared_functions()
+    src = tmp_path / "use_hoccl.c"
+    refs = "\n".join("  fns[n++] = (void (*)(void))%s;" % n for n in names)
+    src.write_text('#include <stdio.h>\n#include <string.h>\n#include "hoccl.h"\nint main(void) {\n  void (*fns[128])(void);\n  int n = 0;\n'
+                   + refs + '\n  if (strcmp(hoccl_error_string(HOCCL_OK), "ok") != 0) return 2;\n'
+                   '  if (hoccl_scratch_bytes(1, 1000, HOCCL_FLOAT32) != 0) return 3;\n'
+                   '  if (hoccl_comm_set_path(0, HOCCL_PATH_CE) != HOCCL_ERR_INVALID_ARG) return 4;\n'
+                   '  for (int k = 0; k < n; k++) if (!fns[k]) return 5;\n'
+                   '  printf("%d entry points\\n", n);\n  return 0;\n}\n')
+    subprocess.run(["gcc", "-std=c99", "-Wall", "-Wextra", "-Werror", "-pedantic", "-fsyntax-only", "-I", inc, str(src)], check=True)
+    subprocess.run(["g++", "-std=c++11", "-Wall", "-Werror", "-fsyntax-only", "-x", "c++", "-I", inc, str(src)], check=True)
+    exe = tmp_path / "use_hoccl"
+    subprocess.run(["gcc", "-std=c99", "-I", inc, str(src), "-o", str(exe), "-L", libdir, "-lhoccl", "-Wl,-rpath," + libdir], check=True)
+    out = subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout
+    assert out.strip() == "%d entry points" % len(names)
