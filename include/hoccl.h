@@ -403,6 +403,13 @@ hoccl_result_t hoccl_copy_launch(const void* src, void* dst, size_t bytes, int c
  * the launch occupied.  Same kernels and launch shapes as the collectives use.
  */
 /*
+ * Memory-port probe behind the 8-SM ceiling quoted for the SUM: `ctas` CTAs of 1024 threads only read (mode 0) or only
+ * write (mode 1) the device buffer `buf` (16-byte aligned, at least 128 KiB; whole 128 KiB tiles are walked) with 16-byte
+ * accesses, 8 in flight per thread.  `sink` is a device word the read mode may write once.  Timed by the caller; together
+ * with hoccl_copy_launch (1 read : 1 write) and hoccl_sum_launch (2 : 1) it gives what one SM's memory port carries.
+ */
+hoccl_result_t hoccl_port_probe(int mode, void* buf, size_t bytes, int ctas, unsigned int* sink, hoccl_stream_t stream);
+/*
  * Host only (no device needed): the flattened view the host passes to a batched SUM (kind 0) or copy (kind 1) launch for
  * `nseg` segments given by their ADDRESSES as integers (a, b, out; b unused for the copy) and lengths (elements for the
  * SUM, bytes for the copy) under the kernel shape that `ctas` selects.  Per segment: head (element-wise items before the

@@ -26,7 +26,7 @@ EXPORTS = [
     "hoccl_comm_init", "hoccl_comm_destroy", "hoccl_scratch_bytes", "hoccl_comm_set_scratch", "hoccl_comm_set_staging", "hoccl_comm_set_host_staging",
     "hoccl_comm_set_path", "hoccl_comm_set_param", "hoccl_comm_get_param", "hoccl_allreduce", "hoccl_reduce_scatter",
     "hoccl_allgather", "hoccl_alltoall", "hoccl_alltoallv", "hoccl_send", "hoccl_recv", "hoccl_comm_pending", "hoccl_comm_async_error", "hoccl_comm_handshakes", "hoccl_selftest_barrier_timeout", "hoccl_host_allreduce", "hoccl_error_string",
-    "hoccl_last_cuda_error", "hoccl_last_stats", "hoccl_profile_reset", "hoccl_probe_move_needs_sm", "hoccl_probe_copy_routes", "hoccl_sum_launch", "hoccl_kernel_sms", "hoccl_flatten_inspect",
+    "hoccl_last_cuda_error", "hoccl_last_stats", "hoccl_profile_reset", "hoccl_probe_move_needs_sm", "hoccl_probe_copy_routes", "hoccl_sum_launch", "hoccl_kernel_sms", "hoccl_flatten_inspect", "hoccl_port_probe",
     "hoccl_copy_launch", "hoccl_plan_build", "hoccl_plan_destroy", "hoccl_plan_num_ops", "hoccl_plan_num_groups",
     "hoccl_plan_get_op", "hoccl_plan_group_deps", "hoccl_plan_slot_bytes", "hoccl_allreduce_static",
     "hoccl_sched_build", "hoccl_sched_destroy", "hoccl_sched_num_stages", "hoccl_sched_stage_tau", "hoccl_sched_total_tau",
@@ -134,6 +134,7 @@ def lib() -> ctypes.CDLL:
         "hoccl_copy_launch": (i, [vp, vp, sz, i, vp]),
         "hoccl_kernel_sms": (i, [i, vp, vp, vp, sz, i, i, vp, vp]),
         "hoccl_selftest_barrier_timeout": (i, [vp, vp, vp, sz, vp]),
+        "hoccl_port_probe": (i, [i, vp, sz, i, vp, vp]),
         "hoccl_flatten_inspect": (i, [i, i, i, i, vp, vp, vp, vp, vp, vp, vp, vp, vp]),
         "hoccl_plan_build": (i, [vpp, i, i, sz, i, i, sz, i, ctypes.c_char_p]),
         "hoccl_plan_slot_bytes": (sz, [vp]),
@@ -366,6 +367,11 @@ def kernel_sms(kind: str, a, b, out, nbytes: int, dtype, ctas: int, smid_out, st
     smid_out (a device array of `ctas` 32-bit words).  Returns the result code."""
     return lib().hoccl_kernel_sms(0 if kind == "sum" else 1, _ptr(a), _ptr(b) if b is not None else None, _ptr(out), nbytes,
                                   _dtype(dtype), ctas, _ptr(smid_out), _stream(stream))
+
+
+def port_probe(mode: str, buf, nbytes: int, ctas: int, sink, stream=None) -> int:
+    """hoccl_port_probe: `ctas` CTAs only read ("read") or only write ("write") the buffer."""
+    return lib().hoccl_port_probe(0 if mode == "read" else 1, _ptr(buf), nbytes, ctas, _ptr(sink), _stream(stream))
 
 
 def flatten_inspect(kind: str, dtype, ctas: int, a_addr, b_addr, out_addr, lens):

@@ -598,6 +598,11 @@ hoccl_result_t hoccl_sum_launch(const void* inbox, const void* local, void* out,
   return launch_sum(b, ctas, (cudaStream_t)stream) == cudaSuccess ? HOCCL_OK : HOCCL_ERR_CUDA;
 }
 
+hoccl_result_t hoccl_port_probe(int mode, void* buf, size_t bytes, int ctas, unsigned int* sink, hoccl_stream_t stream) {
+  if ((mode != 0 && mode != 1) || !buf || !sink || ((uintptr_t)buf & 15) || bytes < (128u << 10) || ctas < 1 || ctas > 1024) return HOCCL_ERR_INVALID_ARG;
+  return launch_port_probe(mode, buf, bytes, ctas, sink, (cudaStream_t)stream) == cudaSuccess ? HOCCL_OK : HOCCL_ERR_CUDA;
+}
+
 hoccl_result_t hoccl_flatten_inspect(int kind, hoccl_dtype_t dtype, int ctas, int nseg, const uint64_t* a_addr, const uint64_t* b_addr,
                                      const uint64_t* out_addr, const uint64_t* len, uint64_t* tiles_end, uint64_t* scalars_end, uint64_t* nvec,
                                      uint32_t* head, uint64_t* tile_vectors) {

@@ -233,6 +233,35 @@ __global__ void __launch_bounds__(THREADS, 1) onepass_kernel(const __grid_consta
   }
 }
 
+// ---- memory-port probe: what one SM can read, or write, when it does nothing else ---------------------------------
+// mode 0: every thread streams 16-byte loads (8 in flight) over its share of the buffer and folds them into one word
+// that is stored once; mode 1: every thread streams 16-byte stores.  Same tile walk as the copy kernel.
+template <int MODE>
+__global__ void __launch_bounds__(1024, 1) port_probe_kernel(uint4* buf, unsigned long long nvec, unsigned int* sink) {
+  constexpr int U = 8;
+  const unsigned long long tile = (unsigned long long)U * 1024, ntiles = nvec / tile;
+  uint4 acc = make_uint4(0, 0, 0, 0);
+  for (unsigned long long t = blockIdx.x; t < ntiles; t += gridDim.x) {
+    uint4* p = buf + t * tile + threadIdx.x;
+    if (MODE == 0) {
+      uint4 v[U];
+#pragma unroll
+      for (int u = 0; u < U; u++) v[u] = __ldcs(p + u * 1024);
+#pragma unroll
+      for (int u = 0; u < U; u++) {
+        acc.x ^= v[u].x;
+        acc.y ^= v[u].y;
+        acc.z ^= v[u].z;
+        acc.w ^= v[u].w;
+      }
+    } else {
+#pragma unroll
+      for (int u = 0; u < U; u++) p[u * 1024] = make_uint4((unsigned)t, u, threadIdx.x, 0);
+    }
+  }
+  if (MODE == 0 && (acc.x ^ acc.y ^ acc.z ^ acc.w) == 0x9e3779b9u) *sink = 1;   // keeps the loads alive
+}
+
 __device__ __forceinline__ unsigned long long global_ns() {
   unsigned long long t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
@@ -322,6 +351,12 @@ cudaError_t launch_copy(const CopyBatch& batch, int ctas, cudaStream_t stream) {
   prepare_copy_batch(&b, ctas);
   if (wide_copy_grid(ctas)) copy_kernel<4, 512><<<ctas, 512, 0, stream>>>(b);
   else copy_kernel<8, 1024><<<ctas, 1024, 0, stream>>>(b);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_port_probe(int mode, void* buf, unsigned long long bytes, int ctas, unsigned int* sink, cudaStream_t stream) {
+  if (mode == 0) port_probe_kernel<0><<<ctas, 1024, 0, stream>>>(static_cast<uint4*>(buf), bytes / 16, sink);
+  else port_probe_kernel<1><<<ctas, 1024, 0, stream>>>(static_cast<uint4*>(buf), bytes / 16, sink);
   return cudaGetLastError();
 }
 

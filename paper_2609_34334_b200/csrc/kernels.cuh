@@ -120,6 +120,9 @@ void prepare_copy_batch(CopyBatch* batch, int ctas);
 const void* sum_kernel_entry(int dtype, int ctas, int* threads);
 const void* copy_kernel_entry(int ctas, int* threads);
 
+// Memory-port probe: `ctas` CTAs only read (mode 0) or only write (mode 1) `bytes` bytes (a multiple of 128 KiB is walked).
+cudaError_t launch_port_probe(int mode, void* buf, unsigned long long bytes, int ctas, unsigned int* sink, cudaStream_t stream);
+
 // Loads every kernel of the library on the current device (no launch).
 cudaError_t preload_kernels();
 

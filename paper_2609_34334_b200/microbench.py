@@ -3,6 +3,7 @@
     python -m paper_2609_34334_b200.microbench --kernel sum --dtype bf16 --mib 200 --ctas 8 --reps 5
     python -m paper_2609_34334_b200.microbench --kernel routes --mib 16      # which same-device copy routes need an SM
     python -m paper_2609_34334_b200.microbench --kernel ring --mib 32 --ctas 148   # all-reduce, R = 8, as one cooperative kernel
+    python -m paper_2609_34334_b200.microbench --kernel port --mib 256 --ctas 8    # what the memory ports of `ctas` SMs carry
 
 Operands are larger than L2 by default; timing uses CUDA events on the launching stream after warm-up.
 Prints one JSON line.  This is the small case used for ncu captures of a single kernel.
@@ -19,7 +20,7 @@ from . import binding as hb
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--kernel", default="sum", choices=["sum", "copy", "routes", "ring"])
+    ap.add_argument("--kernel", default="sum", choices=["sum", "copy", "routes", "ring", "port"])
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "fp32"])
     ap.add_argument("--mib", type=int, default=200, help="MiB per operand")
     ap.add_argument("--ctas", type=int, default=8)
@@ -28,6 +29,33 @@ def main():
     args = ap.parse_args()
     torch.cuda.set_device(0)
     nbytes = args.mib << 20
+    if args.kernel == "port":
+        # read only, write only, 1 : 1 copy and 2 : 1 sum with the same number of CTAs (one CTA occupies one SM)
+        n = nbytes // 2
+        a = torch.empty(n, dtype=torch.bfloat16, device="cuda").normal_(0, 1e-3)
+        b = torch.empty(n, dtype=torch.bfloat16, device="cuda").normal_(0, 1e-3)
+        o = torch.empty(n, dtype=torch.bfloat16, device="cuda")
+        sink = torch.zeros(1, dtype=torch.int32, device="cuda")
+        st = torch.cuda.Stream()
+        cases = {"read_only": (lambda: hb.port_probe("read", a, nbytes, args.ctas, sink, st), nbytes),
+                 "write_only": (lambda: hb.port_probe("write", o, nbytes, args.ctas, sink, st), nbytes),
+                 "copy_1r_1w": (lambda: hb.copy_launch(a, o, nbytes, args.ctas, st), 2 * nbytes),
+                 "sum_2r_1w": (lambda: hb.sum_launch(a, b, o, n, "bf16", args.ctas, st), 3 * nbytes)}
+        out = {"probe": "memory ports of %d SMs (one 1024-thread CTA each), %d MiB operands" % (args.ctas, args.mib), "ctas": args.ctas}
+        for name, (fn, moved) in cases.items():
+            for _ in range(args.warmup):
+                assert fn() == hb.OK
+            st.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(st)
+            for _ in range(args.reps):
+                fn()
+            e1.record(st)
+            st.synchronize()
+            sec = e0.elapsed_time(e1) / 1e3 / args.reps
+            out[name] = {"GBps": moved / sec / 1e9, "GBps_per_sm": moved / sec / 1e9 / args.ctas, "us": sec * 1e6}
+        print(json.dumps(out))
+        return
     if args.kernel == "ring":
         R = 8
         e = 2 if args.dtype == "bf16" else 4

@@ -741,3 +741,23 @@ def test_two_communicators_on_two_streams_at_once(oracle, params):
             assert recvs[k][r].guards_intact() and sends[k][r].guards_intact()
         assert comms[k].async_error() == hb.OK
         assert comms[k].destroy() == hb.OK
+
+
+def test_port_probe_reads_and_writes_what_it_says():
+    """The memory-port probe behind the 8-SM ceiling: write mode stores a known pattern over whole 128 KiB tiles and
+    nothing else; read mode leaves the buffer alone."""
+    nbytes = (3 * 128 << 10) + 4096                     # three tiles and a remainder that must stay untouched
+    buf = torch.full((nbytes // 4,), -1, dtype=torch.int32, device="cuda")
+    sink = torch.zeros(1, dtype=torch.int32, device="cuda")
+    assert hb.port_probe("write", buf, nbytes, 2, sink) == hb.OK
+    torch.cuda.synchronize()
+    v = buf.cpu().numpy().reshape(-1, 4)
+    tile_vecs = 8 * 1024
+    for t, u, tid in ((0, 0, 0), (0, 1, 5), (1, 7, 1023), (2, 3, 77)):
+        assert v[t * tile_vecs + u * 1024 + tid].tolist() == [t, u, tid, 0]
+    assert (v[3 * tile_vecs:] == -1).all()
+    before = buf.clone()
+    assert hb.port_probe("read", buf, nbytes, 2, sink) == hb.OK
+    torch.cuda.synchronize()
+    assert torch.equal(buf, before)
+    assert hb.port_probe("read", buf, 1024, 2, sink) == hb.ERR_INVALID_ARG
