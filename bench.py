@@ -541,6 +541,23 @@ def extras(hb, W, torch, np, new_comm, step, timed, stream, R, S, n, dtype, peak
         fw_rows.append({"path": name, "sum_ctas": sc, "ms_per_step": t * 1e3, "busbw_GBps": S * bus_factor(R) / t / 1e9})
         c1.destroy()
     out["forward_variant"] = fw_rows
+    # direct all-gather: R-1 independent permutation stages r -> r+k instead of R-1 dependent ring hops (rank local, same bytes)
+    ad_rows = []
+    for name, path, sc, cc, fw in (("CE", hb.PATH_CE, 8, 8, 0), ("CE", hb.PATH_CE, 148, 8, 0), ("SM", hb.PATH_SM, 8, 8, 0),
+                                   ("SM", hb.PATH_SM, 8, 48, 0), ("SM", hb.PATH_SM, 148, 148, 0), ("SM", hb.PATH_SM, 148, 148, 1)):
+        c1 = new_comm(path, sum_ctas=sc, copy_ctas=cc, ag_direct=1, forward=fw)
+        t, _ = timed(c1, k, w)
+        # algorithmic bytes: the copy route moves every stage separately (the ring's 2 S (R-1) for the all-gather); the SM path
+        # reads every chunk once and stores it R-1 times (S R); the forward variant is a comparison point, no fraction given
+        ag_bytes = 2.0 * S * (R - 1) if path == hb.PATH_CE else 1.0 * S * R
+        hbm_d = 5.0 * S * (R - 1) + ag_bytes
+        t1, _ = timed(c1, k, w, fn=one_call)
+        ad_rows.append({"path": name, "sum_ctas": sc, "copy_ctas": cc if path == hb.PATH_SM else None, "forward": fw, "ms_per_step": t * 1e3,
+                        "busbw_GBps": S * bus_factor(R) / t / 1e9, "hbm_bytes_per_step": None if fw else hbm_d,
+                        "hbm_frac_of_8TBps": None if fw else hbm_d / t / 1e9 / NOMINAL_HBM_GBS,
+                        "one_allreduce_call_ms": t1 * 1e3, "one_allreduce_call_busbw_GBps": S * bus_factor(R) / t1 / 1e9})
+        c1.destroy()
+    out["direct_allgather"] = ad_rows
     # SM path with the whole collective as one cooperative kernel (grid barriers instead of kernel boundaries)
     fu_rows = []
     for ctas in (8, 148):
@@ -668,10 +685,12 @@ def extras(hb, W, torch, np, new_comm, step, timed, stream, R, S, n, dtype, peak
     for name, path, sc, cc, op, fw in (("CE_sum8", hb.PATH_CE, 8, 8, 0, 0), ("SM_copy8_sum8", hb.PATH_SM, 8, 8, 0, 0),
                                        ("SM_copy32_sum8", hb.PATH_SM, 8, 32, 0, 0), ("SM_copy48_sum8", hb.PATH_SM, 8, 48, 0, 0),
                                        ("SM_copy148_sum148", hb.PATH_SM, 148, 148, 0, 0),
+                                       ("SM_copy48_sum8_direct_allgather", hb.PATH_SM, 8, 48, 0, 3),
                                        ("SM_forward_copy8_sum8", hb.PATH_SM, 8, 8, 0, 1),
                                        ("SM_one_kernel_8", hb.PATH_SM, 8, 8, 0, 2),
                                        ("onepass_8", hb.PATH_CE, 8, 8, 1, 0), ("CE_HOST_sum8", hb.PATH_CE_HOST, 8, 8, 0, 0)):
-        c2 = new_comm(path, sum_ctas=sc, copy_ctas=cc, onepass=op, forward=1 if fw == 1 else 0, fused=1 if fw == 2 else 0)
+        c2 = new_comm(path, sum_ctas=sc, copy_ctas=cc, onepass=op, forward=1 if fw == 1 else 0, fused=1 if fw == 2 else 0,
+                      ag_direct=1 if fw == 3 else 0)
         if path == hb.PATH_CE_HOST:
             c2.set_host_staging(host_stage)
         # the one-pass comparison kernel is one all-reduce call (reduce-scatter + all-gather would add the path's moves)

@@ -153,6 +153,12 @@ hoccl_result_t hoccl_comm_set_path(hoccl_comm_t comm, hoccl_path_t path);
  *                straight into the next rank's inbox, so only step 0 needs moves (3 instead of 5 bytes of traffic per
  *                wire byte in that phase).  Same bits.  A SUM then stores into another rank's memory, as SM-driven
  *                libraries do: it is the second comparison point for what rank locality costs.  0 = off (default).
+ *  "ag_direct"   1 = the all-gather (alone or as the second half of an all-reduce) runs as the stage decomposition of its
+ *                traffic matrix (paper Sec. 3.4): every rank sends its own final chunk to every other rank, R-1
+ *                contention-free permutation stages r -> r+k that depend only on the chunk being final, instead of R-1
+ *                ring hops that each wait for the previous one.  Rank local (a rank sends what it owns), same bytes
+ *                moved, same bits; the moves of all stages can be in flight together (SM path: one batched launch).
+ *                0 = the ring all-gather (default).
  *  "fused"       1 = on HOCCL_PATH_SM the whole collective runs as ONE cooperative kernel that walks the ring steps with a
  *                grid-wide barrier between dependent steps (how an SM-driven library runs a collective: the paper's
  *                "NCCL under an SM budget" baseline, Sec. 5).  The schedule stays rank local and the bits are the same.
@@ -390,11 +396,16 @@ hoccl_result_t hoccl_probe_copy_routes(hoccl_comm_t comm, void* dst, const void*
  * Direct launches of the two kernels (used by kernel-level tests and roofline measurements).
  *  hoccl_sum_launch : out[i] = round_to_dtype(float(inbox[i]) + float(local[i])), i < count, with `ctas` CTAs.
  *  hoccl_copy_launch: dst bytes <- src bytes with `ctas` CTAs.
- * All pointers are device pointers aligned to the element size (any byte alignment for the copy).
+ *  hoccl_fanout_launch: dsts[d] bytes <- src bytes for every d < ndst with `ctas` CTAs; every source byte is read once
+ *                    and stored ndst times (the move of the direct all-gather on the SM path, see "ag_direct").  `dsts`
+ *                    is a HOST array of ndst (1..256) device pointers; destinations must not overlap the source or each
+ *                    other.  Destinations whose address differs from the source's modulo 16 are copied byte by byte.
+ * All pointers are device pointers aligned to the element size (any byte alignment for the copies).
  */
 hoccl_result_t hoccl_sum_launch(const void* inbox, const void* local, void* out, size_t count, hoccl_dtype_t dtype,
                                 int ctas, hoccl_stream_t stream);
 hoccl_result_t hoccl_copy_launch(const void* src, void* dst, size_t bytes, int ctas, hoccl_stream_t stream);
+hoccl_result_t hoccl_fanout_launch(const void* src, void* const* dsts, int ndst, size_t bytes, int ctas, hoccl_stream_t stream);
 /*
  * "SMs used", counted rather than inferred (the paper's Table 1 counts the SMs that communication kernels occupy):
  * launches the SUM kernel (kind 0: out = a + b over bytes / sizeof(dtype) elements) or the copy kernel (kind 1:
@@ -432,14 +443,16 @@ hoccl_result_t hoccl_kernel_sms(int kind, const void* a, const void* b, void* ou
  * relative to.
  */
 typedef enum { HOCCL_PLAN_ALLREDUCE = 0, HOCCL_PLAN_REDUCE_SCATTER = 1, HOCCL_PLAN_ALLGATHER = 2, HOCCL_PLAN_ALLTOALL = 3,
-               HOCCL_PLAN_ALLREDUCE_FWD = 4, HOCCL_PLAN_REDUCE_SCATTER_FWD = 5 /* the "forward" variants */ } hoccl_plan_kind_t;
+               HOCCL_PLAN_ALLREDUCE_FWD = 4, HOCCL_PLAN_REDUCE_SCATTER_FWD = 5, /* the "forward" variants */
+               HOCCL_PLAN_ALLREDUCE_AGD = 6, HOCCL_PLAN_ALLGATHER_DIRECT = 7,   /* the "ag_direct" variants */
+               HOCCL_PLAN_ALLREDUCE_FWD_AGD = 8 /* both */ } hoccl_plan_kind_t;
 typedef enum { HOCCL_OP_MOVE = 0, HOCCL_OP_SUM = 1 } hoccl_plan_op_kind_t;
 typedef enum { HOCCL_BUF_SEND = 0, HOCCL_BUF_RECV = 1, HOCCL_BUF_INBOX = 2, HOCCL_BUF_PARTIAL = 3 } hoccl_buf_kind_t;
 
 typedef struct {
   int kind;      /* hoccl_plan_op_kind_t */
   int phase;     /* 0 reduce-scatter, 1 all-gather, 2 own-chunk / own-block copy, 3 all-to-all stage */
-  int step;      /* ring step s (all-to-all: stage k, destination = rank + k) */
+  int step;      /* ring step s (all-to-all: stage k, destination = rank + k; direct all-gather: stage k - 1) */
   int piece;     /* pipeline piece index */
   int rank;      /* MOVE: source rank; SUM: the rank that sums */
   int dst_rank;  /* MOVE: destination rank; SUM: same as rank (forward variants: the rank whose slot receives the result) */

@@ -17,6 +17,7 @@ FLOAT32, BFLOAT16 = 0, 1
 SUM = 0
 PATH_CE, PATH_SM, PATH_CE_HOST = 0, 1, 2
 PLAN_ALLREDUCE, PLAN_REDUCE_SCATTER, PLAN_ALLGATHER, PLAN_ALLTOALL, PLAN_ALLREDUCE_FWD, PLAN_REDUCE_SCATTER_FWD = range(6)
+PLAN_ALLREDUCE_AGD, PLAN_ALLGATHER_DIRECT, PLAN_ALLREDUCE_FWD_AGD = 6, 7, 8
 OP_MOVE, OP_SUM = 0, 1
 BUF_SEND, BUF_RECV, BUF_INBOX, BUF_PARTIAL = 0, 1, 2, 3
 
@@ -27,7 +28,7 @@ EXPORTS = [
     "hoccl_comm_set_path", "hoccl_comm_set_param", "hoccl_comm_get_param", "hoccl_allreduce", "hoccl_reduce_scatter",
     "hoccl_allgather", "hoccl_alltoall", "hoccl_alltoallv", "hoccl_send", "hoccl_recv", "hoccl_comm_pending", "hoccl_comm_async_error", "hoccl_comm_handshakes", "hoccl_selftest_barrier_timeout", "hoccl_host_allreduce", "hoccl_error_string",
     "hoccl_last_cuda_error", "hoccl_last_stats", "hoccl_profile_reset", "hoccl_probe_move_needs_sm", "hoccl_probe_copy_routes", "hoccl_sum_launch", "hoccl_kernel_sms", "hoccl_flatten_inspect", "hoccl_port_probe",
-    "hoccl_copy_launch", "hoccl_plan_build", "hoccl_plan_destroy", "hoccl_plan_num_ops", "hoccl_plan_num_groups",
+    "hoccl_copy_launch", "hoccl_fanout_launch", "hoccl_plan_build", "hoccl_plan_destroy", "hoccl_plan_num_ops", "hoccl_plan_num_groups",
     "hoccl_plan_get_op", "hoccl_plan_group_deps", "hoccl_plan_slot_bytes", "hoccl_allreduce_static",
     "hoccl_sched_build", "hoccl_sched_destroy", "hoccl_sched_num_stages", "hoccl_sched_stage_tau", "hoccl_sched_total_tau",
     "hoccl_sched_lower_bound", "hoccl_sched_matrix", "hoccl_sched_num_flows", "hoccl_sched_get_flow", "hoccl_sched_queue_len",
@@ -132,6 +133,7 @@ def lib() -> ctypes.CDLL:
         "hoccl_probe_copy_routes": (i, [vp, vp, vp, sz, i, ctypes.POINTER(RouteProbe), i, ctypes.POINTER(i)]),
         "hoccl_sum_launch": (i, [vp, vp, vp, sz, i, i, vp]),
         "hoccl_copy_launch": (i, [vp, vp, sz, i, vp]),
+        "hoccl_fanout_launch": (i, [vp, vp, i, sz, i, vp]),
         "hoccl_kernel_sms": (i, [i, vp, vp, vp, sz, i, i, vp, vp]),
         "hoccl_selftest_barrier_timeout": (i, [vp, vp, vp, sz, vp]),
         "hoccl_port_probe": (i, [i, vp, sz, i, vp, vp]),
@@ -360,6 +362,11 @@ def sum_launch(inbox, local, out, count, dtype, ctas, stream=None) -> int:
 
 def copy_launch(src, dst, nbytes, ctas, stream=None) -> int:
     return lib().hoccl_copy_launch(_ptr(src), _ptr(dst), nbytes, ctas, _stream(stream))
+
+
+def fanout_launch(src, dsts, nbytes, ctas, stream=None) -> int:
+    """hoccl_fanout_launch: every dsts[d] <- src, the source read once.  Returns the result code."""
+    return lib().hoccl_fanout_launch(_ptr(src), _ptr_array(dsts), len(dsts), nbytes, ctas, _stream(stream))
 
 
 def kernel_sms(kind: str, a, b, out, nbytes: int, dtype, ctas: int, smid_out, stream=None) -> int:

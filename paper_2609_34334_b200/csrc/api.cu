@@ -125,6 +125,7 @@ static long* param_slot(hoccl_comm* c, const char* key, long* lo, long* hi) {
               {"ce_sub_bytes", &c->ce_sub_bytes, 0, 1L << 40}, {"handshake", &c->handshake, 0, 1},
               {"watchdog_ms", &c->watchdog_ms, 10, 600000},    {"onepass", &c->onepass, 0, 1},
               {"forward", &c->forward, 0, 1},           {"fused", &c->fused, 0, 1},
+              {"ag_direct", &c->ag_direct, 0, 1},
               {"host_pieces", &c->host_pieces, 1, 64}};
   for (auto& r : rows)
     if (std::strcmp(r.name, key) == 0) {
@@ -673,6 +674,43 @@ hoccl_result_t hoccl_copy_launch(const void* src, void* dst, size_t bytes, int c
   b.pad = 0;
   b.seg[0] = CopySeg{src, dst, (unsigned long long)bytes};
   return launch_copy(b, ctas, (cudaStream_t)stream) == cudaSuccess ? HOCCL_OK : HOCCL_ERR_CUDA;
+}
+
+hoccl_result_t hoccl_fanout_launch(const void* src, void* const* dsts, int ndst, size_t bytes, int ctas, hoccl_stream_t stream) {
+  if (!src || !dsts || ndst < 1 || ndst > kMaxFanDsts || ctas < 1 || ctas > 1024) return HOCCL_ERR_INVALID_ARG;
+  for (int d = 0; d < ndst; d++) {
+    if (!dsts[d] || ranges_overlap((const char*)src, bytes, (const char*)dsts[d], bytes)) return HOCCL_ERR_INVALID_ARG;
+    for (int k = 0; k < d; k++)
+      if (ranges_overlap((const char*)dsts[k], bytes, (const char*)dsts[d], bytes)) return HOCCL_ERR_INVALID_ARG;
+  }
+  if (bytes == 0) return HOCCL_OK;
+  // the same grouping as the collectives use: one segment per 16-byte phase of the destinations
+  RGroup g;
+  g.kind = OP_MOVE;
+  g.piece = 0;
+  g.chain_dep = -1;
+  for (int d = 0; d < ndst; d++) {
+    Seg s = {};
+    s.src = (const char*)src;
+    s.dst = (char*)dsts[d];
+    s.bytes = bytes;
+    g.segs.push_back(s);
+  }
+  std::vector<FanBatch> fans;
+  std::vector<double> hbm;
+  std::vector<long> moves;
+  if (!build_fan_batches(g, &fans, &hbm, &moves)) {   // no two destinations share a phase (or there is only one): plain copies
+    for (size_t first = 0; first < g.segs.size(); first += kMaxSegs) {
+      const size_t n = std::min<size_t>(kMaxSegs, g.segs.size() - first);
+      CopyBatch b;
+      fill_copy_batch(g, first, n, &b);
+      if (launch_copy(b, ctas, (cudaStream_t)stream) != cudaSuccess) return HOCCL_ERR_CUDA;
+    }
+    return HOCCL_OK;
+  }
+  for (const FanBatch& f : fans)
+    if (launch_fan(f, ctas, (cudaStream_t)stream) != cudaSuccess) return HOCCL_ERR_CUDA;
+  return HOCCL_OK;
 }
 
 // ---------------------------------------------------------------- plan inspection ----------------

@@ -39,6 +39,7 @@ struct Seg {
 
 struct RGroup {
   int kind;
+  int piece;
   std::vector<Seg> segs;
   std::vector<int> deps;
   int chain_dep;
@@ -83,7 +84,7 @@ struct hoccl_comm {
   int R = 0, device = 0, num_sms = 0;
   hoccl_path_t path = HOCCL_PATH_CE;
   long sum_ctas = 8, copy_ctas = 8, piece_bytes = 4 << 20, max_pieces = 8, lanes = 4, use_graph = 1, profile = 0, p2p_split = 1, ce_sub_bytes = 0,
-       handshake = 0, watchdog_ms = 10000, onepass = 0, forward = 0, fused = 0, host_pieces = 8;
+       handshake = 0, watchdog_ms = 10000, onepass = 0, forward = 0, fused = 0, host_pieces = 8, ag_direct = 0;
   bool piece_bytes_set = false;  // the caller chose a piece size: no automatic choice
   hoccl::Proxy* proxy = nullptr;
   cudaStream_t lane[hoccl::kMaxLanes] = {};
@@ -167,6 +168,10 @@ struct Tally {
 // exec.cu
 void fill_sum_batch(const RGroup& g, size_t first, size_t n, int dtype, size_t elem, SumBatch* b);
 void fill_copy_batch(const RGroup& g, size_t first, size_t n, CopyBatch* b);
+// Moves of a group that read the same bytes (same source and length; the direct all-gather on the SM path) become fan-out
+// segments: one read, one store per destination.  Returns false (and leaves *out empty) if no source repeats: the plain
+// copy batches are used then.  bytes_out[i] = HBM bytes of batch i (reads + writes), moves_out[i] = moves it carries.
+bool build_fan_batches(const RGroup& g, std::vector<FanBatch>* out, std::vector<double>* bytes_out, std::vector<long>* moves_out);
 // graph.cu
 hoccl_result_t build_graph(hoccl_comm* c, const Plan& P, const std::vector<RGroup>& groups, GraphEntry* entry, int only_piece,
                            cudaGraphExec_t* out_exec);

@@ -11,6 +11,8 @@
 //   * stream executor: internal move lanes plus one sum stream, ordered with CUDA events
 //     (fork from the caller's stream, join back into it).
 // SUM launches are chained (one at a time) so that the SM budget for sums is global, not per piece.
+#include <tuple>
+
 #include "comm.h"
 
 namespace hoccl {
@@ -71,6 +73,7 @@ void resolve(hoccl_comm* c, const Plan& P, const Call& call, std::vector<RGroup>
     const PlanGroup& pg = P.groups[g];
     RGroup& rg = (*out)[g];
     rg.kind = pg.kind;
+    rg.piece = pg.piece;
     rg.deps = pg.deps;
     rg.chain_dep = pg.chain_dep;
     for (int i = 0; i < pg.num_ops; i++) {
@@ -104,6 +107,32 @@ void resolve(hoccl_comm* c, const Plan& P, const Call& call, std::vector<RGroup>
       out->assign(1, all);
     }
   }
+  // SM path, direct all-gather: its stages (the trailing MOVE groups of a piece, nothing depends on them) wait for the same
+  // thing, so consecutive ones with equal dependencies become one group = one batched launch (or one phase of the ring kernel)
+  if (c->path == HOCCL_PATH_SM && P.ag_direct && P.kind != PLAN_ALLTOALL) {
+    std::vector<char> has_user(out->size(), 0);
+    for (const RGroup& g : *out) {
+      for (int d : g.deps) has_user[d] = 1;
+      if (g.chain_dep >= 0) has_user[g.chain_dep] = 1;
+    }
+    std::vector<RGroup> merged;
+    std::vector<int> remap(out->size(), -1);
+    for (size_t g = 0; g < out->size(); g++) {
+      RGroup& cur = (*out)[g];
+      for (int& d : cur.deps) d = remap[d];
+      if (cur.chain_dep >= 0) cur.chain_dep = remap[cur.chain_dep];
+      const bool tail_move = cur.kind == OP_MOVE && !has_user[g] && P.groups[g].phase != PHASE_RS;
+      if (tail_move && !merged.empty() && g > 0 && remap[g - 1] == (int)merged.size() - 1 && merged.back().kind == OP_MOVE &&
+          !has_user[g - 1] && P.groups[g - 1].phase != PHASE_RS && merged.back().piece == cur.piece && merged.back().deps == cur.deps) {
+        merged.back().segs.insert(merged.back().segs.end(), cur.segs.begin(), cur.segs.end());
+        remap[g] = (int)merged.size() - 1;
+      } else {
+        merged.push_back(cur);
+        remap[g] = (int)merged.size() - 1;
+      }
+    }
+    out->swap(merged);
+  }
 }
 
 void fill_sum_batch(const RGroup& g, size_t first, size_t n, int dtype, size_t elem, SumBatch* b) {
@@ -123,6 +152,63 @@ void fill_copy_batch(const RGroup& g, size_t first, size_t n, CopyBatch* b) {
   }
 }
 
+bool build_fan_batches(const RGroup& g, std::vector<FanBatch>* out, std::vector<double>* bytes_out, std::vector<long>* moves_out) {
+  out->clear();
+  bytes_out->clear();
+  moves_out->clear();
+  if (g.kind != OP_MOVE) return false;
+  // classes: same source, same length, same 16-byte phase of the destination (so that a class is all-vector or all-element-wise)
+  struct Class {
+    const char* src;
+    size_t bytes;
+    unsigned phase;
+    std::vector<void*> dsts;
+  };
+  std::vector<Class> classes;
+  std::map<std::tuple<const char*, size_t, unsigned>, size_t> index;
+  bool repeats = false;
+  for (const Seg& s : g.segs) {
+    auto key = std::make_tuple((const char*)s.src, (size_t)s.bytes, (unsigned)((uintptr_t)s.dst & 15));
+    auto it = index.find(key);
+    if (it == index.end()) {
+      index.emplace(key, classes.size());
+      classes.push_back(Class{s.src, s.bytes, std::get<2>(key), {s.dst}});
+    } else {
+      classes[it->second].dsts.push_back(s.dst);
+      repeats = true;
+    }
+  }
+  if (!repeats) return false;
+  FanBatch cur;
+  cur.nseg = 0;
+  cur.ndst_total = 0;
+  double cur_bytes = 0;
+  long cur_moves = 0;
+  auto flush = [&]() {
+    if (cur.nseg == 0) return;
+    out->push_back(cur);
+    bytes_out->push_back(cur_bytes);
+    moves_out->push_back(cur_moves);
+    cur.nseg = 0;
+    cur.ndst_total = 0;
+    cur_bytes = 0;
+    cur_moves = 0;
+  };
+  for (const Class& cl : classes) {
+    size_t done = 0;
+    while (done < cl.dsts.size()) {   // a class with more destinations than a batch holds is cut
+      if (cur.nseg == kMaxSegs || cur.ndst_total == kMaxFanDsts) flush();
+      const size_t n = std::min<size_t>(cl.dsts.size() - done, (size_t)(kMaxFanDsts - cur.ndst_total));
+      cur.seg[cur.nseg++] = FanSeg{cl.src, (unsigned long long)cl.bytes, cur.ndst_total, (int)n};
+      for (size_t i = 0; i < n; i++) cur.dst[cur.ndst_total++] = cl.dsts[done + i];
+      cur_bytes += (double)cl.bytes * (1.0 + (double)n);
+      cur_moves += (long)n;
+      done += n;
+    }
+  }
+  flush();
+  return true;
+}
 
 // ------------------------------------------------------------------ stream executor -------------
 hoccl_result_t run_streams(hoccl_comm* c, const Plan& P, const std::vector<RGroup>& groups, cudaStream_t user, Tally* tally) {
@@ -198,13 +284,24 @@ hoccl_result_t run_streams(hoccl_comm* c, const Plan& P, const std::vector<RGrou
         tally->moves++;
       }
     } else {
-      for (size_t first = 0; first < rg.segs.size(); first += kMaxSegs) {
-        size_t n = std::min<size_t>(kMaxSegs, rg.segs.size() - first);
-        CopyBatch b;
-        fill_copy_batch(rg, first, n, &b);
-        CU_TRY(c, launch_copy(b, (int)c->copy_ctas, s));
-        tally->moves += (long)n;
-        tally->move_launches++;
+      std::vector<FanBatch> fans;
+      std::vector<double> fan_bytes;
+      std::vector<long> fan_moves;
+      if (P.ag_direct && build_fan_batches(rg, &fans, &fan_bytes, &fan_moves)) {
+        for (size_t i = 0; i < fans.size(); i++) {
+          CU_TRY(c, launch_fan(fans[i], (int)c->copy_ctas, s));
+          tally->moves += fan_moves[i];
+          tally->move_launches++;
+        }
+      } else {
+        for (size_t first = 0; first < rg.segs.size(); first += kMaxSegs) {
+          size_t n = std::min<size_t>(kMaxSegs, rg.segs.size() - first);
+          CopyBatch b;
+          fill_copy_batch(rg, first, n, &b);
+          CU_TRY(c, launch_copy(b, (int)c->copy_ctas, s));
+          tally->moves += (long)n;
+          tally->move_launches++;
+        }
       }
     }
     cudaEvent_t ev = next_event(c);
@@ -244,6 +341,7 @@ std::vector<uint64_t> make_key(hoccl_comm* c, const Call& call) {
   k.push_back((uint64_t)c->profile);
   k.push_back((uint64_t)c->ce_sub_bytes);
   k.push_back((uint64_t)c->forward);
+  k.push_back((uint64_t)c->ag_direct);
   k.push_back((uint64_t)(c->fused && c->path == HOCCL_PATH_SM && !c->handshake));
   k.push_back((uint64_t)(uintptr_t)c->scratch);
   k.push_back((uint64_t)c->scratch_bytes);
@@ -442,6 +540,8 @@ hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
   int plan_kind = call->kind;
   if (c->forward && call->kind == PLAN_ALLREDUCE) plan_kind = PLAN_ALLREDUCE_FWD;
   if (c->forward && call->kind == PLAN_REDUCE_SCATTER) plan_kind = PLAN_REDUCE_SCATTER_FWD;
+  if (c->ag_direct && call->kind == PLAN_ALLREDUCE) plan_kind = c->forward ? PLAN_ALLREDUCE_FWD_AGD : PLAN_ALLREDUCE_AGD;
+  if (c->ag_direct && call->kind == PLAN_ALLGATHER) plan_kind = PLAN_ALLGATHER_DIRECT;
   // Piece size: the caller's, else 4 MiB; on the SM path under CTA budgets a reduction is cut into at least two pieces
   // (the copy kernel of one piece then overlaps the sum kernel of the other: measured 1.6x on a 3 MiB chunk with 8 + 8
   // CTAs), which does not pay with driver copies or whole-GPU grids.

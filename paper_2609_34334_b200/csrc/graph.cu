@@ -62,7 +62,7 @@ hoccl_result_t build_graph(hoccl_comm* c, const Plan& P, const std::vector<RGrou
     rc = cuda_fail(c, e, what);
   };
   for (size_t gi = 0; gi < groups.size() && rc == HOCCL_OK; gi++) {
-    if (only_piece >= 0 && P.groups[gi].piece != only_piece) continue;
+    if (only_piece >= 0 && groups[gi].piece != only_piece) continue;
     const RGroup& rg = groups[gi];
     std::vector<cudaGraphNode_t> deps;
     for (int d : rg.deps)
@@ -141,45 +141,62 @@ hoccl_result_t build_graph(hoccl_comm* c, const Plan& P, const std::vector<RGrou
         entry->n_moves++;
       }
     } else {
-      for (size_t first = 0; first < rg.segs.size() && e == cudaSuccess; first += kMaxSegs) {
-        size_t n = std::min<size_t>(kMaxSegs, rg.segs.size() - first);
-        CopyBatch b;
-        fill_copy_batch(rg, first, n, &b);
-        prepare_copy_batch(&b, (int)c->copy_ctas);
-        void* args[] = {&b};
+      // one kernel node per batch; `batch` is copied into the node when it is added
+      auto add_move_node = [&](void* batch, const void* func, int threads, double hbm_bytes, long n_moves) -> cudaError_t {
+        void* args[] = {batch};
         cudaKernelNodeParams kp = {};
-        int copy_threads = 0;
-        kp.func = const_cast<void*>(copy_kernel_entry((int)c->copy_ctas, &copy_threads));
+        kp.func = const_cast<void*>(func);
         kp.gridDim = dim3((unsigned)c->copy_ctas);
-        kp.blockDim = dim3((unsigned)copy_threads);
+        kp.blockDim = dim3((unsigned)threads);
         kp.kernelParams = args;
         // copy launches are chained as well: the CTA budget for copies is global, two never run at the same time
         std::vector<cudaGraphNode_t> d2 = deps;
         if (last_copy_node && std::find(d2.begin(), d2.end(), last_copy_node) == d2.end()) d2.push_back(last_copy_node);
         std::pair<cudaEvent_t, cudaEvent_t> pe{nullptr, nullptr};
+        cudaError_t err;
         if (c->profile) {
-          if ((e = cudaEventCreate(&pe.first)) != cudaSuccess) break;
-          if ((e = cudaEventCreate(&pe.second)) != cudaSuccess) break;
+          if ((err = cudaEventCreate(&pe.first)) != cudaSuccess) return err;
+          if ((err = cudaEventCreate(&pe.second)) != cudaSuccess) return err;
           entry->prof_events.push_back(pe);
-          double bytes = 0;
-          for (size_t i = 0; i < n; i++) bytes += 2.0 * (double)rg.segs[first + i].bytes;
-          entry->prof_bytes.push_back(-bytes);   // negative: a copy launch (read + write), kept apart from the sums
+          entry->prof_bytes.push_back(-hbm_bytes);   // negative: a copy launch (reads + writes), kept apart from the sums
           cudaGraphNode_t start_rec;
-          if ((e = cudaGraphAddEventRecordNode(&start_rec, g, d2.data(), d2.size(), pe.first)) != cudaSuccess) break;
+          if ((err = cudaGraphAddEventRecordNode(&start_rec, g, d2.data(), d2.size(), pe.first)) != cudaSuccess) return err;
           d2.assign(1, start_rec);
         }
         cudaGraphNode_t kn;
-        e = cudaGraphAddKernelNode(&kn, g, d2.data(), d2.size(), &kp);
-        if (e != cudaSuccess) break;
+        if ((err = cudaGraphAddKernelNode(&kn, g, d2.data(), d2.size(), &kp)) != cudaSuccess) return err;
         if (c->profile) {
           cudaGraphNode_t end_rec;
-          if ((e = cudaGraphAddEventRecordNode(&end_rec, g, &kn, 1, pe.second)) != cudaSuccess) break;
+          if ((err = cudaGraphAddEventRecordNode(&end_rec, g, &kn, 1, pe.second)) != cudaSuccess) return err;
           kn = end_rec;
         }
         last_copy_node = kn;
         nodes.push_back(kn);
-        entry->n_moves += (long)n;
+        entry->n_moves += n_moves;
         entry->n_move_launches++;
+        return cudaSuccess;
+      };
+      std::vector<FanBatch> fans;
+      std::vector<double> fan_bytes;
+      std::vector<long> fan_moves;
+      int move_threads = 0;
+      if (P.ag_direct && build_fan_batches(rg, &fans, &fan_bytes, &fan_moves)) {
+        const void* fn = fan_kernel_entry((int)c->copy_ctas, &move_threads);
+        for (size_t i = 0; i < fans.size() && e == cudaSuccess; i++) {
+          prepare_fan_batch(&fans[i], (int)c->copy_ctas);
+          e = add_move_node(&fans[i], fn, move_threads, fan_bytes[i], fan_moves[i]);
+        }
+      } else {
+        const void* fn = copy_kernel_entry((int)c->copy_ctas, &move_threads);
+        for (size_t first = 0; first < rg.segs.size() && e == cudaSuccess; first += kMaxSegs) {
+          size_t n = std::min<size_t>(kMaxSegs, rg.segs.size() - first);
+          CopyBatch b;
+          fill_copy_batch(rg, first, n, &b);
+          prepare_copy_batch(&b, (int)c->copy_ctas);
+          double bytes = 0;
+          for (size_t i = 0; i < n; i++) bytes += 2.0 * (double)rg.segs[first + i].bytes;
+          e = add_move_node(&b, fn, move_threads, bytes, (long)n);
+        }
       }
     }
     if (e != cudaSuccess) {

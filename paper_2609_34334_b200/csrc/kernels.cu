@@ -146,6 +146,70 @@ __global__ void __launch_bounds__(THREADS, 1) copy_kernel(const __grid_constant_
   }
 }
 
+// Fan-out copy: the tile walk of copy_kernel, but a tile that was loaded once is stored to every destination of its segment.
+template <int U, int THREADS>
+__global__ void __launch_bounds__(THREADS, 1) fan_kernel(const __grid_constant__ FanBatch batch) {
+  const Flat& f = batch.flat;
+  const int nseg = batch.nseg;
+  if (batch.smid_out != nullptr && threadIdx.x == 0) {
+    unsigned id;
+    asm volatile("mov.u32 %0, %%smid;" : "=r"(id));
+    batch.smid_out[blockIdx.x] = id;
+  }
+  const unsigned long long total = (unsigned long long)gridDim.x * blockDim.x;
+  const unsigned long long gt = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
+  {
+    const unsigned long long T_all = f.tpre[nseg];
+    const unsigned tile_v = U * blockDim.x;
+    int k = 0;
+    for (unsigned long long t = blockIdx.x; t < T_all; t += gridDim.x) {
+      while (t >= f.tpre[k + 1]) k++;
+      const unsigned long long first = (t - f.tpre[k]) * tile_v;
+      const unsigned long long left = f.nvec[k] - first;
+      const unsigned n_here = left < tile_v ? (unsigned)left : tile_v;
+      const uint4* a = reinterpret_cast<const uint4*>(static_cast<const char*>(batch.seg[k].src) + f.head[k]) + first;
+      void* const* dsts = batch.dst + batch.seg[k].first_dst;
+      const int nd = batch.seg[k].ndst;
+      uint4 va[U];
+      if (n_here == tile_v) {
+#pragma unroll
+        for (int u = 0; u < U; u++) va[u] = __ldcs(a + threadIdx.x + u * blockDim.x);
+        for (int d = 0; d < nd; d++) {
+          uint4* o = reinterpret_cast<uint4*>(static_cast<char*>(dsts[d]) + f.head[k]) + first;
+#pragma unroll
+          for (int u = 0; u < U; u++) o[threadIdx.x + u * blockDim.x] = va[u];
+        }
+      } else {
+#pragma unroll
+        for (int u = 0; u < U; u++) {
+          const unsigned i = threadIdx.x + u * blockDim.x;
+          if (i < n_here) va[u] = __ldcs(a + i);
+        }
+        for (int d = 0; d < nd; d++) {
+          uint4* o = reinterpret_cast<uint4*>(static_cast<char*>(dsts[d]) + f.head[k]) + first;
+#pragma unroll
+          for (int u = 0; u < U; u++) {
+            const unsigned i = threadIdx.x + u * blockDim.x;
+            if (i < n_here) o[i] = va[u];
+          }
+        }
+      }
+    }
+  }
+  {
+    const unsigned long long S = f.spre[nseg];
+    int k = 0;
+    for (unsigned long long j = gt; j < S; j += total) {
+      while (j >= f.spre[k + 1]) k++;
+      unsigned long long i = j - f.spre[k];
+      if (i >= f.head[k]) i += f.nvec[k] * 16;
+      const unsigned char v = static_cast<const unsigned char*>(batch.seg[k].src)[i];
+      void* const* dsts = batch.dst + batch.seg[k].first_dst;
+      for (int d = 0; d < batch.seg[k].ndst; d++) static_cast<unsigned char*>(dsts[d])[i] = v;
+    }
+  }
+}
+
 // ---- one-pass ring reduction (comparison point) -------------------------------------------------------------------
 template <int DT, int THREADS>
 __global__ void __launch_bounds__(THREADS, 1) onepass_kernel(const __grid_constant__ OnePassArgs a) {
@@ -331,6 +395,29 @@ void prepare_copy_batch(CopyBatch* b, int ctas) {
   fill_flat(&b->flat, b->nseg, tile_v, head, nvec, nscalar);
 }
 
+void prepare_fan_batch(FanBatch* b, int ctas) {
+  const unsigned long long tile_v = wide_copy_grid(ctas) ? 4ull * 512 : 8ull * 1024;
+  unsigned head[kMaxSegs];
+  unsigned long long nvec[kMaxSegs], nscalar[kMaxSegs];
+  for (int k = 0; k < b->nseg; k++) {
+    const FanSeg& s = b->seg[k];
+    const unsigned ms = (unsigned)((uintptr_t)s.src & 15);
+    bool same = true;
+    for (int d = 0; d < s.ndst; d++) same = same && ((unsigned)((uintptr_t)b->dst[s.first_dst + d] & 15) == ms);
+    split_segment(s.bytes, ms, same, 1, 16, &head[k], &nvec[k], &nscalar[k]);
+  }
+  fill_flat(&b->flat, b->nseg, tile_v, head, nvec, nscalar);
+}
+
+cudaError_t launch_fan(const FanBatch& batch, int ctas, cudaStream_t stream) {
+  if (batch.nseg <= 0) return cudaSuccess;
+  FanBatch b = batch;
+  prepare_fan_batch(&b, ctas);
+  if (wide_copy_grid(ctas)) fan_kernel<4, 512><<<ctas, 512, 0, stream>>>(b);
+  else fan_kernel<8, 1024><<<ctas, 1024, 0, stream>>>(b);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_sum(const SumBatch& batch, int ctas, cudaStream_t stream) {
   if (batch.nseg <= 0) return cudaSuccess;
   SumBatch b = batch;
@@ -383,6 +470,10 @@ const void* copy_kernel_entry(int ctas, int* threads) {
   *threads = wide_copy_grid(ctas) ? 512 : 1024;
   return wide_copy_grid(ctas) ? reinterpret_cast<const void*>(&copy_kernel<4, 512>) : reinterpret_cast<const void*>(&copy_kernel<8, 1024>);
 }
+const void* fan_kernel_entry(int ctas, int* threads) {
+  *threads = wide_copy_grid(ctas) ? 512 : 1024;
+  return wide_copy_grid(ctas) ? reinterpret_cast<const void*>(&fan_kernel<4, 512>) : reinterpret_cast<const void*>(&fan_kernel<8, 1024>);
+}
 
 // Forces the module that holds these kernels to be loaded now.  Loading a kernel on first launch can synchronise the
 // device; that must never happen while a stream is parked in a hand-over that only the launching thread can finish.
@@ -392,7 +483,8 @@ cudaError_t preload_kernels() {
                        reinterpret_cast<const void*>(&copy_kernel<4, 512>),     reinterpret_cast<const void*>(&copy_kernel<8, 1024>),
                        reinterpret_cast<const void*>(&occupy_kernel),           reinterpret_cast<const void*>(&onepass_kernel<0, 512>),
                        reinterpret_cast<const void*>(&onepass_kernel<1, 512>),  reinterpret_cast<const void*>(&onepass_kernel<0, 1024>),
-                       reinterpret_cast<const void*>(&onepass_kernel<1, 1024>)};
+                       reinterpret_cast<const void*>(&onepass_kernel<1, 1024>), reinterpret_cast<const void*>(&fan_kernel<4, 512>),
+                       reinterpret_cast<const void*>(&fan_kernel<8, 1024>)};
   for (const void* f : fns) {
     cudaFuncAttributes a;
     cudaError_t e = cudaFuncGetAttributes(&a, f);

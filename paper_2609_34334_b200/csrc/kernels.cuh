@@ -49,6 +49,24 @@ struct CopyBatch {
   unsigned int* smid_out = nullptr;  // diagnostics, as in SumBatch
 };
 
+// One fan-out segment: every dst[first_dst + d][0..bytes), d < ndst, <- src[0..bytes).  The source is read once and stored ndst
+// times (the direct all-gather on the SM path: a rank's chunk goes to all its peers, 1 + ndst instead of 2 ndst bytes of
+// traffic per chunk byte).  All addresses of a segment share their 16-byte phase or the segment runs element-wise.
+constexpr int kMaxFanDsts = 256;
+struct FanSeg {
+  const void* src;
+  unsigned long long bytes;
+  int first_dst, ndst;
+};
+struct FanBatch {
+  int nseg;
+  int ndst_total;
+  FanSeg seg[kMaxSegs];
+  void* dst[kMaxFanDsts];
+  Flat flat;  // filled by prepare_fan_batch (launch_fan does it itself)
+  unsigned int* smid_out = nullptr;  // diagnostics, as in SumBatch
+};
+
 // One-pass variant of the ring reduction (comparison point, not rank local): every element is reduced in registers in
 // the ring's order, chunk c as ((x_{c+1} + x_{c+2}) + ... ) + x_c with a rounding to the I/O dtype after every add, and
 // written to its destinations directly.  Same bits as the ring, R reads + R (or 1) writes per element instead of 7(R-1).
@@ -113,6 +131,9 @@ void prepare_ring_phase(RingSeg* seg, int nseg, int kind, int dtype, int threads
 // Enqueue helpers (return the CUDA error of the launch).
 cudaError_t launch_sum(const SumBatch& batch, int ctas, cudaStream_t stream);
 cudaError_t launch_copy(const CopyBatch& batch, int ctas, cudaStream_t stream);
+cudaError_t launch_fan(const FanBatch& batch, int ctas, cudaStream_t stream);
+void prepare_fan_batch(FanBatch* batch, int ctas);
+const void* fan_kernel_entry(int ctas, int* threads);
 // Fill batch->flat for the kernel variant that `ctas` CTAs select (needed before a batch is handed to a graph kernel node).
 void prepare_sum_batch(SumBatch* batch, int ctas);
 void prepare_copy_batch(CopyBatch* batch, int ctas);

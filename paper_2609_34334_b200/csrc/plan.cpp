@@ -83,8 +83,11 @@ void piece_span(const Plan& P, size_t len_bytes, int p, size_t* off, size_t* len
 bool build_plan(Plan* plan, int kind, int R, size_t count, int dtype, bool in_place, size_t piece_bytes, int max_pieces,
                 const unsigned char* send_align) {
   size_t e = dtype_size(dtype);
-  if (!plan || R < 1 || e == 0 || kind < PLAN_ALLREDUCE || kind > PLAN_REDUCE_SCATTER_FWD) return false;
-  const bool forward = (kind == PLAN_ALLREDUCE_FWD || kind == PLAN_REDUCE_SCATTER_FWD);
+  if (!plan || R < 1 || e == 0 || kind < PLAN_ALLREDUCE || kind > PLAN_ALLREDUCE_FWD_AGD) return false;
+  const bool forward = (kind == PLAN_ALLREDUCE_FWD || kind == PLAN_REDUCE_SCATTER_FWD || kind == PLAN_ALLREDUCE_FWD_AGD);
+  const bool ag_direct = (kind == PLAN_ALLREDUCE_AGD || kind == PLAN_ALLGATHER_DIRECT || kind == PLAN_ALLREDUCE_FWD_AGD);
+  if (kind == PLAN_ALLREDUCE_AGD || kind == PLAN_ALLREDUCE_FWD_AGD) kind = PLAN_ALLREDUCE;
+  if (kind == PLAN_ALLGATHER_DIRECT) kind = PLAN_ALLGATHER;
   if (kind == PLAN_ALLREDUCE_FWD) kind = PLAN_ALLREDUCE;
   if (kind == PLAN_REDUCE_SCATTER_FWD) kind = PLAN_REDUCE_SCATTER;
   if (kind == PLAN_ALLTOALL && in_place) return false;  // an in-place exchange would need a staging copy of every block
@@ -94,6 +97,7 @@ bool build_plan(Plan* plan, int kind, int R, size_t count, int dtype, bool in_pl
   P = Plan();
   P.kind = kind;
   P.forward = forward;
+  P.ag_direct = ag_direct;
   P.R = R;
   P.dtype = dtype;
   P.count = count;
@@ -239,6 +243,25 @@ bool build_plan(Plan* plan, int kind, int R, size_t count, int dtype, bool in_pl
         }
         B.end_group();
       }
+    }
+    if (ag_direct) {
+      // ---- direct AG MOVE(k, r, p): rank r sends its own final chunk r to rank r+k, k = 1..R-1.  Stage k is the
+      // contention-free permutation r -> r+k; the stages do not depend on each other, only on the chunk being final.
+      for (int p = 0; p < np_i; p++)
+        for (int k = 1; k < R; k++) {
+          int g = B.begin_group(OP_MOVE, PHASE_AG, k - 1, p);
+          for (int r = 0; r < R; r++) {
+            size_t lo, hi, off, len;
+            P.chunk_range(r, &lo, &hi);
+            piece_span(P, (hi - lo) * e, p, &off, &len);
+            bool from_send = standalone && !in_place;
+            B.add(PlanOp{OP_MOVE, PHASE_AG, k - 1, p, r, (r + k) % R, r, from_send ? BUF_SEND : BUF_RECV, BUF_RECV, -1,
+                         from_send ? off : lo * e + off, lo * e + off, 0, len, 0});
+          }
+          g = B.end_group();
+          if (g >= 0 && !standalone && final_sum[p] >= 0) P.groups[g].deps.push_back(final_sum[p]);
+        }
+      return true;
     }
     std::vector<int> last_ag(np_i, -1);
     for (int s = 0; s <= R - 2; s++) {

@@ -17,7 +17,10 @@ namespace hoccl {
 
 enum PlanKind { PLAN_ALLREDUCE = 0, PLAN_REDUCE_SCATTER = 1, PLAN_ALLGATHER = 2, PLAN_ALLTOALL = 3,
                 // comparison variants: the SUM of step s writes straight into the next rank's inbox (no moves after step 0)
-                PLAN_ALLREDUCE_FWD = 4, PLAN_REDUCE_SCATTER_FWD = 5 };
+                PLAN_ALLREDUCE_FWD = 4, PLAN_REDUCE_SCATTER_FWD = 5,
+                // direct all-gather: the all-gather's traffic matrix (every rank sends its chunk to every other rank) cut into
+                // the R-1 permutation stages r -> r+k (the stage decomposition of Sec. 3.4) instead of R-1 dependent ring hops
+                PLAN_ALLREDUCE_AGD = 6, PLAN_ALLGATHER_DIRECT = 7, PLAN_ALLREDUCE_FWD_AGD = 8 /* both variants */ };
 enum OpKind { OP_MOVE = 0, OP_SUM = 1 };
 enum BufKind { BUF_SEND = 0, BUF_RECV = 1, BUF_INBOX = 2, BUF_PARTIAL = 3 };
 enum Phase { PHASE_RS = 0, PHASE_AG = 1, PHASE_OWN = 2, PHASE_A2A = 3 };
@@ -43,6 +46,7 @@ struct PlanGroup {
 struct Plan {
   int kind = 0, R = 0, dtype = 0;  // kind: the base collective (forward variants are folded into it, see `forward`)
   bool forward = false;            // fused sum-and-forward variant (not rank local)
+  bool ag_direct = false;          // all-gather phase as R-1 independent permutation stages (rank local: rank r sends its own chunk)
   size_t count = 0;
   bool in_place = false;
   size_t elem = 4;

@@ -4,6 +4,7 @@
     python -m paper_2609_34334_b200.microbench --kernel routes --mib 16      # which same-device copy routes need an SM
     python -m paper_2609_34334_b200.microbench --kernel ring --mib 32 --ctas 148   # all-reduce, R = 8, as one cooperative kernel
     python -m paper_2609_34334_b200.microbench --kernel port --mib 256 --ctas 8    # what the memory ports of `ctas` SMs carry
+    python -m paper_2609_34334_b200.microbench --kernel fan --mib 25 --ctas 148    # one source to 7 destinations: fan-out against 7 copies
 
 Operands are larger than L2 by default; timing uses CUDA events on the launching stream after warm-up.
 Prints one JSON line.  This is the small case used for ncu captures of a single kernel.
@@ -20,7 +21,7 @@ from . import binding as hb
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--kernel", default="sum", choices=["sum", "copy", "routes", "ring", "port"])
+    ap.add_argument("--kernel", default="sum", choices=["sum", "copy", "routes", "ring", "port", "fan"])
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "fp32"])
     ap.add_argument("--mib", type=int, default=200, help="MiB per operand")
     ap.add_argument("--ctas", type=int, default=8)
@@ -54,6 +55,36 @@ def main():
             st.synchronize()
             sec = e0.elapsed_time(e1) / 1e3 / args.reps
             out[name] = {"GBps": moved / sec / 1e9, "GBps_per_sm": moved / sec / 1e9 / args.ctas, "us": sec * 1e6}
+        print(json.dumps(out))
+        return
+    if args.kernel == "fan":
+        # the move of the direct all-gather: one chunk to R - 1 = 7 peers, as one fan-out launch and as 7 copy launches
+        nd, sets = 7, 3
+        srcs = [torch.randint(0, 255, (nbytes,), dtype=torch.uint8, device="cuda") for _ in range(sets)]
+        dsts = [[torch.empty(nbytes, dtype=torch.uint8, device="cuda") for _ in range(nd)] for _ in range(sets)]
+        st = torch.cuda.Stream()
+
+        def fan(k):
+            assert hb.fanout_launch(srcs[k], dsts[k], nbytes, args.ctas, st) == hb.OK
+
+        def copies(k):
+            for d in dsts[k]:
+                assert hb.copy_launch(srcs[k], d, nbytes, args.ctas, st) == hb.OK
+
+        out = {"kernel": "fan", "mib_per_operand": args.mib, "destinations": nd, "ctas": args.ctas}
+        for name, fn, moved in (("fan_out", fan, (1 + nd) * nbytes), ("separate_copies", copies, 2 * nd * nbytes)):
+            for k in range(max(args.warmup, sets)):
+                fn(k % sets)
+            st.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(st)
+            for k in range(args.reps):
+                fn(k % sets)
+            e1.record(st)
+            st.synchronize()
+            sec = e0.elapsed_time(e1) / 1e3 / args.reps
+            out[name] = {"us": sec * 1e6, "algorithmic_bytes": moved, "GBps": moved / sec / 1e9, "delivered_GBps": nd * nbytes / sec / 1e9}
+            assert all(torch.equal(d, srcs[0]) for d in dsts[0])
         print(json.dumps(out))
         return
     if args.kernel == "ring":

@@ -40,7 +40,8 @@ def _topo_order(num_groups, deps, rng):
 def _run_plan(plan, kind, R, count, dtype, xs, in_place, rng):
     e = W.elem_size(dtype)
     npdt = np.float32 if dtype == "fp32" else np.uint16
-    base = {hb.PLAN_ALLREDUCE_FWD: hb.PLAN_ALLREDUCE, hb.PLAN_REDUCE_SCATTER_FWD: hb.PLAN_REDUCE_SCATTER}.get(kind, kind)
+    base = {hb.PLAN_ALLREDUCE_FWD: hb.PLAN_ALLREDUCE, hb.PLAN_REDUCE_SCATTER_FWD: hb.PLAN_REDUCE_SCATTER, hb.PLAN_ALLREDUCE_AGD: hb.PLAN_ALLREDUCE,
+            hb.PLAN_ALLREDUCE_FWD_AGD: hb.PLAN_ALLREDUCE, hb.PLAN_ALLGATHER_DIRECT: hb.PLAN_ALLGATHER}.get(kind, kind)
     kind = base
     if kind == hb.PLAN_ALLREDUCE:
         send_n, recv_n = count, count
@@ -262,3 +263,66 @@ def test_forward_variant_plans_execute_to_oracle_bits(oracle, R, n, piece_bytes,
         got = _run_plan(plan, hb.PLAN_REDUCE_SCATTER_FWD, R, n // R, "fp32", xs, False, rng)
         for r in range(R):
             assert (got[r].view(np.uint32) == wrs[r].view(np.uint32)).all()
+
+
+@pytest.mark.parametrize("R,n,piece_bytes,max_pieces", [c for c in CASES if c[0] > 1 and c[1] > 0])
+def test_direct_allgather_plans(oracle, R, n, piece_bytes, max_pieces):
+    """The all-gather as the R-1 permutation stages r -> r+k of its traffic matrix: every rank sends only its own chunk, the
+    stages wait for nothing but the chunk being final, the bytes moved equal the ring's, and any legal order gives the bits."""
+    rng = random.Random(R * 4242 + n)
+    xs = W.rank_inputs("uniform", 29, R, n, "fp32")
+    want = oracle.ring_allreduce(xs)
+    for kind in (hb.PLAN_ALLREDUCE_AGD, hb.PLAN_ALLREDUCE_FWD_AGD):
+        for in_place in (False, True):
+            plan = hb.Plan(kind, R, n, "fp32", in_place, piece_bytes, max_pieces)
+            ring = hb.Plan(hb.PLAN_ALLREDUCE_FWD if kind == hb.PLAN_ALLREDUCE_FWD_AGD else hb.PLAN_ALLREDUCE, R, n, "fp32", in_place, piece_bytes, max_pieces)
+            ag = [op for op in plan.ops if op["phase"] == 1]
+            ring_ag = [op for op in ring.ops if op["phase"] == 1]
+            assert sum(op["bytes"] for op in ag) == sum(op["bytes"] for op in ring_ag)
+            # the reduce-scatter half is the ring's, op for op
+            strip = lambda ops: [{k: v for k, v in op.items() if k != "group"} for op in ops if op["phase"] != 1]
+            assert strip(plan.ops) == strip(ring.ops)
+            sum_groups = {op["group"] for op in plan.ops if op["kind"] == hb.OP_SUM and op["step"] == R - 2}
+            for op in ag:
+                assert op["kind"] == hb.OP_MOVE and op["chunk"] == op["rank"]                  # a rank sends what it owns
+                assert op["dst_rank"] == (op["rank"] + op["step"] + 1) % R != op["rank"]        # stage k = step + 1
+                assert op["src_buf"] == hb.BUF_RECV and op["dst_buf"] == hb.BUF_RECV and op["src_off"] == op["dst_off"]
+                deps = plan.deps[op["group"]]
+                assert len(deps) == 1 and deps[0] in sum_groups                               # no stage waits for another stage
+            # every (destination, chunk) pair is served exactly once per piece
+            seen = {}
+            for op in ag:
+                seen.setdefault((op["dst_rank"], op["chunk"]), []).append((op["dst_off"], op["bytes"]))
+            q = -(-n // R)
+            for d in range(R):
+                for c in range(R):
+                    size = (min((c + 1) * q, n) - min(c * q, n)) * 4
+                    if c == d or size == 0:
+                        assert (d, c) not in seen
+                        continue
+                    spans = sorted(seen[(d, c)])
+                    assert spans[0][0] == min(c * q, n) * 4 and sum(b for _, b in spans) == size
+                    assert all(a[0] + a[1] == b[0] for a, b in zip(spans, spans[1:]))
+            for trial in range(2):
+                got = _run_plan(plan, kind, R, n, "fp32", xs, in_place, rng)
+                for r in range(R):
+                    assert (got[r].view(np.uint32) == want[r].view(np.uint32)).all(), (kind, R, n, in_place, r)
+
+
+@pytest.mark.parametrize("R", [2, 3, 8])
+@pytest.mark.parametrize("count", [1, 7, 3001])
+def test_direct_standalone_allgather_plan(oracle, R, count):
+    rng = random.Random(R * 31 + count)
+    xs = W.rank_inputs("uniform", 37, R, count, "fp32")
+    want = oracle.allgather(xs)
+    for in_place in (False, True):
+        plan = hb.Plan(hb.PLAN_ALLGATHER_DIRECT, R, count, "fp32", in_place, 1024, 8)
+        assert all(not d for d in plan.deps)                     # nothing waits for anything
+        assert plan.slot_bytes == 0
+        for op in plan.ops:
+            assert op["kind"] == hb.OP_MOVE and op["chunk"] == op["rank"]
+            assert op["src_buf"] == (hb.BUF_RECV if in_place else hb.BUF_SEND)
+        for trial in range(2):
+            got = _run_plan(plan, hb.PLAN_ALLGATHER_DIRECT, R, count, "fp32", xs, in_place, rng)
+            for r in range(R):
+                assert (got[r].view(np.uint32) == want[r].view(np.uint32)).all()
