@@ -105,7 +105,10 @@ def sweep_sizes(args):
     ops = ["allreduce", "reduce_scatter", "allgather", "alltoall", "sendrecv"] if args.ops == "all" else args.ops.split(",")
     # name, path, SUM CTAs, copy CTAs, whole collective as one cooperative kernel
     configs = [("CE", hb.PATH_CE, 8, 8, 0), ("SM8", hb.PATH_SM, 8, 8, 0), ("SMall", hb.PATH_SM, 148, 148, 0),
-               ("SM8fused", hb.PATH_SM, 8, 8, 1), ("SMallfused", hb.PATH_SM, 148, 148, 1)]
+               ("SM8fused", hb.PATH_SM, 8, 8, 1), ("SMallfused", hb.PATH_SM, 148, 148, 1),
+               # all-gather as independent stages (fan-out copy on the SM path); the last one adds the forward comparison variant
+               ("CEdirect", hb.PATH_CE, 8, 8, 0), ("SM8direct", hb.PATH_SM, 8, 8, 0), ("SMalldirect", hb.PATH_SM, 148, 148, 0),
+               ("SMallfwddirect", hb.PATH_SM, 148, 148, 0)]
     if args.configs != "all":
         configs = [c for c in configs if c[0] in args.configs.split(",")]
     else:
@@ -137,11 +140,15 @@ def sweep_sizes(args):
                         comm.set_param("sum_ctas", sc)
                         comm.set_param("copy_ctas", cc)
                         comm.set_param("fused", fused)
+                        direct = name.endswith("direct")
+                        comm.set_param("ag_direct", 1 if direct else 0)
+                        comm.set_param("forward", 1 if "fwd" in name else 0)
                         t = time_op(comm, arena, stream)
                         row = {"op": op, "R": R, "dtype": dtype, "S": S, "config": name, "sum_ctas": sc,
                                "copy_ctas": cc if path == hb.PATH_SM else None, "us": t * 1e6, "algbw_GBps": S / t / 1e9,
                                "busbw_GBps": S * _bus_factor(op, R) / t / 1e9,
-                               "hbm_frac_of_8TBps": _hbm_bytes(op, S, R) / t / NOMINAL_HBM, "buffer_sets": nsets}
+                               # the ring's byte count; not given where the variant moves fewer bytes than the ring
+                               "hbm_frac_of_8TBps": None if direct else _hbm_bytes(op, S, R) / t / NOMINAL_HBM, "buffer_sets": nsets}
                         line = json.dumps(row)
                         print(line, flush=True)
                         if out:
