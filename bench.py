@@ -575,6 +575,12 @@ def extras(hb, W, torch, np, new_comm, step, timed, stream, R, S, n, dtype, peak
     t, _ = timed(c1, 6, 3)
     out["host_bounce_path"] = {"ms_per_step": t * 1e3, "busbw_GBps": S * bus_factor(R) / t / 1e9,
                                "pcie_bytes_per_step_each_way": 2.0 * S * (R - 1)}
+    # the same with the direct all-gather: a final chunk goes out to the host once and comes back R-1 times
+    c1.set_param("ag_direct", 1)
+    t, _ = timed(c1, 6, 3)
+    out["host_bounce_path_direct_allgather"] = {"ms_per_step": t * 1e3, "busbw_GBps": S * bus_factor(R) / t / 1e9,
+                                                "pcie_bytes_per_step_outbound": 1.0 * S * (R - 1) + 1.0 * S,
+                                                "pcie_bytes_per_step_inbound": 2.0 * S * (R - 1)}
     c1.destroy()
     # handshake mode (CPU proxy + stream memory operations) on the SM path, against the same path launched directly
     hs = {}

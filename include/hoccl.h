@@ -157,7 +157,9 @@ hoccl_result_t hoccl_comm_set_path(hoccl_comm_t comm, hoccl_path_t path);
  *                traffic matrix (paper Sec. 3.4): every rank sends its own final chunk to every other rank, R-1
  *                contention-free permutation stages r -> r+k that depend only on the chunk being final, instead of R-1
  *                ring hops that each wait for the previous one.  Rank local (a rank sends what it owns), same bytes
- *                moved, same bits; the moves of all stages can be in flight together (SM path: one batched launch).
+ *                moved, same bits; the moves of all stages can be in flight together.  HOCCL_PATH_SM: one batched launch
+ *                in which every chunk is read once and stored R-1 times (S R instead of 2 S (R-1) bytes of traffic);
+ *                HOCCL_PATH_CE_HOST: a chunk goes out to the host staging once and comes back R-1 times.
  *                0 = the ring all-gather (default).
  *  "fused"       1 = on HOCCL_PATH_SM the whole collective runs as ONE cooperative kernel that walks the ring steps with a
  *                grid-wide barrier between dependent steps (how an SM-driven library runs a collective: the paper's

@@ -35,6 +35,7 @@ struct Seg {
   char* dst;
   uint64_t bytes;
   uint64_t host_off = 0;  // HOCCL_PATH_CE_HOST: where this move bounces in the pinned host staging
+  bool host_first = true; // HOCCL_PATH_CE_HOST: this move issues the outbound copy into host_off (false: another move of the group did)
 };
 
 struct RGroup {

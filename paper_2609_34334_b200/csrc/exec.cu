@@ -52,6 +52,29 @@ hoccl_result_t validate(hoccl_comm* c, Call* call) {
   return HOCCL_OK;
 }
 
+// Host-bounce path: moves of one group with the same source and length get the same place in the host staging; the first
+// of them (host_first = true) carries the outbound copy, the others only their inbound copy behind it.  Recomputes *host_need.
+static void share_host_legs(std::vector<RGroup>* groups, size_t* host_need) {
+  *host_need = 0;
+  for (RGroup& g : *groups) {
+    if (g.kind != OP_MOVE) continue;
+    std::map<std::pair<const char*, uint64_t>, size_t> first_of;   // (source, bytes) -> index of the seg that owns the staging
+    for (size_t i = 0; i < g.segs.size(); i++) {
+      Seg& s = g.segs[i];
+      auto it = first_of.find({s.src, s.bytes});
+      if (it == first_of.end()) {
+        first_of.emplace(std::make_pair(s.src, s.bytes), i);
+        s.host_off = *host_need;
+        s.host_first = true;
+        *host_need += (s.bytes + 255) / 256 * 256;
+      } else {
+        s.host_off = g.segs[it->second].host_off;
+        s.host_first = false;
+      }
+    }
+  }
+}
+
 // Turns plan offsets into addresses (the plan already places pieces inside the scratch slots).
 void resolve(hoccl_comm* c, const Plan& P, const Call& call, std::vector<RGroup>* out, size_t* host_need) {
   *host_need = 0;
@@ -108,8 +131,10 @@ void resolve(hoccl_comm* c, const Plan& P, const Call& call, std::vector<RGroup>
     }
   }
   // SM path, direct all-gather: its stages (the trailing MOVE groups of a piece, nothing depends on them) wait for the same
-  // thing, so consecutive ones with equal dependencies become one group = one batched launch (or one phase of the ring kernel)
-  if (c->path == HOCCL_PATH_SM && P.ag_direct && P.kind != PLAN_ALLTOALL) {
+  // thing, so consecutive ones with equal dependencies become one group = one batched launch (or one phase of the ring kernel).
+  // Host-bounce path: the same merge lets the moves of a group that read the same bytes share ONE outbound copy into the
+  // host staging (see share_host_legs): a chunk crosses PCIe once outbound and R-1 times inbound instead of R-1 times each way.
+  if ((c->path == HOCCL_PATH_SM || c->path == HOCCL_PATH_CE_HOST) && P.ag_direct && P.kind != PLAN_ALLTOALL) {
     std::vector<char> has_user(out->size(), 0);
     for (const RGroup& g : *out) {
       for (int d : g.deps) has_user[d] = 1;
@@ -132,6 +157,7 @@ void resolve(hoccl_comm* c, const Plan& P, const Call& call, std::vector<RGroup>
       }
     }
     out->swap(merged);
+    if (c->path == HOCCL_PATH_CE_HOST) share_host_legs(out, host_need);
   }
 }
 
@@ -279,7 +305,8 @@ hoccl_result_t run_streams(hoccl_comm* c, const Plan& P, const std::vector<RGrou
     } else if (c->path == HOCCL_PATH_CE_HOST) {
       // two copy-engine legs through pinned host memory: no SM takes part in the move
       for (const Seg& sg : rg.segs) {
-        CU_TRY(c, cudaMemcpyAsync(c->host_staging + sg.host_off, sg.src, sg.bytes, cudaMemcpyDeviceToHost, s));
+        // a seg that shares another seg's outbound copy comes after it in the same group, hence later on this stream
+        if (sg.host_first) CU_TRY(c, cudaMemcpyAsync(c->host_staging + sg.host_off, sg.src, sg.bytes, cudaMemcpyDeviceToHost, s));
         CU_TRY(c, cudaMemcpyAsync(sg.dst, c->host_staging + sg.host_off, sg.bytes, cudaMemcpyHostToDevice, s));
         tally->moves++;
       }

@@ -130,11 +130,17 @@ hoccl_result_t build_graph(hoccl_comm* c, const Plan& P, const std::vector<RGrou
         if (e != cudaSuccess) break;
       }
     } else if (c->path == HOCCL_PATH_CE_HOST) {
+      std::map<uint64_t, cudaGraphNode_t> outbound;   // staging offset -> the outbound copy that fills it
       for (const Seg& sg : rg.segs) {
         cudaGraphNode_t d2h, h2d;
-        e = cudaGraphAddMemcpyNode1D(&d2h, g, deps.data(), deps.size(), c->host_staging + sg.host_off, sg.src, sg.bytes,
-                                     cudaMemcpyDeviceToHost);
-        if (e != cudaSuccess) break;
+        if (sg.host_first) {
+          e = cudaGraphAddMemcpyNode1D(&d2h, g, deps.data(), deps.size(), c->host_staging + sg.host_off, sg.src, sg.bytes,
+                                       cudaMemcpyDeviceToHost);
+          if (e != cudaSuccess) break;
+          outbound[sg.host_off] = d2h;
+        } else {
+          d2h = outbound[sg.host_off];   // filled by an earlier move of this group (same source, same bytes)
+        }
         e = cudaGraphAddMemcpyNode1D(&h2d, g, &d2h, 1, sg.dst, c->host_staging + sg.host_off, sg.bytes, cudaMemcpyHostToDevice);
         if (e != cudaSuccess) break;
         nodes.push_back(h2d);

@@ -141,3 +141,20 @@ def test_fanout_kernel_moves_exact_bytes(ctas):
     assert hb.fanout_launch(big.ptr, [big.ptr + 1024, big.ptr + 1500], 1024, 8) == hb.ERR_INVALID_ARG
     assert hb.fanout_launch(big.ptr, [big.ptr + 512], 1024, 8) == hb.ERR_INVALID_ARG
     assert hb.fanout_launch(big.ptr, [big.ptr + 2048] * 257, 16, 8) == hb.ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("use_graph", [0, 1])
+def test_many_ranks_need_several_fan_out_launches(oracle, use_graph):
+    """R = 20 and 40: R (R-1) = 380 and 1560 destinations, more than one launch carries (256), so chunks and even the
+    destinations of one chunk are spread over several launches; odd send alignments put some destinations out of phase."""
+    dtype, e = "fp32", 4
+    for R, n in [(20, 20 * 300 + 7), (40, 40 * 64 + 1)]:
+        xs = W.rank_inputs("uniform", 95, R, n, dtype)
+        want = oracle.ring_allreduce(xs)
+        comm = make_comm(R, n, dtype, hb.PATH_SM, ag_direct=1, sum_ctas=16, copy_ctas=16, use_graph=use_graph)
+        got = run_allreduce(comm, xs, dtype, in_place=True, offs=[(r % 3) * e for r in range(R)])
+        for r in range(R):
+            assert same_bits(got[r], want[r], dtype), (R, r)
+        st = comm.last_stats()
+        assert st["n_moves"] == 2 * R * (R - 1)
+        comm.destroy()

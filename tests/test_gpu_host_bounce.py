@@ -28,7 +28,9 @@ def _comm(R, n, dtype, host_bytes):
 
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
 @pytest.mark.parametrize("use_graph", [0, 1])
-def test_collectives_over_host_bounce(oracle, dtype, use_graph):
+@pytest.mark.parametrize("ag_direct", [0, 1])
+def test_collectives_over_host_bounce(oracle, dtype, use_graph, ag_direct):
+    """ag_direct = 1: the all-gather's moves that read the same chunk share one outbound copy into the host staging."""
     torch.cuda.set_device(0)
     e = W.elem_size(dtype)
     for R, n in [(2, 4099), (4, 4 * 30_000 + 4), (8, 8 * 8192), (3, 10)]:
@@ -36,6 +38,7 @@ def test_collectives_over_host_bounce(oracle, dtype, use_graph):
         want = oracle.ring_allreduce(xs)
         comm = _comm(R, n, dtype, 4 * R * (n * e + 4096))
         comm.set_param("use_graph", use_graph)
+        comm.set_param("ag_direct", ag_direct)
         comm.set_param("piece_bytes", 16384)
         send = [DevBuf(n * e).put(xs[r]) for r in range(R)]
         recv = [DevBuf(n * e) for _ in range(R)]
