@@ -134,9 +134,11 @@ hoccl_result_t hoccl_comm_set_path(hoccl_comm_t comm, hoccl_path_t path);
  * Tuning and diagnostics.  Keys:
  *  "sum_ctas"    CTAs of a SUM launch, 1..1024 (default 8: the SM budget for sums)
  *  "copy_ctas"   CTAs of an SM copy launch, 1..1024 (default 8)
- *  "piece_bytes" pipeline piece size in bytes (rounded to a multiple of 1024).  Default 4 MiB; on the SM path with
- *                CTA budgets below 64 a reduction whose ring chunk is 1 MiB or more is cut into at least two pieces
- *                so that one piece's copy kernel overlaps the other's sum kernel.  Setting the key turns that off.
+ *  "piece_bytes" pipeline piece size in bytes (rounded to a multiple of 1024).  If the key is not set: whole ring chunks
+ *                on HOCCL_PATH_CE and on HOCCL_PATH_SM when both CTA budgets are 128 or more (pieces exist to overlap one
+ *                piece's move with another piece's sum, which neither driver copies nor whole-GPU grids do); otherwise
+ *                4 MiB, and on the SM path with CTA budgets below 64 a reduction whose ring chunk is 1 MiB or more is
+ *                cut into at least two pieces so that one piece's copy kernel overlaps the other's sum kernel.
  *  "max_pieces"  cap on pieces per ring chunk (default 8)
  *  "lanes"       internal move streams of the stream executor, 1..8 (default 4)
  *  "p2p_split"   a send/recv message of 32 MiB or more on the CE path is cut into up to this many slices that

@@ -314,12 +314,15 @@ def gradients(args):
         for b in [int(x) for x in args.budgets.split(",")]:
             configs.append(("SM_copy%d_sum%d" % (b, min(b, 8)), hb.PATH_SM, min(b, 8), b))
         configs.append(("SM_copy148_sum148", hb.PATH_SM, 148, 148))
+    if getattr(args, "direct", False):   # every SM-path configuration once more with the direct (fan-out) all-gather
+        configs = configs + [(n_ + "_direct", p_, s_, c_) for n_, p_, s_, c_ in configs if p_ == hb.PATH_SM]
     for name, path, sc, cc in configs:
         comm = hb.Comm(R, 0)
         comm.set_scratch(scratch.data_ptr() + pad, scratch.numel() - 256)
         comm.set_path(path)
         comm.set_param("sum_ctas", sc)
         comm.set_param("copy_ctas", cc)
+        comm.set_param("ag_direct", 1 if name.endswith("_direct") else 0)
         for k in range(pool):
             comm.allreduce(send[k], recv[k], per, dtype, stream)
         stream.synchronize()
@@ -472,6 +475,7 @@ def main():
     g = sub.add_parser("gradients")
     g.add_argument("--buckets", type=int, default=32)
     g.add_argument("--budgets", default="", help="comma list of copy-kernel CTA budgets, e.g. 1,2,4,8,16,32,64")
+    g.add_argument("--direct", action="store_true", help="repeat every SM-path configuration with ag_direct = 1")
     sub.add_parser("launch-cost")
     a2 = sub.add_parser("alltoallv")
     a2.add_argument("--mib", default="4,64,256", help="comma list of MiB sent per rank")
