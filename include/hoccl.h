@@ -169,8 +169,8 @@ hoccl_result_t hoccl_comm_set_path(hoccl_comm_t comm, hoccl_path_t path);
  *                Its grid is min(sum_ctas, copy_ctas) CTAs (copy_ctas for pure moves), fewer for small messages.
  *                Measured on B200 (R = 8, bf16, whole GPU): a grid barrier costs ~4 us against ~1.5 us for a kernel
  *                boundary inside a CUDA graph, so below 128 MiB per rank the graph of per-step kernels is faster (4 KiB
- *                all-reduce: 31 against 96 us); from 128 MiB on the one-kernel form is 3-10 % faster (no ramp and tail
- *                per step: 0.78-0.80 against 0.73-0.77 of the 8 TB/s roofline).  Under an 8-CTA budget the graph is
+ *                all-reduce: 31 against 96 us); from 128 MiB on the one-kernel form is 1-3 % faster (no ramp and tail
+ *                per step: 0.78-0.80 against 0.76-0.78 of the 8 TB/s roofline).  Under an 8-CTA budget the graph is
  *                faster at every size, because it overlaps a copy kernel with a sum kernel.
  *                Every barrier wait is bounded; a wait that runs out ends the kernel and is reported by
  *                hoccl_comm_async_error as HOCCL_ERR_TIMEOUT.  The library allocates 16 bytes of device memory and 4 bytes
