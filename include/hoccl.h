@@ -134,8 +134,8 @@ hoccl_result_t hoccl_comm_set_path(hoccl_comm_t comm, hoccl_path_t path);
  * Tuning and diagnostics.  Keys:
  *  "sum_ctas"    CTAs of a SUM launch, 1..1024 (default 8: the SM budget for sums)
  *  "copy_ctas"   CTAs of an SM copy launch, 1..1024 (default 8)
- *  "piece_bytes" pipeline piece size in bytes (rounded to a multiple of 1024).  If the key is not set: whole ring chunks
- *                on HOCCL_PATH_CE and on HOCCL_PATH_SM when both CTA budgets are 128 or more (pieces exist to overlap one
+ *  "piece_bytes" pipeline piece size in bytes (rounded to a multiple of 1024).  If the key is not set: for reductions, whole
+ *                ring chunks (up to 256 MiB) on HOCCL_PATH_CE and on HOCCL_PATH_SM when both CTA budgets are 128 or more (pieces exist to overlap one
  *                piece's move with another piece's sum, which neither driver copies nor whole-GPU grids do); otherwise
  *                4 MiB, and on the SM path with CTA budgets below 64 a reduction whose ring chunk is 1 MiB or more is
  *                cut into at least two pieces so that one piece's copy kernel overlaps the other's sum kernel.

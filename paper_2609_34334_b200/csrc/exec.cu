@@ -573,7 +573,7 @@ hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
   // pieces (the copy kernel of one piece then overlaps the sum kernel of the other: measured 1.6x on a 3 MiB chunk with
   // 8 + 8 CTAs) of at most 4 MiB.  That does not pay with driver copies (they take the whole GPU and never overlap a sum:
   // every extra copy only adds its start-up) nor with whole-GPU grids (two kernels then share the same SMs), so the
-  // copy route and the SM path with 128 CTAs or more for both kernels keep whole chunks at every size (measured, R = 8,
+  // copy route and the SM path with 128 CTAs or more for both kernels keep whole chunks up to 256 MiB (measured, R = 8,
   // bf16, 64 MiB to 1 GiB per rank: 7-15 % faster than 4 MiB pieces on the copy route with 8-CTA sums, 19-33 % with
   // 148-CTA sums, 3-14 % on the whole-GPU SM path).
   size_t piece_bytes = (size_t)c->piece_bytes;
@@ -586,8 +586,10 @@ hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
   } else if (fused) {   // one kernel walks the steps in order; whole chunks measured faster than pieces (fewer barriers and tails)
     piece_bytes = (size_t)1 << 60;
     max_pieces = 1;
-  } else if (!c->piece_bytes_set && (c->path == HOCCL_PATH_CE || (c->path == HOCCL_PATH_SM && std::min(c->sum_ctas, c->copy_ctas) >= 128))) {
-    piece_bytes = (size_t)1 << 60;
+  } else if (!c->piece_bytes_set && (call->kind == PLAN_ALLREDUCE || call->kind == PLAN_REDUCE_SCATTER) &&
+             (c->path == HOCCL_PATH_CE || (c->path == HOCCL_PATH_SM && std::min(c->sum_ctas, c->copy_ctas) >= 128))) {
+    // "whole" stops at 256 MiB: several concurrent driver copies of 512 MiB each ran at half speed (R = 2, 1 GiB per rank)
+    piece_bytes = (size_t)256 << 20;
   } else if (!c->piece_bytes_set && c->path == HOCCL_PATH_SM && std::max(c->sum_ctas, c->copy_ctas) < 64 &&
       (call->kind == PLAN_ALLREDUCE || call->kind == PLAN_REDUCE_SCATTER)) {
     const size_t q = call->kind == PLAN_ALLREDUCE ? (call->count + c->R - 1) / c->R : call->count;

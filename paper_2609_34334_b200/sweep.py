@@ -107,6 +107,7 @@ def sweep_sizes(args):
     configs = [("CE", hb.PATH_CE, 8, 8, 0), ("SM8", hb.PATH_SM, 8, 8, 0), ("SMall", hb.PATH_SM, 148, 148, 0),
                ("SM8fused", hb.PATH_SM, 8, 8, 1), ("SMallfused", hb.PATH_SM, 148, 148, 1),
                # all-gather as independent stages (fan-out copy on the SM path); the last one adds the forward comparison variant
+               ("CEall", hb.PATH_CE, 148, 8, 0),   # copy route with whole-GPU sums: what the route reaches without the 8-CTA SUM budget
                ("CEdirect", hb.PATH_CE, 8, 8, 0), ("SM8direct", hb.PATH_SM, 8, 8, 0), ("SMalldirect", hb.PATH_SM, 148, 148, 0),
                ("SMallfwddirect", hb.PATH_SM, 148, 148, 0)]
     if args.configs != "all":
