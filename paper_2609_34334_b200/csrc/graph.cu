@@ -119,6 +119,12 @@ hoccl_result_t build_graph(hoccl_comm* c, const Plan& P, const std::vector<RGrou
         size_t sub = sg.bytes;
         if (c->ce_sub_bytes > 0 && sg.bytes > (size_t)c->ce_sub_bytes && sg.bytes < ((size_t)16 << 20))
           sub = ((size_t)c->ce_sub_bytes + 255) / 256 * 256;
+        // All-to-all: its R (R-1) copies are all independent, and that many concurrent driver copies of 4-16 MiB run one
+        // after the other at ~5 us each (measured, R = 8: 348 us for 4 MiB blocks, 448 us for 8 MiB blocks); as 2 MiB
+        // sub-copies they take 107 and 211 us.  A ring stage (R copies at a time) does not show this and is left alone, and
+        // with 16 copies or fewer (R <= 4; R = 5 was not measured) sub-copies were as often slower as faster.
+        else if (c->ce_sub_bytes == 0 && P.kind == PLAN_ALLTOALL && P.R * P.R > 32 && sg.bytes >= ((size_t)4 << 20) && sg.bytes < ((size_t)16 << 20))
+          sub = (size_t)2 << 20;
         for (size_t off = 0; off < sg.bytes && e == cudaSuccess; off += sub) {
           cudaGraphNode_t n;
           e = cudaGraphAddMemcpyNode1D(&n, g, deps.data(), deps.size(), sg.dst + off, sg.src + off, std::min(sub, sg.bytes - off),
