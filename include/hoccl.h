@@ -437,6 +437,17 @@ hoccl_result_t hoccl_port_probe(int mode, void* buf, size_t bytes, int ctas, uns
 hoccl_result_t hoccl_flatten_inspect(int kind, hoccl_dtype_t dtype, int ctas, int nseg, const uint64_t* a_addr, const uint64_t* b_addr,
                                      const uint64_t* out_addr, const uint64_t* len, uint64_t* tiles_end, uint64_t* scalars_end,
                                      uint64_t* nvec, uint32_t* head, uint64_t* tile_vectors);
+/*
+ * Host only (no device needed): how a group of `n` moves, given by their ADDRESSES as integers (src[i] -> dst[i], len[i]
+ * bytes), is packed into fan-out launches.  Moves with the same source, length and 16-byte phase of the destination share
+ * one segment (one read, one store per destination); a launch carries at most 32 segments and 256 destinations.
+ * Output, one entry per segment in launch order (arrays of capacity seg_cap): its launch index, source, length, number
+ * of destinations, head / nvec of its split under the kernel shape `ctas` selects; its destinations follow each other in
+ * dst_out (capacity n).  *n_seg = 0 means no source repeats: the moves go as plain copies.  Nothing is read or written.
+ */
+hoccl_result_t hoccl_fanout_inspect(int n, const uint64_t* src, const uint64_t* dst, const uint64_t* len, int ctas, int seg_cap,
+                                    int* seg_launch, uint64_t* seg_src, uint64_t* seg_len, int* seg_ndst, uint32_t* seg_head,
+                                    uint64_t* seg_nvec, uint64_t* dst_out, int* n_seg, int* n_launch);
 hoccl_result_t hoccl_kernel_sms(int kind, const void* a, const void* b, void* out, size_t bytes, hoccl_dtype_t dtype, int ctas,
                                 unsigned int* smid_out, hoccl_stream_t stream);
 

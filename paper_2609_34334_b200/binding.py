@@ -28,7 +28,7 @@ EXPORTS = [
     "hoccl_comm_set_path", "hoccl_comm_set_param", "hoccl_comm_get_param", "hoccl_allreduce", "hoccl_reduce_scatter",
     "hoccl_allgather", "hoccl_alltoall", "hoccl_alltoallv", "hoccl_send", "hoccl_recv", "hoccl_comm_pending", "hoccl_comm_async_error", "hoccl_comm_handshakes", "hoccl_selftest_barrier_timeout", "hoccl_host_allreduce", "hoccl_error_string",
     "hoccl_last_cuda_error", "hoccl_last_stats", "hoccl_profile_reset", "hoccl_probe_move_needs_sm", "hoccl_probe_copy_routes", "hoccl_sum_launch", "hoccl_kernel_sms", "hoccl_flatten_inspect", "hoccl_port_probe",
-    "hoccl_copy_launch", "hoccl_fanout_launch", "hoccl_plan_build", "hoccl_plan_destroy", "hoccl_plan_num_ops", "hoccl_plan_num_groups",
+    "hoccl_copy_launch", "hoccl_fanout_launch", "hoccl_fanout_inspect", "hoccl_plan_build", "hoccl_plan_destroy", "hoccl_plan_num_ops", "hoccl_plan_num_groups",
     "hoccl_plan_get_op", "hoccl_plan_group_deps", "hoccl_plan_slot_bytes", "hoccl_allreduce_static",
     "hoccl_sched_build", "hoccl_sched_destroy", "hoccl_sched_num_stages", "hoccl_sched_stage_tau", "hoccl_sched_total_tau",
     "hoccl_sched_lower_bound", "hoccl_sched_matrix", "hoccl_sched_num_flows", "hoccl_sched_get_flow", "hoccl_sched_queue_len",
@@ -134,6 +134,7 @@ def lib() -> ctypes.CDLL:
         "hoccl_sum_launch": (i, [vp, vp, vp, sz, i, i, vp]),
         "hoccl_copy_launch": (i, [vp, vp, sz, i, vp]),
         "hoccl_fanout_launch": (i, [vp, vp, i, sz, i, vp]),
+        "hoccl_fanout_inspect": (i, [i, vp, vp, vp, i, i, vp, vp, vp, vp, vp, vp, vp, ctypes.POINTER(i), ctypes.POINTER(i)]),
         "hoccl_kernel_sms": (i, [i, vp, vp, vp, sz, i, i, vp, vp]),
         "hoccl_selftest_barrier_timeout": (i, [vp, vp, vp, sz, vp]),
         "hoccl_port_probe": (i, [i, vp, sz, i, vp, vp]),
@@ -367,6 +368,28 @@ def copy_launch(src, dst, nbytes, ctas, stream=None) -> int:
 def fanout_launch(src, dsts, nbytes, ctas, stream=None) -> int:
     """hoccl_fanout_launch: every dsts[d] <- src, the source read once.  Returns the result code."""
     return lib().hoccl_fanout_launch(_ptr(src), _ptr_array(dsts), len(dsts), nbytes, ctas, _stream(stream))
+
+
+def fanout_inspect(moves, ctas: int = 8):
+    """hoccl_fanout_inspect (host only): moves = [(src_addr, dst_addr, nbytes), ...] -> (segments, launches) where a segment is
+    (launch, src_addr, nbytes, [dst_addr, ...], head, nvec); no segments means the moves go as plain copies."""
+    n = len(moves)
+    u64 = ctypes.c_uint64 * n
+    src, dst, ln = u64(*[m[0] for m in moves]), u64(*[m[1] for m in moves]), u64(*[m[2] for m in moves])
+    cap = n
+    seg_launch, seg_nd = (ctypes.c_int * cap)(), (ctypes.c_int * cap)()
+    seg_src, seg_len, seg_nvec, dst_out = (ctypes.c_uint64 * cap)(), (ctypes.c_uint64 * cap)(), (ctypes.c_uint64 * cap)(), u64()
+    seg_head = (ctypes.c_uint32 * cap)()
+    n_seg, n_launch = ctypes.c_int(0), ctypes.c_int(0)
+    rc = lib().hoccl_fanout_inspect(n, src, dst, ln, ctas, cap, seg_launch, seg_src, seg_len, seg_nd, seg_head, seg_nvec, dst_out,
+                                    ctypes.byref(n_seg), ctypes.byref(n_launch))
+    if rc != OK:
+        raise HocclError(rc, "hoccl_fanout_inspect", "")
+    segs, at = [], 0
+    for k in range(n_seg.value):
+        segs.append((seg_launch[k], seg_src[k], seg_len[k], [dst_out[at + d] for d in range(seg_nd[k])], seg_head[k], seg_nvec[k]))
+        at += seg_nd[k]
+    return segs, n_launch.value
 
 
 def kernel_sms(kind: str, a, b, out, nbytes: int, dtype, ctas: int, smid_out, stream=None) -> int:

@@ -643,6 +643,51 @@ hoccl_result_t hoccl_flatten_inspect(int kind, hoccl_dtype_t dtype, int ctas, in
   return HOCCL_OK;
 }
 
+hoccl_result_t hoccl_fanout_inspect(int n, const uint64_t* src, const uint64_t* dst, const uint64_t* len, int ctas, int seg_cap,
+                                    int* seg_launch, uint64_t* seg_src, uint64_t* seg_len, int* seg_ndst, uint32_t* seg_head,
+                                    uint64_t* seg_nvec, uint64_t* dst_out, int* n_seg, int* n_launch) {
+  if (n < 1 || !src || !dst || !len || ctas < 1 || seg_cap < 1 || !seg_launch || !seg_src || !seg_len || !seg_ndst || !seg_head ||
+      !seg_nvec || !dst_out || !n_seg || !n_launch)
+    return HOCCL_ERR_INVALID_ARG;
+  RGroup g;
+  g.kind = OP_MOVE;
+  g.piece = 0;
+  g.chain_dep = -1;
+  for (int i = 0; i < n; i++) {
+    Seg sg = {};
+    sg.src = (const char*)(uintptr_t)src[i];
+    sg.dst = (char*)(uintptr_t)dst[i];
+    sg.bytes = len[i];
+    g.segs.push_back(sg);
+  }
+  std::vector<FanBatch> fans;
+  std::vector<double> hbm;
+  std::vector<long> moves;
+  *n_seg = 0;
+  *n_launch = 0;
+  if (!build_fan_batches(g, &fans, &hbm, &moves)) return HOCCL_OK;
+  int k = 0;
+  size_t nd = 0;
+  for (size_t b = 0; b < fans.size(); b++) {
+    prepare_fan_batch(&fans[b], ctas);
+    for (int j = 0; j < fans[b].nseg; j++) {
+      const FanSeg& fs = fans[b].seg[j];
+      if (k >= seg_cap || nd + (size_t)fs.ndst > (size_t)n) return HOCCL_ERR_INVALID_ARG;
+      seg_launch[k] = (int)b;
+      seg_src[k] = (uint64_t)(uintptr_t)fs.src;
+      seg_len[k] = fs.bytes;
+      seg_ndst[k] = fs.ndst;
+      seg_head[k] = fans[b].flat.head[j];
+      seg_nvec[k] = fans[b].flat.nvec[j];
+      for (int d = 0; d < fs.ndst; d++) dst_out[nd++] = (uint64_t)(uintptr_t)fans[b].dst[fs.first_dst + d];
+      k++;
+    }
+  }
+  *n_seg = k;
+  *n_launch = (int)fans.size();
+  return HOCCL_OK;
+}
+
 hoccl_result_t hoccl_kernel_sms(int kind, const void* a, const void* b, void* out, size_t bytes, hoccl_dtype_t dtype, int ctas,
                                 unsigned int* smid_out, hoccl_stream_t stream) {
   size_t e = dtype_size((int)dtype);

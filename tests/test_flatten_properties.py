@@ -78,3 +78,64 @@ def test_aligned_segments_take_the_vector_path():
     assert tile_v == 4 * 512 and view[0][0] == 13 and view[0][1] == (100_000 - 13) // 16
     view, _ = hb.flatten_inspect("copy", "bf16", 8, [4096 + 3], None, [8192 + 4], [100_000])
     assert view[0][1] == 0 and view[0][3] == 100_000                         # no common phase: element-wise fallback
+
+
+# ---- fan-out packing (hoccl_fanout_inspect): the moves of a direct all-gather that read the same bytes share one segment
+move_set = st.lists(st.tuples(st.integers(0, 5), st.integers(0, 15), st.sampled_from([0, 0, 0, 3, 8]), st.integers(1, 40)),
+                    min_size=1, max_size=700)
+
+
+@settings(max_examples=150, deadline=None, suppress_health_check=list(HealthCheck), derandomize=True)
+@given(moves=move_set, n_len=st.integers(1, 3), ctas=st.sampled_from([8, 148]))
+def test_fan_out_packing_serves_every_move_exactly_once(moves, n_len, ctas):
+    """Random groups of moves (few sources, few lengths, many destinations with a few 16-byte phases).  Every move must
+    appear exactly once, a segment's destinations share their phase, its split follows that phase, and a launch carries
+    at most 32 segments and 256 destinations."""
+    base, lens = 1 << 32, [4096 + 16 * 7, 100_000, 17][:n_len]
+    src_phase = {}
+    flat = []
+    for k, (s, sp, dp, l) in enumerate(moves):
+        src = base + s * (1 << 24) + src_phase.setdefault(s, sp)      # one address per source
+        dst = base + (64 + k) * (1 << 24) + (src % 16 + dp) % 16      # mostly in phase with the source
+        flat.append((src, dst, lens[l % n_len]))
+    segs, launches = hb.fanout_inspect(flat, ctas)
+    repeats = len({(m[0], m[2], m[1] % 16) for m in flat}) < len(flat)
+    if not repeats:
+        assert segs == [] and launches == 0
+        return
+    served = sorted((src, d, ln) for (_, src, ln, dsts, _, _) in segs for d in dsts)
+    assert served == sorted(flat)
+    per_launch = {}
+    for launch, src, ln, dsts, head, nvec in segs:
+        assert 1 <= len(dsts) <= 256
+        assert len({d % 16 for d in dsts}) == 1
+        in_phase = dsts[0] % 16 == src % 16
+        if in_phase:
+            assert head == min((16 - src % 16) % 16, ln) and nvec == (ln - head) // 16
+        else:
+            assert nvec == 0                                         # element-wise: no vector access on a misaligned pair
+        acc = per_launch.setdefault(launch, [0, 0])
+        acc[0] += 1
+        acc[1] += len(dsts)
+    assert sorted(per_launch) == list(range(launches))
+    for nseg, nd in per_launch.values():
+        assert nseg <= 32 and nd <= 256
+
+
+def test_fan_out_packing_of_a_direct_all_gather():
+    """R = 8 ranks, chunk of 3,276,800 bytes: 56 moves become 8 segments of 7 destinations in one launch."""
+    R, chunk = 8, 3_276_800
+    recv = [(1 << 33) + r * (1 << 28) for r in range(R)]
+    moves = [(recv[r] + r * chunk, recv[(r + k) % R] + r * chunk, chunk) for k in range(1, R) for r in range(R)]
+    segs, launches = hb.fanout_inspect(moves, 148)
+    assert launches == 1 and len(segs) == R
+    for launch, src, ln, dsts, head, nvec in segs:
+        r = (src - recv[0]) // (1 << 28)
+        assert ln == chunk and head == 0 and nvec == chunk // 16 and len(dsts) == R - 1
+        assert sorted(dsts) == sorted(recv[d] + r * chunk for d in range(R) if d != r)
+    # R = 40: 1560 destinations need 7 launches of at most 256
+    R = 40
+    recv = [(1 << 33) + r * (1 << 26) for r in range(R)]
+    moves = [(recv[r] + r * 4096, recv[(r + k) % R] + r * 4096, 4096) for k in range(1, R) for r in range(R)]
+    segs, launches = hb.fanout_inspect(moves, 16)
+    assert launches == -(-R * (R - 1) // 256) and sum(len(s[3]) for s in segs) == R * (R - 1)
