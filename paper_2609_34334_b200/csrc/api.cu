@@ -125,7 +125,7 @@ static long* param_slot(hoccl_comm* c, const char* key, long* lo, long* hi) {
               {"ce_sub_bytes", &c->ce_sub_bytes, 0, 1L << 40}, {"handshake", &c->handshake, 0, 1},
               {"watchdog_ms", &c->watchdog_ms, 10, 600000},    {"onepass", &c->onepass, 0, 1},
               {"forward", &c->forward, 0, 1},           {"fused", &c->fused, 0, 1},
-              {"ag_direct", &c->ag_direct, 0, 1},
+              {"ag_direct", &c->ag_direct, 0, 2},
               {"host_pieces", &c->host_pieces, 1, 64}};
   for (auto& r : rows)
     if (std::strcmp(r.name, key) == 0) {

@@ -567,8 +567,16 @@ hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
   int plan_kind = call->kind;
   if (c->forward && call->kind == PLAN_ALLREDUCE) plan_kind = PLAN_ALLREDUCE_FWD;
   if (c->forward && call->kind == PLAN_REDUCE_SCATTER) plan_kind = PLAN_REDUCE_SCATTER_FWD;
-  if (c->ag_direct && call->kind == PLAN_ALLREDUCE) plan_kind = c->forward ? PLAN_ALLREDUCE_FWD_AGD : PLAN_ALLREDUCE_AGD;
-  if (c->ag_direct && call->kind == PLAN_ALLGATHER) plan_kind = PLAN_ALLGATHER_DIRECT;
+  // ag_direct = 2: where it was measured faster.  Kernels of this library (SM path) and the host bounce: always (fewer
+  // bytes, fewer launches or hops).  Copy route: only while a chunk is at most 4 MiB (R (R-1) concurrent driver copies
+  // of 4-16 MiB serialise; beyond that the two forms are within a few percent).
+  bool direct = c->ag_direct == 1;
+  if (c->ag_direct == 2 && (call->kind == PLAN_ALLREDUCE || call->kind == PLAN_ALLGATHER)) {
+    const size_t q = call->kind == PLAN_ALLREDUCE ? (call->count + c->R - 1) / c->R : call->count;
+    direct = c->path != HOCCL_PATH_CE || q * dtype_size(call->dtype) <= ((size_t)4 << 20);
+  }
+  if (direct && call->kind == PLAN_ALLREDUCE) plan_kind = c->forward ? PLAN_ALLREDUCE_FWD_AGD : PLAN_ALLREDUCE_AGD;
+  if (direct && call->kind == PLAN_ALLGATHER) plan_kind = PLAN_ALLGATHER_DIRECT;
   // Piece size: the caller's if set.  Otherwise: on the SM path under CTA budgets a reduction is cut into at least two
   // pieces (the copy kernel of one piece then overlaps the sum kernel of the other: measured 1.6x on a 3 MiB chunk with
   // 8 + 8 CTAs) of at most 4 MiB.  That does not pay with driver copies (they take the whole GPU and never overlap a sum:
@@ -637,12 +645,18 @@ hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
         for (const PlanGroup& pg : P.groups) any = any || pg.piece == p;
         if (!any) continue;   // e.g. one rank copying in place: nothing to run between the copies
         rc = build_graph(c, P, groups, &entry, p, &entry.piece_exec[p]);
-        if (rc != HOCCL_OK) return rc;
+        if (rc != HOCCL_OK) {
+          destroy_entry(&entry);   // the pieces built so far, and any profile events
+          return rc;
+        }
       }
     } else {
       rc = fused ? build_ring(c, P, groups, &entry) : HOCCL_ERR_UNSUPPORTED;
       if (rc == HOCCL_ERR_UNSUPPORTED) rc = build_graph(c, P, groups, &entry, -1, &entry.exec);   // not asked for, or too many ranks for one launch
-      if (rc != HOCCL_OK) return rc;
+      if (rc != HOCCL_OK) {
+        destroy_entry(&entry);
+        return rc;
+      }
     }
     // handshake mode: place the graph on the device now; the proxy must not meet first-launch work later
     if (c->handshake) {

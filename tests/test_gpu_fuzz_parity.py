@@ -51,7 +51,7 @@ case = st.fixed_dictionaries({
     "offs": st.lists(st.integers(0, 3), min_size=9, max_size=9),
     "flavour": st.sampled_from(["normal", "wide", "special"]),
     "seed": st.integers(0, 2 ** 31 - 1),
-    "ag_direct": st.integers(0, 1),
+    "ag_direct": st.integers(0, 2),
 })
 
 
