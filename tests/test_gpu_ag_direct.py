@@ -180,3 +180,40 @@ def test_automatic_choice(oracle):
         got = run_allreduce(comm, xs, dtype, in_place=True)
         assert all(same_bits(got[r], want[r], dtype) for r in range(R)), chunk_bytes
         comm.destroy()
+
+
+def test_config2_bucket_full_size_every_timed_variant(oracle):
+    """The gradient bucket at full size (R = 8, 25 MiB bf16 per rank), reduce-scatter then all-gather as the benchmark runs
+    it, in every configuration its variant tables time with the direct all-gather (and the ring beside it): all bits
+    equal the oracle's."""
+    c = W.C2_DP_BUCKET
+    R, n, e = c.R, c.count, 2
+    xs = W.rank_inputs(c.dist, c.seed, R, n, c.dtype, c.sigma)
+    want = oracle.ring_allreduce(xs, threads=oracle.max_threads())
+    count = n // R
+    send = [DevBuf(n * e).put(xs[r]) for r in range(R)]
+    recv = [DevBuf(n * e) for _ in range(R)]
+    host = torch.empty(400 << 20, dtype=torch.uint8).pin_memory()
+    variants = [(hb.PATH_CE, dict(sum_ctas=8, ag_direct=1)), (hb.PATH_CE, dict(sum_ctas=148, ag_direct=1)),
+                (hb.PATH_SM, dict(sum_ctas=8, copy_ctas=8, ag_direct=1)), (hb.PATH_SM, dict(sum_ctas=8, copy_ctas=48, ag_direct=1)),
+                (hb.PATH_SM, dict(sum_ctas=148, copy_ctas=148, ag_direct=1)), (hb.PATH_SM, dict(sum_ctas=148, copy_ctas=148, ag_direct=1, forward=1)),
+                (hb.PATH_SM, dict(sum_ctas=148, copy_ctas=148, ag_direct=0)), (hb.PATH_SM, dict(sum_ctas=8, copy_ctas=48, ag_direct=2)),
+                (hb.PATH_CE_HOST, dict(sum_ctas=8, ag_direct=1))]
+    for path, params in variants:
+        comm = make_comm(R, n, c.dtype, path, **params)
+        if path == hb.PATH_CE_HOST:
+            comm.set_host_staging(host)
+        for two_calls in (True, False):
+            for b in recv:
+                b.view.fill_(0)
+            if two_calls:
+                rs_out = [recv[r].ptr + r * count * e for r in range(R)]
+                comm.reduce_scatter(send, rs_out, count, c.dtype)
+                comm.allgather(rs_out, recv, count, c.dtype)
+            else:
+                comm.allreduce(send, recv, n, c.dtype)
+            torch.cuda.synchronize()
+            for r in range(R):
+                assert same_bits(recv[r].get(np.uint16), want[r], c.dtype), (path, params, two_calls, r)
+                assert recv[r].guards_intact() and send[r].guards_intact()
+        comm.destroy()
