@@ -269,11 +269,17 @@ def main():
     win.sort()
     windows = {"n": 10, "steps_each": max(5, steps // 10), "median_ms_per_step": win[len(win) // 2], "best_ms_per_step": win[0],
                "worst_ms_per_step": win[-1]}
-    # launches of our kernels per step: the SUM launches of the reduce-scatter (the all-gather has none on this path)
-    comm.reduce_scatter(send_sets[0], [recv_sets[0][r].data_ptr() + r * count * e for r in range(R)], count, dtype, stream)
+    # launches of our kernels per step: the SUM launches of the reduce-scatter, plus the empty one-warp kernel that each of
+    # the two graphs puts in front of its first copies (the all-gather has no other kernel of ours on this path)
+    rs_out0 = [recv_sets[0][r].data_ptr() + r * count * e for r in range(R)]
+    comm.allgather(rs_out0, recv_sets[0], count, dtype, stream)
+    stream.synchronize()
+    ag_stats = comm.last_stats()
+    comm.reduce_scatter(send_sets[0], rs_out0, count, dtype, stream)
     stream.synchronize()
     rs_stats = comm.last_stats()
-    launches_per_step = rs_stats["n_sum_launches"] + rs_stats["n_move_launches"]
+    launches_per_step = (rs_stats["n_sum_launches"] + rs_stats["n_move_launches"] + rs_stats["n_order_launches"] +
+                         ag_stats["n_sum_launches"] + ag_stats["n_move_launches"] + ag_stats["n_order_launches"])
 
     # results of the timed configuration on bucket set 0 (ranks 0 and 5, full vectors), kept for the comparison with the
     # oracle, which happens where the oracle runs: in the CPU-baseline leg below

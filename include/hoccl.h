@@ -96,6 +96,7 @@ typedef struct {
   double copy_kernel_ms;   /* the same for copy_kernel launches (SM path, graph executor) */
   long copy_kernel_launches_timed;
   double copy_kernel_bytes; /* algorithmic bytes (1 read + 1 write per byte) of those launches */
+  long n_order_launches;    /* empty one-warp kernels of the last call that only order copy nodes inside its graph (copy routes) */
 } hoccl_stats_t;
 
 /* ---------------------------------------------------------------- communicator ----------------- */
@@ -145,9 +146,7 @@ hoccl_result_t hoccl_comm_set_path(hoccl_comm_t comm, hoccl_path_t path);
  *                run on different lanes, 1..8 (default 1 = one copy per message; measured: slices do not help
  *                on one device because every driver copy already spreads over the whole GPU)
  *  "ce_sub_bytes" graph executor, CE path: a move between this many bytes and 16 MiB is issued as sub-copies of
- *                this size.  0 (default) = automatic: only the blocks of an all-to-all over 6 or more ranks between 4 and 16 MiB are cut, into
- *                2 MiB sub-copies (its R (R-1) independent driver copies of that size otherwise run one after the other);
- *                16 MiB or more = never cut
+ *                this size (0 = off, the default; measured: no gain once a graph's first copies share one predecessor)
  *  "onepass"     1 = all-reduce and reduce-scatter run as ONE kernel ("sum_ctas" CTAs) that reduces every element in
  *                registers in the ring's order and rounding and writes it to its destinations: the same bits, R reads
  *                + R (or 1) writes per element instead of 7(R-1) bytes per wire byte, no moves, no scratch.  It is not

@@ -47,6 +47,7 @@ class Stats(ctypes.Structure):
         ("n_pieces", ctypes.c_long), ("graph_hit", ctypes.c_long), ("sum_kernel_ms", ctypes.c_double),
         ("sum_kernel_launches_timed", ctypes.c_long), ("sum_kernel_bytes", ctypes.c_double),
         ("copy_kernel_ms", ctypes.c_double), ("copy_kernel_launches_timed", ctypes.c_long), ("copy_kernel_bytes", ctypes.c_double),
+        ("n_order_launches", ctypes.c_long),
     ]
 
     def as_dict(self):

@@ -65,7 +65,7 @@ struct GraphEntry {
   std::vector<uint64_t> key;
   cudaGraphExec_t exec = nullptr;
   uint64_t last_use = 0;
-  long n_moves = 0, n_move_launches = 0, n_sum_launches = 0, n_pieces = 0;
+  long n_moves = 0, n_move_launches = 0, n_sum_launches = 0, n_pieces = 0, n_order_launches = 0;
   std::vector<std::pair<cudaEvent_t, cudaEvent_t>> prof_events;  // owned; only with profile = 1
   std::vector<double> prof_bytes;
   bool prof_pending = false;  // replayed since the profile events were last read

@@ -498,6 +498,7 @@ static hoccl_result_t launch_entry(hoccl_comm* c, GraphEntry* hit, cudaStream_t 
   c->stats.n_moves = hit->n_moves;
   c->stats.n_move_launches = hit->n_move_launches;
   c->stats.n_sum_launches = hit->n_sum_launches;
+  c->stats.n_order_launches = hit->n_order_launches;
   c->stats.max_sum_ctas = hit->n_sum_launches ? c->sum_ctas : 0;
   c->stats.max_copy_ctas = hit->n_move_launches ? c->copy_ctas : 0;
   c->stats.host_launch_us = now_us() - t0;

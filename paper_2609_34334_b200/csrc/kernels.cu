@@ -326,6 +326,9 @@ __global__ void __launch_bounds__(1024, 1) port_probe_kernel(uint4* buf, unsigne
   if (MODE == 0 && (acc.x ^ acc.y ^ acc.z ^ acc.w) == 0x9e3779b9u) *sink = 1;   // keeps the loads alive
 }
 
+// Does nothing: a graph node that only orders (see build_graph).
+__global__ void graph_root_kernel() {}
+
 __device__ __forceinline__ unsigned long long global_ns() {
   unsigned long long t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
@@ -470,6 +473,7 @@ const void* copy_kernel_entry(int ctas, int* threads) {
   *threads = wide_copy_grid(ctas) ? 512 : 1024;
   return wide_copy_grid(ctas) ? reinterpret_cast<const void*>(&copy_kernel<4, 512>) : reinterpret_cast<const void*>(&copy_kernel<8, 1024>);
 }
+const void* graph_root_kernel_entry() { return reinterpret_cast<const void*>(&graph_root_kernel); }
 const void* fan_kernel_entry(int ctas, int* threads) {
   *threads = wide_copy_grid(ctas) ? 512 : 1024;
   return wide_copy_grid(ctas) ? reinterpret_cast<const void*>(&fan_kernel<4, 512>) : reinterpret_cast<const void*>(&fan_kernel<8, 1024>);
@@ -484,7 +488,7 @@ cudaError_t preload_kernels() {
                        reinterpret_cast<const void*>(&occupy_kernel),           reinterpret_cast<const void*>(&onepass_kernel<0, 512>),
                        reinterpret_cast<const void*>(&onepass_kernel<1, 512>),  reinterpret_cast<const void*>(&onepass_kernel<0, 1024>),
                        reinterpret_cast<const void*>(&onepass_kernel<1, 1024>), reinterpret_cast<const void*>(&fan_kernel<4, 512>),
-                       reinterpret_cast<const void*>(&fan_kernel<8, 1024>)};
+                       reinterpret_cast<const void*>(&fan_kernel<8, 1024>), reinterpret_cast<const void*>(&graph_root_kernel)};
   for (const void* f : fns) {
     cudaFuncAttributes a;
     cudaError_t e = cudaFuncGetAttributes(&a, f);

@@ -140,6 +140,7 @@ void prepare_copy_batch(CopyBatch* batch, int ctas);
 // Kernel entry addresses and parameter blocks for CUDA graph kernel nodes.
 const void* sum_kernel_entry(int dtype, int ctas, int* threads);
 const void* copy_kernel_entry(int ctas, int* threads);
+const void* graph_root_kernel_entry();   // an empty kernel (1 CTA of 32 threads): common predecessor of many root copy nodes
 
 // Memory-port probe: `ctas` CTAs only read (mode 0) or only write (mode 1) `bytes` bytes (a multiple of 128 KiB is walked).
 cudaError_t launch_port_probe(int mode, void* buf, unsigned long long bytes, int ctas, unsigned int* sink, cudaStream_t stream);

@@ -26,6 +26,7 @@ def test_bench_line_has_the_contract_keys():
     assert d["e2e"]["h2d_bytes_per_step"] == 8 * 26214400 and d["e2e"]["value"] < d["value"]
     r = d["roofline"]
     assert r["bound"] == "hbm" and r["unit"] == "GB/s" and abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-9 and r["traffic"] > 0
-    assert d["gpu_launches"] == 7 * 8                         # seven SUM launches per step, nothing else is ours on this path
+    # per step: seven SUM launches plus the empty ordering kernel in front of each of the two graphs' first copies
+    assert d["gpu_launches"] == (7 + 2) * 8
     c = d["cpu_baseline"]
     assert c["kind"] == "oracle" and c["cores"] >= 1 and c["value"] > 0
