@@ -164,7 +164,7 @@ hoccl_result_t hoccl_comm_set_path(hoccl_comm_t comm, hoccl_path_t path);
  *                in which every chunk is read once and stored R-1 times (S R instead of 2 S (R-1) bytes of traffic);
  *                HOCCL_PATH_CE_HOST: a chunk goes out to the host staging once and comes back R-1 times.
  *                0 = the ring all-gather (default).  2 = automatic: direct where it was measured faster on B200 (always on
- *                HOCCL_PATH_SM and HOCCL_PATH_CE_HOST; on HOCCL_PATH_CE while a ring chunk is at most 4 MiB), ring elsewhere.
+ *                HOCCL_PATH_SM and HOCCL_PATH_CE_HOST; on HOCCL_PATH_CE while a ring chunk is at most 64 MiB), ring elsewhere.
  *  "fused"       1 = on HOCCL_PATH_SM the whole collective runs as ONE cooperative kernel that walks the ring steps with a
  *                grid-wide barrier between dependent steps (how an SM-driven library runs a collective: the paper's
  *                "NCCL under an SM budget" baseline, Sec. 5).  The schedule stays rank local and the bits are the same.

@@ -568,13 +568,13 @@ hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
   int plan_kind = call->kind;
   if (c->forward && call->kind == PLAN_ALLREDUCE) plan_kind = PLAN_ALLREDUCE_FWD;
   if (c->forward && call->kind == PLAN_REDUCE_SCATTER) plan_kind = PLAN_REDUCE_SCATTER_FWD;
-  // ag_direct = 2: where it was measured faster.  Kernels of this library (SM path) and the host bounce: always (fewer
-  // bytes, fewer launches or hops).  Copy route: only while a chunk is at most 4 MiB (R (R-1) concurrent driver copies
-  // of 4-16 MiB serialise; beyond that the two forms are within a few percent).
+  // ag_direct = 2: where it was measured faster or equal.  Kernels of this library (SM path) and the host bounce: always
+  // (fewer bytes, fewer launches or hops).  Copy route: the bytes are the same, the gain is the missing chain of stages,
+  // which fades with size (equal within 2 % from 64 MiB per rank at R = 8), so it is taken while a chunk is at most 64 MiB.
   bool direct = c->ag_direct == 1;
   if (c->ag_direct == 2 && (call->kind == PLAN_ALLREDUCE || call->kind == PLAN_ALLGATHER)) {
     const size_t q = call->kind == PLAN_ALLREDUCE ? (call->count + c->R - 1) / c->R : call->count;
-    direct = c->path != HOCCL_PATH_CE || q * dtype_size(call->dtype) <= ((size_t)4 << 20);
+    direct = c->path != HOCCL_PATH_CE || q * dtype_size(call->dtype) <= ((size_t)64 << 20);
   }
   if (direct && call->kind == PLAN_ALLREDUCE) plan_kind = c->forward ? PLAN_ALLREDUCE_FWD_AGD : PLAN_ALLREDUCE_AGD;
   if (direct && call->kind == PLAN_ALLGATHER) plan_kind = PLAN_ALLGATHER_DIRECT;

@@ -162,7 +162,7 @@ def test_many_ranks_need_several_fan_out_launches(oracle, use_graph):
 
 def test_automatic_choice(oracle):
     """ag_direct = 2: the SM path takes the direct form (one fan-out launch), the copy route takes it only while a ring
-    chunk is at most 4 MiB; the bits are the oracle's on both sides of that switch."""
+    chunk is at most 64 MiB; the bits are the oracle's on both sides of that switch."""
     R, dtype = 8, "bf16"
     n = 8 * 100_000
     xs = W.rank_inputs("normal", 96, R, n, dtype, 1e-3)
@@ -172,10 +172,11 @@ def test_automatic_choice(oracle):
     assert all(same_bits(got[r], want[r], dtype) for r in range(R))
     assert comm.last_stats()["n_move_launches"] == 7 + 1
     comm.destroy()
-    for chunk_bytes in ((4 << 20), (4 << 20) + 4096):          # the last size at which the copy route goes direct, and the next
+    R = 2
+    for chunk_bytes in ((64 << 20), (64 << 20) + 4096):        # the last size at which the copy route goes direct, and the next
         n = R * chunk_bytes // 2
         xs = W.rank_inputs("normal", 97, R, n, dtype, 1e-3)
-        want = oracle.ring_allreduce(xs)
+        want = oracle.ring_allreduce(xs, threads=oracle.max_threads())
         comm = make_comm(R, n, dtype, hb.PATH_CE, ag_direct=2)
         got = run_allreduce(comm, xs, dtype, in_place=True)
         assert all(same_bits(got[r], want[r], dtype) for r in range(R)), chunk_bytes
