@@ -269,8 +269,8 @@ def main():
     win.sort()
     windows = {"n": 10, "steps_each": max(5, steps // 10), "median_ms_per_step": win[len(win) // 2], "best_ms_per_step": win[0],
                "worst_ms_per_step": win[-1]}
-    # launches of our kernels per step: the SUM launches of the reduce-scatter, plus the empty one-warp kernel that each of
-    # the two graphs puts in front of its first copies (the all-gather has no other kernel of ours on this path)
+    # launches of our kernels per step: the SUM launches of the reduce-scatter, plus the empty one-warp kernels that order
+    # copy nodes inside the two graphs (in front of each graph's first copies and behind each all-gather stage)
     rs_out0 = [recv_sets[0][r].data_ptr() + r * count * e for r in range(R)]
     comm.allgather(rs_out0, recv_sets[0], count, dtype, stream)
     stream.synchronize()
@@ -498,6 +498,15 @@ def extras(hb, W, torch, np, new_comm, step, timed, stream, R, S, n, dtype, peak
                      "busbw_GBps": S * bus_factor(R) / t / 1e9, "hbm_frac_of_8TBps": hbm / t / 1e9 / NOMINAL_HBM_GBS})
         cm.destroy()
     out["variants"] = rows
+    # the same copy-route graphs without their empty ordering kernels (parameter "order_kernels" = 0): the comparison point
+    pg_rows = []
+    for sc in (8, 148):
+        cm = new_comm(hb.PATH_CE, sum_ctas=sc, order_kernels=0)
+        t, _ = timed(cm, k, w)
+        pg_rows.append({"path": "CE", "sum_ctas": sc, "ms_per_step": t * 1e3, "busbw_GBps": S * bus_factor(R) / t / 1e9,
+                        "hbm_frac_of_8TBps": hbm / t / 1e9 / NOMINAL_HBM_GBS})
+        cm.destroy()
+    out["plain_graphs_no_order_kernels"] = pg_rows
     # SM footprint of this library's kernels on the SM path (SMs x busy time per step), per-launch CUDA events in the graph
     fp_rows = []
     for sc, cc in ((8, 8), (8, 32), (8, 48), (148, 148)):
@@ -694,7 +703,8 @@ def extras(hb, W, torch, np, new_comm, step, timed, stream, R, S, n, dtype, peak
     probe = {}
     alone, _ = gemm_tflops(None)
     probe["alone_TFLOPs"] = alone
-    for name, path, sc, cc, op, fw in (("CE_sum8", hb.PATH_CE, 8, 8, 0, 0), ("SM_copy8_sum8", hb.PATH_SM, 8, 8, 0, 0),
+    for name, path, sc, cc, op, fw in (("CE_sum8", hb.PATH_CE, 8, 8, 0, 0), ("CE_sum8_plain_graphs_no_order_kernels", hb.PATH_CE, 8, 8, 0, 4),
+                                       ("SM_copy8_sum8", hb.PATH_SM, 8, 8, 0, 0),
                                        ("SM_copy32_sum8", hb.PATH_SM, 8, 32, 0, 0), ("SM_copy48_sum8", hb.PATH_SM, 8, 48, 0, 0),
                                        ("SM_copy148_sum148", hb.PATH_SM, 148, 148, 0, 0),
                                        ("SM_copy48_sum8_direct_allgather", hb.PATH_SM, 8, 48, 0, 3),
@@ -702,7 +712,7 @@ def extras(hb, W, torch, np, new_comm, step, timed, stream, R, S, n, dtype, peak
                                        ("SM_one_kernel_8", hb.PATH_SM, 8, 8, 0, 2),
                                        ("onepass_8", hb.PATH_CE, 8, 8, 1, 0), ("CE_HOST_sum8", hb.PATH_CE_HOST, 8, 8, 0, 0)):
         c2 = new_comm(path, sum_ctas=sc, copy_ctas=cc, onepass=op, forward=1 if fw == 1 else 0, fused=1 if fw == 2 else 0,
-                      ag_direct=1 if fw == 3 else 0)
+                      ag_direct=1 if fw == 3 else 0, order_kernels=0 if fw == 4 else 1)
         if path == hb.PATH_CE_HOST:
             c2.set_host_staging(host_stage)
         # the one-pass comparison kernel is one all-reduce call (reduce-scatter + all-gather would add the path's moves)

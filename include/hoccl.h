@@ -165,6 +165,11 @@ hoccl_result_t hoccl_comm_set_path(hoccl_comm_t comm, hoccl_path_t path);
  *                HOCCL_PATH_CE_HOST: a chunk goes out to the host staging once and comes back R-1 times.
  *                0 = the ring all-gather (default).  2 = automatic: direct where it was measured faster on B200 (always on
  *                HOCCL_PATH_SM and HOCCL_PATH_CE_HOST; on HOCCL_PATH_CE while a ring chunk is at most 64 MiB), ring elsewhere.
+ *  "order_kernels" 1 (default) = on the copy routes the graph executor puts an empty one-warp kernel in front of a graph's
+ *                first copies and behind every group of copies that other copies (or the end of the graph) wait for.
+ *                Measured on B200: a copy node that waits for earlier stream work or for several copy nodes starts ~4 us
+ *                late per node, and a GEMM on another stream loses half of its throughput beside such graphs (54 %
+ *                against 8 % for the gradient bucket).  0 = plain graphs (the comparison point).
  *  "fused"       1 = on HOCCL_PATH_SM the whole collective runs as ONE cooperative kernel that walks the ring steps with a
  *                grid-wide barrier between dependent steps (how an SM-driven library runs a collective: the paper's
  *                "NCCL under an SM budget" baseline, Sec. 5).  The schedule stays rank local and the bits are the same.

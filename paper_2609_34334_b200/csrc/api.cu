@@ -126,6 +126,7 @@ static long* param_slot(hoccl_comm* c, const char* key, long* lo, long* hi) {
               {"watchdog_ms", &c->watchdog_ms, 10, 600000},    {"onepass", &c->onepass, 0, 1},
               {"forward", &c->forward, 0, 1},           {"fused", &c->fused, 0, 1},
               {"ag_direct", &c->ag_direct, 0, 2},
+              {"order_kernels", &c->order_kernels, 0, 1},
               {"host_pieces", &c->host_pieces, 1, 64}};
   for (auto& r : rows)
     if (std::strcmp(r.name, key) == 0) {
@@ -307,6 +308,7 @@ hoccl_result_t hoccl_alltoallv(const void* const* send, const size_t* sendcounts
     key.push_back((uint64_t)c->path);
     key.push_back((uint64_t)c->copy_ctas);
     key.push_back((uint64_t)c->piece_bytes);
+    key.push_back((uint64_t)c->order_kernels);
     for (int r = 0; r < R; r++) {
       key.push_back((uint64_t)(uintptr_t)send[r]);
       key.push_back((uint64_t)(uintptr_t)recv[r]);

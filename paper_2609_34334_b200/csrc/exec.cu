@@ -369,6 +369,7 @@ std::vector<uint64_t> make_key(hoccl_comm* c, const Call& call) {
   k.push_back((uint64_t)c->ce_sub_bytes);
   k.push_back((uint64_t)c->forward);
   k.push_back((uint64_t)c->ag_direct);
+  k.push_back((uint64_t)c->order_kernels);
   k.push_back((uint64_t)(c->fused && c->path == HOCCL_PATH_SM && !c->handshake));
   k.push_back((uint64_t)(uintptr_t)c->scratch);
   k.push_back((uint64_t)c->scratch_bytes);

@@ -55,7 +55,7 @@ hoccl_result_t build_graph(hoccl_comm* c, const Plan& P, const std::vector<RGrou
                            cudaGraphExec_t* out_exec) {
   cudaGraph_t g = nullptr;
   CU_TRY(c, cudaGraphCreate(&g, 0));
-  std::vector<cudaGraphNode_t> tail(groups.size(), nullptr);
+  std::vector<std::vector<cudaGraphNode_t>> tail(groups.size());   // the node(s) a consumer of the group waits for
   cudaGraphNode_t last_copy_node = nullptr;
   // Copy nodes without a predecessor each wait for the stream's earlier work on their own, which costs ~4 us per node when
   // that work is still running (measured behind a reduce-scatter: 240 instead of 65 us for the 56 root copies of a direct
@@ -63,12 +63,28 @@ hoccl_result_t build_graph(hoccl_comm* c, const Plan& P, const std::vector<RGrou
   // their common predecessor takes that wait once (an empty graph node does not: it changes nothing).
   cudaGraphNode_t root = nullptr;
   bool many_root_copies = false;
-  if (c->path == HOCCL_PATH_CE || c->path == HOCCL_PATH_CE_HOST) {
+  if (c->order_kernels && (c->path == HOCCL_PATH_CE || c->path == HOCCL_PATH_CE_HOST)) {
     size_t n_root = 0;
     for (size_t gi = 0; gi < groups.size(); gi++)
       if ((only_piece < 0 || groups[gi].piece == only_piece) && groups[gi].kind == OP_MOVE && groups[gi].deps.empty() && groups[gi].chain_dep < 0)
         n_root += groups[gi].segs.size();
     many_root_copies = n_root >= 2;
+  }
+  // The same holds behind a group of copies: copy nodes (or the end of the graph) that wait for several copy nodes start
+  // late; an empty kernel as the join of such a group fixes it (ring all-gather of the gradient bucket, seven stages of eight
+  // copies: 88 -> 68 us; the 56 copies of the direct one: 61 -> 51 us).  A SUM kernel that waits for its copies directly does
+  // not need it (a kernel in between costs ~1 us per step there), so groups that only feed SUMs keep the empty join.
+  std::vector<char> kernel_join(groups.size(), 0);
+  if (c->order_kernels && (c->path == HOCCL_PATH_CE || c->path == HOCCL_PATH_CE_HOST)) {
+    std::vector<char> move_user(groups.size(), 0), any_user(groups.size(), 0);
+    for (size_t gi = 0; gi < groups.size(); gi++) {
+      if (only_piece >= 0 && groups[gi].piece != only_piece) continue;
+      for (int d : groups[gi].deps) {
+        any_user[d] = 1;
+        if (groups[gi].kind == OP_MOVE) move_user[d] = 1;
+      }
+    }
+    for (size_t gi = 0; gi < groups.size(); gi++) kernel_join[gi] = groups[gi].kind == OP_MOVE && (move_user[gi] || !any_user[gi]);
   }
   hoccl_result_t rc = HOCCL_OK;
   auto fail = [&](cudaError_t e, const char* what) {
@@ -79,9 +95,9 @@ hoccl_result_t build_graph(hoccl_comm* c, const Plan& P, const std::vector<RGrou
     const RGroup& rg = groups[gi];
     std::vector<cudaGraphNode_t> deps;
     for (int d : rg.deps)
-      if (tail[d]) deps.push_back(tail[d]);
-    if (rg.chain_dep >= 0 && tail[rg.chain_dep] && std::find(rg.deps.begin(), rg.deps.end(), rg.chain_dep) == rg.deps.end())
-      deps.push_back(tail[rg.chain_dep]);
+      deps.insert(deps.end(), tail[d].begin(), tail[d].end());
+    if (rg.chain_dep >= 0 && std::find(rg.deps.begin(), rg.deps.end(), rg.chain_dep) == rg.deps.end())
+      deps.insert(deps.end(), tail[rg.chain_dep].begin(), tail[rg.chain_dep].end());
     std::vector<cudaGraphNode_t> nodes;
     cudaError_t e = cudaSuccess;
     if (deps.empty() && many_root_copies && rg.kind == OP_MOVE) {
@@ -239,15 +255,25 @@ hoccl_result_t build_graph(hoccl_comm* c, const Plan& P, const std::vector<RGrou
       break;
     }
     if (nodes.size() == 1) {
-      tail[gi] = nodes[0];
+      tail[gi].assign(1, nodes[0]);
     } else if (nodes.size() > 1) {
       cudaGraphNode_t join;
-      e = cudaGraphAddEmptyNode(&join, g, nodes.data(), nodes.size());
+      if (kernel_join[gi]) {
+        cudaKernelNodeParams kp = {};
+        kp.func = const_cast<void*>(graph_root_kernel_entry());
+        kp.gridDim = dim3(1);
+        kp.blockDim = dim3(32);
+        kp.kernelParams = nullptr;
+        e = cudaGraphAddKernelNode(&join, g, nodes.data(), nodes.size(), &kp);
+        if (e == cudaSuccess) entry->n_order_launches++;
+      } else {
+        e = cudaGraphAddEmptyNode(&join, g, nodes.data(), nodes.size());
+      }
       if (e != cudaSuccess) {
         fail(e, "graph join node");
         break;
       }
-      tail[gi] = join;
+      tail[gi].assign(1, join);
     }
   }
   if (rc == HOCCL_OK) {
@@ -283,7 +309,7 @@ hoccl_result_t build_pattern_graph(hoccl_comm* c, const Schedule& S, const void*
   CU_TRY(c, cudaGraphCreate(&g, 0));
   cudaError_t err = cudaSuccess;
   cudaGraphNode_t stage_dep = nullptr;
-  if (c->path == HOCCL_PATH_CE) {   // one empty kernel in front of the first stage's copy chains (see build_graph)
+  if (c->path == HOCCL_PATH_CE && c->order_kernels) {   // one empty kernel in front of the first stage's copy chains (see build_graph)
     cudaKernelNodeParams kp = {};
     kp.func = const_cast<void*>(graph_root_kernel_entry());
     kp.gridDim = dim3(1);
@@ -367,7 +393,17 @@ hoccl_result_t build_pattern_graph(hoccl_comm* c, const Schedule& S, const void*
       stage_dep = tails[0];
     } else if (tails.size() > 1) {
       cudaGraphNode_t join;
-      err = cudaGraphAddEmptyNode(&join, g, tails.data(), tails.size());
+      if (c->path == HOCCL_PATH_CE && c->order_kernels) {   // copy chains wait for copy chains: an empty kernel as the join (see build_graph)
+        cudaKernelNodeParams kp = {};
+        kp.func = const_cast<void*>(graph_root_kernel_entry());
+        kp.gridDim = dim3(1);
+        kp.blockDim = dim3(32);
+        kp.kernelParams = nullptr;
+        err = cudaGraphAddKernelNode(&join, g, tails.data(), tails.size(), &kp);
+        if (err == cudaSuccess) entry->n_order_launches++;
+      } else {
+        err = cudaGraphAddEmptyNode(&join, g, tails.data(), tails.size());
+      }
       if (err == cudaSuccess) stage_dep = join;
     }
   }

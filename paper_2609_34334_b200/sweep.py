@@ -307,11 +307,11 @@ def gradients(args):
     alone, _, _ = gemm_tflops(40)
     print(json.dumps({"workload": g.name, "buckets_total": len(sizes), "bucket_MiB": S >> 20, "last_bucket_MiB": sizes[-1] * 2 >> 20,
                       "gemm_probe": [M, K, N], "gemm_alone_TFLOPs": alone}), flush=True)
-    configs = [("CE_sum8", hb.PATH_CE, 8, 8), ("SM_copy8_sum8", hb.PATH_SM, 8, 8), ("SM_copy32_sum8", hb.PATH_SM, 8, 32),
-               ("SM_copy148_sum148", hb.PATH_SM, 148, 148)]
+    configs = [("CE_sum8", hb.PATH_CE, 8, 8), ("CE_sum8_plain_graphs", hb.PATH_CE, 8, 8), ("SM_copy8_sum8", hb.PATH_SM, 8, 8),
+               ("SM_copy32_sum8", hb.PATH_SM, 8, 32), ("SM_copy148_sum148", hb.PATH_SM, 148, 148)]
     if getattr(args, "budgets", ""):
         # the copy-route path, then the SM-copy path under every CTA budget (SUM budget: the same, at most 8), then the whole GPU
-        configs = [("CE_sum8", hb.PATH_CE, 8, 8)]
+        configs = [("CE_sum8", hb.PATH_CE, 8, 8), ("CE_sum8_plain_graphs", hb.PATH_CE, 8, 8)]
         for b in [int(x) for x in args.budgets.split(",")]:
             configs.append(("SM_copy%d_sum%d" % (b, min(b, 8)), hb.PATH_SM, min(b, 8), b))
         configs.append(("SM_copy148_sum148", hb.PATH_SM, 148, 148))
@@ -324,6 +324,7 @@ def gradients(args):
         comm.set_param("sum_ctas", sc)
         comm.set_param("copy_ctas", cc)
         comm.set_param("ag_direct", 1 if name.endswith("_direct") else 0)
+        comm.set_param("order_kernels", 0 if name.endswith("_plain_graphs") else 1)   # the copy-route graphs without ordering kernels
         for k in range(pool):
             comm.allreduce(send[k], recv[k], per, dtype, stream)
         stream.synchronize()

@@ -16,6 +16,9 @@ class DevBuf:
         self.view = self.raw[GUARD + off:GUARD + off + nbytes]
         if nbytes:
             self.view.fill_(fill)
+        # the fills run on torch's current stream; tests hand these buffers to calls on other (non-blocking) streams, which are
+        # not ordered behind it, so the buffer is made ready here
+        torch.cuda.current_stream().synchronize()
 
     @property
     def ptr(self) -> int:
@@ -28,6 +31,7 @@ class DevBuf:
         b = torch.from_numpy(arr.view(np.uint8).copy())
         assert b.numel() == self.nbytes
         self.view.copy_(b)
+        torch.cuda.current_stream().synchronize()
         return self
 
     def get(self, dtype) -> np.ndarray:

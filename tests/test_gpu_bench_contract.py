@@ -26,7 +26,8 @@ def test_bench_line_has_the_contract_keys():
     assert d["e2e"]["h2d_bytes_per_step"] == 8 * 26214400 and d["e2e"]["value"] < d["value"]
     r = d["roofline"]
     assert r["bound"] == "hbm" and r["unit"] == "GB/s" and abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-9 and r["traffic"] > 0
-    # per step: seven SUM launches plus the empty ordering kernel in front of each of the two graphs' first copies
-    assert d["gpu_launches"] == (7 + 2) * 8
+    # per step: seven SUM launches, and the empty ordering kernels of the two graphs: one in front of each graph's first
+    # copies, one behind each of the seven copy stages of the ring all-gather
+    assert d["gpu_launches"] == (7 + 2 + 7) * 8
     c = d["cpu_baseline"]
     assert c["kind"] == "oracle" and c["cores"] >= 1 and c["value"] > 0

@@ -64,12 +64,14 @@ def test_collectives_through_the_proxy_match_the_oracle(oracle):
         for r in range(R):
             assert same_bits(after[r].cpu().numpy().view(np.uint16), want[r], dtype), (rep, r)
             recv[r].zero_()
+        torch.cuda.synchronize()                       # zero_ ran on torch's current stream, the next repetition runs on st
     assert comm.handshakes() == 3
     assert comm.async_error() == hb.OK
     # all-gather and all-to-all go the same way
     ys = W.rank_inputs("uniform", 92, R, 4096, dtype)
     gs = [torch.from_numpy(y.view(np.int16)).cuda() for y in ys]
     gr = [torch.zeros(R * 4096, dtype=torch.int16, device="cuda") for _ in range(R)]
+    torch.cuda.synchronize()
     comm.allgather(gs, gr, 4096, dtype, st)
     _wait(st)
     cat = np.concatenate(ys)

