@@ -107,6 +107,7 @@ def sweep_sizes(args):
     configs = [("CE", hb.PATH_CE, 8, 8, 0), ("SM8", hb.PATH_SM, 8, 8, 0), ("SMall", hb.PATH_SM, 148, 148, 0),
                ("SM8fused", hb.PATH_SM, 8, 8, 1), ("SMallfused", hb.PATH_SM, 148, 148, 1),
                # all-gather as independent stages (fan-out copy on the SM path); the last one adds the forward comparison variant
+               ("CEplain", hb.PATH_CE, 8, 8, 0),   # copy route, plain graphs: no empty ordering kernels (order_kernels = 0)
                ("CEall", hb.PATH_CE, 148, 8, 0),   # copy route with whole-GPU sums: what the route reaches without the 8-CTA SUM budget
                ("CEdirect", hb.PATH_CE, 8, 8, 0), ("SM8direct", hb.PATH_SM, 8, 8, 0), ("SMalldirect", hb.PATH_SM, 148, 148, 0),
                ("SMallfwddirect", hb.PATH_SM, 148, 148, 0)]
@@ -144,6 +145,7 @@ def sweep_sizes(args):
                         direct = name.endswith("direct")
                         comm.set_param("ag_direct", 1 if direct else 0)
                         comm.set_param("forward", 1 if "fwd" in name else 0)
+                        comm.set_param("order_kernels", 0 if name == "CEplain" else 1)
                         t = time_op(comm, arena, stream)
                         row = {"op": op, "R": R, "dtype": dtype, "S": S, "config": name, "sum_ctas": sc,
                                "copy_ctas": cc if path == hb.PATH_SM else None, "us": t * 1e6, "algbw_GBps": S / t / 1e9,
