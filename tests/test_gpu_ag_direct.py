@@ -218,3 +218,29 @@ def test_config2_bucket_full_size_every_timed_variant(oracle):
                 assert same_bits(recv[r].get(np.uint16), want[r], c.dtype), (path, params, two_calls, r)
                 assert recv[r].guards_intact() and send[r].guards_intact()
         comm.destroy()
+
+
+def test_ordering_kernels_are_counted_and_optional(oracle):
+    """Copy route: the graphs carry empty one-warp kernels in front of their first copies and behind groups of copies that
+    other copies (or the graph's end) wait for; "order_kernels" = 0 builds the plain graphs.  Same bits either way."""
+    R, n, dtype = 8, 8 * 50_000 + 5, "bf16"
+    count = n // R
+    xs = W.rank_inputs("normal", 98, R, n, dtype, 1e-3)
+    want = oracle.ring_allreduce(xs)
+    for order, direct in ((1, 0), (0, 0), (1, 1), (0, 1)):
+        comm = make_comm(R, n, dtype, hb.PATH_CE, order_kernels=order, ag_direct=direct)
+        got = run_allreduce(comm, xs, dtype)
+        assert all(same_bits(got[r], want[r], dtype) for r in range(R)), (order, direct)
+        st = comm.last_stats()
+        # one all-reduce graph: a root in front of the 8 first copies and a join behind each of the 7 all-gather stages
+        # (ring: the next stage waits for it; direct: the stages are separate groups here and each ends the graph)
+        assert st["n_order_launches"] == (1 + 7 if order else 0), (order, direct, st)
+        assert st["n_sum_launches"] == 7 and st["n_move_launches"] == 0 and st["n_moves"] == 112
+        comm.destroy()
+    # the SM path and the stream executor have none
+    for path, params in ((hb.PATH_SM, dict()), (hb.PATH_CE, dict(use_graph=0))):
+        comm = make_comm(R, n, dtype, path, **params)
+        got = run_allreduce(comm, xs, dtype)
+        assert all(same_bits(got[r], want[r], dtype) for r in range(R))
+        assert comm.last_stats()["n_order_launches"] == 0
+        comm.destroy()
