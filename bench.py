@@ -328,7 +328,9 @@ def main():
             "frac_of_8TBps": algorithmic_hbm_bytes_allreduce(S, R) / t_step / 1e9 / NOMINAL_HBM_GBS,
             "frac_of_measured_copy": algorithmic_hbm_bytes_allreduce(S, R) / t_step / 1e9 / peaks["hbm_gbs"],
         },
-        "sms_used": {"sum_ctas": int(rs_stats["max_sum_ctas"]), "moves": "driver copy route (see move_needs_sm)"},
+        "sms_used": {"sum_ctas": int(rs_stats["max_sum_ctas"]), "moves": "driver copy route (see move_needs_sm)",
+                     "ordering_kernels_per_step": int(rs_stats["n_order_launches"] + ag_stats["n_order_launches"]),
+                     "ordering_kernel": "empty, 1 CTA of 32 threads, ~2 us each (orders copy nodes inside the graphs)"},
         "e2e": {"value": e2e_value, "unit": "GB/s", "h2d_bytes_per_step": R * S, "d2h_bytes_per_step": R * S,
                 "ms_per_step": t_e2e_slowest * 1e3, "call": "hoccl_host_allreduce (pinned host buffers; inbound copies, ring and outbound copies pipelined over 8 pieces per chunk)", "steps": k_e2e,
                 "matches_oracle": e2e_ok},
