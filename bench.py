@@ -449,12 +449,15 @@ def small_case(hb, W, torch, np, stream):
     nb = hb.scratch_bytes(R, n, c.dtype)
     scratch = torch.empty(nb + 256, dtype=torch.uint8, device="cuda")
     rows = {}
-    for name, path, ctas, fused in (("CE_sum8", hb.PATH_CE, 8, 0), ("SM_8", hb.PATH_SM, 8, 0), ("SM_148", hb.PATH_SM, 148, 0),
-                                    ("SM_148_one_kernel", hb.PATH_SM, 148, 1)):
+    for name, path, ctas, fused, direct, fwd in (("CE_sum8", hb.PATH_CE, 8, 0, 0, 0), ("CE_sum8_direct_allgather", hb.PATH_CE, 8, 0, 1, 0),
+                                                 ("SM_8", hb.PATH_SM, 8, 0, 0, 0), ("SM_148", hb.PATH_SM, 148, 0, 0, 0),
+                                                 ("SM_148_one_kernel", hb.PATH_SM, 148, 1, 0, 0),
+                                                 ("SM_148_direct_allgather", hb.PATH_SM, 148, 0, 1, 0),
+                                                 ("SM_148_direct_allgather_forward", hb.PATH_SM, 148, 0, 1, 1)):
         cm = hb.Comm(R, 0)
         cm.set_scratch(scratch.data_ptr() + (-scratch.data_ptr()) % 256, nb)
         cm.set_path(path)
-        for key, v in (("sum_ctas", ctas), ("copy_ctas", ctas), ("fused", fused)):
+        for key, v in (("sum_ctas", ctas), ("copy_ctas", ctas), ("fused", fused), ("ag_direct", direct), ("forward", fwd)):
             cm.set_param(key, v)
         for b in range(sets):
             cm.allreduce(send[b], recv[b], n, c.dtype, stream)
@@ -469,8 +472,11 @@ def small_case(hb, W, torch, np, stream):
         stream.synchronize()
         t = e0.elapsed_time(e1) / 1e3 / reps
         S1 = n * 4
+        # algorithmic bytes: the ring's 7 S (R-1); the direct all-gather on the SM path reads a chunk once and stores it R-1
+        # times (5 S (R-1) + S R); no figure for the forward comparison variant
+        moved = None if fwd else (5.0 * S1 * (R - 1) + S1 * R if (direct and path == hb.PATH_SM) else 7.0 * S1 * (R - 1))
         rows[name] = {"us_per_call": t * 1e6, "busbw_GBps": S1 * 2 * (R - 1) / R / t / 1e9,
-                      "hbm_frac_of_8TBps": 7.0 * S1 * (R - 1) / t / 1e9 / NOMINAL_HBM_GBS, "matches_oracle": ok}
+                      "hbm_frac_of_8TBps": None if moved is None else moved / t / 1e9 / NOMINAL_HBM_GBS, "matches_oracle": ok}
         cm.destroy()
     # the oracle on the host cores for the same configuration (a reported baseline, as for the headline workload)
     thr = oracle_ring.max_threads()
