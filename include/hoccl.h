@@ -116,6 +116,9 @@ hoccl_result_t hoccl_comm_destroy(hoccl_comm_t comm);
  * per rank buffer (allreduce convention) with R ranks: per rank one inbox and one partial slot of
  * one ring chunk each, padded.  0 for R == 1. */
 size_t hoccl_scratch_bytes(int R, size_t max_count, hoccl_dtype_t dtype);
+/* The same bound with the "rs_direct" parameter set: per rank R-1 inbox slots of one ring chunk each, padded.  It also covers
+ * every call without that parameter when R >= 3. */
+size_t hoccl_scratch_bytes_direct(int R, size_t max_count, hoccl_dtype_t dtype);
 
 /* Attaches caller-owned device scratch (256-byte aligned).  Reductions need it; all-gather and p2p do
  * not.  Contents are undefined between calls.  Collectives that overlap in time on different streams
@@ -165,6 +168,15 @@ hoccl_result_t hoccl_comm_set_path(hoccl_comm_t comm, hoccl_path_t path);
  *                HOCCL_PATH_CE_HOST: a chunk goes out to the host staging once and comes back R-1 times.
  *                0 = the ring all-gather (default).  2 = automatic: direct where it was measured faster on B200 (always on
  *                HOCCL_PATH_SM and HOCCL_PATH_CE_HOST; on HOCCL_PATH_CE while a ring chunk is at most 64 MiB), ring elsewhere.
+ *  "rs_direct"   1 = the reduce-scatter (alone or as the first half of an all-reduce) runs as the stage decomposition of its
+ *                traffic matrix (paper Sec. 3.4: rank r owes its contribution to chunk d to rank d): R-1 contention-free
+ *                permutation stages r -> r+k that wait for nothing, into R-1 inbox slots of the owner, and then ONE sum
+ *                per rank that adds the R-1 arrived contributions and its own in the ring's order, rounding into the I/O
+ *                dtype after every add (chain_kernel, "sum_ctas" CTAs).  Rank local, the ring's bits; every output byte is
+ *                written once instead of R-1 times: 2 S (R-1) + S (R+1) bytes of traffic instead of 5 S (R-1), and under
+ *                an SM budget, where a sum is bound by the SMs' memory ports, R reads + 1 write per output instead of
+ *                (R-1) x (2 reads + 1 write).  Needs hoccl_scratch_bytes_direct bytes of scratch (R-1 slots per rank
+ *                instead of 2).  "forward" and "fused" do not apply to it.  0 = the ring reduce-scatter (default).
  *  "order_kernels" 1 (default) = on the copy routes the graph executor puts an empty one-warp kernel in front of a graph's
  *                first copies and behind every group of copies that other copies (or the end of the graph) wait for.
  *                Measured on B200: a copy node that waits for earlier stream work or for several copy nodes starts ~4 us
@@ -453,6 +465,14 @@ hoccl_result_t hoccl_flatten_inspect(int kind, hoccl_dtype_t dtype, int ctas, in
 hoccl_result_t hoccl_fanout_inspect(int n, const uint64_t* src, const uint64_t* dst, const uint64_t* len, int ctas, int seg_cap,
                                     int* seg_launch, uint64_t* seg_src, uint64_t* seg_len, int* seg_ndst, uint32_t* seg_head,
                                     uint64_t* seg_nvec, uint64_t* dst_out, int* n_seg, int* n_launch);
+/*
+ * Self-test of the arithmetic: the chain sum of the direct reduce-scatter adds bf16 operands with the native packed add
+ * (add.rn.bf16x2); this call compares it on the device with the reference add of every SUM (binary32 add of the widened
+ * operands, rounded to nearest even into bf16) for ALL 2^32 pairs of bf16 bit patterns.  counts: DEVICE array of two 64-bit
+ * words, zeroed by the caller; after the stream has run it holds {pairs whose results differ, pairs where both results are
+ * NaN with different payloads}.  Both must be 0.
+ */
+hoccl_result_t hoccl_selftest_bf16_add(unsigned long long* counts, hoccl_stream_t stream);
 hoccl_result_t hoccl_kernel_sms(int kind, const void* a, const void* b, void* out, size_t bytes, hoccl_dtype_t dtype, int ctas,
                                 unsigned int* smid_out, hoccl_stream_t stream);
 
@@ -468,7 +488,10 @@ typedef enum { HOCCL_PLAN_ALLREDUCE = 0, HOCCL_PLAN_REDUCE_SCATTER = 1, HOCCL_PL
                HOCCL_PLAN_ALLREDUCE_FWD = 4, HOCCL_PLAN_REDUCE_SCATTER_FWD = 5, /* the "forward" variants */
                HOCCL_PLAN_ALLREDUCE_AGD = 6, HOCCL_PLAN_ALLGATHER_DIRECT = 7,   /* the "ag_direct" variants */
                HOCCL_PLAN_ALLREDUCE_FWD_AGD = 8 /* both */ } hoccl_plan_kind_t;
-typedef enum { HOCCL_OP_MOVE = 0, HOCCL_OP_SUM = 1 } hoccl_plan_op_kind_t;
+/* General form: a base kind (0..3) OR-ed with flags; the numbered variants above are shorthands. */
+typedef enum { HOCCL_PLAN_FLAG_FORWARD = 16, HOCCL_PLAN_FLAG_AG_DIRECT = 32, HOCCL_PLAN_FLAG_RS_DIRECT = 64 /* "rs_direct" */ } hoccl_plan_flag_t;
+/* CHAIN: out = (((s_0 + s_1) + ...) + s_{nsrc-1}) + local, every add rounded into the I/O dtype; s_j at src_off + j * src_stride */
+typedef enum { HOCCL_OP_MOVE = 0, HOCCL_OP_SUM = 1, HOCCL_OP_CHAIN = 2 } hoccl_plan_op_kind_t;
 typedef enum { HOCCL_BUF_SEND = 0, HOCCL_BUF_RECV = 1, HOCCL_BUF_INBOX = 2, HOCCL_BUF_PARTIAL = 3 } hoccl_buf_kind_t;
 
 typedef struct {
@@ -483,6 +506,8 @@ typedef struct {
   uint64_t src_off, dst_off, local_off; /* byte offsets from the start of those buffers (scratch: from the start of the rank's slot) */
   uint64_t bytes;
   int group;     /* ops of one group are issued together (one batched kernel launch or R copies) */
+  int nsrc;      /* CHAIN: number of inbox operands (R-1); 1 otherwise */
+  uint64_t src_stride; /* CHAIN: bytes between consecutive inbox operands (one scratch slot) */
 } hoccl_plan_op_t;
 
 typedef struct hoccl_plan* hoccl_plan_t;
@@ -493,8 +518,12 @@ typedef struct hoccl_plan* hoccl_plan_t;
  * scratch region a piece is placed so that SUM operands share their 16-byte phase.  Free with hoccl_plan_destroy. */
 hoccl_result_t hoccl_plan_build(hoccl_plan_t* plan, int kind, int R, size_t count, hoccl_dtype_t dtype, int in_place,
                                 size_t piece_bytes, int max_pieces, const unsigned char* send_align);
-/* Bytes of one rank's scratch slot (inbox or partial) under this plan; slots of rank r start at r * that. */
+/* Bytes of one rank's scratch slot (inbox or partial) under this plan.  Rank r's inbox is hoccl_plan_inbox_slots slots at
+ * r * slots * slot bytes (1 slot; R-1 for the direct reduce-scatter); the partial slots, one per rank, follow all inboxes. */
 size_t hoccl_plan_slot_bytes(hoccl_plan_t plan);
+int hoccl_plan_inbox_slots(hoccl_plan_t plan);
+/* Scratch bytes a call with this plan needs. */
+size_t hoccl_plan_scratch_bytes(hoccl_plan_t plan);
 void hoccl_plan_destroy(hoccl_plan_t plan);
 int hoccl_plan_num_ops(hoccl_plan_t plan);
 int hoccl_plan_num_groups(hoccl_plan_t plan);

@@ -18,17 +18,18 @@ SUM = 0
 PATH_CE, PATH_SM, PATH_CE_HOST = 0, 1, 2
 PLAN_ALLREDUCE, PLAN_REDUCE_SCATTER, PLAN_ALLGATHER, PLAN_ALLTOALL, PLAN_ALLREDUCE_FWD, PLAN_REDUCE_SCATTER_FWD = range(6)
 PLAN_ALLREDUCE_AGD, PLAN_ALLGATHER_DIRECT, PLAN_ALLREDUCE_FWD_AGD = 6, 7, 8
-OP_MOVE, OP_SUM = 0, 1
+OP_MOVE, OP_SUM, OP_CHAIN = 0, 1, 2
+PLAN_FLAG_FORWARD, PLAN_FLAG_AG_DIRECT, PLAN_FLAG_RS_DIRECT = 16, 32, 64
 BUF_SEND, BUF_RECV, BUF_INBOX, BUF_PARTIAL = 0, 1, 2, 3
 
 DTYPES = {"fp32": FLOAT32, "bf16": BFLOAT16}
 
 EXPORTS = [
-    "hoccl_comm_init", "hoccl_comm_destroy", "hoccl_scratch_bytes", "hoccl_comm_set_scratch", "hoccl_comm_set_staging", "hoccl_comm_set_host_staging",
+    "hoccl_comm_init", "hoccl_comm_destroy", "hoccl_scratch_bytes", "hoccl_scratch_bytes_direct", "hoccl_plan_inbox_slots", "hoccl_plan_scratch_bytes", "hoccl_comm_set_scratch", "hoccl_comm_set_staging", "hoccl_comm_set_host_staging",
     "hoccl_comm_set_path", "hoccl_comm_set_param", "hoccl_comm_get_param", "hoccl_allreduce", "hoccl_reduce_scatter",
     "hoccl_allgather", "hoccl_alltoall", "hoccl_alltoallv", "hoccl_send", "hoccl_recv", "hoccl_comm_pending", "hoccl_comm_async_error", "hoccl_comm_handshakes", "hoccl_selftest_barrier_timeout", "hoccl_host_allreduce", "hoccl_error_string",
     "hoccl_last_cuda_error", "hoccl_last_stats", "hoccl_profile_reset", "hoccl_probe_move_needs_sm", "hoccl_probe_copy_routes", "hoccl_sum_launch", "hoccl_kernel_sms", "hoccl_flatten_inspect", "hoccl_port_probe",
-    "hoccl_copy_launch", "hoccl_fanout_launch", "hoccl_fanout_inspect", "hoccl_plan_build", "hoccl_plan_destroy", "hoccl_plan_num_ops", "hoccl_plan_num_groups",
+    "hoccl_copy_launch", "hoccl_fanout_launch", "hoccl_fanout_inspect", "hoccl_selftest_bf16_add", "hoccl_plan_build", "hoccl_plan_destroy", "hoccl_plan_num_ops", "hoccl_plan_num_groups",
     "hoccl_plan_get_op", "hoccl_plan_group_deps", "hoccl_plan_slot_bytes", "hoccl_allreduce_static",
     "hoccl_sched_build", "hoccl_sched_destroy", "hoccl_sched_num_stages", "hoccl_sched_stage_tau", "hoccl_sched_total_tau",
     "hoccl_sched_lower_bound", "hoccl_sched_matrix", "hoccl_sched_num_flows", "hoccl_sched_get_flow", "hoccl_sched_queue_len",
@@ -60,6 +61,7 @@ class PlanOp(ctypes.Structure):
         ("rank", ctypes.c_int), ("dst_rank", ctypes.c_int), ("chunk", ctypes.c_int), ("src_buf", ctypes.c_int),
         ("dst_buf", ctypes.c_int), ("local_buf", ctypes.c_int), ("src_off", ctypes.c_uint64), ("dst_off", ctypes.c_uint64),
         ("local_off", ctypes.c_uint64), ("bytes", ctypes.c_uint64), ("group", ctypes.c_int),
+        ("nsrc", ctypes.c_int), ("src_stride", ctypes.c_uint64),
     ]
 
 
@@ -97,6 +99,9 @@ def lib() -> ctypes.CDLL:
         "hoccl_comm_init": (i, [vpp, i, i]),
         "hoccl_comm_destroy": (i, [vp]),
         "hoccl_scratch_bytes": (sz, [i, sz, i]),
+        "hoccl_scratch_bytes_direct": (sz, [i, sz, i]),
+        "hoccl_plan_inbox_slots": (i, [vp]),
+        "hoccl_plan_scratch_bytes": (sz, [vp]),
         "hoccl_comm_set_scratch": (i, [vp, vp, sz]),
         "hoccl_comm_set_staging": (i, [vp, vp, sz]),
         "hoccl_comm_set_host_staging": (i, [vp, vp, sz]),
@@ -135,6 +140,7 @@ def lib() -> ctypes.CDLL:
         "hoccl_sum_launch": (i, [vp, vp, vp, sz, i, i, vp]),
         "hoccl_copy_launch": (i, [vp, vp, sz, i, vp]),
         "hoccl_fanout_launch": (i, [vp, vp, i, sz, i, vp]),
+        "hoccl_selftest_bf16_add": (i, [vp, vp]),
         "hoccl_fanout_inspect": (i, [i, vp, vp, vp, i, i, vp, vp, vp, vp, vp, vp, vp, ctypes.POINTER(i), ctypes.POINTER(i)]),
         "hoccl_kernel_sms": (i, [i, vp, vp, vp, sz, i, i, vp, vp]),
         "hoccl_selftest_barrier_timeout": (i, [vp, vp, vp, sz, vp]),
@@ -358,6 +364,11 @@ def scratch_bytes(R: int, max_count: int, dtype) -> int:
     return int(lib().hoccl_scratch_bytes(R, max_count, _dtype(dtype)))
 
 
+def scratch_bytes_direct(R: int, max_count: int, dtype) -> int:
+    """Scratch bound with "rs_direct" set (R-1 inbox slots per rank)."""
+    return int(lib().hoccl_scratch_bytes_direct(R, max_count, _dtype(dtype)))
+
+
 def sum_launch(inbox, local, out, count, dtype, ctas, stream=None) -> int:
     return lib().hoccl_sum_launch(_ptr(inbox), _ptr(local), _ptr(out), count, _dtype(dtype), ctas, _stream(stream))
 
@@ -369,6 +380,11 @@ def copy_launch(src, dst, nbytes, ctas, stream=None) -> int:
 def fanout_launch(src, dsts, nbytes, ctas, stream=None) -> int:
     """hoccl_fanout_launch: every dsts[d] <- src, the source read once.  Returns the result code."""
     return lib().hoccl_fanout_launch(_ptr(src), _ptr_array(dsts), len(dsts), nbytes, ctas, _stream(stream))
+
+
+def selftest_bf16_add(counts, stream=None) -> int:
+    """hoccl_selftest_bf16_add: counts = device array of two zeroed 64-bit words.  Returns the result code."""
+    return lib().hoccl_selftest_bf16_add(_ptr(counts), _stream(stream))
 
 
 def fanout_inspect(moves, ctas: int = 8):
@@ -432,6 +448,8 @@ class Plan:
             raise HocclError(rc, "hoccl_plan_build")
         L = lib()
         self.slot_bytes = int(L.hoccl_plan_slot_bytes(self._h))
+        self.inbox_slots = int(L.hoccl_plan_inbox_slots(self._h))
+        self.scratch_bytes = int(L.hoccl_plan_scratch_bytes(self._h))
         self.ops = []
         for k in range(L.hoccl_plan_num_ops(self._h)):
             op = PlanOp()

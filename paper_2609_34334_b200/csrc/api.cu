@@ -79,6 +79,12 @@ size_t hoccl_scratch_bytes(int R, size_t max_count, hoccl_dtype_t dtype) {
   return 2 * (size_t)R * slot_bytes_for(R, max_count, e);
 }
 
+size_t hoccl_scratch_bytes_direct(int R, size_t max_count, hoccl_dtype_t dtype) {
+  size_t e = dtype_size((int)dtype);
+  if (R <= 1 || e == 0 || max_count == 0) return 0;
+  return (size_t)std::max(2, R - 1) * (size_t)R * slot_bytes_for(R, max_count, e);
+}
+
 hoccl_result_t hoccl_comm_set_scratch(hoccl_comm_t c, void* dev_ptr, size_t bytes) {
   if (!c || ((uintptr_t)dev_ptr & 255)) return HOCCL_ERR_INVALID_ARG;
   c->scratch = dev_ptr;
@@ -127,6 +133,7 @@ static long* param_slot(hoccl_comm* c, const char* key, long* lo, long* hi) {
               {"forward", &c->forward, 0, 1},           {"fused", &c->fused, 0, 1},
               {"ag_direct", &c->ag_direct, 0, 2},
               {"order_kernels", &c->order_kernels, 0, 1},
+              {"rs_direct", &c->rs_direct, 0, 1},
               {"host_pieces", &c->host_pieces, 1, 64}};
   for (auto& r : rows)
     if (std::strcmp(r.name, key) == 0) {
@@ -645,6 +652,11 @@ hoccl_result_t hoccl_flatten_inspect(int kind, hoccl_dtype_t dtype, int ctas, in
   return HOCCL_OK;
 }
 
+hoccl_result_t hoccl_selftest_bf16_add(unsigned long long* counts, hoccl_stream_t stream) {
+  if (!counts) return HOCCL_ERR_INVALID_ARG;
+  return launch_bf16_add_selftest(counts, (cudaStream_t)stream) == cudaSuccess ? HOCCL_OK : HOCCL_ERR_CUDA;
+}
+
 hoccl_result_t hoccl_fanout_inspect(int n, const uint64_t* src, const uint64_t* dst, const uint64_t* len, int ctas, int seg_cap,
                                     int* seg_launch, uint64_t* seg_src, uint64_t* seg_len, int* seg_ndst, uint32_t* seg_head,
                                     uint64_t* seg_nvec, uint64_t* dst_out, int* n_seg, int* n_launch) {
@@ -782,6 +794,8 @@ hoccl_result_t hoccl_plan_build(hoccl_plan_t* plan, int kind, int R, size_t coun
 
 void hoccl_plan_destroy(hoccl_plan_t plan) { delete plan; }
 size_t hoccl_plan_slot_bytes(hoccl_plan_t plan) { return plan ? plan->p.slot_bytes : 0; }
+int hoccl_plan_inbox_slots(hoccl_plan_t plan) { return plan ? plan->p.inbox_slots : 0; }
+size_t hoccl_plan_scratch_bytes(hoccl_plan_t plan) { return plan ? plan->p.scratch_need() : 0; }
 int hoccl_plan_num_ops(hoccl_plan_t plan) { return plan ? (int)plan->p.ops.size() : 0; }
 int hoccl_plan_num_groups(hoccl_plan_t plan) { return plan ? (int)plan->p.groups.size() : 0; }
 
@@ -803,6 +817,8 @@ hoccl_result_t hoccl_plan_get_op(hoccl_plan_t plan, int index, hoccl_plan_op_t* 
   out->local_off = o.local_off;
   out->bytes = o.bytes;
   out->group = o.group;
+  out->nsrc = o.nsrc;
+  out->src_stride = o.src_stride;
   return HOCCL_OK;
 }
 

@@ -35,6 +35,8 @@ struct Seg {
   char* dst;
   uint64_t bytes;
   uint64_t host_off = 0;  // HOCCL_PATH_CE_HOST: where this move bounces in the pinned host staging
+  int nsrc = 1;           // OP_CHAIN: inbox operands at src + j * src_stride
+  uint64_t src_stride = 0;
   bool host_first = true; // HOCCL_PATH_CE_HOST: this move issues the outbound copy into host_off (false: another move of the group did)
 };
 
@@ -85,7 +87,7 @@ struct hoccl_comm {
   int R = 0, device = 0, num_sms = 0;
   hoccl_path_t path = HOCCL_PATH_CE;
   long sum_ctas = 8, copy_ctas = 8, piece_bytes = 4 << 20, max_pieces = 8, lanes = 4, use_graph = 1, profile = 0, p2p_split = 1, ce_sub_bytes = 0,
-       handshake = 0, watchdog_ms = 10000, onepass = 0, forward = 0, fused = 0, host_pieces = 8, ag_direct = 0, order_kernels = 1;
+       handshake = 0, watchdog_ms = 10000, onepass = 0, forward = 0, fused = 0, host_pieces = 8, ag_direct = 0, order_kernels = 1, rs_direct = 0;
   bool piece_bytes_set = false;  // the caller chose a piece size: no automatic choice
   hoccl::Proxy* proxy = nullptr;
   cudaStream_t lane[hoccl::kMaxLanes] = {};
@@ -169,6 +171,7 @@ struct Tally {
 // exec.cu
 void fill_sum_batch(const RGroup& g, size_t first, size_t n, int dtype, size_t elem, SumBatch* b);
 void fill_copy_batch(const RGroup& g, size_t first, size_t n, CopyBatch* b);
+void fill_chain_batch(const RGroup& g, size_t first, size_t n, int dtype, size_t elem, ChainBatch* b);
 // Moves of a group that read the same bytes (same source and length; the direct all-gather on the SM path) become fan-out
 // segments: one read, one store per destination.  Returns false (and leaves *out empty) if no source repeats: the plain
 // copy batches are used then.  bytes_out[i] = HBM bytes of batch i (reads + writes), moves_out[i] = moves it carries.

@@ -36,6 +36,21 @@ __device__ __forceinline__ uint32_t add_bf16x2(uint32_t a, uint32_t b) {
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
   return d;
 }
+// The same add as one instruction.  add.rn.bf16x2 gives the bits of add_bf16x2 for ALL 2^32 operand pairs, NaN payloads
+// included (checked exhaustively on the device: hoccl_selftest_bf16_add); a long chain of adds is issue bound without it.
+__device__ __forceinline__ uint32_t add_bf16x2_native(uint32_t a, uint32_t b) {
+  uint32_t d;
+  asm("add.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
+__device__ __forceinline__ uint4 add_vec_bf16_native(uint4 a, uint4 b) {
+  uint4 r;
+  r.x = add_bf16x2_native(a.x, b.x);
+  r.y = add_bf16x2_native(a.y, b.y);
+  r.z = add_bf16x2_native(a.z, b.z);
+  r.w = add_bf16x2_native(a.w, b.w);
+  return r;
+}
 template <>
 struct Traits<1> {  // bf16
   static constexpr int E = 2;

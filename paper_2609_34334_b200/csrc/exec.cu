@@ -80,13 +80,14 @@ void resolve(hoccl_comm* c, const Plan& P, const Call& call, std::vector<RGroup>
   *host_need = 0;
   const int R = P.R;
   char* inbox0 = (char*)c->scratch;
-  char* partial0 = inbox0 + (size_t)R * P.slot_bytes;
+  const size_t inbox_bytes = (size_t)P.inbox_slots * P.slot_bytes;   // one rank's inbox: 1 slot, or R-1 for the direct reduce-scatter
+  char* partial0 = inbox0 + (size_t)R * inbox_bytes;
   auto addr = [&](int buf, int rank, int chunk, uint64_t off) -> char* {
     (void)chunk;
     switch (buf) {
       case BUF_SEND: return (char*)call.send[rank] + off;
       case BUF_RECV: return (char*)call.recv[rank] + off;
-      case BUF_INBOX: return inbox0 + (size_t)rank * P.slot_bytes + off;
+      case BUF_INBOX: return inbox0 + (size_t)rank * inbox_bytes + off;
       default: return partial0 + (size_t)rank * P.slot_bytes + off;
     }
   };
@@ -111,6 +112,8 @@ void resolve(hoccl_comm* c, const Plan& P, const Call& call, std::vector<RGroup>
         s.src = addr(op.src_buf, op.rank, op.chunk, op.src_off);
         s.local = addr(op.local_buf, op.rank, op.chunk, op.local_off);
         s.dst = addr(op.dst_buf, op.dst_rank, op.chunk, op.dst_off);  // dst_rank == rank except in the forward variant
+        s.nsrc = op.nsrc;
+        s.src_stride = op.src_stride;
       }
       if (op.kind == OP_MOVE && c->path == HOCCL_PATH_CE_HOST) {
         s.host_off = *host_need;
@@ -167,6 +170,14 @@ void fill_sum_batch(const RGroup& g, size_t first, size_t n, int dtype, size_t e
   for (size_t i = 0; i < n; i++) {
     const Seg& s = g.segs[first + i];
     b->seg[i] = SumSeg{s.src, s.local, s.dst, (unsigned long long)(s.bytes / elem)};
+  }
+}
+void fill_chain_batch(const RGroup& g, size_t first, size_t n, int dtype, size_t elem, ChainBatch* b) {
+  b->nseg = (int)n;
+  b->dtype = dtype;
+  for (size_t i = 0; i < n; i++) {
+    const Seg& s = g.segs[first + i];
+    b->seg[i] = ChainSeg{s.src, s.local, s.dst, (unsigned long long)(s.bytes / elem), (unsigned long long)s.src_stride, s.nsrc, 0};
   }
 }
 void fill_copy_batch(const RGroup& g, size_t first, size_t n, CopyBatch* b) {
@@ -256,7 +267,7 @@ hoccl_result_t run_streams(hoccl_comm* c, const Plan& P, const std::vector<RGrou
   for (size_t g = 0; g < groups.size(); g++) {
     const RGroup& rg = groups[g];
     cudaStream_t s;
-    if (rg.kind == OP_SUM) {
+    if (rg.kind != OP_MOVE) {
       s = c->sum_stream;
       char u = sum_used ? 1 : 0;
       CU_TRY(c, touch(s, &u));
@@ -270,7 +281,15 @@ hoccl_result_t run_streams(hoccl_comm* c, const Plan& P, const std::vector<RGrou
     for (int d : rg.deps)
       if (where[d] != s) CU_TRY(c, cudaStreamWaitEvent(s, done[d], 0));
     // chain_dep needs no event here: every SUM is on the one sum stream
-    if (rg.kind == OP_SUM) {
+    if (rg.kind == OP_CHAIN) {
+      for (size_t first = 0; first < rg.segs.size(); first += kMaxSegs) {
+        size_t n = std::min<size_t>(kMaxSegs, rg.segs.size() - first);
+        ChainBatch b;
+        fill_chain_batch(rg, first, n, P.dtype, P.elem, &b);
+        CU_TRY(c, launch_chain(b, (int)c->sum_ctas, s));
+        tally->sum_launches++;
+      }
+    } else if (rg.kind == OP_SUM) {
       for (size_t first = 0; first < rg.segs.size(); first += kMaxSegs) {
         size_t n = std::min<size_t>(kMaxSegs, rg.segs.size() - first);
         SumBatch b;
@@ -370,6 +389,7 @@ std::vector<uint64_t> make_key(hoccl_comm* c, const Call& call) {
   k.push_back((uint64_t)c->forward);
   k.push_back((uint64_t)c->ag_direct);
   k.push_back((uint64_t)c->order_kernels);
+  k.push_back((uint64_t)c->rs_direct);
   k.push_back((uint64_t)(c->fused && c->path == HOCCL_PATH_SM && !c->handshake));
   k.push_back((uint64_t)(uintptr_t)c->scratch);
   k.push_back((uint64_t)c->scratch_bytes);
@@ -512,7 +532,8 @@ hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
   if (dtype_size(call->dtype) == 0) return HOCCL_ERR_UNSUPPORTED;
   if (!call->send || !call->recv) return HOCCL_ERR_INVALID_ARG;
   const bool onepass_case = c->onepass && !c->handshake && (call->kind == PLAN_ALLREDUCE || call->kind == PLAN_REDUCE_SCATTER);
-  const bool fused = c->fused && c->path == HOCCL_PATH_SM && !c->handshake && !onepass_case && !call->h_send;
+  const bool direct_rs = c->rs_direct && (call->kind == PLAN_ALLREDUCE || call->kind == PLAN_REDUCE_SCATTER);
+  const bool fused = c->fused && c->path == HOCCL_PATH_SM && !c->handshake && !onepass_case && !call->h_send && !direct_rs;   // the ring kernel has no chain phase
   const bool graphs = (c->use_graph || c->handshake || fused) && !onepass_case;
   std::vector<uint64_t> key;
   if (graphs && call->count != 0) {
@@ -579,6 +600,8 @@ hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
   }
   if (direct && call->kind == PLAN_ALLREDUCE) plan_kind = c->forward ? PLAN_ALLREDUCE_FWD_AGD : PLAN_ALLREDUCE_AGD;
   if (direct && call->kind == PLAN_ALLGATHER) plan_kind = PLAN_ALLGATHER_DIRECT;
+  if (c->rs_direct && (call->kind == PLAN_ALLREDUCE || call->kind == PLAN_REDUCE_SCATTER))
+    plan_kind = call->kind | PLAN_FLAG_RS_DIRECT | (direct ? PLAN_FLAG_AG_DIRECT : 0);
   // Piece size: the caller's if set.  Otherwise: on the SM path under CTA budgets a reduction is cut into at least two
   // pieces (the copy kernel of one piece then overlaps the sum kernel of the other: measured 1.6x on a 3 MiB chunk with
   // 8 + 8 CTAs) of at most 4 MiB.  That does not pay with driver copies (they take the whole GPU and never overlap a sum:
@@ -609,7 +632,7 @@ hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
   if (!build_plan(&P, plan_kind, c->R, call->count, call->dtype, call->in_place, piece_bytes, max_pieces, align))
     return HOCCL_ERR_INVALID_ARG;
   if (P.slot_bytes) {
-    size_t need = 2 * (size_t)c->R * P.slot_bytes;
+    size_t need = P.scratch_need();
     if (!c->scratch || c->scratch_bytes < need) return HOCCL_ERR_SCRATCH;
     // scratch must not overlap any rank buffer
     for (int r = 0; r < c->R; r++)

@@ -116,16 +116,28 @@ hoccl_result_t build_graph(hoccl_comm* c, const Plan& P, const std::vector<RGrou
       }
       deps.push_back(root);
     }
-    if (rg.kind == OP_SUM) {
+    if (rg.kind == OP_SUM || rg.kind == OP_CHAIN) {
       for (size_t first = 0; first < rg.segs.size() && e == cudaSuccess; first += kMaxSegs) {
         size_t n = std::min<size_t>(kMaxSegs, rg.segs.size() - first);
         SumBatch b;
-        fill_sum_batch(rg, first, n, P.dtype, P.elem, &b);
-        prepare_sum_batch(&b, (int)c->sum_ctas);
-        void* args[] = {&b};
+        ChainBatch cb;
+        void* args[1];
         cudaKernelNodeParams kp = {};
         int sum_threads = 0;
-        kp.func = const_cast<void*>(sum_kernel_entry(P.dtype, (int)c->sum_ctas, &sum_threads));
+        double bytes = 0;
+        if (rg.kind == OP_SUM) {
+          fill_sum_batch(rg, first, n, P.dtype, P.elem, &b);
+          prepare_sum_batch(&b, (int)c->sum_ctas);
+          args[0] = &b;
+          kp.func = const_cast<void*>(sum_kernel_entry(P.dtype, (int)c->sum_ctas, &sum_threads));
+          for (size_t i = 0; i < n; i++) bytes += 3.0 * (double)rg.segs[first + i].bytes;
+        } else {
+          fill_chain_batch(rg, first, n, P.dtype, P.elem, &cb);
+          prepare_chain_batch(&cb, (int)c->sum_ctas);
+          args[0] = &cb;
+          kp.func = const_cast<void*>(chain_kernel_entry(P.dtype, &sum_threads));
+          for (size_t i = 0; i < n; i++) bytes += (2.0 + (double)rg.segs[first + i].nsrc) * (double)rg.segs[first + i].bytes;
+        }
         kp.gridDim = dim3((unsigned)c->sum_ctas);
         kp.blockDim = dim3((unsigned)sum_threads);
         kp.kernelParams = args;
@@ -137,8 +149,6 @@ hoccl_result_t build_graph(hoccl_comm* c, const Plan& P, const std::vector<RGrou
           if ((e = cudaEventCreate(&pe.first)) != cudaSuccess) break;
           if ((e = cudaEventCreate(&pe.second)) != cudaSuccess) break;
           entry->prof_events.push_back(pe);
-          double bytes = 0;
-          for (size_t i = 0; i < n; i++) bytes += 3.0 * (double)rg.segs[first + i].bytes;
           entry->prof_bytes.push_back(bytes);
           if ((e = cudaGraphAddEventRecordNode(&start_rec, g, d2.data(), d2.size(), pe.first)) != cudaSuccess) break;
           d2.assign(1, start_rec);

@@ -146,6 +146,79 @@ __global__ void __launch_bounds__(THREADS, 1) copy_kernel(const __grid_constant_
   }
 }
 
+// Chain sum of the direct reduce-scatter: per element nsrc inbox operands and the local one, added in the ring's order with a
+// rounding into the I/O dtype after every add.  One 16-byte vector per thread and tile; the operands are loaded in batches of
+// up to 8 before they are added, so up to 8 x 16 KiB are in flight per CTA.  Store bound under a CTA budget like every kernel
+// here, but it writes each output byte once instead of R-1 times, which is the point of the direct form.
+template <int DT, int THREADS>
+__global__ void __launch_bounds__(THREADS, 1) chain_kernel(const __grid_constant__ ChainBatch batch) {
+  using T = Traits<DT>;
+  const Flat& f = batch.flat;
+  const int nseg = batch.nseg;
+  if (batch.smid_out != nullptr && threadIdx.x == 0) {
+    unsigned id;
+    asm volatile("mov.u32 %0, %%smid;" : "=r"(id));
+    batch.smid_out[blockIdx.x] = id;
+  }
+  const unsigned long long total = (unsigned long long)gridDim.x * blockDim.x;
+  const unsigned long long gt = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
+  {
+    const unsigned long long T_all = f.tpre[nseg];
+    int k = 0;
+    for (unsigned long long t = blockIdx.x; t < T_all; t += gridDim.x) {
+      while (t >= f.tpre[k + 1]) k++;
+      const unsigned long long v = (t - f.tpre[k]) * blockDim.x + threadIdx.x;   // vector of segment k
+      if (v >= f.nvec[k]) continue;
+      const ChainSeg& sg = batch.seg[k];
+      const size_t off = (size_t)f.head[k] * T::E + (size_t)v * 16;
+      const char* src = static_cast<const char*>(sg.first) + off;
+      const int n_ops = sg.nsrc + 1;   // operand j < nsrc: inbox slot j; operand nsrc: the local contribution
+      uint4 acc;
+      for (int j0 = 0; j0 < n_ops; j0 += 8) {
+        uint4 buf[8];
+#pragma unroll
+        for (int j = 0; j < 8; j++) {
+          const int q = j0 + j;
+          if (q < sg.nsrc) buf[j] = __ldcs(reinterpret_cast<const uint4*>(src + (size_t)q * sg.stride));
+          else if (q == sg.nsrc) buf[j] = __ldcs(reinterpret_cast<const uint4*>(static_cast<const char*>(sg.local) + off));
+        }
+#pragma unroll
+        for (int j = 0; j < 8; j++) {
+          const int q = j0 + j;
+          if (q < n_ops) acc = (q == 0) ? buf[j] : (DT == 1 ? add_vec_bf16_native(acc, buf[j]) : T::add_vec(acc, buf[j]));
+        }
+      }
+      *reinterpret_cast<uint4*>(static_cast<char*>(sg.out) + off) = acc;
+    }
+  }
+  // element-wise items: heads, tails and segments without a common 16-byte phase
+  {
+    const unsigned long long S = f.spre[nseg];
+    int k = 0;
+    for (unsigned long long j = gt; j < S; j += total) {
+      while (j >= f.spre[k + 1]) k++;
+      unsigned long long i = j - f.spre[k];
+      if (i >= f.head[k]) i += f.nvec[k] * T::VE;
+      const ChainSeg& sg = batch.seg[k];
+      if (DT == 0) {
+        float acc = static_cast<const float*>(sg.first)[i];
+        for (int q = 1; q < sg.nsrc; q++)
+          acc = __fadd_rn(acc, reinterpret_cast<const float*>(static_cast<const char*>(sg.first) + (size_t)q * sg.stride)[i]);
+        static_cast<float*>(sg.out)[i] = __fadd_rn(acc, static_cast<const float*>(sg.local)[i]);
+      } else {
+        unsigned short acc = static_cast<const unsigned short*>(sg.first)[i];
+        for (int q = 1; q <= sg.nsrc; q++) {
+          const unsigned short b = q < sg.nsrc ? reinterpret_cast<const unsigned short*>(static_cast<const char*>(sg.first) + (size_t)q * sg.stride)[i]
+                                               : static_cast<const unsigned short*>(sg.local)[i];
+          const float s2 = __fadd_rn(__uint_as_float((uint32_t)acc << 16), __uint_as_float((uint32_t)b << 16));
+          acc = __bfloat16_as_ushort(__float2bfloat16_rn(s2));
+        }
+        static_cast<unsigned short*>(sg.out)[i] = acc;
+      }
+    }
+  }
+}
+
 // Fan-out copy: the tile walk of copy_kernel, but a tile that was loaded once is stored to every destination of its segment.
 template <int U, int THREADS>
 __global__ void __launch_bounds__(THREADS, 1) fan_kernel(const __grid_constant__ FanBatch batch) {
@@ -326,6 +399,27 @@ __global__ void __launch_bounds__(1024, 1) port_probe_kernel(uint4* buf, unsigne
   if (MODE == 0 && (acc.x ^ acc.y ^ acc.z ^ acc.w) == 0x9e3779b9u) *sink = 1;   // keeps the loads alive
 }
 
+// Self-test: add.rn.bf16x2 against the reference add (binary32 add of the widened operands, rounded to nearest even into
+// bf16) for every pair of bf16 bit patterns.  Block a handles all b; counts[0] = value mismatches, counts[1] = pairs where
+// both are NaN with different payloads.
+__global__ void bf16_add_selftest_kernel(unsigned long long* counts) {
+  const uint32_t a = blockIdx.x;
+  unsigned long long nb = 0, np = 0;
+  for (uint32_t b = threadIdx.x * 2; b < 65536; b += blockDim.x * 2) {
+    const uint32_t A = a | (a << 16), B = b | ((b + 1) << 16);
+    const uint32_t r = add_bf16x2(A, B), h = add_bf16x2_native(A, B);
+    for (int l = 0; l < 2; l++) {
+      const uint32_t rr = (r >> (16 * l)) & 0xffffu, hh = (h >> (16 * l)) & 0xffffu;
+      if (rr != hh) {
+        if ((rr & 0x7fffu) > 0x7f80u && (hh & 0x7fffu) > 0x7f80u) np++;
+        else nb++;
+      }
+    }
+  }
+  if (nb) atomicAdd(&counts[0], nb);
+  if (np) atomicAdd(&counts[1], np);
+}
+
 // Does nothing: a graph node that only orders (see build_graph).
 __global__ void graph_root_kernel() {}
 
@@ -396,6 +490,29 @@ void prepare_copy_batch(CopyBatch* b, int ctas) {
     split_segment(s.bytes, ms, ms == md, 1, 16, &head[k], &nvec[k], &nscalar[k]);
   }
   fill_flat(&b->flat, b->nseg, tile_v, head, nvec, nscalar);
+}
+
+void prepare_chain_batch(ChainBatch* b, int ctas) {
+  (void)ctas;
+  const int E = b->dtype == 0 ? 4 : 2, VE = 16 / E;
+  const unsigned long long tile_v = 1024;   // one vector per thread and tile
+  unsigned head[kMaxSegs];
+  unsigned long long nvec[kMaxSegs], nscalar[kMaxSegs];
+  for (int k = 0; k < b->nseg; k++) {
+    const ChainSeg& s = b->seg[k];
+    const unsigned ma = (unsigned)((uintptr_t)s.first & 15), mb = (unsigned)((uintptr_t)s.local & 15), mo = (unsigned)((uintptr_t)s.out & 15);
+    split_segment(s.n, ma, ma == mb && mb == mo && (s.stride & 15) == 0, E, VE, &head[k], &nvec[k], &nscalar[k]);
+  }
+  fill_flat(&b->flat, b->nseg, tile_v, head, nvec, nscalar);
+}
+
+cudaError_t launch_chain(const ChainBatch& batch, int ctas, cudaStream_t stream) {
+  if (batch.nseg <= 0) return cudaSuccess;
+  ChainBatch b = batch;
+  prepare_chain_batch(&b, ctas);
+  if (b.dtype == 0) chain_kernel<0, 1024><<<ctas, 1024, 0, stream>>>(b);
+  else chain_kernel<1, 1024><<<ctas, 1024, 0, stream>>>(b);
+  return cudaGetLastError();
 }
 
 void prepare_fan_batch(FanBatch* b, int ctas) {
@@ -473,6 +590,14 @@ const void* copy_kernel_entry(int ctas, int* threads) {
   *threads = wide_copy_grid(ctas) ? 512 : 1024;
   return wide_copy_grid(ctas) ? reinterpret_cast<const void*>(&copy_kernel<4, 512>) : reinterpret_cast<const void*>(&copy_kernel<8, 1024>);
 }
+cudaError_t launch_bf16_add_selftest(unsigned long long* counts, cudaStream_t stream) {
+  bf16_add_selftest_kernel<<<65536, 256, 0, stream>>>(counts);
+  return cudaGetLastError();
+}
+const void* chain_kernel_entry(int dtype, int* threads) {
+  *threads = 1024;
+  return dtype == 0 ? reinterpret_cast<const void*>(&chain_kernel<0, 1024>) : reinterpret_cast<const void*>(&chain_kernel<1, 1024>);
+}
 const void* graph_root_kernel_entry() { return reinterpret_cast<const void*>(&graph_root_kernel); }
 const void* fan_kernel_entry(int ctas, int* threads) {
   *threads = wide_copy_grid(ctas) ? 512 : 1024;
@@ -488,7 +613,8 @@ cudaError_t preload_kernels() {
                        reinterpret_cast<const void*>(&occupy_kernel),           reinterpret_cast<const void*>(&onepass_kernel<0, 512>),
                        reinterpret_cast<const void*>(&onepass_kernel<1, 512>),  reinterpret_cast<const void*>(&onepass_kernel<0, 1024>),
                        reinterpret_cast<const void*>(&onepass_kernel<1, 1024>), reinterpret_cast<const void*>(&fan_kernel<4, 512>),
-                       reinterpret_cast<const void*>(&fan_kernel<8, 1024>), reinterpret_cast<const void*>(&graph_root_kernel)};
+                       reinterpret_cast<const void*>(&fan_kernel<8, 1024>), reinterpret_cast<const void*>(&graph_root_kernel),
+                       reinterpret_cast<const void*>(&chain_kernel<0, 1024>), reinterpret_cast<const void*>(&chain_kernel<1, 1024>)};
   for (const void* f : fns) {
     cudaFuncAttributes a;
     cudaError_t e = cudaFuncGetAttributes(&a, f);

@@ -35,6 +35,27 @@ struct SumBatch {
   unsigned int* smid_out = nullptr;  // diagnostics: if set, CTA b stores the id of the SM it runs on to smid_out[b]
 };
 
+// One chain segment (direct reduce-scatter): out[i] = (((s_0[i] + s_1[i]) + ...) + s_{nsrc-1}[i]) + local[i], every add one
+// binary32 add rounded into the I/O dtype: the ring's order and rounding for one chunk, done by its owner in one pass.
+// s_j = first + j * stride bytes: the owner's inbox slots, filled by the R-1 direct moves.
+struct ChainSeg {
+  const void* first;
+  const void* local;
+  void* out;
+  unsigned long long n;       // elements
+  unsigned long long stride;  // bytes, a multiple of 16
+  int nsrc;                   // 1..kMaxChainSrcs
+  int pad;
+};
+constexpr int kMaxChainSrcs = 63;
+struct ChainBatch {
+  int nseg;
+  int dtype;
+  ChainSeg seg[kMaxSegs];
+  Flat flat;  // filled by prepare_chain_batch (launch_chain does it itself)
+  unsigned int* smid_out = nullptr;
+};
+
 // One copy segment: dst[0..bytes) <- src[0..bytes).
 struct CopySeg {
   const void* src;
@@ -131,6 +152,11 @@ void prepare_ring_phase(RingSeg* seg, int nseg, int kind, int dtype, int threads
 // Enqueue helpers (return the CUDA error of the launch).
 cudaError_t launch_sum(const SumBatch& batch, int ctas, cudaStream_t stream);
 cudaError_t launch_copy(const CopyBatch& batch, int ctas, cudaStream_t stream);
+cudaError_t launch_chain(const ChainBatch& batch, int ctas, cudaStream_t stream);
+void prepare_chain_batch(ChainBatch* batch, int ctas);
+const void* chain_kernel_entry(int dtype, int* threads);
+// counts: two device words, zeroed by the caller; see bf16_add_selftest_kernel
+cudaError_t launch_bf16_add_selftest(unsigned long long* counts, cudaStream_t stream);
 cudaError_t launch_fan(const FanBatch& batch, int ctas, cudaStream_t stream);
 void prepare_fan_batch(FanBatch* batch, int ctas);
 const void* fan_kernel_entry(int ctas, int* threads);

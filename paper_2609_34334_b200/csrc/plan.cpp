@@ -83,13 +83,25 @@ void piece_span(const Plan& P, size_t len_bytes, int p, size_t* off, size_t* len
 bool build_plan(Plan* plan, int kind, int R, size_t count, int dtype, bool in_place, size_t piece_bytes, int max_pieces,
                 const unsigned char* send_align) {
   size_t e = dtype_size(dtype);
-  if (!plan || R < 1 || e == 0 || kind < PLAN_ALLREDUCE || kind > PLAN_ALLREDUCE_FWD_AGD) return false;
-  const bool forward = (kind == PLAN_ALLREDUCE_FWD || kind == PLAN_REDUCE_SCATTER_FWD || kind == PLAN_ALLREDUCE_FWD_AGD);
-  const bool ag_direct = (kind == PLAN_ALLREDUCE_AGD || kind == PLAN_ALLGATHER_DIRECT || kind == PLAN_ALLREDUCE_FWD_AGD);
-  if (kind == PLAN_ALLREDUCE_AGD || kind == PLAN_ALLREDUCE_FWD_AGD) kind = PLAN_ALLREDUCE;
-  if (kind == PLAN_ALLGATHER_DIRECT) kind = PLAN_ALLGATHER;
-  if (kind == PLAN_ALLREDUCE_FWD) kind = PLAN_ALLREDUCE;
-  if (kind == PLAN_REDUCE_SCATTER_FWD) kind = PLAN_REDUCE_SCATTER;
+  if (!plan || R < 1 || e == 0 || kind < 0) return false;
+  int flags = 0;
+  if (kind >= 16) {
+    flags = kind & ~15;
+    kind &= 15;
+    if (kind > PLAN_ALLTOALL || (flags & ~(PLAN_FLAG_FORWARD | PLAN_FLAG_AG_DIRECT | PLAN_FLAG_RS_DIRECT))) return false;
+  } else {
+    if (kind > PLAN_ALLREDUCE_FWD_AGD) return false;
+    if (kind == PLAN_ALLREDUCE_FWD || kind == PLAN_REDUCE_SCATTER_FWD || kind == PLAN_ALLREDUCE_FWD_AGD) flags |= PLAN_FLAG_FORWARD;
+    if (kind == PLAN_ALLREDUCE_AGD || kind == PLAN_ALLGATHER_DIRECT || kind == PLAN_ALLREDUCE_FWD_AGD) flags |= PLAN_FLAG_AG_DIRECT;
+    if (kind == PLAN_ALLREDUCE_FWD || kind == PLAN_ALLREDUCE_AGD || kind == PLAN_ALLREDUCE_FWD_AGD) kind = PLAN_ALLREDUCE;
+    if (kind == PLAN_REDUCE_SCATTER_FWD) kind = PLAN_REDUCE_SCATTER;
+    if (kind == PLAN_ALLGATHER_DIRECT) kind = PLAN_ALLGATHER;
+  }
+  const bool reduces = (kind == PLAN_ALLREDUCE || kind == PLAN_REDUCE_SCATTER);
+  const bool gathers = (kind == PLAN_ALLREDUCE || kind == PLAN_ALLGATHER);
+  const bool rs_direct = reduces && (flags & PLAN_FLAG_RS_DIRECT) && R > 1;
+  const bool forward = reduces && (flags & PLAN_FLAG_FORWARD) && !rs_direct;   // the direct form has no per-step sums to forward
+  const bool ag_direct = gathers && (flags & PLAN_FLAG_AG_DIRECT);
   if (kind == PLAN_ALLTOALL && in_place) return false;  // an in-place exchange would need a staging copy of every block
   if (max_pieces < 1) max_pieces = 1;
   if (piece_bytes < 1024) piece_bytes = 1024;
@@ -98,6 +110,9 @@ bool build_plan(Plan* plan, int kind, int R, size_t count, int dtype, bool in_pl
   P.kind = kind;
   P.forward = forward;
   P.ag_direct = ag_direct;
+  P.rs_direct = rs_direct;
+  P.inbox_slots = rs_direct ? R - 1 : 1;
+  P.uses_partial = !rs_direct;
   P.R = R;
   P.dtype = dtype;
   P.count = count;
@@ -176,7 +191,44 @@ bool build_plan(Plan* plan, int kind, int R, size_t count, int dtype, bool in_pl
   std::vector<int> final_sum(np_i, -1);  // SUM group of step R-2, per piece
   int prev_sum_group = -1;
 
-  if (kind != PLAN_ALLGATHER) {
+  if (rs_direct) {
+    // ---- direct MOVE(k, r, p): rank r sends its contribution to chunk d = r + k to rank d, k = 1..R-1 (stage k is the
+    // contention-free permutation r -> r+k).  Rank d keeps source (d+1+j) in inbox slot j, the order in which the ring
+    // would have added them.  All moves of a piece form one group: none waits for anything.
+    // ---- CHAIN(d, p): out = (((s_0 + s_1) + ...) + s_{R-2}) + own contribution, one pass, rounded after every add.
+    for (int p = 0; p < np_i; p++) {
+      int gm = B.begin_group(OP_MOVE, PHASE_RS, 0, p);
+      for (int k = 1; k < R; k++)
+        for (int r = 0; r < R; r++) {
+          int d = (r + k) % R;
+          size_t lo, hi, off, len;
+          P.chunk_range(d, &lo, &hi);
+          piece_span(P, (hi - lo) * e, p, &off, &len);
+          PlanOp op{OP_MOVE, PHASE_RS, k - 1, p, r, d, d, BUF_SEND, BUF_INBOX, -1, lo * e + off,
+                    (uint64_t)(R - 1 - k) * P.slot_bytes + slot_off(d, d, p), 0, len, 0};
+          B.add(op);
+        }
+      gm = B.end_group();
+      int gs = B.begin_group(OP_CHAIN, PHASE_RS, R - 2, p);
+      for (int d = 0; d < R; d++) {
+        size_t lo, hi, off, len;
+        P.chunk_range(d, &lo, &hi);
+        piece_span(P, (hi - lo) * e, p, &off, &len);
+        PlanOp op{OP_CHAIN, PHASE_RS, R - 2, p, d, d, d, BUF_INBOX, BUF_RECV, BUF_SEND, slot_off(d, d, p),
+                  (kind == PLAN_ALLREDUCE ? lo * e : 0) + off, lo * e + off, len, 0};
+        op.nsrc = R - 1;
+        op.src_stride = P.slot_bytes;
+        B.add(op);
+      }
+      gs = B.end_group();
+      if (gs >= 0) {
+        if (gm >= 0) P.groups[gs].deps.push_back(gm);
+        P.groups[gs].chain_dep = prev_sum_group;
+        prev_sum_group = gs;
+        final_sum[p] = gs;
+      }
+    }
+  } else if (kind != PLAN_ALLGATHER) {
     for (int s = 0; s <= R - 2; s++) {
       for (int p = 0; p < np_i; p++) {
         // ---- MOVE(s, r, p): chunk c = (r-1-s) mod R leaves rank r for the inbox of rank r+1.

@@ -21,7 +21,15 @@ enum PlanKind { PLAN_ALLREDUCE = 0, PLAN_REDUCE_SCATTER = 1, PLAN_ALLGATHER = 2,
                 // direct all-gather: the all-gather's traffic matrix (every rank sends its chunk to every other rank) cut into
                 // the R-1 permutation stages r -> r+k (the stage decomposition of Sec. 3.4) instead of R-1 dependent ring hops
                 PLAN_ALLREDUCE_AGD = 6, PLAN_ALLGATHER_DIRECT = 7, PLAN_ALLREDUCE_FWD_AGD = 8 /* both variants */ };
-enum OpKind { OP_MOVE = 0, OP_SUM = 1 };
+// General form of a variant: base kind (0..3) | flags.  The numbered variants above are shorthands for some combinations.
+enum PlanFlag { PLAN_FLAG_FORWARD = 16, PLAN_FLAG_AG_DIRECT = 32,
+                // direct reduce-scatter: the reduce-scatter's traffic matrix (rank r owes chunk d to rank d) cut into the R-1
+                // permutation stages r -> r+k (Sec. 3.4); rank d keeps the R-1 contributions in R-1 inbox slots and sums them
+                // in the ring's order in one pass (OP_CHAIN): same bits, 2 S (R-1) + S (R+1) instead of 5 S (R-1) bytes
+                PLAN_FLAG_RS_DIRECT = 64 };
+enum OpKind { OP_MOVE = 0, OP_SUM = 1,
+              // out = (((s_0 + s_1) + ...) + s_{nsrc-1}) + local, rounded to the I/O dtype after every add; s_j at src_off + j * src_stride
+              OP_CHAIN = 2 };
 enum BufKind { BUF_SEND = 0, BUF_RECV = 1, BUF_INBOX = 2, BUF_PARTIAL = 3 };
 enum Phase { PHASE_RS = 0, PHASE_AG = 1, PHASE_OWN = 2, PHASE_A2A = 3 };
 
@@ -33,6 +41,8 @@ struct PlanOp {
   uint64_t src_off, dst_off, local_off;  // bytes from the start of the buffer (scratch: from the start of the rank's slot)
   uint64_t bytes;
   int group;
+  int nsrc = 1;             // OP_CHAIN: number of inbox operands (R-1)
+  uint64_t src_stride = 0;  // OP_CHAIN: bytes between consecutive inbox operands (one scratch slot)
 };
 
 struct PlanGroup {
@@ -47,6 +57,10 @@ struct Plan {
   int kind = 0, R = 0, dtype = 0;  // kind: the base collective (forward variants are folded into it, see `forward`)
   bool forward = false;            // fused sum-and-forward variant (not rank local)
   bool ag_direct = false;          // all-gather phase as R-1 independent permutation stages (rank local: rank r sends its own chunk)
+  bool rs_direct = false;          // reduce-scatter phase as R-1 independent permutation stages + one chain sum per rank
+  int inbox_slots = 1;             // scratch slots of one rank's inbox (rs_direct: R-1); the partial slots follow all inboxes
+  bool uses_partial = true;        // false: no partial slots in the scratch (rs_direct)
+  size_t scratch_need() const { return (size_t)R * slot_bytes * ((size_t)inbox_slots + (uses_partial ? 1 : 0)); }
   size_t count = 0;
   bool in_place = false;
   size_t elem = 4;

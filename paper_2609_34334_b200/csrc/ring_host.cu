@@ -75,7 +75,10 @@ hoccl_result_t build_ring(hoccl_comm* c, const Plan& P, const std::vector<RGroup
   if (rc != HOCCL_OK) return rc;
   size_t max_phase_bytes = 0;
   bool has_sum = false;
-  for (const RGroup& g : groups) has_sum = has_sum || g.kind == OP_SUM;
+  for (const RGroup& g : groups) {
+    if (g.kind == OP_CHAIN) return HOCCL_ERR_UNSUPPORTED;   // the ring kernel walks ring steps only
+    has_sum = has_sum || g.kind == OP_SUM;
+  }
   // CTA budget: never more than either budget of the SM path; never more CTAs than the largest phase has tiles for
   // (a barrier costs more the more CTAs take part); never more than can be resident together.
   long budget = has_sum ? std::min(c->sum_ctas, c->copy_ctas) : c->copy_ctas;

@@ -52,6 +52,7 @@ case = st.fixed_dictionaries({
     "flavour": st.sampled_from(["normal", "wide", "special"]),
     "seed": st.integers(0, 2 ** 31 - 1),
     "ag_direct": st.integers(0, 2),
+    "rs_direct": st.integers(0, 1),
 })
 
 
@@ -67,7 +68,7 @@ def test_random_cases_match_the_oracle(oracle, c):
     total = count if op == "allreduce" else count * R
     offs = [o * e for o in c["offs"][:R]]
     params = dict(use_graph=c["use_graph"], piece_bytes=c["piece_kib"] << 10, max_pieces=c["max_pieces"], sum_ctas=c["ctas"],
-                  copy_ctas=c["ctas"], ag_direct=c["ag_direct"])
+                  copy_ctas=c["ctas"], ag_direct=c["ag_direct"], rs_direct=c["rs_direct"])
     if c["variant"] != "plain":
         params[c["variant"]] = 1
     comm = make_comm(R, max(total, 1), dtype, c["path"], **params)

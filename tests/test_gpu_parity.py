@@ -29,7 +29,7 @@ def make_comm(R, count, dtype, path=hb.PATH_CE, **params):
     comm.set_path(path)
     for k, v in params.items():
         comm.set_param(k, v)
-    nb = hb.scratch_bytes(R, count, dtype)
+    nb = hb.scratch_bytes_direct(R, count, dtype) if params.get("rs_direct") else hb.scratch_bytes(R, count, dtype)
     scratch = DevBuf(nb + 256)
     pad = (-scratch.ptr) % 256
     comm._scratch_keep = scratch

@@ -1,0 +1,161 @@
+"""GPU parity for the direct reduce-scatter ("rs_direct" = 1): the reduce-scatter as the R-1 permutation stages r -> r+k of its
+traffic matrix (the paper's stage decomposition, Sec. 3.4) into R-1 inbox slots of the owner, then one chain sum per rank in
+the ring's order with a rounding after every add.
+
+The order of addition and every rounding are the ring's, so all results must carry the oracle's bits: on every path and
+executor, for both dtypes, in place, with ragged sizes and misaligned buffers, alone and combined with the direct all-gather."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2609_34334_b200 import binding as hb
+from paper_2609_34334_b200 import workloads as W
+from gpu_util import DevBuf, np_dtype, same_bits
+from test_gpu_parity import make_comm, run_allreduce
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(autouse=True)
+def _need_gpu():
+    assert torch.cuda.is_available(), "these tests need a CUDA device"
+    torch.cuda.set_device(0)
+    yield
+    torch.cuda.synchronize()
+
+
+CONFIGS = [
+    (hb.PATH_CE, dict()),
+    (hb.PATH_CE, dict(ag_direct=1)),
+    (hb.PATH_CE, dict(use_graph=0)),
+    (hb.PATH_CE, dict(order_kernels=0)),
+    (hb.PATH_SM, dict(sum_ctas=8, copy_ctas=8)),
+    (hb.PATH_SM, dict(sum_ctas=8, copy_ctas=8, ag_direct=1)),
+    (hb.PATH_SM, dict(sum_ctas=148, copy_ctas=148, ag_direct=1)),
+    (hb.PATH_SM, dict(sum_ctas=3, copy_ctas=5, use_graph=0)),
+    (hb.PATH_SM, dict(fused=1, sum_ctas=148, copy_ctas=148)),             # not available as one kernel: runs as a graph
+    (hb.PATH_SM, dict(forward=1, sum_ctas=32, copy_ctas=32)),              # forward does not apply: ignored
+    (hb.PATH_SM, dict(handshake=1, watchdog_ms=5000)),
+    (hb.PATH_CE_HOST, dict(ag_direct=1)),
+]
+
+
+@pytest.mark.parametrize("path,params", CONFIGS)
+def test_allreduce_with_direct_reduce_scatter(oracle, path, params):
+    for dtype in ("fp32", "bf16"):
+        e = W.elem_size(dtype)
+        for R, n in [(2, 1), (2, 100_003), (3, 5), (4, 262_144 + 9), (8, 8 * 70_000 + 3), (8, 7), (5, 99_999)]:
+            xs = W.rank_inputs("uniform", 190 + R, R, n, dtype)
+            want = oracle.ring_allreduce(xs)
+            comm = make_comm(R, n, dtype, path, rs_direct=1, piece_bytes=65536, max_pieces=4, **params)
+            if path == hb.PATH_CE_HOST:
+                comm.set_host_staging(torch.empty(4 * R * (n * e + 4096), dtype=torch.uint8).pin_memory())
+            for in_place in (False, True):
+                offs = [(r % 4) * e for r in range(R)] if in_place else None
+                got = run_allreduce(comm, xs, dtype, in_place=in_place, offs=offs)
+                for r in range(R):
+                    assert same_bits(got[r], want[r], dtype), (dtype, R, n, in_place, r)
+            st = comm.last_stats()
+            if R > 1 and n >= R:
+                assert st["n_sum_launches"] == st["n_pieces"], st          # one chain launch per piece instead of R-1 sums
+            comm.destroy()
+
+
+@pytest.mark.parametrize("path", [hb.PATH_CE, hb.PATH_SM])
+def test_reduce_scatter_call_direct(oracle, path):
+    for dtype in ("fp32", "bf16"):
+        e = W.elem_size(dtype)
+        for R, count in [(1, 9), (2, 1), (4, 1025), (8, 4099), (3, 77)]:
+            xs = W.rank_inputs("uniform", 141, R, R * count, dtype)
+            want = oracle.ring_reduce_scatter(xs)
+            comm = make_comm(R, R * count, dtype, path, rs_direct=1, piece_bytes=2048, max_pieces=5)
+            send = [DevBuf(R * count * e).put(xs[r]) for r in range(R)]
+            recv = [DevBuf(count * e, (r % 2) * e) for r in range(R)]
+            comm.reduce_scatter(send, recv, count, dtype)
+            torch.cuda.synchronize()
+            for r in range(R):
+                assert same_bits(recv[r].get(np_dtype(dtype)), want[r], dtype), (dtype, R, count, r)
+                assert recv[r].guards_intact() and send[r].guards_intact()
+                assert (send[r].get(np_dtype(dtype)).view(np.uint8) == xs[r].view(np.uint8)).all(), "send buffer was written"
+            comm.reduce_scatter(send, [send[r].ptr + r * count * e for r in range(R)], count, dtype)      # in place
+            torch.cuda.synchronize()
+            for r in range(R):
+                assert same_bits(send[r].get(np_dtype(dtype))[r * count:(r + 1) * count], want[r], dtype)
+            comm.destroy()
+
+
+def test_special_values_and_many_ranks(oracle):
+    """NaN, infinities, signed zeros and subnormals go through the chain like through the ring; R = 20 and 40 need several
+    operand batches per element (more than 8 operands) and several launches per group."""
+    for dtype in ("fp32", "bf16"):
+        for R, n in [(4, 4 * 2048 + 3), (20, 20 * 300 + 7), (40, 40 * 64 + 1)]:
+            xs = W.rank_inputs("uniform", 195, R, n, dtype)
+            special = np.array([np.nan, np.inf, -np.inf, 0.0, -0.0, 1e-40, -1e-40, 3.0e38, -3.0e38, 1.0], dtype=np.float32)
+            for r in range(R):
+                v = np.roll(special, r)
+                if dtype == "fp32":
+                    xs[r][:v.size] = v
+                else:
+                    xs[r][:v.size] = (v.view(np.uint32) >> 16).astype(np.uint16)
+            want = oracle.ring_allreduce(xs)
+            for path, params in ((hb.PATH_CE, dict()), (hb.PATH_SM, dict(sum_ctas=16, copy_ctas=16, ag_direct=1))):
+                comm = make_comm(R, n, dtype, path, rs_direct=1, **params)
+                got = run_allreduce(comm, xs, dtype, in_place=True, offs=[(r % 3) * W.elem_size(dtype) for r in range(R)])
+                for r in range(R):
+                    assert same_bits(got[r], want[r], dtype), (dtype, R, path, r)
+                comm.destroy()
+
+
+def test_scratch_bound_is_checked():
+    R, n, dtype = 8, 8 * 10_000, "fp32"
+    comm = make_comm(R, n, dtype, hb.PATH_CE)                       # scratch for the ring: two slots per rank
+    a = [DevBuf(n * 4) for _ in range(R)]
+    b = [DevBuf(n * 4) for _ in range(R)]
+    assert comm.allreduce_rc(a, b, n, dtype) == hb.OK
+    comm.set_param("rs_direct", 1)
+    assert comm.allreduce_rc(a, b, n, dtype) == hb.ERR_SCRATCH      # R-1 slots per rank do not fit
+    torch.cuda.synchronize()
+    comm.destroy()
+    assert hb.scratch_bytes_direct(R, n, dtype) >= (R - 1) * hb.scratch_bytes(R, n, dtype) // 2
+    assert hb.scratch_bytes_direct(2, n, dtype) == hb.scratch_bytes(2, n, dtype)
+    assert hb.scratch_bytes_direct(1, n, dtype) == 0
+
+
+def test_config2_bucket_full_size(oracle):
+    """The gradient bucket at full size, two calls and one call, copy route with 8-CTA sums and the SM path."""
+    c = W.C2_DP_BUCKET
+    R, n, e = c.R, c.count, 2
+    xs = W.rank_inputs(c.dist, c.seed, R, n, c.dtype, c.sigma)
+    want = oracle.ring_allreduce(xs, threads=oracle.max_threads())
+    count = n // R
+    send = [DevBuf(n * e).put(xs[r]) for r in range(R)]
+    recv = [DevBuf(n * e) for _ in range(R)]
+    for path, params in [(hb.PATH_CE, dict(sum_ctas=8)), (hb.PATH_CE, dict(sum_ctas=8, ag_direct=1)),
+                         (hb.PATH_SM, dict(sum_ctas=8, copy_ctas=48, ag_direct=1)), (hb.PATH_SM, dict(sum_ctas=148, copy_ctas=148, ag_direct=1))]:
+        comm = make_comm(R, n, c.dtype, path, rs_direct=1, **params)
+        for two_calls in (True, False):
+            for b in recv:
+                b.view.fill_(0)
+            torch.cuda.synchronize()
+            if two_calls:
+                rs_out = [recv[r].ptr + r * count * e for r in range(R)]
+                comm.reduce_scatter(send, rs_out, count, c.dtype)
+                comm.allgather(rs_out, recv, count, c.dtype)
+            else:
+                comm.allreduce(send, recv, n, c.dtype)
+            torch.cuda.synchronize()
+            for r in range(R):
+                assert same_bits(recv[r].get(np.uint16), want[r], c.dtype), (path, params, two_calls, r)
+                assert recv[r].guards_intact() and send[r].guards_intact()
+        assert comm._scratch_keep.guards_intact()
+        comm.destroy()
+
+
+def test_native_bf16_add_equals_the_reference_add_for_all_operand_pairs():
+    """The chain kernel adds bf16 with add.rn.bf16x2.  It must give the bits of every other SUM (binary32 add of the widened
+    operands, rounded to nearest even) for all 2^32 pairs of bf16 bit patterns, NaN payloads included."""
+    counts = torch.zeros(2, dtype=torch.int64, device="cuda")
+    torch.cuda.synchronize()
+    assert hb.selftest_bf16_add(counts) == hb.OK
+    torch.cuda.synchronize()
+    assert counts.tolist() == [0, 0]

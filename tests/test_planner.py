@@ -42,7 +42,7 @@ def _run_plan(plan, kind, R, count, dtype, xs, in_place, rng):
     npdt = np.float32 if dtype == "fp32" else np.uint16
     base = {hb.PLAN_ALLREDUCE_FWD: hb.PLAN_ALLREDUCE, hb.PLAN_REDUCE_SCATTER_FWD: hb.PLAN_REDUCE_SCATTER, hb.PLAN_ALLREDUCE_AGD: hb.PLAN_ALLREDUCE,
             hb.PLAN_ALLREDUCE_FWD_AGD: hb.PLAN_ALLREDUCE, hb.PLAN_ALLGATHER_DIRECT: hb.PLAN_ALLGATHER}.get(kind, kind)
-    kind = base
+    kind = base if base < 16 else (base & 15)
     if kind == hb.PLAN_ALLREDUCE:
         send_n, recv_n = count, count
     elif kind == hb.PLAN_ALLTOALL:
@@ -54,6 +54,8 @@ def _run_plan(plan, kind, R, count, dtype, xs, in_place, rng):
     slot = plan.slot_bytes
     if R > 1 and count > 0 and kind in (hb.PLAN_ALLREDUCE, hb.PLAN_REDUCE_SCATTER):
         assert 0 < slot <= hb.scratch_bytes(R, send_n, dtype) // (2 * R)      # the advertised bound covers any piece setting
+        bound = hb.scratch_bytes_direct(R, send_n, dtype) if plan.inbox_slots > 1 else hb.scratch_bytes(R, send_n, dtype)
+        assert plan.scratch_bytes <= bound
     send = [x.copy().view(np.uint8) for x in xs]
     if in_place:
         if kind == hb.PLAN_ALLREDUCE:
@@ -67,7 +69,7 @@ def _run_plan(plan, kind, R, count, dtype, xs, in_place, rng):
                 send[r] = recv[r][r * count * e:(r + 1) * count * e]
     else:
         recv = [np.full(recv_n * e, 0xAB, dtype=np.uint8) for _ in range(R)]
-    inbox = [np.full(slot, 0xCD, dtype=np.uint8) for _ in range(R)]
+    inbox = [np.full(slot * plan.inbox_slots, 0xCD, dtype=np.uint8) for _ in range(R)]
     partial = [np.full(slot, 0xEF, dtype=np.uint8) for _ in range(R)]
     bufs = {hb.BUF_SEND: send, hb.BUF_RECV: recv, hb.BUF_INBOX: inbox, hb.BUF_PARTIAL: partial}
     by_group = {}
@@ -85,6 +87,19 @@ def _run_plan(plan, kind, R, count, dtype, xs, in_place, rng):
                 dst = bufs[op["dst_buf"]][op["dst_rank"]]
                 assert op["dst_off"] + n <= dst.size
                 dst[op["dst_off"]:op["dst_off"] + n] = src
+            elif op["kind"] == hb.OP_CHAIN:
+                assert dtype == "fp32" and op["rank"] == op["dst_rank"] and op["src_buf"] == hb.BUF_INBOX
+                box = bufs[hb.BUF_INBOX][op["rank"]]
+                acc = box[op["src_off"]:op["src_off"] + n].view(np.float32).copy()
+                for j in range(1, op["nsrc"]):
+                    lo = op["src_off"] + j * op["src_stride"]
+                    assert lo + n <= box.size
+                    acc = acc + box[lo:lo + n].view(np.float32)
+                loc = bufs[op["local_buf"]][op["rank"]][op["local_off"]:op["local_off"] + n]
+                res = (acc + loc.view(np.float32)).view(np.uint8)
+                out = bufs[op["dst_buf"]][op["dst_rank"]]
+                assert op["dst_off"] + n <= out.size
+                out[op["dst_off"]:op["dst_off"] + n] = res
             else:
                 assert dtype == "fp32"
                 loc = bufs[op["local_buf"]][op["rank"]][op["local_off"]:op["local_off"] + n]
@@ -326,3 +341,53 @@ def test_direct_standalone_allgather_plan(oracle, R, count):
             got = _run_plan(plan, hb.PLAN_ALLGATHER_DIRECT, R, count, "fp32", xs, in_place, rng)
             for r in range(R):
                 assert (got[r].view(np.uint32) == want[r].view(np.uint32)).all()
+
+
+@pytest.mark.parametrize("R,n,piece_bytes,max_pieces", [c for c in CASES if c[0] > 1 and c[1] > 0])
+def test_direct_reduce_scatter_plans(oracle, R, n, piece_bytes, max_pieces):
+    """The reduce-scatter as the R-1 permutation stages of its traffic matrix plus one chain sum per rank: every move leaves
+    the sender's own send buffer for the owner's inbox slot (the slot order is the ring's order of addition), nothing waits
+    for anything but the moves of its own piece, and any legal order gives the ring's bits."""
+    rng = random.Random(R * 515 + n)
+    xs = W.rank_inputs("uniform", 41, R, n, "fp32")
+    want = oracle.ring_allreduce(xs)
+    for flags in (hb.PLAN_FLAG_RS_DIRECT, hb.PLAN_FLAG_RS_DIRECT | hb.PLAN_FLAG_AG_DIRECT):
+        kind = hb.PLAN_ALLREDUCE | flags
+        for in_place in (False, True):
+            align = [(4 * rng.randrange(4)) for _ in range(R)] if in_place else None
+            plan = hb.Plan(kind, R, n, "fp32", in_place, piece_bytes, max_pieces, align)
+            assert plan.inbox_slots == R - 1
+            q = -(-n // R)
+            rs_moves = [op for op in plan.ops if op["kind"] == hb.OP_MOVE and op["phase"] == 0]
+            chains = [op for op in plan.ops if op["kind"] == hb.OP_CHAIN]
+            assert not [op for op in plan.ops if op["kind"] == hb.OP_SUM]
+            for op in rs_moves:
+                k = op["step"] + 1
+                assert op["dst_rank"] == (op["rank"] + k) % R == op["chunk"] and op["src_buf"] == hb.BUF_SEND and op["dst_buf"] == hb.BUF_INBOX
+                assert not plan.deps[op["group"]]
+                slot = op["dst_off"] // plan.slot_bytes
+                assert (op["dst_rank"] + 1 + slot) % R == op["rank"]            # slot j holds source d+1+j: the ring's order
+            for op in chains:
+                assert op["rank"] == op["dst_rank"] == op["chunk"] and op["nsrc"] == R - 1 and op["src_stride"] == plan.slot_bytes
+                assert op["local_buf"] == hb.BUF_SEND and op["dst_buf"] == hb.BUF_RECV
+                a = align[op["rank"]] if align else 0
+                assert op["src_off"] % 16 == (a + op["local_off"]) % 16          # operands share their 16-byte phase
+            moved = sum(op["bytes"] for op in rs_moves)
+            assert moved == sum((min((c + 1) * q, n) - min(c * q, n)) * 4 for c in range(R)) * (R - 1)
+            for trial in range(2):
+                got = _run_plan(plan, kind, R, n, "fp32", xs, in_place, rng)
+                for r in range(R):
+                    assert (got[r].view(np.uint32) == want[r].view(np.uint32)).all(), (flags, R, n, in_place, r)
+    if n % R == 0:
+        wrs = oracle.ring_reduce_scatter(xs)
+        kind = hb.PLAN_REDUCE_SCATTER | hb.PLAN_FLAG_RS_DIRECT
+        for in_place in (False, True):
+            plan = hb.Plan(kind, R, n // R, "fp32", in_place, piece_bytes, max_pieces)
+            got = _run_plan(plan, kind, R, n // R, "fp32", xs, in_place, rng)
+            for r in range(R):
+                res = got[r] if not in_place else got[r]
+                assert (res.view(np.uint32) == wrs[r].view(np.uint32)).all(), (R, n, in_place, r)
+    # flags that do not apply are ignored, unknown ones refused
+    assert hb.Plan(hb.PLAN_ALLGATHER | hb.PLAN_FLAG_RS_DIRECT, R, 8, "fp32").inbox_slots == 1
+    with pytest.raises(hb.HocclError):
+        hb.Plan(hb.PLAN_ALLREDUCE | 128, R, 8, "fp32")
