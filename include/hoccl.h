@@ -429,6 +429,11 @@ hoccl_result_t hoccl_sum_launch(const void* inbox, const void* local, void* out,
                                 int ctas, hoccl_stream_t stream);
 hoccl_result_t hoccl_copy_launch(const void* src, void* dst, size_t bytes, int ctas, hoccl_stream_t stream);
 hoccl_result_t hoccl_fanout_launch(const void* src, void* const* dsts, int ndst, size_t bytes, int ctas, hoccl_stream_t stream);
+/* Direct launch of the chain sum of the direct reduce-scatter ("rs_direct"): out[i] = (((s_0[i] + s_1[i]) + ...) + s_{nsrc-1}[i])
+ * + local[i], i < count, every add rounded into `dtype`; s_j = first + j * stride_bytes (a multiple of 16), nsrc in 1..63,
+ * `ctas` CTAs of 1024 threads.  Device pointers aligned to the element size; out may equal local. */
+hoccl_result_t hoccl_chain_launch(const void* first, size_t stride_bytes, int nsrc, const void* local, void* out, size_t count,
+                                  hoccl_dtype_t dtype, int ctas, hoccl_stream_t stream);
 /*
  * "SMs used", counted rather than inferred (the paper's Table 1 counts the SMs that communication kernels occupy):
  * launches the SUM kernel (kind 0: out = a + b over bytes / sizeof(dtype) elements) or the copy kernel (kind 1:

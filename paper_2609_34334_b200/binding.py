@@ -29,7 +29,7 @@ EXPORTS = [
     "hoccl_comm_set_path", "hoccl_comm_set_param", "hoccl_comm_get_param", "hoccl_allreduce", "hoccl_reduce_scatter",
     "hoccl_allgather", "hoccl_alltoall", "hoccl_alltoallv", "hoccl_send", "hoccl_recv", "hoccl_comm_pending", "hoccl_comm_async_error", "hoccl_comm_handshakes", "hoccl_selftest_barrier_timeout", "hoccl_host_allreduce", "hoccl_error_string",
     "hoccl_last_cuda_error", "hoccl_last_stats", "hoccl_profile_reset", "hoccl_probe_move_needs_sm", "hoccl_probe_copy_routes", "hoccl_sum_launch", "hoccl_kernel_sms", "hoccl_flatten_inspect", "hoccl_port_probe",
-    "hoccl_copy_launch", "hoccl_fanout_launch", "hoccl_fanout_inspect", "hoccl_selftest_bf16_add", "hoccl_plan_build", "hoccl_plan_destroy", "hoccl_plan_num_ops", "hoccl_plan_num_groups",
+    "hoccl_copy_launch", "hoccl_fanout_launch", "hoccl_fanout_inspect", "hoccl_selftest_bf16_add", "hoccl_chain_launch", "hoccl_plan_build", "hoccl_plan_destroy", "hoccl_plan_num_ops", "hoccl_plan_num_groups",
     "hoccl_plan_get_op", "hoccl_plan_group_deps", "hoccl_plan_slot_bytes", "hoccl_allreduce_static",
     "hoccl_sched_build", "hoccl_sched_destroy", "hoccl_sched_num_stages", "hoccl_sched_stage_tau", "hoccl_sched_total_tau",
     "hoccl_sched_lower_bound", "hoccl_sched_matrix", "hoccl_sched_num_flows", "hoccl_sched_get_flow", "hoccl_sched_queue_len",
@@ -141,6 +141,7 @@ def lib() -> ctypes.CDLL:
         "hoccl_copy_launch": (i, [vp, vp, sz, i, vp]),
         "hoccl_fanout_launch": (i, [vp, vp, i, sz, i, vp]),
         "hoccl_selftest_bf16_add": (i, [vp, vp]),
+        "hoccl_chain_launch": (i, [vp, sz, i, vp, vp, sz, i, i, vp]),
         "hoccl_fanout_inspect": (i, [i, vp, vp, vp, i, i, vp, vp, vp, vp, vp, vp, vp, ctypes.POINTER(i), ctypes.POINTER(i)]),
         "hoccl_kernel_sms": (i, [i, vp, vp, vp, sz, i, i, vp, vp]),
         "hoccl_selftest_barrier_timeout": (i, [vp, vp, vp, sz, vp]),
@@ -380,6 +381,11 @@ def copy_launch(src, dst, nbytes, ctas, stream=None) -> int:
 def fanout_launch(src, dsts, nbytes, ctas, stream=None) -> int:
     """hoccl_fanout_launch: every dsts[d] <- src, the source read once.  Returns the result code."""
     return lib().hoccl_fanout_launch(_ptr(src), _ptr_array(dsts), len(dsts), nbytes, ctas, _stream(stream))
+
+
+def chain_launch(first, stride_bytes, nsrc, local, out, count, dtype, ctas, stream=None) -> int:
+    """hoccl_chain_launch: out = (((s_0 + s_1) + ...) + s_{nsrc-1}) + local with s_j = first + j * stride_bytes."""
+    return lib().hoccl_chain_launch(_ptr(first), stride_bytes, nsrc, _ptr(local), _ptr(out), count, _dtype(dtype), ctas, _stream(stream))
 
 
 def selftest_bf16_add(counts, stream=None) -> int:

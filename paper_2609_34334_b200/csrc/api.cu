@@ -652,6 +652,21 @@ hoccl_result_t hoccl_flatten_inspect(int kind, hoccl_dtype_t dtype, int ctas, in
   return HOCCL_OK;
 }
 
+hoccl_result_t hoccl_chain_launch(const void* first, size_t stride_bytes, int nsrc, const void* local, void* out, size_t count,
+                                  hoccl_dtype_t dtype, int ctas, hoccl_stream_t stream) {
+  const size_t e = dtype_size((int)dtype);
+  if (e == 0) return HOCCL_ERR_UNSUPPORTED;
+  if (!first || !local || !out || nsrc < 1 || nsrc > kMaxChainSrcs || (stride_bytes & 15) || ctas < 1 || ctas > 1024 ||
+      ((uintptr_t)first % e) || ((uintptr_t)local % e) || ((uintptr_t)out % e))
+    return HOCCL_ERR_INVALID_ARG;
+  if (count == 0) return HOCCL_OK;
+  ChainBatch b;
+  b.nseg = 1;
+  b.dtype = (int)dtype;
+  b.seg[0] = ChainSeg{first, local, out, (unsigned long long)count, (unsigned long long)stride_bytes, nsrc, 0};
+  return launch_chain(b, ctas, (cudaStream_t)stream) == cudaSuccess ? HOCCL_OK : HOCCL_ERR_CUDA;
+}
+
 hoccl_result_t hoccl_selftest_bf16_add(unsigned long long* counts, hoccl_stream_t stream) {
   if (!counts) return HOCCL_ERR_INVALID_ARG;
   return launch_bf16_add_selftest(counts, (cudaStream_t)stream) == cudaSuccess ? HOCCL_OK : HOCCL_ERR_CUDA;

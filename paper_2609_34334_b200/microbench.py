@@ -5,6 +5,7 @@
     python -m paper_2609_34334_b200.microbench --kernel ring --mib 32 --ctas 148   # all-reduce, R = 8, as one cooperative kernel
     python -m paper_2609_34334_b200.microbench --kernel port --mib 256 --ctas 8    # what the memory ports of `ctas` SMs carry
     python -m paper_2609_34334_b200.microbench --kernel fan --mib 25 --ctas 148    # one source to 7 destinations: fan-out against 7 copies
+    python -m paper_2609_34334_b200.microbench --kernel chain --mib 25 --ctas 8    # 7 inbox operands + the local one into one output
 
 Operands are larger than L2 by default; timing uses CUDA events on the launching stream after warm-up.
 Prints one JSON line.  This is the small case used for ncu captures of a single kernel.
@@ -21,7 +22,7 @@ from . import binding as hb
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--kernel", default="sum", choices=["sum", "copy", "routes", "ring", "port", "fan"])
+    ap.add_argument("--kernel", default="sum", choices=["sum", "copy", "routes", "ring", "port", "fan", "chain"])
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "fp32"])
     ap.add_argument("--mib", type=int, default=200, help="MiB per operand")
     ap.add_argument("--ctas", type=int, default=8)
@@ -56,6 +57,41 @@ def main():
             sec = e0.elapsed_time(e1) / 1e3 / args.reps
             out[name] = {"GBps": moved / sec / 1e9, "GBps_per_sm": moved / sec / 1e9 / args.ctas, "us": sec * 1e6}
         print(json.dumps(out))
+        return
+    if args.kernel == "chain":
+        # the sum of the direct reduce-scatter for R = 8: seven inbox operands and the local one, one output (8 reads : 1 write)
+        nsrc, sets = 7, 3
+        tdt = torch.bfloat16 if args.dtype == "bf16" else torch.float32
+        e = 2 if args.dtype == "bf16" else 4
+        n = nbytes // e
+        st = torch.cuda.Stream()
+        inbox = [torch.empty(nsrc * n, dtype=tdt, device="cuda").normal_(0, 1e-3) for _ in range(sets)]
+        local = [torch.empty(n, dtype=tdt, device="cuda").normal_(0, 1e-3) for _ in range(sets)]
+        out_t = [torch.empty(n, dtype=tdt, device="cuda") for _ in range(sets)]
+        torch.cuda.synchronize()
+
+        def chain(k):
+            assert hb.chain_launch(inbox[k], nbytes, nsrc, local[k], out_t[k], n, args.dtype, args.ctas, st) == hb.OK
+
+        for k in range(max(args.warmup, sets)):
+            chain(k % sets)
+        st.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(st)
+        for k in range(args.reps):
+            chain(k % sets)
+        e1.record(st)
+        st.synchronize()
+        sec = e0.elapsed_time(e1) / 1e3 / args.reps
+        acc = inbox[0][:n].clone()
+        for j in range(1, nsrc):
+            acc = (acc.float() + inbox[0][j * n:(j + 1) * n].float()).to(tdt)
+        acc = (acc.float() + local[0].float()).to(tdt)
+        assert torch.equal(out_t[0], acc), "kernel result differs from torch's fp32 add + RNE, taken step by step"
+        moved = (nsrc + 2) * nbytes
+        print(json.dumps({"kernel": "chain", "dtype": args.dtype, "mib_per_operand": args.mib, "inbox_operands": nsrc, "ctas": args.ctas,
+                          "us_per_launch": sec * 1e6, "algorithmic_bytes_per_launch": moved, "GBps": moved / sec / 1e9,
+                          "GBps_per_cta": moved / sec / 1e9 / args.ctas, "output_GBps_per_cta": nbytes / sec / 1e9 / args.ctas}))
         return
     if args.kernel == "fan":
         # the move of the direct all-gather: one chunk to R - 1 = 7 peers, as one fan-out launch and as 7 copy launches

@@ -159,3 +159,34 @@ def test_native_bf16_add_equals_the_reference_add_for_all_operand_pairs():
     assert hb.selftest_bf16_add(counts) == hb.OK
     torch.cuda.synchronize()
     assert counts.tolist() == [0, 0]
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+@pytest.mark.parametrize("ctas", [1, 8, 148])
+def test_chain_kernel_against_the_oracles_chain(oracle, dtype, ctas):
+    """hoccl_chain_launch against the oracle's closed form of the ring order, ((x_{c+1} + x_{c+2}) + ...) + x_c with a rounding
+    after every add: R = 2..12 operands, ragged lengths, operands off the 16-byte grid together (vector path) or not."""
+    e = W.elem_size(dtype)
+    for R, n in [(2, 1), (3, 1023), (8, 4096 * 5 + 3), (8, 1_000_003), (12, 70_001)]:
+        xs = W.rank_inputs("uniform", 230 + R, R, n, dtype)
+        c = R // 2
+        want = oracle.chain_sum(xs, c, 0, n)
+        stride = (n * e + 255) // 256 * 256 + 256
+        for offs in ((0, 0, 0), (e, e, e), (0, e, 0)):
+            inbox = DevBuf(stride * (R - 1), offs[0])
+            for j in range(R - 1):                                   # slot j holds source c + 1 + j: the ring's order
+                src = xs[(c + 1 + j) % R].view(np.uint8)
+                inbox.view[j * stride:j * stride + n * e].copy_(torch.from_numpy(src.copy()))
+            local = DevBuf(n * e, offs[1]).put(xs[c])
+            out = DevBuf(n * e, offs[2])
+            torch.cuda.synchronize()
+            assert hb.chain_launch(inbox, stride, R - 1, local, out, n, dtype, ctas) == hb.OK
+            torch.cuda.synchronize()
+            assert same_bits(out.get(np_dtype(dtype)), want, dtype), (dtype, R, n, offs)
+            assert out.guards_intact() and inbox.guards_intact() and local.guards_intact()
+            # in place on the local operand
+            assert hb.chain_launch(inbox, stride, R - 1, local, local, n, dtype, ctas) == hb.OK
+            torch.cuda.synchronize()
+            assert same_bits(local.get(np_dtype(dtype)), want, dtype), ("in place", dtype, R, n, offs)
+    assert hb.chain_launch(inbox, 24, 1, local, out, 4, dtype, 8) == hb.ERR_INVALID_ARG      # stride not a multiple of 16
+    assert hb.chain_launch(inbox, 32, 64, local, out, 4, dtype, 8) == hb.ERR_INVALID_ARG     # too many operands
