@@ -218,7 +218,7 @@ def main():
             send = [torch.roll(t, 4099 * b) for t in send_sets[0]]
         send_sets.append(send)
         recv_sets.append([torch.zeros(n, dtype=torch.int16, device="cuda") for _ in range(R)])
-    scratch = torch.empty(hb.scratch_bytes(R, n, dtype) + 256, dtype=torch.uint8, device="cuda")
+    scratch = torch.empty(hb.scratch_bytes_direct(R, n, dtype) + 256, dtype=torch.uint8, device="cuda")   # covers every variant
     spad = (-scratch.data_ptr()) % 256
 
     def new_comm(path=hb.PATH_CE, **params):
@@ -446,7 +446,7 @@ def small_case(hb, W, torch, np, stream):
     sets = 8      # 8 x 32 MiB of buffers in rotation: larger than L2
     send = [[torch.from_numpy(x).cuda() for x in xs] for _ in range(sets)]
     recv = [[torch.zeros(n, dtype=torch.float32, device="cuda") for _ in range(R)] for _ in range(sets)]
-    nb = hb.scratch_bytes(R, n, c.dtype)
+    nb = hb.scratch_bytes_direct(R, n, c.dtype)
     scratch = torch.empty(nb + 256, dtype=torch.uint8, device="cuda")
     rows = {}
     for name, path, ctas, fused, direct, fwd in (("CE_sum8", hb.PATH_CE, 8, 0, 0, 0), ("CE_sum8_direct_allgather", hb.PATH_CE, 8, 0, 1, 0),
@@ -581,6 +581,24 @@ def extras(hb, W, torch, np, new_comm, step, timed, stream, R, S, n, dtype, peak
                         "one_allreduce_call_ms": t1 * 1e3, "one_allreduce_call_busbw_GBps": S * bus_factor(R) / t1 / 1e9})
         c1.destroy()
     out["direct_allgather"] = ad_rows
+    # direct schedule: the reduce-scatter too as independent permutation stages, into R-1 inbox slots of the owner, and ONE chain
+    # sum per rank in the ring's order (rank local, the ring's bits); with the ring or the direct all-gather behind it
+    ds_rows = []
+    for name, path, sc, cc, agd in (("CE", hb.PATH_CE, 8, 8, 0), ("CE", hb.PATH_CE, 8, 8, 1), ("CE", hb.PATH_CE, 32, 8, 1), ("CE", hb.PATH_CE, 148, 8, 1),
+                                    ("SM", hb.PATH_SM, 8, 8, 1), ("SM", hb.PATH_SM, 8, 48, 1), ("SM", hb.PATH_SM, 148, 148, 1)):
+        c1 = new_comm(path, sum_ctas=sc, copy_ctas=cc, rs_direct=1, ag_direct=agd)
+        t, _ = timed(c1, k, w)
+        t1, _ = timed(c1, k, w, fn=one_call)
+        # algorithmic bytes: moves 2 S (R-1), chain sum S (R+1) (R reads and one write per output byte), all-gather 2 S (R-1) as
+        # copies or S R as a fan-out launch
+        ag_bytes = 1.0 * S * R if (agd and path == hb.PATH_SM) else 2.0 * S * (R - 1)
+        hbm_d = 2.0 * S * (R - 1) + 1.0 * S * (R + 1) + ag_bytes
+        ds_rows.append({"path": name, "sum_ctas": sc, "copy_ctas": cc if path == hb.PATH_SM else None, "ag_direct": agd, "ms_per_step": t * 1e3,
+                        "busbw_GBps": S * bus_factor(R) / t / 1e9, "hbm_bytes_per_step": hbm_d, "hbm_frac_of_8TBps": hbm_d / t / 1e9 / NOMINAL_HBM_GBS,
+                        "one_allreduce_call_ms": t1 * 1e3, "one_allreduce_call_busbw_GBps": S * bus_factor(R) / t1 / 1e9,
+                        "sum_launches_per_step": int(c1.last_stats()["n_sum_launches"])})
+        c1.destroy()
+    out["direct_schedule"] = ds_rows
     # SM path with the whole collective as one cooperative kernel (grid barriers instead of kernel boundaries)
     fu_rows = []
     for ctas in (8, 148):
@@ -716,11 +734,12 @@ def extras(hb, W, torch, np, new_comm, step, timed, stream, R, S, n, dtype, peak
                                        ("SM_copy32_sum8", hb.PATH_SM, 8, 32, 0, 0), ("SM_copy48_sum8", hb.PATH_SM, 8, 48, 0, 0),
                                        ("SM_copy148_sum148", hb.PATH_SM, 148, 148, 0, 0),
                                        ("SM_copy48_sum8_direct_allgather", hb.PATH_SM, 8, 48, 0, 3),
+                                       ("CE_sum8_direct_schedule", hb.PATH_CE, 8, 8, 0, 5), ("SM_copy48_sum8_direct_schedule", hb.PATH_SM, 8, 48, 0, 5),
                                        ("SM_forward_copy8_sum8", hb.PATH_SM, 8, 8, 0, 1),
                                        ("SM_one_kernel_8", hb.PATH_SM, 8, 8, 0, 2),
                                        ("onepass_8", hb.PATH_CE, 8, 8, 1, 0), ("CE_HOST_sum8", hb.PATH_CE_HOST, 8, 8, 0, 0)):
         c2 = new_comm(path, sum_ctas=sc, copy_ctas=cc, onepass=op, forward=1 if fw == 1 else 0, fused=1 if fw == 2 else 0,
-                      ag_direct=1 if fw == 3 else 0, order_kernels=0 if fw == 4 else 1)
+                      ag_direct=1 if fw in (3, 5) else 0, order_kernels=0 if fw == 4 else 1, rs_direct=1 if fw == 5 else 0)
         if path == hb.PATH_CE_HOST:
             c2.set_host_staging(host_stage)
         # the one-pass comparison kernel is one all-reduce call (reduce-scatter + all-gather would add the path's moves)

@@ -110,7 +110,10 @@ def sweep_sizes(args):
                ("CEplain", hb.PATH_CE, 8, 8, 0),   # copy route, plain graphs: no empty ordering kernels (order_kernels = 0)
                ("CEall", hb.PATH_CE, 148, 8, 0),   # copy route with whole-GPU sums: what the route reaches without the 8-CTA SUM budget
                ("CEdirect", hb.PATH_CE, 8, 8, 0), ("SM8direct", hb.PATH_SM, 8, 8, 0), ("SMalldirect", hb.PATH_SM, 148, 148, 0),
-               ("SMallfwddirect", hb.PATH_SM, 148, 148, 0)]
+               ("SMallfwddirect", hb.PATH_SM, 148, 148, 0),
+               # direct schedule: reduce-scatter and all-gather both as independent stages, one chain sum per rank
+               ("CErsdirect", hb.PATH_CE, 8, 8, 0), ("CEallrsdirect", hb.PATH_CE, 148, 8, 0), ("SM8rsdirect", hb.PATH_SM, 8, 8, 0),
+               ("SMallrsdirect", hb.PATH_SM, 148, 148, 0)]
     if args.configs != "all":
         configs = [c for c in configs if c[0] in args.configs.split(",")]
     else:
@@ -132,7 +135,7 @@ def sweep_sizes(args):
                     if footprint * nsets > (48 << 30):
                         nsets = 1
                     arena = Arena(op, R, S, dtype, nsets)
-                    scratch = torch.empty(hb.scratch_bytes(R, S // e, dtype) + 256, dtype=torch.uint8, device="cuda")
+                    scratch = torch.empty(hb.scratch_bytes_direct(R, S // e, dtype) + 256, dtype=torch.uint8, device="cuda")
                     pad = (-scratch.data_ptr()) % 256
                     for name, path, sc, cc, fused in configs:
                         comm = hb.Comm(R, 0)
@@ -146,6 +149,7 @@ def sweep_sizes(args):
                         comm.set_param("ag_direct", 1 if direct else 0)
                         comm.set_param("forward", 1 if "fwd" in name else 0)
                         comm.set_param("order_kernels", 0 if name == "CEplain" else 1)
+                        comm.set_param("rs_direct", 1 if name.endswith("rsdirect") else 0)
                         t = time_op(comm, arena, stream)
                         row = {"op": op, "R": R, "dtype": dtype, "S": S, "config": name, "sum_ctas": sc,
                                "copy_ctas": cc if path == hb.PATH_SM else None, "us": t * 1e6, "algbw_GBps": S / t / 1e9,
@@ -277,7 +281,7 @@ def gradients(args):
     pool = 3     # reusable per-rank bucket buffers
     send = [[torch.empty(per, dtype=torch.bfloat16, device="cuda").normal_(0, 1e-3) for _ in range(R)] for _ in range(pool)]
     recv = [[torch.empty(per, dtype=torch.bfloat16, device="cuda") for _ in range(R)] for _ in range(pool)]
-    scratch = torch.empty(hb.scratch_bytes(R, per, dtype) + 256, dtype=torch.uint8, device="cuda")
+    scratch = torch.empty(hb.scratch_bytes_direct(R, per, dtype) + 256, dtype=torch.uint8, device="cuda")
     pad = (-scratch.data_ptr()) % 256
     M, K, N = g.gemm_probe
     A = torch.randn(M, K, dtype=torch.bfloat16, device="cuda")
@@ -318,14 +322,16 @@ def gradients(args):
             configs.append(("SM_copy%d_sum%d" % (b, min(b, 8)), hb.PATH_SM, min(b, 8), b))
         configs.append(("SM_copy148_sum148", hb.PATH_SM, 148, 148))
     if getattr(args, "direct", False):   # every SM-path configuration once more with the direct (fan-out) all-gather
-        configs = configs + [(n_ + "_direct", p_, s_, c_) for n_, p_, s_, c_ in configs if p_ == hb.PATH_SM]
+        configs = (configs + [(n_ + "_direct", p_, s_, c_) for n_, p_, s_, c_ in configs if p_ == hb.PATH_SM] +
+                   [(n_ + "_rsdirect", p_, s_, c_) for n_, p_, s_, c_ in configs if not n_.endswith("_plain_graphs")])
     for name, path, sc, cc in configs:
         comm = hb.Comm(R, 0)
         comm.set_scratch(scratch.data_ptr() + pad, scratch.numel() - 256)
         comm.set_path(path)
         comm.set_param("sum_ctas", sc)
         comm.set_param("copy_ctas", cc)
-        comm.set_param("ag_direct", 1 if name.endswith("_direct") else 0)
+        comm.set_param("ag_direct", 1 if name.endswith("direct") else 0)
+        comm.set_param("rs_direct", 1 if name.endswith("_rsdirect") else 0)
         comm.set_param("order_kernels", 0 if name.endswith("_plain_graphs") else 1)   # the copy-route graphs without ordering kernels
         for k in range(pool):
             comm.allreduce(send[k], recv[k], per, dtype, stream)
