@@ -292,6 +292,24 @@ def main():
     units = replicas.sum_over_ranks(world, S * bus_factor(R))
     value = units / t_slowest / 1e9
 
+    # ---- the same workload, constraints and bits as the stage-decomposed ("direct") schedule: the reduce-scatter as R-1
+    # independent permutation stages into R-1 inbox slots and one chain sum per rank in the ring's order, the all-gather as
+    # R-1 independent stages; copy route, 8 SUM CTAs.  Timed like the headline (same steps, same bucket sets).
+    comm_d = new_comm(hb.PATH_CE, sum_ctas=8, rs_direct=1, ag_direct=1)
+    t_direct, _ = timed(comm_d, steps, warmup)
+    step(comm_d, 0, stream)
+    stream.synchronize()
+    got_direct = {r: recv_sets[0][r].cpu().numpy().view(np.uint16).copy() for r in (0, 5)}
+    comm_d.reduce_scatter(send_sets[0], rs_out0, count, dtype, stream)
+    stream.synchronize()
+    direct_sum_launches = int(comm_d.last_stats()["n_sum_launches"])
+    comm_d.destroy()
+    t_direct_slowest = replicas.max_over_ranks(world, t_direct)
+    direct_line = {"schedule": "rs_direct + ag_direct (rank local; the ring's order of addition and rounding)", "path": "CE (driver copy route)",
+                   "sum_ctas": 8, "value": units / t_direct_slowest / 1e9, "unit": "GB/s", "ms_per_step": t_direct_slowest * 1e3,
+                   "sum_launches_per_step": direct_sum_launches,
+                   "algorithmic_bytes_per_step": 2.0 * S * (R - 1) + 1.0 * S * (R + 1) + 2.0 * S * (R - 1), "matches_oracle": None}
+
     # ---- end to end: host buffers through hoccl_host_allreduce (H2D and D2H inside the timed region)
     per = (S + 255) // 256 * 256
     staging = torch.empty(2 * R * per + 256, dtype=torch.uint8, device="cuda")
@@ -339,6 +357,7 @@ def main():
         "host_launch_us_per_call": st["host_launch_us"],
         "windows": windows,
         "matches_oracle": parity,
+        "direct_schedule": direct_line,
         "peaks": peaks,
     }
 
@@ -417,6 +436,7 @@ def main():
         # the oracle's result against what the device produced in the timed configuration and end to end
         line["matches_oracle"] = all(bool((got_parity[r] == want[r]).all()) for r in got_parity)
         line["e2e"]["matches_oracle"] = bool((got_e2e == want[3]).all())
+        line["direct_schedule"]["matches_oracle"] = all(bool((got_direct[r] == want[r]).all()) for r in got_direct)
         t1 = time.perf_counter()
         oracle_ring.ring_allreduce(xs, threads=1)          # the canonical single-thread run (the parity reference)
         t_single = time.perf_counter() - t1

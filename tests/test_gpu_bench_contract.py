@@ -29,5 +29,7 @@ def test_bench_line_has_the_contract_keys():
     # per step: seven SUM launches, and the empty ordering kernels of the two graphs: one in front of each graph's first
     # copies, one behind each of the seven copy stages of the ring all-gather
     assert d["gpu_launches"] == (7 + 2 + 7) * 8
+    ds = d["direct_schedule"]
+    assert ds["matches_oracle"] is True and ds["sum_launches_per_step"] == 1 and ds["value"] > d["value"]
     c = d["cpu_baseline"]
     assert c["kind"] == "oracle" and c["cores"] >= 1 and c["value"] > 0
