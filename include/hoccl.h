@@ -176,7 +176,9 @@ hoccl_result_t hoccl_comm_set_path(hoccl_comm_t comm, hoccl_path_t path);
  *                written once instead of R-1 times: 2 S (R-1) + S (R+1) bytes of traffic instead of 5 S (R-1), and under
  *                an SM budget, where a sum is bound by the SMs' memory ports, R reads + 1 write per output instead of
  *                (R-1) x (2 reads + 1 write).  Needs hoccl_scratch_bytes_direct bytes of scratch (R-1 slots per rank
- *                instead of 2).  "forward" and "fused" do not apply to it.  0 = the ring reduce-scatter (default).
+ *                instead of 2).  "forward" and "fused" do not apply to it.  0 = the ring reduce-scatter (default).  2 = automatic:
+ *                direct whenever the attached scratch is large enough for it (it was measured faster than the ring at every
+ *                size and on every path), the ring otherwise.
  *  "order_kernels" 1 (default) = on the copy routes the graph executor puts an empty one-warp kernel in front of a graph's
  *                first copies and behind every group of copies that other copies (or the end of the graph) wait for.
  *                Measured on B200: a copy node that waits for earlier stream work or for several copy nodes starts ~4 us

@@ -133,7 +133,7 @@ static long* param_slot(hoccl_comm* c, const char* key, long* lo, long* hi) {
               {"forward", &c->forward, 0, 1},           {"fused", &c->fused, 0, 1},
               {"ag_direct", &c->ag_direct, 0, 2},
               {"order_kernels", &c->order_kernels, 0, 1},
-              {"rs_direct", &c->rs_direct, 0, 1},
+              {"rs_direct", &c->rs_direct, 0, 2},
               {"host_pieces", &c->host_pieces, 1, 64}};
   for (auto& r : rows)
     if (std::strcmp(r.name, key) == 0) {

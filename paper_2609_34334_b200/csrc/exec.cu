@@ -532,7 +532,13 @@ hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
   if (dtype_size(call->dtype) == 0) return HOCCL_ERR_UNSUPPORTED;
   if (!call->send || !call->recv) return HOCCL_ERR_INVALID_ARG;
   const bool onepass_case = c->onepass && !c->handshake && (call->kind == PLAN_ALLREDUCE || call->kind == PLAN_REDUCE_SCATTER);
-  const bool direct_rs = c->rs_direct && (call->kind == PLAN_ALLREDUCE || call->kind == PLAN_REDUCE_SCATTER);
+  // rs_direct = 2: the direct reduce-scatter whenever the attached scratch holds its R-1 inbox slots per rank (it was faster
+  // than the ring at every size and on every path measured), the ring otherwise
+  bool direct_rs = c->rs_direct == 1 && (call->kind == PLAN_ALLREDUCE || call->kind == PLAN_REDUCE_SCATTER);
+  if (c->rs_direct == 2 && (call->kind == PLAN_ALLREDUCE || call->kind == PLAN_REDUCE_SCATTER) && c->R > 1) {
+    const size_t cnt = call->kind == PLAN_ALLREDUCE ? call->count : call->count * (size_t)c->R;
+    direct_rs = c->scratch && c->scratch_bytes >= (size_t)(c->R - 1) * (size_t)c->R * slot_bytes_for(c->R, cnt, dtype_size(call->dtype));
+  }
   const bool fused = c->fused && c->path == HOCCL_PATH_SM && !c->handshake && !onepass_case && !call->h_send && !direct_rs;   // the ring kernel has no chain phase
   const bool graphs = (c->use_graph || c->handshake || fused) && !onepass_case;
   std::vector<uint64_t> key;
@@ -600,8 +606,7 @@ hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
   }
   if (direct && call->kind == PLAN_ALLREDUCE) plan_kind = c->forward ? PLAN_ALLREDUCE_FWD_AGD : PLAN_ALLREDUCE_AGD;
   if (direct && call->kind == PLAN_ALLGATHER) plan_kind = PLAN_ALLGATHER_DIRECT;
-  if (c->rs_direct && (call->kind == PLAN_ALLREDUCE || call->kind == PLAN_REDUCE_SCATTER))
-    plan_kind = call->kind | PLAN_FLAG_RS_DIRECT | (direct ? PLAN_FLAG_AG_DIRECT : 0);
+  if (direct_rs) plan_kind = call->kind | PLAN_FLAG_RS_DIRECT | (direct ? PLAN_FLAG_AG_DIRECT : 0);
   // Piece size: the caller's if set.  Otherwise: on the SM path under CTA budgets a reduction is cut into at least two
   // pieces (the copy kernel of one piece then overlaps the sum kernel of the other: measured 1.6x on a 3 MiB chunk with
   // 8 + 8 CTAs) of at most 4 MiB.  That does not pay with driver copies (they take the whole GPU and never overlap a sum:

@@ -52,7 +52,7 @@ case = st.fixed_dictionaries({
     "flavour": st.sampled_from(["normal", "wide", "special"]),
     "seed": st.integers(0, 2 ** 31 - 1),
     "ag_direct": st.integers(0, 2),
-    "rs_direct": st.integers(0, 1),
+    "rs_direct": st.integers(0, 2),
 })
 
 

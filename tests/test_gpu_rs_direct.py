@@ -190,3 +190,18 @@ def test_chain_kernel_against_the_oracles_chain(oracle, dtype, ctas):
             assert same_bits(local.get(np_dtype(dtype)), want, dtype), ("in place", dtype, R, n, offs)
     assert hb.chain_launch(inbox, 24, 1, local, out, 4, dtype, 8) == hb.ERR_INVALID_ARG      # stride not a multiple of 16
     assert hb.chain_launch(inbox, 32, 64, local, out, 4, dtype, 8) == hb.ERR_INVALID_ARG     # too many operands
+
+
+def test_automatic_choice_follows_the_scratch(oracle):
+    """rs_direct = 2: the direct form when the attached scratch holds R-1 inbox slots per rank, the ring otherwise."""
+    R, n, dtype = 8, 8 * 60_000 + 1, "bf16"
+    xs = W.rank_inputs("normal", 199, R, n, dtype, 1e-3)
+    want = oracle.ring_allreduce(xs)
+    for big, sums in ((True, 1), (False, R - 1)):
+        params = dict(rs_direct=1) if big else dict()            # make_comm sizes the scratch from this
+        comm = make_comm(R, n, dtype, hb.PATH_CE, piece_bytes=1 << 30, max_pieces=1, **params)
+        comm.set_param("rs_direct", 2)
+        got = run_allreduce(comm, xs, dtype)
+        assert all(same_bits(got[r], want[r], dtype) for r in range(R)), big
+        assert comm.last_stats()["n_sum_launches"] == sums, (big, comm.last_stats())
+        comm.destroy()
