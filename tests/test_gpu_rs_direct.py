@@ -205,3 +205,24 @@ def test_automatic_choice_follows_the_scratch(oracle):
         assert all(same_bits(got[r], want[r], dtype) for r in range(R)), big
         assert comm.last_stats()["n_sum_launches"] == sums, (big, comm.last_stats())
         comm.destroy()
+
+
+def test_host_allreduce_with_the_direct_schedule(oracle):
+    """The pipelined host entry point cuts chunks into pieces; every piece runs its own direct reduce-scatter and all-gather."""
+    from test_gpu_host_allreduce import _pinned, _with_staging
+    R, n, dtype = 8, 8 * 200_000 + 5, "bf16"
+    xs = W.rank_inputs("normal", 198, R, n, dtype, 1e-3)
+    want = oracle.ring_allreduce(xs)
+    for path, params in [(hb.PATH_CE, dict()), (hb.PATH_SM, dict(sum_ctas=8, copy_ctas=8))]:
+        comm = make_comm(R, n, dtype, path, rs_direct=1, ag_direct=1, host_pieces=4, **params)
+        _with_staging(comm, R, n, dtype)
+        h_send = [_pinned(x) for x in xs]
+        h_recv = [torch.zeros(n * 2, dtype=torch.uint8).pin_memory() for _ in range(R)]
+        for rep in range(2):
+            comm.host_allreduce(h_send, h_recv, n, dtype)
+            torch.cuda.synchronize()
+            for r in range(R):
+                assert same_bits(h_recv[r].numpy().view(np.uint16), want[r], dtype), (path, r, rep)
+        st = comm.last_stats()
+        assert st["n_pieces"] > 1 and st["n_sum_launches"] == st["n_pieces"], st
+        comm.destroy()
