@@ -362,6 +362,29 @@ def main():
     }
 
     if world.rank == 0:
+        # ---- the direct schedule's dominant kernel, the chain sum, timed per launch the same way (one launch per step)
+        prof_d = new_comm(hb.PATH_CE, sum_ctas=8, profile=1, rs_direct=1, ag_direct=1)
+        for k in range(3):
+            step(prof_d, k % N_BUCKET_SETS, stream)
+        stream.synchronize()
+        prof_d.profile_reset()
+        for k in range(min(steps, 40)):
+            step(prof_d, k % N_BUCKET_SETS, stream)
+            stream.synchronize()
+            prof_d.last_stats()
+        pd = prof_d.last_stats()
+        nld = max(1, pd["sum_kernel_launches_timed"])
+        avg_d = pd["sum_kernel_ms"] / nld
+        bytes_d = pd["sum_kernel_bytes"] / nld
+        ach_d = bytes_d / (avg_d * 1e-3) / 1e9 if avg_d > 0 else 0.0
+        # traffic: the ncu capture of profiles/chain_kernel_bf16_8cta_25MiB.md (216.7 MB of DRAM traffic for 235.9 MB of
+        # algorithmic bytes; the output of one launch is still in L2 when it ends), scaled by the bytes of this launch
+        line["direct_schedule"]["roofline"] = {
+            "kernel": "chain_kernel<bf16>", "bound": "hbm", "achieved": ach_d, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+            "frac": ach_d / peaks["hbm_gbs"], "peak_source": "of " + peaks["source"], "traffic": bytes_d * (216.72 / 235.93),
+            "algorithmic_bytes_per_launch": bytes_d, "avg_launch_us": avg_d * 1e3, "launches_timed": int(nld), "ctas": 8,
+            "note": "8 CTAs by design; 8 reads : 1 write per output byte, 111 GB/s per SM (profiles/chain_kernel_bf16_8cta_25MiB.md)"}
+        prof_d.destroy()
         # ---- roofline of the dominant kernel (the only kernel of this path): SUM, timed per launch with CUDA events
         prof = new_comm(hb.PATH_CE, sum_ctas=8, profile=1)
         for k in range(3):
