@@ -368,7 +368,11 @@ hoccl_result_t hoccl_host_allreduce(const void* const* h_send, void* const* h_re
  * overlap in time on the GPU (different streams, no ordering between them) race on the array: order them.
  *
  * First call.  The first call on each device looks up the array's device address (once per device, with
- * that device current) before it launches anything; make that first call before any stream capture.
+ * that device current) before it launches anything.  If the library's device code has not been loaded on that
+ * device yet, this look-up loads it: that is when the device reserves the HOCCL_STATIC_SCRATCH_BYTES of the array,
+ * and loading may synchronise the device.  "Allocates nothing" therefore holds from the second call on; make the
+ * first call on every device at start-up (a call with a few elements will do), and before any stream capture.
+ * The look-up uses the device that is current at the call; `stream` is not checked against it.
  *
  * Errors: INVALID_ARG (NULL or misaligned pointer, overlapping buffers, R out of range), UNSUPPORTED
  * (dtype, op), SCRATCH (beyond the maximum), CUDA (no device, address lookup or launch failed).

@@ -88,6 +88,56 @@ def small_integers(seed: int, rank: int, n: int, dtype: str, bound: int = 8, sta
     return _finish(_blocked(block, n, start), dtype)
 
 
+# ---- position-dependent inputs that can also be produced ON THE DEVICE (full-size parity runs) --------------------
+# A 32-bit integer hash of (seed, rank, element index) written with 64-bit integer operations that never overflow, so
+# numpy (host windows for the oracle) and torch (whole buffers, generated where they are used) give the same values.
+_H_A, _H_B, _H_C, _H_M1, _H_M2 = 2654435761, 0x9E3779B1, 0x85EBCA6B, 0x7FEB352D, 0x2C1B3C6D
+
+
+def _hash32(xp, idx, seed: int, rank: int):
+    """idx: int64 array/tensor of element indices below 2^31.  Returns int64 values in [0, 2^32)."""
+    m = 0xFFFFFFFF
+    h = (idx * _H_A + ((rank + 1) * _H_B + (seed + 1) * _H_C) % (1 << 32)) & m
+    h = h ^ (h >> 16)
+    h = (h * _H_M1) & m
+    h = h ^ (h >> 15)
+    h = (h * _H_M2) & m
+    return h ^ (h >> 16)
+
+
+def hashed(kind: str, seed: int, rank: int, start: int, n: int, dtype: str) -> np.ndarray:
+    """Elements start..start+n-1 of rank `rank`: kind "int" = integers in [-8, 8] (every partial sum over up to 8 ranks is
+    exact in bf16 and fp32, so the all-reduce result is the exact integer sum whatever the order), kind "uniform" =
+    k / 2^23 - 1 with k the top 24 bits of the hash.  No period: the value depends on the element's position."""
+    h = _hash32(np, np.arange(start, start + n, dtype=np.int64), seed, rank)
+    if kind == "int":
+        x = (h % 17 - 8).astype(np.float32)
+    elif kind == "uniform":
+        x = (h >> 8).astype(np.float32) * np.float32(2.0 ** -23) - np.float32(1.0)
+    else:
+        raise ValueError(kind)
+    return _finish(x, dtype)
+
+
+def hashed_device(kind: str, seed: int, rank: int, n: int, dtype: str, device="cuda", block: int = 1 << 25):
+    """The same values as hashed(kind, seed, rank, 0, n, dtype) as a torch tensor on `device` (float32, or bfloat16 for
+    "bf16"), generated block by block so that the 64-bit temporaries stay small."""
+    import torch
+
+    out = torch.empty(n, dtype=torch.float32 if dtype == "fp32" else torch.bfloat16, device=device)
+    for lo in range(0, n, block):
+        m = min(block, n - lo)
+        h = _hash32(torch, torch.arange(lo, lo + m, dtype=torch.int64, device=device), seed, rank)
+        if kind == "int":
+            x = (h % 17 - 8).to(torch.float32)
+        elif kind == "uniform":
+            x = (h >> 8).to(torch.float32) * (2.0 ** -23) - 1.0
+        else:
+            raise ValueError(kind)
+        out[lo:lo + m] = x.to(out.dtype)      # float32 -> bfloat16 rounds to nearest even, as _finish does
+    return out
+
+
 def _finish(x: np.ndarray, dtype: str) -> np.ndarray:
     if dtype == "fp32":
         return np.ascontiguousarray(x, dtype=np.float32)

@@ -79,6 +79,48 @@ def _python_chain(vals, c, dtype):
     return acc
 
 
+def _literal_chunk(n, R, c):
+    """Ring chunk c of n elements over R ranks: q = ceil(n / R) elements per chunk, clipped to n."""
+    q = -(-n // R)
+    return min(c * q, n), min((c + 1) * q, n)
+
+
+# (n, R) -> the R chunk ranges, typed out by hand from q = ceil(n / R): trailing chunks are short or empty
+CHUNK_TABLE = {
+    (10, 4): [(0, 3), (3, 6), (6, 9), (9, 10)],
+    (7, 3): [(0, 3), (3, 6), (6, 7)],
+    (5, 4): [(0, 2), (2, 4), (4, 5), (5, 5)],
+    (9, 8): [(0, 2), (2, 4), (4, 6), (6, 8), (8, 9), (9, 9), (9, 9), (9, 9)],
+    (3, 8): [(0, 1), (1, 2), (2, 3), (3, 3), (3, 3), (3, 3), (3, 3), (3, 3)],
+    (1, 4): [(0, 1), (1, 1), (1, 1), (1, 1)],
+    (0, 3): [(0, 0), (0, 0), (0, 0)],
+    (12, 4): [(0, 3), (3, 6), (6, 9), (9, 12)],
+    (13, 1): [(0, 13)],
+    (1_000_001, 8): [(0, 125001), (125001, 250002), (250002, 375003), (375003, 500004), (500004, 625005), (625005, 750006),
+                     (750006, 875007), (875007, 1000001)],
+}
+
+
+@pytest.mark.parametrize("n,R", sorted(CHUNK_TABLE))
+def test_chunk_partition_against_literal_values(oracle, n, R):
+    """The partition for counts that R does not divide (and n < R, where trailing chunks are empty)."""
+    for c, want in enumerate(CHUNK_TABLE[(n, R)]):
+        assert oracle.chunk_range(n, R, c) == want, (n, R, c)
+        assert _literal_chunk(n, R, c) == want
+
+
+def test_a_wrong_chunk_owner_changes_the_bits(oracle):
+    """The order fingerprint depends on which chunk an element is in, so a wrong partition for R that does not divide n
+    cannot hide: with x = (1e8, 1, -1e8, 1) on ranks 0..3 the chain of chunk c gives (0, 1, 0, 1)[c]."""
+    R, n = 4, 10
+    xs = [np.full(n, v, dtype=np.float32) for v in (1e8, 1.0, -1e8, 1.0)]
+    y = oracle.ring_allreduce(xs)[0]
+    want = np.empty(n, dtype=np.float32)
+    for c, (lo, hi) in enumerate(CHUNK_TABLE[(n, R)]):
+        want[lo:hi] = (0.0, 1.0, 0.0, 1.0)[c]
+    assert (y == want).all()
+
+
 @pytest.mark.parametrize("name,dtype", [("ring_order_w1_fp32.txt", "fp32"), ("ring_order_w2_bf16.txt", "bf16")])
 def test_worked_order_fingerprints(oracle, name, dtype):
     g = _read_golden(name)
@@ -136,7 +178,8 @@ def test_chain_closed_form_bruteforce(oracle, dtype, R):
         for r in range(1, R):
             assert (ys[r] == ys[0]).all()
         for c in range(R):
-            lo, hi = oracle.chunk_range(n, R, c)
+            lo, hi = _literal_chunk(n, R, c)      # the partition written out here, not taken from the oracle
+            assert oracle.chunk_range(n, R, c) == (lo, hi)
             for i in range(lo, hi):
                 vals = [x[i] if dtype == "fp32" else int(x[i]) for x in xs]
                 expect = _python_chain(vals, c, dtype)
