@@ -437,7 +437,8 @@ hoccl_result_t hoccl_copy_launch(const void* src, void* dst, size_t bytes, int c
 hoccl_result_t hoccl_fanout_launch(const void* src, void* const* dsts, int ndst, size_t bytes, int ctas, hoccl_stream_t stream);
 /* Direct launch of the chain sum of the direct reduce-scatter ("rs_direct"): out[i] = (((s_0[i] + s_1[i]) + ...) + s_{nsrc-1}[i])
  * + local[i], i < count, every add rounded into `dtype`; s_j = first + j * stride_bytes (a multiple of 16), nsrc in 1..63,
- * `ctas` CTAs of 1024 threads.  Device pointers aligned to the element size; out may equal local. */
+ * `ctas` CTAs (512 threads each, three tiles of loads in flight per thread, for up to 7 inbox operands and fewer than 128
+ * CTAs; 1024 threads otherwise).  Device pointers aligned to the element size; out may equal local. */
 hoccl_result_t hoccl_chain_launch(const void* first, size_t stride_bytes, int nsrc, const void* local, void* out, size_t count,
                                   hoccl_dtype_t dtype, int ctas, hoccl_stream_t stream);
 /*

@@ -135,7 +135,7 @@ hoccl_result_t build_graph(hoccl_comm* c, const Plan& P, const std::vector<RGrou
           fill_chain_batch(rg, first, n, P.dtype, P.elem, &cb);
           prepare_chain_batch(&cb, (int)c->sum_ctas);
           args[0] = &cb;
-          kp.func = const_cast<void*>(chain_kernel_entry(P.dtype, &sum_threads));
+          kp.func = const_cast<void*>(chain_kernel_entry(cb, (int)c->sum_ctas, &sum_threads));
           for (size_t i = 0; i < n; i++) bytes += (2.0 + (double)rg.segs[first + i].nsrc) * (double)rg.segs[first + i].bytes;
         }
         kp.gridDim = dim3((unsigned)c->sum_ctas);

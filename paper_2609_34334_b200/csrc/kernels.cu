@@ -146,6 +146,26 @@ __global__ void __launch_bounds__(THREADS, 1) copy_kernel(const __grid_constant_
   }
 }
 
+// One element of a chain segment, element-wise: the same adds in the same order as the vector body.
+template <int DT>
+__device__ __forceinline__ void chain_scalar(const ChainSeg& sg, unsigned long long i) {
+  if (DT == 0) {
+    float acc = static_cast<const float*>(sg.first)[i];
+    for (int q = 1; q < sg.nsrc; q++)
+      acc = __fadd_rn(acc, reinterpret_cast<const float*>(static_cast<const char*>(sg.first) + (size_t)q * sg.stride)[i]);
+    static_cast<float*>(sg.out)[i] = __fadd_rn(acc, static_cast<const float*>(sg.local)[i]);
+  } else {
+    unsigned short acc = static_cast<const unsigned short*>(sg.first)[i];
+    for (int q = 1; q <= sg.nsrc; q++) {
+      const unsigned short b = q < sg.nsrc ? reinterpret_cast<const unsigned short*>(static_cast<const char*>(sg.first) + (size_t)q * sg.stride)[i]
+                                           : static_cast<const unsigned short*>(sg.local)[i];
+      const float s2 = __fadd_rn(__uint_as_float((uint32_t)acc << 16), __uint_as_float((uint32_t)b << 16));
+      acc = __bfloat16_as_ushort(__float2bfloat16_rn(s2));
+    }
+    static_cast<unsigned short*>(sg.out)[i] = acc;
+  }
+}
+
 // Chain sum of the direct reduce-scatter: per element nsrc inbox operands and the local one, added in the ring's order with a
 // rounding into the I/O dtype after every add.  One 16-byte vector per thread and tile; the operands are loaded in batches of
 // up to 8 before they are added, so up to 8 x 16 KiB are in flight per CTA.  Store bound under a CTA budget like every kernel
@@ -199,22 +219,99 @@ __global__ void __launch_bounds__(THREADS, 1) chain_kernel(const __grid_constant
       while (j >= f.spre[k + 1]) k++;
       unsigned long long i = j - f.spre[k];
       if (i >= f.head[k]) i += f.nvec[k] * T::VE;
+      chain_scalar<DT>(batch.seg[k], i);
+    }
+  }
+}
+
+// Software-pipelined form of the chain sum for a compile-time operand count NOPS (inbox operands + the local one) that all
+// segments of the launch share.  Under a CTA budget the chain sum is bound by the bytes one SM keeps in flight: a load takes
+// the better part of a microsecond to come back, so a thread that loads a tile, adds it, stores it and only then loads the
+// next one leaves the memory port idle most of the time.  Here every thread keeps P tiles in registers: the loads of tile
+// t + P - 1 are issued before the adds and the store of tile t, so P - 1 to P tiles of NOPS x 16 bytes per thread are in
+// flight all the time.  That only works when the steady state is straight-line code: with a branch or a segment look-up
+// between the loads and the adds the compiler waits for every outstanding load at the join (measured: 89 GB/s per SM, the
+// rate of ONE tile in flight, whatever P).  So a CTA takes a CONTIGUOUS range of the flattened tile space, walks it segment
+// by segment, and inside a segment the full tiles run through a loop whose body has no branch: unconditional loads, adds,
+// store (measured: 163 GB/s per SM for 8 operands with P = 3 and 512 threads, against 111 for chain_kernel).  The ragged
+// last tile of a segment and ranges shorter than P tiles take a plain guarded path.  The order of the adds and their
+// rounding are those of chain_kernel (operand 0 first, the local contribution last).  Tiles are THREADS vectors.
+template <int DT, int NOPS, int P, int THREADS>
+__global__ void __launch_bounds__(THREADS, 1) chain_pipe_kernel(const __grid_constant__ ChainBatch batch) {
+  using T = Traits<DT>;
+  const Flat& f = batch.flat;
+  const int nseg = batch.nseg;
+  if (batch.smid_out != nullptr && threadIdx.x == 0) {
+    unsigned id;
+    asm volatile("mov.u32 %0, %%smid;" : "=r"(id));
+    batch.smid_out[blockIdx.x] = id;
+  }
+  {
+    const unsigned long long T_all = f.tpre[nseg];
+    // this CTA's share of the flattened tile space: [A, B)
+    const unsigned long long A = T_all / gridDim.x * blockIdx.x + min((unsigned long long)blockIdx.x, T_all % gridDim.x);
+    const unsigned long long B = A + T_all / gridDim.x + (blockIdx.x < T_all % gridDim.x ? 1 : 0);
+    int k = 0;
+    while (k < nseg && f.tpre[k + 1] <= A) k++;
+    for (; k < nseg && f.tpre[k] < B; k++) {
+      const unsigned long long a = (A > f.tpre[k] ? A : f.tpre[k]) - f.tpre[k];                 // tiles [a, b) of segment k
+      const unsigned long long b = (B < f.tpre[k + 1] ? B : f.tpre[k + 1]) - f.tpre[k];
+      const unsigned long long nvec = f.nvec[k];
+      const unsigned long long bf = b < nvec / THREADS ? b : nvec / THREADS;                    // full tiles end here
       const ChainSeg& sg = batch.seg[k];
-      if (DT == 0) {
-        float acc = static_cast<const float*>(sg.first)[i];
-        for (int q = 1; q < sg.nsrc; q++)
-          acc = __fadd_rn(acc, reinterpret_cast<const float*>(static_cast<const char*>(sg.first) + (size_t)q * sg.stride)[i]);
-        static_cast<float*>(sg.out)[i] = __fadd_rn(acc, static_cast<const float*>(sg.local)[i]);
-      } else {
-        unsigned short acc = static_cast<const unsigned short*>(sg.first)[i];
-        for (int q = 1; q <= sg.nsrc; q++) {
-          const unsigned short b = q < sg.nsrc ? reinterpret_cast<const unsigned short*>(static_cast<const char*>(sg.first) + (size_t)q * sg.stride)[i]
-                                               : static_cast<const unsigned short*>(sg.local)[i];
-          const float s2 = __fadd_rn(__uint_as_float((uint32_t)acc << 16), __uint_as_float((uint32_t)b << 16));
-          acc = __bfloat16_as_ushort(__float2bfloat16_rn(s2));
+      const size_t off0 = (size_t)f.head[k] * T::E + (size_t)threadIdx.x * 16;
+      const char* src = static_cast<const char*>(sg.first) + off0;
+      const char* loc = static_cast<const char*>(sg.local) + off0;
+      char* out = static_cast<char*>(sg.out) + off0;
+      const size_t stride = sg.stride;
+      uint4 buf[P][NOPS];
+      auto load = [&](uint4(&bb)[NOPS], unsigned long long t) {
+        const size_t o = (size_t)t * THREADS * 16;
+#pragma unroll
+        for (int q = 0; q < NOPS - 1; q++) bb[q] = __ldcs(reinterpret_cast<const uint4*>(src + (size_t)q * stride + o));
+        bb[NOPS - 1] = __ldcs(reinterpret_cast<const uint4*>(loc + o));
+      };
+      auto finish = [&](const uint4(&bb)[NOPS], unsigned long long t) {
+        uint4 acc = bb[0];
+#pragma unroll
+        for (int q = 1; q < NOPS; q++) acc = DT == 1 ? add_vec_bf16_native(acc, bb[q]) : T::add_vec(acc, bb[q]);
+        *reinterpret_cast<uint4*>(out + (size_t)t * THREADS * 16) = acc;
+      };
+      unsigned long long i = a;
+      if (bf > a && bf - a >= (unsigned long long)P) {
+#pragma unroll
+        for (int p = 0; p < P - 1; p++) load(buf[p], i + p);
+        for (; i + 2 * P - 1 <= bf; i += P) {   // steady state: no branch between a tile's loads and the adds of an older tile
+#pragma unroll
+          for (int p = 0; p < P; p++) {
+            load(buf[(p + P - 1) % P], i + p + P - 1);
+            finish(buf[p], i + p);
+          }
         }
-        static_cast<unsigned short*>(sg.out)[i] = acc;
+#pragma unroll
+        for (int p = 0; p < P - 1; p++) finish(buf[p], i + p);
+        i += P - 1;
       }
+      for (; i < bf; i++) {   // what is left of the full tiles
+        load(buf[0], i);
+        finish(buf[0], i);
+      }
+      if (i < b && i * THREADS + threadIdx.x < nvec) {   // the ragged last tile of the segment
+        load(buf[0], i);
+        finish(buf[0], i);
+      }
+    }
+  }
+  // element-wise items: heads, tails and segments without a common 16-byte phase (as in chain_kernel)
+  {
+    const unsigned long long total = (unsigned long long)gridDim.x * blockDim.x;
+    const unsigned long long S = f.spre[nseg];
+    int k = 0;
+    for (unsigned long long j = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; j < S; j += total) {
+      while (j >= f.spre[k + 1]) k++;
+      unsigned long long i = j - f.spre[k];
+      if (i >= f.head[k]) i += f.nvec[k] * T::VE;
+      chain_scalar<DT>(batch.seg[k], i);
     }
   }
 }
@@ -492,10 +589,43 @@ void prepare_copy_batch(CopyBatch* b, int ctas) {
   fill_flat(&b->flat, b->nseg, tile_v, head, nvec, nscalar);
 }
 
+// Which chain kernel serves a batch.  The software-pipelined form needs one operand count for the whole launch (the usual
+// case: every rank's chain has R - 1 inbox operands and the local one) and is compiled for 2 to 8 operands.  Measured on
+// B200 (8 operands, 25 MiB each, bf16): 163 against 111 GB/s per SM with 8 CTAs, 158 / 107 with 16, 138 / 99 with 32,
+// 113 / 89 with 48, 88 / 80 with 64, 59 / 58 with 96; with 148 CTAs both are HBM bound (5.7 TB/s).  Variants with the same
+// or more bytes in flight (P = 2 with 640 threads, P = 4 with 384, P = 4 and 6 with 256) end at the same 159-163 GB/s per
+// SM with 8 CTAs: that is the SM's memory port at 8 reads : 1 write, no longer the bytes in flight.
+struct ChainVariant {
+  const void* fn;
+  int threads;
+};
+template <int DT>
+static ChainVariant chain_pipe_variant(int nops) {
+  // P x NOPS vectors per thread: 16 to 24, i.e. 128 to 192 KiB per SM with 512 threads
+  switch (nops) {
+    case 2: return {reinterpret_cast<const void*>(&chain_pipe_kernel<DT, 2, 8, 512>), 512};
+    case 3: return {reinterpret_cast<const void*>(&chain_pipe_kernel<DT, 3, 6, 512>), 512};
+    case 4: return {reinterpret_cast<const void*>(&chain_pipe_kernel<DT, 4, 5, 512>), 512};
+    case 5: return {reinterpret_cast<const void*>(&chain_pipe_kernel<DT, 5, 4, 512>), 512};
+    case 6: return {reinterpret_cast<const void*>(&chain_pipe_kernel<DT, 6, 3, 512>), 512};
+    case 7: return {reinterpret_cast<const void*>(&chain_pipe_kernel<DT, 7, 3, 512>), 512};
+    case 8: return {reinterpret_cast<const void*>(&chain_pipe_kernel<DT, 8, 3, 512>), 512};
+    default: return {nullptr, 0};
+  }
+}
+static ChainVariant chain_variant(const ChainBatch& b, int ctas) {
+  ChainVariant plain{b.dtype == 0 ? reinterpret_cast<const void*>(&chain_kernel<0, 1024>) : reinterpret_cast<const void*>(&chain_kernel<1, 1024>), 1024};
+  if (ctas >= 128 || b.nseg <= 0) return plain;
+  const int nops = b.seg[0].nsrc + 1;
+  for (int k = 1; k < b.nseg; k++)
+    if (b.seg[k].nsrc + 1 != nops) return plain;
+  ChainVariant pv = b.dtype == 0 ? chain_pipe_variant<0>(nops) : chain_pipe_variant<1>(nops);
+  return pv.fn ? pv : plain;
+}
+
 void prepare_chain_batch(ChainBatch* b, int ctas) {
-  (void)ctas;
   const int E = b->dtype == 0 ? 4 : 2, VE = 16 / E;
-  const unsigned long long tile_v = 1024;   // one vector per thread and tile
+  const unsigned long long tile_v = (unsigned long long)chain_variant(*b, ctas).threads;   // one vector per thread and tile
   unsigned head[kMaxSegs];
   unsigned long long nvec[kMaxSegs], nscalar[kMaxSegs];
   for (int k = 0; k < b->nseg; k++) {
@@ -510,9 +640,9 @@ cudaError_t launch_chain(const ChainBatch& batch, int ctas, cudaStream_t stream)
   if (batch.nseg <= 0) return cudaSuccess;
   ChainBatch b = batch;
   prepare_chain_batch(&b, ctas);
-  if (b.dtype == 0) chain_kernel<0, 1024><<<ctas, 1024, 0, stream>>>(b);
-  else chain_kernel<1, 1024><<<ctas, 1024, 0, stream>>>(b);
-  return cudaGetLastError();
+  const ChainVariant v = chain_variant(b, ctas);
+  void* args[1] = {&b};
+  return cudaLaunchKernel(v.fn, dim3((unsigned)ctas), dim3((unsigned)v.threads), args, 0, stream);
 }
 
 void prepare_fan_batch(FanBatch* b, int ctas) {
@@ -594,9 +724,10 @@ cudaError_t launch_bf16_add_selftest(unsigned long long* counts, cudaStream_t st
   bf16_add_selftest_kernel<<<65536, 256, 0, stream>>>(counts);
   return cudaGetLastError();
 }
-const void* chain_kernel_entry(int dtype, int* threads) {
-  *threads = 1024;
-  return dtype == 0 ? reinterpret_cast<const void*>(&chain_kernel<0, 1024>) : reinterpret_cast<const void*>(&chain_kernel<1, 1024>);
+const void* chain_kernel_entry(const ChainBatch& batch, int ctas, int* threads) {
+  const ChainVariant v = chain_variant(batch, ctas);
+  *threads = v.threads;
+  return v.fn;
 }
 const void* graph_root_kernel_entry() { return reinterpret_cast<const void*>(&graph_root_kernel); }
 const void* fan_kernel_entry(int ctas, int* threads) {
@@ -620,6 +751,12 @@ cudaError_t preload_kernels() {
     cudaError_t e = cudaFuncGetAttributes(&a, f);
     if (e != cudaSuccess) return e;
   }
+  for (int nops = 2; nops <= 8; nops++)
+    for (const void* f : {chain_pipe_variant<0>(nops).fn, chain_pipe_variant<1>(nops).fn}) {
+      cudaFuncAttributes a;
+      cudaError_t e = cudaFuncGetAttributes(&a, f);
+      if (e != cudaSuccess) return e;
+    }
   return cudaSuccess;
 }
 

@@ -154,7 +154,8 @@ cudaError_t launch_sum(const SumBatch& batch, int ctas, cudaStream_t stream);
 cudaError_t launch_copy(const CopyBatch& batch, int ctas, cudaStream_t stream);
 cudaError_t launch_chain(const ChainBatch& batch, int ctas, cudaStream_t stream);
 void prepare_chain_batch(ChainBatch* batch, int ctas);
-const void* chain_kernel_entry(int dtype, int* threads);
+// kernel and thread count that serve `batch` with `ctas` CTAs (the batch must have been prepared for the same `ctas`)
+const void* chain_kernel_entry(const ChainBatch& batch, int ctas, int* threads);
 // counts: two device words, zeroed by the caller; see bf16_add_selftest_kernel
 cudaError_t launch_bf16_add_selftest(unsigned long long* counts, cudaStream_t stream);
 cudaError_t launch_fan(const FanBatch& batch, int ctas, cudaStream_t stream);

@@ -162,12 +162,19 @@ def test_native_bf16_add_equals_the_reference_add_for_all_operand_pairs():
 
 
 @pytest.mark.parametrize("dtype", ["fp32", "bf16"])
-@pytest.mark.parametrize("ctas", [1, 8, 148])
+@pytest.mark.parametrize("ctas", [1, 3, 8, 148])
 def test_chain_kernel_against_the_oracles_chain(oracle, dtype, ctas):
     """hoccl_chain_launch against the oracle's closed form of the ring order, ((x_{c+1} + x_{c+2}) + ...) + x_c with a rounding
-    after every add: R = 2..12 operands, ragged lengths, operands off the 16-byte grid together (vector path) or not."""
+    after every add: R = 2..12 operands (every operand count the software-pipelined kernel is compiled for, and beyond it the
+    plain one), ragged lengths, operands off the 16-byte grid together (vector path) or not.  The lengths give a CTA fewer
+    tiles than its pipeline is deep, exactly as many, many more with a ragged last tile, and an uneven split over 3 CTAs."""
     e = W.elem_size(dtype)
-    for R, n in [(2, 1), (3, 1023), (8, 4096 * 5 + 3), (8, 1_000_003), (12, 70_001)]:
+    vec = 16 // e
+    tile = 512 * vec                      # elements of one tile of the pipelined kernel
+    cases = [(2, 1), (3, 1023), (8, 4096 * 5 + 3), (8, 1_000_003), (12, 70_001),
+             (4, 3 * tile), (5, 2 * tile + 7), (6, 9 * tile + vec), (7, 25 * tile - vec + 1), (8, 3 * ctas * tile),
+             (8, (3 * ctas + 1) * tile + 5), (2, 40 * tile + 3), (3, 17 * tile)]
+    for R, n in cases:
         xs = W.rank_inputs("uniform", 230 + R, R, n, dtype)
         c = R // 2
         want = oracle.chain_sum(xs, c, 0, n)
