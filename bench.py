@@ -190,6 +190,7 @@ def main():
     import torch
 
     from paper_2609_34334_b200 import binding as hb
+    from paper_2609_34334_b200 import diag as hd
     from paper_2609_34334_b200 import workloads as W
 
     if not torch.cuda.is_available():
@@ -424,18 +425,18 @@ def main():
         o = torch.empty(big, dtype=torch.bfloat16, device="cuda")
         # SMs used, counted: every CTA of an 8-CTA SUM launch (the launch shape of the timed path) reports its SM id
         ids = torch.full((8,), -1, dtype=torch.int32, device="cuda")
-        if hb.kernel_sms("sum", a, b2, o, 8 * 3276800, dtype, 8, ids, stream) == hb.OK:
+        if hd.kernel_sms("sum", a, b2, o, 8 * 3276800, dtype, 8, ids, stream) == hb.OK:
             stream.synchronize()
             line["sms_used"]["distinct_sms_of_one_sum_launch"] = len(set(ids.cpu().tolist()))
         full = {}
         for ctas in (8, 16, 32, 48, 64, 96, 128, 148, 296, 592):
             for _ in range(3):
-                hb.sum_launch(a, b2, o, big, dtype, ctas, stream)
+                hd.sum_launch(a, b2, o, big, dtype, ctas, stream)
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record(stream)
             reps = 3 if ctas == 8 else 10
             for _ in range(reps):
-                hb.sum_launch(a, b2, o, big, dtype, ctas, stream)
+                hd.sum_launch(a, b2, o, big, dtype, ctas, stream)
             e1.record(stream)
             stream.synchronize()
             full[str(ctas)] = 3.0 * big * 2 / (e0.elapsed_time(e1) / 1e3 / reps) / 1e9
@@ -469,7 +470,7 @@ def main():
                                 "single_thread_ms_per_step": t_single * 1e3}
 
         if not args.no_extras:
-            line["extras"] = extras(hb, W, torch, np, new_comm, step, timed, stream, R, S, n, dtype, peaks, send_sets, recv_sets)
+            line["extras"] = extras(hb, hd, W, torch, np, new_comm, step, timed, stream, R, S, n, dtype, peaks, send_sets, recv_sets)
 
     comm.destroy()
     if world.rank == 0:
@@ -534,7 +535,7 @@ def small_case(hb, W, torch, np, stream):
     return rows
 
 
-def extras(hb, W, torch, np, new_comm, step, timed, stream, R, S, n, dtype, peaks, send_sets, recv_sets):
+def extras(hb, hd, W, torch, np, new_comm, step, timed, stream, R, S, n, dtype, peaks, send_sets, recv_sets):
     """Context lines: path / CTA-budget variants, whether a move needs an SM, p2p, and the co-running GEMM probe."""
     out = {}
     k, w = 40, 5
@@ -687,19 +688,19 @@ def extras(hb, W, torch, np, new_comm, step, timed, stream, R, S, n, dtype, peak
     src = send_sets[0][0]
     dst = recv_sets[0][0]
     nb = min(64 << 20, src.numel() * 2)
-    ce_needs, ce_end = cm.probe_move_needs_sm(hb.PATH_CE, dst, src, nb, 3000)
-    sm_needs, sm_end = cm.probe_move_needs_sm(hb.PATH_SM, dst, src, nb, 3000)
+    ce_needs, ce_end = hd.probe_move_needs_sm(cm, hb.PATH_CE, dst, src, nb, 3000)
+    sm_needs, sm_end = hd.probe_move_needs_sm(cm, hb.PATH_SM, dst, src, nb, 3000)
     pinned = torch.empty(8 << 20, dtype=torch.uint8).pin_memory()
-    h2d_needs, h2d_end = cm.probe_move_needs_sm(hb.PATH_CE, dst, pinned, pinned.numel(), 3000)
+    h2d_needs, h2d_end = hd.probe_move_needs_sm(cm, hb.PATH_CE, dst, pinned, pinned.numel(), 3000)
     cm.set_host_staging(host_stage)
-    hb_needs, hb_end = cm.probe_move_needs_sm(hb.PATH_CE_HOST, dst, src, min(nb, 16 << 20), 3000)
+    hb_needs, hb_end = hd.probe_move_needs_sm(cm, hb.PATH_CE_HOST, dst, src, min(nb, 16 << 20), 3000)
     out["move_needs_sm"] = {"CE_HOST_bounce_16MiB": hb_needs, "CE_HOST_move_end_us": hb_end,
                             "CE_driver_copy_same_device_64MiB": ce_needs, "CE_move_end_us": ce_end, "SM_copy_kernel": sm_needs,
                             "SM_move_end_us": sm_end, "control_pinned_host_to_device_8MiB": h2d_needs,
                             "control_move_end_us": h2d_end, "occupancy_kernel_us": 3000,
                             "note": "true = the move finished only after a kernel holding every SM had ended"}
     out["copy_routes_16MiB"] = [{"route": n_, "needs_sm": s_, "end_us": round(t_, 1)}
-                                for n_, s_, t_ in cm.probe_copy_routes(dst, src, min(nb, 16 << 20), 3000)]
+                                for n_, s_, t_ in hd.probe_copy_routes(cm, dst, src, min(nb, 16 << 20), 3000)]
     # host cost of one call with an idle queue (the paper's CPU launch overhead axis)
     host_us = {}
     for label, use_graph in (("graph_replay", 1), ("stream_executor", 0)):

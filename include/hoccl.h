@@ -30,6 +30,7 @@
  *    attached with hoccl_comm_set_scratch / hoccl_comm_set_staging.  The two exceptions are stated where
  *    they apply: handshake mode allocates 512 bytes once, and hoccl_allreduce_static uses a fixed array
  *    that is part of the library image.
+ *  - Probes, self-tests, direct kernel launches and plan inspection are declared in hoccl_diag.h.
  *  - The CUDA device must be present: every entry point that touches the device returns
  *    HOCCL_ERR_CUDA otherwise.  There is no CPU fallback.
  */
@@ -109,7 +110,12 @@ typedef struct {
 hoccl_result_t hoccl_comm_init(hoccl_comm_t* comm, int R, int device);
 
 /* Frees host state, streams, events and cached graphs.  Synchronises the internal streams.
- * HOCCL_ERR_PENDING (and nothing freed) if unmatched send/recv posts remain. */
+ * HOCCL_ERR_PENDING (and nothing freed) if unmatched send/recv posts remain.
+ * Handshake mode: hand-overs that are still open after one watchdog period (a stream that has not reached its call yet
+ * because it is busy with earlier work, a schedule that has not finished) are released by force, so that no stream
+ * waits on a communicator that is gone: such a stream goes on WITHOUT the result of that call, everything is freed as
+ * usual, and the call returns HOCCL_ERR_TIMEOUT to say so.  (The few hundred bytes of pinned counters stay allocated
+ * for the life of the process in that case: the late stream still reads them when it gets there.) */
 hoccl_result_t hoccl_comm_destroy(hoccl_comm_t comm);
 
 /* Upper bound of the scratch bytes any collective needs for up to `max_count` elements of `dtype`
@@ -166,19 +172,32 @@ hoccl_result_t hoccl_comm_set_path(hoccl_comm_t comm, hoccl_path_t path);
  *                moved, same bits; the moves of all stages can be in flight together.  HOCCL_PATH_SM: one batched launch
  *                in which every chunk is read once and stored R-1 times (S R instead of 2 S (R-1) bytes of traffic);
  *                HOCCL_PATH_CE_HOST: a chunk goes out to the host staging once and comes back R-1 times.
- *                0 = the ring all-gather (default).  2 = automatic: direct where it was measured faster on B200 (always on
+ *                0 = the ring all-gather.  2 (default) = automatic: direct where it was measured faster on B200 (always on
  *                HOCCL_PATH_SM and HOCCL_PATH_CE_HOST; on HOCCL_PATH_CE while a ring chunk is at most 64 MiB), ring elsewhere.
  *  "rs_direct"   1 = the reduce-scatter (alone or as the first half of an all-reduce) runs as the stage decomposition of its
  *                traffic matrix (paper Sec. 3.4: rank r owes its contribution to chunk d to rank d): R-1 contention-free
  *                permutation stages r -> r+k that wait for nothing, into R-1 inbox slots of the owner, and then ONE sum
  *                per rank that adds the R-1 arrived contributions and its own in the ring's order, rounding into the I/O
- *                dtype after every add (chain_kernel, "sum_ctas" CTAs).  Rank local, the ring's bits; every output byte is
+ *                dtype after every add (the chain sum, "sum_ctas" CTAs).  Rank local, the ring's bits; every output byte is
  *                written once instead of R-1 times: 2 S (R-1) + S (R+1) bytes of traffic instead of 5 S (R-1), and under
  *                an SM budget, where a sum is bound by the SMs' memory ports, R reads + 1 write per output instead of
  *                (R-1) x (2 reads + 1 write).  Needs hoccl_scratch_bytes_direct bytes of scratch (R-1 slots per rank
- *                instead of 2).  "forward" and "fused" do not apply to it.  0 = the ring reduce-scatter (default).  2 = automatic:
- *                direct whenever the attached scratch is large enough for it (it was measured faster than the ring at every
- *                size and on every path), the ring otherwise.
+ *                instead of 2); with less the call returns HOCCL_ERR_SCRATCH.  0 = the ring reduce-scatter, step by step.
+ *                2 (default) = automatic: direct whenever the attached scratch is large enough for it and neither "forward",
+ *                "fused" nor "onepass" is set (it was measured faster than the ring at every size and on every path), the ring
+ *                otherwise.  So a communicator with hoccl_scratch_bytes of scratch runs the ring, one with
+ *                hoccl_scratch_bytes_direct runs the direct form; the bits are the same.
+ *  "ce_small_bytes" on HOCCL_PATH_CE a call whose per-rank message (S in the convention of each collective: all-reduce
+ *                count, reduce-scatter / all-gather / all-to-all R * count elements) is at most this many bytes issues its
+ *                moves as batched launches of the SM copy kernel with "ce_small_ctas" CTAs instead of driver copies, i.e.
+ *                it runs on the route of HOCCL_PATH_SM (hoccl_last_stats shows the launches).  Inside one device a driver
+ *                copy spares no SM (hoccl_probe_move_needs_sm) and takes microseconds to start, so below a crossover the
+ *                kernel is a pure gain: measured on B200 with the default schedule and 8-CTA sums, R = 8 bf16 all-reduce of
+ *                4 KiB 34 -> 10 us, 1 MiB 48 -> 25 us, 4 MiB 88 -> 54 us, 8 MiB 107 -> 97 us, equal from 16 MiB on; R = 4 fp32
+ *                all-reduce of 4 MiB 37 -> 33 us.  Default 8 MiB; 0 = driver copies at every size.  "HOCCL_PATH_CE" therefore
+ *                means: the copy route above this size.  Not applied to hoccl_host_allreduce, send/recv or hoccl_alltoallv.
+ *  "ce_small_ctas" CTAs of those launches, 1..1024 (default 148: like the driver's own copies they may use the whole GPU,
+ *                for tens of microseconds)
  *  "order_kernels" 1 (default) = on the copy routes the graph executor puts an empty one-warp kernel in front of a graph's
  *                first copies and behind every group of copies that other copies (or the end of the graph) wait for.
  *                Measured on B200: a copy node that waits for earlier stream work or for several copy nodes starts ~4 us
@@ -196,31 +215,47 @@ hoccl_result_t hoccl_comm_set_path(hoccl_comm_t comm, hoccl_path_t path);
  *                Every barrier wait is bounded; a wait that runs out ends the kernel and is reported by
  *                hoccl_comm_async_error as HOCCL_ERR_TIMEOUT.  The library allocates 16 bytes of device memory and 4 bytes
  *                of pinned host memory of its own on first use (the third exception to "device memory is the caller's").
- *                Ignored on the other paths, in handshake mode, and for plans too large for one launch (more than 480
- *                chunk operations or 96 steps: an all-reduce beyond 12 ranks), which run as a graph.  0 = off (default).
+ *                Refused on the other paths and in handshake mode (see the rules below); plans too large for one launch (more
+ *                than 480 chunk operations or 96 steps: an all-reduce beyond 12 ranks) run as a graph.  0 = off (default).
  *  "host_pieces" pieces per ring chunk of the pipelined hoccl_host_allreduce (1..64, default 8; 1 = not pipelined)
  *  "use_graph"   1 = run a cached CUDA graph built from the plan (default), 0 = streams and events
- *  "handshake"   1 = the paper's stream manager (Sec. 3.2, Listing 1): instead of launching into the caller's
- *                stream, the call enqueues four stream memory operations (write start flag, wait for the CPU's
- *                acknowledgement, wait for the finish flag, reset it) and hands the schedule to a CPU proxy thread
- *                that polls the flags in pinned host memory, runs the schedule on an internal stream and hands the
- *                stream back.  send/recv posts are matched by the proxy AFTER each stream has reached its post, so a
+ *  "handshake"   1 = the paper's stream manager (Sec. 3.2): instead of launching into the caller's stream, the call
+ *                enqueues three stream memory operations (write "hand-over n has arrived", wait for "hand-over n is
+ *                released", write "hand-over n is behind me"; the counters live in pinned host memory and only grow) and
+ *                hands the schedule to a CPU proxy thread that polls the counters, runs the schedule on an internal stream
+ *                and then releases the caller's stream.  send/recv posts are matched by the proxy AFTER each stream has reached its post, so a
  *                post may wait for a partner that is posted later (the paper's semantics, Sec. 3.3.2); count/dtype
  *                mismatches and unmatched posts are then reported asynchronously (hoccl_comm_async_error).
  *                0 = off (default).  Results are identical bit for bit.  Handshake mode needs HOCCL_PATH_SM: calls on
- *                the CE path return HOCCL_ERR_UNSUPPORTED, because on one device a driver copy issued by the proxy
+ *                the other paths return HOCCL_ERR_UNSUPPORTED, because on one device a driver copy issued by the proxy
  *                can queue up behind copies that the parked stream itself has waiting and then never start.
  *                The two sides of a send/recv must be
  *                posted on different streams (a stream parked in its own post cannot reach the partner's).  The
- *                first use creates the proxy: a thread, pinned host memory for 64 flag pairs and 512 bytes of
+ *                first use creates the proxy: a thread, pinned host memory for 64 sets of counters and 512 bytes of
  *                device memory (one of the library's own device allocations stated in this header), and loads every kernel, because
  *                first-use work in the driver must not happen while a stream is parked.
- *  "watchdog_ms" handshake mode: after this long (default 10000) an unmatched post is released with an abort
- *                value and HOCCL_ERR_TIMEOUT is recorded, so no stream can wait on this library forever
+ *  "watchdog_ms" handshake mode: after this long (default 10000) the stream of an unmatched post is released without its
+ *                transfer and HOCCL_ERR_TIMEOUT is recorded, so no stream can wait on this library forever
+ *  "p2p_strict"  1 = send/recv posts go through the CPU proxy as in handshake mode while collectives are launched directly:
+ *                a post then holds its stream at the post until the transfer is done, whichever side posts first (the
+ *                paper's semantics, Sec. 3.3.2), instead of parking on the host (see hoccl_send).  Needs HOCCL_PATH_SM,
+ *                like handshake mode.  0 = off (default).
  *  "profile"     1 = time every SUM launch with CUDA events; read the totals with hoccl_last_stats after
  *                synchronising (with graphs only the latest replay of each cached graph is readable, so
  *                read after every step)
- * None of them changes a single result bit.  Errors: UNSUPPORTED (unknown key), INVALID_ARG (range).
+ * How the settings combine (one rule set, applied by every collective before it plans; hoccl_options_resolve in
+ * hoccl_diag.h evaluates it without a device).  A value of 1 asks for something, 2 is automatic and yields to whatever was
+ * asked for; a combination that does not fit together makes the CALL return HOCCL_ERR_UNSUPPORTED with nothing enqueued,
+ * it is never changed silently:
+ *   - "handshake" needs HOCCL_PATH_SM and cannot be combined with "onepass" or "fused" (the proxy replays graphs);
+ *   - "fused" is an executor of HOCCL_PATH_SM: refused on the other paths; refused with "rs_direct" = 1 (the one-kernel
+ *     form has no chain phase); it ignores "use_graph" and is not used by hoccl_host_allreduce; plans beyond its capacity
+ *     (see "fused") run as a graph;
+ *   - "onepass" applies to all-reduce and reduce-scatter calls, ignores the path, and for those calls is refused together
+ *     with "forward", "fused", "rs_direct" = 1 or (all-reduce) "ag_direct" = 1; other collectives ignore it;
+ *   - "forward" applies to all-reduce and reduce-scatter calls and is refused with "rs_direct" = 1;
+ *   - "use_graph" chooses between graph replay and the stream executor where neither "handshake" nor "fused" decides.
+ * None of them changes a single result bit.  Errors of set_param itself: UNSUPPORTED (unknown key), INVALID_ARG (range).
  */
 hoccl_result_t hoccl_comm_set_param(hoccl_comm_t comm, const char* key, long value);
 hoccl_result_t hoccl_comm_get_param(hoccl_comm_t comm, const char* key, long* value);
@@ -295,10 +330,14 @@ hoccl_result_t hoccl_alltoallv(const void* const* send, const size_t* sendcounts
  * Non-blocking matched send/recv between logical ranks (paper Sec. 3.3.2 "Intra-node
  * Communication": a post does not block the caller while the peer has not posted; the transfer
  * happens once both sides are known).  Posts are matched per (src, dst) pair in FIFO order; either
- * side may come first.  The first post parks {buffer, count, dtype, stream} and enqueues nothing.
- * The second post enqueues ONE device-to-device move of count elements that runs after both
- * posting streams have reached their post (for the first poster: its stream position at the time of
- * the match) and that both streams then wait for.
+ * side may come first.  The first post parks {buffer, count, dtype, stream} on the host and marks its place in its
+ * stream with an event; nothing else is enqueued.  The second post enqueues ONE device-to-device move of count
+ * elements that runs after both streams have reached their posts and that both streams then wait for.
+ * What this cannot give: work that the FIRST poster enqueues on its stream between its own post and the partner's is
+ * not ordered against the transfer (a stream cannot be made to wait, after the fact, for something that is enqueued
+ * later): a consumer of the receive buffer, or a writer of the send buffer, must be enqueued after the partner has
+ * posted.  Callers that cannot arrange that set "p2p_strict" = 1 (or "handshake" = 1): the post then holds its stream
+ * until the transfer is done, whoever posts first, bounded by the watchdog.
  * Mismatch of count or dtype at match time: HOCCL_ERR_MISMATCH from the second call, nothing is
  * enqueued and the parked post is dropped.  Unmatched posts can never hang a stream; their number is
  * hoccl_comm_pending().  Errors: INVALID_ARG (NULL buf, rank out of range, src == dst), CUDA.
@@ -311,16 +350,13 @@ int hoccl_comm_pending(hoccl_comm_t comm);
 /* First asynchronous failure: handshake mode, as seen by the proxy (OK, TIMEOUT, MISMATCH or CUDA); "fused" setting,
  * TIMEOUT if a barrier wait of the whole-collective kernel ran out.  clear != 0 resets it. */
 hoccl_result_t hoccl_comm_async_error(hoccl_comm_t comm, int clear);
-/*
- * Failure-detection self-test of the "fused" kernel's bounded waits, without faulting the GPU: enqueues the
- * whole-collective kernel with two copy phases (first and second half of `bytes`, src -> dst, device pointers, bytes a
- * multiple of 32) separated by a grid barrier that waits for one arrival more than the grid delivers.  Every CTA polls
- * for its bounded number of rounds (a second or two), gives up, the kernel ends by itself, the second half is NOT
- * copied, and hoccl_comm_async_error then reports HOCCL_ERR_TIMEOUT; the barrier words are clean for the next call.
- */
-hoccl_result_t hoccl_selftest_barrier_timeout(hoccl_comm_t comm, void* dst, const void* src, size_t bytes, hoccl_stream_t stream);
 /* Handshake mode: number of stream hand-overs the proxy has served so far. */
 long hoccl_comm_handshakes(hoccl_comm_t comm);
+/* Handshake mode: how busy the proxy thread is.  *busy_us = time it spent working (launching schedules and moves, writing
+ * counters), *span_us = wall time from the first task it accepted to its latest release, since creation or the last reset
+ * (reset != 0 zeroes both after reading).  1 - busy / span is the share of the time the thread merely polled: the analogue
+ * of the CPU slack the paper reports for its proxy (Sec. 5 "End-to-end workloads").  Both 0 without a proxy. */
+hoccl_result_t hoccl_comm_proxy_stats(hoccl_comm_t comm, double* busy_us, double* span_us, int reset);
 
 /* ---------------------------------------------------------------- host-buffer entry points ----- */
 
@@ -381,167 +417,13 @@ hoccl_result_t hoccl_host_allreduce(const void* const* h_send, void* const* h_re
 hoccl_result_t hoccl_allreduce_static(const void* const* send, void* const* recv, size_t count, hoccl_dtype_t dtype,
                                       hoccl_op_t op, int R, hoccl_stream_t stream);
 
-/* ---------------------------------------------------------------- diagnostics ------------------ */
+/* ---------------------------------------------------------------- errors and statistics -------- */
 
 const char* hoccl_error_string(hoccl_result_t code);
 /* Text of the last CUDA error seen by this communicator ("" if none); valid until the next call. */
 const char* hoccl_last_cuda_error(hoccl_comm_t comm);
 hoccl_result_t hoccl_last_stats(hoccl_comm_t comm, hoccl_stats_t* out);
 hoccl_result_t hoccl_profile_reset(hoccl_comm_t comm);
-
-/*
- * Measures whether a MOVE of `bytes` bytes on the given path needs an SM.  A kernel that fills every
- * thread slot of every SM sleeps for a fixed `spin_us` microseconds (bounded; it never waits on
- * anything) while the move is enqueued on another stream; *needs_sm is 1 if the move finished only
- * after that kernel ended, 0 if it finished while all SMs were taken.  *move_end_us is the move's
- * completion time measured from the kernel's start.  Synchronises the device.  This is the
- * single-GPU form of the paper's claim that copy-engine transfers occupy no SM (Sec. 2.3).
- * src and dst are device buffers of at least `bytes` bytes.  On the CE path src may also be PINNED HOST
- * memory: a host-to-device copy is driven by a copy engine, which makes it the control of the measurement
- * (it must report needs_sm = 0).
- */
-hoccl_result_t hoccl_probe_move_needs_sm(hoccl_comm_t comm, hoccl_path_t path, void* dst, const void* src, size_t bytes,
-                                         int spin_us, int* needs_sm, double* move_end_us);
-
-/*
- * The same measurement for every way the CUDA API offers to move bytes inside one device, one after the other:
- * cudaMemcpyAsync, cudaMemcpyPeerAsync with both ends on this device, cuMemcpyDtoDAsync, a memcpy node of a CUDA
- * graph, cudaMemcpy2DAsync, cudaMemsetAsync, this library's copy_kernel, and as controls a 32-bit stream memory
- * write (what the paper's handshake uses, Listing 1) and, when pinned host staging is attached
- * (hoccl_comm_set_host_staging, at least `bytes` bytes), a copy in each direction between device and pinned host.
- * Writes one record per route that could be tried (at most max_out) and their number to *n_out.
- * dst and src are disjoint device buffers of `bytes` bytes (bytes >= 4; dst is overwritten).  Synchronises the device.
- * Errors: INVALID_ARG (null pointer, bytes < 4, spin_us outside [100, 20000]), CUDA.
- */
-typedef struct {
-  char name[56];   /* which route */
-  int needs_sm;    /* 1: finished only after the SM-occupying kernel ended */
-  double end_us;   /* completion time, measured from the start of that kernel */
-} hoccl_route_probe_t;
-hoccl_result_t hoccl_probe_copy_routes(hoccl_comm_t comm, void* dst, const void* src, size_t bytes, int spin_us,
-                                       hoccl_route_probe_t* out, int max_out, int* n_out);
-
-/*
- * Direct launches of the two kernels (used by kernel-level tests and roofline measurements).
- *  hoccl_sum_launch : out[i] = round_to_dtype(float(inbox[i]) + float(local[i])), i < count, with `ctas` CTAs.
- *  hoccl_copy_launch: dst bytes <- src bytes with `ctas` CTAs.
- *  hoccl_fanout_launch: dsts[d] bytes <- src bytes for every d < ndst with `ctas` CTAs; every source byte is read once
- *                    and stored ndst times (the move of the direct all-gather on the SM path, see "ag_direct").  `dsts`
- *                    is a HOST array of ndst (1..256) device pointers; destinations must not overlap the source or each
- *                    other.  Destinations whose address differs from the source's modulo 16 are copied byte by byte.
- * All pointers are device pointers aligned to the element size (any byte alignment for the copies).
- */
-hoccl_result_t hoccl_sum_launch(const void* inbox, const void* local, void* out, size_t count, hoccl_dtype_t dtype,
-                                int ctas, hoccl_stream_t stream);
-hoccl_result_t hoccl_copy_launch(const void* src, void* dst, size_t bytes, int ctas, hoccl_stream_t stream);
-hoccl_result_t hoccl_fanout_launch(const void* src, void* const* dsts, int ndst, size_t bytes, int ctas, hoccl_stream_t stream);
-/* Direct launch of the chain sum of the direct reduce-scatter ("rs_direct"): out[i] = (((s_0[i] + s_1[i]) + ...) + s_{nsrc-1}[i])
- * + local[i], i < count, every add rounded into `dtype`; s_j = first + j * stride_bytes (a multiple of 16), nsrc in 1..63,
- * `ctas` CTAs (512 threads each, three tiles of loads in flight per thread, for up to 7 inbox operands and fewer than 128
- * CTAs; 1024 threads otherwise).  Device pointers aligned to the element size; out may equal local. */
-hoccl_result_t hoccl_chain_launch(const void* first, size_t stride_bytes, int nsrc, const void* local, void* out, size_t count,
-                                  hoccl_dtype_t dtype, int ctas, hoccl_stream_t stream);
-/*
- * "SMs used", counted rather than inferred (the paper's Table 1 counts the SMs that communication kernels occupy):
- * launches the SUM kernel (kind 0: out = a + b over bytes / sizeof(dtype) elements) or the copy kernel (kind 1:
- * out <- a, b ignored) with `ctas` CTAs, and every CTA additionally stores the id of the SM it runs on (%smid) to
- * smid_out[block index], a device array of `ctas` 32-bit words.  The number of distinct values is the number of SMs
- * the launch occupied.  Same kernels and launch shapes as the collectives use.
- */
-/*
- * Memory-port probe behind the 8-SM ceiling quoted for the SUM: `ctas` CTAs of 1024 threads only read (mode 0) or only
- * write (mode 1) the device buffer `buf` (16-byte aligned, at least 128 KiB; whole 128 KiB tiles are walked) with 16-byte
- * accesses, 8 in flight per thread.  `sink` is a device word the read mode may write once.  Timed by the caller; together
- * with hoccl_copy_launch (1 read : 1 write) and hoccl_sum_launch (2 : 1) it gives what one SM's memory port carries.
- */
-hoccl_result_t hoccl_port_probe(int mode, void* buf, size_t bytes, int ctas, unsigned int* sink, hoccl_stream_t stream);
-/*
- * Host only (no device needed): the flattened view the host passes to a batched SUM (kind 0) or copy (kind 1) launch for
- * `nseg` segments given by their ADDRESSES as integers (a, b, out; b unused for the copy) and lengths (elements for the
- * SUM, bytes for the copy) under the kernel shape that `ctas` selects.  Per segment: head (element-wise items before the
- * 16-byte vector body), nvec (vectors in the body), and the running totals of tiles and of element-wise items;
- * *tile_vectors is the tile size in vectors.  The kernels trust this view for every address they form, so tests check its
- * invariants on the CPU: nothing is read or written.
- */
-hoccl_result_t hoccl_flatten_inspect(int kind, hoccl_dtype_t dtype, int ctas, int nseg, const uint64_t* a_addr, const uint64_t* b_addr,
-                                     const uint64_t* out_addr, const uint64_t* len, uint64_t* tiles_end, uint64_t* scalars_end,
-                                     uint64_t* nvec, uint32_t* head, uint64_t* tile_vectors);
-/*
- * Host only (no device needed): how a group of `n` moves, given by their ADDRESSES as integers (src[i] -> dst[i], len[i]
- * bytes), is packed into fan-out launches.  Moves with the same source, length and 16-byte phase of the destination share
- * one segment (one read, one store per destination); a launch carries at most 32 segments and 256 destinations.
- * Output, one entry per segment in launch order (arrays of capacity seg_cap): its launch index, source, length, number
- * of destinations, head / nvec of its split under the kernel shape `ctas` selects; its destinations follow each other in
- * dst_out (capacity n).  *n_seg = 0 means no source repeats: the moves go as plain copies.  Nothing is read or written.
- */
-hoccl_result_t hoccl_fanout_inspect(int n, const uint64_t* src, const uint64_t* dst, const uint64_t* len, int ctas, int seg_cap,
-                                    int* seg_launch, uint64_t* seg_src, uint64_t* seg_len, int* seg_ndst, uint32_t* seg_head,
-                                    uint64_t* seg_nvec, uint64_t* dst_out, int* n_seg, int* n_launch);
-/*
- * Self-test of the arithmetic: the chain sum of the direct reduce-scatter adds bf16 operands with the native packed add
- * (add.rn.bf16x2); this call compares it on the device with the reference add of every SUM (binary32 add of the widened
- * operands, rounded to nearest even into bf16) for ALL 2^32 pairs of bf16 bit patterns.  counts: DEVICE array of two 64-bit
- * words, zeroed by the caller; after the stream has run it holds {pairs whose results differ, pairs where both results are
- * NaN with different payloads}.  Both must be 0.
- */
-hoccl_result_t hoccl_selftest_bf16_add(unsigned long long* counts, hoccl_stream_t stream);
-hoccl_result_t hoccl_kernel_sms(int kind, const void* a, const void* b, void* out, size_t bytes, hoccl_dtype_t dtype, int ctas,
-                                unsigned int* smid_out, hoccl_stream_t stream);
-
-/* ---------------------------------------------------------------- plan inspection (host only) --- */
-
-/*
- * The planner (paper Sec. 3.4: a collective becomes stages of point-to-point flows that are cut into
- * chunks for the copy queue) is pure host code; these calls expose its output so that it can be
- * checked without a GPU.  Addresses in a plan are byte offsets: buffer kinds below say what they are
- * relative to.
- */
-typedef enum { HOCCL_PLAN_ALLREDUCE = 0, HOCCL_PLAN_REDUCE_SCATTER = 1, HOCCL_PLAN_ALLGATHER = 2, HOCCL_PLAN_ALLTOALL = 3,
-               HOCCL_PLAN_ALLREDUCE_FWD = 4, HOCCL_PLAN_REDUCE_SCATTER_FWD = 5, /* the "forward" variants */
-               HOCCL_PLAN_ALLREDUCE_AGD = 6, HOCCL_PLAN_ALLGATHER_DIRECT = 7,   /* the "ag_direct" variants */
-               HOCCL_PLAN_ALLREDUCE_FWD_AGD = 8 /* both */ } hoccl_plan_kind_t;
-/* General form: a base kind (0..3) OR-ed with flags; the numbered variants above are shorthands. */
-typedef enum { HOCCL_PLAN_FLAG_FORWARD = 16, HOCCL_PLAN_FLAG_AG_DIRECT = 32, HOCCL_PLAN_FLAG_RS_DIRECT = 64 /* "rs_direct" */ } hoccl_plan_flag_t;
-/* CHAIN: out = (((s_0 + s_1) + ...) + s_{nsrc-1}) + local, every add rounded into the I/O dtype; s_j at src_off + j * src_stride */
-typedef enum { HOCCL_OP_MOVE = 0, HOCCL_OP_SUM = 1, HOCCL_OP_CHAIN = 2 } hoccl_plan_op_kind_t;
-typedef enum { HOCCL_BUF_SEND = 0, HOCCL_BUF_RECV = 1, HOCCL_BUF_INBOX = 2, HOCCL_BUF_PARTIAL = 3 } hoccl_buf_kind_t;
-
-typedef struct {
-  int kind;      /* hoccl_plan_op_kind_t */
-  int phase;     /* 0 reduce-scatter, 1 all-gather, 2 own-chunk / own-block copy, 3 all-to-all stage */
-  int step;      /* ring step s (all-to-all: stage k, destination = rank + k; direct all-gather: stage k - 1) */
-  int piece;     /* pipeline piece index */
-  int rank;      /* MOVE: source rank; SUM: the rank that sums */
-  int dst_rank;  /* MOVE: destination rank; SUM: same as rank (forward variants: the rank whose slot receives the result) */
-  int chunk;     /* ring chunk index */
-  int src_buf, dst_buf, local_buf; /* hoccl_buf_kind_t; local_buf only for SUM */
-  uint64_t src_off, dst_off, local_off; /* byte offsets from the start of those buffers (scratch: from the start of the rank's slot) */
-  uint64_t bytes;
-  int group;     /* ops of one group are issued together (one batched kernel launch or R copies) */
-  int nsrc;      /* CHAIN: number of inbox operands (R-1); 1 otherwise */
-  uint64_t src_stride; /* CHAIN: bytes between consecutive inbox operands (one scratch slot) */
-} hoccl_plan_op_t;
-
-typedef struct hoccl_plan* hoccl_plan_t;
-
-/* Builds the plan for `kind` over R ranks.  `count` as in the collective; in_place as defined at the top of
- * this file; piece_bytes / max_pieces as the parameters of the same name.  send_align: HOST array of R bytes,
- * the low 4 bits of each rank's send pointer (NULL = all 16-byte aligned); it only decides where inside its
- * scratch region a piece is placed so that SUM operands share their 16-byte phase.  Free with hoccl_plan_destroy. */
-hoccl_result_t hoccl_plan_build(hoccl_plan_t* plan, int kind, int R, size_t count, hoccl_dtype_t dtype, int in_place,
-                                size_t piece_bytes, int max_pieces, const unsigned char* send_align);
-/* Bytes of one rank's scratch slot (inbox or partial) under this plan.  Rank r's inbox is hoccl_plan_inbox_slots slots at
- * r * slots * slot bytes (1 slot; R-1 for the direct reduce-scatter); the partial slots, one per rank, follow all inboxes. */
-size_t hoccl_plan_slot_bytes(hoccl_plan_t plan);
-int hoccl_plan_inbox_slots(hoccl_plan_t plan);
-/* Scratch bytes a call with this plan needs. */
-size_t hoccl_plan_scratch_bytes(hoccl_plan_t plan);
-void hoccl_plan_destroy(hoccl_plan_t plan);
-int hoccl_plan_num_ops(hoccl_plan_t plan);
-int hoccl_plan_num_groups(hoccl_plan_t plan);
-hoccl_result_t hoccl_plan_get_op(hoccl_plan_t plan, int index, hoccl_plan_op_t* out);
-/* Dependencies are between groups: writes up to `cap` predecessor group ids of `group` into deps, returns their number. */
-int hoccl_plan_group_deps(hoccl_plan_t plan, int group, int* deps, int cap);
 
 /* ---------------------------------------------------------------- collective scheduler (host only) --- */
 

@@ -1,4 +1,5 @@
-"""Thin ctypes binding of libhoccl.so: same names as include/hoccl.h, argument marshalling only.
+"""Thin ctypes binding of libhoccl.so: same names as include/hoccl.h, argument marshalling only (the diagnostics of
+include/hoccl_diag.h are bound in diag.py).
 
 Buffers are given as objects with a `data_ptr()` method (torch tensors) or as integer device
 addresses; streams as `torch.cuda.Stream`, raw integer handles or None (the current torch stream).
@@ -16,29 +17,20 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_CUDA, ERR_MISMATCH, ERR_PENDING, ERR_S
 FLOAT32, BFLOAT16 = 0, 1
 SUM = 0
 PATH_CE, PATH_SM, PATH_CE_HOST = 0, 1, 2
-PLAN_ALLREDUCE, PLAN_REDUCE_SCATTER, PLAN_ALLGATHER, PLAN_ALLTOALL, PLAN_ALLREDUCE_FWD, PLAN_REDUCE_SCATTER_FWD = range(6)
-PLAN_ALLREDUCE_AGD, PLAN_ALLGATHER_DIRECT, PLAN_ALLREDUCE_FWD_AGD = 6, 7, 8
-OP_MOVE, OP_SUM, OP_CHAIN = 0, 1, 2
-PLAN_FLAG_FORWARD, PLAN_FLAG_AG_DIRECT, PLAN_FLAG_RS_DIRECT = 16, 32, 64
-BUF_SEND, BUF_RECV, BUF_INBOX, BUF_PARTIAL = 0, 1, 2, 3
 
 DTYPES = {"fp32": FLOAT32, "bf16": BFLOAT16}
 
-EXPORTS = [
-    "hoccl_comm_init", "hoccl_comm_destroy", "hoccl_scratch_bytes", "hoccl_scratch_bytes_direct", "hoccl_plan_inbox_slots", "hoccl_plan_scratch_bytes", "hoccl_comm_set_scratch", "hoccl_comm_set_staging", "hoccl_comm_set_host_staging",
-    "hoccl_comm_set_path", "hoccl_comm_set_param", "hoccl_comm_get_param", "hoccl_allreduce", "hoccl_reduce_scatter",
-    "hoccl_allgather", "hoccl_alltoall", "hoccl_alltoallv", "hoccl_send", "hoccl_recv", "hoccl_comm_pending", "hoccl_comm_async_error", "hoccl_comm_handshakes", "hoccl_selftest_barrier_timeout", "hoccl_host_allreduce", "hoccl_error_string",
-    "hoccl_last_cuda_error", "hoccl_last_stats", "hoccl_profile_reset", "hoccl_probe_move_needs_sm", "hoccl_probe_copy_routes", "hoccl_sum_launch", "hoccl_kernel_sms", "hoccl_flatten_inspect", "hoccl_port_probe",
-    "hoccl_copy_launch", "hoccl_fanout_launch", "hoccl_fanout_inspect", "hoccl_selftest_bf16_add", "hoccl_chain_launch", "hoccl_plan_build", "hoccl_plan_destroy", "hoccl_plan_num_ops", "hoccl_plan_num_groups",
-    "hoccl_plan_get_op", "hoccl_plan_group_deps", "hoccl_plan_slot_bytes", "hoccl_allreduce_static",
-    "hoccl_sched_build", "hoccl_sched_destroy", "hoccl_sched_num_stages", "hoccl_sched_stage_tau", "hoccl_sched_total_tau",
-    "hoccl_sched_lower_bound", "hoccl_sched_matrix", "hoccl_sched_num_flows", "hoccl_sched_get_flow", "hoccl_sched_queue_len",
+EXPORTS = [   # every function include/hoccl.h declares
+    "hoccl_comm_init", "hoccl_comm_destroy", "hoccl_scratch_bytes", "hoccl_scratch_bytes_direct",
+    "hoccl_comm_set_scratch", "hoccl_comm_set_staging", "hoccl_comm_set_host_staging", "hoccl_comm_set_path",
+    "hoccl_comm_set_param", "hoccl_comm_get_param", "hoccl_allreduce", "hoccl_reduce_scatter", "hoccl_allgather",
+    "hoccl_alltoall", "hoccl_alltoallv", "hoccl_send", "hoccl_recv", "hoccl_comm_pending", "hoccl_comm_async_error",
+    "hoccl_comm_handshakes", "hoccl_comm_proxy_stats", "hoccl_host_allreduce", "hoccl_error_string", "hoccl_last_cuda_error", "hoccl_last_stats",
+    "hoccl_profile_reset", "hoccl_allreduce_static", "hoccl_sched_build", "hoccl_sched_destroy",
+    "hoccl_sched_num_stages", "hoccl_sched_stage_tau", "hoccl_sched_total_tau", "hoccl_sched_lower_bound",
+    "hoccl_sched_matrix", "hoccl_sched_num_flows", "hoccl_sched_get_flow", "hoccl_sched_queue_len",
     "hoccl_sched_queue_get",
 ]
-
-
-class RouteProbe(ctypes.Structure):
-    _fields_ = [("name", ctypes.c_char * 56), ("needs_sm", ctypes.c_int), ("end_us", ctypes.c_double)]
 
 
 class Stats(ctypes.Structure):
@@ -53,16 +45,6 @@ class Stats(ctypes.Structure):
 
     def as_dict(self):
         return {k: getattr(self, k) for k, _ in self._fields_}
-
-
-class PlanOp(ctypes.Structure):
-    _fields_ = [
-        ("kind", ctypes.c_int), ("phase", ctypes.c_int), ("step", ctypes.c_int), ("piece", ctypes.c_int),
-        ("rank", ctypes.c_int), ("dst_rank", ctypes.c_int), ("chunk", ctypes.c_int), ("src_buf", ctypes.c_int),
-        ("dst_buf", ctypes.c_int), ("local_buf", ctypes.c_int), ("src_off", ctypes.c_uint64), ("dst_off", ctypes.c_uint64),
-        ("local_off", ctypes.c_uint64), ("bytes", ctypes.c_uint64), ("group", ctypes.c_int),
-        ("nsrc", ctypes.c_int), ("src_stride", ctypes.c_uint64),
-    ]
 
 
 class SchedFlow(ctypes.Structure):
@@ -100,8 +82,6 @@ def lib() -> ctypes.CDLL:
         "hoccl_comm_destroy": (i, [vp]),
         "hoccl_scratch_bytes": (sz, [i, sz, i]),
         "hoccl_scratch_bytes_direct": (sz, [i, sz, i]),
-        "hoccl_plan_inbox_slots": (i, [vp]),
-        "hoccl_plan_scratch_bytes": (sz, [vp]),
         "hoccl_comm_set_scratch": (i, [vp, vp, sz]),
         "hoccl_comm_set_staging": (i, [vp, vp, sz]),
         "hoccl_comm_set_host_staging": (i, [vp, vp, sz]),
@@ -129,31 +109,13 @@ def lib() -> ctypes.CDLL:
         "hoccl_comm_pending": (i, [vp]),
         "hoccl_comm_async_error": (i, [vp, i]),
         "hoccl_comm_handshakes": (l, [vp]),
+        "hoccl_comm_proxy_stats": (i, [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double), i]),
         "hoccl_host_allreduce": (i, [vpp, vpp, sz, i, i, vp, vp]),
         "hoccl_allreduce_static": (i, [vpp, vpp, sz, i, i, i, vp]),
         "hoccl_error_string": (ctypes.c_char_p, [i]),
         "hoccl_last_cuda_error": (ctypes.c_char_p, [vp]),
         "hoccl_last_stats": (i, [vp, ctypes.POINTER(Stats)]),
         "hoccl_profile_reset": (i, [vp]),
-        "hoccl_probe_move_needs_sm": (i, [vp, i, vp, vp, sz, i, ctypes.POINTER(i), ctypes.POINTER(ctypes.c_double)]),
-        "hoccl_probe_copy_routes": (i, [vp, vp, vp, sz, i, ctypes.POINTER(RouteProbe), i, ctypes.POINTER(i)]),
-        "hoccl_sum_launch": (i, [vp, vp, vp, sz, i, i, vp]),
-        "hoccl_copy_launch": (i, [vp, vp, sz, i, vp]),
-        "hoccl_fanout_launch": (i, [vp, vp, i, sz, i, vp]),
-        "hoccl_selftest_bf16_add": (i, [vp, vp]),
-        "hoccl_chain_launch": (i, [vp, sz, i, vp, vp, sz, i, i, vp]),
-        "hoccl_fanout_inspect": (i, [i, vp, vp, vp, i, i, vp, vp, vp, vp, vp, vp, vp, ctypes.POINTER(i), ctypes.POINTER(i)]),
-        "hoccl_kernel_sms": (i, [i, vp, vp, vp, sz, i, i, vp, vp]),
-        "hoccl_selftest_barrier_timeout": (i, [vp, vp, vp, sz, vp]),
-        "hoccl_port_probe": (i, [i, vp, sz, i, vp, vp]),
-        "hoccl_flatten_inspect": (i, [i, i, i, i, vp, vp, vp, vp, vp, vp, vp, vp, vp]),
-        "hoccl_plan_build": (i, [vpp, i, i, sz, i, i, sz, i, ctypes.c_char_p]),
-        "hoccl_plan_slot_bytes": (sz, [vp]),
-        "hoccl_plan_destroy": (None, [vp]),
-        "hoccl_plan_num_ops": (i, [vp]),
-        "hoccl_plan_num_groups": (i, [vp]),
-        "hoccl_plan_get_op": (i, [vp, i, ctypes.POINTER(PlanOp)]),
-        "hoccl_plan_group_deps": (i, [vp, i, ctypes.POINTER(i), i]),
     }
     for name, (res, args) in sigs.items():
         fn = getattr(L, name)
@@ -221,7 +183,7 @@ class Comm:
     def destroy(self):
         if self._h:
             rc = lib().hoccl_comm_destroy(self._h)
-            if rc == OK:
+            if rc != ERR_PENDING:      # PENDING is the one case in which nothing was freed
                 self._h = ctypes.c_void_p()
             return rc
         return OK
@@ -321,11 +283,14 @@ class Comm:
     def async_error(self, clear: bool = False) -> int:
         return lib().hoccl_comm_async_error(self._h, int(clear))
 
-    def selftest_barrier_timeout(self, dst, src, nbytes, stream=None) -> int:
-        return lib().hoccl_selftest_barrier_timeout(self._h, _ptr(dst), _ptr(src), nbytes, _stream(stream))
-
     def handshakes(self) -> int:
         return int(lib().hoccl_comm_handshakes(self._h))
+
+    def proxy_stats(self, reset: bool = False):
+        """(busy_us, span_us) of the proxy thread: see hoccl_comm_proxy_stats."""
+        b, s = ctypes.c_double(), ctypes.c_double()
+        self._check(lib().hoccl_comm_proxy_stats(self._h, ctypes.byref(b), ctypes.byref(s), int(reset)), "hoccl_comm_proxy_stats")
+        return b.value, s.value
 
     # -- diagnostics
     def last_stats(self) -> dict:
@@ -335,22 +300,6 @@ class Comm:
 
     def profile_reset(self):
         self._check(lib().hoccl_profile_reset(self._h), "hoccl_profile_reset")
-
-    def probe_move_needs_sm(self, path, dst, src, nbytes, spin_us=3000):
-        needs = ctypes.c_int()
-        end_us = ctypes.c_double()
-        self._check(lib().hoccl_probe_move_needs_sm(self._h, path, _ptr(dst), _ptr(src), nbytes, spin_us, ctypes.byref(needs),
-                                                    ctypes.byref(end_us)), "hoccl_probe_move_needs_sm")
-        return bool(needs.value), end_us.value
-
-    def probe_copy_routes(self, dst, src, nbytes, spin_us=3000):
-        """[(route name, needs an SM, completion time in us)] for every same-device way of moving bytes."""
-        out = (RouteProbe * 16)()
-        n = ctypes.c_int()
-        self._check(lib().hoccl_probe_copy_routes(self._h, _ptr(dst), _ptr(src), nbytes, spin_us, out, 16, ctypes.byref(n)),
-                    "hoccl_probe_copy_routes")
-        return [(out[k].name.decode(), bool(out[k].needs_sm), out[k].end_us) for k in range(n.value)]
-
 
 STATIC_SCRATCH_BYTES = 32 << 20
 
@@ -368,107 +317,6 @@ def scratch_bytes(R: int, max_count: int, dtype) -> int:
 def scratch_bytes_direct(R: int, max_count: int, dtype) -> int:
     """Scratch bound with "rs_direct" set (R-1 inbox slots per rank)."""
     return int(lib().hoccl_scratch_bytes_direct(R, max_count, _dtype(dtype)))
-
-
-def sum_launch(inbox, local, out, count, dtype, ctas, stream=None) -> int:
-    return lib().hoccl_sum_launch(_ptr(inbox), _ptr(local), _ptr(out), count, _dtype(dtype), ctas, _stream(stream))
-
-
-def copy_launch(src, dst, nbytes, ctas, stream=None) -> int:
-    return lib().hoccl_copy_launch(_ptr(src), _ptr(dst), nbytes, ctas, _stream(stream))
-
-
-def fanout_launch(src, dsts, nbytes, ctas, stream=None) -> int:
-    """hoccl_fanout_launch: every dsts[d] <- src, the source read once.  Returns the result code."""
-    return lib().hoccl_fanout_launch(_ptr(src), _ptr_array(dsts), len(dsts), nbytes, ctas, _stream(stream))
-
-
-def chain_launch(first, stride_bytes, nsrc, local, out, count, dtype, ctas, stream=None) -> int:
-    """hoccl_chain_launch: out = (((s_0 + s_1) + ...) + s_{nsrc-1}) + local with s_j = first + j * stride_bytes."""
-    return lib().hoccl_chain_launch(_ptr(first), stride_bytes, nsrc, _ptr(local), _ptr(out), count, _dtype(dtype), ctas, _stream(stream))
-
-
-def selftest_bf16_add(counts, stream=None) -> int:
-    """hoccl_selftest_bf16_add: counts = device array of two zeroed 64-bit words.  Returns the result code."""
-    return lib().hoccl_selftest_bf16_add(_ptr(counts), _stream(stream))
-
-
-def fanout_inspect(moves, ctas: int = 8):
-    """hoccl_fanout_inspect (host only): moves = [(src_addr, dst_addr, nbytes), ...] -> (segments, launches) where a segment is
-    (launch, src_addr, nbytes, [dst_addr, ...], head, nvec); no segments means the moves go as plain copies."""
-    n = len(moves)
-    u64 = ctypes.c_uint64 * n
-    src, dst, ln = u64(*[m[0] for m in moves]), u64(*[m[1] for m in moves]), u64(*[m[2] for m in moves])
-    cap = n
-    seg_launch, seg_nd = (ctypes.c_int * cap)(), (ctypes.c_int * cap)()
-    seg_src, seg_len, seg_nvec, dst_out = (ctypes.c_uint64 * cap)(), (ctypes.c_uint64 * cap)(), (ctypes.c_uint64 * cap)(), u64()
-    seg_head = (ctypes.c_uint32 * cap)()
-    n_seg, n_launch = ctypes.c_int(0), ctypes.c_int(0)
-    rc = lib().hoccl_fanout_inspect(n, src, dst, ln, ctas, cap, seg_launch, seg_src, seg_len, seg_nd, seg_head, seg_nvec, dst_out,
-                                    ctypes.byref(n_seg), ctypes.byref(n_launch))
-    if rc != OK:
-        raise HocclError(rc, "hoccl_fanout_inspect", "")
-    segs, at = [], 0
-    for k in range(n_seg.value):
-        segs.append((seg_launch[k], seg_src[k], seg_len[k], [dst_out[at + d] for d in range(seg_nd[k])], seg_head[k], seg_nvec[k]))
-        at += seg_nd[k]
-    return segs, n_launch.value
-
-
-def kernel_sms(kind: str, a, b, out, nbytes: int, dtype, ctas: int, smid_out, stream=None) -> int:
-    """hoccl_kernel_sms: run the SUM ("sum") or copy ("copy") kernel with `ctas` CTAs; every CTA writes its SM id to
-    smid_out (a device array of `ctas` 32-bit words).  Returns the result code."""
-    return lib().hoccl_kernel_sms(0 if kind == "sum" else 1, _ptr(a), _ptr(b) if b is not None else None, _ptr(out), nbytes,
-                                  _dtype(dtype), ctas, _ptr(smid_out), _stream(stream))
-
-
-def port_probe(mode: str, buf, nbytes: int, ctas: int, sink, stream=None) -> int:
-    """hoccl_port_probe: `ctas` CTAs only read ("read") or only write ("write") the buffer."""
-    return lib().hoccl_port_probe(0 if mode == "read" else 1, _ptr(buf), nbytes, ctas, _ptr(sink), _stream(stream))
-
-
-def flatten_inspect(kind: str, dtype, ctas: int, a_addr, b_addr, out_addr, lens):
-    """hoccl_flatten_inspect (host only): per segment (head, nvec, tiles_end, scalars_end) and the tile size in vectors."""
-    n = len(lens)
-    U64 = ctypes.c_uint64 * n
-    a, o, ln = U64(*a_addr), U64(*out_addr), U64(*lens)
-    b = U64(*(b_addr if b_addr is not None else [0] * n))
-    tiles, scal, nvec = U64(), U64(), U64()
-    head = (ctypes.c_uint32 * n)()
-    tv = ctypes.c_uint64()
-    rc = lib().hoccl_flatten_inspect(0 if kind == "sum" else 1, _dtype(dtype), ctas, n, a, b, o, ln, tiles, scal, nvec, head, ctypes.byref(tv))
-    if rc != OK:
-        raise HocclError(rc, "hoccl_flatten_inspect", "")
-    return [(int(head[k]), int(nvec[k]), int(tiles[k]), int(scal[k])) for k in range(n)], int(tv.value)
-
-
-class Plan:
-    """Host-only view of the planner's output."""
-
-    def __init__(self, kind, R, count, dtype, in_place=False, piece_bytes=4 << 20, max_pieces=8, send_align=None):
-        self._h = ctypes.c_void_p()
-        align = bytes(send_align) if send_align is not None else None
-        rc = lib().hoccl_plan_build(ctypes.byref(self._h), kind, R, count, _dtype(dtype), int(in_place), piece_bytes, max_pieces,
-                                    align)
-        if rc != OK:
-            raise HocclError(rc, "hoccl_plan_build")
-        L = lib()
-        self.slot_bytes = int(L.hoccl_plan_slot_bytes(self._h))
-        self.inbox_slots = int(L.hoccl_plan_inbox_slots(self._h))
-        self.scratch_bytes = int(L.hoccl_plan_scratch_bytes(self._h))
-        self.ops = []
-        for k in range(L.hoccl_plan_num_ops(self._h)):
-            op = PlanOp()
-            assert L.hoccl_plan_get_op(self._h, k, ctypes.byref(op)) == OK
-            self.ops.append({f: getattr(op, f) for f, _ in PlanOp._fields_})
-        self.num_groups = L.hoccl_plan_num_groups(self._h)
-        self.deps = []
-        for g in range(self.num_groups):
-            buf = (ctypes.c_int * 64)()
-            n = L.hoccl_plan_group_deps(self._h, g, buf, 64)
-            self.deps.append([buf[k] for k in range(n)])
-        L.hoccl_plan_destroy(self._h)
-        self._h = None
 
 
 class Schedule:

@@ -1,6 +1,8 @@
 // The C ABI declared in include/hoccl.h: communicator life cycle, parameters, collectives, send/recv, the user-defined
 // pattern executor, diagnostics, and the host-only planner / scheduler inspection calls.
 #include "comm.h"
+#include "options.h"
+#include "../../include/hoccl_diag.h"
 
 using namespace hoccl;
 
@@ -41,9 +43,15 @@ hoccl_result_t hoccl_comm_init(hoccl_comm_t* comm, int R, int device) {
 hoccl_result_t hoccl_comm_destroy(hoccl_comm_t c) {
   if (!c) return HOCCL_ERR_INVALID_ARG;
   if (c->n_pending > 0) return HOCCL_ERR_PENDING;
+  bool forced = false;
   if (c->proxy) {
-    c->proxy->drain(c->watchdog_ms);
+    const bool drained = c->proxy->drain(c->watchdog_ms);
     if (c->proxy->pending_p2p() > 0) return HOCCL_ERR_PENDING;
+    // Hand-overs that are still open (a stream that has not reached its post yet, work that has not finished) are
+    // released by the proxy on its way out, so no stream keeps waiting on a communicator that is gone; if a stream could
+    // not be seen past its hand-over in time, the flag memory outlives the proxy (see Proxy::shutdown).
+    const bool passed = c->proxy->shutdown(2 * c->watchdog_ms + 100);
+    forced = !drained || !passed;
     delete c->proxy;
     c->proxy = nullptr;
   }
@@ -61,6 +69,7 @@ hoccl_result_t hoccl_comm_destroy(hoccl_comm_t c) {
   if (c->ring_bar) cudaFree(c->ring_bar);
   if (c->ring_err) cudaFreeHost(c->ring_err);
   for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
+  for (cudaEvent_t e : c->post_events) cudaEventDestroy(e);
   for (auto& p : c->prof_pool) {
     cudaEventDestroy(p.first);
     cudaEventDestroy(p.second);
@@ -70,7 +79,7 @@ hoccl_result_t hoccl_comm_destroy(hoccl_comm_t c) {
     cudaEventDestroy(p.first.second);
   }
   delete c;
-  return HOCCL_OK;
+  return forced ? HOCCL_ERR_TIMEOUT : HOCCL_OK;
 }
 
 size_t hoccl_scratch_bytes(int R, size_t max_count, hoccl_dtype_t dtype) {
@@ -134,6 +143,9 @@ static long* param_slot(hoccl_comm* c, const char* key, long* lo, long* hi) {
               {"ag_direct", &c->ag_direct, 0, 2},
               {"order_kernels", &c->order_kernels, 0, 1},
               {"rs_direct", &c->rs_direct, 0, 2},
+              {"ce_small_bytes", &c->ce_small_bytes, 0, 1L << 40},
+              {"ce_small_ctas", &c->ce_small_ctas, 1, 1024},
+              {"p2p_strict", &c->p2p_strict, 0, 1},
               {"host_pieces", &c->host_pieces, 1, 64}};
   for (auto& r : rows)
     if (std::strcmp(r.name, key) == 0) {
@@ -239,6 +251,16 @@ hoccl_result_t hoccl_selftest_barrier_timeout(hoccl_comm_t c, void* dst, const v
 
 long hoccl_comm_handshakes(hoccl_comm_t c) { return (c && c->proxy) ? c->proxy->handshakes() : 0; }
 
+hoccl_result_t hoccl_comm_proxy_stats(hoccl_comm_t c, double* busy_us, double* span_us, int reset) {
+  if (!c) return HOCCL_ERR_INVALID_ARG;
+  if (busy_us) *busy_us = 0;
+  if (span_us) *span_us = 0;
+  if (!c->proxy) return HOCCL_OK;
+  c->proxy->work_stats(busy_us, span_us);
+  if (reset) c->proxy->reset_work_stats();
+  return HOCCL_OK;
+}
+
 hoccl_result_t hoccl_host_allreduce(const void* const* h_send, void* const* h_recv, size_t count, hoccl_dtype_t dtype, hoccl_op_t op,
                                     hoccl_comm_t c, hoccl_stream_t stream) {
   if (!c || !h_send || !h_recv) return HOCCL_ERR_INVALID_ARG;
@@ -274,6 +296,10 @@ hoccl_result_t hoccl_host_allreduce(const void* const* h_send, void* const* h_re
     call.h_send = h_send;
     call.h_recv = h_recv;
     return run_collective(c, &call, st);
+  }
+  {   // a combination of settings that the all-reduce will refuse must be refused before the inbound copies are enqueued
+    hoccl_result_t orc = check_options(c, PLAN_ALLREDUCE, count, (int)dtype);
+    if (orc != HOCCL_OK) return orc;
   }
   for (int r = 0; r < R; r++) CU_TRY(c, cudaMemcpyAsync(const_cast<void*>(dsend[r]), h_send[r], count * e, cudaMemcpyHostToDevice, st));
   hoccl_result_t rc = hoccl_allreduce(dsend, drecv, count, dtype, op, c, stream);
@@ -854,3 +880,18 @@ int hoccl_plan_group_deps(hoccl_plan_t plan, int group, int* deps, int cap) {
 
 
 }  // extern "C"
+
+extern "C" hoccl_result_t hoccl_options_resolve(const hoccl_options_t* o, hoccl_resolved_t* out) {
+  if (!o || !out) return HOCCL_ERR_INVALID_ARG;
+  hoccl::OptionsIn in{o->kind, o->R, o->count, o->dtype, o->path, o->onepass, o->forward, o->fused, o->rs_direct, o->ag_direct,
+                      o->handshake, o->use_graph, o->ce_small_bytes, o->ce_small_ctas, o->copy_ctas, o->scratch_bytes, o->host_call};
+  hoccl::OptionsOut r;
+  hoccl_result_t rc = hoccl::resolve_options(in, &r);
+  if (rc != HOCCL_OK) return rc;
+  out->plan_kind = r.plan_kind;
+  out->executor = r.executor;
+  out->path = r.path;
+  out->copy_ctas = r.copy_ctas;
+  out->small_switch = r.small_switch;
+  return HOCCL_OK;
+}

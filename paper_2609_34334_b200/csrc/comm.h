@@ -14,6 +14,7 @@
 #include <vector>
 
 #include "../../include/hoccl.h"
+#include "../../include/hoccl_diag.h"
 #include "kernels.cuh"
 #include "plan.h"
 #include "proxy.h"
@@ -54,6 +55,7 @@ struct Post {
   size_t count;
   int dtype;
   cudaStream_t stream;
+  cudaEvent_t at_post;   // recorded on `stream` when the post was made: the move waits for this point, not for later work
 };
 
 // One host <-> staging copy of the pipelined host all-reduce: `rows` rows of `width` bytes at `pitch` (rows == 1: plain).
@@ -87,7 +89,8 @@ struct hoccl_comm {
   int R = 0, device = 0, num_sms = 0;
   hoccl_path_t path = HOCCL_PATH_CE;
   long sum_ctas = 8, copy_ctas = 8, piece_bytes = 4 << 20, max_pieces = 8, lanes = 4, use_graph = 1, profile = 0, p2p_split = 1, ce_sub_bytes = 0,
-       handshake = 0, watchdog_ms = 10000, onepass = 0, forward = 0, fused = 0, host_pieces = 8, ag_direct = 0, order_kernels = 1, rs_direct = 0;
+       handshake = 0, watchdog_ms = 10000, onepass = 0, forward = 0, fused = 0, host_pieces = 8, ag_direct = 2, order_kernels = 1, rs_direct = 2,
+       ce_small_bytes = 8 << 20, ce_small_ctas = 148, p2p_strict = 0;
   bool piece_bytes_set = false;  // the caller chose a piece size: no automatic choice
   hoccl::Proxy* proxy = nullptr;
   cudaStream_t lane[hoccl::kMaxLanes] = {};
@@ -105,6 +108,7 @@ struct hoccl_comm {
   char* host_staging = nullptr;  // pinned host memory of the CE_HOST path
   size_t host_staging_bytes = 0;
   std::map<std::pair<int, int>, std::deque<hoccl::Post>> pending;
+  std::vector<cudaEvent_t> post_events;   // free list of the events that mark parked posts
   int n_pending = 0;
   unsigned p2p_rr = 0;
   std::vector<hoccl::GraphEntry> cache;
@@ -185,6 +189,8 @@ cudaError_t enqueue_host_copy(const HostCopy& hc, bool to_device, cudaStream_t s
 hoccl_result_t build_ring(hoccl_comm* c, const Plan& P, const std::vector<RGroup>& groups, GraphEntry* entry);
 // exec.cu
 hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user);
+// HOCCL_OK if the communicator's settings fit together for such a call (see options.h); nothing is enqueued
+hoccl_result_t check_options(hoccl_comm* c, int kind, size_t count, int dtype);
 hoccl_result_t ensure_proxy(hoccl_comm* c);
 void harvest_profile(hoccl_comm* c);
 void destroy_entry(GraphEntry* e);

@@ -14,6 +14,7 @@
 #include <tuple>
 
 #include "comm.h"
+#include "options.h"
 
 namespace hoccl {
 
@@ -526,26 +527,48 @@ static hoccl_result_t launch_entry(hoccl_comm* c, GraphEntry* hit, cudaStream_t 
   return HOCCL_OK;
 }
 
+static OptionsIn options_of(hoccl_comm* c, int kind, size_t count, int dtype, bool host_call) {
+  return OptionsIn{kind, c->R, count, dtype, (int)c->path, c->onepass, c->forward, c->fused, c->rs_direct, c->ag_direct,
+                   c->handshake, c->use_graph, c->ce_small_bytes, c->ce_small_ctas, c->copy_ctas, c->scratch ? c->scratch_bytes : 0,
+                   host_call ? 1 : 0};
+}
+
+hoccl_result_t check_options(hoccl_comm* c, int kind, size_t count, int dtype) {
+  OptionsOut o;
+  return resolve_options(options_of(c, kind, count, dtype, false), &o);
+}
+
 hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
   const double t0 = now_us();
   if (!c) return HOCCL_ERR_INVALID_ARG;
   if (dtype_size(call->dtype) == 0) return HOCCL_ERR_UNSUPPORTED;
   if (!call->send || !call->recv) return HOCCL_ERR_INVALID_ARG;
-  const bool onepass_case = c->onepass && !c->handshake && (call->kind == PLAN_ALLREDUCE || call->kind == PLAN_REDUCE_SCATTER);
-  // rs_direct = 2: the direct reduce-scatter whenever the attached scratch holds its R-1 inbox slots per rank (it was faster
-  // than the ring at every size and on every path measured), the ring otherwise
-  bool direct_rs = c->rs_direct == 1 && (call->kind == PLAN_ALLREDUCE || call->kind == PLAN_REDUCE_SCATTER);
-  if (c->rs_direct == 2 && (call->kind == PLAN_ALLREDUCE || call->kind == PLAN_REDUCE_SCATTER) && c->R > 1) {
-    const size_t cnt = call->kind == PLAN_ALLREDUCE ? call->count : call->count * (size_t)c->R;
-    direct_rs = c->scratch && c->scratch_bytes >= (size_t)(c->R - 1) * (size_t)c->R * slot_bytes_for(c->R, cnt, dtype_size(call->dtype));
+  // One place decides how the settings combine for this call (options.h); a contradictory combination is refused here.
+  const OptionsIn oin = options_of(c, call->kind, call->count, call->dtype, call->h_send != nullptr);
+  OptionsOut opt;
+  {
+    hoccl_result_t orc = resolve_options(oin, &opt);
+    if (orc != HOCCL_OK) return orc;
   }
-  const bool fused = c->fused && c->path == HOCCL_PATH_SM && !c->handshake && !onepass_case && !call->h_send && !direct_rs;   // the ring kernel has no chain phase
-  const bool graphs = (c->use_graph || c->handshake || fused) && !onepass_case;
+  // a small message on the copy route runs on the copy kernel's route: the communicator shows that route for this call only
+  struct RouteGuard {
+    hoccl_comm* c;
+    hoccl_path_t path;
+    long ctas;
+    ~RouteGuard() {
+      c->path = path;
+      c->copy_ctas = ctas;
+    }
+  } guard{c, c->path, c->copy_ctas};
+  c->path = (hoccl_path_t)opt.path;
+  c->copy_ctas = opt.copy_ctas;
+  const bool onepass_case = opt.executor == EXEC_ONEPASS;
+  const bool fused = opt.executor == EXEC_ONE_KERNEL;
+  const bool graphs = opt.executor != EXEC_STREAMS && !onepass_case;
   std::vector<uint64_t> key;
   if (graphs && call->count != 0) {
     // Fast path: a call whose signature (operation, count, dtype, every pointer, every setting that shapes the graph)
     // was seen before was validated and planned then; replaying its graph is all that is left to do.
-    if (c->handshake && c->path != HOCCL_PATH_SM) return HOCCL_ERR_UNSUPPORTED;
     key = make_key(c, *call);
     for (auto& e : c->cache)
       if (e.key == key) {
@@ -565,7 +588,7 @@ hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
   if (call->count == 0) return HOCCL_OK;
   CU_TRY(c, cudaSetDevice(c->device));
 
-  if (c->onepass && !c->handshake && (call->kind == PLAN_ALLREDUCE || call->kind == PLAN_REDUCE_SCATTER)) {
+  if (onepass_case) {
     // comparison point: the whole reduction in one kernel, same order and rounding as the ring, no moves, no scratch
     OnePassArgs a;
     a.R = c->R;
@@ -593,20 +616,7 @@ hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
   Plan P;
   unsigned char align[kMaxRanks];
   for (int r = 0; r < c->R; r++) align[r] = (unsigned char)((uintptr_t)call->send[r] & 15);
-  int plan_kind = call->kind;
-  if (c->forward && call->kind == PLAN_ALLREDUCE) plan_kind = PLAN_ALLREDUCE_FWD;
-  if (c->forward && call->kind == PLAN_REDUCE_SCATTER) plan_kind = PLAN_REDUCE_SCATTER_FWD;
-  // ag_direct = 2: where it was measured faster or equal.  Kernels of this library (SM path) and the host bounce: always
-  // (fewer bytes, fewer launches or hops).  Copy route: the bytes are the same, the gain is the missing chain of stages,
-  // which fades with size (equal within 2 % from 64 MiB per rank at R = 8), so it is taken while a chunk is at most 64 MiB.
-  bool direct = c->ag_direct == 1;
-  if (c->ag_direct == 2 && (call->kind == PLAN_ALLREDUCE || call->kind == PLAN_ALLGATHER)) {
-    const size_t q = call->kind == PLAN_ALLREDUCE ? (call->count + c->R - 1) / c->R : call->count;
-    direct = c->path != HOCCL_PATH_CE || q * dtype_size(call->dtype) <= ((size_t)64 << 20);
-  }
-  if (direct && call->kind == PLAN_ALLREDUCE) plan_kind = c->forward ? PLAN_ALLREDUCE_FWD_AGD : PLAN_ALLREDUCE_AGD;
-  if (direct && call->kind == PLAN_ALLGATHER) plan_kind = PLAN_ALLGATHER_DIRECT;
-  if (direct_rs) plan_kind = call->kind | PLAN_FLAG_RS_DIRECT | (direct ? PLAN_FLAG_AG_DIRECT : 0);
+  const int plan_kind = opt.plan_kind;
   // Piece size: the caller's if set.  Otherwise: on the SM path under CTA budgets a reduction is cut into at least two
   // pieces (the copy kernel of one piece then overlaps the sum kernel of the other: measured 1.6x on a 3 MiB chunk with
   // 8 + 8 CTAs) of at most 4 MiB.  That does not pay with driver copies (they take the whole GPU and never overlap a sum:

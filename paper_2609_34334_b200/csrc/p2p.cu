@@ -11,7 +11,7 @@ hoccl_result_t p2p_post(hoccl_comm* c, bool is_send, void* buf, size_t count, in
   if (e == 0) return HOCCL_ERR_UNSUPPORTED;
   if (src < 0 || src >= c->R || dst < 0 || dst >= c->R || src == dst) return HOCCL_ERR_INVALID_ARG;
   if ((uintptr_t)buf % e) return HOCCL_ERR_INVALID_ARG;
-  if (c->handshake) {
+  if (c->handshake || c->p2p_strict) {
     // the post is handed to the proxy at once; matching happens there, after the stream has reached the post
     if (c->path != HOCCL_PATH_SM) return HOCCL_ERR_UNSUPPORTED;   // see run_collective
     hoccl_result_t rc = ensure_proxy(c);
@@ -37,13 +37,29 @@ hoccl_result_t p2p_post(hoccl_comm* c, bool is_send, void* buf, size_t count, in
   auto key = std::make_pair(src, dst);
   std::deque<Post>& q = c->pending[key];
   if (q.empty() || q.front().is_send == is_send) {
-    q.push_back(Post{is_send, buf, count, dtype, stream});
+    // No partner yet: the post parks on the host.  Its place in its stream is marked now, so that the move, whenever the
+    // partner comes, waits for exactly this point of the stream and not for whatever the stream is given afterwards.
+    CU_TRY(c, cudaSetDevice(c->device));
+    cudaEvent_t ev = nullptr;
+    if (!c->post_events.empty()) {
+      ev = c->post_events.back();
+      c->post_events.pop_back();
+    } else {
+      CU_TRY(c, cudaEventCreateWithFlags(&ev, cudaEventDisableTiming));
+    }
+    cudaError_t re = cudaEventRecord(ev, stream);
+    if (re != cudaSuccess) {
+      c->post_events.push_back(ev);
+      return cuda_fail(c, re, "cudaEventRecord (post)");
+    }
+    q.push_back(Post{is_send, buf, count, dtype, stream, ev});
     c->n_pending++;
     return HOCCL_OK;
   }
   Post peer = q.front();
   q.pop_front();
   c->n_pending--;
+  c->post_events.push_back(peer.at_post);   // waits enqueued below capture the record made at post time; the event itself is free again
   if (peer.count != count || peer.dtype != dtype) return HOCCL_ERR_MISMATCH;
   c->stats = hoccl_stats_t{};
   if (count == 0) return HOCCL_OK;
@@ -58,15 +74,13 @@ hoccl_result_t p2p_post(hoccl_comm* c, bool is_send, void* buf, size_t count, in
     // the staging area, so they run one after the other.
     if (!c->host_staging || bytes > c->host_staging_bytes) return HOCCL_ERR_SCRATCH;
     c->ev_next = 0;
-    cudaEvent_t ea = next_event(c), eb = two_streams ? next_event(c) : nullptr, ed = next_event(c);
-    if (!ea || (two_streams && !eb) || !ed) return cuda_fail(c, cudaErrorMemoryAllocation, "event pool");
+    // ea: where the first poster's stream was when it posted; eb: where this (the second) poster's stream is now
+    cudaEvent_t ea = peer.at_post, eb = next_event(c), ed = next_event(c);
+    if (!eb || !ed) return cuda_fail(c, cudaErrorMemoryAllocation, "event pool");
     cudaStream_t run = c->lane[0];
-    CU_TRY(c, cudaEventRecord(ea, peer.stream));
-    CU_TRY(c, cudaStreamWaitEvent(run, ea, 0));
-    if (two_streams) {
-      CU_TRY(c, cudaEventRecord(eb, stream));
-      CU_TRY(c, cudaStreamWaitEvent(run, eb, 0));
-    }
+    if (two_streams) CU_TRY(c, cudaStreamWaitEvent(run, ea, 0));
+    CU_TRY(c, cudaEventRecord(eb, stream));
+    CU_TRY(c, cudaStreamWaitEvent(run, eb, 0));
     // Chunk pipelining through the staging area (paper Sec. 3.3.1: one engine fills a staging chunk while the other
     // drains the previous one): the outbound leg of chunk k+1 runs on lane 0 while the inbound leg of chunk k runs on
     // lane 1; PCIe carries both directions at once.
@@ -127,10 +141,9 @@ hoccl_result_t p2p_post(hoccl_comm* c, bool is_send, void* buf, size_t count, in
   } else {
     // the move runs on internal lanes after both posting streams, and both wait for it
     c->ev_next = 0;
-    cudaEvent_t ea = next_event(c), eb = two_streams ? next_event(c) : nullptr;
-    if (!ea || (two_streams && !eb)) return cuda_fail(c, cudaErrorMemoryAllocation, "event pool");
-    CU_TRY(c, cudaEventRecord(ea, peer.stream));
-    if (two_streams) CU_TRY(c, cudaEventRecord(eb, stream));
+    cudaEvent_t ea = peer.at_post, eb = next_event(c);
+    if (!eb) return cuda_fail(c, cudaErrorMemoryAllocation, "event pool");
+    CU_TRY(c, cudaEventRecord(eb, stream));
     const size_t slice = ((bytes + nsplit - 1) / nsplit + 255) / 256 * 256;
     for (int i = 0; i < nsplit; i++) {
       const size_t off = (size_t)i * slice;
@@ -139,8 +152,8 @@ hoccl_result_t p2p_post(hoccl_comm* c, bool is_send, void* buf, size_t count, in
       // copy route: rotate lanes so that independent messages overlap; SM copies share one lane so that the CTA
       // budget stays global (two copy kernels never run at the same time)
       cudaStream_t run = c->path == HOCCL_PATH_CE ? c->lane[(c->p2p_rr++) % kMaxLanes] : c->lane[0];
-      CU_TRY(c, cudaStreamWaitEvent(run, ea, 0));
-      if (two_streams) CU_TRY(c, cudaStreamWaitEvent(run, eb, 0));
+      if (two_streams) CU_TRY(c, cudaStreamWaitEvent(run, ea, 0));
+      CU_TRY(c, cudaStreamWaitEvent(run, eb, 0));
       if (c->path == HOCCL_PATH_CE) {
         CU_TRY(c, cudaMemcpyAsync((char*)dbuf + off, (const char*)sbuf + off, len, cudaMemcpyDeviceToDevice, run));
       } else {

@@ -1,5 +1,6 @@
-// CPU proxy thread and the two-flag stream handshake (see proxy.h; paper Sec. 3.2, Listing 1, and Sec. 3.3.2 for
-// the matched send/recv that the proxy completes once both sides have posted).
+// CPU proxy thread and the sequence-numbered stream hand-over (see proxy.h; the idea of a stream that hands itself to a
+// CPU thread is the paper's, Sec. 3.2; Sec. 3.3.2 for the matched send/recv that the proxy completes once both sides
+// have posted).
 #include "proxy.h"
 
 #include <cuda.h>
@@ -38,12 +39,16 @@ bool trace_on() {
 double now_ms() {
   return std::chrono::duration<double, std::milli>(std::chrono::steady_clock::now().time_since_epoch()).count();
 }
+long long now_ns() {
+  return std::chrono::duration_cast<std::chrono::nanoseconds>(std::chrono::steady_clock::now().time_since_epoch()).count();
+}
 
 }  // namespace
 
 Proxy::Proxy(int device, long watchdog_ms) : device_(device), watchdog_ms_(watchdog_ms) {
   slots_.resize(kFlagPairs);
   pair_busy_.assign(kFlagPairs, 0);
+  last_seq_.assign(kFlagPairs, 0);
 }
 
 cudaError_t Proxy::init() {
@@ -55,10 +60,10 @@ cudaError_t Proxy::init() {
   e = cudaGetDriverEntryPoint("cuStreamWaitValue32", &fn_wait_, cudaEnableDefault, &qr);
   if (e != cudaSuccess || !fn_wait_) return e != cudaSuccess ? e : cudaErrorNotSupported;
   void* host = nullptr;
-  e = cudaHostAlloc(&host, sizeof(uint32_t) * 2 * kFlagPairs, cudaHostAllocMapped | cudaHostAllocPortable);
+  e = cudaHostAlloc(&host, sizeof(uint32_t) * kFlagWords * kFlagPairs, cudaHostAllocMapped | cudaHostAllocPortable);
   if (e != cudaSuccess) return e;
   flags_ = static_cast<volatile uint32_t*>(host);
-  for (int i = 0; i < 2 * kFlagPairs; i++) flags_[i] = 0;
+  for (int i = 0; i < kFlagWords * kFlagPairs; i++) flags_[i] = 0;
   void* dev = nullptr;
   e = cudaHostGetDevicePointer(&dev, host, 0);
   if (e != cudaSuccess) return e;
@@ -102,10 +107,32 @@ cudaError_t Proxy::init() {
   return cudaSuccess;
 }
 
-Proxy::~Proxy() {
+bool Proxy::all_passed() {
+  std::lock_guard<std::mutex> lock(mu_);
+  for (int i = 0; i < kFlagPairs; i++)
+    if (*passed(i) != last_seq_[i]) return false;
+  return true;
+}
+
+bool Proxy::shutdown(long timeout_ms) {
   stop_ = true;
   cv_.notify_all();
-  if (th_.joinable()) th_.join();
+  if (th_.joinable()) th_.join();   // the loop releases whatever is still open before it ends
+  if (!flags_) return true;
+  if (keep_flags_) return false;
+  const double t0 = now_ms();
+  while (!all_passed()) {
+    if (now_ms() - t0 > (double)timeout_ms) {
+      keep_flags_ = true;   // a stream will still come and look at its pair: the counters stay where they are
+      return false;
+    }
+    std::this_thread::sleep_for(std::chrono::microseconds(100));
+  }
+  return true;
+}
+
+Proxy::~Proxy() {
+  shutdown(2 * watchdog_ms_.load() + 100);
   cudaSetDevice(device_);
   if (stream_) {
     cudaStreamSynchronize(stream_);
@@ -113,13 +140,14 @@ Proxy::~Proxy() {
   }
   for (auto& s : slots_)
     if (s.done) cudaEventDestroy(s.done);
-  if (flags_) cudaFreeHost(const_cast<uint32_t*>(flags_));
+  if (flags_ && !keep_flags_) cudaFreeHost(const_cast<uint32_t*>(flags_));
   if (warm_) cudaFree(warm_);
 }
 
 cudaError_t Proxy::submit(cudaStream_t user, ProxyTask task) {
   if (stop_) return cudaErrorUnknown;
   int pair = -1;
+  uint32_t seq = 0;
   {
     std::unique_lock<std::mutex> lock(mu_);
     const double t0 = now_ms();
@@ -137,25 +165,25 @@ cudaError_t Proxy::submit(cudaStream_t user, ProxyTask task) {
     }
     pair_busy_[pair] = 1;
     next_pair_ = (pair + 1) % kFlagPairs;
+    seq = ++last_seq_[pair];
   }
-  *start_flag(pair) = 0;
-  *finish_flag(pair) = 0;
-  std::atomic_thread_fence(std::memory_order_seq_cst);
-  const CUdeviceptr ds = (CUdeviceptr)(uintptr_t)(flags_dev_ + 2 * pair);
-  const CUdeviceptr df = (CUdeviceptr)(uintptr_t)(flags_dev_ + 2 * pair + 1);
+  const CUdeviceptr d_arrived = (CUdeviceptr)(uintptr_t)(flags_dev_ + kFlagWords * pair);
+  const CUdeviceptr d_released = d_arrived + 4, d_passed = d_arrived + 8;
   WriteValue32Fn wr = reinterpret_cast<WriteValue32Fn>(fn_write_);
   WaitValue32Fn wt = reinterpret_cast<WaitValue32Fn>(fn_wait_);
   CUstream cs = (CUstream)user;
-  CUresult r = wr(cs, ds, kFlagStart, CU_STREAM_WRITE_VALUE_DEFAULT);
-  if (r == CUDA_SUCCESS) r = wt(cs, ds, 0, CU_STREAM_WAIT_VALUE_EQ);
-  if (r == CUDA_SUCCESS) r = wt(cs, df, kFlagFinish, CU_STREAM_WAIT_VALUE_GEQ);
-  if (r == CUDA_SUCCESS) r = wr(cs, df, 0, CU_STREAM_WRITE_VALUE_DEFAULT);
+  // arrive, wait for the release of this very hand-over (cyclic >=, so the counters may wrap), tell the host we are past it
+  CUresult r = wr(cs, d_arrived, seq, CU_STREAM_WRITE_VALUE_DEFAULT);
+  if (r == CUDA_SUCCESS) r = wt(cs, d_released, seq, CU_STREAM_WAIT_VALUE_GEQ);
+  if (r == CUDA_SUCCESS) r = wr(cs, d_passed, seq, CU_STREAM_WRITE_VALUE_DEFAULT);
   if (r != CUDA_SUCCESS) {
-    // Whatever part was enqueued still has to be served: hand the proxy a task that does no work.
+    // Whatever part was enqueued still has to be served: hand the proxy a task that does no work and is released at once.
     task.kind = ProxyTask::GRAPH;
     task.exec = nullptr;
+    *passed(pair) = seq;   // nothing on the stream will write it
   }
   task.pair = pair;
+  task.seq = seq;
   {
     std::lock_guard<std::mutex> lock(mu_);
     inbox_.push_back(task);
@@ -169,6 +197,17 @@ int Proxy::pending_p2p() { return parked_.load(); }
 int Proxy::async_error() { return error_.load(); }
 void Proxy::clear_error() { error_ = 0; }
 
+void Proxy::work_stats(double* busy_us, double* span_us) const {
+  if (busy_us) *busy_us = (double)busy_ns_.load() / 1e3;
+  const long long a = first_ns_.load(), b = last_ns_.load();
+  if (span_us) *span_us = (a && b > a) ? (double)(b - a) / 1e3 : 0.0;
+}
+void Proxy::reset_work_stats() {
+  busy_ns_ = 0;
+  first_ns_ = 0;
+  last_ns_ = 0;
+}
+
 bool Proxy::drain(long timeout_ms) {
   const double t0 = now_ms();
   while (active_.load() > parked_.load()) {
@@ -178,12 +217,24 @@ bool Proxy::drain(long timeout_ms) {
   return true;
 }
 
-void Proxy::release_with_abort(int i, int err) {
-  int zero = 0;
-  error_.compare_exchange_strong(zero, err);
-  *finish_flag(i) = kFlagAbort;
+// The stream of slot i may go on (err != PROXY_OK: it is let go without its result, and the first such error sticks).
+void Proxy::release(int i, int err) {
+  if (err != PROXY_OK) {
+    int zero = 0;
+    error_.compare_exchange_strong(zero, err);
+  }
   std::atomic_thread_fence(std::memory_order_seq_cst);
-  slots_[i].state = WAIT_ACK;
+  *released(i) = slots_[i].task.seq;
+  std::atomic_thread_fence(std::memory_order_seq_cst);
+  slots_[i].state = FREE;
+  last_ns_ = now_ns();
+  {
+    std::lock_guard<std::mutex> lock(mu_);
+    pair_busy_[i] = 0;
+    active_--;
+  }
+  cv_.notify_all();
+  PTRACE("pair %d: hand-over %u released (%d)", i, slots_[i].task.seq, err);
 }
 
 void Proxy::loop() {
@@ -199,11 +250,13 @@ void Proxy::loop() {
         inbox_.pop_front();
         Slot& s = slots_[t.pair];
         s.task = t;
-        s.state = WAIT_START;
+        // a task without work comes from a hand-over that could not be enqueued completely: nothing may arrive, release it
+        s.state = (t.kind == ProxyTask::GRAPH && !t.exec) ? READY : WAIT_ARRIVE;
         s.t0 = now_ms();
         s.partner = -1;
         order[t.pair] = seq++;
-        PTRACE("pair %d: task kind %d accepted", t.pair, t.kind);
+        if (first_ns_.load() == 0) first_ns_ = now_ns();
+        PTRACE("pair %d: task kind %d accepted as hand-over %u", t.pair, t.kind, t.seq);
       }
       if (active_.load() == 0) {
         if (stop_) break;
@@ -212,9 +265,17 @@ void Proxy::loop() {
       }
     }
     if (stop_) {
-      // shutting down with work still in flight: serve it for at most one watchdog period, then give up
+      // Shutting down with hand-overs still open: they are served for at most one watchdog period; then every stream
+      // that is still held, or has not even arrived yet, is let go (it finds its release whenever it gets there).
       if (stop_since == 0) stop_since = now_ms();
-      if (now_ms() - stop_since > (double)watchdog_ms_) break;
+      if (now_ms() - stop_since > (double)watchdog_ms_) {
+        for (int i = 0; i < kFlagPairs; i++)
+          if (slots_[i].state != FREE) {
+            if (slots_[i].state == PARKED) parked_--;
+            release(i, PROXY_TIMEOUT);
+          }
+        break;
+      }
     }
     const double now = now_ms();
     const double limit = (double)watchdog_ms_;
@@ -224,12 +285,11 @@ void Proxy::loop() {
       switch (s.state) {
         case FREE:
           break;
-        case WAIT_START:
-          if (*start_flag(i) == kFlagStart) {
+        case WAIT_ARRIVE:
+          if (*arrived(i) == s.task.seq) {
             std::atomic_thread_fence(std::memory_order_seq_cst);
-            *start_flag(i) = 0;  // acknowledgement: the stream moves on to its wait for the finish flag
             handshakes_++;
-            PTRACE("pair %d: start seen, acknowledged", i);
+            PTRACE("pair %d: the stream has arrived", i);
             s.state = READY;
             s.t0 = now;
           } else if (now - s.t0 > limit) {
@@ -238,17 +298,19 @@ void Proxy::loop() {
           }
           break;
         case READY: {
+          const long long w0 = now_ns();
           if (s.task.kind == ProxyTask::GRAPH) {
             cudaError_t e = cudaSuccess;
             if (s.task.exec) e = cudaGraphLaunch(s.task.exec, stream_);
             if (e == cudaSuccess) e = cudaEventRecord(s.done, stream_);
             PTRACE("pair %d: schedule launched on the proxy stream (%s)", i, cudaGetErrorString(e));
             if (e != cudaSuccess) {
-              release_with_abort(i, PROXY_CUDA);
+              release(i, PROXY_CUDA);
             } else {
               s.state = RUNNING;
               s.t0 = now;
             }
+            busy_ns_ += now_ns() - w0;
             break;
           }
           // send/recv: look for the oldest parked partner of the same (src, dst) pair and the other direction
@@ -263,13 +325,15 @@ void Proxy::loop() {
             s.state = PARKED;
             s.t0 = now;
             parked_++;
+            busy_ns_ += now_ns() - w0;
             break;
           }
           Slot& o = slots_[best];
           parked_--;
           if (o.task.count != s.task.count || o.task.dtype != s.task.dtype) {
-            release_with_abort(best, PROXY_MISMATCH);
-            release_with_abort(i, PROXY_MISMATCH);
+            release(best, PROXY_MISMATCH);
+            release(i, PROXY_MISMATCH);
+            busy_ns_ += now_ns() - w0;
             break;
           }
           const void* src = s.task.is_send ? s.task.buf : o.task.buf;
@@ -289,8 +353,9 @@ void Proxy::loop() {
           }
           if (e == cudaSuccess) e = cudaEventRecord(s.done, stream_);
           if (e != cudaSuccess) {
-            release_with_abort(best, PROXY_CUDA);
-            release_with_abort(i, PROXY_CUDA);
+            release(best, PROXY_CUDA);
+            release(i, PROXY_CUDA);
+            busy_ns_ += now_ns() - w0;
             break;
           }
           s.partner = best;
@@ -298,12 +363,13 @@ void Proxy::loop() {
           s.t0 = now;
           o.state = RUNNING;  // passive: finished by slot i
           o.partner = -2;
+          busy_ns_ += now_ns() - w0;
           break;
         }
         case PARKED:
           if (now - s.t0 > limit) {  // nobody posted the other side: let the stream go and report it
             parked_--;
-            release_with_abort(i, PROXY_TIMEOUT);
+            release(i, PROXY_TIMEOUT);
           }
           break;
         case RUNNING: {
@@ -315,38 +381,19 @@ void Proxy::loop() {
               error_.compare_exchange_strong(zero, PROXY_TIMEOUT);  // reported; the work may still be making progress
             }
             if (now - s.t0 <= 4 * limit) break;
-            // Four watchdog periods without completion: the work is considered stuck.  The stream is released with
-            // the abort value so that nothing waits on this library forever; the result is undefined and the sticky
-            // error says so.
+            // Four watchdog periods without completion: the work is considered stuck.  The stream is let go so that
+            // nothing waits on this library forever; the result is undefined and the sticky error says so.
             q = cudaErrorTimeout;
           }
-          PTRACE("pair %d: work complete (%s), finish flag written", i, cudaGetErrorString(q));
-          const uint32_t v = (q == cudaSuccess) ? kFlagFinish : kFlagAbort;
-          if (q != cudaSuccess) {
-            int zero = 0;
-            error_.compare_exchange_strong(zero, PROXY_CUDA);
-          }
-          std::atomic_thread_fence(std::memory_order_seq_cst);
-          *finish_flag(i) = v;
-          s.state = WAIT_ACK;
-          if (s.partner >= 0) {
-            *finish_flag(s.partner) = v;
-            slots_[s.partner].state = WAIT_ACK;
-          }
+          const long long w0 = now_ns();
+          PTRACE("pair %d: work complete (%s)", i, cudaGetErrorString(q));
+          const int err = (q == cudaSuccess) ? PROXY_OK : PROXY_CUDA;
+          const int partner = s.partner;
+          release(i, err);
+          if (partner >= 0) release(partner, err);
+          busy_ns_ += now_ns() - w0;
           break;
         }
-        case WAIT_ACK:
-          if (*finish_flag(i) == 0) {  // the stream has taken the result and reset the flag: the pair is free again
-            PTRACE("pair %d: stream acknowledged, pair free", i);
-            s.state = FREE;
-            {
-              std::lock_guard<std::mutex> lock(mu_);
-              pair_busy_[i] = 0;
-              active_--;
-            }
-            cv_.notify_all();
-          }
-          break;
       }
     }
   }

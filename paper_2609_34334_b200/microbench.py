@@ -18,6 +18,7 @@ import json
 import torch
 
 from . import binding as hb
+from . import diag as hd
 
 
 def main():
@@ -39,10 +40,10 @@ def main():
         o = torch.empty(n, dtype=torch.bfloat16, device="cuda")
         sink = torch.zeros(1, dtype=torch.int32, device="cuda")
         st = torch.cuda.Stream()
-        cases = {"read_only": (lambda: hb.port_probe("read", a, nbytes, args.ctas, sink, st), nbytes),
-                 "write_only": (lambda: hb.port_probe("write", o, nbytes, args.ctas, sink, st), nbytes),
-                 "copy_1r_1w": (lambda: hb.copy_launch(a, o, nbytes, args.ctas, st), 2 * nbytes),
-                 "sum_2r_1w": (lambda: hb.sum_launch(a, b, o, n, "bf16", args.ctas, st), 3 * nbytes)}
+        cases = {"read_only": (lambda: hd.port_probe("read", a, nbytes, args.ctas, sink, st), nbytes),
+                 "write_only": (lambda: hd.port_probe("write", o, nbytes, args.ctas, sink, st), nbytes),
+                 "copy_1r_1w": (lambda: hd.copy_launch(a, o, nbytes, args.ctas, st), 2 * nbytes),
+                 "sum_2r_1w": (lambda: hd.sum_launch(a, b, o, n, "bf16", args.ctas, st), 3 * nbytes)}
         out = {"probe": "memory ports of %d SMs (one 1024-thread CTA each), %d MiB operands" % (args.ctas, args.mib), "ctas": args.ctas}
         for name, (fn, moved) in cases.items():
             for _ in range(args.warmup):
@@ -71,7 +72,7 @@ def main():
         torch.cuda.synchronize()
 
         def chain(k):
-            assert hb.chain_launch(inbox[k], nbytes, nsrc, local[k], out_t[k], n, args.dtype, args.ctas, st) == hb.OK
+            assert hd.chain_launch(inbox[k], nbytes, nsrc, local[k], out_t[k], n, args.dtype, args.ctas, st) == hb.OK
 
         for k in range(max(args.warmup, sets)):
             chain(k % sets)
@@ -101,11 +102,11 @@ def main():
         st = torch.cuda.Stream()
 
         def fan(k):
-            assert hb.fanout_launch(srcs[k], dsts[k], nbytes, args.ctas, st) == hb.OK
+            assert hd.fanout_launch(srcs[k], dsts[k], nbytes, args.ctas, st) == hb.OK
 
         def copies(k):
             for d in dsts[k]:
-                assert hb.copy_launch(srcs[k], d, nbytes, args.ctas, st) == hb.OK
+                assert hd.copy_launch(srcs[k], d, nbytes, args.ctas, st) == hb.OK
 
         out = {"kernel": "fan", "mib_per_operand": args.mib, "destinations": nd, "ctas": args.ctas}
         for name, fn, moved in (("fan_out", fan, (1 + nd) * nbytes), ("separate_copies", copies, 2 * nd * nbytes)):
@@ -165,7 +166,7 @@ def main():
         comm = hb.Comm(2, 0)
         comm.set_param("copy_ctas", args.ctas)
         comm.set_host_staging(host)
-        rows = comm.probe_copy_routes(dst, src, nbytes, 3000)
+        rows = hd.probe_copy_routes(comm, dst, src, nbytes, 3000)
         comm.destroy()
         print(json.dumps({"probe": "copy routes under a kernel that holds every SM for 3000 us", "mib": args.mib,
                           "routes": [{"route": n, "needs_sm": s, "end_us": round(t, 1)} for n, s, t in rows]}))
@@ -180,9 +181,9 @@ def main():
 
     def launch():
         if args.kernel == "sum":
-            rc = hb.sum_launch(a, b, o, n, args.dtype, args.ctas, st)
+            rc = hd.sum_launch(a, b, o, n, args.dtype, args.ctas, st)
         else:
-            rc = hb.copy_launch(a, o, nbytes, args.ctas, st)
+            rc = hd.copy_launch(a, o, nbytes, args.ctas, st)
         assert rc == hb.OK, rc
 
     for _ in range(args.warmup):

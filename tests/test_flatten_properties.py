@@ -10,13 +10,14 @@ from hypothesis import HealthCheck, given, settings
 from hypothesis import strategies as st
 
 from paper_2609_34334_b200 import binding as hb
+from paper_2609_34334_b200 import diag as hd
 
 
 def _replay(kind, dtype, ctas, addrs_a, addrs_b, addrs_o, lens):
     """Returns per segment a byte-coverage count array, replaying the device loops for every CTA and thread."""
     e = 1 if kind == "copy" else (4 if dtype == "fp32" else 2)
     ve = 16 // e
-    view, tile_v = hb.flatten_inspect(kind, dtype, ctas, addrs_a, addrs_b, addrs_o, lens)
+    view, tile_v = hd.flatten_inspect(kind, dtype, ctas, addrs_a, addrs_b, addrs_o, lens)
     cover = [np.zeros(n * e, dtype=np.int32) for n in lens]
     tiles_prev, scal_prev = 0, 0
     for k, (head, nvec, tiles_end, scal_end) in enumerate(view):
@@ -69,14 +70,14 @@ def test_every_byte_of_every_segment_is_touched_exactly_once(kind, dtype, ctas, 
 
 
 def test_aligned_segments_take_the_vector_path():
-    view, tile_v = hb.flatten_inspect("sum", "bf16", 8, [4096, 8192 + 6], [1 << 20, (1 << 20) + 6], [2 << 20, (2 << 20) + 6], [8000, 8003])
+    view, tile_v = hd.flatten_inspect("sum", "bf16", 8, [4096, 8192 + 6], [1 << 20, (1 << 20) + 6], [2 << 20, (2 << 20) + 6], [8000, 8003])
     assert tile_v == 4 * 1024
     (h0, v0, t0, s0), (h1, v1, t1, s1) = view
     assert (h0, v0, s0) == (0, 1000, 0) and t0 == 1
     assert h1 == 5 and v1 == (8003 - 5) // 8 and s1 == 8003 - v1 * 8       # 6 bytes off: 5 bf16 elements up to the next 16-byte line
-    view, tile_v = hb.flatten_inspect("copy", "bf16", 148, [4096 + 3], None, [8192 + 3], [100_000])
+    view, tile_v = hd.flatten_inspect("copy", "bf16", 148, [4096 + 3], None, [8192 + 3], [100_000])
     assert tile_v == 4 * 512 and view[0][0] == 13 and view[0][1] == (100_000 - 13) // 16
-    view, _ = hb.flatten_inspect("copy", "bf16", 8, [4096 + 3], None, [8192 + 4], [100_000])
+    view, _ = hd.flatten_inspect("copy", "bf16", 8, [4096 + 3], None, [8192 + 4], [100_000])
     assert view[0][1] == 0 and view[0][3] == 100_000                         # no common phase: element-wise fallback
 
 
@@ -98,7 +99,7 @@ def test_fan_out_packing_serves_every_move_exactly_once(moves, n_len, ctas):
         src = base + s * (1 << 24) + src_phase.setdefault(s, sp)      # one address per source
         dst = base + (64 + k) * (1 << 24) + (src % 16 + dp) % 16      # mostly in phase with the source
         flat.append((src, dst, lens[l % n_len]))
-    segs, launches = hb.fanout_inspect(flat, ctas)
+    segs, launches = hd.fanout_inspect(flat, ctas)
     repeats = len({(m[0], m[2], m[1] % 16) for m in flat}) < len(flat)
     if not repeats:
         assert segs == [] and launches == 0
@@ -127,7 +128,7 @@ def test_fan_out_packing_of_a_direct_all_gather():
     R, chunk = 8, 3_276_800
     recv = [(1 << 33) + r * (1 << 28) for r in range(R)]
     moves = [(recv[r] + r * chunk, recv[(r + k) % R] + r * chunk, chunk) for k in range(1, R) for r in range(R)]
-    segs, launches = hb.fanout_inspect(moves, 148)
+    segs, launches = hd.fanout_inspect(moves, 148)
     assert launches == 1 and len(segs) == R
     for launch, src, ln, dsts, head, nvec in segs:
         r = (src - recv[0]) // (1 << 28)
@@ -137,5 +138,5 @@ def test_fan_out_packing_of_a_direct_all_gather():
     R = 40
     recv = [(1 << 33) + r * (1 << 26) for r in range(R)]
     moves = [(recv[r] + r * 4096, recv[(r + k) % R] + r * 4096, 4096) for k in range(1, R) for r in range(R)]
-    segs, launches = hb.fanout_inspect(moves, 16)
+    segs, launches = hd.fanout_inspect(moves, 16)
     assert launches == -(-R * (R - 1) // 256) and sum(len(s[3]) for s in segs) == R * (R - 1)

@@ -9,6 +9,7 @@ import pytest
 import torch
 
 from paper_2609_34334_b200 import binding as hb
+from paper_2609_34334_b200 import diag as hd
 from paper_2609_34334_b200 import workloads as W
 from gpu_util import DevBuf, np_dtype, same_bits
 from test_gpu_parity import make_comm, run_allreduce
@@ -130,7 +131,7 @@ def test_fanout_kernel_moves_exact_bytes(ctas):
         for offs in ([0] * (ndst + 1), [3] * (ndst + 1), [(5 * k) % 16 for k in range(ndst + 1)]):
             src = DevBuf(nbytes, offs[0]).put(data)
             dsts = [DevBuf(nbytes, offs[1 + d]) for d in range(ndst)]
-            assert hb.fanout_launch(src, dsts, nbytes, ctas) == hb.OK
+            assert hd.fanout_launch(src, dsts, nbytes, ctas) == hb.OK
             torch.cuda.synchronize()
             assert (src.get(np.uint8) == data).all() and src.guards_intact()
             for d in dsts:
@@ -138,9 +139,9 @@ def test_fanout_kernel_moves_exact_bytes(ctas):
                 assert d.guards_intact()
     # refused: overlapping destinations, destination over the source, too many destinations
     big = DevBuf(4096)
-    assert hb.fanout_launch(big.ptr, [big.ptr + 1024, big.ptr + 1500], 1024, 8) == hb.ERR_INVALID_ARG
-    assert hb.fanout_launch(big.ptr, [big.ptr + 512], 1024, 8) == hb.ERR_INVALID_ARG
-    assert hb.fanout_launch(big.ptr, [big.ptr + 2048] * 257, 16, 8) == hb.ERR_INVALID_ARG
+    assert hd.fanout_launch(big.ptr, [big.ptr + 1024, big.ptr + 1500], 1024, 8) == hb.ERR_INVALID_ARG
+    assert hd.fanout_launch(big.ptr, [big.ptr + 512], 1024, 8) == hb.ERR_INVALID_ARG
+    assert hd.fanout_launch(big.ptr, [big.ptr + 2048] * 257, 16, 8) == hb.ERR_INVALID_ARG
 
 
 @pytest.mark.parametrize("use_graph", [0, 1])

@@ -6,6 +6,7 @@ import pytest
 import torch
 
 from paper_2609_34334_b200 import binding as hb
+from paper_2609_34334_b200 import diag as hd
 from paper_2609_34334_b200 import workloads as W
 from gpu_util import DevBuf, np_dtype, same_bits
 from test_gpu_parity import make_comm, run_allreduce, SMALL
@@ -170,7 +171,7 @@ def test_bounded_barrier_wait_runs_out_and_is_reported(oracle):
     dst = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")
     assert comm.async_error() == hb.OK
     t0 = time.time()
-    assert comm.selftest_barrier_timeout(dst, src, nbytes) == hb.OK
+    assert hd.selftest_barrier_timeout(comm, dst, src, nbytes) == hb.OK
     torch.cuda.synchronize()
     waited = time.time() - t0
     assert 0.05 < waited < 30.0, waited                       # it really waited, and it really stopped by itself

@@ -1,13 +1,15 @@
 """Randomised GPU parity (hypothesis, derandomised so that every run draws the same cases): operation, rank count,
 element count, dtype, path, executor, piece settings, variants, in-place form and per-rank byte offsets are drawn
 together, values include signed zeros, subnormals, infinities and NaNs, and every result is compared with the
-oracle bit for bit (any NaN matches any NaN).  What must hold: no setting and no layout changes a bit."""
+oracle bit for bit (any NaN matches any NaN).  What must hold: no setting and no layout changes a bit, and a combination
+of settings that does not fit together (as the host-only option rules say) is refused with nothing enqueued."""
 import numpy as np
 import pytest
 import torch
 from hypothesis import given, settings, strategies as st, HealthCheck
 
 from paper_2609_34334_b200 import binding as hb
+from paper_2609_34334_b200 import diag as hd
 from paper_2609_34334_b200 import workloads as W
 from gpu_util import DevBuf, np_dtype, same_bits
 from test_gpu_parity import make_comm
@@ -53,6 +55,7 @@ case = st.fixed_dictionaries({
     "seed": st.integers(0, 2 ** 31 - 1),
     "ag_direct": st.integers(0, 2),
     "rs_direct": st.integers(0, 2),
+    "ce_small_kib": st.sampled_from([0, 0, 64, 8192]),
 })
 
 
@@ -68,11 +71,29 @@ def test_random_cases_match_the_oracle(oracle, c):
     total = count if op == "allreduce" else count * R
     offs = [o * e for o in c["offs"][:R]]
     params = dict(use_graph=c["use_graph"], piece_bytes=c["piece_kib"] << 10, max_pieces=c["max_pieces"], sum_ctas=c["ctas"],
-                  copy_ctas=c["ctas"], ag_direct=c["ag_direct"], rs_direct=c["rs_direct"])
+                  copy_ctas=c["ctas"], ag_direct=c["ag_direct"], rs_direct=c["rs_direct"], ce_small_bytes=c["ce_small_kib"] << 10)
     if c["variant"] != "plain":
         params[c["variant"]] = 1
     comm = make_comm(R, max(total, 1), dtype, c["path"], **params)
     npd = np_dtype(dtype)
+    # what the option rules say about this combination, without a device
+    kind = {"allreduce": hd.PLAN_ALLREDUCE, "reduce_scatter": hd.PLAN_REDUCE_SCATTER, "allgather": hd.PLAN_ALLGATHER,
+            "alltoall": hd.PLAN_ALLTOALL}[op]
+    verdict, _ = hd.options_resolve(kind, R, count, dtype, c["path"], **{k: v for k, v in params.items()
+                                                                     if k in ("use_graph", "ag_direct", "rs_direct", "onepass", "forward",
+                                                                              "fused", "ce_small_bytes", "copy_ctas")})
+    if verdict != hb.OK:
+        assert verdict == hb.ERR_UNSUPPORTED
+        send = [DevBuf(max(total, 1) * e) for _ in range(R)]
+        recv = [DevBuf(max(total, 1) * e, fill=0x3C) for _ in range(R)]
+        fn = {"allreduce": comm.allreduce_rc, "reduce_scatter": comm.reduce_scatter_rc, "allgather": comm.allgather_rc,
+              "alltoall": comm.alltoall_rc}[op]
+        assert fn(send, recv, count, dtype) == hb.ERR_UNSUPPORTED, c
+        torch.cuda.synchronize()
+        for b in recv:
+            assert (b.get(np.uint8) == 0x3C).all() and b.guards_intact(), c      # nothing was enqueued
+        assert comm.destroy() == hb.OK
+        return
     if op == "allreduce":
         xs = [_values(rng, count, dtype, c["flavour"]) for _ in range(R)]
         want = oracle.ring_allreduce(xs)

@@ -6,6 +6,7 @@ import pytest
 import torch
 
 from paper_2609_34334_b200 import binding as hb
+from paper_2609_34334_b200 import diag as hd
 from paper_2609_34334_b200 import workloads as W
 from gpu_util import DevBuf, np_dtype, same_bits
 
@@ -83,7 +84,7 @@ def test_host_bounce_moves_need_no_sm_and_staging_is_checked():
     comm.set_host_staging(torch.empty(32 << 20, dtype=torch.uint8).pin_memory())
     src = torch.ones(8 << 20, dtype=torch.uint8, device="cuda")
     dst = torch.zeros(8 << 20, dtype=torch.uint8, device="cuda")
-    needs_sm, end_us = comm.probe_move_needs_sm(hb.PATH_CE_HOST, dst, src, src.numel(), 3000)
+    needs_sm, end_us = hd.probe_move_needs_sm(comm, hb.PATH_CE_HOST, dst, src, src.numel(), 3000)
     assert needs_sm is False and end_us < 2700            # finished while a kernel held every SM: copy engines only
     assert torch.equal(src, dst)
     comm.set_param("handshake", 1)

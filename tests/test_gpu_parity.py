@@ -9,6 +9,7 @@ import pytest
 import torch
 
 from paper_2609_34334_b200 import binding as hb
+from paper_2609_34334_b200 import diag as hd
 from paper_2609_34334_b200 import workloads as W
 from gpu_util import DevBuf, np_dtype, same_bits
 
@@ -27,6 +28,9 @@ def make_comm(R, count, dtype, path=hb.PATH_CE, **params):
     """Communicator with guarded scratch for buffers of up to `count` elements (allreduce convention)."""
     comm = hb.Comm(R, 0)
     comm.set_path(path)
+    # these tests are small: without this, every call on the copy route would take the small-message rule and run on the
+    # copy kernel; the rule has tests of its own (test_small_messages_on_the_copy_route)
+    params.setdefault("ce_small_bytes", 0)
     for k, v in params.items():
         comm.set_param(k, v)
     nb = hb.scratch_bytes_direct(R, count, dtype) if params.get("rs_direct") else hb.scratch_bytes(R, count, dtype)
@@ -67,7 +71,7 @@ def test_sum_kernel_against_oracle(oracle, dtype, ctas):
             A = DevBuf(n * e, offs[0]).put(a)
             B = DevBuf(n * e, offs[1]).put(b)
             O = DevBuf(n * e, offs[2])
-            assert hb.sum_launch(A, B, O, n, dtype, ctas) == hb.OK
+            assert hd.sum_launch(A, B, O, n, dtype, ctas) == hb.OK
             torch.cuda.synchronize()
             assert same_bits(O.get(np_dtype(dtype)), want, dtype), (n, offs)
             assert A.guards_intact() and B.guards_intact() and O.guards_intact()
@@ -81,7 +85,7 @@ def test_copy_kernel_is_identity(ctas):
         for so, do in ((0, 0), (1, 1), (3, 3), (5, 2), (0, 9)):
             S = DevBuf(nbytes, so).put(src)
             D = DevBuf(nbytes, do)
-            assert hb.copy_launch(S, D, nbytes, ctas) == hb.OK
+            assert hd.copy_launch(S, D, nbytes, ctas) == hb.OK
             torch.cuda.synchronize()
             assert (D.get(np.uint8) == src).all() and D.guards_intact() and S.guards_intact()
 
@@ -93,7 +97,7 @@ def test_sum_kernel_special_values(oracle):
     b = np.array([1.0, 1.0, -0.0, tiny, -1.0, inf, 3e38, -3e-41, -1e-45] * 5, dtype=np.float32)
     want = oracle.ring_allreduce([b, a])[0]
     A, B, O = DevBuf(a.nbytes).put(a), DevBuf(b.nbytes).put(b), DevBuf(a.nbytes)
-    assert hb.sum_launch(A, B, O, a.size, "fp32", 8) == hb.OK
+    assert hd.sum_launch(A, B, O, a.size, "fp32", 8) == hb.OK
     torch.cuda.synchronize()
     got = O.get(np.float32)
     assert same_bits(got, want, "fp32")
@@ -103,7 +107,7 @@ def test_sum_kernel_special_values(oracle):
     gb16 = np.array([0x0001, 0x0001, 0x8001, 0x7F7F, 0x3F80, 0x3B80, 0xFF80, 0x3F80, 0x8000] * 3, dtype=np.uint16)
     want = oracle.ring_allreduce([gb16, hb16])[0]
     A, B, O = DevBuf(hb16.nbytes).put(hb16), DevBuf(gb16.nbytes).put(gb16), DevBuf(hb16.nbytes)
-    assert hb.sum_launch(A, B, O, hb16.size, "bf16", 8) == hb.OK
+    assert hd.sum_launch(A, B, O, hb16.size, "bf16", 8) == hb.OK
     torch.cuda.synchronize()
     assert same_bits(O.get(np.uint16), want, "bf16")
 
@@ -453,6 +457,50 @@ def test_large_periodic_inputs_full_compare(oracle):
         torch.cuda.empty_cache()
 
 
+def test_small_messages_on_the_copy_route(oracle):
+    """Default settings on HOCCL_PATH_CE: a message of at most ce_small_bytes (8 MiB) per rank moves through batched copy-kernel
+    launches (the statistics show them), a larger one through driver copies; ce_small_bytes = 0 keeps driver copies at every
+    size.  The bits are the oracle's either way, for every collective."""
+    R, dtype = 4, "fp32"
+    for n, small in ((4096, True), (2 * 1024 * 1024, True), (2 * 1024 * 1024 + 4, False)):     # 16 KiB, 8 MiB, just above
+        xs = W.rank_inputs("uniform", 300, R, n, dtype)
+        want = oracle.ring_allreduce(xs)
+        for limit in (None, 0):
+            comm = make_comm(R, n, dtype, hb.PATH_CE, **({"ce_small_bytes": 8 << 20} if limit is None else {"ce_small_bytes": 0}))
+            got = run_allreduce(comm, xs, dtype)
+            st = comm.last_stats()
+            for r in range(R):
+                assert same_bits(got[r], want[r], dtype), (n, limit, r)
+            if small and limit is None:
+                assert st["n_move_launches"] > 0 and st["max_copy_ctas"] == 148, st
+            else:
+                assert st["n_move_launches"] == 0 and st["n_moves"] > 0, st
+            assert comm.get_param("copy_ctas") == 8       # the communicator's own settings are untouched by the rule
+            comm.destroy()
+    # the other collectives under the rule
+    n = 4 * 3000
+    xs = W.rank_inputs("uniform", 301, R, n, dtype)
+    comm = make_comm(R, n, dtype, hb.PATH_CE, ce_small_bytes=8 << 20)
+    send = [DevBuf(n * 4).put(x) for x in xs]
+    rs = [DevBuf(n) for _ in range(R)]
+    comm.reduce_scatter(send, rs, n // R, dtype)
+    assert comm.last_stats()["n_move_launches"] > 0
+    ag = [DevBuf(n * 4) for _ in range(R)]
+    comm.allgather([s.ptr for s in send], ag, n // R, dtype)
+    assert comm.last_stats()["n_move_launches"] > 0
+    a2a = [DevBuf(n * 4) for _ in range(R)]
+    comm.alltoall(send, a2a, n // R, dtype)
+    assert comm.last_stats()["n_move_launches"] > 0
+    torch.cuda.synchronize()
+    wrs, wag, wa2a = oracle.ring_reduce_scatter(xs), oracle.allgather([x[:n // R] for x in xs]), oracle.alltoall(xs)
+    for r in range(R):
+        assert same_bits(rs[r].get(np.float32), wrs[r], dtype)
+        assert (ag[r].get(np.float32).view(np.uint32) == wag[r].view(np.uint32)).all()
+        assert (a2a[r].get(np.float32).view(np.uint32) == wa2a[r].view(np.uint32)).all()
+        assert rs[r].guards_intact() and ag[r].guards_intact() and a2a[r].guards_intact()
+    comm.destroy()
+
+
 # ------------------------------------------------------------------------------- ordering ---------
 def test_stream_ordering_with_neighbouring_kernels(oracle):
     """Work enqueued before the call on the same stream is seen by it; work enqueued after sees its result."""
@@ -637,10 +685,10 @@ def test_probe_move_needs_sm_terminates():
     comm.set_param("copy_ctas", 8)
     a = torch.ones(1 << 22, dtype=torch.uint8, device="cuda")
     b = torch.zeros(1 << 22, dtype=torch.uint8, device="cuda")
-    needs_sm_kernel, end_us = comm.probe_move_needs_sm(hb.PATH_SM, b, a, a.numel(), 1500)
+    needs_sm_kernel, end_us = hd.probe_move_needs_sm(comm, hb.PATH_SM, b, a, a.numel(), 1500)
     assert needs_sm_kernel is True and end_us >= 1300        # an SM copy cannot start while every SM is taken
     assert torch.equal(a, b)
-    needs_ce, end_ce = comm.probe_move_needs_sm(hb.PATH_CE, b, a, a.numel(), 1500)
+    needs_ce, end_ce = hd.probe_move_needs_sm(comm, hb.PATH_CE, b, a, a.numel(), 1500)
     assert isinstance(needs_ce, bool) and end_ce > 0         # the answer is the driver's; it is reported, not asserted
     comm.destroy()
 
@@ -655,7 +703,7 @@ def test_probe_copy_routes_controls_and_copy_kernel():
     b = torch.zeros(n, dtype=torch.uint8, device="cuda")
     host = torch.empty(n, dtype=torch.uint8).pin_memory()
     comm.set_host_staging(host)
-    rows = {name: (needs, end) for name, needs, end in comm.probe_copy_routes(b, a, n, 3000)}
+    rows = {name: (needs, end) for name, needs, end in hd.probe_copy_routes(comm, b, a, n, 3000)}
     assert len(rows) >= 9
     for name, (needs, end) in rows.items():
         assert end > 0, name
@@ -678,7 +726,7 @@ def test_kernels_occupy_as_many_sms_as_their_cta_budget(kind):
     n_sm = torch.cuda.get_device_properties(0).multi_processor_count
     for ctas in (1, 8, 32, n_sm):
         ids = torch.full((ctas,), 0xFFFF, dtype=torch.int32, device="cuda")
-        assert hb.kernel_sms(kind, a, b if kind == "sum" else None, out, n * 2, "bf16", ctas, ids) == hb.OK
+        assert hd.kernel_sms(kind, a, b if kind == "sum" else None, out, n * 2, "bf16", ctas, ids) == hb.OK
         torch.cuda.synchronize()
         got = ids.cpu().numpy()
         assert (got >= 0).all() and (got < n_sm).all()
@@ -749,7 +797,7 @@ def test_port_probe_reads_and_writes_what_it_says():
     nbytes = (3 * 128 << 10) + 4096                     # three tiles and a remainder that must stay untouched
     buf = torch.full((nbytes // 4,), -1, dtype=torch.int32, device="cuda")
     sink = torch.zeros(1, dtype=torch.int32, device="cuda")
-    assert hb.port_probe("write", buf, nbytes, 2, sink) == hb.OK
+    assert hd.port_probe("write", buf, nbytes, 2, sink) == hb.OK
     torch.cuda.synchronize()
     v = buf.cpu().numpy().reshape(-1, 4)
     tile_vecs = 8 * 1024
@@ -757,7 +805,7 @@ def test_port_probe_reads_and_writes_what_it_says():
         assert v[t * tile_vecs + u * 1024 + tid].tolist() == [t, u, tid, 0]
     assert (v[3 * tile_vecs:] == -1).all()
     before = buf.clone()
-    assert hb.port_probe("read", buf, nbytes, 2, sink) == hb.OK
+    assert hd.port_probe("read", buf, nbytes, 2, sink) == hb.OK
     torch.cuda.synchronize()
     assert torch.equal(buf, before)
-    assert hb.port_probe("read", buf, 1024, 2, sink) == hb.ERR_INVALID_ARG
+    assert hd.port_probe("read", buf, 1024, 2, sink) == hb.ERR_INVALID_ARG

@@ -9,6 +9,7 @@ import pytest
 import torch
 
 from paper_2609_34334_b200 import binding as hb
+from paper_2609_34334_b200 import diag as hd
 from paper_2609_34334_b200 import workloads as W
 from gpu_util import DevBuf, np_dtype, same_bits
 from test_gpu_parity import make_comm, run_allreduce
@@ -33,8 +34,6 @@ CONFIGS = [
     (hb.PATH_SM, dict(sum_ctas=8, copy_ctas=8, ag_direct=1)),
     (hb.PATH_SM, dict(sum_ctas=148, copy_ctas=148, ag_direct=1)),
     (hb.PATH_SM, dict(sum_ctas=3, copy_ctas=5, use_graph=0)),
-    (hb.PATH_SM, dict(fused=1, sum_ctas=148, copy_ctas=148)),             # not available as one kernel: runs as a graph
-    (hb.PATH_SM, dict(forward=1, sum_ctas=32, copy_ctas=32)),              # forward does not apply: ignored
     (hb.PATH_SM, dict(handshake=1, watchdog_ms=5000)),
     (hb.PATH_CE_HOST, dict(ag_direct=1)),
 ]
@@ -59,6 +58,28 @@ def test_allreduce_with_direct_reduce_scatter(oracle, path, params):
             if R > 1 and n >= R:
                 assert st["n_sum_launches"] == st["n_pieces"], st          # one chain launch per piece instead of R-1 sums
             comm.destroy()
+
+
+def test_what_does_not_combine_with_the_direct_reduce_scatter_is_refused():
+    """The one-kernel form has no chain phase and the direct form has no steps to forward between: asking for either together
+    with rs_direct = 1 is an error, nothing is enqueued; with rs_direct = 2 (automatic) the option that was asked for wins."""
+    R, n, dtype = 4, 4096, "fp32"
+    send = [DevBuf(n * 4) for _ in range(R)]
+    recv = [DevBuf(n * 4, fill=0x3C) for _ in range(R)]
+    for extra in (dict(fused=1), dict(forward=1), dict(onepass=1)):
+        comm = make_comm(R, n, dtype, hb.PATH_SM, rs_direct=1, **extra)
+        assert comm.allreduce_rc(send, recv, n, dtype) == hb.ERR_UNSUPPORTED, extra
+        assert comm.reduce_scatter_rc(send, [r.ptr for r in recv], n // R, dtype) == hb.ERR_UNSUPPORTED, extra
+        torch.cuda.synchronize()
+        assert all((b.get(np.uint8) == 0x3C).all() for b in recv)
+        comm.set_param("rs_direct", 2)
+        assert comm.allreduce_rc(send, recv, n, dtype) == hb.OK, extra
+        torch.cuda.synchronize()
+        assert comm.last_stats()["n_sum_launches"] != 1 or extra.get("onepass")       # not the one chain launch of the direct form
+        for b in recv:
+            b.view.fill_(0x3C)
+        torch.cuda.synchronize()
+        comm.destroy()
 
 
 @pytest.mark.parametrize("path", [hb.PATH_CE, hb.PATH_SM])
@@ -156,7 +177,7 @@ def test_native_bf16_add_equals_the_reference_add_for_all_operand_pairs():
     operands, rounded to nearest even) for all 2^32 pairs of bf16 bit patterns, NaN payloads included."""
     counts = torch.zeros(2, dtype=torch.int64, device="cuda")
     torch.cuda.synchronize()
-    assert hb.selftest_bf16_add(counts) == hb.OK
+    assert hd.selftest_bf16_add(counts) == hb.OK
     torch.cuda.synchronize()
     assert counts.tolist() == [0, 0]
 
@@ -187,16 +208,16 @@ def test_chain_kernel_against_the_oracles_chain(oracle, dtype, ctas):
             local = DevBuf(n * e, offs[1]).put(xs[c])
             out = DevBuf(n * e, offs[2])
             torch.cuda.synchronize()
-            assert hb.chain_launch(inbox, stride, R - 1, local, out, n, dtype, ctas) == hb.OK
+            assert hd.chain_launch(inbox, stride, R - 1, local, out, n, dtype, ctas) == hb.OK
             torch.cuda.synchronize()
             assert same_bits(out.get(np_dtype(dtype)), want, dtype), (dtype, R, n, offs)
             assert out.guards_intact() and inbox.guards_intact() and local.guards_intact()
             # in place on the local operand
-            assert hb.chain_launch(inbox, stride, R - 1, local, local, n, dtype, ctas) == hb.OK
+            assert hd.chain_launch(inbox, stride, R - 1, local, local, n, dtype, ctas) == hb.OK
             torch.cuda.synchronize()
             assert same_bits(local.get(np_dtype(dtype)), want, dtype), ("in place", dtype, R, n, offs)
-    assert hb.chain_launch(inbox, 24, 1, local, out, 4, dtype, 8) == hb.ERR_INVALID_ARG      # stride not a multiple of 16
-    assert hb.chain_launch(inbox, 32, 64, local, out, 4, dtype, 8) == hb.ERR_INVALID_ARG     # too many operands
+    assert hd.chain_launch(inbox, 24, 1, local, out, 4, dtype, 8) == hb.ERR_INVALID_ARG      # stride not a multiple of 16
+    assert hd.chain_launch(inbox, 32, 64, local, out, 4, dtype, 8) == hb.ERR_INVALID_ARG     # too many operands
 
 
 def test_automatic_choice_follows_the_scratch(oracle):

@@ -40,10 +40,14 @@ def test_sweep_points_match_the_oracle(oracle, R, dtype):
         send = [_dev(x, dtype) for x in xs]
         scratch = torch.empty(hb.scratch_bytes(R, n, dtype) + 256, dtype=torch.uint8, device="cuda")
         pad = (-scratch.data_ptr()) % 256
-        for path in (hb.PATH_CE, hb.PATH_SM):
+        # the copy route with its small-message rule (default: up to 8 MiB per rank the moves are copy-kernel launches), the
+        # copy route with driver copies at every size, and the SM path
+        for path, small in ((hb.PATH_CE, None), (hb.PATH_CE, 0), (hb.PATH_SM, None)):
             comm = hb.Comm(R, 0)
             comm.set_scratch(scratch.data_ptr() + pad, scratch.numel() - 256)
             comm.set_path(path)
+            if small is not None:
+                comm.set_param("ce_small_bytes", small)
             recv = [torch.zeros(n, dtype=tdt, device="cuda") for _ in range(R)]
             comm.allreduce(send, recv, n, dtype)
             torch.cuda.synchronize()

@@ -1,4 +1,4 @@
-"""The C-ABI library builds, loads and exports every symbol include/hoccl.h declares (no GPU needed)."""
+"""The C-ABI library builds, loads and exports every symbol include/hoccl.h and include/hoccl_diag.h declare (no GPU needed)."""
 import ctypes
 import os
 import re
@@ -6,12 +6,13 @@ import re
 import pytest
 
 from paper_2609_34334_b200 import binding as hb
+from paper_2609_34334_b200 import diag as hd
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
-def _declared_functions():
-    text = open(os.path.join(ROOT, "include", "hoccl.h")).read()
+def _declared_functions(header="hoccl.h"):
+    text = open(os.path.join(ROOT, "include", header)).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
     return sorted(set(re.findall(r"\b(hoccl_[a-z0-9_]+)\s*\(", text)))
 
@@ -23,6 +24,13 @@ def test_every_declared_symbol_is_exported():
     for n in names:
         assert hasattr(L, n), n
     assert sorted(hb.EXPORTS) == names, (set(names) ^ set(hb.EXPORTS))
+    # the diagnostics header and its binding
+    hd.lib()
+    dnames = _declared_functions("hoccl_diag.h")
+    assert len(dnames) >= 15 and not set(dnames) & set(names)
+    for n in dnames:
+        assert hasattr(L, n), n
+    assert sorted(hd.EXPORTS) == dnames, (set(dnames) ^ set(hd.EXPORTS))
 
 
 def test_error_strings_and_sizes():
@@ -46,12 +54,12 @@ def test_argument_errors_need_no_device():
     assert L.hoccl_comm_init(ctypes.byref(h), 0, 0) == hb.ERR_INVALID_ARG
     assert L.hoccl_comm_init(ctypes.byref(h), 65, 0) == hb.ERR_INVALID_ARG
     assert L.hoccl_comm_destroy(None) == hb.ERR_INVALID_ARG
-    assert L.hoccl_sum_launch(None, None, None, 4, 0, 8, None) == hb.ERR_INVALID_ARG
-    assert L.hoccl_sum_launch(16, 32, 48, 4, 7, 8, None) == hb.ERR_UNSUPPORTED
-    assert L.hoccl_sum_launch(18, 32, 48, 4, 0, 8, None) == hb.ERR_INVALID_ARG      # misaligned for fp32
+    assert hd.lib().hoccl_sum_launch(None, None, None, 4, 0, 8, None) == hb.ERR_INVALID_ARG
+    assert hd.lib().hoccl_sum_launch(16, 32, 48, 4, 7, 8, None) == hb.ERR_UNSUPPORTED
+    assert hd.lib().hoccl_sum_launch(18, 32, 48, 4, 0, 8, None) == hb.ERR_INVALID_ARG      # misaligned for fp32
     p = ctypes.c_void_p()
-    assert L.hoccl_plan_build(ctypes.byref(p), 0, 0, 10, 0, 0, 4096, 8, None) == hb.ERR_INVALID_ARG
-    assert L.hoccl_plan_build(ctypes.byref(p), 0, 4, 10, 9, 0, 4096, 8, None) == hb.ERR_UNSUPPORTED
+    assert hd.lib().hoccl_plan_build(ctypes.byref(p), 0, 0, 10, 0, 0, 4096, 8, None) == hb.ERR_INVALID_ARG
+    assert hd.lib().hoccl_plan_build(ctypes.byref(p), 0, 4, 10, 9, 0, 4096, 8, None) == hb.ERR_UNSUPPORTED
 
 
 def test_no_device_fails_loudly():
@@ -73,10 +81,10 @@ def test_header_is_plain_c_and_a_c_program_links_against_the_library(tmp_path):
         pytest.skip("no C compiler")
     inc = os.path.join(ROOT, "include")
     libdir = os.path.dirname(hb.library_path())
-    names = _declared_functions()
+    names = _declared_functions() + _declared_functions("hoccl_diag.h")
     src = tmp_path / "use_hoccl.c"
     refs = "\n".join("  fns[n++] = (void (*)(void))%s;" % n for n in names)
-    src.write_text('#include <stdio.h>\n#include <string.h>\n#include "hoccl.h"\nint main(void) {\n  void (*fns[128])(void);\n  int n = 0;\n'
+    src.write_text('#include <stdio.h>\n#include <string.h>\n#include "hoccl.h"\n#include "hoccl_diag.h"\nint main(void) {\n  void (*fns[128])(void);\n  int n = 0;\n'
                    + refs + '\n  if (strcmp(hoccl_error_string(HOCCL_OK), "ok") != 0) return 2;\n'
                    '  if (hoccl_scratch_bytes(1, 1000, HOCCL_FLOAT32) != 0) return 3;\n'
                    '  if (hoccl_comm_set_path(0, HOCCL_PATH_CE) != HOCCL_ERR_INVALID_ARG) return 4;\n'

@@ -12,6 +12,7 @@ import numpy as np
 import pytest
 
 from paper_2609_34334_b200 import binding as hb
+from paper_2609_34334_b200 import diag as hd
 from paper_2609_34334_b200 import workloads as W
 
 PHASE_RS, PHASE_AG, PHASE_OWN = 0, 1, 2
@@ -40,27 +41,27 @@ def _topo_order(num_groups, deps, rng):
 def _run_plan(plan, kind, R, count, dtype, xs, in_place, rng):
     e = W.elem_size(dtype)
     npdt = np.float32 if dtype == "fp32" else np.uint16
-    base = {hb.PLAN_ALLREDUCE_FWD: hb.PLAN_ALLREDUCE, hb.PLAN_REDUCE_SCATTER_FWD: hb.PLAN_REDUCE_SCATTER, hb.PLAN_ALLREDUCE_AGD: hb.PLAN_ALLREDUCE,
-            hb.PLAN_ALLREDUCE_FWD_AGD: hb.PLAN_ALLREDUCE, hb.PLAN_ALLGATHER_DIRECT: hb.PLAN_ALLGATHER}.get(kind, kind)
+    base = {hd.PLAN_ALLREDUCE_FWD: hd.PLAN_ALLREDUCE, hd.PLAN_REDUCE_SCATTER_FWD: hd.PLAN_REDUCE_SCATTER, hd.PLAN_ALLREDUCE_AGD: hd.PLAN_ALLREDUCE,
+            hd.PLAN_ALLREDUCE_FWD_AGD: hd.PLAN_ALLREDUCE, hd.PLAN_ALLGATHER_DIRECT: hd.PLAN_ALLGATHER}.get(kind, kind)
     kind = base if base < 16 else (base & 15)
-    if kind == hb.PLAN_ALLREDUCE:
+    if kind == hd.PLAN_ALLREDUCE:
         send_n, recv_n = count, count
-    elif kind == hb.PLAN_ALLTOALL:
+    elif kind == hd.PLAN_ALLTOALL:
         send_n, recv_n = R * count, R * count
-    elif kind == hb.PLAN_REDUCE_SCATTER:
+    elif kind == hd.PLAN_REDUCE_SCATTER:
         send_n, recv_n = R * count, count
     else:
         send_n, recv_n = count, R * count
     slot = plan.slot_bytes
-    if R > 1 and count > 0 and kind in (hb.PLAN_ALLREDUCE, hb.PLAN_REDUCE_SCATTER):
+    if R > 1 and count > 0 and kind in (hd.PLAN_ALLREDUCE, hd.PLAN_REDUCE_SCATTER):
         assert 0 < slot <= hb.scratch_bytes(R, send_n, dtype) // (2 * R)      # the advertised bound covers any piece setting
         bound = hb.scratch_bytes_direct(R, send_n, dtype) if plan.inbox_slots > 1 else hb.scratch_bytes(R, send_n, dtype)
         assert plan.scratch_bytes <= bound
     send = [x.copy().view(np.uint8) for x in xs]
     if in_place:
-        if kind == hb.PLAN_ALLREDUCE:
+        if kind == hd.PLAN_ALLREDUCE:
             recv = send
-        elif kind == hb.PLAN_REDUCE_SCATTER:
+        elif kind == hd.PLAN_REDUCE_SCATTER:
             recv = [send[r][r * count * e:(r + 1) * count * e] for r in range(R)]
         else:
             recv = [np.zeros(recv_n * e, dtype=np.uint8) for _ in range(R)]
@@ -71,7 +72,7 @@ def _run_plan(plan, kind, R, count, dtype, xs, in_place, rng):
         recv = [np.full(recv_n * e, 0xAB, dtype=np.uint8) for _ in range(R)]
     inbox = [np.full(slot * plan.inbox_slots, 0xCD, dtype=np.uint8) for _ in range(R)]
     partial = [np.full(slot, 0xEF, dtype=np.uint8) for _ in range(R)]
-    bufs = {hb.BUF_SEND: send, hb.BUF_RECV: recv, hb.BUF_INBOX: inbox, hb.BUF_PARTIAL: partial}
+    bufs = {hd.BUF_SEND: send, hd.BUF_RECV: recv, hd.BUF_INBOX: inbox, hd.BUF_PARTIAL: partial}
     by_group = {}
     for op in plan.ops:
         by_group.setdefault(op["group"], []).append(op)
@@ -83,13 +84,13 @@ def _run_plan(plan, kind, R, count, dtype, xs, in_place, rng):
             assert n > 0 and n % e == 0
             src = bufs[op["src_buf"]][op["rank"]][op["src_off"]:op["src_off"] + n]
             assert src.size == n
-            if op["kind"] == hb.OP_MOVE:
+            if op["kind"] == hd.OP_MOVE:
                 dst = bufs[op["dst_buf"]][op["dst_rank"]]
                 assert op["dst_off"] + n <= dst.size
                 dst[op["dst_off"]:op["dst_off"] + n] = src
-            elif op["kind"] == hb.OP_CHAIN:
-                assert dtype == "fp32" and op["rank"] == op["dst_rank"] and op["src_buf"] == hb.BUF_INBOX
-                box = bufs[hb.BUF_INBOX][op["rank"]]
+            elif op["kind"] == hd.OP_CHAIN:
+                assert dtype == "fp32" and op["rank"] == op["dst_rank"] and op["src_buf"] == hd.BUF_INBOX
+                box = bufs[hd.BUF_INBOX][op["rank"]]
                 acc = box[op["src_off"]:op["src_off"] + n].view(np.float32).copy()
                 for j in range(1, op["nsrc"]):
                     lo = op["src_off"] + j * op["src_stride"]
@@ -121,16 +122,16 @@ def test_allreduce_plan_executes_to_oracle_bits(oracle, R, n, piece_bytes, max_p
     want = oracle.ring_allreduce(xs)
     for in_place in (False, True):
         align = [(4 * rng.randrange(4)) for _ in range(R)] if in_place else None
-        plan = hb.Plan(hb.PLAN_ALLREDUCE, R, n, "fp32", in_place, piece_bytes, max_pieces, align)
+        plan = hd.Plan(hd.PLAN_ALLREDUCE, R, n, "fp32", in_place, piece_bytes, max_pieces, align)
         # SUM operands share their 16-byte phase (vector path), whatever the send pointers' alignment
         for op in plan.ops:
-            if op["kind"] == hb.OP_SUM:
+            if op["kind"] == hd.OP_SUM:
                 a = align[op["rank"]] if align else 0
                 assert op["src_off"] % 16 == (a + op["local_off"]) % 16
-                if op["dst_buf"] == hb.BUF_PARTIAL:
+                if op["dst_buf"] == hd.BUF_PARTIAL:
                     assert op["dst_off"] % 16 == op["src_off"] % 16
         for trial in range(2):
-            got = _run_plan(plan, hb.PLAN_ALLREDUCE, R, n, "fp32", xs, in_place, rng)
+            got = _run_plan(plan, hd.PLAN_ALLREDUCE, R, n, "fp32", xs, in_place, rng)
             for r in range(R):
                 assert (got[r].view(np.uint32) == want[r].view(np.uint32)).all(), (R, n, in_place, r)
 
@@ -142,17 +143,17 @@ def test_reduce_scatter_and_allgather_plans(oracle, R, count):
     xs = W.rank_inputs("uniform", 23, R, R * count, "fp32")
     want = oracle.ring_reduce_scatter(xs)
     for in_place in (False, True):
-        plan = hb.Plan(hb.PLAN_REDUCE_SCATTER, R, count, "fp32", in_place, 2048, 4)
-        got = _run_plan(plan, hb.PLAN_REDUCE_SCATTER, R, count, "fp32", xs, in_place, rng)
+        plan = hd.Plan(hd.PLAN_REDUCE_SCATTER, R, count, "fp32", in_place, 2048, 4)
+        got = _run_plan(plan, hd.PLAN_REDUCE_SCATTER, R, count, "fp32", xs, in_place, rng)
         for r in range(R):
             assert (got[r].view(np.uint32) == want[r].view(np.uint32)).all()
     for dtype in ("fp32", "bf16"):
         ys = W.rank_inputs("uniform", 29, R, count, dtype)
         cat = np.concatenate(ys)
         for in_place in (False, True):
-            plan = hb.Plan(hb.PLAN_ALLGATHER, R, count, dtype, in_place, 1024, 8)
-            assert all(op["kind"] == hb.OP_MOVE for op in plan.ops)
-            got = _run_plan(plan, hb.PLAN_ALLGATHER, R, count, dtype, ys, in_place, rng)
+            plan = hd.Plan(hd.PLAN_ALLGATHER, R, count, dtype, in_place, 1024, 8)
+            assert all(op["kind"] == hd.OP_MOVE for op in plan.ops)
+            got = _run_plan(plan, hd.PLAN_ALLGATHER, R, count, dtype, ys, in_place, rng)
             for r in range(R):
                 assert (got[r] == cat).all()
 
@@ -160,18 +161,18 @@ def test_reduce_scatter_and_allgather_plans(oracle, R, count):
 @pytest.mark.parametrize("R,n", [(2, 100), (4, 1 << 20), (8, 13_107_200), (8, 1001), (5, 12345)])
 def test_structure_rules(R, n):
     e = 4
-    plan = hb.Plan(hb.PLAN_ALLREDUCE, R, n, "fp32", False, 1 << 20, 8)
+    plan = hd.Plan(hd.PLAN_ALLREDUCE, R, n, "fp32", False, 1 << 20, 8)
     q = -(-n // R)
     lo = [min(c * q, n) for c in range(R)]
     hi = [min((c + 1) * q, n) for c in range(R)]
-    sums = [op for op in plan.ops if op["kind"] == hb.OP_SUM]
-    moves = [op for op in plan.ops if op["kind"] == hb.OP_MOVE]
+    sums = [op for op in plan.ops if op["kind"] == hd.OP_SUM]
+    moves = [op for op in plan.ops if op["kind"] == hd.OP_MOVE]
     # rank locality: a SUM touches one rank only; its operands are inbox + own send data
     for op in sums:
         assert op["rank"] == op["dst_rank"]
-        assert op["src_buf"] == hb.BUF_INBOX and op["local_buf"] == hb.BUF_SEND
+        assert op["src_buf"] == hd.BUF_INBOX and op["local_buf"] == hd.BUF_SEND
         assert op["chunk"] == (op["rank"] - 2 - op["step"]) % R
-        assert op["dst_buf"] == (hb.BUF_RECV if op["step"] == R - 2 else hb.BUF_PARTIAL)
+        assert op["dst_buf"] == (hd.BUF_RECV if op["step"] == R - 2 else hd.BUF_PARTIAL)
         assert op["src_off"] + op["bytes"] <= plan.slot_bytes
     # every ring MOVE crosses exactly one rank boundary, towards rank+1
     for op in moves:
@@ -179,11 +180,11 @@ def test_structure_rules(R, n):
         assert op["dst_rank"] == (op["rank"] + 1) % R and op["dst_rank"] != op["rank"]
         if op["phase"] == PHASE_RS:
             assert op["chunk"] == (op["rank"] - 1 - op["step"]) % R
-            assert op["dst_buf"] == hb.BUF_INBOX
-            assert op["src_buf"] == (hb.BUF_SEND if op["step"] == 0 else hb.BUF_PARTIAL)
+            assert op["dst_buf"] == hd.BUF_INBOX
+            assert op["src_buf"] == (hd.BUF_SEND if op["step"] == 0 else hd.BUF_PARTIAL)
         else:
             assert op["chunk"] == (op["rank"] - op["step"]) % R
-            assert op["src_buf"] == hb.BUF_RECV and op["dst_buf"] == hb.BUF_RECV and op["src_off"] == op["dst_off"]
+            assert op["src_buf"] == hd.BUF_RECV and op["dst_buf"] == hd.BUF_RECV and op["src_off"] == op["dst_off"]
     # coverage: per (phase, step, rank) the pieces tile the chunk exactly once
     for kind_ops, phase in ((moves, PHASE_RS), (moves, PHASE_AG), (sums, PHASE_RS)):
         seen = {}
@@ -195,7 +196,7 @@ def test_structure_rules(R, n):
         for (s, r, c), ops in seen.items():
             total = sum(o["bytes"] for o in ops)
             assert total == (hi[c] - lo[c]) * e
-            if all(o["dst_buf"] == hb.BUF_RECV for o in ops):
+            if all(o["dst_buf"] == hd.BUF_RECV for o in ops):
                 spans = sorted((o["dst_off"] - lo[c] * e, o["bytes"]) for o in ops)
                 pos = 0
                 for off, b in spans:
@@ -220,14 +221,14 @@ def test_structure_rules(R, n):
 
 def test_piece_geometry():
     # 25 MiB bf16 bucket over 8 ranks: chunk 3,276,800 B
-    plan = hb.Plan(hb.PLAN_ALLREDUCE, 8, 13_107_200, "bf16", False, 1 << 20, 8)
+    plan = hd.Plan(hd.PLAN_ALLREDUCE, 8, 13_107_200, "bf16", False, 1 << 20, 8)
     pieces = sorted({op["piece"] for op in plan.ops})
     assert pieces == [0, 1, 2, 3]
     sizes = {op["bytes"] for op in plan.ops}
     assert max(sizes) % 1024 == 0 and sum(sorted({(op["piece"], op["bytes"]) for op in plan.ops if op["rank"] == 0 and op["step"] == 0 and op["kind"] == 1}, key=lambda t: t[0])[k][1] for k in range(4)) == 3_276_800
-    one = hb.Plan(hb.PLAN_ALLREDUCE, 8, 13_107_200, "bf16", False, 64 << 20, 8)
+    one = hd.Plan(hd.PLAN_ALLREDUCE, 8, 13_107_200, "bf16", False, 64 << 20, 8)
     assert {op["piece"] for op in one.ops} == {0}
-    capped = hb.Plan(hb.PLAN_ALLREDUCE, 2, 1 << 28, "fp32", False, 1 << 20, 8)
+    capped = hd.Plan(hd.PLAN_ALLREDUCE, 2, 1 << 28, "fp32", False, 1 << 20, 8)
     assert len({op["piece"] for op in capped.ops}) == 8
 
 
@@ -238,8 +239,8 @@ def test_alltoall_plan(oracle, R, count):
     for dtype in ("fp32", "bf16"):
         xs = W.rank_inputs("uniform", 37, R, R * count, dtype)
         want = oracle.alltoall(xs)
-        plan = hb.Plan(hb.PLAN_ALLTOALL, R, count, dtype, False, 1024, 8)
-        assert all(op["kind"] == hb.OP_MOVE for op in plan.ops) and all(len(d) == 0 for d in plan.deps)
+        plan = hd.Plan(hd.PLAN_ALLTOALL, R, count, dtype, False, 1024, 8)
+        assert all(op["kind"] == hd.OP_MOVE for op in plan.ops) and all(len(d) == 0 for d in plan.deps)
         # every stage is a permutation: each rank sends one block and receives one block
         stages = {}
         for op in plan.ops:
@@ -248,11 +249,11 @@ def test_alltoall_plan(oracle, R, count):
             assert sorted(o["rank"] for o in ops) == list(range(R)) and sorted(o["dst_rank"] for o in ops) == list(range(R))
             for o in ops:
                 assert o["dst_rank"] == (o["rank"] + (k if phase == 3 else 0)) % R
-        got = _run_plan(plan, hb.PLAN_ALLTOALL, R, count, dtype, xs, False, rng)
+        got = _run_plan(plan, hd.PLAN_ALLTOALL, R, count, dtype, xs, False, rng)
         for r in range(R):
             assert (got[r] == want[r]).all()
     with pytest.raises(hb.HocclError):
-        hb.Plan(hb.PLAN_ALLTOALL, R, count, "fp32", True, 1024, 8)      # no in-place form
+        hd.Plan(hd.PLAN_ALLTOALL, R, count, "fp32", True, 1024, 8)      # no in-place form
 
 
 @pytest.mark.parametrize("R,n,piece_bytes,max_pieces", [c for c in CASES if c[0] > 1 and c[1] > 0])
@@ -262,20 +263,20 @@ def test_forward_variant_plans_execute_to_oracle_bits(oracle, R, n, piece_bytes,
     xs = W.rank_inputs("uniform", 19, R, n, "fp32")
     want = oracle.ring_allreduce(xs)
     for in_place in (False, True):
-        plan = hb.Plan(hb.PLAN_ALLREDUCE_FWD, R, n, "fp32", in_place, piece_bytes, max_pieces)
-        rs_moves = [op for op in plan.ops if op["kind"] == hb.OP_MOVE and op["phase"] == 0]
+        plan = hd.Plan(hd.PLAN_ALLREDUCE_FWD, R, n, "fp32", in_place, piece_bytes, max_pieces)
+        rs_moves = [op for op in plan.ops if op["kind"] == hd.OP_MOVE and op["phase"] == 0]
         assert all(op["step"] == 0 for op in rs_moves)
         for op in plan.ops:
-            if op["kind"] == hb.OP_SUM and op["step"] < R - 2:
+            if op["kind"] == hd.OP_SUM and op["step"] < R - 2:
                 assert op["dst_rank"] == (op["rank"] + 1) % R and op["dst_buf"] != op["src_buf"]
         for trial in range(2):
-            got = _run_plan(plan, hb.PLAN_ALLREDUCE_FWD, R, n, "fp32", xs, in_place, rng)
+            got = _run_plan(plan, hd.PLAN_ALLREDUCE_FWD, R, n, "fp32", xs, in_place, rng)
             for r in range(R):
                 assert (got[r].view(np.uint32) == want[r].view(np.uint32)).all(), (R, n, in_place, r)
     if n % R == 0:
         wrs = oracle.ring_reduce_scatter(xs)
-        plan = hb.Plan(hb.PLAN_REDUCE_SCATTER_FWD, R, n // R, "fp32", False, piece_bytes, max_pieces)
-        got = _run_plan(plan, hb.PLAN_REDUCE_SCATTER_FWD, R, n // R, "fp32", xs, False, rng)
+        plan = hd.Plan(hd.PLAN_REDUCE_SCATTER_FWD, R, n // R, "fp32", False, piece_bytes, max_pieces)
+        got = _run_plan(plan, hd.PLAN_REDUCE_SCATTER_FWD, R, n // R, "fp32", xs, False, rng)
         for r in range(R):
             assert (got[r].view(np.uint32) == wrs[r].view(np.uint32)).all()
 
@@ -287,21 +288,21 @@ def test_direct_allgather_plans(oracle, R, n, piece_bytes, max_pieces):
     rng = random.Random(R * 4242 + n)
     xs = W.rank_inputs("uniform", 29, R, n, "fp32")
     want = oracle.ring_allreduce(xs)
-    for kind in (hb.PLAN_ALLREDUCE_AGD, hb.PLAN_ALLREDUCE_FWD_AGD):
+    for kind in (hd.PLAN_ALLREDUCE_AGD, hd.PLAN_ALLREDUCE_FWD_AGD):
         for in_place in (False, True):
-            plan = hb.Plan(kind, R, n, "fp32", in_place, piece_bytes, max_pieces)
-            ring = hb.Plan(hb.PLAN_ALLREDUCE_FWD if kind == hb.PLAN_ALLREDUCE_FWD_AGD else hb.PLAN_ALLREDUCE, R, n, "fp32", in_place, piece_bytes, max_pieces)
+            plan = hd.Plan(kind, R, n, "fp32", in_place, piece_bytes, max_pieces)
+            ring = hd.Plan(hd.PLAN_ALLREDUCE_FWD if kind == hd.PLAN_ALLREDUCE_FWD_AGD else hd.PLAN_ALLREDUCE, R, n, "fp32", in_place, piece_bytes, max_pieces)
             ag = [op for op in plan.ops if op["phase"] == 1]
             ring_ag = [op for op in ring.ops if op["phase"] == 1]
             assert sum(op["bytes"] for op in ag) == sum(op["bytes"] for op in ring_ag)
             # the reduce-scatter half is the ring's, op for op
             strip = lambda ops: [{k: v for k, v in op.items() if k != "group"} for op in ops if op["phase"] != 1]
             assert strip(plan.ops) == strip(ring.ops)
-            sum_groups = {op["group"] for op in plan.ops if op["kind"] == hb.OP_SUM and op["step"] == R - 2}
+            sum_groups = {op["group"] for op in plan.ops if op["kind"] == hd.OP_SUM and op["step"] == R - 2}
             for op in ag:
-                assert op["kind"] == hb.OP_MOVE and op["chunk"] == op["rank"]                  # a rank sends what it owns
+                assert op["kind"] == hd.OP_MOVE and op["chunk"] == op["rank"]                  # a rank sends what it owns
                 assert op["dst_rank"] == (op["rank"] + op["step"] + 1) % R != op["rank"]        # stage k = step + 1
-                assert op["src_buf"] == hb.BUF_RECV and op["dst_buf"] == hb.BUF_RECV and op["src_off"] == op["dst_off"]
+                assert op["src_buf"] == hd.BUF_RECV and op["dst_buf"] == hd.BUF_RECV and op["src_off"] == op["dst_off"]
                 deps = plan.deps[op["group"]]
                 assert len(deps) == 1 and deps[0] in sum_groups                               # no stage waits for another stage
             # every (destination, chunk) pair is served exactly once per piece
@@ -331,14 +332,14 @@ def test_direct_standalone_allgather_plan(oracle, R, count):
     xs = W.rank_inputs("uniform", 37, R, count, "fp32")
     want = oracle.allgather(xs)
     for in_place in (False, True):
-        plan = hb.Plan(hb.PLAN_ALLGATHER_DIRECT, R, count, "fp32", in_place, 1024, 8)
+        plan = hd.Plan(hd.PLAN_ALLGATHER_DIRECT, R, count, "fp32", in_place, 1024, 8)
         assert all(not d for d in plan.deps)                     # nothing waits for anything
         assert plan.slot_bytes == 0
         for op in plan.ops:
-            assert op["kind"] == hb.OP_MOVE and op["chunk"] == op["rank"]
-            assert op["src_buf"] == (hb.BUF_RECV if in_place else hb.BUF_SEND)
+            assert op["kind"] == hd.OP_MOVE and op["chunk"] == op["rank"]
+            assert op["src_buf"] == (hd.BUF_RECV if in_place else hd.BUF_SEND)
         for trial in range(2):
-            got = _run_plan(plan, hb.PLAN_ALLGATHER_DIRECT, R, count, "fp32", xs, in_place, rng)
+            got = _run_plan(plan, hd.PLAN_ALLGATHER_DIRECT, R, count, "fp32", xs, in_place, rng)
             for r in range(R):
                 assert (got[r].view(np.uint32) == want[r].view(np.uint32)).all()
 
@@ -351,25 +352,25 @@ def test_direct_reduce_scatter_plans(oracle, R, n, piece_bytes, max_pieces):
     rng = random.Random(R * 515 + n)
     xs = W.rank_inputs("uniform", 41, R, n, "fp32")
     want = oracle.ring_allreduce(xs)
-    for flags in (hb.PLAN_FLAG_RS_DIRECT, hb.PLAN_FLAG_RS_DIRECT | hb.PLAN_FLAG_AG_DIRECT):
-        kind = hb.PLAN_ALLREDUCE | flags
+    for flags in (hd.PLAN_FLAG_RS_DIRECT, hd.PLAN_FLAG_RS_DIRECT | hd.PLAN_FLAG_AG_DIRECT):
+        kind = hd.PLAN_ALLREDUCE | flags
         for in_place in (False, True):
             align = [(4 * rng.randrange(4)) for _ in range(R)] if in_place else None
-            plan = hb.Plan(kind, R, n, "fp32", in_place, piece_bytes, max_pieces, align)
+            plan = hd.Plan(kind, R, n, "fp32", in_place, piece_bytes, max_pieces, align)
             assert plan.inbox_slots == R - 1
             q = -(-n // R)
-            rs_moves = [op for op in plan.ops if op["kind"] == hb.OP_MOVE and op["phase"] == 0]
-            chains = [op for op in plan.ops if op["kind"] == hb.OP_CHAIN]
-            assert not [op for op in plan.ops if op["kind"] == hb.OP_SUM]
+            rs_moves = [op for op in plan.ops if op["kind"] == hd.OP_MOVE and op["phase"] == 0]
+            chains = [op for op in plan.ops if op["kind"] == hd.OP_CHAIN]
+            assert not [op for op in plan.ops if op["kind"] == hd.OP_SUM]
             for op in rs_moves:
                 k = op["step"] + 1
-                assert op["dst_rank"] == (op["rank"] + k) % R == op["chunk"] and op["src_buf"] == hb.BUF_SEND and op["dst_buf"] == hb.BUF_INBOX
+                assert op["dst_rank"] == (op["rank"] + k) % R == op["chunk"] and op["src_buf"] == hd.BUF_SEND and op["dst_buf"] == hd.BUF_INBOX
                 assert not plan.deps[op["group"]]
                 slot = op["dst_off"] // plan.slot_bytes
                 assert (op["dst_rank"] + 1 + slot) % R == op["rank"]            # slot j holds source d+1+j: the ring's order
             for op in chains:
                 assert op["rank"] == op["dst_rank"] == op["chunk"] and op["nsrc"] == R - 1 and op["src_stride"] == plan.slot_bytes
-                assert op["local_buf"] == hb.BUF_SEND and op["dst_buf"] == hb.BUF_RECV
+                assert op["local_buf"] == hd.BUF_SEND and op["dst_buf"] == hd.BUF_RECV
                 a = align[op["rank"]] if align else 0
                 assert op["src_off"] % 16 == (a + op["local_off"]) % 16          # operands share their 16-byte phase
             moved = sum(op["bytes"] for op in rs_moves)
@@ -380,14 +381,14 @@ def test_direct_reduce_scatter_plans(oracle, R, n, piece_bytes, max_pieces):
                     assert (got[r].view(np.uint32) == want[r].view(np.uint32)).all(), (flags, R, n, in_place, r)
     if n % R == 0:
         wrs = oracle.ring_reduce_scatter(xs)
-        kind = hb.PLAN_REDUCE_SCATTER | hb.PLAN_FLAG_RS_DIRECT
+        kind = hd.PLAN_REDUCE_SCATTER | hd.PLAN_FLAG_RS_DIRECT
         for in_place in (False, True):
-            plan = hb.Plan(kind, R, n // R, "fp32", in_place, piece_bytes, max_pieces)
+            plan = hd.Plan(kind, R, n // R, "fp32", in_place, piece_bytes, max_pieces)
             got = _run_plan(plan, kind, R, n // R, "fp32", xs, in_place, rng)
             for r in range(R):
                 res = got[r] if not in_place else got[r]
                 assert (res.view(np.uint32) == wrs[r].view(np.uint32)).all(), (R, n, in_place, r)
     # flags that do not apply are ignored, unknown ones refused
-    assert hb.Plan(hb.PLAN_ALLGATHER | hb.PLAN_FLAG_RS_DIRECT, R, 8, "fp32").inbox_slots == 1
+    assert hd.Plan(hd.PLAN_ALLGATHER | hd.PLAN_FLAG_RS_DIRECT, R, 8, "fp32").inbox_slots == 1
     with pytest.raises(hb.HocclError):
-        hb.Plan(hb.PLAN_ALLREDUCE | 128, R, 8, "fp32")
+        hd.Plan(hd.PLAN_ALLREDUCE | 128, R, 8, "fp32")

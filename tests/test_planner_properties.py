@@ -8,6 +8,7 @@ from hypothesis import HealthCheck, given, settings
 from hypothesis import strategies as st
 
 from paper_2609_34334_b200 import binding as hb
+from paper_2609_34334_b200 import diag as hd
 from paper_2609_34334_b200 import workloads as W
 from test_planner import _run_plan
 
@@ -20,20 +21,20 @@ def test_allreduce_plans(oracle, R, n, piece_kib, max_pieces, in_place, forward,
     xs = W.rank_inputs("uniform", seed % 1000, R, n, "fp32")
     want = oracle.ring_allreduce(xs)
     align = [4 * rng.randrange(4) for _ in range(R)]
-    kind = hb.PLAN_ALLREDUCE_FWD if forward else hb.PLAN_ALLREDUCE
-    plan = hb.Plan(kind, R, n, "fp32", in_place, piece_kib * 1024, max_pieces, align)
+    kind = hd.PLAN_ALLREDUCE_FWD if forward else hd.PLAN_ALLREDUCE
+    plan = hd.Plan(kind, R, n, "fp32", in_place, piece_kib * 1024, max_pieces, align)
     if n == 0:
         assert plan.ops == []
         return
     by = {}
     for op in plan.ops:
         assert op["bytes"] > 0
-        if op["kind"] == hb.OP_SUM and not forward:
+        if op["kind"] == hd.OP_SUM and not forward:
             assert op["rank"] == op["dst_rank"]
         for buf, rank, off in ((op["src_buf"], op["rank"], op["src_off"]), (op["dst_buf"], op["dst_rank"], op["dst_off"])):
-            if buf in (hb.BUF_INBOX, hb.BUF_PARTIAL):
+            if buf in (hd.BUF_INBOX, hd.BUF_PARTIAL):
                 assert off + op["bytes"] <= plan.slot_bytes
-        if op["kind"] == hb.OP_SUM:                      # pieces of one (step, rank) never overlap in the inbox slot
+        if op["kind"] == hd.OP_SUM:                      # pieces of one (step, rank) never overlap in the inbox slot
             by.setdefault((op["step"], op["rank"]), []).append((op["src_off"], op["bytes"]))
     for spans in by.values():
         spans.sort()
@@ -52,17 +53,17 @@ def test_other_collective_plans(oracle, R, count, kind, in_place, seed):
     if kind == "rs":
         xs = W.rank_inputs("uniform", seed % 997, R, R * count, "fp32")
         want = oracle.ring_reduce_scatter(xs)
-        plan = hb.Plan(hb.PLAN_REDUCE_SCATTER, R, count, "fp32", in_place, 2048, 5)
-        got = _run_plan(plan, hb.PLAN_REDUCE_SCATTER, R, count, "fp32", xs, in_place, rng)
+        plan = hd.Plan(hd.PLAN_REDUCE_SCATTER, R, count, "fp32", in_place, 2048, 5)
+        got = _run_plan(plan, hd.PLAN_REDUCE_SCATTER, R, count, "fp32", xs, in_place, rng)
     elif kind == "ag":
         xs = W.rank_inputs("uniform", seed % 997, R, count, "bf16")
         want = oracle.allgather(xs)
-        plan = hb.Plan(hb.PLAN_ALLGATHER, R, count, "bf16", in_place, 1024, 4)
-        got = _run_plan(plan, hb.PLAN_ALLGATHER, R, count, "bf16", xs, in_place, rng)
+        plan = hd.Plan(hd.PLAN_ALLGATHER, R, count, "bf16", in_place, 1024, 4)
+        got = _run_plan(plan, hd.PLAN_ALLGATHER, R, count, "bf16", xs, in_place, rng)
     else:
         xs = W.rank_inputs("uniform", seed % 997, R, R * count, "bf16")
         want = oracle.alltoall(xs)
-        plan = hb.Plan(hb.PLAN_ALLTOALL, R, count, "bf16", False, 1024, 4)
-        got = _run_plan(plan, hb.PLAN_ALLTOALL, R, count, "bf16", xs, False, rng)
+        plan = hd.Plan(hd.PLAN_ALLTOALL, R, count, "bf16", False, 1024, 4)
+        got = _run_plan(plan, hd.PLAN_ALLTOALL, R, count, "bf16", xs, False, rng)
     for r in range(R):
         assert (got[r].view(np.uint8) == want[r].view(np.uint8)).all()
