@@ -250,6 +250,18 @@ class GradientStream:
 C4_GRADIENTS = GradientStream()
 
 
+def gradient_bucket(g: GradientStream, b: int):
+    """The R per-rank arrays of bucket b of the gradient stream: elements [b * per, b * per + len) of every rank's flat
+    gradient, normal(0, sigma) from the stream's seed (position independent, so any bucket can be produced alone)."""
+    sizes = g.buckets()
+    per = sizes[0]
+    n = sizes[b]
+    from concurrent.futures import ThreadPoolExecutor
+
+    with ThreadPoolExecutor(max_workers=min(g.R, 8)) as pool:
+        return list(pool.map(lambda r: normal(g.seed, r, n, g.dtype, g.sigma, start=b * per), range(g.R)))
+
+
 @dataclass(frozen=True)
 class Sweep:
     name: str = "c5_size_sweep"
