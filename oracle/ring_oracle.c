@@ -5,8 +5,8 @@
  * What it follows.  The paper (HOCCL) moves collective data with copy engines and treats
  * AllGather and point-to-point send/recv as pure byte moves (Sec. 3.3 "Zero-SM Point-to-Point
  * Executor", Sec. 5 "Communication benchmarks"); it states that reductions are outside its scope
- * (Sec. 4 "Limitations").  The reduction is therefore the textbook ring reduce-scatter defined by
- * this build's problem statement: R ranks, R ring chunks, data travels r -> (r+1) mod R, rank r
+ * (Sec. 4 "Limitations").  The reduction is therefore the textbook ring reduce-scatter in a fixed
+ * order: R ranks, R ring chunks, data travels r -> (r+1) mod R, rank r
  * ends the reduce-scatter owning chunk r, the travelling partial is stored in the I/O dtype at every
  * hop, and each hop is ONE IEEE binary32 add followed by round-to-nearest-even to the I/O dtype.
  *

@@ -146,6 +146,8 @@ static long* param_slot(hoccl_comm* c, const char* key, long* lo, long* hi) {
               {"ce_small_bytes", &c->ce_small_bytes, 0, 1L << 40},
               {"ce_small_ctas", &c->ce_small_ctas, 1, 1024},
               {"p2p_strict", &c->p2p_strict, 0, 1},
+              {"model_gpus_per_node", &c->model_gpus_per_node, 0, kMaxRanks},
+              {"model_rdma_sub_bytes", &c->model_rdma_sub_bytes, 0, 1L << 40},
               {"host_pieces", &c->host_pieces, 1, 64}};
   for (auto& r : rows)
     if (std::strcmp(r.name, key) == 0) {
@@ -323,7 +325,9 @@ hoccl_result_t hoccl_alltoallv(const void* const* send, const size_t* sendcounts
   // the flows of the user-defined pattern as the origin traffic matrix C (bytes); one NVLink domain, no RDMA
   Topology topo;
   topo.G = R;
-  topo.gpus_per_node = R;
+  topo.gpus_per_node = (c->model_gpus_per_node > 0 && c->model_gpus_per_node < R) ? (int)c->model_gpus_per_node : R;
+  const bool modelled = topo.gpus_per_node < R;   // more than one modelled node: forwarding copies and "RDMA" legs exist
+  if (modelled && !c->use_graph) return HOCCL_ERR_UNSUPPORTED;
   std::vector<uint64_t> C((size_t)R * R);
   uint64_t total = 0;
   for (int u = 0; u < R; u++)
@@ -342,6 +346,10 @@ hoccl_result_t hoccl_alltoallv(const void* const* send, const size_t* sendcounts
     key.push_back((uint64_t)c->copy_ctas);
     key.push_back((uint64_t)c->piece_bytes);
     key.push_back((uint64_t)c->order_kernels);
+    key.push_back((uint64_t)topo.gpus_per_node);
+    key.push_back((uint64_t)c->model_rdma_sub_bytes);
+    key.push_back((uint64_t)(uintptr_t)c->staging);
+    key.push_back((uint64_t)c->staging_bytes);
     for (int r = 0; r < R; r++) {
       key.push_back((uint64_t)(uintptr_t)send[r]);
       key.push_back((uint64_t)(uintptr_t)recv[r]);
@@ -380,13 +388,33 @@ hoccl_result_t hoccl_alltoallv(const void* const* send, const size_t* sendcounts
   c->stats = hoccl_stats_t{};
   if (total == 0) return HOCCL_OK;
   Schedule S;
-  if (!build_schedule(topo, C, (uint64_t)std::max<long>(c->piece_bytes, 65536), &S)) return HOCCL_ERR_INTERNAL;
+  const uint64_t chunk_bytes = (uint64_t)std::max<long>(c->piece_bytes, 65536);
+  if (!build_schedule(topo, C, chunk_bytes, &S)) return HOCCL_ERR_INTERNAL;
   CU_TRY(c, cudaSetDevice(c->device));
   cudaStream_t user = (cudaStream_t)stream;
   if (c->use_graph) {
     GraphEntry entry;
     entry.key = key;
-    hoccl_result_t grc = build_pattern_graph(c, S, send, sdispls, recv, rdispls, e, &entry);
+    hoccl_result_t grc;
+    if (modelled) {
+      // staging for the flows between modelled nodes: what has left the sender's side and what has arrived at the receiver's
+      std::vector<uint64_t> off((size_t)R * R, 0);
+      uint64_t need = 0;
+      for (int u = 0; u < R; u++)
+        for (int v = 0; v < R; v++)
+          if (u != v && !topo.same_node(u, v) && C[(size_t)u * R + v]) {
+            off[(size_t)u * R + v] = need;
+            need += (C[(size_t)u * R + v] + 255) / 256 * 256;
+          }
+      if (need && (!c->staging || c->staging_bytes < 2 * need)) return HOCCL_ERR_SCRATCH;
+      for (int r = 0; r < R && need; r++)
+        if (ranges_overlap((const char*)c->staging, 2 * need, (const char*)send[r], 1) || ranges_overlap((const char*)c->staging, 2 * need, (const char*)recv[r], 1))
+          return HOCCL_ERR_INVALID_ARG;
+      grc = build_pattern_graph_modelled(c, S, send, sdispls, recv, rdispls, e, (char*)c->staging, (char*)c->staging + need, off,
+                                         (size_t)chunk_bytes, (size_t)c->model_rdma_sub_bytes, &entry);
+    } else {
+      grc = build_pattern_graph(c, S, send, sdispls, recv, rdispls, e, &entry);
+    }
     if (grc != HOCCL_OK) return grc;
     GraphEntry* en = cache_put(c, std::move(entry));
     en->last_use = ++c->use_counter;

@@ -90,7 +90,7 @@ struct hoccl_comm {
   hoccl_path_t path = HOCCL_PATH_CE;
   long sum_ctas = 8, copy_ctas = 8, piece_bytes = 4 << 20, max_pieces = 8, lanes = 4, use_graph = 1, profile = 0, p2p_split = 1, ce_sub_bytes = 0,
        handshake = 0, watchdog_ms = 10000, onepass = 0, forward = 0, fused = 0, host_pieces = 8, ag_direct = 2, order_kernels = 1, rs_direct = 2,
-       ce_small_bytes = 8 << 20, ce_small_ctas = 148, p2p_strict = 0;
+       ce_small_bytes = 8 << 20, ce_small_ctas = 148, p2p_strict = 0, model_gpus_per_node = 0, model_rdma_sub_bytes = 0;
   bool piece_bytes_set = false;  // the caller chose a piece size: no automatic choice
   hoccl::Proxy* proxy = nullptr;
   cudaStream_t lane[hoccl::kMaxLanes] = {};
@@ -197,6 +197,10 @@ void destroy_entry(GraphEntry* e);
 GraphEntry* cache_put(hoccl_comm* c, GraphEntry&& entry);
 hoccl_result_t build_pattern_graph(hoccl_comm* c, const Schedule& S, const void* const* send, const size_t* sdispls, void* const* recv,
                                    const size_t* rdispls, size_t e, GraphEntry* entry);
+hoccl_result_t build_pattern_graph_modelled(hoccl_comm* c, const Schedule& S, const void* const* send, const size_t* sdispls,
+                                            void* const* recv, const size_t* rdispls, size_t e, char* out_stage, char* in_stage,
+                                            const std::vector<uint64_t>& flow_stage_off, size_t chunk_bytes, size_t rdma_sub,
+                                            GraphEntry* entry);
 hoccl_result_t ring_barrier_selftest(hoccl_comm* c, void* dst, const void* src, size_t bytes, cudaStream_t stream);
 // p2p.cu
 hoccl_result_t p2p_post(hoccl_comm* c, bool is_send, void* buf, size_t count, int dtype, int src, int dst, cudaStream_t stream);

@@ -1,6 +1,8 @@
 // Graph side of libhoccl: a resolved plan (or the schedule of a user-defined pattern) becomes an explicit CUDA graph:
 // memcpy nodes for moves on the copy route, kernel nodes for sums and SM copies, empty nodes as joins.  Also the graph
 // cache and the host copies of the pipelined host all-reduce.
+#include <tuple>
+
 #include "comm.h"
 
 namespace hoccl {
@@ -420,6 +422,185 @@ hoccl_result_t build_pattern_graph(hoccl_comm* c, const Schedule& S, const void*
   hoccl_result_t rc = HOCCL_OK;
   if (err == cudaSuccess) err = cudaGraphInstantiate(&entry->exec, g, 0);
   if (err != cudaSuccess) rc = cuda_fail(c, err, "pattern graph");
+  cudaGraphDestroy(g);
+  entry->n_pieces = (long)S.stages.size();
+  if (rc != HOCCL_OK) destroy_entry(entry);
+  return rc;
+}
+
+// The same for a MODELLED topology with more than one node (paper Sec. 3.4, Eq. 2-4 and Algorithm 1 run as real copies on one
+// device).  A logical flow u -> v between two nodes is carried, portion by portion as Algorithm 1 stages it, by three copies
+// per chunk: the sender-side forwarding copy f' from u's send buffer into a staging slot at u's symmetric peer, the "RDMA"
+// leg f from that slot into a staging slot at v's symmetric peer (optionally cut into serial sub-copies of `rdma_sub` bytes, a
+// crude stand-in for the slower domain), and the receiver-side forwarding copy f'' from there into v's receive buffer.
+// Staging: `out_stage` + the flow's offset holds what left u, `in_stage` + the same offset what arrived at v's side.
+// Copy route: chunk-level DAG; a source GPU's native and forwarding chunks form one serial queue in the scheduler's
+// interleaved order (its DMA engine), the RDMA legs of one source form a second serial queue (its NIC), and chunk k of f
+// waits for chunk k of f', chunk k of f'' for chunk k of f.  SM path: per stage three batched phases (all f' and native
+// chunks, all f, all f'') in one chain of launches.  Stages run one after the other.
+hoccl_result_t build_pattern_graph_modelled(hoccl_comm* c, const Schedule& S, const void* const* send, const size_t* sdispls,
+                                            void* const* recv, const size_t* rdispls, size_t e, char* out_stage, char* in_stage,
+                                            const std::vector<uint64_t>& flow_stage_off, size_t chunk_bytes, size_t rdma_sub,
+                                            GraphEntry* entry) {
+  const int R = c->R;
+  const Topology& topo = S.topo;
+  cudaGraph_t g = nullptr;
+  CU_TRY(c, cudaGraphCreate(&g, 0));
+  cudaError_t err = cudaSuccess;
+  auto order_kernel = [&](cudaGraphNode_t* out, const cudaGraphNode_t* deps, size_t nd) {
+    cudaKernelNodeParams kp = {};
+    kp.func = const_cast<void*>(graph_root_kernel_entry());
+    kp.gridDim = dim3(1);
+    kp.blockDim = dim3(32);
+    kp.kernelParams = nullptr;
+    cudaError_t e2 = cudaGraphAddKernelNode(out, g, deps, nd, &kp);
+    if (e2 == cudaSuccess) entry->n_order_launches++;
+    return e2;
+  };
+  cudaGraphNode_t stage_dep = nullptr;
+  const bool ce = c->path == HOCCL_PATH_CE;
+  if (ce && c->order_kernels) err = order_kernel(&stage_dep, nullptr, 0);
+  // where the bytes [off, off + n) of the logical flow (u, v) sit at each of the four places they pass through
+  auto place = [&](int cls_src, int u, int v, uint64_t off) -> char* {
+    // cls_src: 0 = u's send buffer, 1 = staging at u's peer, 2 = staging at v's peer, 3 = v's receive buffer
+    switch (cls_src) {
+      case 0: return (char*)send[u] + sdispls[(size_t)u * R + v] * e + off;
+      case 1: return out_stage + flow_stage_off[(size_t)u * R + v] + off;
+      case 2: return in_stage + flow_stage_off[(size_t)u * R + v] + off;
+      default: return (char*)recv[v] + rdispls[(size_t)v * R + u] * e + off;
+    }
+  };
+  struct Op {
+    const char* src;
+    char* dst;
+    uint64_t bytes;
+  };
+  for (size_t si = 0; si < S.stages.size() && err == cudaSuccess; si++) {
+    const Stage& st = S.stages[si];
+    auto op_of = [&](const StageFlow& f, uint64_t off, uint64_t n) -> Op {
+      const int u = f.origin_src, v = f.origin_dst;
+      const uint64_t o = f.origin_offset + off;
+      const bool has_pu = topo.peer_of(u) != u, has_pv = topo.peer_of(v) != v;
+      switch (f.cls) {
+        case FLOW_NATIVE: return Op{place(0, u, v, o), place(3, u, v, o), n};
+        case FLOW_FWD_SEND: return Op{place(0, u, v, o), place(1, u, v, o), n};
+        case FLOW_FWD_RECV: return Op{place(2, u, v, o), place(3, u, v, o), n};
+        default: return Op{place(has_pu ? 1 : 0, u, v, o), place(has_pv ? 2 : 3, u, v, o), n};   // the RDMA leg
+      }
+    };
+    auto key_of = [&](const StageFlow& f, uint64_t off) { return std::make_tuple(f.origin_src, f.origin_dst, f.origin_offset + off); };
+    std::vector<cudaGraphNode_t> tails;
+    if (ce) {
+      std::map<std::tuple<int, int, uint64_t>, cudaGraphNode_t> sent, arrived;   // chunk -> its f' node, its f node
+      auto add_copy = [&](const Op& op, std::vector<cudaGraphNode_t> deps, size_t sub, cudaGraphNode_t* last) {
+        const size_t step = sub ? sub : op.bytes;
+        for (uint64_t o = 0; o < op.bytes && err == cudaSuccess; o += step) {
+          const uint64_t n = std::min<uint64_t>(step, op.bytes - o);
+          cudaGraphNode_t nd;
+          err = cudaGraphAddMemcpyNode1D(&nd, g, deps.data(), deps.size(), op.dst + o, op.src + o, n, cudaMemcpyDeviceToDevice);
+          if (err != cudaSuccess) return;
+          deps.assign(1, nd);
+          *last = nd;
+          entry->n_moves++;
+        }
+      };
+      // pass 1: the DMA queues' native and sender-side chunks; pass 2: the NIC queues; pass 3: the receiver-side chunks, in
+      // their queues' order behind whatever that queue issued in pass 1
+      std::vector<cudaGraphNode_t> qtail(R, nullptr);
+      for (int pass = 0; pass < 3 && err == cudaSuccess; pass++) {
+        if (pass == 1) {
+          for (int u = 0; u < R && err == cudaSuccess; u++) {
+            cudaGraphNode_t nic = nullptr;
+            for (const StageFlow& f : st.flows) {
+              if (f.cls != FLOW_RDMA || f.u != u) continue;
+              for (uint64_t off = 0; off < f.bytes && err == cudaSuccess; off += chunk_bytes) {
+                const uint64_t n = std::min<uint64_t>(chunk_bytes, f.bytes - off);
+                std::vector<cudaGraphNode_t> deps;
+                if (nic) deps.push_back(nic);
+                auto it = sent.find(key_of(f, off));
+                if (it != sent.end()) deps.push_back(it->second);
+                if (deps.empty() && stage_dep) deps.push_back(stage_dep);
+                cudaGraphNode_t last = nullptr;
+                add_copy(op_of(f, off, n), deps, rdma_sub, &last);
+                if (err != cudaSuccess) break;
+                nic = last;
+                arrived[key_of(f, off)] = last;
+              }
+            }
+            if (nic) tails.push_back(nic);
+          }
+          continue;
+        }
+        for (int q = 0; q < R && err == cudaSuccess; q++) {
+          for (const ChunkItem& it : st.queues[q]) {
+            const StageFlow& f = st.flows[it.flow];
+            const bool recv_side = f.cls == FLOW_FWD_RECV;
+            if ((pass == 0) == recv_side) continue;
+            std::vector<cudaGraphNode_t> deps;
+            if (qtail[q]) deps.push_back(qtail[q]);
+            if (recv_side) {
+              auto a = arrived.find(key_of(f, it.offset));
+              if (a != arrived.end()) deps.push_back(a->second);
+            }
+            if (deps.empty() && stage_dep) deps.push_back(stage_dep);
+            cudaGraphNode_t last = nullptr;
+            add_copy(op_of(f, it.offset, it.bytes), deps, 0, &last);
+            if (err != cudaSuccess) break;
+            qtail[q] = last;
+            if (f.cls == FLOW_FWD_SEND) sent[key_of(f, it.offset)] = last;
+          }
+        }
+      }
+      for (int q = 0; q < R; q++)
+        if (qtail[q]) tails.push_back(qtail[q]);
+    } else {
+      cudaGraphNode_t prev = stage_dep;
+      auto run_phase = [&](const std::vector<Op>& ops) {
+        for (size_t first = 0; first < ops.size() && err == cudaSuccess; first += kMaxSegs) {
+          CopyBatch b;
+          b.nseg = (int)std::min<size_t>(kMaxSegs, ops.size() - first);
+          b.pad = 0;
+          for (int i = 0; i < b.nseg; i++) b.seg[i] = CopySeg{ops[first + i].src, ops[first + i].dst, (unsigned long long)ops[first + i].bytes};
+          prepare_copy_batch(&b, (int)c->copy_ctas);
+          void* args[] = {&b};
+          cudaKernelNodeParams kp = {};
+          int threads = 0;
+          kp.func = const_cast<void*>(copy_kernel_entry((int)c->copy_ctas, &threads));
+          kp.gridDim = dim3((unsigned)c->copy_ctas);
+          kp.blockDim = dim3((unsigned)threads);
+          kp.kernelParams = args;
+          cudaGraphNode_t n;
+          err = cudaGraphAddKernelNode(&n, g, prev ? &prev : nullptr, prev ? 1 : 0, &kp);
+          if (err == cudaSuccess) {
+            prev = n;
+            entry->n_move_launches++;
+            entry->n_moves += b.nseg;
+          }
+        }
+      };
+      std::vector<Op> a, b, d;
+      for (const StageFlow& f : st.flows) {
+        if (!f.bytes) continue;
+        (f.cls == FLOW_RDMA ? b : f.cls == FLOW_FWD_RECV ? d : a).push_back(op_of(f, 0, f.bytes));
+      }
+      run_phase(a);
+      run_phase(b);
+      run_phase(d);
+      if (prev && prev != stage_dep) tails.push_back(prev);
+    }
+    if (err != cudaSuccess) break;
+    if (tails.size() == 1) {
+      stage_dep = tails[0];
+    } else if (tails.size() > 1) {
+      cudaGraphNode_t join;
+      if (ce && c->order_kernels) err = order_kernel(&join, tails.data(), tails.size());
+      else err = cudaGraphAddEmptyNode(&join, g, tails.data(), tails.size());
+      if (err == cudaSuccess) stage_dep = join;
+    }
+  }
+  hoccl_result_t rc = HOCCL_OK;
+  if (err == cudaSuccess) err = cudaGraphInstantiate(&entry->exec, g, 0);
+  if (err != cudaSuccess) rc = cuda_fail(c, err, "modelled pattern graph");
   cudaGraphDestroy(g);
   entry->n_pieces = (long)S.stages.size();
   if (rc != HOCCL_OK) destroy_entry(entry);

@@ -5,7 +5,7 @@ pipeline / gradient-stream workloads (third and fourth), through the C ABI.
     python -m paper_2609_34334_b200.sweep pipeline [--microbatches 16]
     python -m paper_2609_34334_b200.sweep gradients [--buckets 32] [--budgets 1,2,4,8,16,32,64]
     python -m paper_2609_34334_b200.sweep launch-cost
-    python -m paper_2609_34334_b200.sweep alltoallv [--mib 4,64,256]
+    python -m paper_2609_34334_b200.sweep alltoallv [--mib 4,64,256] [--model 4,2]
 
 Sizes are per-rank buffer bytes S in the nccl-tests convention (all-reduce: send = recv = S; reduce-scatter:
 send = S; all-gather: recv = S; all-to-all: send = recv = S; send/recv: S), like the sweeps the paper reports (Sec. 5 "Communication
@@ -423,11 +423,26 @@ def alltoallv(args):
             rdispls = np.concatenate([np.zeros((R, 1), dtype=np.int64), np.cumsum(recv_counts, axis=1)[:, :-1]], axis=1)
             recv = [torch.zeros(int(recv_counts[v].sum()) + 8, dtype=torch.bfloat16, device="cuda") for v in range(R)]
             moved = int(counts.sum()) * e
-            configs = [("CE", hb.PATH_CE, 8), ("SM8", hb.PATH_SM, 8), ("SMall", hb.PATH_SM, 148)]
-            for name, path, ctas in configs:
+            configs = [("CE", hb.PATH_CE, 8, 0, 0), ("SM8", hb.PATH_SM, 8, 0, 0), ("SMall", hb.PATH_SM, 148, 0, 0)]
+            # the same pattern over a modelled topology of two (or four) nodes: forwarding copies and "RDMA" legs as real copies
+            for gpn in [int(x) for x in args.model.split(",") if x]:
+                configs += [("CE_model%d" % gpn, hb.PATH_CE, 8, gpn, 0), ("CE_model%d_sub256K" % gpn, hb.PATH_CE, 8, gpn, 256 << 10),
+                            ("SMall_model%d" % gpn, hb.PATH_SM, 148, gpn, 0)]
+            stage_buf = None
+            for name, path, ctas, gpn, sub in configs:
                 comm = hb.Comm(R, 0)
                 comm.set_path(path)
                 comm.set_param("copy_ctas", ctas)
+                tau = None
+                if gpn:
+                    comm.set_param("model_gpus_per_node", gpn)
+                    comm.set_param("model_rdma_sub_bytes", sub)
+                    if stage_buf is None:
+                        stage_buf = torch.empty(2 * moved + 2 * R * R * 256 + 256, dtype=torch.uint8, device="cuda")
+                    comm.set_staging(stage_buf.data_ptr() + (-stage_buf.data_ptr()) % 256, stage_buf.numel() - 256)
+                    sch = hb.Schedule(counts.astype(np.uint64) * e, gpn, chunk_bytes=4 << 20)
+                    tau = {"stages_host": len(sch.stages), "total_tau_us_at_400_and_50_GBps": sch.total_tau * 1e6,
+                           "lower_bound_us": sch.lower_bound * 1e6}
 
                 def call():
                     comm.alltoallv(send, counts.reshape(-1), sdispls.reshape(-1), recv, rdispls.reshape(-1), dtype, stream)
@@ -450,6 +465,10 @@ def alltoallv(args):
                        "hbm_frac_of_8TBps": 2.0 * moved / t / NOMINAL_HBM, "stages": int(st["n_pieces"]), "moves": int(st["n_moves"]),
                        "launches": int(st["n_move_launches"]), "host_us_per_call": st["host_launch_us"], "delivered_bit_exact": ok,
                        "largest_flow_MiB": float(counts.max() * e / 2 ** 20), "smallest_flow_MiB": float(counts.min() * e / 2 ** 20)}
+                if tau:
+                    row.update(tau)
+                    row["model_gpus_per_node"] = gpn
+                    row["model_rdma_sub_bytes"] = sub
                 if pattern == "uniform":
                     r2 = [torch.zeros(n, dtype=torch.bfloat16, device="cuda") for _ in range(R)]
                     for _ in range(3):
@@ -489,6 +508,7 @@ def main():
     sub.add_parser("launch-cost")
     a2 = sub.add_parser("alltoallv")
     a2.add_argument("--mib", default="4,64,256", help="comma list of MiB sent per rank")
+    a2.add_argument("--model", default="", help="comma list of modelled GPUs per node (e.g. 4,2): also run the pattern over that topology")
     args = ap.parse_args()
     if not torch.cuda.is_available():
         sys.stderr.write("sweep: no CUDA device\n")
