@@ -196,6 +196,12 @@ hoccl_result_t hoccl_comm_set_path(hoccl_comm_t comm, hoccl_path_t path);
  *                4 KiB 34 -> 10 us, 1 MiB 48 -> 25 us, 4 MiB 88 -> 54 us, 8 MiB 107 -> 97 us, equal from 16 MiB on; R = 4 fp32
  *                all-reduce of 4 MiB 37 -> 33 us.  Default 8 MiB; 0 = driver copies at every size.  "HOCCL_PATH_CE" therefore
  *                means: the copy route above this size.  Not applied to hoccl_host_allreduce, send/recv or hoccl_alltoallv.
+ *  "ce_overlap"  HOCCL_PATH_CE, direct reduce-scatter: the ring chunks are cut into this many pieces and every piece's three
+ *                parts (the reduce-scatter's moves, the chain sum, the all-gather's moves) become graphs of their own that
+ *                run on three internal streams, ordered by events, so that one piece's driver copies run beside another
+ *                piece's sum (inside ONE graph, and on plain streams, they were never seen to overlap).  Sums still run one
+ *                at a time.  Costs ~8 us of host time per piece and call.  -1 (default) = automatic: 4 pieces from 4 MiB per
+ *                ring chunk, 8 from 16 MiB, off below; 0 = off; 2..64 = that many pieces.  Ignored when "piece_bytes" is set.
  *  "ce_small_ctas" CTAs of those launches, 1..1024 (default 148: like the driver's own copies they may use the whole GPU,
  *                for tens of microseconds)
  *  "order_kernels" 1 (default) = on the copy routes the graph executor puts an empty one-warp kernel in front of a graph's

@@ -44,6 +44,7 @@ struct Seg {
 struct RGroup {
   int kind;
   int piece;
+  int phase = 0;   // plan phase of the group (reduce-scatter, all-gather, own chunk, all-to-all stage)
   std::vector<Seg> segs;
   std::vector<int> deps;
   int chain_dep;
@@ -76,6 +77,9 @@ struct GraphEntry {
   // pipelined host all-reduce: one graph per piece, and the host copies in front of and behind each of them
   std::vector<cudaGraphExec_t> piece_exec;
   std::vector<std::vector<HostCopy>> h2d, d2h;   // [piece]
+  // "ce_overlap" setting: per piece three graphs (the reduce-scatter's moves, the sum, the all-gather's moves) that run on three
+  // internal streams, so that one piece's driver copies overlap another piece's sum (inside ONE graph they never did)
+  std::vector<cudaGraphExec_t> part_exec;   // [piece * 3 + part], null where a part is empty
   // "fused" setting: the whole plan as one cooperative kernel instead of a graph (exec stays null)
   std::vector<char> ring_args;  // a RingArgsSmall or RingArgsLarge, by value
   bool ring_large = false;
@@ -90,7 +94,7 @@ struct hoccl_comm {
   hoccl_path_t path = HOCCL_PATH_CE;
   long sum_ctas = 8, copy_ctas = 8, piece_bytes = 4 << 20, max_pieces = 8, lanes = 4, use_graph = 1, profile = 0, p2p_split = 1, ce_sub_bytes = 0,
        handshake = 0, watchdog_ms = 10000, onepass = 0, forward = 0, fused = 0, host_pieces = 8, ag_direct = 2, order_kernels = 1, rs_direct = 2,
-       ce_small_bytes = 8 << 20, ce_small_ctas = 148, p2p_strict = 0, model_gpus_per_node = 0, model_rdma_sub_bytes = 0;
+       ce_small_bytes = 8 << 20, ce_small_ctas = 148, p2p_strict = 0, ce_overlap = -1, model_gpus_per_node = 0, model_rdma_sub_bytes = 0;
   bool piece_bytes_set = false;  // the caller chose a piece size: no automatic choice
   hoccl::Proxy* proxy = nullptr;
   cudaStream_t lane[hoccl::kMaxLanes] = {};
@@ -181,8 +185,11 @@ void fill_chain_batch(const RGroup& g, size_t first, size_t n, int dtype, size_t
 // copy batches are used then.  bytes_out[i] = HBM bytes of batch i (reads + writes), moves_out[i] = moves it carries.
 bool build_fan_batches(const RGroup& g, std::vector<FanBatch>* out, std::vector<double>* bytes_out, std::vector<long>* moves_out);
 // graph.cu
+// part < 0: every group (of `only_piece`, if that is >= 0); part 0 / 1 / 2: only the reduce-scatter's MOVE groups / the SUM and
+// CHAIN groups / the remaining MOVE groups; dependencies on groups outside the part are left to the caller (events).
+// *out_exec stays null when nothing falls into the selection.
 hoccl_result_t build_graph(hoccl_comm* c, const Plan& P, const std::vector<RGroup>& groups, GraphEntry* entry, int only_piece,
-                           cudaGraphExec_t* out_exec);
+                           cudaGraphExec_t* out_exec, int part = -1);
 void add_host_copies(const Plan& P, int p, char* dev, char* host, std::vector<HostCopy>* out);
 cudaError_t enqueue_host_copy(const HostCopy& hc, bool to_device, cudaStream_t s);
 // ring_host.cu

@@ -99,6 +99,7 @@ void resolve(hoccl_comm* c, const Plan& P, const Call& call, std::vector<RGroup>
     RGroup& rg = (*out)[g];
     rg.kind = pg.kind;
     rg.piece = pg.piece;
+    rg.phase = pg.phase;
     rg.deps = pg.deps;
     rg.chain_dep = pg.chain_dep;
     for (int i = 0; i < pg.num_ops; i++) {
@@ -391,6 +392,7 @@ std::vector<uint64_t> make_key(hoccl_comm* c, const Call& call) {
   k.push_back((uint64_t)c->ag_direct);
   k.push_back((uint64_t)c->order_kernels);
   k.push_back((uint64_t)c->rs_direct);
+  k.push_back((uint64_t)c->ce_overlap);
   k.push_back((uint64_t)(c->fused && c->path == HOCCL_PATH_SM && !c->handshake));
   k.push_back((uint64_t)(uintptr_t)c->scratch);
   k.push_back((uint64_t)c->scratch_bytes);
@@ -475,7 +477,44 @@ static hoccl_result_t launch_entry(hoccl_comm* c, GraphEntry* hit, cudaStream_t 
     c->stats.host_launch_us = now_us() - t0;
     return HOCCL_OK;
   }
-  if (!hit->piece_exec.empty()) {
+  if (!hit->part_exec.empty()) {
+    // Copy route with overlap: the reduce-scatter's moves of every piece on one internal stream, the sums on the sum stream
+    // (one at a time: the SM budget stays global), the all-gather's moves on a second internal stream; events carry the
+    // per-piece dependencies between them.
+    cudaStream_t rs = c->lane[0], sm = c->sum_stream, ag = c->lane[1];
+    c->ev_next = 0;
+    cudaEvent_t fork = next_event(c);
+    if (!fork) return cuda_fail(c, cudaErrorMemoryAllocation, "event pool");
+    CU_TRY(c, cudaEventRecord(fork, user));
+    CU_TRY(c, cudaStreamWaitEvent(rs, fork, 0));
+    CU_TRY(c, cudaStreamWaitEvent(sm, fork, 0));
+    CU_TRY(c, cudaStreamWaitEvent(ag, fork, 0));
+    const size_t np = hit->part_exec.size() / 3;
+    for (size_t p = 0; p < np; p++) {
+      cudaGraphExec_t g_rs = hit->part_exec[3 * p], g_sum = hit->part_exec[3 * p + 1], g_ag = hit->part_exec[3 * p + 2];
+      if (g_rs) {
+        CU_TRY(c, cudaGraphLaunch(g_rs, rs));
+        cudaEvent_t moved = next_event(c);
+        if (!moved) return cuda_fail(c, cudaErrorMemoryAllocation, "event pool");
+        CU_TRY(c, cudaEventRecord(moved, rs));
+        CU_TRY(c, cudaStreamWaitEvent(sm, moved, 0));
+      }
+      if (g_sum) CU_TRY(c, cudaGraphLaunch(g_sum, sm));
+      if (g_ag) {
+        cudaEvent_t summed = next_event(c);
+        if (!summed) return cuda_fail(c, cudaErrorMemoryAllocation, "event pool");
+        CU_TRY(c, cudaEventRecord(summed, sm));
+        CU_TRY(c, cudaStreamWaitEvent(ag, summed, 0));
+        CU_TRY(c, cudaGraphLaunch(g_ag, ag));
+      }
+    }
+    for (cudaStream_t s : {rs, sm, ag}) {
+      cudaEvent_t done = next_event(c);
+      if (!done) return cuda_fail(c, cudaErrorMemoryAllocation, "event pool");
+      CU_TRY(c, cudaEventRecord(done, s));
+      CU_TRY(c, cudaStreamWaitEvent(user, done, 0));
+    }
+  } else if (!hit->piece_exec.empty()) {
     // Pipelined host all-reduce: the inbound copies run on one internal stream, the outbound copies on another, and the
     // caller's stream runs the ring piece by piece as each piece arrives; PCIe carries both directions at once.
     cudaStream_t in = c->lane[0], out = c->lane[1];
@@ -626,7 +665,28 @@ hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
   // 148-CTA sums, 3-14 % on the whole-GPU SM path).
   size_t piece_bytes = (size_t)c->piece_bytes;
   int max_pieces = (int)c->max_pieces;
-  if (call->h_send) {   // pipelined host all-reduce: host_pieces pieces per chunk, whatever the chunk size
+  const bool reduction = call->kind == PLAN_ALLREDUCE || call->kind == PLAN_REDUCE_SCATTER;
+  const size_t ring_chunk = (call->kind == PLAN_ALLREDUCE ? (call->count + c->R - 1) / c->R : call->count) * dtype_size(call->dtype);
+  // Copy route with overlap ("ce_overlap"): the direct schedule cut into pieces whose three parts run on three internal
+  // streams (see launch_entry).  Automatic (-1): 4 pieces from 4 MiB per ring chunk, 8 from 16 MiB; below that the ~30 us of
+  // host time per call and the extra copies cost more than the overlap gives (measured on B200, R = 8, bf16, 8-CTA sums:
+  // 40 MiB per rank 0.469 -> 0.426 ms with 4 pieces, 256 MiB 2.97 -> 2.48 ms with 8; 25 MiB 0.290 -> 0.281 with 2).
+  long overlap_pieces = c->ce_overlap;
+  if (overlap_pieces < 0) overlap_pieces = ring_chunk >= ((size_t)16 << 20) ? 8 : ring_chunk >= ((size_t)4 << 20) ? 4 : 0;
+  const bool overlap = overlap_pieces > 1 && c->path == HOCCL_PATH_CE && opt.executor == EXEC_GRAPH && !call->h_send &&
+                       (plan_kind & PLAN_FLAG_RS_DIRECT) && c->R > 1 && !c->piece_bytes_set;
+  if (overlap) {
+    max_pieces = (int)overlap_pieces;
+    piece_bytes = std::max<size_t>((size_t)64 << 10, ((ring_chunk + max_pieces - 1) / max_pieces + 1023) / 1024 * 1024);
+  } else if (!c->piece_bytes_set && c->path == HOCCL_PATH_SM && opt.executor == EXEC_GRAPH && !call->h_send && reduction &&
+             (plan_kind & PLAN_FLAG_RS_DIRECT) && c->sum_ctas < 64 && c->copy_ctas < 128 && ring_chunk >= ((size_t)1 << 20)) {
+    // SM path, direct schedule under CTA budgets: pieces of an eighth of a ring chunk, between 512 KiB and 2 MiB, issued as a
+    // software pipeline (see build_graph): a piece's copies run beside another piece's chain sum (measured, 8-CTA sums and
+    // 40 copy CTAs: 40 MiB per rank 0.47 ms with 2 pieces, 0.42 with 4, 0.39 with 8, 0.58 with 16; 256 MiB 2.99 / 2.72 / 2.57 /
+    // 2.50 ms with 2 / 4 / 8 / 16 pieces)
+    piece_bytes = std::min<size_t>((size_t)2 << 20, std::max<size_t>((size_t)512 << 10, (ring_chunk / 8 + 1023) / 1024 * 1024));
+    max_pieces = 64;
+  } else if (call->h_send) {   // pipelined host all-reduce: host_pieces pieces per chunk, whatever the chunk size
     const size_t q = (call->count + c->R - 1) / c->R;
     const size_t chunk = q * dtype_size(call->dtype);
     max_pieces = (int)c->host_pieces;
@@ -634,7 +694,7 @@ hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
   } else if (fused) {   // one kernel walks the steps in order; whole chunks measured faster than pieces (fewer barriers and tails)
     piece_bytes = (size_t)1 << 60;
     max_pieces = 1;
-  } else if (!c->piece_bytes_set && (call->kind == PLAN_ALLREDUCE || call->kind == PLAN_REDUCE_SCATTER) &&
+  } else if (!c->piece_bytes_set && reduction &&
              (c->path == HOCCL_PATH_CE || (c->path == HOCCL_PATH_SM && std::min(c->sum_ctas, c->copy_ctas) >= 128))) {
     // "whole" stops at 256 MiB: several concurrent driver copies of 512 MiB each ran at half speed (R = 2, 1 GiB per rank)
     piece_bytes = (size_t)256 << 20;
@@ -689,6 +749,14 @@ hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
           destroy_entry(&entry);   // the pieces built so far, and any profile events
           return rc;
         }
+      }
+    } else if (overlap && P.pieces > 1) {   // with one piece there is nothing to overlap: one graph
+      entry.part_exec.assign((size_t)P.pieces * 3, nullptr);
+      for (int p = 0; p < P.pieces && rc == HOCCL_OK; p++)
+        for (int part = 0; part < 3 && rc == HOCCL_OK; part++) rc = build_graph(c, P, groups, &entry, p, &entry.part_exec[(size_t)p * 3 + part], part);
+      if (rc != HOCCL_OK) {
+        destroy_entry(&entry);
+        return rc;
       }
     } else {
       rc = fused ? build_ring(c, P, groups, &entry) : HOCCL_ERR_UNSUPPORTED;

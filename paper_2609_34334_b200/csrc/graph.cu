@@ -12,6 +12,9 @@ void destroy_entry(GraphEntry* e) {
   for (cudaGraphExec_t pe : e->piece_exec)
     if (pe) cudaGraphExecDestroy(pe);
   e->piece_exec.clear();
+  for (cudaGraphExec_t pe : e->part_exec)
+    if (pe) cudaGraphExecDestroy(pe);
+  e->part_exec.clear();
   for (auto& p : e->prof_events) {
     cudaEventDestroy(p.first);
     cudaEventDestroy(p.second);
@@ -54,7 +57,23 @@ cudaError_t enqueue_host_copy(const HostCopy& hc, bool to_device, cudaStream_t s
 
 // only_piece >= 0 builds the graph of that piece alone (dependencies never cross pieces) and stores it in *out_exec.
 hoccl_result_t build_graph(hoccl_comm* c, const Plan& P, const std::vector<RGroup>& groups, GraphEntry* entry, int only_piece,
-                           cudaGraphExec_t* out_exec) {
+                           cudaGraphExec_t* out_exec, int part) {
+  // which groups this graph holds
+  auto included = [&](size_t gi) {
+    const RGroup& rg = groups[gi];
+    if (only_piece >= 0 && rg.piece != only_piece) return false;
+    if (part < 0) return true;
+    const int cls = rg.kind != OP_MOVE ? 1 : (rg.phase == PHASE_RS ? 0 : 2);
+    return cls == part;
+  };
+  {
+    bool any = false;
+    for (size_t gi = 0; gi < groups.size(); gi++) any = any || (included(gi) && !groups[gi].segs.empty());
+    if (!any && part >= 0) {
+      *out_exec = nullptr;
+      return HOCCL_OK;
+    }
+  }
   cudaGraph_t g = nullptr;
   CU_TRY(c, cudaGraphCreate(&g, 0));
   std::vector<std::vector<cudaGraphNode_t>> tail(groups.size());   // the node(s) a consumer of the group waits for
@@ -65,11 +84,16 @@ hoccl_result_t build_graph(hoccl_comm* c, const Plan& P, const std::vector<RGrou
   // their common predecessor takes that wait once (an empty graph node does not: it changes nothing).
   cudaGraphNode_t root = nullptr;
   bool many_root_copies = false;
+  auto inner_deps = [&](size_t gi) {   // dependencies of group gi on groups of this graph
+    size_t n = 0;
+    for (int d : groups[gi].deps) n += included((size_t)d) ? 1 : 0;
+    if (groups[gi].chain_dep >= 0 && included((size_t)groups[gi].chain_dep)) n++;
+    return n;
+  };
   if (c->order_kernels && (c->path == HOCCL_PATH_CE || c->path == HOCCL_PATH_CE_HOST)) {
     size_t n_root = 0;
     for (size_t gi = 0; gi < groups.size(); gi++)
-      if ((only_piece < 0 || groups[gi].piece == only_piece) && groups[gi].kind == OP_MOVE && groups[gi].deps.empty() && groups[gi].chain_dep < 0)
-        n_root += groups[gi].segs.size();
+      if (included(gi) && groups[gi].kind == OP_MOVE && inner_deps(gi) == 0) n_root += groups[gi].segs.size();
     many_root_copies = n_root >= 2;
   }
   // The same holds behind a group of copies: copy nodes (or the end of the graph) that wait for several copy nodes start
@@ -80,7 +104,7 @@ hoccl_result_t build_graph(hoccl_comm* c, const Plan& P, const std::vector<RGrou
   if (c->order_kernels && (c->path == HOCCL_PATH_CE || c->path == HOCCL_PATH_CE_HOST)) {
     std::vector<char> move_user(groups.size(), 0), any_user(groups.size(), 0);
     for (size_t gi = 0; gi < groups.size(); gi++) {
-      if (only_piece >= 0 && groups[gi].piece != only_piece) continue;
+      if (!included(gi)) continue;
       for (int d : groups[gi].deps) {
         any_user[d] = 1;
         if (groups[gi].kind == OP_MOVE) move_user[d] = 1;
@@ -92,10 +116,27 @@ hoccl_result_t build_graph(hoccl_comm* c, const Plan& P, const std::vector<RGrou
   auto fail = [&](cudaError_t e, const char* what) {
     rc = cuda_fail(c, e, what);
   };
-  for (size_t gi = 0; gi < groups.size() && rc == HOCCL_OK; gi++) {
-    if (only_piece >= 0 && groups[gi].piece != only_piece) continue;
+  // Issue order.  Copy launches of the SM path form one chain (the CTA budget for copies is global), so the order in which
+  // the groups are added is the order in which their copies run.  For the direct schedule cut into pieces the plan lists a
+  // piece's reduce-scatter moves, its sum and its all-gather moves together; taken in that order the next piece's moves would
+  // wait behind this piece's all-gather, which waits for this piece's sum: nothing would overlap.  So the moves are ordered
+  // as a software pipeline: RS(0), RS(1), AG(0), RS(2), AG(1), ...; every dependency still points to an earlier position.
+  std::vector<size_t> order(groups.size());
+  for (size_t gi = 0; gi < groups.size(); gi++) order[gi] = gi;
+  if (c->path == HOCCL_PATH_SM && P.rs_direct && P.pieces > 1 && only_piece < 0 && part < 0) {
+    auto key = [&](size_t gi) {
+      const RGroup& rg = groups[gi];
+      const long p = rg.piece;
+      if (rg.kind != OP_MOVE) return 8 * p + 2;
+      return rg.phase == PHASE_RS ? 8 * p : 8 * p + 9;
+    };
+    std::stable_sort(order.begin(), order.end(), [&](size_t a, size_t b) { return key(a) < key(b); });
+  }
+  for (size_t oi = 0; oi < order.size() && rc == HOCCL_OK; oi++) {
+    const size_t gi = order[oi];
+    if (!included(gi)) continue;
     const RGroup& rg = groups[gi];
-    std::vector<cudaGraphNode_t> deps;
+    std::vector<cudaGraphNode_t> deps;   // groups outside this graph have no tail here: their order is the caller's (events)
     for (int d : rg.deps)
       deps.insert(deps.end(), tail[d].begin(), tail[d].end());
     if (rg.chain_dep >= 0 && std::find(rg.deps.begin(), rg.deps.end(), rg.chain_dep) == rg.deps.end())

@@ -27,9 +27,10 @@ def test_bench_line_has_the_contract_keys():
     assert d["e2e"]["h2d_bytes_per_step"] == 8 * (40 << 20) and d["e2e"]["value"] < d["value"]
     r = d["roofline"]
     assert r["bound"] == "hbm" and r["unit"] == "GB/s" and abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-9 and r["traffic"] > 0
-    # per step of the default (stage-decomposed) schedule: one chain sum launch and the empty ordering kernels of the graph
-    assert d["sms_used"]["sum_launches_per_step"] == 1 and d["sms_used"]["sum_ctas"] == 8
-    assert d["gpu_launches"] == (1 + d["sms_used"]["ordering_kernels_per_step"]) * 8
+    # per step of the default (stage-decomposed) schedule: one chain sum launch per piece (the copy route cuts a 5 MiB ring
+    # chunk into 4 pieces so that copies and sums overlap) and the empty ordering kernels of the graphs
+    assert d["sms_used"]["sum_launches_per_step"] == d["config"]["pieces_per_chunk"] == 4 and d["sms_used"]["sum_ctas"] == 8
+    assert d["gpu_launches"] == (4 + d["sms_used"]["ordering_kernels_per_step"]) * 8
     rs = d["ring_schedule"]
     assert rs["matches_oracle"] is True and rs["sum_launches_per_step"] == 7 and rs["value"] < d["value"]
     assert rs["roofline"]["kernel"].startswith("sum2_kernel")

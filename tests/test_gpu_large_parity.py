@@ -11,8 +11,9 @@ place would go unseen.  Here every element depends on (rank, position):
 * uniform[-1, 1) inputs, hashed the same way: the whole result against the oracle's step-by-step ring on the same bytes
   (order sensitive), at 64 MiB, 256 MiB and 1 GiB per rank.
 
-Both the copy route and the SM path; R = 2 and R = 8; the R = 2, 1 GiB case is the one that cuts a ring chunk of more
-than 256 MiB into two pieces.
+The copy route (default schedule, which at these sizes runs its pieces on three overlapping streams; the ring step by
+step; the direct schedule in one graph) and the SM path; R = 2 and R = 8; the ring at R = 2 and 1 GiB is the case that cuts a
+ring chunk of more than 256 MiB into two pieces.
 """
 import numpy as np
 import pytest
@@ -77,8 +78,9 @@ def _boundaries(comm, R, n, e):
 
 CONFIGS = [
     ("copy_route_sum8", hb.PATH_CE, {}),
+    ("copy_route_ring", hb.PATH_CE, {"rs_direct": 0, "ag_direct": 0}),
     ("sm_path_whole_gpu", hb.PATH_SM, {"sum_ctas": 148, "copy_ctas": 148}),
-    ("copy_route_direct", hb.PATH_CE, {"rs_direct": 1, "ag_direct": 1}),
+    ("copy_route_direct_one_graph", hb.PATH_CE, {"rs_direct": 1, "ag_direct": 1, "ce_overlap": 0}),
 ]
 
 
@@ -121,7 +123,7 @@ def test_position_dependent_integer_inputs_give_the_exact_sum_everywhere(oracle,
             ow = oracle.ring_allreduce(win)[0]
             assert (_np(recv[0][lo:hi]).view(np.uint8) == ow.view(np.uint8)).all(), (name, "boundary", b)
             assert (_np(recv[R - 1][lo:hi]).view(np.uint8) == ow.view(np.uint8)).all(), (name, "boundary", b)
-        if R == 2 and mib == 1024 and path == hb.PATH_CE and not params:
+        if R == 2 and mib == 1024 and name == "copy_route_ring":
             assert comm.last_stats()["n_pieces"] == 2      # the branch that cuts a 512 MiB ring chunk in two
         assert comm.destroy() == hb.OK
         del comm

@@ -254,3 +254,64 @@ def test_host_allreduce_with_the_direct_schedule(oracle):
         st = comm.last_stats()
         assert st["n_pieces"] > 1 and st["n_sum_launches"] == st["n_pieces"], st
         comm.destroy()
+
+
+@pytest.mark.parametrize("dtype", ["fp32", "bf16"])
+def test_overlapped_copy_route_and_pipelined_sm_path_give_the_oracle_bits(oracle, dtype):
+    """The direct schedule cut into pieces: on the copy route the three parts of every piece run as graphs of their own on three
+    internal streams ("ce_overlap"), on the SM path under CTA budgets the copy launches are issued as a software pipeline.
+    Both are scheduling only: the bits are the oracle's, for ragged sizes and piece counts, in place, repeated, and for the
+    reduce-scatter call alone; sums still run one launch at a time."""
+    e = W.elem_size(dtype)
+    cases = [(8, 8 * 70_000 + 3, dict(ce_overlap=5)), (4, 4 * 300_000, dict(ce_overlap=2)), (3, 100_001, dict(ce_overlap=16)),
+             (2, (8 << 20) // e + 8, dict()),                         # 4 MiB ring chunks: the automatic choice (4 pieces)
+             (8, 8 * 600_000 + 8, dict(path=hb.PATH_SM, sum_ctas=8, copy_ctas=40)),      # > 1 MiB chunks: pipelined pieces
+             (5, 5 * 700_000 + 1, dict(path=hb.PATH_SM, sum_ctas=3, copy_ctas=5))]
+    for R, n, params in cases:
+        params = dict(params)
+        path = params.pop("path", hb.PATH_CE)
+        xs = W.rank_inputs("uniform", 400 + R, R, n, dtype)
+        want = oracle.ring_allreduce(xs)
+        comm = make_comm(R, n, dtype, path, rs_direct=1, **params)
+        for in_place in (False, True, False):
+            got = run_allreduce(comm, xs, dtype, in_place=in_place)
+            for r in range(R):
+                assert same_bits(got[r], want[r], dtype), (dtype, R, n, params, in_place, r)
+        st = comm.last_stats()
+        assert st["n_pieces"] > 1 and st["n_sum_launches"] == st["n_pieces"], st
+        if n % R == 0:
+            count = n // R
+            wrs = oracle.ring_reduce_scatter(xs)
+            send = [DevBuf(n * e).put(xs[r]) for r in range(R)]
+            recv = [DevBuf(count * e) for _ in range(R)]
+            comm.reduce_scatter(send, recv, count, dtype)
+            torch.cuda.synchronize()
+            for r in range(R):
+                assert same_bits(recv[r].get(np_dtype(dtype)), wrs[r], dtype) and recv[r].guards_intact()
+        comm.destroy()
+    # ordering against the caller's stream: producers before, consumers after, on a side stream
+    R, n = 4, (16 << 20) // e
+    xs = W.rank_inputs("uniform", 410, R, n, dtype)
+    want = oracle.ring_allreduce(xs)
+    comm = make_comm(R, n, dtype, hb.PATH_CE, rs_direct=1)
+    tdt = torch.float32 if dtype == "fp32" else torch.int16
+    base = [torch.from_numpy(x if dtype == "fp32" else x.view(np.int16)).cuda() for x in xs]
+    send = [torch.zeros(n, dtype=tdt, device="cuda") for _ in range(R)]
+    recv = [torch.zeros(n, dtype=tdt, device="cuda") for _ in range(R)]
+    after = [torch.zeros(n, dtype=tdt, device="cuda") for _ in range(R)]
+    st = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    for rep in range(3):
+        with torch.cuda.stream(st):
+            for r in range(R):
+                send[r].copy_(base[r])
+            comm.allreduce(send, recv, n, dtype, st)
+            for r in range(R):
+                after[r].copy_(recv[r])
+                recv[r].zero_()
+        st.synchronize()
+        assert comm.last_stats()["n_pieces"] == 4
+        for r in range(R):
+            got = after[r].cpu().numpy()
+            assert same_bits(got if dtype == "fp32" else got.view(np.uint16), want[r], dtype), (rep, r)
+    comm.destroy()
