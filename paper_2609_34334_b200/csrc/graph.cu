@@ -100,7 +100,7 @@ hoccl_result_t build_graph(hoccl_comm* c, const Plan& P, const std::vector<RGrou
   // late; an empty kernel as the join of such a group fixes it (ring all-gather of the gradient bucket, seven stages of eight
   // copies: 88 -> 68 us; the 56 copies of the direct one: 61 -> 51 us).  A SUM kernel that waits for its copies directly does
   // not need it (a kernel in between costs ~1 us per step there), so groups that only feed SUMs keep the empty join.
-  std::vector<char> kernel_join(groups.size(), 0);
+  std::vector<char> kernel_join(groups.size(), 0), terminal(groups.size(), 0);
   if (c->order_kernels && (c->path == HOCCL_PATH_CE || c->path == HOCCL_PATH_CE_HOST)) {
     std::vector<char> move_user(groups.size(), 0), any_user(groups.size(), 0);
     for (size_t gi = 0; gi < groups.size(); gi++) {
@@ -110,8 +110,14 @@ hoccl_result_t build_graph(hoccl_comm* c, const Plan& P, const std::vector<RGrou
         if (groups[gi].kind == OP_MOVE) move_user[d] = 1;
       }
     }
-    for (size_t gi = 0; gi < groups.size(); gi++) kernel_join[gi] = groups[gi].kind == OP_MOVE && (move_user[gi] || !any_user[gi]);
+    // groups of copies that nothing in this graph waits for share ONE such kernel at the end of the graph (one per group cost
+    // 2 us of kernel time each and bought nothing more)
+    for (size_t gi = 0; gi < groups.size(); gi++) {
+      kernel_join[gi] = groups[gi].kind == OP_MOVE && move_user[gi];
+      terminal[gi] = groups[gi].kind == OP_MOVE && !any_user[gi];
+    }
   }
+  std::vector<cudaGraphNode_t> terminal_nodes;
   hoccl_result_t rc = HOCCL_OK;
   auto fail = [&](cudaError_t e, const char* what) {
     rc = cuda_fail(c, e, what);
@@ -307,7 +313,9 @@ hoccl_result_t build_graph(hoccl_comm* c, const Plan& P, const std::vector<RGrou
       fail(e, "graph node");
       break;
     }
-    if (nodes.size() == 1) {
+    if (terminal[gi]) {
+      terminal_nodes.insert(terminal_nodes.end(), nodes.begin(), nodes.end());
+    } else if (nodes.size() == 1) {
       tail[gi].assign(1, nodes[0]);
     } else if (nodes.size() > 1) {
       cudaGraphNode_t join;
@@ -328,6 +336,17 @@ hoccl_result_t build_graph(hoccl_comm* c, const Plan& P, const std::vector<RGrou
       }
       tail[gi].assign(1, join);
     }
+  }
+  if (rc == HOCCL_OK && terminal_nodes.size() > 1) {
+    cudaGraphNode_t join;
+    cudaKernelNodeParams kp = {};
+    kp.func = const_cast<void*>(graph_root_kernel_entry());
+    kp.gridDim = dim3(1);
+    kp.blockDim = dim3(32);
+    kp.kernelParams = nullptr;
+    cudaError_t e = cudaGraphAddKernelNode(&join, g, terminal_nodes.data(), terminal_nodes.size(), &kp);
+    if (e == cudaSuccess) entry->n_order_launches++;
+    else rc = cuda_fail(c, e, "graph end node");
   }
   if (rc == HOCCL_OK) {
     cudaError_t e = cudaGraphInstantiate(out_exec, g, 0);

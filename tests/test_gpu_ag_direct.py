@@ -233,9 +233,10 @@ def test_ordering_kernels_are_counted_and_optional(oracle):
         got = run_allreduce(comm, xs, dtype)
         assert all(same_bits(got[r], want[r], dtype) for r in range(R)), (order, direct)
         st = comm.last_stats()
-        # one all-reduce graph: a root in front of the 8 first copies and a join behind each of the 7 all-gather stages
-        # (ring: the next stage waits for it; direct: the stages are separate groups here and each ends the graph)
-        assert st["n_order_launches"] == (1 + 7 if order else 0), (order, direct, st)
+        # one all-reduce graph: a root in front of the 8 first copies; ring all-gather: a join behind each of the first 6 stages
+        # (the next stage waits for it) and one at the end of the graph; direct all-gather: its 7 stages all end the graph and
+        # share the one join there
+        assert st["n_order_launches"] == ((1 + (1 if direct else 7)) if order else 0), (order, direct, st)
         assert st["n_sum_launches"] == 7 and st["n_move_launches"] == 0 and st["n_moves"] == 112
         comm.destroy()
     # the SM path and the stream executor have none

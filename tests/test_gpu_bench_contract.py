@@ -53,4 +53,4 @@ def test_large_message_and_gemm_rows_carry_oracle_flags():
     gm = d["gemm_loss_matched"]
     names = [r["config"] for r in gm["rows"]]
     assert "CE_sum8" in names and all("SM_copy%d_sum8" % b in names for b in (8, 16, 32, 64, 148))
-    assert all(r["matches_oracle"] is True and 0.0 <= r["gemm_loss"] < 1.0 for r in gm["rows"])
+    assert all(r["matches_oracle"] is True and -0.05 < r["gemm_loss"] < 1.0 for r in gm["rows"])      # a loss of zero is measured within ~1 %
