@@ -561,7 +561,7 @@ def gemm_loss_matched(torch, hb, W, B, want_dev):
     alone, _, _ = corun(n_gemm)
     rows = []
     configs = [("CE_sum8", hb.PATH_CE, 8, 8, {}), ("CE_sum8_ring", hb.PATH_CE, 8, 8, {"rs_direct": 0, "ag_direct": 0}),
-               ("CE_sum8_plain_graphs", hb.PATH_CE, 8, 8, {"order_kernels": 0})]
+               ("CE_sum8_plain_graphs", hb.PATH_CE, 8, 8, {"order_kernels": 0, "ce_overlap": 0})]
     configs += [("SM_copy%d_sum8" % b, hb.PATH_SM, 8, b, {}) for b in (8, 16, 32, 64, 148)]
     configs += [("SM_copy148_sum148", hb.PATH_SM, 148, 148, {})]
     for name, path, sc, cc, extra in configs:

@@ -6,6 +6,7 @@
     python -m paper_2609_34334_b200.microbench --kernel port --mib 256 --ctas 8    # what the memory ports of `ctas` SMs carry
     python -m paper_2609_34334_b200.microbench --kernel fan --mib 25 --ctas 148    # one source to 7 destinations: fan-out against 7 copies
     python -m paper_2609_34334_b200.microbench --kernel chain --mib 25 --ctas 8    # 7 inbox operands + the local one into one output
+    python -m paper_2609_34334_b200.microbench --kernel beside --mib 40 --ctas 8   # the chain sum while a 1 GiB copy runs on another stream
 
 Operands are larger than L2 by default; timing uses CUDA events on the launching stream after warm-up.
 Prints one JSON line.  This is the small case used for ncu captures of a single kernel.
@@ -23,7 +24,7 @@ from . import diag as hd
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--kernel", default="sum", choices=["sum", "copy", "routes", "ring", "port", "fan", "chain"])
+    ap.add_argument("--kernel", default="sum", choices=["sum", "copy", "routes", "ring", "port", "fan", "chain", "beside"])
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "fp32"])
     ap.add_argument("--mib", type=int, default=200, help="MiB per operand")
     ap.add_argument("--ctas", type=int, default=8)
@@ -58,6 +59,50 @@ def main():
             sec = e0.elapsed_time(e1) / 1e3 / args.reps
             out[name] = {"GBps": moved / sec / 1e9, "GBps_per_sm": moved / sec / 1e9 / args.ctas, "us": sec * 1e6}
         print(json.dumps(out))
+        return
+    if args.kernel == "beside":
+        # what concurrent copies cost a sum under a CTA budget: the chain sum (7 inbox operands + the local one) is timed while a
+        # 1 GiB copy runs on another stream, as copy_kernel launches of several CTA budgets and as one driver copy
+        nsrc = 7
+        n = nbytes // 2
+        inbox = torch.empty(nsrc * n, dtype=torch.bfloat16, device="cuda").normal_(0, 1e-3)
+        local = torch.empty(n, dtype=torch.bfloat16, device="cuda").normal_(0, 1e-3)
+        out_t = torch.empty(n, dtype=torch.bfloat16, device="cuda")
+        big = 1 << 30
+        src = torch.empty(big, dtype=torch.uint8, device="cuda")
+        dst = torch.empty(big, dtype=torch.uint8, device="cuda")
+        sa, sb = torch.cuda.Stream(), torch.cuda.Stream()
+        torch.cuda.synchronize()
+
+        def chain():
+            assert hd.chain_launch(inbox, nbytes, nsrc, local, out_t, n, "bf16", args.ctas, sa) == hb.OK
+
+        rows = []
+        for what in ("none", "copy_16", "copy_32", "copy_48", "copy_64", "copy_100", "copy_140", "driver"):
+            best = None
+            for _ in range(max(1, args.reps)):
+                chain()
+                torch.cuda.synchronize()
+                k0, k1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                c0.record(sb)
+                if what == "driver":
+                    with torch.cuda.stream(sb):
+                        dst.copy_(src, non_blocking=True)
+                elif what != "none":
+                    assert hd.copy_launch(src, dst, big, int(what.split("_")[1]), sb) == hb.OK
+                c1.record(sb)
+                k0.record(sa)
+                chain()
+                k1.record(sa)
+                torch.cuda.synchronize()
+                row = {"background": what, "chain_us": k0.elapsed_time(k1) * 1e3, "background_us": c0.elapsed_time(c1) * 1e3}
+                if best is None or row["chain_us"] < best["chain_us"]:
+                    best = row
+            best["background_GBps"] = 2.0 * big / best["background_us"] / 1e3 if what != "none" else 0.0
+            rows.append(best)
+        print(json.dumps({"probe": "chain sum (%d CTAs, output of %d MiB, 8 operands) beside a 1 GiB copy on another stream" % (args.ctas, args.mib),
+                          "rows": rows}))
         return
     if args.kernel == "chain":
         # the sum of the direct reduce-scatter for R = 8: seven inbox operands and the local one, one output (8 reads : 1 write)

@@ -103,21 +103,23 @@ def sweep_sizes(args):
     torch.cuda.set_device(0)
     stream = torch.cuda.Stream()
     ops = ["allreduce", "reduce_scatter", "allgather", "alltoall", "sendrecv"] if args.ops == "all" else args.ops.split(",")
-    # name, path, SUM CTAs, copy CTAs, whole collective as one cooperative kernel
-    configs = [("CE", hb.PATH_CE, 8, 8, 0), ("SM8", hb.PATH_SM, 8, 8, 0), ("SMall", hb.PATH_SM, 148, 148, 0),
-               ("SM8fused", hb.PATH_SM, 8, 8, 1), ("SMallfused", hb.PATH_SM, 148, 148, 1),
-               # all-gather as independent stages (fan-out copy on the SM path); the last one adds the forward comparison variant
-               ("CEplain", hb.PATH_CE, 8, 8, 0),   # copy route, plain graphs: no empty ordering kernels (order_kernels = 0)
-               ("CEall", hb.PATH_CE, 148, 8, 0),   # copy route with whole-GPU sums: what the route reaches without the 8-CTA SUM budget
-               ("CEdirect", hb.PATH_CE, 8, 8, 0), ("SM8direct", hb.PATH_SM, 8, 8, 0), ("SMalldirect", hb.PATH_SM, 148, 148, 0),
-               ("SMallfwddirect", hb.PATH_SM, 148, 148, 0),
-               # direct schedule: reduce-scatter and all-gather both as independent stages, one chain sum per rank
-               ("CErsdirect", hb.PATH_CE, 8, 8, 0), ("CEallrsdirect", hb.PATH_CE, 148, 8, 0), ("SM8rsdirect", hb.PATH_SM, 8, 8, 0),
-               ("SMallrsdirect", hb.PATH_SM, 148, 148, 0)]
-    if args.configs != "all":
-        configs = [c for c in configs if c[0] in args.configs.split(",")]
-    else:
-        configs = configs[:3]
+    # name -> (path, SUM CTAs, copy CTAs, further parameters).  Default schedule unless "ring" is in the name.
+    ring = {"rs_direct": 0, "ag_direct": 0}
+    table = {
+        "CE": (hb.PATH_CE, 8, 8, {}),                                   # copy route as a new communicator has it
+        "CEring": (hb.PATH_CE, 8, 8, dict(ring)),                       # the ring step by step
+        "CEdriver": (hb.PATH_CE, 8, 8, {"ce_small_bytes": 0}),          # driver copies at every size (no small-message rule)
+        "CEonegraph": (hb.PATH_CE, 8, 8, {"ce_overlap": 0}),            # the direct schedule as one graph (no overlap of copies and sums)
+        "CEplain": (hb.PATH_CE, 8, 8, {"order_kernels": 0, "ce_overlap": 0}),   # plain graphs: no empty ordering kernels
+        "CEall": (hb.PATH_CE, 148, 8, {}),                              # copy route with whole-GPU sums
+        "SM8": (hb.PATH_SM, 8, 8, {}), "SM8ring": (hb.PATH_SM, 8, 8, dict(ring)),
+        "SM40": (hb.PATH_SM, 8, 40, {}),                                # 8-CTA sums beside 40 copy CTAs
+        "SMall": (hb.PATH_SM, 148, 148, {}), "SMallring": (hb.PATH_SM, 148, 148, dict(ring)),
+        "SMallfused": (hb.PATH_SM, 148, 148, {"fused": 1}),             # the ring as one cooperative kernel
+        "SM8fused": (hb.PATH_SM, 8, 8, {"fused": 1}),
+    }
+    names = ["CE", "SM8", "SMall"] if args.configs == "all" else args.configs.split(",")
+    configs = [(nm,) + table[nm] for nm in names]
     out = open(args.out, "w") if args.out else None
     for dtype in args.dtypes.split(","):
         for R in [int(r) for r in args.ranks.split(",")]:
@@ -137,25 +139,22 @@ def sweep_sizes(args):
                     arena = Arena(op, R, S, dtype, nsets)
                     scratch = torch.empty(hb.scratch_bytes_direct(R, S // e, dtype) + 256, dtype=torch.uint8, device="cuda")
                     pad = (-scratch.data_ptr()) % 256
-                    for name, path, sc, cc, fused in configs:
+                    for name, path, sc, cc, extra in configs:
                         comm = hb.Comm(R, 0)
                         if scratch.numel() > 256:
                             comm.set_scratch(scratch.data_ptr() + pad, scratch.numel() - 256)
                         comm.set_path(path)
                         comm.set_param("sum_ctas", sc)
                         comm.set_param("copy_ctas", cc)
-                        comm.set_param("fused", fused)
-                        direct = name.endswith("direct")
-                        comm.set_param("ag_direct", 1 if direct else 0)
-                        comm.set_param("forward", 1 if "fwd" in name else 0)
-                        comm.set_param("order_kernels", 0 if name == "CEplain" else 1)
-                        comm.set_param("rs_direct", 1 if name.endswith("rsdirect") else 0)
+                        for k_, v_ in extra.items():
+                            comm.set_param(k_, v_)
                         t = time_op(comm, arena, stream)
                         row = {"op": op, "R": R, "dtype": dtype, "S": S, "config": name, "sum_ctas": sc,
                                "copy_ctas": cc if path == hb.PATH_SM else None, "us": t * 1e6, "algbw_GBps": S / t / 1e9,
                                "busbw_GBps": S * _bus_factor(op, R) / t / 1e9,
-                               # the ring's byte count; not given where the variant moves fewer bytes than the ring
-                               "hbm_frac_of_8TBps": None if direct else _hbm_bytes(op, S, R) / t / NOMINAL_HBM, "buffer_sets": nsets}
+                               # the bytes the rank-local RING must move for this operation, over the time
+                               "hbm_frac_of_8TBps": _hbm_bytes(op, S, R) / t / NOMINAL_HBM, "buffer_sets": nsets,
+                               "pieces": int(comm.last_stats()["n_pieces"])}
                         line = json.dumps(row)
                         print(line, flush=True)
                         if out:
@@ -321,17 +320,17 @@ def gradients(args):
         for b in [int(x) for x in args.budgets.split(",")]:
             configs.append(("SM_copy%d_sum%d" % (b, min(b, 8)), hb.PATH_SM, min(b, 8), b))
         configs.append(("SM_copy148_sum148", hb.PATH_SM, 148, 148))
-    if getattr(args, "direct", False):   # every SM-path configuration once more with the direct (fan-out) all-gather
-        configs = (configs + [(n_ + "_direct", p_, s_, c_) for n_, p_, s_, c_ in configs if p_ == hb.PATH_SM] +
-                   [(n_ + "_rsdirect", p_, s_, c_) for n_, p_, s_, c_ in configs if not n_.endswith("_plain_graphs")])
+    if getattr(args, "ring", False):   # every configuration once more on the ring schedule, step by step
+        configs = configs + [(n_ + "_ring", p_, s_, c_) for n_, p_, s_, c_ in configs if not n_.endswith("_plain_graphs")]
     for name, path, sc, cc in configs:
         comm = hb.Comm(R, 0)
         comm.set_scratch(scratch.data_ptr() + pad, scratch.numel() - 256)
         comm.set_path(path)
         comm.set_param("sum_ctas", sc)
         comm.set_param("copy_ctas", cc)
-        comm.set_param("ag_direct", 1 if name.endswith("direct") else 0)
-        comm.set_param("rs_direct", 1 if name.endswith("_rsdirect") else 0)
+        if name.endswith("_ring"):
+            comm.set_param("ag_direct", 0)
+            comm.set_param("rs_direct", 0)
         comm.set_param("order_kernels", 0 if name.endswith("_plain_graphs") else 1)   # the copy-route graphs without ordering kernels
         for k in range(pool):
             comm.allreduce(send[k], recv[k], per, dtype, stream)
@@ -504,7 +503,7 @@ def main():
     g = sub.add_parser("gradients")
     g.add_argument("--buckets", type=int, default=32)
     g.add_argument("--budgets", default="", help="comma list of copy-kernel CTA budgets, e.g. 1,2,4,8,16,32,64")
-    g.add_argument("--direct", action="store_true", help="repeat every SM-path configuration with ag_direct = 1")
+    g.add_argument("--ring", action="store_true", help="repeat every configuration on the ring schedule (rs_direct = 0, ag_direct = 0)")
     sub.add_parser("launch-cost")
     a2 = sub.add_parser("alltoallv")
     a2.add_argument("--mib", default="4,64,256", help="comma list of MiB sent per rank")
