@@ -124,6 +124,16 @@ hoccl_result_t hoccl_selftest_bf16_add(unsigned long long* counts, hoccl_stream_
  */
 hoccl_result_t hoccl_selftest_barrier_timeout(hoccl_comm_t comm, void* dst, const void* src, size_t bytes, hoccl_stream_t stream);
 
+/*
+ * The same for the bounded waits of the "roles" kernel (communicator parameter "roles" = 1, else HOCCL_ERR_UNSUPPORTED):
+ * enqueues the all-reduce the arguments describe (as hoccl_allreduce) with summing CTAs that wait for one mover more than
+ * the grid has.  They poll for their bounded number of rounds (a second or two) and give up, every other CTA sees the
+ * give-up flag and leaves, the kernel ends by itself (the receive buffers are then NOT the all-reduce), and
+ * hoccl_comm_async_error reports HOCCL_ERR_TIMEOUT; the counters are clean for the next call.
+ */
+hoccl_result_t hoccl_selftest_roles_timeout(const void* const* sendbufs, void* const* recvbufs, size_t count, hoccl_dtype_t dtype,
+                                            hoccl_comm_t comm, hoccl_stream_t stream);
+
 /* ---------------------------------------------------------------- plan inspection (host only) --- */
 
 /*
@@ -197,8 +207,10 @@ typedef struct {
   long onepass, forward, fused, rs_direct, ag_direct, handshake, use_graph, ce_small_bytes, ce_small_ctas, copy_ctas;
   size_t scratch_bytes;
   int host_call;
+  long roles;
 } hoccl_options_t;
-typedef enum { HOCCL_EXEC_GRAPH = 0, HOCCL_EXEC_STREAMS = 1, HOCCL_EXEC_ONE_KERNEL = 2, HOCCL_EXEC_ONEPASS = 3, HOCCL_EXEC_PROXY = 4 } hoccl_executor_t;
+typedef enum { HOCCL_EXEC_GRAPH = 0, HOCCL_EXEC_STREAMS = 1, HOCCL_EXEC_ONE_KERNEL = 2, HOCCL_EXEC_ONEPASS = 3, HOCCL_EXEC_PROXY = 4,
+               HOCCL_EXEC_ROLES = 5 } hoccl_executor_t;
 typedef struct {
   int plan_kind;    /* base collective | hoccl_plan_flag_t bits: what hoccl_plan_build is given */
   int executor;     /* hoccl_executor_t */

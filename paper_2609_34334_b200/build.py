@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libhoccl.so")
-SOURCES = ["api.cu", "exec.cu", "p2p.cu", "kernels.cu", "plan.cpp", "static_scratch.cu", "proxy.cu", "sched.cpp", "probe.cu", "ring.cu", "graph.cu", "ring_host.cu", "options.cpp"]
+SOURCES = ["api.cu", "exec.cu", "p2p.cu", "kernels.cu", "plan.cpp", "static_scratch.cu", "proxy.cu", "sched.cpp", "probe.cu", "ring.cu", "graph.cu", "ring_host.cu", "options.cpp", "roles.cu"]
 HEADERS = ["comm.h", "kernels.cuh", "device_common.cuh", "plan.h", "proxy.h", "sched.h", "options.h", os.path.join("..", "..", "include", "hoccl.h"), os.path.join("..", "..", "include", "hoccl_diag.h")]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

@@ -68,6 +68,8 @@ hoccl_result_t hoccl_comm_destroy(hoccl_comm_t c) {
   for (auto& e : c->cache) destroy_entry(&e);
   if (c->ring_bar) cudaFree(c->ring_bar);
   if (c->ring_err) cudaFreeHost(c->ring_err);
+  if (c->roles_ctl) cudaFree(c->roles_ctl);
+  if (c->roles_err) cudaFreeHost(c->roles_err);
   for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
   for (cudaEvent_t e : c->post_events) cudaEventDestroy(e);
   for (auto& p : c->prof_pool) {
@@ -146,6 +148,7 @@ static long* param_slot(hoccl_comm* c, const char* key, long* lo, long* hi) {
               {"ce_small_bytes", &c->ce_small_bytes, 0, 1L << 40},
               {"ce_small_ctas", &c->ce_small_ctas, 1, 1024},
               {"p2p_strict", &c->p2p_strict, 0, 1},
+              {"roles", &c->roles, 0, 1},
               {"ce_overlap", &c->ce_overlap, -1, 64},
               {"model_gpus_per_node", &c->model_gpus_per_node, 0, kMaxRanks},
               {"model_rdma_sub_bytes", &c->model_rdma_sub_bytes, 0, 1L << 40},
@@ -235,6 +238,10 @@ hoccl_result_t hoccl_comm_async_error(hoccl_comm_t c, int clear) {
     if (clear) *reinterpret_cast<volatile int*>(c->ring_err) = 0;
     return HOCCL_ERR_TIMEOUT;   // a barrier wait of the whole-collective kernel ran out
   }
+  if (c->roles_err && *reinterpret_cast<volatile int*>(c->roles_err) != 0) {
+    if (clear) *reinterpret_cast<volatile int*>(c->roles_err) = 0;
+    return HOCCL_ERR_TIMEOUT;   // a wait of the roles kernel ran out
+  }
   if (!c->proxy) return HOCCL_OK;
   int e = c->proxy->async_error();
   if (clear) c->proxy->clear_error();
@@ -250,6 +257,16 @@ hoccl_result_t hoccl_selftest_barrier_timeout(hoccl_comm_t c, void* dst, const v
   if (!c || !dst || !src || bytes < 32 || (bytes & 31)) return HOCCL_ERR_INVALID_ARG;
   CU_TRY(c, cudaSetDevice(c->device));
   return ring_barrier_selftest(c, dst, src, bytes, (cudaStream_t)stream);
+}
+
+hoccl_result_t hoccl_selftest_roles_timeout(const void* const* send, void* const* recv, size_t count, hoccl_dtype_t dtype, hoccl_comm_t c,
+                                            hoccl_stream_t stream) {
+  if (!c) return HOCCL_ERR_INVALID_ARG;
+  if (!c->roles) return HOCCL_ERR_UNSUPPORTED;
+  c->roles_missing = 1;
+  hoccl_result_t rc = hoccl_allreduce(send, recv, count, dtype, HOCCL_SUM, c, stream);
+  c->roles_missing = 0;
+  return rc;
 }
 
 long hoccl_comm_handshakes(hoccl_comm_t c) { return (c && c->proxy) ? c->proxy->handshakes() : 0; }
@@ -913,7 +930,7 @@ int hoccl_plan_group_deps(hoccl_plan_t plan, int group, int* deps, int cap) {
 extern "C" hoccl_result_t hoccl_options_resolve(const hoccl_options_t* o, hoccl_resolved_t* out) {
   if (!o || !out) return HOCCL_ERR_INVALID_ARG;
   hoccl::OptionsIn in{o->kind, o->R, o->count, o->dtype, o->path, o->onepass, o->forward, o->fused, o->rs_direct, o->ag_direct,
-                      o->handshake, o->use_graph, o->ce_small_bytes, o->ce_small_ctas, o->copy_ctas, o->scratch_bytes, o->host_call};
+                      o->handshake, o->use_graph, o->ce_small_bytes, o->ce_small_ctas, o->copy_ctas, o->scratch_bytes, o->host_call, o->roles};
   hoccl::OptionsOut r;
   hoccl_result_t rc = hoccl::resolve_options(in, &r);
   if (rc != HOCCL_OK) return rc;

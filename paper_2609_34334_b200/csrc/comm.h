@@ -85,6 +85,12 @@ struct GraphEntry {
   bool ring_large = false;
   int ring_grid = 0, ring_threads = 0;
   bool ring_has_sum = false;
+  // "roles" setting: the direct schedule as one cooperative kernel with summing and moving CTAs (exec stays null)
+  char* roles_tab = nullptr;    // owned device memory: the segment tables of this call signature
+  std::vector<char> roles_args; // a RolesArgs, by value
+  const void* roles_fn = nullptr;
+  int roles_grid = 0, roles_sum_ctas = 0;
+  size_t roles_smem = 0;        // dynamic shared memory of the launch = size of the tables
 };
 
 }  // namespace hoccl
@@ -94,7 +100,8 @@ struct hoccl_comm {
   hoccl_path_t path = HOCCL_PATH_CE;
   long sum_ctas = 8, copy_ctas = 8, piece_bytes = 4 << 20, max_pieces = 8, lanes = 4, use_graph = 1, profile = 0, p2p_split = 1, ce_sub_bytes = 0,
        handshake = 0, watchdog_ms = 10000, onepass = 0, forward = 0, fused = 0, host_pieces = 8, ag_direct = 2, order_kernels = 1, rs_direct = 2,
-       ce_small_bytes = 8 << 20, ce_small_ctas = 148, p2p_strict = 0, ce_overlap = -1, model_gpus_per_node = 0, model_rdma_sub_bytes = 0;
+       ce_small_bytes = 8 << 20, ce_small_ctas = 148, p2p_strict = 0, ce_overlap = -1, model_gpus_per_node = 0, model_rdma_sub_bytes = 0, roles = 0,
+       roles_missing = 0 /* self-test only: summing CTAs wait for this many movers that do not exist */;
   bool piece_bytes_set = false;  // the caller chose a piece size: no automatic choice
   hoccl::Proxy* proxy = nullptr;
   cudaStream_t lane[hoccl::kMaxLanes] = {};
@@ -109,6 +116,9 @@ struct hoccl_comm {
   unsigned* ring_bar = nullptr;  // "fused" setting: three device words of the grid barrier (library owned, 16 bytes)
   int* ring_err = nullptr;       // mapped pinned host word the ring kernel sets when a barrier wait ran out
   int* ring_err_dev = nullptr;   // the same word as the device sees it
+  char* roles_ctl = nullptr;     // "roles" setting: control words and per-piece counters of the roles kernel (library owned, 1 KiB)
+  int* roles_err = nullptr;      // mapped pinned host word the roles kernel sets when a wait ran out
+  int* roles_err_dev = nullptr;
   char* host_staging = nullptr;  // pinned host memory of the CE_HOST path
   size_t host_staging_bytes = 0;
   std::map<std::pair<int, int>, std::deque<hoccl::Post>> pending;
@@ -194,6 +204,9 @@ void add_host_copies(const Plan& P, int p, char* dev, char* host, std::vector<Ho
 cudaError_t enqueue_host_copy(const HostCopy& hc, bool to_device, cudaStream_t s);
 // ring_host.cu
 hoccl_result_t build_ring(hoccl_comm* c, const Plan& P, const std::vector<RGroup>& groups, GraphEntry* entry);
+// roles.cu
+hoccl_result_t build_roles(hoccl_comm* c, const Plan& P, const std::vector<RGroup>& groups, GraphEntry* entry);
+hoccl_result_t launch_roles(hoccl_comm* c, GraphEntry* entry, cudaStream_t stream);
 // exec.cu
 hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user);
 // HOCCL_OK if the communicator's settings fit together for such a call (see options.h); nothing is enqueued

@@ -394,6 +394,8 @@ std::vector<uint64_t> make_key(hoccl_comm* c, const Call& call) {
   k.push_back((uint64_t)c->rs_direct);
   k.push_back((uint64_t)c->ce_overlap);
   k.push_back((uint64_t)(c->fused && c->path == HOCCL_PATH_SM && !c->handshake));
+  k.push_back((uint64_t)c->roles);
+  k.push_back((uint64_t)c->roles_missing);
   k.push_back((uint64_t)(uintptr_t)c->scratch);
   k.push_back((uint64_t)c->scratch_bytes);
   k.push_back((uint64_t)(uintptr_t)c->host_staging);
@@ -474,6 +476,18 @@ static hoccl_result_t launch_entry(hoccl_comm* c, GraphEntry* hit, cudaStream_t 
     c->stats.n_sum_launches = 0;
     c->stats.max_copy_ctas = hit->ring_grid;
     c->stats.max_sum_ctas = hit->ring_has_sum ? hit->ring_grid : 0;
+    c->stats.host_launch_us = now_us() - t0;
+    return HOCCL_OK;
+  }
+  if (hit->roles_fn) {
+    hoccl_result_t rrc = launch_roles(c, hit, user);
+    if (rrc != HOCCL_OK) return rrc;
+    c->stats.n_pieces = hit->n_pieces;
+    c->stats.n_moves = hit->n_moves;
+    c->stats.n_move_launches = 1;
+    c->stats.n_sum_launches = 0;
+    c->stats.max_copy_ctas = hit->roles_grid - hit->roles_sum_ctas;
+    c->stats.max_sum_ctas = hit->roles_sum_ctas;
     c->stats.host_launch_us = now_us() - t0;
     return HOCCL_OK;
   }
@@ -569,7 +583,7 @@ static hoccl_result_t launch_entry(hoccl_comm* c, GraphEntry* hit, cudaStream_t 
 static OptionsIn options_of(hoccl_comm* c, int kind, size_t count, int dtype, bool host_call) {
   return OptionsIn{kind, c->R, count, dtype, (int)c->path, c->onepass, c->forward, c->fused, c->rs_direct, c->ag_direct,
                    c->handshake, c->use_graph, c->ce_small_bytes, c->ce_small_ctas, c->copy_ctas, c->scratch ? c->scratch_bytes : 0,
-                   host_call ? 1 : 0};
+                   host_call ? 1 : 0, c->roles};
 }
 
 hoccl_result_t check_options(hoccl_comm* c, int kind, size_t count, int dtype) {
@@ -603,6 +617,7 @@ hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
   c->copy_ctas = opt.copy_ctas;
   const bool onepass_case = opt.executor == EXEC_ONEPASS;
   const bool fused = opt.executor == EXEC_ONE_KERNEL;
+  const bool roles = opt.executor == EXEC_ROLES;
   const bool graphs = opt.executor != EXEC_STREAMS && !onepass_case;
   std::vector<uint64_t> key;
   if (graphs && call->count != 0) {
@@ -691,6 +706,14 @@ hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
     const size_t chunk = q * dtype_size(call->dtype);
     max_pieces = (int)c->host_pieces;
     piece_bytes = std::max<size_t>((size_t)64 << 10, ((chunk + max_pieces - 1) / max_pieces + 1023) / 1024 * 1024);
+  } else if (roles) {
+    // pieces cost no launch here, but every piece drains and refills the register pipelines of both roles (measured ~6 us per piece
+    // for the sums): about twelve per ring chunk, a multiple of the movers' tile (128 KiB) so that no segment ends in a short tile
+    if (!c->piece_bytes_set) {
+      const size_t tile = (size_t)128 << 10;
+      piece_bytes = std::min<size_t>((size_t)2 << 20, std::max<size_t>(2 * tile, (ring_chunk / 12 + tile - 1) / tile * tile));
+    }
+    max_pieces = 32;   // the tables of all pieces must fit into a CTA's shared memory
   } else if (fused) {   // one kernel walks the steps in order; whole chunks measured faster than pieces (fewer barriers and tails)
     piece_bytes = (size_t)1 << 60;
     max_pieces = 1;
@@ -759,8 +782,9 @@ hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
         return rc;
       }
     } else {
-      rc = fused ? build_ring(c, P, groups, &entry) : HOCCL_ERR_UNSUPPORTED;
-      if (rc == HOCCL_ERR_UNSUPPORTED) rc = build_graph(c, P, groups, &entry, -1, &entry.exec);   // not asked for, or too many ranks for one launch
+      rc = fused ? build_ring(c, P, groups, &entry) : roles ? build_roles(c, P, groups, &entry) : HOCCL_ERR_UNSUPPORTED;
+      // not asked for, too many ranks for one launch (fused), or more CTAs than can be resident together (roles)
+      if (rc == HOCCL_ERR_UNSUPPORTED) rc = build_graph(c, P, groups, &entry, -1, &entry.exec);
       if (rc != HOCCL_OK) {
         destroy_entry(&entry);
         return rc;

@@ -21,6 +21,11 @@ void destroy_entry(GraphEntry* e) {
   }
   e->exec = nullptr;
   e->prof_events.clear();
+  if (e->roles_tab) {
+    cudaFree(e->roles_tab);   // waits for launches still in flight
+    e->roles_tab = nullptr;
+    e->roles_fn = nullptr;
+  }
 }
 
 // Host <-> staging copies of one piece of one rank (all-reduce layout): piece p of every ring chunk, i.e. rows of

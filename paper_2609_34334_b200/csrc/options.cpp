@@ -32,14 +32,19 @@ hoccl_result_t resolve_options(const OptionsIn& in, OptionsOut* out) {
     return HOCCL_ERR_UNSUPPORTED;
   if (reduction && in.rs_direct == 1 && (in.forward || in.fused)) return HOCCL_ERR_UNSUPPORTED;
 
+  const bool roles = in.roles && reduction && !in.host_call;
+  if (roles && (in.path != HOCCL_PATH_SM || in.R < 2 || in.R > 8 || in.handshake || in.onepass || in.forward || in.fused || in.rs_direct == 0 ||
+                (in.kind == PLAN_ALLREDUCE && in.ag_direct == 0)))
+    return HOCCL_ERR_UNSUPPORTED;
+
   const bool forward = in.forward && reduction;
   const bool fused = in.fused && !in.host_call;   // the pipelined host entry runs its pieces as graphs
-  bool direct_rs = reduction && in.rs_direct == 1;
-  if (reduction && in.rs_direct == 2 && in.R > 1 && !forward && !in.fused && !onepass) {
+  bool direct_rs = reduction && (in.rs_direct == 1 || roles);
+  if (reduction && in.rs_direct == 2 && in.R > 1 && !forward && !in.fused && !onepass && !roles) {
     const size_t cnt = in.kind == PLAN_ALLREDUCE ? in.count : in.count * (size_t)in.R;
     direct_rs = in.scratch_bytes >= (size_t)(in.R - 1) * (size_t)in.R * slot_bytes_for(in.R, cnt, e);
   }
-  bool direct_ag = gathers && in.ag_direct == 1;
+  bool direct_ag = gathers && (in.ag_direct == 1 || roles);
   if (gathers && in.ag_direct == 2) {
     const size_t q = in.kind == PLAN_ALLREDUCE ? (in.count + in.R - 1) / in.R : in.count;
     direct_ag = path != HOCCL_PATH_CE || q * e <= ((size_t)64 << 20);
@@ -49,6 +54,7 @@ hoccl_result_t resolve_options(const OptionsIn& in, OptionsOut* out) {
   if (onepass) out->executor = EXEC_ONEPASS;
   else if (in.handshake) out->executor = EXEC_PROXY;
   else if (fused) out->executor = EXEC_ONE_KERNEL;
+  else if (roles) out->executor = EXEC_ROLES;
   else out->executor = in.use_graph ? EXEC_GRAPH : EXEC_STREAMS;
   out->path = path;
   out->copy_ctas = copy_ctas;

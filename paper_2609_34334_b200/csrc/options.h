@@ -10,6 +10,11 @@
 //   fused       one cooperative kernel on HOCCL_PATH_SM: refused on the other paths; it has no chain phase and does not
 //               forward, so "rs_direct" = 1 is refused with it; "forward" with "fused" is served (the ring kernel walks the
 //               forward plan).  It ignores "use_graph".
+//   roles       all-reduce and reduce-scatter calls as ONE cooperative kernel with summing and moving CTAs (roles.cu).  It runs
+//               the direct schedule on HOCCL_PATH_SM for 2 to 8 ranks: refused on the other paths, for other rank counts, with
+//               "handshake", "onepass", "forward", "fused", "rs_direct" = 0 and (all-reduce) "ag_direct" = 0.  Like "rs_direct"
+//               = 1 it needs the scratch of the direct form (HOCCL_ERR_SCRATCH otherwise).  Other calls ignore it; so does the
+//               pipelined host entry.  It ignores "use_graph".
 //   forward     applies to all-reduce and reduce-scatter; "rs_direct" = 1 is refused with it (the direct form has no steps
 //               to forward between).
 //   rs_direct   2 takes the direct reduce-scatter when nothing above excludes it and the attached scratch holds its R - 1
@@ -27,7 +32,7 @@
 
 namespace hoccl {
 
-enum Executor { EXEC_GRAPH = 0, EXEC_STREAMS = 1, EXEC_ONE_KERNEL = 2, EXEC_ONEPASS = 3, EXEC_PROXY = 4 };
+enum Executor { EXEC_GRAPH = 0, EXEC_STREAMS = 1, EXEC_ONE_KERNEL = 2, EXEC_ONEPASS = 3, EXEC_PROXY = 4, EXEC_ROLES = 5 };
 
 struct OptionsIn {
   int kind;          // PlanKind base: 0 all-reduce, 1 reduce-scatter, 2 all-gather, 3 all-to-all
@@ -39,6 +44,7 @@ struct OptionsIn {
   long ce_small_bytes, ce_small_ctas, copy_ctas;
   size_t scratch_bytes;   // attached scratch (0: none)
   int host_call;          // hoccl_host_allreduce
+  long roles = 0;
 };
 
 struct OptionsOut {

@@ -12,14 +12,14 @@ PLAN_ALLREDUCE_AGD, PLAN_ALLGATHER_DIRECT, PLAN_ALLREDUCE_FWD_AGD = 6, 7, 8
 OP_MOVE, OP_SUM, OP_CHAIN = 0, 1, 2
 PLAN_FLAG_FORWARD, PLAN_FLAG_AG_DIRECT, PLAN_FLAG_RS_DIRECT = 16, 32, 64
 BUF_SEND, BUF_RECV, BUF_INBOX, BUF_PARTIAL = 0, 1, 2, 3
-EXEC_GRAPH, EXEC_STREAMS, EXEC_ONE_KERNEL, EXEC_ONEPASS, EXEC_PROXY = range(5)
+EXEC_GRAPH, EXEC_STREAMS, EXEC_ONE_KERNEL, EXEC_ONEPASS, EXEC_PROXY, EXEC_ROLES = range(6)
 
 EXPORTS = [   # every function include/hoccl_diag.h declares
     "hoccl_chain_launch", "hoccl_copy_launch", "hoccl_fanout_inspect", "hoccl_fanout_launch", "hoccl_flatten_inspect",
     "hoccl_kernel_sms", "hoccl_options_resolve", "hoccl_plan_build", "hoccl_plan_destroy", "hoccl_plan_get_op",
     "hoccl_plan_group_deps", "hoccl_plan_inbox_slots", "hoccl_plan_num_groups", "hoccl_plan_num_ops",
     "hoccl_plan_scratch_bytes", "hoccl_plan_slot_bytes", "hoccl_port_probe", "hoccl_probe_copy_routes",
-    "hoccl_probe_move_needs_sm", "hoccl_selftest_barrier_timeout", "hoccl_selftest_bf16_add", "hoccl_sum_launch",
+    "hoccl_probe_move_needs_sm", "hoccl_selftest_barrier_timeout", "hoccl_selftest_roles_timeout", "hoccl_selftest_bf16_add", "hoccl_sum_launch",
 ]
 
 
@@ -42,7 +42,7 @@ class Options(ctypes.Structure):
                 ("onepass", ctypes.c_long), ("forward", ctypes.c_long), ("fused", ctypes.c_long), ("rs_direct", ctypes.c_long),
                 ("ag_direct", ctypes.c_long), ("handshake", ctypes.c_long), ("use_graph", ctypes.c_long),
                 ("ce_small_bytes", ctypes.c_long), ("ce_small_ctas", ctypes.c_long), ("copy_ctas", ctypes.c_long),
-                ("scratch_bytes", ctypes.c_size_t), ("host_call", ctypes.c_int)]
+                ("scratch_bytes", ctypes.c_size_t), ("host_call", ctypes.c_int), ("roles", ctypes.c_long)]
 
 
 class Resolved(ctypes.Structure):
@@ -73,6 +73,7 @@ def lib() -> ctypes.CDLL:
         "hoccl_fanout_inspect": (i, [i, vp, vp, vp, i, i, vp, vp, vp, vp, vp, vp, vp, ctypes.POINTER(i), ctypes.POINTER(i)]),
         "hoccl_kernel_sms": (i, [i, vp, vp, vp, sz, i, i, vp, vp]),
         "hoccl_selftest_barrier_timeout": (i, [vp, vp, vp, sz, vp]),
+        "hoccl_selftest_roles_timeout": (i, [vpp, vpp, sz, i, vp, vp]),
         "hoccl_port_probe": (i, [i, vp, sz, i, vp, vp]),
         "hoccl_flatten_inspect": (i, [i, i, i, i, vp, vp, vp, vp, vp, vp, vp, vp, vp]),
         "hoccl_plan_build": (i, [vpp, i, i, sz, i, i, sz, i, ctypes.c_char_p]),
@@ -97,11 +98,11 @@ def options_resolve(kind, R, count, dtype, path=_b.PATH_CE, scratch_bytes=0, hos
     params: the communicator parameters of the same names (defaults as a new communicator has them).
     Returns (code, dict or None)."""
     vals = dict(onepass=0, forward=0, fused=0, rs_direct=2, ag_direct=2, handshake=0, use_graph=1, ce_small_bytes=8 << 20, ce_small_ctas=148,
-                copy_ctas=8)
+                copy_ctas=8, roles=0)
     vals.update(params)
     o = Options(kind, R, count, _dtype(dtype), path, vals["onepass"], vals["forward"], vals["fused"], vals["rs_direct"], vals["ag_direct"],
                 vals["handshake"], vals["use_graph"], vals["ce_small_bytes"], vals["ce_small_ctas"], vals["copy_ctas"], scratch_bytes,
-                host_call)
+                host_call, vals["roles"])
     r = Resolved()
     rc = lib().hoccl_options_resolve(ctypes.byref(o), ctypes.byref(r))
     if rc != OK:
@@ -111,6 +112,10 @@ def options_resolve(kind, R, count, dtype, path=_b.PATH_CE, scratch_bytes=0, hos
 
 def selftest_barrier_timeout(comm, dst, src, nbytes, stream=None) -> int:
     return lib().hoccl_selftest_barrier_timeout(comm._h, _ptr(dst), _ptr(src), nbytes, _stream(stream))
+
+
+def selftest_roles_timeout(comm, send, recv, count, dtype, stream=None) -> int:
+    return lib().hoccl_selftest_roles_timeout(_b._ptr_array(send), _b._ptr_array(recv), count, _dtype(dtype), comm._h, _stream(stream))
 
 
 

@@ -34,10 +34,15 @@ def _must_refuse(kind, path, o):
             return True                   # the one-pass kernel replaces the whole schedule
     if reduction and o["rs_direct"] == 1 and (o["forward"] or o["fused"]):
         return True                       # no chain phase in the ring kernel, no steps to forward between
+    if reduction and o.get("roles"):
+        if path != hb.PATH_SM or o["handshake"] or o["onepass"] or o["forward"] or o["fused"] or o["rs_direct"] == 0:
+            return True                   # the roles kernel runs the direct schedule on the SM path, nothing else
+        if kind == "allreduce" and o["ag_direct"] == 0:
+            return True
     return False
 
 
-GRID = list(itertools.product([0, 1], [0, 1], [0, 1], [0, 1, 2], [0, 1, 2], [0, 1], [0, 1]))   # onepass forward fused rs ag handshake graph
+GRID = list(itertools.product([0, 1], [0, 1], [0, 1], [0, 1, 2], [0, 1, 2], [0, 1], [0, 1], [0, 1]))   # onepass forward fused rs ag handshake graph roles
 
 
 @pytest.mark.parametrize("kind", sorted(KINDS))
@@ -60,9 +65,9 @@ def test_every_combination_is_served_as_asked_or_refused(oracle, kind, path):
     small = hb.scratch_bytes(R, n_send, dtype)
     served = refused = 0
     plans = {}
-    for onepass, forward, fused, rs, ag, handshake, graph in GRID:
+    for onepass, forward, fused, rs, ag, handshake, graph, roles in GRID:
         o = dict(onepass=onepass, forward=forward, fused=fused, rs_direct=rs, ag_direct=ag, handshake=handshake, use_graph=graph,
-                 ce_small_bytes=0)
+                 roles=roles, ce_small_bytes=0)
         for scratch in (big, small):
             rc, res = hd.options_resolve(KINDS[kind], R, count, dtype, path, scratch_bytes=scratch, **o)
             if _must_refuse(kind, path, o):
@@ -74,6 +79,10 @@ def test_every_combination_is_served_as_asked_or_refused(oracle, kind, path):
             pk = res["plan_kind"]
             assert pk & 15 == KINDS[kind]
             reduction = kind in ("allreduce", "reduce_scatter")
+            if roles and reduction:       # the roles kernel: the direct schedule, whatever the scratch (a call fails later if it is too small)
+                assert pk & hd.PLAN_FLAG_RS_DIRECT and res["executor"] == hd.EXEC_ROLES and res["path"] == hb.PATH_SM
+                assert kind != "allreduce" or pk & hd.PLAN_FLAG_AG_DIRECT
+                continue
             # what was asked for is in the plan; "automatic" yields to it
             assert bool(pk & hd.PLAN_FLAG_FORWARD) == bool(forward and reduction)
             if rs == 1 and reduction:
@@ -138,4 +147,9 @@ def test_argument_errors():
     assert hd.options_resolve(7, 4, 10, "fp32")[0] == hb.ERR_INVALID_ARG
     assert hd.options_resolve(0, 0, 10, "fp32")[0] == hb.ERR_INVALID_ARG
     assert hd.options_resolve(0, 4, 10, 9)[0] == hb.ERR_UNSUPPORTED
+    # the roles kernel has chain loops for 2 to 8 ranks
+    assert hd.options_resolve(0, 9, 1000, "fp32", hb.PATH_SM, roles=1)[0] == hb.ERR_UNSUPPORTED
+    assert hd.options_resolve(0, 1, 1000, "fp32", hb.PATH_SM, roles=1)[0] == hb.ERR_UNSUPPORTED
+    assert hd.options_resolve(0, 8, 1000, "fp32", hb.PATH_SM, roles=1)[0] == hb.OK
+    assert hd.options_resolve(0, 8, 1000, "fp32", hb.PATH_SM, roles=1, host_call=1)[1]["executor"] == hd.EXEC_GRAPH
     assert hd.lib().hoccl_options_resolve(None, None) == hb.ERR_INVALID_ARG
