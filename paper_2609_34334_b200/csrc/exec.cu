@@ -683,11 +683,11 @@ hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
   const bool reduction = call->kind == PLAN_ALLREDUCE || call->kind == PLAN_REDUCE_SCATTER;
   const size_t ring_chunk = (call->kind == PLAN_ALLREDUCE ? (call->count + c->R - 1) / c->R : call->count) * dtype_size(call->dtype);
   // Copy route with overlap ("ce_overlap"): the direct schedule cut into pieces whose three parts run on three internal
-  // streams (see launch_entry).  Automatic (-1): 4 pieces from 4 MiB per ring chunk, 8 from 16 MiB; below that the ~30 us of
-  // host time per call and the extra copies cost more than the overlap gives (measured on B200, R = 8, bf16, 8-CTA sums:
-  // 40 MiB per rank 0.469 -> 0.426 ms with 4 pieces, 256 MiB 2.97 -> 2.48 ms with 8; 25 MiB 0.290 -> 0.281 with 2).
+  // streams (see launch_entry).  Automatic (-1): 2 pieces from 2 MiB per ring chunk, 4 from 4 MiB, 8 from 16 MiB; below that the
+  // ~30 us of host time per call and the extra copies cost more than the overlap gives (measured on B200, R = 8, bf16, 8-CTA
+  // sums: 40 MiB per rank 0.468 -> 0.425 ms with 4 pieces, 256 MiB 2.97 -> 2.45 ms with 8; 25 MiB 0.290 -> 0.280 with 2).
   long overlap_pieces = c->ce_overlap;
-  if (overlap_pieces < 0) overlap_pieces = ring_chunk >= ((size_t)16 << 20) ? 8 : ring_chunk >= ((size_t)4 << 20) ? 4 : 0;
+  if (overlap_pieces < 0) overlap_pieces = ring_chunk >= ((size_t)16 << 20) ? 8 : ring_chunk >= ((size_t)4 << 20) ? 4 : ring_chunk >= ((size_t)2 << 20) ? 2 : 0;
   const bool overlap = overlap_pieces > 1 && c->path == HOCCL_PATH_CE && opt.executor == EXEC_GRAPH && !call->h_send &&
                        (plan_kind & PLAN_FLAG_RS_DIRECT) && c->R > 1 && !c->piece_bytes_set;
   if (overlap) {
@@ -695,11 +695,11 @@ hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
     piece_bytes = std::max<size_t>((size_t)64 << 10, ((ring_chunk + max_pieces - 1) / max_pieces + 1023) / 1024 * 1024);
   } else if (!c->piece_bytes_set && c->path == HOCCL_PATH_SM && opt.executor == EXEC_GRAPH && !call->h_send && reduction &&
              (plan_kind & PLAN_FLAG_RS_DIRECT) && c->sum_ctas < 64 && c->copy_ctas < 128 && ring_chunk >= ((size_t)1 << 20)) {
-    // SM path, direct schedule under CTA budgets: pieces of an eighth of a ring chunk, between 512 KiB and 2 MiB, issued as a
+    // SM path, direct schedule under CTA budgets: pieces of an eighth of a ring chunk, between 640 KiB and 2 MiB, issued as a
     // software pipeline (see build_graph): a piece's copies run beside another piece's chain sum (measured, 8-CTA sums and
-    // 40 copy CTAs: 40 MiB per rank 0.47 ms with 2 pieces, 0.42 with 4, 0.39 with 8, 0.58 with 16; 256 MiB 2.99 / 2.72 / 2.57 /
-    // 2.50 ms with 2 / 4 / 8 / 16 pieces)
-    piece_bytes = std::min<size_t>((size_t)2 << 20, std::max<size_t>((size_t)512 << 10, (ring_chunk / 8 + 1023) / 1024 * 1024));
+    // 40 copy CTAs: 40 MiB per rank 0.46 ms with 2 pieces, 0.41 with 4, 0.38 with 8, 0.45 with 10; 25 MiB 0.30 / 0.26 / 0.245 /
+    // 0.29 ms with 2 / 4 / 5 / 7 pieces; 256 MiB 2.92 / 2.57 / 2.40 / 2.32 ms with 2 / 4 / 8 / 16 pieces)
+    piece_bytes = std::min<size_t>((size_t)2 << 20, std::max<size_t>((size_t)640 << 10, (ring_chunk / 8 + 1023) / 1024 * 1024));
     max_pieces = 64;
   } else if (call->h_send) {   // pipelined host all-reduce: host_pieces pieces per chunk, whatever the chunk size
     const size_t q = (call->count + c->R - 1) / c->R;
@@ -707,13 +707,10 @@ hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
     max_pieces = (int)c->host_pieces;
     piece_bytes = std::max<size_t>((size_t)64 << 10, ((chunk + max_pieces - 1) / max_pieces + 1023) / 1024 * 1024);
   } else if (roles) {
-    // pieces cost no launch here, but every piece drains and refills the register pipelines of both roles (measured ~6 us per piece
-    // for the sums): about twelve per ring chunk, a multiple of the movers' tile (128 KiB) so that no segment ends in a short tile
-    if (!c->piece_bytes_set) {
-      const size_t tile = (size_t)128 << 10;
-      piece_bytes = std::min<size_t>((size_t)2 << 20, std::max<size_t>(2 * tile, (ring_chunk / 12 + tile - 1) / tile * tile));
-    }
-    max_pieces = 32;   // the tables of all pieces must fit into a CTA's shared memory
+    // the piece rule of the graph form of the same schedule (above): both forms measured best with the same pieces
+    if (!c->piece_bytes_set)
+      piece_bytes = std::min<size_t>((size_t)2 << 20, std::max<size_t>((size_t)640 << 10, (ring_chunk / 8 + 1023) / 1024 * 1024));
+    max_pieces = 64;   // (when the tables of that many pieces do not fit into shared memory the graph form runs the plan)
   } else if (fused) {   // one kernel walks the steps in order; whole chunks measured faster than pieces (fewer barriers and tails)
     piece_bytes = (size_t)1 << 60;
     max_pieces = 1;

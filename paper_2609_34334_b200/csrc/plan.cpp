@@ -127,6 +127,9 @@ bool build_plan(Plan* plan, int kind, int R, size_t count, int dtype, bool in_pl
   size_t want = (chunk_bytes + piece_bytes - 1) / piece_bytes;
   size_t np = std::max<size_t>(1, std::min<size_t>(want, (size_t)max_pieces));
   size_t plen = round_up((chunk_bytes + np - 1) / np, 1024);
+  // pieces of 256 KiB or more are whole multiples of 128 KiB (the copy kernels' tile): measured on B200, R = 8, 40 MiB per rank,
+  // pieces of 1708 or 854 KiB (a third, a sixth of the ring chunk) ran 15 % slower than the same schedule with 1280 or 640 KiB
+  if (np > 1 && plen >= ((size_t)256 << 10)) plen = round_up(plen, (size_t)128 << 10);
   if (plen == 0) plen = 1024;
   P.piece_bytes = plen;
   P.pieces = (int)std::max<size_t>(1, (chunk_bytes + plen - 1) / plen);

@@ -2,8 +2,9 @@
 //
 // Why.  Under the SM budget for sums the chain sum is the long pole (a 40 MiB bucket over 8 ranks: 292 us on 8 SMs), and the
 // moves (the reduce-scatter's copies into the owners' inbox slots, the all-gather's fan-out) can run beside it as long as they
-// stay below ~3.5 TB/s (faster copies lengthen the loads of the few summing SMs and slow the sum down).  As a graph of kernels
-// that overlap pays a launch and a ramp per piece and per kernel; here the pieces are pipelined inside one kernel instead:
+// stay below ~3.5 TB/s (faster copies lengthen the loads of the few summing SMs and slow the sum down).  The graph form gets
+// that overlap from kernels of different pieces that run side by side and pays a launch and a pipeline ramp per piece and
+// kernel; here the pieces are pipelined inside one kernel through counters instead:
 //   * the first `n_sum` CTAs only sum: for piece p they wait until every mover has finished the reduce-scatter moves of piece p,
 //     run the chain sum of that piece (the software-pipelined loop of chain_pipe_kernel) and count themselves done;
 //   * the other CTAs only move: RS(0), RS(1), AG(0), RS(2), AG(1), ...; before the all-gather moves of piece p they wait until
@@ -16,6 +17,15 @@
 // kernel ends by itself and the host reads the error word; the last CTA out clears the counters for the next launch.
 // Rank locality holds as in the graph form: a mover copies a rank's own data, a summing CTA works in the owner's memory.
 // The order of the adds and their rounding are those of chain_kernel: the bits are the oracle's.
+//
+// Measured (B200, R = 8, bf16, 8 summing + 40 moving CTAs, against the graph form with the same pieces and budgets): 25 MiB per
+// rank 0.248 vs 0.245 ms, 40 MiB 0.377 vs 0.380, 64 MiB 0.599 vs 0.613, 128 MiB 1.14 vs 1.22, 256 MiB 2.28 vs 2.32.  So one
+// launch instead of 24 to 48 buys a few per cent at best: every piece still drains and refills the register pipelines of both
+// roles (4 to 5 us per piece for the sums, measured with the movers switched off), which is what the launches cost the graph
+// form too.  Three things mattered more than the form: tables in shared memory (walking them in device memory cost the movers
+// 24 us per piece), the three role bodies as functions of their own (inlined into one kernel the chain loop was scheduled
+// 8 % slower, and any added variable pushed the kernel over its 128 registers), and scratch regions that start on 128-byte
+// lines (plan.cpp).
 #include <cuda_bf16.h>
 
 #include "comm.h"
@@ -123,7 +133,7 @@ __device__ __noinline__ void copy_ragged(const uint4* a, uint4* o, unsigned n_he
 // vectors per thread, all loads of a tile issued before its stores).  Equal contiguous byte ranges per mover instead were tried:
 // the extra live 64-bit values pushed the kernel over its 128 registers and every role got slower.
 template <bool CG>
-__device__ __forceinline__ void copy_share(const RolesCopySeg* seg, int nseg, unsigned m, unsigned M) {
+__device__ __noinline__ void copy_share(const RolesCopySeg* seg, int nseg, unsigned m, unsigned M) {
   if (nseg <= 0) return;
   constexpr unsigned tile_v = kCopyU * kRolesThreads;
   {
@@ -161,7 +171,7 @@ __device__ __forceinline__ void copy_share(const RolesCopySeg* seg, int nseg, un
 }
 
 // ---- a mover's share of the fan-out segments of one piece (a tile is loaded once and stored to every destination)
-__device__ __forceinline__ void fan_share(const RolesFanSeg* seg, int nseg, void* const* dst_all, unsigned m, unsigned M) {
+__device__ __noinline__ void fan_share(const RolesFanSeg* seg, int nseg, void* const* dst_all, unsigned m, unsigned M) {
   if (nseg <= 0) return;
   constexpr unsigned tile_v = kFanU * kRolesThreads;
   {
@@ -228,7 +238,7 @@ __device__ __forceinline__ void chain_scalar_cg(const RolesChainSeg& sg, unsigne
 // ---- a summing CTA's share of the chain sums of one piece: a contiguous range of the flattened tile space, the full tiles of a
 // segment through a branch-free loop with kChainP tiles of loads in flight per thread (see chain_pipe_kernel)
 template <int DT, int NOPS>
-__device__ __forceinline__ void chain_share(const RolesChainSeg* seg, int nseg, unsigned s, unsigned S) {
+__device__ __noinline__ void chain_share(const RolesChainSeg* seg, int nseg, unsigned s, unsigned S) {
   using T = Traits<DT>;
   if (nseg <= 0) return;
   constexpr int P = kChainP, THREADS = kRolesThreads;
