@@ -525,7 +525,8 @@ def main():
 def gemm_loss_matched(torch, hb, W, B, want_dev):
     """What a co-running bf16 GEMM (8192 x 4096 x 16384, on another stream) loses while the gradient stream's buckets are
     all-reduced back to back, against the collective's bus bandwidth beside it: the copy route, and the SM-copy path under
-    copy-kernel budgets of 8 to 148 CTAs, every one with 8-CTA sums and the default schedule.  `interpolated` reads the SM
+    copy-kernel budgets of 8 to 148 CTAs (and as one kernel with roles, 8 + 40 CTAs), every one with 8-CTA sums and the default
+    schedule.  `interpolated` reads the SM
     path's loss at the copy route's throughput, so that the two are compared at equal bandwidth."""
     g = W.C4_GRADIENTS
     R, S, stream = B.R, B.S, B.stream
@@ -562,10 +563,11 @@ def gemm_loss_matched(torch, hb, W, B, want_dev):
     rows = []
     configs = [("CE_sum8", hb.PATH_CE, 8, 8, {}), ("CE_sum8_ring", hb.PATH_CE, 8, 8, {"rs_direct": 0, "ag_direct": 0}),
                ("CE_sum8_plain_graphs", hb.PATH_CE, 8, 8, {"order_kernels": 0, "ce_overlap": 0})]
-    configs += [("SM_copy%d_sum8" % b, hb.PATH_SM, 8, b, {}) for b in (8, 16, 32, 64, 148)]
-    configs += [("SM_copy148_sum148", hb.PATH_SM, 148, 148, {})]
+    configs += [("SM_copy%d_sum8" % b, hb.PATH_SM, 8, b, {}) for b in (8, 16, 32, 40, 64, 148)]
+    configs += [("SM_roles_copy40_sum8", hb.PATH_SM, 8, 40, {"roles": 1}), ("SM_copy148_sum148", hb.PATH_SM, 148, 148, {})]
     for name, path, sc, cc, extra in configs:
         cm = B.comm(path, sum_ctas=sc, copy_ctas=cc, **extra)
+        time.sleep(0.5)   # the stand-alone figure must not inherit the clocks the previous row's GEMM left behind (power cap)
         t, _ = B.timed(cm, 12, 3)
         t_g = n_gemm * flops / (alone * 1e12)
         n_bucket = max(1, int(1.3 * t_g / t) + 1)
@@ -592,14 +594,18 @@ def gemm_loss_matched(torch, hb, W, B, want_dev):
             if x0 <= x <= x1:
                 interp = y0 if x1 == x0 else y0 + (y1 - y0) * (x - x0) / (x1 - x0)
                 break
+    near = min((r for r in rows if r["config"].startswith("SM_copy") and r["sum_ctas"] == 8), key=lambda r: abs(r["busbw_beside_GBps"] - x))
     return {"workload": g.name, "gemm_probe": [M, K, N], "gemm_alone_TFLOPs": alone, "gemms_per_run": n_gemm, "rows": rows,
             "interpolated": {"at_busbw_beside_GBps": x, "copy_route_gemm_loss": ce["gemm_loss"], "sm_copy_path_gemm_loss_at_that_bandwidth": interp,
-                             "note": "null: the copy route's bandwidth lies outside the range the copy-kernel budgets cover"}}
+                             "nearest_sm_copy_row": {"config": near["config"], "busbw_beside_GBps": near["busbw_beside_GBps"],
+                                                     "gemm_loss": near["gemm_loss"]},
+                             "note": "null: the copy route's bandwidth lies outside the range the copy-kernel budgets cover; the nearest "
+                                     "budget row is given beside it"}}
 
 
 def large_messages(torch, hb, W, np, peaks):
     """All-reduce, reduce-scatter, all-gather and send/recv at 64 MiB, 256 MiB and 1 GiB per rank (R = 8, bf16, per-rank sizes in
-    the nccl-tests convention), copy route against SM path.  Inputs depend on (rank, position), generated on the device; every
+    the nccl-tests convention), copy route against SM path (graphs of kernels, and the one kernel with roles).  Inputs depend on (rank, position), generated on the device; every
     row's output is compared, on the device, with what the CPU oracle computes from the same bytes."""
     from oracle import ring as oracle_ring
 
@@ -607,7 +613,8 @@ def large_messages(torch, hb, W, np, peaks):
     stream = torch.cuda.Stream()
     thr = oracle_ring.max_threads()
     configs = [("CE_sum8", hb.PATH_CE, 8, 8, {}), ("CE_sum8_ring", hb.PATH_CE, 8, 8, {"rs_direct": 0, "ag_direct": 0}),
-               ("CE_sum148", hb.PATH_CE, 148, 8, {}), ("SM_copy8_sum8", hb.PATH_SM, 8, 8, {}), ("SM_copy148_sum148", hb.PATH_SM, 148, 148, {})]
+               ("CE_sum148", hb.PATH_CE, 148, 8, {}), ("SM_copy8_sum8", hb.PATH_SM, 8, 8, {}), ("SM_copy40_sum8", hb.PATH_SM, 8, 40, {}),
+               ("SM_roles_copy40_sum8", hb.PATH_SM, 8, 40, {"roles": 1}), ("SM_copy148_sum148", hb.PATH_SM, 148, 148, {})]
     rows = []
 
     def bits(t):
@@ -671,8 +678,8 @@ def large_messages(torch, hb, W, np, peaks):
             if name in ("CE_sum8", "SM_copy8_sum8", "SM_copy148_sum148"):
                 ops.append(("sendrecv", p2p, check_p2p, 2.0 * S, 1.0))
             for op, fn, check, ring_bytes, bf in ops:
-                if op in ("allgather", "sendrecv") and name in ("CE_sum148",):
-                    continue                     # no sums in these: the row would repeat CE_sum8
+                if op in ("allgather", "sendrecv") and name in ("CE_sum148", "SM_roles_copy40_sum8"):
+                    continue                     # no sums in these: the row would repeat CE_sum8 / SM_copy40_sum8
                 for t in recv + small:
                     t.zero_()
                 torch.cuda.synchronize()

@@ -223,6 +223,20 @@ hoccl_result_t hoccl_comm_set_path(hoccl_comm_t comm, hoccl_path_t path);
  *                of pinned host memory of its own on first use (the third exception to "device memory is the caller's").
  *                Refused on the other paths and in handshake mode (see the rules below); plans too large for one launch (more
  *                than 480 chunk operations or 96 steps: an all-reduce beyond 12 ranks) run as a graph.  0 = off (default).
+ *  "roles"       1 = on HOCCL_PATH_SM all-reduce and reduce-scatter calls of 2 to 8 ranks run the stage-decomposed schedule
+ *                ("rs_direct", "ag_direct") as ONE cooperative kernel whose CTAs have roles: the first min(sum_ctas, 64) CTAs
+ *                only sum, copy_ctas further CTAs only move, and the pieces of a chunk are pipelined between them through
+ *                counters in device memory (moves of piece p + 1 run beside the sums of piece p; paper Sec. 3.3, chunk
+ *                pipelining, without a launch per piece and kernel).  Rank local, same bits.  Measured on B200 (R = 8, bf16,
+ *                8 + 40 CTAs) it equals the graph of kernels with the same budgets within a few per cent (40 MiB per rank
+ *                0.377 against 0.380 ms, 256 MiB 2.28 against 2.32 ms).  It needs the scratch of the direct form
+ *                (hoccl_scratch_bytes_direct; HOCCL_ERR_SCRATCH otherwise).  Every wait is bounded; a wait that runs out ends
+ *                the kernel and is reported by hoccl_comm_async_error as HOCCL_ERR_TIMEOUT.  The library allocates 1 KiB of
+ *                device memory and 4 bytes of pinned host memory per communicator on first use, and per cached call
+ *                signature a table of at most 200 KiB in device memory (further exceptions to "device memory is the
+ *                caller's").  When sum_ctas + copy_ctas CTAs cannot be resident together, or the tables of a call's pieces
+ *                exceed 200 KiB (more than ~40 pieces at 8 ranks), the same plan runs as a graph.  Other calls ignore the
+ *                setting.  0 = off (default).
  *  "host_pieces" pieces per ring chunk of the pipelined hoccl_host_allreduce (1..64, default 8; 1 = not pipelined)
  *  "use_graph"   1 = run a cached CUDA graph built from the plan (default), 0 = streams and events
  *  "handshake"   1 = the paper's stream manager (Sec. 3.2): instead of launching into the caller's stream, the call
@@ -246,6 +260,11 @@ hoccl_result_t hoccl_comm_set_path(hoccl_comm_t comm, hoccl_path_t path);
  *                a post then holds its stream at the post until the transfer is done, whichever side posts first (the
  *                paper's semantics, Sec. 3.3.2), instead of parking on the host (see hoccl_send).  Needs HOCCL_PATH_SM,
  *                like handshake mode.  0 = off (default).
+ *  "model_gpus_per_node"  hoccl_alltoallv only: 0 (default) or >= R = all ranks in one NVLink domain; g in 1..R-1 = the ranks are
+ *                modelled as nodes of g GPUs each and inter-node flows take the forwarding copies and the RDMA leg of the
+ *                paper's scheduler as real copies through the staging memory (see hoccl_alltoallv)
+ *  "model_rdma_sub_bytes" modelled topology: the RDMA leg of a chunk is issued in sub-copies of this many bytes, one after the
+ *                other, as a NIC serialises its queue (0 = one copy per chunk, default)
  *  "profile"     1 = time every SUM launch with CUDA events; read the totals with hoccl_last_stats after
  *                synchronising (with graphs only the latest replay of each cached graph is readable, so
  *                read after every step)
@@ -257,6 +276,9 @@ hoccl_result_t hoccl_comm_set_path(hoccl_comm_t comm, hoccl_path_t path);
  *   - "fused" is an executor of HOCCL_PATH_SM: refused on the other paths; refused with "rs_direct" = 1 (the one-kernel
  *     form has no chain phase); it ignores "use_graph" and is not used by hoccl_host_allreduce; plans beyond its capacity
  *     (see "fused") run as a graph;
+ *   - "roles" applies to all-reduce and reduce-scatter calls (hoccl_host_allreduce excepted) and runs the direct schedule
+ *     on HOCCL_PATH_SM: refused on the other paths, for fewer than 2 or more than 8 ranks, and together with "handshake",
+ *     "onepass", "forward", "fused", "rs_direct" = 0 or (all-reduce) "ag_direct" = 0; it ignores "use_graph";
  *   - "onepass" applies to all-reduce and reduce-scatter calls, ignores the path, and for those calls is refused together
  *     with "forward", "fused", "rs_direct" = 1 or (all-reduce) "ag_direct" = 1; other collectives ignore it;
  *   - "forward" applies to all-reduce and reduce-scatter calls and is refused with "rs_direct" = 1;
@@ -324,8 +346,15 @@ hoccl_result_t hoccl_alltoall(const void* const* send, void* const* recv, size_t
  * run one after the other.  With "use_graph" = 1 (default) the schedule becomes a CUDA graph that is cached under the
  * call's full signature (every pointer, count and displacement), so a pattern that repeats on the same buffers replays
  * it; otherwise, and with "use_graph" = 0, it is issued with streams and events.  No scratch.
+ * Modelled topology ("model_gpus_per_node" = g with 0 < g < R): the R logical ranks are treated as GPUs of R / g nodes (rank r
+ * sits on node r / g, the last node may be smaller) and the scheduler runs the paper's full expansion (Eq. 2-4, Algorithm 1):
+ * a flow between two nodes is carried, portion by portion as Algorithm 1 stages it, by a forwarding copy to the sender's
+ * symmetric peer, the "RDMA" leg to the receiver's symmetric peer and a forwarding copy to the receiver, all as real copies
+ * through the memory attached with hoccl_comm_set_staging, while native flows fill the NVLink slack of the stages.  The
+ * received bytes are the same.  Needs staging of at least twice the inter-node bytes of the call, every flow rounded up to 256
+ * (HOCCL_ERR_SCRATCH otherwise), and "use_graph" = 1 (HOCCL_ERR_UNSUPPORTED otherwise).
  * Errors: INVALID_ARG (NULL, misaligned, overlapping receive regions, a send region overlapping a receive region),
- * UNSUPPORTED (dtype; handshake mode).
+ * UNSUPPORTED (dtype; handshake mode; a modelled topology without graphs), SCRATCH (modelled topology, staging too small).
  */
 hoccl_result_t hoccl_alltoallv(const void* const* send, const size_t* sendcounts, const size_t* sdispls, void* const* recv,
                                const size_t* rdispls, hoccl_dtype_t dtype, hoccl_comm_t comm, hoccl_stream_t stream);
@@ -353,8 +382,8 @@ hoccl_result_t hoccl_send(const void* buf, size_t count, hoccl_dtype_t dtype, in
 hoccl_result_t hoccl_recv(void* buf, size_t count, hoccl_dtype_t dtype, int src, int dst, hoccl_comm_t comm,
                           hoccl_stream_t stream);
 int hoccl_comm_pending(hoccl_comm_t comm);
-/* First asynchronous failure: handshake mode, as seen by the proxy (OK, TIMEOUT, MISMATCH or CUDA); "fused" setting,
- * TIMEOUT if a barrier wait of the whole-collective kernel ran out.  clear != 0 resets it. */
+/* First asynchronous failure: handshake mode, as seen by the proxy (OK, TIMEOUT, MISMATCH or CUDA); "fused" and "roles"
+ * settings, TIMEOUT if a bounded wait inside the kernel ran out.  clear != 0 resets it. */
 hoccl_result_t hoccl_comm_async_error(hoccl_comm_t comm, int clear);
 /* Handshake mode: number of stream hand-overs the proxy has served so far. */
 long hoccl_comm_handshakes(hoccl_comm_t comm);

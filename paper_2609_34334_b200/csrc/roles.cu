@@ -76,6 +76,29 @@ struct RolesArgs {
   int npieces, n_sum, missing, pad;
 };
 
+// L2 eviction hints: what a mover puts into an inbox slot is read once, by a summing CTA, a piece later: it should stay in
+// L2 until then and go first afterwards; what the all-gather stores is not read again in this launch.  (Measured: 2 % at
+// 40 MiB per rank, nothing at 256 MiB; the L2 hit rate of the launch stays near 10 %.)
+constexpr bool kL2Hints = true;
+__device__ __forceinline__ unsigned long long policy_evict_last() {
+  unsigned long long p;
+  asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ unsigned long long policy_evict_first() {
+  unsigned long long p;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+  return p;
+}
+__device__ __forceinline__ void st_hint(uint4* a, uint4 v, unsigned long long pol) {
+  asm volatile("st.global.L2::cache_hint.v4.u32 [%0], {%1,%2,%3,%4}, %5;" ::"l"(a), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w), "l"(pol) : "memory");
+}
+__device__ __forceinline__ uint4 ldcg_hint(const uint4* a, unsigned long long pol) {
+  uint4 v;
+  asm volatile("ld.global.cg.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %5;" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(a), "l"(pol));
+  return v;
+}
+
 __device__ __forceinline__ unsigned ld_acquire(const unsigned* p) {
   unsigned v;
   asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
@@ -136,6 +159,7 @@ template <bool CG>
 __device__ __noinline__ void copy_share(const RolesCopySeg* seg, int nseg, unsigned m, unsigned M) {
   if (nseg <= 0) return;
   constexpr unsigned tile_v = kCopyU * kRolesThreads;
+  const unsigned long long keep = policy_evict_last();
   {
     const unsigned long long T_all = seg[nseg - 1].tiles_end;
     int k = 0;
@@ -151,7 +175,10 @@ __device__ __noinline__ void copy_share(const RolesCopySeg* seg, int nseg, unsig
 #pragma unroll
         for (int u = 0; u < kCopyU; u++) v[u] = CG ? __ldcg(a + threadIdx.x + u * kRolesThreads) : __ldcs(a + threadIdx.x + u * kRolesThreads);
 #pragma unroll
-        for (int u = 0; u < kCopyU; u++) o[threadIdx.x + u * kRolesThreads] = v[u];
+        for (int u = 0; u < kCopyU; u++) {
+          if (kL2Hints && !CG) st_hint(o + threadIdx.x + u * kRolesThreads, v[u], keep);
+          else o[threadIdx.x + u * kRolesThreads] = v[u];
+        }
       } else {
         copy_ragged(a, o, n_here, CG);
       }
@@ -196,7 +223,10 @@ __device__ __noinline__ void fan_share(const RolesFanSeg* seg, int nseg, void* c
 #pragma unroll
         for (int u = 0; u < kFanU; u++) {
           const unsigned i = threadIdx.x + u * kRolesThreads;
-          if (i < n_here) o[i] = v[u];
+          if (i < n_here) {
+            if (kL2Hints) __stcs(o + i, v[u]);
+            else o[i] = v[u];
+          }
         }
       }
     }
@@ -242,6 +272,7 @@ __device__ __noinline__ void chain_share(const RolesChainSeg* seg, int nseg, uns
   using T = Traits<DT>;
   if (nseg <= 0) return;
   constexpr int P = kChainP, THREADS = kRolesThreads;
+  const unsigned long long drop = policy_evict_first();
   {
     const unsigned long long T_all = seg[nseg - 1].tiles_end;
     const unsigned long long A = T_all / S * s + min((unsigned long long)s, T_all % S);
@@ -263,7 +294,9 @@ __device__ __noinline__ void chain_share(const RolesChainSeg* seg, int nseg, uns
       auto load = [&](uint4(&bb)[NOPS], unsigned long long t) {
         const size_t o = (size_t)t * THREADS * 16;
 #pragma unroll
-        for (int q = 0; q < NOPS - 1; q++) bb[q] = __ldcg(reinterpret_cast<const uint4*>(src + (size_t)q * stride + o));
+        for (int q = 0; q < NOPS - 1; q++)
+          bb[q] = kL2Hints ? ldcg_hint(reinterpret_cast<const uint4*>(src + (size_t)q * stride + o), drop)
+                                 : __ldcg(reinterpret_cast<const uint4*>(src + (size_t)q * stride + o));
         bb[NOPS - 1] = __ldcg(reinterpret_cast<const uint4*>(loc + o));
       };
       auto finish = [&](const uint4(&bb)[NOPS], unsigned long long t) {

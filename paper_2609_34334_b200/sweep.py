@@ -17,6 +17,7 @@ from __future__ import annotations
 import argparse
 import json
 import sys
+import time
 
 import torch
 
@@ -114,6 +115,7 @@ def sweep_sizes(args):
         "CEall": (hb.PATH_CE, 148, 8, {}),                              # copy route with whole-GPU sums
         "SM8": (hb.PATH_SM, 8, 8, {}), "SM8ring": (hb.PATH_SM, 8, 8, dict(ring)),
         "SM40": (hb.PATH_SM, 8, 40, {}),                                # 8-CTA sums beside 40 copy CTAs
+        "SMroles40": (hb.PATH_SM, 8, 40, {"roles": 1}),                 # the same as one cooperative kernel with roles
         "SMall": (hb.PATH_SM, 148, 148, {}), "SMallring": (hb.PATH_SM, 148, 148, dict(ring)),
         "SMallfused": (hb.PATH_SM, 148, 148, {"fused": 1}),             # the ring as one cooperative kernel
         "SM8fused": (hb.PATH_SM, 8, 8, {"fused": 1}),
@@ -332,6 +334,11 @@ def gradients(args):
             comm.set_param("ag_direct", 0)
             comm.set_param("rs_direct", 0)
         comm.set_param("order_kernels", 0 if name.endswith("_plain_graphs") else 1)   # the copy-route graphs without ordering kernels
+        for k in range(pool):
+            comm.allreduce(send[k], recv[k], per, dtype, stream)
+        stream.synchronize()
+        # the stand-alone figure must not inherit the clocks the previous configuration's GEMM left behind (power cap)
+        time.sleep(0.5)
         for k in range(pool):
             comm.allreduce(send[k], recv[k], per, dtype, stream)
         stream.synchronize()
