@@ -68,7 +68,13 @@ def _boundaries(comm, R, n, e):
         lo, hi = min(c * q, n), min((c + 1) * q, n)
         out.add(lo)
         if pieces > 1 and hi > lo:
-            pb = (-(-(q * e) // pieces) + 1023) // 1024 * 1024      # equal pieces, a multiple of 1024 bytes
+            # equal pieces, a multiple of 1024 bytes, from 256 KiB on a multiple of 128 KiB (the planner's rule)
+            for want in range(pieces, pieces + 16):
+                pb = (-(-(q * e) // want) + 1023) // 1024 * 1024
+                if pb >= 256 << 10:
+                    pb = -(-pb // (128 << 10)) * (128 << 10)
+                if -(-(q * e) // pb) == pieces:
+                    break
             for p in range(1, pieces):
                 out.add(min(hi, lo + (p * pb) // e))
     out.discard(0)
@@ -81,6 +87,11 @@ CONFIGS = [
     ("copy_route_ring", hb.PATH_CE, {"rs_direct": 0, "ag_direct": 0}),
     ("sm_path_whole_gpu", hb.PATH_SM, {"sum_ctas": 148, "copy_ctas": 148}),
     ("copy_route_direct_one_graph", hb.PATH_CE, {"rs_direct": 1, "ag_direct": 1, "ce_overlap": 0}),
+    # with the scratch of the direct form attached (rs_direct = 2 is the default; naming it makes _comm attach that scratch):
+    # the configurations bench.py times
+    ("copy_route_default_overlapped", hb.PATH_CE, {"rs_direct": 2}),
+    ("sm_path_sum8_copy40", hb.PATH_SM, {"rs_direct": 2, "sum_ctas": 8, "copy_ctas": 40}),
+    ("sm_path_roles_sum8_copy40", hb.PATH_SM, {"rs_direct": 2, "sum_ctas": 8, "copy_ctas": 40, "roles": 1}),
 ]
 
 
