@@ -200,8 +200,9 @@ hoccl_result_t hoccl_comm_set_path(hoccl_comm_t comm, hoccl_path_t path);
  *                parts (the reduce-scatter's moves, the chain sum, the all-gather's moves) become graphs of their own that
  *                run on three internal streams, ordered by events, so that one piece's driver copies run beside another
  *                piece's sum (inside ONE graph, and on plain streams, they were never seen to overlap).  Sums still run one
- *                at a time.  Costs ~8 us of host time per piece and call.  -1 (default) = automatic: 4 pieces from 4 MiB per
- *                ring chunk, 8 from 16 MiB, off below; 0 = off; 2..64 = that many pieces.  Ignored when "piece_bytes" is set.
+ *                at a time.  Costs ~8 us of host time per piece and call.  -1 (default) = automatic: 2 pieces from 2 MiB per
+ *                ring chunk, from 4 MiB on pieces of about 4 MiB (at least 4, at most 32 of them), off below; 0 = off;
+ *                2..64 = that many pieces.  Ignored when "piece_bytes" is set.
  *  "ce_small_ctas" CTAs of those launches, 1..1024 (default 148: like the driver's own copies they may use the whole GPU,
  *                for tens of microseconds)
  *  "order_kernels" 1 (default) = on the copy routes the graph executor puts an empty one-warp kernel in front of a graph's
@@ -237,6 +238,11 @@ hoccl_result_t hoccl_comm_set_path(hoccl_comm_t comm, hoccl_path_t path);
  *                caller's").  When sum_ctas + copy_ctas CTAs cannot be resident together, or the tables of a call's pieces
  *                exceed 200 KiB (more than ~40 pieces at 8 ranks), the same plan runs as a graph.  Other calls ignore the
  *                setting.  0 = off (default).
+ *  "piece_grade" all-reduce and reduce-scatter on the stage-decomposed schedule: 1 = the pieces of a ring chunk are graded, the
+ *                first and the last ones smaller (a third, two thirds of a middle piece; pieces of 256 KiB or more only), so that
+ *                less of the moves in front of the first sum and behind the last one is exposed; 0 = equal pieces; -1 (default)
+ *                = automatic: graded from 8 MiB per ring chunk on, where it was measured to gain 1-5 %, equal below, where the
+ *                small outer pieces cost more than they save.  Same operations, same bits.
  *  "host_pieces" pieces per ring chunk of the pipelined hoccl_host_allreduce (1..64, default 8; 1 = not pipelined)
  *  "use_graph"   1 = run a cached CUDA graph built from the plan (default), 0 = streams and events
  *  "handshake"   1 = the paper's stream manager (Sec. 3.2): instead of launching into the caller's stream, the call

@@ -147,7 +147,8 @@ typedef enum { HOCCL_PLAN_ALLREDUCE = 0, HOCCL_PLAN_REDUCE_SCATTER = 1, HOCCL_PL
                HOCCL_PLAN_ALLREDUCE_AGD = 6, HOCCL_PLAN_ALLGATHER_DIRECT = 7,   /* the "ag_direct" variants */
                HOCCL_PLAN_ALLREDUCE_FWD_AGD = 8 /* both */ } hoccl_plan_kind_t;
 /* General form: a base kind (0..3) OR-ed with flags; the numbered variants above are shorthands. */
-typedef enum { HOCCL_PLAN_FLAG_FORWARD = 16, HOCCL_PLAN_FLAG_AG_DIRECT = 32, HOCCL_PLAN_FLAG_RS_DIRECT = 64 /* "rs_direct" */ } hoccl_plan_flag_t;
+typedef enum { HOCCL_PLAN_FLAG_FORWARD = 16, HOCCL_PLAN_FLAG_AG_DIRECT = 32, HOCCL_PLAN_FLAG_RS_DIRECT = 64 /* "rs_direct" */,
+               HOCCL_PLAN_FLAG_GRADED = 128 /* "piece_grade": smaller first and last pieces */ } hoccl_plan_flag_t;
 /* CHAIN: out = (((s_0 + s_1) + ...) + s_{nsrc-1}) + local, every add rounded into the I/O dtype; s_j at src_off + j * src_stride */
 typedef enum { HOCCL_OP_MOVE = 0, HOCCL_OP_SUM = 1, HOCCL_OP_CHAIN = 2 } hoccl_plan_op_kind_t;
 typedef enum { HOCCL_BUF_SEND = 0, HOCCL_BUF_RECV = 1, HOCCL_BUF_INBOX = 2, HOCCL_BUF_PARTIAL = 3 } hoccl_buf_kind_t;

@@ -149,6 +149,7 @@ static long* param_slot(hoccl_comm* c, const char* key, long* lo, long* hi) {
               {"ce_small_ctas", &c->ce_small_ctas, 1, 1024},
               {"p2p_strict", &c->p2p_strict, 0, 1},
               {"roles", &c->roles, 0, 1},
+              {"piece_grade", &c->piece_grade, -1, 1},
               {"ce_overlap", &c->ce_overlap, -1, 64},
               {"model_gpus_per_node", &c->model_gpus_per_node, 0, kMaxRanks},
               {"model_rdma_sub_bytes", &c->model_rdma_sub_bytes, 0, 1L << 40},

@@ -100,7 +100,7 @@ struct hoccl_comm {
   hoccl_path_t path = HOCCL_PATH_CE;
   long sum_ctas = 8, copy_ctas = 8, piece_bytes = 4 << 20, max_pieces = 8, lanes = 4, use_graph = 1, profile = 0, p2p_split = 1, ce_sub_bytes = 0,
        handshake = 0, watchdog_ms = 10000, onepass = 0, forward = 0, fused = 0, host_pieces = 8, ag_direct = 2, order_kernels = 1, rs_direct = 2,
-       ce_small_bytes = 8 << 20, ce_small_ctas = 148, p2p_strict = 0, ce_overlap = -1, model_gpus_per_node = 0, model_rdma_sub_bytes = 0, roles = 0,
+       ce_small_bytes = 8 << 20, ce_small_ctas = 148, p2p_strict = 0, ce_overlap = -1, model_gpus_per_node = 0, model_rdma_sub_bytes = 0, roles = 0, piece_grade = -1,
        roles_missing = 0 /* self-test only: summing CTAs wait for this many movers that do not exist */;
   bool piece_bytes_set = false;  // the caller chose a piece size: no automatic choice
   hoccl::Proxy* proxy = nullptr;

@@ -395,6 +395,7 @@ std::vector<uint64_t> make_key(hoccl_comm* c, const Call& call) {
   k.push_back((uint64_t)c->ce_overlap);
   k.push_back((uint64_t)(c->fused && c->path == HOCCL_PATH_SM && !c->handshake));
   k.push_back((uint64_t)c->roles);
+  k.push_back((uint64_t)c->piece_grade);
   k.push_back((uint64_t)c->roles_missing);
   k.push_back((uint64_t)(uintptr_t)c->scratch);
   k.push_back((uint64_t)c->scratch_bytes);
@@ -683,11 +684,14 @@ hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
   const bool reduction = call->kind == PLAN_ALLREDUCE || call->kind == PLAN_REDUCE_SCATTER;
   const size_t ring_chunk = (call->kind == PLAN_ALLREDUCE ? (call->count + c->R - 1) / c->R : call->count) * dtype_size(call->dtype);
   // Copy route with overlap ("ce_overlap"): the direct schedule cut into pieces whose three parts run on three internal
-  // streams (see launch_entry).  Automatic (-1): 2 pieces from 2 MiB per ring chunk, 4 from 4 MiB, 8 from 16 MiB; below that the
-  // ~30 us of host time per call and the extra copies cost more than the overlap gives (measured on B200, R = 8, bf16, 8-CTA
-  // sums: 40 MiB per rank 0.468 -> 0.425 ms with 4 pieces, 256 MiB 2.97 -> 2.45 ms with 8; 25 MiB 0.290 -> 0.280 with 2).
+  // streams (see launch_entry).  Automatic (-1): 2 pieces from 2 MiB per ring chunk, from 4 MiB on pieces of about 4 MiB, at
+  // least 4 and at most 32 of them; below that the ~30 us of host time per call and the extra copies cost more than the overlap
+  // gives (measured on B200, R = 8, bf16, 8-CTA sums: 25 MiB per rank 0.290 -> 0.280 ms with 2 pieces; 40 MiB 0.468 -> 0.421 with
+  // 4; 256 MiB 2.97 -> 2.44 with 8; 1 GiB 11.8 -> 9.72 with 8, 9.52 with 32).
   long overlap_pieces = c->ce_overlap;
-  if (overlap_pieces < 0) overlap_pieces = ring_chunk >= ((size_t)16 << 20) ? 8 : ring_chunk >= ((size_t)4 << 20) ? 4 : ring_chunk >= ((size_t)2 << 20) ? 2 : 0;
+  if (overlap_pieces < 0)
+    overlap_pieces = ring_chunk >= ((size_t)4 << 20) ? (long)std::min<size_t>(32, std::max<size_t>(4, ring_chunk >> 22))
+                                                     : ring_chunk >= ((size_t)2 << 20) ? 2 : 0;
   const bool overlap = overlap_pieces > 1 && c->path == HOCCL_PATH_CE && opt.executor == EXEC_GRAPH && !call->h_send &&
                        (plan_kind & PLAN_FLAG_RS_DIRECT) && c->R > 1 && !c->piece_bytes_set;
   if (overlap) {
@@ -724,7 +728,13 @@ hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
     const size_t chunk = q * dtype_size(call->dtype);
     if (chunk >= ((size_t)1 << 20)) piece_bytes = std::min(piece_bytes, (chunk / 2 + 1023) / 1024 * 1024);
   }
-  if (!build_plan(&P, plan_kind, c->R, call->count, call->dtype, call->in_place, piece_bytes, max_pieces, align))
+  // graded pieces ("piece_grade"; -1 = automatic): measured on B200 (R = 8, bf16, 8-CTA sums) they gain 1-5 % from 64 MiB per rank
+  // on (256 MiB: copy route 2.46 -> 2.44 ms, SM path 8 + 40 CTAs 2.32 -> 2.27, roles kernel 2.32 -> 2.25) and lose below (40 MiB
+  // buckets: copy route 0.423 -> 0.444 ms, SM path 0.380 -> 0.431: the small outer pieces cost more in fixed time per piece than
+  // their shorter fill saves), so automatic means: from 8 MiB per ring chunk
+  const bool graded = reduction && !call->h_send && !fused && (plan_kind & PLAN_FLAG_RS_DIRECT) &&
+                      (c->piece_grade == 1 || (c->piece_grade < 0 && ring_chunk >= ((size_t)8 << 20)));
+  if (!build_plan(&P, plan_kind | (graded ? PLAN_FLAG_GRADED : 0), c->R, call->count, call->dtype, call->in_place, piece_bytes, max_pieces, align))
     return HOCCL_ERR_INVALID_ARG;
   if (P.slot_bytes) {
     size_t need = P.scratch_need();

@@ -33,13 +33,13 @@ void destroy_entry(GraphEntry* e) {
 // as a 1-D copy.
 void add_host_copies(const Plan& P, int p, char* dev, char* host, std::vector<HostCopy>* out) {
   const size_t e = P.elem, q_bytes = P.chunk_elems * e;
-  const size_t off = (size_t)p * P.piece_bytes;
+  const size_t off = (size_t)P.piece_off[(size_t)p], end = (size_t)P.piece_off[(size_t)p + 1];
   size_t full_rows = 0, full_len = 0;
   for (int cidx = 0; cidx < P.R; cidx++) {
     size_t lo, hi;
     P.chunk_range(cidx, &lo, &hi);
     const size_t len_bytes = (hi - lo) * e;
-    const size_t a = std::min(off, len_bytes), b = std::min(off + P.piece_bytes, len_bytes);
+    const size_t a = std::min(off, len_bytes), b = std::min(end, len_bytes);
     const size_t len = b - a;
     if (len == 0) continue;
     if (cidx == 0) full_len = len;

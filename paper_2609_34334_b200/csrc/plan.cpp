@@ -70,8 +70,8 @@ struct Builder {
 
 // piece p of a chunk of len_bytes bytes: [off, off+len)
 void piece_span(const Plan& P, size_t len_bytes, int p, size_t* off, size_t* len) {
-  size_t a = (size_t)p * P.piece_bytes;
-  size_t b = a + P.piece_bytes;
+  size_t a = (size_t)P.piece_off[(size_t)p];
+  size_t b = (size_t)P.piece_off[(size_t)p + 1];
   a = std::min(a, len_bytes);
   b = std::min(b, len_bytes);
   *off = a;
@@ -88,7 +88,7 @@ bool build_plan(Plan* plan, int kind, int R, size_t count, int dtype, bool in_pl
   if (kind >= 16) {
     flags = kind & ~15;
     kind &= 15;
-    if (kind > PLAN_ALLTOALL || (flags & ~(PLAN_FLAG_FORWARD | PLAN_FLAG_AG_DIRECT | PLAN_FLAG_RS_DIRECT))) return false;
+    if (kind > PLAN_ALLTOALL || (flags & ~(PLAN_FLAG_FORWARD | PLAN_FLAG_AG_DIRECT | PLAN_FLAG_RS_DIRECT | PLAN_FLAG_GRADED))) return false;
   } else {
     if (kind > PLAN_ALLREDUCE_FWD_AGD) return false;
     if (kind == PLAN_ALLREDUCE_FWD || kind == PLAN_REDUCE_SCATTER_FWD || kind == PLAN_ALLREDUCE_FWD_AGD) flags |= PLAN_FLAG_FORWARD;
@@ -102,6 +102,7 @@ bool build_plan(Plan* plan, int kind, int R, size_t count, int dtype, bool in_pl
   const bool rs_direct = reduces && (flags & PLAN_FLAG_RS_DIRECT) && R > 1;
   const bool forward = reduces && (flags & PLAN_FLAG_FORWARD) && !rs_direct;   // the direct form has no per-step sums to forward
   const bool ag_direct = gathers && (flags & PLAN_FLAG_AG_DIRECT);
+  const bool graded = reduces && (flags & PLAN_FLAG_GRADED);
   if (kind == PLAN_ALLTOALL && in_place) return false;  // an in-place exchange would need a staging copy of every block
   if (max_pieces < 1) max_pieces = 1;
   if (piece_bytes < 1024) piece_bytes = 1024;
@@ -133,6 +134,48 @@ bool build_plan(Plan* plan, int kind, int R, size_t count, int dtype, bool in_pl
   if (plen == 0) plen = 1024;
   P.piece_bytes = plen;
   P.pieces = (int)std::max<size_t>(1, (chunk_bytes + plen - 1) / plen);
+  P.piece_off.assign((size_t)P.pieces + 1, 0);
+  for (int p = 0; p <= P.pieces; p++) P.piece_off[(size_t)p] = std::min<uint64_t>((uint64_t)p * plen, chunk_bytes);
+  if (graded && P.pieces >= 3 && plen >= ((size_t)256 << 10)) {
+    // Graded pieces, in units of 128 KiB: weights 1/3, 2/3, 1, ..., 1, 2/3, 1/3 (with three or four pieces only the outer ones
+    // shrink).  The count stays; the middle pieces grow by what the outer ones give up.
+    const size_t u = (size_t)128 << 10;
+    const size_t units = (chunk_bytes + u - 1) / u;
+    const int n = P.pieces;
+    std::vector<double> w((size_t)n, 1.0);
+    const int ramp = n >= 6 ? 2 : 1;
+    for (int k = 0; k < ramp; k++) {
+      w[(size_t)k] = w[(size_t)(n - 1 - k)] = (double)(k + 1) / (double)(ramp + 1);
+    }
+    double wsum = 0;
+    for (double x : w) wsum += x;
+    std::vector<size_t> sz((size_t)n, 0);
+    size_t used = 0;
+    for (int k = 0; k < n; k++) {
+      sz[(size_t)k] = std::max<size_t>(1, (size_t)((double)units * w[(size_t)k] / wsum));
+      used += sz[(size_t)k];
+    }
+    // what rounding left over goes to (or comes from) the middle pieces, one unit at a time
+    for (int k = ramp; used < units; k = (k + 1 - ramp) % std::max(1, n - 2 * ramp) + ramp) {
+      sz[(size_t)k]++;
+      used++;
+    }
+    size_t guard = 0;
+    for (int k = ramp; used > units && guard < units * (size_t)n; k = (k + 1 - ramp) % std::max(1, n - 2 * ramp) + ramp, guard++) {
+      if (sz[(size_t)k] > 1) {
+        sz[(size_t)k]--;
+        used--;
+      }
+    }
+    size_t off = 0, biggest = 0;
+    for (int k = 0; k < n; k++) {
+      P.piece_off[(size_t)k] = std::min<uint64_t>(off, chunk_bytes);
+      off += sz[(size_t)k] * u;
+      biggest = std::max(biggest, sz[(size_t)k] * u);
+    }
+    P.piece_off[(size_t)n] = chunk_bytes;
+    P.piece_bytes = biggest;
+  }
   // Slack between the regions of consecutive pieces inside a scratch slot: 16 bytes hold the phase shift (below); pieces of
   // 16 KiB or more get 128, so that every region starts on a 128-byte line like the operands it is summed with.  (With 16 the
   // region of piece p sat 16 p bytes off the line grid: a warp's 512-byte load then touched five lines instead of four, and the
@@ -148,7 +191,7 @@ bool build_plan(Plan* plan, int kind, int R, size_t count, int dtype, bool in_pl
     size_t lo, hi;
     P.chunk_range(c, &lo, &hi);
     size_t phase = ((send_align ? (size_t)(send_align[r] & 15) : 0) + lo * e) & 15;
-    return (uint64_t)p * (P.piece_bytes + slack) + phase;
+    return P.piece_off[(size_t)p] + (uint64_t)p * slack + phase;
   };
 
   Builder B{&P};

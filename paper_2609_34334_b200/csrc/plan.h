@@ -26,7 +26,11 @@ enum PlanFlag { PLAN_FLAG_FORWARD = 16, PLAN_FLAG_AG_DIRECT = 32,
                 // direct reduce-scatter: the reduce-scatter's traffic matrix (rank r owes chunk d to rank d) cut into the R-1
                 // permutation stages r -> r+k (Sec. 3.4); rank d keeps the R-1 contributions in R-1 inbox slots and sums them
                 // in the ring's order in one pass (OP_CHAIN): same bits, 2 S (R-1) + S (R+1) instead of 5 S (R-1) bytes
-                PLAN_FLAG_RS_DIRECT = 64 };
+                PLAN_FLAG_RS_DIRECT = 64,
+                // graded pieces (reductions): the first and the last pieces of a chunk are smaller than the middle ones (a third,
+                // two thirds of a middle piece), so that less of the pipeline's fill and drain (the moves in front of the first
+                // sum and behind the last one) is exposed.  Pieces of 256 KiB or more only; same operations, same bits.
+                PLAN_FLAG_GRADED = 128 };
 enum OpKind { OP_MOVE = 0, OP_SUM = 1,
               // out = (((s_0 + s_1) + ...) + s_{nsrc-1}) + local, rounded to the I/O dtype after every add; s_j at src_off + j * src_stride
               OP_CHAIN = 2 };
@@ -65,8 +69,9 @@ struct Plan {
   bool in_place = false;
   size_t elem = 4;
   size_t chunk_elems = 0;   // q: elements of a full ring chunk
-  size_t piece_bytes = 0;   // bytes of a full piece (multiple of 1024 unless the chunk is one piece)
+  size_t piece_bytes = 0;   // bytes of the largest piece (multiple of 1024 unless the chunk is one piece)
   int pieces = 1;
+  std::vector<uint64_t> piece_off;   // pieces + 1 byte offsets inside a full ring chunk; piece p is [piece_off[p], piece_off[p+1])
   size_t slot_bytes = 0;    // bytes of one scratch slot (inbox or partial) of one rank, padded
   std::vector<PlanOp> ops;
   std::vector<PlanGroup> groups;

@@ -10,7 +10,7 @@ from .binding import OK, HocclError, _dtype, _ptr, _ptr_array, _stream
 PLAN_ALLREDUCE, PLAN_REDUCE_SCATTER, PLAN_ALLGATHER, PLAN_ALLTOALL, PLAN_ALLREDUCE_FWD, PLAN_REDUCE_SCATTER_FWD = range(6)
 PLAN_ALLREDUCE_AGD, PLAN_ALLGATHER_DIRECT, PLAN_ALLREDUCE_FWD_AGD = 6, 7, 8
 OP_MOVE, OP_SUM, OP_CHAIN = 0, 1, 2
-PLAN_FLAG_FORWARD, PLAN_FLAG_AG_DIRECT, PLAN_FLAG_RS_DIRECT = 16, 32, 64
+PLAN_FLAG_FORWARD, PLAN_FLAG_AG_DIRECT, PLAN_FLAG_RS_DIRECT, PLAN_FLAG_GRADED = 16, 32, 64, 128
 BUF_SEND, BUF_RECV, BUF_INBOX, BUF_PARTIAL = 0, 1, 2, 3
 EXEC_GRAPH, EXEC_STREAMS, EXEC_ONE_KERNEL, EXEC_ONEPASS, EXEC_PROXY, EXEC_ROLES = range(6)
 

@@ -60,23 +60,17 @@ def _exact_integer_sum(send):
 
 
 def _boundaries(comm, R, n, e):
-    """Element indices where a ring chunk or a pipeline piece of the last call starts."""
+    """Element indices where a ring chunk or a pipeline piece of the last call starts: the planner's own piece offsets for the
+    piece count the call reports, for equal and for graded pieces (the call may have used either)."""
+    from paper_2609_34334_b200 import diag as hd
     q = -(-n // R)
     pieces = max(1, int(comm.last_stats()["n_pieces"]))
-    out = set()
-    for c in range(R):
-        lo, hi = min(c * q, n), min((c + 1) * q, n)
-        out.add(lo)
-        if pieces > 1 and hi > lo:
-            # equal pieces, a multiple of 1024 bytes, from 256 KiB on a multiple of 128 KiB (the planner's rule)
-            for want in range(pieces, pieces + 16):
-                pb = (-(-(q * e) // want) + 1023) // 1024 * 1024
-                if pb >= 256 << 10:
-                    pb = -(-pb // (128 << 10)) * (128 << 10)
-                if -(-(q * e) // pb) == pieces:
-                    break
-            for p in range(1, pieces):
-                out.add(min(hi, lo + (p * pb) // e))
+    dtype = "fp32" if e == 4 else "bf16"
+    out = set(min(c * q, n) for c in range(R))
+    if pieces > 1:
+        for flags in (hd.PLAN_FLAG_RS_DIRECT, hd.PLAN_FLAG_RS_DIRECT | hd.PLAN_FLAG_GRADED):
+            plan = hd.Plan(hd.PLAN_ALLREDUCE | flags, R, n, dtype, False, -(-(q * e) // pieces), pieces)
+            out.update(op["local_off"] // e for op in plan.ops if op["kind"] == hd.OP_CHAIN)
     out.discard(0)
     out.discard(n)
     return sorted(out)

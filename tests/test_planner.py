@@ -391,4 +391,45 @@ def test_direct_reduce_scatter_plans(oracle, R, n, piece_bytes, max_pieces):
     # flags that do not apply are ignored, unknown ones refused
     assert hd.Plan(hd.PLAN_ALLGATHER | hd.PLAN_FLAG_RS_DIRECT, R, 8, "fp32").inbox_slots == 1
     with pytest.raises(hb.HocclError):
-        hd.Plan(hd.PLAN_ALLREDUCE | 128, R, 8, "fp32")
+        hd.Plan(hd.PLAN_ALLREDUCE | 256, R, 8, "fp32")
+
+
+@pytest.mark.parametrize("R,n,piece_bytes,max_pieces", [(4, 4 * (3 << 20) // 4 + 5, 256 << 10, 64), (8, 8 * 700_000 + 3, 384 << 10, 6),
+                                                        (2, 2 * 1_000_000, 512 << 10, 3), (3, 3 * 90_000, 256 << 10, 8)])
+def test_graded_pieces_cover_the_chunk_and_give_the_ring_bits(oracle, R, n, piece_bytes, max_pieces):
+    """PLAN_FLAG_GRADED: the same operations on pieces of unequal size (the outer ones a third and two thirds of a middle one, in
+    units of 128 KiB).  The pieces still tile every chunk exactly, every piece keeps its own region of the scratch slots (no
+    two regions overlap, every region starts on a 128-byte line), and any legal order gives the ring's bits."""
+    rng = random.Random(R * 77 + max_pieces)
+    dtype, e = "fp32", 4
+    xs = W.rank_inputs("uniform", 43, R, n, dtype)
+    want = oracle.ring_allreduce(xs)
+    q = -(-n // R)
+    for flags in (hd.PLAN_FLAG_RS_DIRECT | hd.PLAN_FLAG_AG_DIRECT, 0):
+        kind = hd.PLAN_ALLREDUCE | flags
+        plain = hd.Plan(kind, R, n, dtype, False, piece_bytes, max_pieces)
+        plan = hd.Plan(kind | hd.PLAN_FLAG_GRADED, R, n, dtype, False, piece_bytes, max_pieces)
+        assert plan.scratch_bytes <= hb.scratch_bytes_direct(R, n, dtype) if flags else plan.scratch_bytes <= hb.scratch_bytes(R, n, dtype)
+        # the pieces of chunk 0 as the sums see them: contiguous, complete, and (when the chunk is large enough) graded
+        sums = sorted((op["local_off"], op["bytes"]) for op in plan.ops if op["kind"] in (hd.OP_CHAIN, hd.OP_SUM) and op["chunk"] == 0
+                      and op["rank"] == 0 and (op["kind"] == hd.OP_CHAIN or op["step"] == R - 2))
+        assert sums[0][0] == 0 and sum(b for _, b in sums) == min(q, n) * e
+        for (o0, b0), (o1, _) in zip(sums, sums[1:]):
+            assert o0 + b0 == o1
+        sizes = [b for _, b in sums]
+        if len(sizes) >= 3 and q * e // len(sizes) >= 256 << 10:
+            assert sizes[0] < sizes[1] and sizes[-1] < sizes[-2] and all(b % (128 << 10) == 0 for b in sizes[:-1])
+            assert len(sizes) == len([1 for op in plain.ops if op["kind"] in (hd.OP_CHAIN, hd.OP_SUM) and op["chunk"] == 0 and op["rank"] == 0
+                                      and (op["kind"] == hd.OP_CHAIN or op["step"] == R - 2)])
+        else:
+            assert [op for op in plan.ops] == [op for op in plain.ops]          # too small to grade: the plain plan
+        # regions of one inbox slot do not overlap and start on 128-byte lines
+        regions = sorted((op["dst_off"], op["bytes"]) for op in plan.ops if op["kind"] == hd.OP_MOVE and op["dst_buf"] == hd.BUF_INBOX
+                         and op["dst_rank"] == 1 and op["dst_off"] < plan.slot_bytes and (flags or op["step"] == 0))
+        for (o0, b0), (o1, _) in zip(regions, regions[1:]):
+            assert o0 + b0 <= o1
+            if len(sizes) > 1 and min(sizes[:-1]) >= 16 << 10:
+                assert (o1 - regions[0][0]) % 128 == 0                 # regions[0][0] is the 16-byte phase of this rank's operand
+        got = _run_plan(plan, kind, R, n, dtype, xs, False, rng)
+        for r in range(R):
+            assert (got[r].view(np.uint32) == want[r].view(np.uint32)).all(), (R, n, flags, r)
