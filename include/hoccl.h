@@ -241,8 +241,9 @@ hoccl_result_t hoccl_comm_set_path(hoccl_comm_t comm, hoccl_path_t path);
  *  "piece_grade" all-reduce and reduce-scatter on the stage-decomposed schedule: 1 = the pieces of a ring chunk are graded, the
  *                first and the last ones smaller (a third, two thirds of a middle piece; pieces of 256 KiB or more only), so that
  *                less of the moves in front of the first sum and behind the last one is exposed; 0 = equal pieces; -1 (default)
- *                = automatic: graded from 8 MiB per ring chunk on, where it was measured to gain 1-5 %, equal below, where the
- *                small outer pieces cost more than they save.  Same operations, same bits.
+ *                = automatic: graded from 8 MiB per ring chunk on under a SUM budget (sum_ctas < 64), where it was measured to
+ *                gain 1-5 %, equal otherwise (below that size the small outer pieces cost more than they save).  Same
+ *                operations, same bits.
  *  "host_pieces" pieces per ring chunk of the pipelined hoccl_host_allreduce (1..64, default 8; 1 = not pipelined)
  *  "use_graph"   1 = run a cached CUDA graph built from the plan (default), 0 = streams and events
  *  "handshake"   1 = the paper's stream manager (Sec. 3.2): instead of launching into the caller's stream, the call

@@ -689,9 +689,12 @@ hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
   // gives (measured on B200, R = 8, bf16, 8-CTA sums: 25 MiB per rank 0.290 -> 0.280 ms with 2 pieces; 40 MiB 0.468 -> 0.421 with
   // 4; 256 MiB 2.97 -> 2.44 with 8; 1 GiB 11.8 -> 9.72 with 8, 9.52 with 32).
   long overlap_pieces = c->ce_overlap;
-  if (overlap_pieces < 0)
-    overlap_pieces = ring_chunk >= ((size_t)4 << 20) ? (long)std::min<size_t>(32, std::max<size_t>(4, ring_chunk >> 22))
+  if (overlap_pieces < 0) {
+    // (whole-GPU sums are short: beside them more than 8 pieces only add copies; 1 GiB per rank 6.34 ms with 8, 6.80 with 32)
+    const size_t most = c->sum_ctas >= 64 ? 8 : 32;
+    overlap_pieces = ring_chunk >= ((size_t)4 << 20) ? (long)std::min<size_t>(most, std::max<size_t>(4, ring_chunk >> 22))
                                                      : ring_chunk >= ((size_t)2 << 20) ? 2 : 0;
+  }
   const bool overlap = overlap_pieces > 1 && c->path == HOCCL_PATH_CE && opt.executor == EXEC_GRAPH && !call->h_send &&
                        (plan_kind & PLAN_FLAG_RS_DIRECT) && c->R > 1 && !c->piece_bytes_set;
   if (overlap) {
@@ -731,9 +734,10 @@ hoccl_result_t run_collective(hoccl_comm* c, Call* call, cudaStream_t user) {
   // graded pieces ("piece_grade"; -1 = automatic): measured on B200 (R = 8, bf16, 8-CTA sums) they gain 1-5 % from 64 MiB per rank
   // on (256 MiB: copy route 2.46 -> 2.44 ms, SM path 8 + 40 CTAs 2.32 -> 2.27, roles kernel 2.32 -> 2.25) and lose below (40 MiB
   // buckets: copy route 0.423 -> 0.444 ms, SM path 0.380 -> 0.431: the small outer pieces cost more in fixed time per piece than
-  // their shorter fill saves), so automatic means: from 8 MiB per ring chunk
+  // their shorter fill saves), so automatic means: from 8 MiB per ring chunk, under a SUM budget (with whole-GPU sums the outer
+  // pieces' moves are no longer what is exposed: 256 MiB per rank, copy route, 148-CTA sums 1.51 -> 1.53 ms)
   const bool graded = reduction && !call->h_send && !fused && (plan_kind & PLAN_FLAG_RS_DIRECT) &&
-                      (c->piece_grade == 1 || (c->piece_grade < 0 && ring_chunk >= ((size_t)8 << 20)));
+                      (c->piece_grade == 1 || (c->piece_grade < 0 && ring_chunk >= ((size_t)8 << 20) && c->sum_ctas < 64));
   if (!build_plan(&P, plan_kind | (graded ? PLAN_FLAG_GRADED : 0), c->R, call->count, call->dtype, call->in_place, piece_bytes, max_pieces, align))
     return HOCCL_ERR_INVALID_ARG;
   if (P.slot_bytes) {
