@@ -41,13 +41,14 @@ def _values(rng, n, dtype, flavour):
 case = st.fixed_dictionaries({
     "op": st.sampled_from(["allreduce", "allreduce", "reduce_scatter", "allgather", "alltoall"]),
     "R": st.integers(1, 9),
-    "n": st.one_of(st.integers(0, 40), st.integers(41, 5000), st.integers(5001, 300_000)),
+    "n": st.one_of(st.integers(0, 40), st.integers(41, 5000), st.integers(5001, 300_000), st.integers(300_001, 2_500_000)),
     "dtype": st.sampled_from(["fp32", "bf16"]),
     "path": st.sampled_from([hb.PATH_CE, hb.PATH_SM]),
     "use_graph": st.integers(0, 1),
-    "piece_kib": st.sampled_from([1, 4, 64, 4096]),
+    "piece_kib": st.sampled_from([1, 4, 64, 256, 4096]),
     "max_pieces": st.integers(1, 6),
-    "variant": st.sampled_from(["plain", "plain", "fused", "forward", "onepass"]),
+    "variant": st.sampled_from(["plain", "plain", "fused", "forward", "onepass", "roles"]),
+    "piece_grade": st.integers(-1, 1),
     "ctas": st.sampled_from([1, 3, 8, 148]),
     "in_place": st.booleans(),
     "offs": st.lists(st.integers(0, 3), min_size=9, max_size=9),
@@ -71,7 +72,8 @@ def test_random_cases_match_the_oracle(oracle, c):
     total = count if op == "allreduce" else count * R
     offs = [o * e for o in c["offs"][:R]]
     params = dict(use_graph=c["use_graph"], piece_bytes=c["piece_kib"] << 10, max_pieces=c["max_pieces"], sum_ctas=c["ctas"],
-                  copy_ctas=c["ctas"], ag_direct=c["ag_direct"], rs_direct=c["rs_direct"], ce_small_bytes=c["ce_small_kib"] << 10)
+                  copy_ctas=c["ctas"], ag_direct=c["ag_direct"], rs_direct=c["rs_direct"], ce_small_bytes=c["ce_small_kib"] << 10,
+                  piece_grade=c["piece_grade"])
     if c["variant"] != "plain":
         params[c["variant"]] = 1
     comm = make_comm(R, max(total, 1), dtype, c["path"], **params)
@@ -81,7 +83,7 @@ def test_random_cases_match_the_oracle(oracle, c):
             "alltoall": hd.PLAN_ALLTOALL}[op]
     verdict, _ = hd.options_resolve(kind, R, count, dtype, c["path"], **{k: v for k, v in params.items()
                                                                      if k in ("use_graph", "ag_direct", "rs_direct", "onepass", "forward",
-                                                                              "fused", "ce_small_bytes", "copy_ctas")})
+                                                                              "fused", "roles", "ce_small_bytes", "copy_ctas")})
     if verdict != hb.OK:
         assert verdict == hb.ERR_UNSUPPORTED
         send = [DevBuf(max(total, 1) * e) for _ in range(R)]
