@@ -199,7 +199,7 @@ int hoccl_plan_group_deps(hoccl_plan_t plan, int group, int* deps, int cap);
  * this function, so a combination is either served as asked or refused, never changed silently.
  * kind: 0 all-reduce, 1 reduce-scatter, 2 all-gather, 3 all-to-all; count in that collective's convention; the option
  * fields carry the values of the parameters of the same name; scratch_bytes = attached scratch (0: none); host_call = 1
- * for hoccl_host_allreduce.
+ * for hoccl_host_allreduce.  (HOCCL_PLAN_FLAG_GRADED is not part of the answer: a call adds it by message size, "piece_grade".)
  */
 typedef struct {
   int kind, R;
