@@ -818,6 +818,11 @@ def extras(torch, hb, hd, W, np, replicas, world, dev, peaks):
         for label, extra in (("direct", {}), ("ring", {"rs_direct": 0, "ag_direct": 0}), ("ring_direct_allgather", {"rs_direct": 0, "ag_direct": 1})):
             cm = B.comm(path, sum_ctas=sc, copy_ctas=cc, **extra)
             r = row(cm, path=name, sum_ctas=sc, copy_ctas=cc if path == hb.PATH_SM else None, schedule=label)
+            # the sums are in the first of the two calls: its statistics, not the all-gather's
+            cnt = B.n // R
+            rs_out = [B.recv_sets[0][q].data_ptr() + q * cnt * B.e for q in range(R)]
+            cm.reduce_scatter(B.send_sets[0], rs_out, cnt, B.dtype, stream)
+            stream.synchronize()
             r["sum_launches_per_step"] = int(cm.last_stats()["n_sum_launches"])
             sched.append(r)
             cm.destroy()
